@@ -1,0 +1,520 @@
+/*
+ * CPU oracle for the FP8 transformer-block hot path (test infrastructure, NOT a product path).
+ *
+ * Plain, slow, double-accumulating C.  It shares no code with the CUDA library and must never be
+ * called from it; only the tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * What it follows in the paper:
+ *   - FP8 formats E4M3 / E5M2 and their roles (forward / backward tensors): Section 2 (Background).
+ *   - per-tensor scaling s(x) = FP8Max / absmax(x): Appendix C (definition before Theorem 1);
+ *     rho(X) = FP8Max / (2^m max H): Appendix E.
+ *   - end-to-end GEMM(X,Y) = 1/(rho_X rho_Y) * FP8GEMM(cast(rho_X X), cast(rho_Y Y)): Appendix E.
+ *   - linear operators Y = XW and which products run in FP8 (QK^T and PV included): Appendix E, Table
+ *     "Comparison between FP8 methods".
+ *   - attention P = Softmax(s QK^T + M), selfattn = PV, grouped-query heads: Appendix B, Eq. (P).
+ * Where the paper is silent (rounding mode, saturation, where FP8 enters inside attention, the backward
+ * pass) the reading taken is written at the function.
+ *
+ * Parity status: codec, amax, scale, cast, GEMM, attention forward and the un-quantised attention
+ * backward are pinned by tests (tables, worked values, brute force, closed forms, finite differences).
+ * The *placement* of the two FP8 encodes inside the attention backward is our reading of "FP8 in forward
+ * and backward"; no published value exists for it: "parity unpinned" for that placement only.
+ */
+#include <float.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_E4M3 0
+#define ORACLE_E5M2 1
+
+/* ------------------------------------------------------------------------------------------------
+ * Codec (Section 2: E4M3 = 1 sign, 4 exponent, 3 mantissa bits; E5M2 = 1-5-2).
+ * E4M3 has no infinities and a single NaN mantissa pattern (S.1111.111); E5M2 is IEEE-like.
+ * ---------------------------------------------------------------------------------------------- */
+static int fmt_mbits(int fmt) { return fmt == ORACLE_E4M3 ? 3 : 2; }
+static int fmt_ebits(int fmt) { return fmt == ORACLE_E4M3 ? 4 : 5; }
+static int fmt_bias(int fmt) { return fmt == ORACLE_E4M3 ? 7 : 15; }
+
+double oracle_fp8_max(int fmt) { return fmt == ORACLE_E4M3 ? 448.0 : 57344.0; }
+
+double oracle_fp8_decode(uint8_t code, int fmt)
+{
+    const int mb = fmt_mbits(fmt), eb = fmt_ebits(fmt), bias = fmt_bias(fmt);
+    const int sign = code >> 7;
+    const int E = (code >> mb) & ((1 << eb) - 1);
+    const int M = code & ((1 << mb) - 1);
+    double v;
+    if (fmt == ORACLE_E4M3) {
+        if (E == 15 && M == 7) return NAN;
+    } else {
+        if (E == 31) return M == 0 ? (sign ? -INFINITY : INFINITY) : NAN;
+    }
+    if (E == 0)
+        v = ldexp((double)M, 1 - bias - mb);                       /* subnormal: M * 2^(1-bias-mbits) */
+    else
+        v = ldexp(1.0 + (double)M / (double)(1 << mb), E - bias);  /* normal */
+    return sign ? -v : v;
+}
+
+/* binary32 -> FP8 code, round-to-nearest-even, saturating to the largest finite value.
+ * Reading (paper silent on rounding/overflow): finite inputs never produce Inf/NaN; +-Inf saturates;
+ * NaN gives the NaN pattern 0x7F; the sign of zero and of values that round to zero is kept. */
+uint8_t oracle_fp8_encode(float v, int fmt)
+{
+    const int mb = fmt_mbits(fmt), bias = fmt_bias(fmt);
+    const double maxv = oracle_fp8_max(fmt);
+    const double min_normal = ldexp(1.0, 1 - bias);
+    const double min_sub = ldexp(1.0, 1 - bias - mb);
+    if (isnan(v)) return 0x7F;
+    const uint8_t sign = signbit(v) ? 0x80 : 0x00;
+    const double a = fabs((double)v);
+    uint8_t code;
+    if (a > maxv) {
+        code = (fmt == ORACLE_E4M3) ? 0x7E : 0x7B;
+    } else if (a < min_normal) {
+        /* fixed-point grid of step min_sub; nearbyint rounds half to even in the default mode;
+         * q == 2^mbits is the code of min_normal by continuity of the encoding */
+        code = (uint8_t)nearbyint(a / min_sub);
+    } else {
+        int ex;
+        (void)frexp(a, &ex);          /* a = f * 2^ex, f in [0.5,1) */
+        int e = ex - 1;               /* a = (1+frac) * 2^e */
+        double frac = a / ldexp(1.0, e) - 1.0;
+        int q = (int)nearbyint(frac * (double)(1 << mb));
+        if (q == (1 << mb)) { q = 0; e += 1; }
+        code = (uint8_t)(((e + bias) << mb) | q);
+    }
+    return (uint8_t)(code | sign);
+}
+
+void oracle_fp8_decode_table(int fmt, double *out256)
+{
+    for (int c = 0; c < 256; ++c) out256[c] = oracle_fp8_decode((uint8_t)c, fmt);
+}
+
+void oracle_fp8_encode_array(const float *v, size_t n, int fmt, uint8_t *out)
+{
+    for (size_t i = 0; i < n; ++i) out[i] = oracle_fp8_encode(v[i], fmt);
+}
+
+static float bf16_bits_to_float(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * amax: absmax(x) of Appendix C / max|x| of Appendix E, over a BF16 tensor.
+ * |x| ordering of finite BF16 values equals the ordering of (bits & 0x7FFF) as integers.
+ * ---------------------------------------------------------------------------------------------- */
+float oracle_amax_bf16(const uint16_t *x, size_t n)
+{
+    uint16_t best = 0;
+    for (size_t i = 0; i < n; ++i) {
+        uint16_t m = (uint16_t)(x[i] & 0x7FFF);
+        if (m > best) best = m;
+    }
+    return bf16_bits_to_float(best);
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * scale: s = FP8Max / (2^margin * amax) (Appendix C with margin 0; Appendix E with H = {amax}).
+ * One binary32 division, then an exact power-of-two factor; scale_inv is one more binary32 division.
+ * Readings (paper silent): amax == 0 or non-finite -> scale 1; an overflowing quotient -> FLT_MAX.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_scale(float amax, int fmt, int margin, float *scale, float *scale_inv)
+{
+    volatile float s;
+    if (!(amax > 0.0f) || isinf(amax)) {
+        s = 1.0f;
+    } else {
+        volatile float q = (float)oracle_fp8_max(fmt) / amax;
+        s = q * ldexpf(1.0f, -margin);
+        if (isinf(s)) s = FLT_MAX;
+    }
+    volatile float inv = 1.0f / s;
+    *scale = s;
+    *scale_inv = inv;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * cast: FP8cast(rho * X) of Appendix E.  Reading of the precision (paper silent): the BF16 value is
+ * widened exactly to binary32, multiplied by the scale in binary32 (round-to-nearest), and the product
+ * is rounded once more to FP8 by oracle_fp8_encode.  out_t, if not NULL, is the same codes laid out
+ * [cols, rows].
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_cast_bf16(const uint16_t *x, size_t rows, size_t cols, float scale, int fmt,
+                      uint8_t *out, uint8_t *out_t)
+{
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < (long)rows; ++r) {
+        for (size_t c = 0; c < cols; ++c) {
+            volatile float p = bf16_bits_to_float(x[(size_t)r * cols + c]) * scale;
+            uint8_t code = oracle_fp8_encode(p, fmt);
+            if (out) out[(size_t)r * cols + c] = code;
+            if (out_t) out_t[c * rows + (size_t)r] = code;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * FP8 GEMM with descale (Appendix E): ref[i,j] = sa_inv*sb_inv * sum_k dec(A[i,k]) * dec(B[j,k]),
+ * accumulated in double, on a list of output rows and columns.  A and B are addressed through
+ * (row stride, reduction stride) so that the three linear products are this one routine on three
+ * index patterns (see the wrappers below).  mag is the same sum over absolute values.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_gemm_sampled(const uint8_t *A, int fmtA, int64_t a_rs, int64_t a_ks,
+                         const uint8_t *B, int fmtB, int64_t b_rs, int64_t b_ks,
+                         double sa_inv, double sb_inv, int64_t kred,
+                         const int64_t *rows, int64_t nrows, const int64_t *cols, int64_t ncols,
+                         const double *prev, double *ref, double *mag)
+{
+    double ta[256], tb[256];
+    oracle_fp8_decode_table(fmtA, ta);
+    oracle_fp8_decode_table(fmtB, tb);
+#pragma omp parallel for collapse(2) schedule(dynamic, 16)
+    for (int64_t ii = 0; ii < nrows; ++ii) {
+        for (int64_t jj = 0; jj < ncols; ++jj) {
+            const uint8_t *pa = A + rows[ii] * a_rs;
+            const uint8_t *pb = B + cols[jj] * b_rs;
+            double acc = 0.0, am = 0.0;
+            for (int64_t k = 0; k < kred; ++k) {
+                double a = ta[pa[k * a_ks]], b = tb[pb[k * b_ks]];
+                acc += a * b;
+                am += fabs(a) * fabs(b);
+            }
+            double r = sa_inv * sb_inv * acc;
+            if (prev) r += prev[ii * ncols + jj];
+            ref[ii * ncols + jj] = r;
+            if (mag) mag[ii * ncols + jj] = sa_inv * sb_inv * am;
+        }
+    }
+}
+
+/* Y[t,n] = sum_k X8[t,k] W8[n,k]   (Linear_W(X) = XW with W stored [out,in]; X, W in E4M3) */
+void oracle_linear_fwd(const uint8_t *X8, const uint8_t *W8, double sx_inv, double sw_inv,
+                       int64_t T, int64_t N, int64_t K,
+                       const int64_t *rows, int64_t nrows, const int64_t *cols, int64_t ncols,
+                       double *ref, double *mag)
+{
+    (void)T; (void)N;
+    oracle_gemm_sampled(X8, ORACLE_E4M3, K, 1, W8, ORACLE_E4M3, K, 1, sx_inv, sw_inv, K,
+                        rows, nrows, cols, ncols, NULL, ref, mag);
+}
+
+/* dX[t,k] = sum_n dY8[t,n] W8[n,k]   (dY in E5M2, W in E4M3) */
+void oracle_linear_dgrad(const uint8_t *dY8, const uint8_t *W8, double sdy_inv, double sw_inv,
+                         int64_t T, int64_t N, int64_t K,
+                         const int64_t *rows, int64_t nrows, const int64_t *cols, int64_t ncols,
+                         double *ref, double *mag)
+{
+    (void)T;
+    oracle_gemm_sampled(dY8, ORACLE_E5M2, N, 1, W8, ORACLE_E4M3, 1, K, sdy_inv, sw_inv, N,
+                        rows, nrows, cols, ncols, NULL, ref, mag);
+}
+
+/* dW[n,k] = (prev[n,k]) + sum_t dY8[t,n] X8[t,k]   (dY in E5M2, X in E4M3) */
+void oracle_linear_wgrad(const uint8_t *dY8, const uint8_t *X8, double sdy_inv, double sx_inv,
+                         int64_t T, int64_t N, int64_t K,
+                         const int64_t *rows, int64_t nrows, const int64_t *cols, int64_t ncols,
+                         const double *prev, double *ref, double *mag)
+{
+    oracle_gemm_sampled(dY8, ORACLE_E5M2, 1, N, X8, ORACLE_E4M3, 1, K, sdy_inv, sx_inv, T,
+                        rows, nrows, cols, ncols, prev, ref, mag);
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Attention (Appendix B, Eq. (P): P = Softmax(s QK^T + M), output PV; grouped-query heads).
+ * Tensors are [B, N, H, d]; query head h reads key/value head h / (Hq/Hkv).  M is the causal mask
+ * (0 for key <= query, -inf otherwise) or absent.
+ *
+ * An operand is either FP8 codes (decoded through a table) or real values in double; the second form
+ * exists so that the un-quantised arithmetic can be checked by finite differences.
+ * ---------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t B, N, Hq, Hkv, d;
+    int32_t causal;
+    int32_t quant;     /* 1: P -> E4M3 and dS -> E5M2 are applied; 0: both encodes dropped */
+    int32_t kv_block;  /* forward: 0 = whole row at once, else keys are taken in blocks of this length */
+    int32_t max_mode;  /* forward: 0 = exact running maximum; 1 = maximum of x*log2(e) rounded up to an integer */
+    int32_t pad_;
+    double s;          /* softmax scale */
+    double c_P;        /* quantisation scale of P~ = exp(x - m) in (0,1]; 448 = FP8Max/amax with amax = 1 */
+    double q_inv, k_inv, v_inv, do_inv;  /* descales of Q8, K8, V8, dO8 */
+    double ds_scale;   /* backward: quantisation scale of dS */
+} oracle_attn_params;
+
+typedef struct {
+    const uint8_t *codes;   /* used when vals == NULL */
+    const double *vals;
+    double table[256];
+} operand;
+
+static void operand_init(operand *o, const uint8_t *codes, const double *vals, int fmt)
+{
+    o->codes = codes;
+    o->vals = vals;
+    oracle_fp8_decode_table(fmt, o->table);
+}
+static inline double ld(const operand *o, int64_t idx)
+{
+    return o->vals ? o->vals[idx] : o->table[o->codes[idx]];
+}
+static inline int64_t idx4(const oracle_attn_params *p, int H, int b, int n, int h, int dd)
+{
+    return (((int64_t)b * p->N + n) * H + h) * p->d + dd;
+}
+
+/* x_ij = s * q_inv * k_inv * sum_d Q[i,h,d] K[j,g,d] */
+static double score(const oracle_attn_params *p, const operand *Q, const operand *K,
+                    int b, int h, int g, int i, int j)
+{
+    double acc = 0.0;
+    for (int dd = 0; dd < p->d; ++dd)
+        acc += ld(Q, idx4(p, p->Hq, b, i, h, dd)) * ld(K, idx4(p, p->Hkv, b, j, g, dd));
+    return p->s * p->q_inv * p->k_inv * acc;
+}
+
+static double quant_p(const oracle_attn_params *p, double pt)
+{
+    /* P~ * c_P is formed as a binary32 product and rounded once to E4M3; returned still scaled by c_P */
+    if (!p->quant) return pt;
+    volatile float prod = (float)pt * (float)p->c_P;
+    return oracle_fp8_decode(oracle_fp8_encode(prod, ORACLE_E4M3), ORACLE_E4M3);
+}
+
+/* Forward for the listed (batch, query head) pairs and query rows [r0, r1).
+ * Reading of where FP8 enters (paper: "QK^T and PV in FP8", nothing more): Q, K, V arrive as E4M3 codes;
+ * scores and the softmax are real-valued; P~ = exp(x - m) is re-quantised to E4M3 with scale c_P right
+ * before the PV product; the row sum l uses the un-quantised P~, so LSE is the true log-sum-exp.
+ * Outputs: O[pair][row][d], LSE[pair][row], mag (sum of |P8||V| with the same normalisation; may be NULL). */
+static void attention_fwd_core(const operand *Q, const operand *K, const operand *V,
+                               const oracle_attn_params *p, const int32_t *bh, int nbh, int r0, int r1,
+                               double *O, double *LSE, double *mag)
+{
+    const int d = p->d, nr = r1 - r0, G = p->Hq / p->Hkv;
+    const double LOG2E = 1.4426950408889634074, LN2 = 0.69314718055994530942;
+    const double cP = p->quant ? p->c_P : 1.0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 8)
+    for (int pi = 0; pi < nbh; ++pi) {
+        for (int i = r0; i < r1; ++i) {
+            const int b = bh[2 * pi], h = bh[2 * pi + 1], g = h / G;
+            const int jlast = p->causal ? i : p->N - 1;
+            const int Bc = p->kv_block > 0 ? p->kv_block : p->N;
+            double *x = (double *)malloc(sizeof(double) * (size_t)Bc);
+            double *acc = (double *)calloc((size_t)d, sizeof(double));
+            double *am = (double *)calloc((size_t)d, sizeof(double));
+            double m = -INFINITY, l = 0.0;
+            for (int j0 = 0; j0 <= jlast; j0 += Bc) {
+                const int j1 = (j0 + Bc - 1 < jlast) ? j0 + Bc - 1 : jlast;
+                double bm = -INFINITY;
+                for (int j = j0; j <= j1; ++j) {
+                    x[j - j0] = score(p, Q, K, b, h, g, i, j);
+                    if (x[j - j0] > bm) bm = x[j - j0];
+                }
+                double cand = (p->max_mode == 1) ? ceil(bm * LOG2E) * LN2 : bm;
+                if (cand > m) {
+                    double f = isinf(m) ? 0.0 : exp(m - cand);
+                    l *= f;
+                    for (int dd = 0; dd < d; ++dd) { acc[dd] *= f; am[dd] *= f; }
+                    m = cand;
+                }
+                for (int j = j0; j <= j1; ++j) {
+                    double pt = exp(x[j - j0] - m);
+                    l += pt;
+                    double w = quant_p(p, pt);
+                    for (int dd = 0; dd < d; ++dd) {
+                        double v = ld(V, idx4(p, p->Hkv, b, j, g, dd));
+                        acc[dd] += w * v;
+                        am[dd] += w * fabs(v);
+                    }
+                }
+            }
+            int64_t o = ((int64_t)pi * nr + (i - r0));
+            for (int dd = 0; dd < d; ++dd) {
+                O[o * d + dd] = p->v_inv * acc[dd] / (cP * l);
+                if (mag) mag[o * d + dd] = p->v_inv * am[dd] / (cP * l);
+            }
+            LSE[o] = m + log(l);
+            free(x); free(acc); free(am);
+        }
+    }
+}
+
+void oracle_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8,
+                          const oracle_attn_params *p, const int32_t *bh, int nbh, int r0, int r1,
+                          double *O, double *LSE, double *mag)
+{
+    operand Q, K, V;
+    operand_init(&Q, Q8, NULL, ORACLE_E4M3);
+    operand_init(&K, K8, NULL, ORACLE_E4M3);
+    operand_init(&V, V8, NULL, ORACLE_E4M3);
+    attention_fwd_core(&Q, &K, &V, p, bh, nbh, r0, r1, O, LSE, mag);
+}
+
+/* Same arithmetic on real-valued operands (used with quant = 0 for the finite-difference pin). */
+void oracle_attention_fwd_real(const double *Qd, const double *Kd, const double *Vd,
+                               const oracle_attn_params *p, const int32_t *bh, int nbh, int r0, int r1,
+                               double *O, double *LSE, double *mag)
+{
+    operand Q, K, V;
+    operand_init(&Q, NULL, Qd, ORACLE_E4M3);
+    operand_init(&K, NULL, Kd, ORACLE_E4M3);
+    operand_init(&V, NULL, Vd, ORACLE_E4M3);
+    attention_fwd_core(&Q, &K, &V, p, bh, nbh, r0, r1, O, LSE, mag);
+}
+
+/* Backward of O = PV through the softmax (the paper runs it in FP8 too but gives no formula; this is the
+ * textbook derivative with the FP8 encodes placed where a GEMM operand is produced):
+ *   D_i  = sum_d dO_id O_id                    P_ij = exp(x_ij - LSE_i)
+ *   dV_j = sum_i P8_ij/c_P * dO_i              dP_ij = dO_i . V_j
+ *   dS_ij = P_ij (dP_ij - D_i)                 dS8 = E5M2(dS * ds_scale)
+ *   dQ_i = s sum_j dS8_ij/ds_scale * K_j       dK_j = s sum_i dS8_ij/ds_scale * Q_i
+ * with dO = do_inv*dec(dO8), V = v_inv*dec(V8) and so on; dK, dV sum over the query heads of a group.
+ * Covers query rows [q0,q1) x key rows [k0,k1) for the listed (batch, kv head) pairs: dQ is complete
+ * when the key range holds every key the rows attend to, dK/dV when the query range holds every query
+ * that attends to the keys.  O is [B,N,Hq,d] and LSE [B,Hq,N], given by the caller.
+ * Outputs: dQ[pair][G][q1-q0][d], dK,dV[pair][k1-k0][d], their magnitude sums (nullable), amax of |dS|. */
+static void attention_bwd_core(const operand *Q, const operand *K, const operand *V, const operand *dO,
+                               const double *O, const double *LSE, const oracle_attn_params *p,
+                               const int32_t *bg, int nbg, int q0, int q1, int k0, int k1,
+                               double *dQ, double *dK, double *dV,
+                               double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS)
+{
+    const int d = p->d, G = p->Hq / p->Hkv, nq = q1 - q0, nk = k1 - k0;
+    const double cP = p->quant ? p->c_P : 1.0;
+    double amax = 0.0;
+    /* D_i for every (pair, head in group, row) */
+    double *D = (double *)malloc(sizeof(double) * (size_t)nbg * G * nq);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int pi = 0; pi < nbg; ++pi)
+        for (int r = 0; r < G * nq; ++r) {
+            const int b = bg[2 * pi], g = bg[2 * pi + 1], h = g * G + r / nq, i = q0 + r % nq;
+            double acc = 0.0;
+            for (int dd = 0; dd < d; ++dd)
+                acc += p->do_inv * ld(dO, idx4(p, p->Hq, b, i, h, dd)) * O[idx4(p, p->Hq, b, i, h, dd)];
+            D[((int64_t)pi * G + r / nq) * nq + r % nq] = acc;
+        }
+
+    /* row-local pass: dQ_i, and amax|dS| */
+#pragma omp parallel for collapse(2) schedule(dynamic, 8) reduction(max : amax)
+    for (int pi = 0; pi < nbg; ++pi)
+        for (int r = 0; r < G * nq; ++r) {
+            const int b = bg[2 * pi], g = bg[2 * pi + 1], hg = r / nq, h = g * G + hg, i = q0 + r % nq;
+            const double lse = LSE[((int64_t)b * p->Hq + h) * p->N + i];
+            const double Di = D[((int64_t)pi * G + hg) * nq + (i - q0)];
+            double *out = dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d;
+            double *mout = mag_dQ ? mag_dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d : NULL;
+            for (int dd = 0; dd < d; ++dd) { out[dd] = 0.0; if (mout) mout[dd] = 0.0; }
+            for (int j = k0; j < k1; ++j) {
+                if (p->causal && j > i) break;
+                double P = exp(score(p, Q, K, b, h, g, i, j) - lse);
+                double dP = 0.0;
+                for (int dd = 0; dd < d; ++dd)
+                    dP += ld(dO, idx4(p, p->Hq, b, i, h, dd)) * ld(V, idx4(p, p->Hkv, b, j, g, dd));
+                dP *= p->do_inv * p->v_inv;
+                double dS = P * (dP - Di);
+                if (fabs(dS) > amax) amax = fabs(dS);
+                double u = dS;
+                if (p->quant) {
+                    volatile float prod = (float)dS * (float)p->ds_scale;
+                    u = oracle_fp8_decode(oracle_fp8_encode(prod, ORACLE_E5M2), ORACLE_E5M2) / p->ds_scale;
+                }
+                for (int dd = 0; dd < d; ++dd) {
+                    double kv = ld(K, idx4(p, p->Hkv, b, j, g, dd));
+                    out[dd] += p->s * p->k_inv * u * kv;
+                    if (mout) mout[dd] += p->s * p->k_inv * fabs(u) * fabs(kv);
+                }
+            }
+        }
+
+    /* column-local pass: dK_j, dV_j (sum over the group's query heads and the query rows) */
+#pragma omp parallel for collapse(2) schedule(dynamic, 8)
+    for (int pi = 0; pi < nbg; ++pi)
+        for (int j = k0; j < k1; ++j) {
+            const int b = bg[2 * pi], g = bg[2 * pi + 1];
+            double *oK = dK + ((int64_t)pi * nk + (j - k0)) * d;
+            double *oV = dV + ((int64_t)pi * nk + (j - k0)) * d;
+            double *mK = mag_dK ? mag_dK + ((int64_t)pi * nk + (j - k0)) * d : NULL;
+            double *mV = mag_dV ? mag_dV + ((int64_t)pi * nk + (j - k0)) * d : NULL;
+            for (int dd = 0; dd < d; ++dd) {
+                oK[dd] = 0.0; oV[dd] = 0.0;
+                if (mK) mK[dd] = 0.0;
+                if (mV) mV[dd] = 0.0;
+            }
+            for (int hg = 0; hg < G; ++hg) {
+                const int h = g * G + hg;
+                for (int i = q0; i < q1; ++i) {
+                    if (p->causal && j > i) continue;
+                    const double lse = LSE[((int64_t)b * p->Hq + h) * p->N + i];
+                    const double Di = D[((int64_t)pi * G + hg) * nq + (i - q0)];
+                    double P = exp(score(p, Q, K, b, h, g, i, j) - lse);
+                    double w = quant_p(p, P) / cP;
+                    double dP = 0.0;
+                    for (int dd = 0; dd < d; ++dd)
+                        dP += ld(dO, idx4(p, p->Hq, b, i, h, dd)) * ld(V, idx4(p, p->Hkv, b, j, g, dd));
+                    dP *= p->do_inv * p->v_inv;
+                    double dS = P * (dP - Di);
+                    double u = dS;
+                    if (p->quant) {
+                        volatile float prod = (float)dS * (float)p->ds_scale;
+                        u = oracle_fp8_decode(oracle_fp8_encode(prod, ORACLE_E5M2), ORACLE_E5M2) / p->ds_scale;
+                    }
+                    for (int dd = 0; dd < d; ++dd) {
+                        double dov = ld(dO, idx4(p, p->Hq, b, i, h, dd));
+                        double qv = ld(Q, idx4(p, p->Hq, b, i, h, dd));
+                        oV[dd] += p->do_inv * w * dov;
+                        oK[dd] += p->s * p->q_inv * u * qv;
+                        if (mV) mV[dd] += p->do_inv * w * fabs(dov);
+                        if (mK) mK[dd] += p->s * p->q_inv * fabs(u) * fabs(qv);
+                    }
+                }
+            }
+        }
+    free(D);
+    if (amax_dS) *amax_dS = amax;
+}
+
+void oracle_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const uint8_t *dO8,
+                          const double *O, const double *LSE, const oracle_attn_params *p,
+                          const int32_t *bg, int nbg, int q0, int q1, int k0, int k1,
+                          double *dQ, double *dK, double *dV,
+                          double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS)
+{
+    operand Q, K, V, dO;
+    operand_init(&Q, Q8, NULL, ORACLE_E4M3);
+    operand_init(&K, K8, NULL, ORACLE_E4M3);
+    operand_init(&V, V8, NULL, ORACLE_E4M3);
+    operand_init(&dO, dO8, NULL, ORACLE_E5M2);
+    attention_bwd_core(&Q, &K, &V, &dO, O, LSE, p, bg, nbg, q0, q1, k0, k1,
+                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS);
+}
+
+void oracle_attention_bwd_real(const double *Qd, const double *Kd, const double *Vd, const double *dOd,
+                               const double *O, const double *LSE, const oracle_attn_params *p,
+                               const int32_t *bg, int nbg, int q0, int q1, int k0, int k1,
+                               double *dQ, double *dK, double *dV,
+                               double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS)
+{
+    operand Q, K, V, dO;
+    operand_init(&Q, NULL, Qd, ORACLE_E4M3);
+    operand_init(&K, NULL, Kd, ORACLE_E4M3);
+    operand_init(&V, NULL, Vd, ORACLE_E4M3);
+    operand_init(&dO, NULL, dOd, ORACLE_E5M2);
+    attention_bwd_core(&Q, &K, &V, &dO, O, LSE, p, bg, nbg, q0, q1, k0, k1,
+                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS);
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,219 @@
+"""Pins of the oracle's attention (Appendix B, Eq. (P): P = Softmax(s QK^T + M), selfattn = PV)."""
+import numpy as np
+import pytest
+
+import oracle as o
+
+ONE = 0x38  # E4M3 code of 1.0
+
+
+def rand_codes(shape, seed, lo=0x20, hi=0x48):
+    """E4M3 codes of moderate magnitude with random signs."""
+    rng = np.random.default_rng(seed)
+    c = rng.integers(lo, hi, size=shape).astype(np.uint8)
+    return c | (rng.integers(0, 2, size=shape).astype(np.uint8) << 7)
+
+
+def dec(c, fmt=o.E4M3):
+    return o.decode_array(c, fmt)
+
+
+def softmax_reference(Q, K, V, s, causal):
+    """Textbook float64 attention for one head: numpy only."""
+    x = s * Q @ K.T
+    if causal:
+        x = np.where(np.tril(np.ones_like(x, dtype=bool)), x, -np.inf)
+    x = x - x.max(axis=1, keepdims=True)
+    P = np.exp(x)
+    P /= P.sum(axis=1, keepdims=True)
+    lse = None
+    return P, P @ V
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("max_mode,kv_block", [(0, 0), (1, 0), (0, 3), (1, 4), (0, 1)])
+def test_unquantised_forward_is_textbook_softmax_attention(causal, max_mode, kv_block):
+    B, N, Hq, Hkv, d = 2, 11, 4, 2, 8
+    q, k, v = rand_codes((B, N, Hq, d), 1), rand_codes((B, N, Hkv, d), 2), rand_codes((B, N, Hkv, d), 3)
+    p = o.attn_params(B, N, Hq, Hkv, d, causal=causal, quant=False, kv_block=kv_block, max_mode=max_mode,
+                      s=0.3, q_inv=0.5, k_inv=2.0, v_inv=0.25)
+    O, LSE, _ = o.attention_fwd(q, k, v, p)
+    Q, K, V = dec(q) * 0.5, dec(k) * 2.0, dec(v) * 0.25
+    for b in range(B):
+        for h in range(Hq):
+            g = h // (Hq // Hkv)                        # grouped-query mapping
+            P, ref = softmax_reference(Q[b, :, h], K[b, :, g], V[b, :, g], 0.3, causal)
+            assert np.allclose(O[b * Hq + h], ref, rtol=1e-12, atol=1e-13)
+            x = 0.3 * Q[b, :, h] @ K[b, :, g].T
+            if causal:
+                x = np.where(np.tril(np.ones_like(x, dtype=bool)), x, -np.inf)
+            assert np.allclose(LSE[b * Hq + h], np.log(np.exp(x).sum(axis=1)), rtol=1e-12)
+
+
+def test_rows_of_P_sum_to_one():
+    """V = identity (d = N) makes O equal to P."""
+    N = 16
+    q, k = rand_codes((1, N, 1, N), 4), rand_codes((1, N, 1, N), 5)
+    v = np.where(np.eye(N, dtype=bool), ONE, 0).astype(np.uint8).reshape(1, N, 1, N)
+    for causal in (True, False):
+        p = o.attn_params(1, N, 1, 1, N, causal=causal, quant=False, s=0.2)
+        O, _, _ = o.attention_fwd(q, k, v, p)
+        assert np.allclose(O[0].sum(axis=1), 1.0, atol=1e-12)
+        if causal:
+            assert np.all(np.triu(O[0], 1) == 0.0)
+
+
+@pytest.mark.parametrize("quant", [True, False])
+def test_closed_forms_single_key_zero_query_first_row(quant):
+    B, N, H, d = 1, 9, 2, 8
+    q, k, v = rand_codes((B, N, H, d), 6), rand_codes((B, N, H, d), 7), rand_codes((B, N, H, d), 8)
+    V = dec(v) * 0.125
+    # N = 1: O = V exactly (P~ = 1 -> code 0x7E = 448 = c_P)
+    p1 = o.attn_params(1, 1, H, H, d, quant=quant, v_inv=0.125, max_mode=0)
+    O, LSE, _ = o.attention_fwd(q[:, :1], k[:, :1], v[:, :1], p1)
+    assert np.array_equal(O[:, 0], V[0, 0])
+    # causal row 0 attends to key 0 only
+    p = o.attn_params(B, N, H, H, d, quant=quant, v_inv=0.125, max_mode=0)
+    O, LSE, _ = o.attention_fwd(q, k, v, p)
+    assert np.array_equal(O[:, 0], V[0, 0])
+    # Q == 0: uniform weights, O_i = mean of V_0..V_i, LSE_i = ln(i+1); exact in FP8 mode as well
+    O, LSE, _ = o.attention_fwd(np.zeros_like(q), k, v, p)
+    for h in range(H):
+        pref = np.cumsum(V[0, :, h], axis=0) / np.arange(1, N + 1)[:, None]
+        assert np.allclose(O[h], pref, rtol=1e-13, atol=0)
+        assert np.allclose(LSE[h], np.log(np.arange(1, N + 1)), rtol=1e-13)
+
+
+def test_key_permutation_invariance_non_causal():
+    B, N, H, d = 1, 12, 1, 8
+    q, k, v = rand_codes((B, N, H, d), 9), rand_codes((B, N, H, d), 10), rand_codes((B, N, H, d), 11)
+    perm = np.random.default_rng(0).permutation(N)
+    for quant in (False, True):
+        p = o.attn_params(B, N, H, H, d, causal=False, quant=quant, kv_block=0)
+        O1, L1, _ = o.attention_fwd(q, k, v, p)
+        O2, L2, _ = o.attention_fwd(q, k[:, perm], v[:, perm], p)
+        assert np.allclose(O1, O2, rtol=1e-12, atol=1e-14) and np.allclose(L1, L2, rtol=1e-13)
+
+
+def test_quantised_forward_matches_stepwise_definition():
+    """quant=on differs from the textbook form only by P8 = E4M3(P~ c_P) in the numerator."""
+    B, N, H, d = 1, 10, 1, 8
+    q, k, v = rand_codes((B, N, H, d), 12), rand_codes((B, N, H, d), 13), rand_codes((B, N, H, d), 14)
+    for max_mode in (0, 1):
+        p = o.attn_params(B, N, H, H, d, quant=True, s=0.4, max_mode=max_mode)
+        O, LSE, mag = o.attention_fwd(q, k, v, p)
+        Q, K, V = dec(q)[0, :, 0], dec(k)[0, :, 0], dec(v)[0, :, 0]
+        x = np.where(np.tril(np.ones((N, N), dtype=bool)), 0.4 * Q @ K.T, -np.inf)
+        m = x.max(axis=1, keepdims=True)
+        if max_mode == 1:
+            m = np.ceil(m * np.log2(np.e)) * np.log(2.0)
+        Pt = np.exp(x - m)
+        P8 = dec(o.encode_array((Pt.astype(np.float32) * np.float32(448.0)), o.E4M3))
+        ref = (P8 @ V) / (448.0 * Pt.sum(axis=1, keepdims=True))
+        assert np.allclose(O[0], ref, rtol=1e-12, atol=1e-14)
+        assert np.allclose(LSE[0], (m + np.log(Pt.sum(axis=1, keepdims=True)))[:, 0], rtol=1e-13)
+        assert np.allclose(mag[0], (P8 @ np.abs(V)) / (448.0 * Pt.sum(axis=1, keepdims=True)), rtol=1e-12)
+        if max_mode == 1:   # reference maximum is an integer number of octaves above the true one
+            assert np.all((Pt.max(axis=1) > 0.5) & (Pt.max(axis=1) <= 1.0))
+
+
+def _fd_setup():
+    rng = np.random.default_rng(21)
+    B, N, Hq, Hkv, d = 1, 8, 2, 1, 4
+    Q, K, V = rng.normal(size=(B, N, Hq, d)), rng.normal(size=(B, N, Hkv, d)), rng.normal(size=(B, N, Hkv, d))
+    dO = rng.normal(size=(B, N, Hq, d))
+    return B, N, Hq, Hkv, d, Q, K, V, dO
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_unquantised_backward_matches_finite_differences(causal):
+    B, N, Hq, Hkv, d, Q, K, V, dO = _fd_setup()
+    s = 0.7
+    p = o.attn_params(B, N, Hq, Hkv, d, causal=causal, quant=False, s=s, max_mode=0)
+
+    def loss(Q_, K_, V_):
+        O, _, _ = o.attention_fwd(Q_, K_, V_, p, real=True)       # [pair=(b,h), row, d]
+        return float((O.reshape(B, Hq, N, d).transpose(0, 2, 1, 3) * dO).sum())
+
+    O, LSE, _ = o.attention_fwd(Q, K, V, p, real=True)
+    Ofull = O.reshape(B, Hq, N, d).transpose(0, 2, 1, 3)
+    g = o.attention_bwd(Q, K, V, dO, Ofull, LSE.reshape(B, Hq, N), p, real=True)
+    dQ = g["dQ"].reshape(B, Hkv, Hq // Hkv, N, d)
+    h = 1e-5
+    for name, T_, grad in (("Q", Q, None), ("K", K, g["dK"]), ("V", V, g["dV"])):
+        for idx in np.ndindex(T_.shape):
+            Tp, Tm = T_.copy(), T_.copy()
+            Tp[idx] += h
+            Tm[idx] -= h
+            args_p = {"Q": (Tp, K, V), "K": (Q, Tp, V), "V": (Q, K, Tp)}[name]
+            args_m = {"Q": (Tm, K, V), "K": (Q, Tm, V), "V": (Q, K, Tm)}[name]
+            fd = (loss(*args_p) - loss(*args_m)) / (2 * h)
+            b, n, hh, dd = idx
+            if name == "Q":
+                an = dQ[b, hh // (Hq // Hkv), hh % (Hq // Hkv), n, dd]
+            else:
+                an = grad[b * Hkv + hh, n, dd]
+            assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (name, idx, fd, an)
+
+
+def test_backward_rows_of_dS_sum_to_zero():
+    """K = identity (d = N) makes dQ_i = s * dS_i, and every row of dS sums to zero."""
+    rng = np.random.default_rng(5)
+    N = 8
+    Q, V, dO = rng.normal(size=(1, N, 1, N)), rng.normal(size=(1, N, 1, N)), rng.normal(size=(1, N, 1, N))
+    K = np.eye(N).reshape(1, N, 1, N)
+    p = o.attn_params(1, N, 1, 1, N, causal=True, quant=False, s=0.9)
+    O, LSE, _ = o.attention_fwd(Q, K, V, p, real=True)
+    g = o.attention_bwd(Q, K, V, dO, O.reshape(1, N, 1, N), LSE.reshape(1, 1, N), p, real=True)
+    assert np.allclose(g["dQ"][0, 0].sum(axis=1), 0.0, atol=1e-13)
+    assert g["amax_dS"] == pytest.approx(np.abs(g["dQ"]).max() / 0.9, rel=1e-12)
+
+
+@pytest.mark.parametrize("quant", [False, True])
+def test_backward_zero_query_closed_form(quant):
+    """Q == 0: P_ij = 1/(i+1); dV_j = sum_{i>=j} P8_ij/c_P dO_i with P8 = E4M3(448/(i+1))."""
+    B, N, H, d = 1, 12, 1, 8
+    k, v = rand_codes((B, N, H, d), 30), rand_codes((B, N, H, d), 31)
+    do = rand_codes((B, N, H, d), 32, 0x10, 0x30)            # read as E5M2 codes
+    q = np.zeros_like(k)
+    p = o.attn_params(B, N, H, H, d, quant=quant, max_mode=0, do_inv=0.5, ds_scale=64.0)
+    O, LSE, _ = o.attention_fwd(q, k, v, p)
+    g = o.attention_bwd(q, k, v, do, O.reshape(B, N, H, d), LSE.reshape(B, H, N), p)
+    dO = dec(do, o.E5M2)[0, :, 0] * 0.5
+    w = 1.0 / np.arange(1, N + 1)
+    if quant:
+        w = dec(o.encode_array((w.astype(np.float32) * np.float32(448.0)), o.E4M3)) / 448.0
+    exp = np.array([(w[j:, None] * dO[j:]).sum(axis=0) for j in range(N)])
+    assert np.allclose(g["dV"][0], exp, rtol=1e-12, atol=1e-15)
+    assert np.all(g["dK"] == 0.0)                            # dK_j = s sum_i dS_ij Q_i with Q = 0
+
+
+def test_backward_ranges_compose():
+    """Partial (query range x key range) results add up to the full backward."""
+    B, N, Hq, Hkv, d = 1, 12, 2, 1, 8
+    q, k, v = rand_codes((B, N, Hq, d), 40), rand_codes((B, N, Hkv, d), 41), rand_codes((B, N, Hkv, d), 42)
+    do = rand_codes((B, N, Hq, d), 43, 0x10, 0x30)
+    p = o.attn_params(B, N, Hq, Hkv, d, quant=True, ds_scale=16.0, do_inv=0.01)
+    O, LSE, _ = o.attention_fwd(q, k, v, p)
+    Of = O.reshape(B, Hq, N, d).transpose(0, 2, 1, 3)
+    L = LSE.reshape(B, Hq, N)
+    full = o.attention_bwd(q, k, v, do, Of, L, p)
+    # causal: rows [0,6) see keys [0,6) only; keys [6,12) are seen by rows [6,12) only
+    a = o.attention_bwd(q, k, v, do, Of, L, p, q_rows=(0, 6), k_rows=(0, 6))
+    b = o.attention_bwd(q, k, v, do, Of, L, p, q_rows=(6, 12), k_rows=(6, 12))
+    assert np.allclose(a["dQ"], full["dQ"][:, :, :6], rtol=1e-13, atol=1e-300)
+    assert np.allclose(b["dK"], full["dK"][:, 6:], rtol=1e-13, atol=1e-300)
+    assert np.allclose(b["dV"], full["dV"][:, 6:], rtol=1e-13, atol=1e-300)
+
+
+def test_softmax_scale_fold_identity():
+    """Section 3 (QK regularisation): a frozen gain g on normalised Q and K equals scaling s by g^2."""
+    B, N, H, d = 1, 6, 1, 8
+    q, k, v = rand_codes((B, N, H, d), 50), rand_codes((B, N, H, d), 51), rand_codes((B, N, H, d), 52)
+    g2 = 2.0 ** 0.5                     # s = 0.125 at d = 128 corresponds to gamma^2 = sqrt(2)
+    p1 = o.attn_params(B, N, H, H, d, quant=False, s=g2 / d ** 0.5)
+    p2 = o.attn_params(B, N, H, H, d, quant=False, s=1 / d ** 0.5, q_inv=g2 ** 0.5, k_inv=g2 ** 0.5)
+    O1, _, _ = o.attention_fwd(q, k, v, p1)
+    O2, _, _ = o.attention_fwd(q, k, v, p2)
+    assert np.allclose(O1, O2, rtol=1e-12)
+    assert abs(0.125 * 128 ** 0.5 - g2) < 1e-12
