@@ -1,0 +1,141 @@
+/*
+ * fp8dpa — C ABI of the FP8 transformer-block hot path on one B200 (sm_100a).
+ *
+ * Every GEMM of the block runs on FP8 operands (forward and backward), fed by per-tensor scaling:
+ *   amax -> scale -> saturating cast (BF16 -> E4M3 for activations/weights, E5M2 for gradients),
+ *   linear forward / dgrad / wgrad, and attention forward / backward with QK^T and PV in FP8.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless it says "host".  The library
+ *     allocates no device memory; scratch comes from the caller (`ws`, sized by the *_workspace_bytes
+ *     functions, 256-byte aligned).
+ *   - Tensor pointers must be 16-byte aligned and row pitches multiples of 16 bytes (128-bit access and
+ *     TMA).  Violations return FP8_ERR_ALIGN / FP8_ERR_SHAPE before anything is launched.
+ *   - `stream` is a cudaStream_t passed as void*; every call only enqueues work on it and returns.
+ *     Scales and amax values are device scalars so that amax -> scale -> cast -> GEMM never syncs the host.
+ *   - Return value: FP8_OK or a negative fp8_status.  fp8_last_error() gives a host string for the last
+ *     failure on the calling thread.  Kernels never spin without bound: a wait that runs out records
+ *     FP8_ERR_TIMEOUT in a device status word, read (and cleared) by fp8_device_status().
+ *   - BF16 tensors are raw 16-bit words; FP8 tensors are raw bytes (codes).
+ *   - There is no CPU fallback: on a device that is not compute capability 10.x every call returns
+ *     FP8_ERR_ARCH.
+ */
+#ifndef FP8DPA_H
+#define FP8DPA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define FP8_API __attribute__((visibility("default")))
+#else
+#define FP8_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { FP8_E4M3 = 0, FP8_E5M2 = 1 } fp8_fmt;
+
+typedef enum {
+    FP8_OK = 0,
+    FP8_ERR_NULL = -1,       /* a required pointer is NULL */
+    FP8_ERR_ALIGN = -2,      /* pointer not 16-byte aligned */
+    FP8_ERR_SHAPE = -3,      /* size zero, pitch not a multiple of 16 bytes, unsupported head_dim, Hq % Hkv != 0 */
+    FP8_ERR_ENUM = -4,       /* bad fp8_fmt */
+    FP8_ERR_WORKSPACE = -5,  /* ws NULL / too small / misaligned */
+    FP8_ERR_CUDA = -6,       /* CUDA runtime or driver error; see fp8_last_error() */
+    FP8_ERR_TIMEOUT = -7,    /* a bounded device-side wait expired (reported by fp8_device_status) */
+    FP8_ERR_ARCH = -8        /* current device is not sm_100 */
+} fp8_status;
+
+/* Host string describing the last non-OK return on this thread (never NULL). */
+FP8_API const char *fp8_last_error(void);
+
+/* Synchronises `stream`, copies the device status word of the current device to *status_out (host; FP8_OK
+ * or FP8_ERR_TIMEOUT) and clears it. */
+FP8_API int fp8_device_status(int *status_out, void *stream);
+
+/* ---- per-tensor scaling ---------------------------------------------------------------------------
+ * Appendix C (definition above Theorem 1): s(x) = MaxFP8Value / absmax(x); Appendix E: rho(X) =
+ * FP8MaxValue / (2^m max H) and FP8cast(rho(X) X).  MaxFP8Value is 448 (E4M3) / 57344 (E5M2). */
+
+/* *amax = max_i |x_i| over n BF16 values (overwritten; exact). */
+FP8_API int fp8_amax(const void *x_bf16, size_t n, float *amax, void *stream);
+
+/* *scale = FP8Max(fmt) / (2^margin * *amax) in binary32 (one IEEE division), *scale_inv = 1 / *scale.
+ * amax == 0 or non-finite gives scale 1; an overflowing quotient gives FLT_MAX. */
+FP8_API int fp8_scale(const float *amax, int fmt, int margin, float *scale, float *scale_inv, void *stream);
+
+/* out[r,c] = sat_rne_fmt( float(x[r,c]) * *scale ): binary32 product, one round-to-nearest-even to FP8,
+ * saturating at +-FP8Max (no Inf/NaN from finite input).  x is [rows, cols] row-major BF16.
+ * out_t (nullable) receives the same codes as [cols, rows]; it needs rows % 16 == 0.
+ * amax_out (nullable) is overwritten with amax(x) in the same pass (for delayed scaling).
+ * cols % 16 == 0 unless rows == 1 (a flat tensor may have any length). */
+FP8_API int fp8_cast(const void *x_bf16, size_t rows, size_t cols, const float *scale, int fmt,
+             uint8_t *out, uint8_t *out_t, float *amax_out, void *stream);
+
+/* Just-in-time scaling of one tensor: fp8_amax, fp8_scale (margin 0) and fp8_cast chained on `stream`
+ * (two passes over x, as Section 2 notes for JIT scaling).  amax, scale, scale_inv are outputs. */
+FP8_API int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fmt, uint8_t *out, uint8_t *out_t,
+                 float *amax, float *scale, float *scale_inv, void *stream);
+
+/* ---- linear layers --------------------------------------------------------------------------------
+ * Appendix E: GEMM(X,Y) = 1/(rho_X rho_Y) * FP8GEMM(FP8cast(rho_X X), FP8cast(rho_Y Y)), BF16 result;
+ * Table "Comparison between FP8 methods": Linear_W(X) = XW for the FFN, QKV and output projections.
+ * Weights are stored [out, in] = [N, K].  Operands are FP8 codes whose reduction index is contiguous;
+ * where the stored tensor has the other orientation, pass the transposed copy fp8_cast produced.
+ * sA_inv / sB_inv are device scalars (1/scale of each operand).  Accumulation is FP32 on the tensor
+ * cores.  Output is BF16 (out_is_fp32 == 0) or FP32, row-major, fully overwritten unless `accumulate`.
+ * Reduction lengths and output widths must be multiples of 16.  ws may be NULL (none needed today). */
+
+/* Y[T,N] = sX_inv*sW_inv * X8[T,K] . W8[N,K]^T         (X8, W8: E4M3) */
+FP8_API int fp8_linear_fwd(const uint8_t *X8, const uint8_t *W8, const float *sX_inv, const float *sW_inv,
+                   void *Y, int out_is_fp32, int T, int N, int K, void *ws, size_t ws_bytes, void *stream);
+
+/* dX[T,K] = sdY_inv*sW_inv * dY8[T,N] . W8t[K,N]^T     (dY8: E5M2; W8t = transposed copy of W8, E4M3) */
+FP8_API int fp8_linear_dgrad(const uint8_t *dY8, const uint8_t *W8t, const float *sdY_inv, const float *sW_inv,
+                     void *dX, int out_is_fp32, int T, int N, int K, void *ws, size_t ws_bytes, void *stream);
+
+/* dW[N,K] (+)= sdY_inv*sX_inv * dY8t[N,T] . X8t[K,T]^T (dY8t: E5M2 [N,T]; X8t: E4M3 [K,T]) */
+FP8_API int fp8_linear_wgrad(const uint8_t *dY8t, const uint8_t *X8t, const float *sdY_inv, const float *sX_inv,
+                     void *dW, int out_is_fp32, int accumulate, int T, int N, int K,
+                     void *ws, size_t ws_bytes, void *stream);
+
+/* ---- attention ------------------------------------------------------------------------------------
+ * Appendix B, Eq. (P): P = Softmax(s Q K^T + M), output P V, grouped-query heads; Appendix E table: both
+ * products in FP8, forward and backward.  Tensors are [B, N, H, d] row-major; query head h reads KV head
+ * h / (Hq/Hkv).  M is the causal mask when `causal` != 0.  d is 64 or 128; N % 16 == 0.
+ *
+ * Forward: scores and softmax in FP32; P~ = exp(x - running max) in (0,1] is re-quantised to E4M3 with
+ * scale p_scale (448 = FP8Max / amax(P~)) before the PV product, keys taken in blocks of 128 in ascending
+ * order; the row sum uses the un-quantised P~.  O is BF16, LSE[b,h,i] the FP32 log-sum-exp (natural log).
+ * Backward: recomputes P = exp(x - LSE); dV = P8^T dO, dP = dO V^T, dS = P o (dP - D) with
+ * D = rowsum(dO o O), dS -> E5M2 with *ds_scale, dQ = s dS8 K, dK = s dS8^T Q; dK, dV summed over the
+ * query heads of a group; *ds_amax (nullable) is overwritten with max|dS|. */
+typedef struct {
+    const float *q_inv, *k_inv, *v_inv; /* device scalars: 1/scale of Q8, K8, V8 */
+    const float *do_inv;                /* device scalar: 1/scale of dO8 (backward only) */
+    float softmax_scale;                /* host value s; 1/sqrt(d) for Llama-style blocks */
+    float p_scale;                      /* host value c_P; 448 */
+    const float *ds_scale;              /* device scalar: quantisation scale of dS (backward only) */
+    float *ds_amax;                     /* device scalar out, nullable (backward only) */
+} fp8_attn_scales;
+
+/* Scratch bytes the attention calls need (op: 0 = forward, 1 = backward). */
+FP8_API size_t fp8_attention_workspace_bytes(int op, int B, int N, int Hq, int Hkv, int d);
+
+FP8_API int fp8_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const fp8_attn_scales *sc,
+                      int causal, int B, int N, int Hq, int Hkv, int d,
+                      void *O_bf16, float *LSE, void *ws, size_t ws_bytes, void *stream);
+
+FP8_API int fp8_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const uint8_t *dO8,
+                      const void *O_bf16, const float *LSE, const fp8_attn_scales *sc,
+                      int causal, int B, int N, int Hq, int Hkv, int d,
+                      void *dQ_bf16, void *dK_bf16, void *dV_bf16, void *ws, size_t ws_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP8DPA_H */

@@ -1,0 +1,11 @@
+"""FP8 transformer-block hot path for one B200 (sm_100a): per-tensor quantize, FP8 linear GEMMs and FP8
+attention behind a C ABI (``include/fp8dpa.h``), with a thin Python binding of the same names.
+
+``binding``  the C-ABI calls (ctypes; torch only supplies device memory and streams)
+``synth``    seeded synthetic inputs shaped like the paper's workloads
+``build``    compiles ``csrc/*.cu`` into ``csrc/libfp8dpa.so``
+"""
+from . import binding  # noqa: F401
+from .binding import (E4M3, E5M2, Fp8Error, fp8_amax, fp8_attention_bwd, fp8_attention_fwd,  # noqa: F401
+                      fp8_attention_workspace_bytes, fp8_cast, fp8_device_status, fp8_last_error,
+                      fp8_linear_dgrad, fp8_linear_fwd, fp8_linear_wgrad, fp8_quantize, fp8_scale)

@@ -1,0 +1,171 @@
+"""ctypes binding of ``libfp8dpa.so`` with the names of ``include/fp8dpa.h``.
+
+Argument marshalling only: every function takes torch CUDA tensors (device memory and streams are torch's),
+passes their addresses through the C ABI and raises ``Fp8Error`` on a non-zero status.  There is no
+fallback of any kind: if the CUDA library is missing or fails to load, importing is fine but the first
+call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+E4M3 = 0
+E5M2 = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
+_lib = None
+
+SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_cast", "fp8_quantize",
+           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_attention_workspace_bytes",
+           "fp8_attention_fwd", "fp8_attention_bwd"]
+
+STATUS_NAMES = {0: "FP8_OK", -1: "FP8_ERR_NULL", -2: "FP8_ERR_ALIGN", -3: "FP8_ERR_SHAPE", -4: "FP8_ERR_ENUM",
+                -5: "FP8_ERR_WORKSPACE", -6: "FP8_ERR_CUDA", -7: "FP8_ERR_TIMEOUT", -8: "FP8_ERR_ARCH"}
+
+
+class Fp8Error(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {msg}")
+        self.status = status
+
+
+class AttnScales(C.Structure):
+    _fields_ = [("q_inv", C.c_void_p), ("k_inv", C.c_void_p), ("v_inv", C.c_void_p), ("do_inv", C.c_void_p),
+                ("softmax_scale", C.c_float), ("p_scale", C.c_float),
+                ("ds_scale", C.c_void_p), ("ds_amax", C.c_void_p)]
+
+
+def load() -> C.CDLL:
+    """Loads the CUDA library; raises if it has not been built (there is nothing to fall back to)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2505_20524_b200.build`")
+        lib = C.CDLL(LIB_PATH)
+        lib.fp8_last_error.restype = C.c_char_p
+        if hasattr(lib, "fp8_attention_workspace_bytes"):
+            lib.fp8_attention_workspace_bytes.restype = C.c_size_t
+            lib.fp8_attention_workspace_bytes.argtypes = [C.c_int] * 6
+        _lib = lib
+    return _lib
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise Fp8Error(rc, load().fp8_last_error().decode())
+
+
+def _ptr(t):
+    if t is None:
+        return C.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous(), "expects contiguous CUDA tensors"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def fp8_last_error() -> str:
+    return load().fp8_last_error().decode()
+
+
+def fp8_device_status(stream=None) -> int:
+    out = C.c_int(0)
+    _check(load().fp8_device_status(C.byref(out), _stream(stream)))
+    return out.value
+
+
+def fp8_amax(x, amax, stream=None):
+    _check(load().fp8_amax(_ptr(x), C.c_size_t(x.numel()), _ptr(amax), _stream(stream)))
+
+
+def fp8_scale(amax, fmt, margin, scale, scale_inv, stream=None):
+    _check(load().fp8_scale(_ptr(amax), C.c_int(fmt), C.c_int(margin), _ptr(scale), _ptr(scale_inv), _stream(stream)))
+
+
+def _rows_cols(x):
+    if x.dim() == 1:
+        return 1, x.numel()
+    return x.numel() // x.shape[-1], x.shape[-1]
+
+
+def fp8_cast(x, scale, fmt, out, out_t=None, amax_out=None, stream=None):
+    rows, cols = _rows_cols(x)
+    _check(load().fp8_cast(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), _ptr(scale), C.c_int(fmt), _ptr(out),
+                           _ptr(out_t), _ptr(amax_out), _stream(stream)))
+
+
+def fp8_quantize(x, fmt, out, out_t, amax, scale, scale_inv, stream=None):
+    rows, cols = _rows_cols(x)
+    _check(load().fp8_quantize(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), C.c_int(fmt), _ptr(out), _ptr(out_t),
+                               _ptr(amax), _ptr(scale), _ptr(scale_inv), _stream(stream)))
+
+
+def _is_fp32(t):
+    if t.dtype == torch.float32:
+        return 1
+    assert t.dtype in (torch.bfloat16, torch.int16, torch.uint16), "output must be BF16 or FP32"
+    return 0
+
+
+def fp8_linear_fwd(x8, w8, sx_inv, sw_inv, y, ws=None, stream=None):
+    T, K = x8.shape
+    N = w8.shape[0]
+    _check(load().fp8_linear_fwd(_ptr(x8), _ptr(w8), _ptr(sx_inv), _ptr(sw_inv), _ptr(y), C.c_int(_is_fp32(y)),
+                                 C.c_int(T), C.c_int(N), C.c_int(K), _ptr(ws),
+                                 C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()), _stream(stream)))
+
+
+def fp8_linear_dgrad(dy8, w8t, sdy_inv, sw_inv, dx, ws=None, stream=None):
+    T, N = dy8.shape
+    K = w8t.shape[0]
+    _check(load().fp8_linear_dgrad(_ptr(dy8), _ptr(w8t), _ptr(sdy_inv), _ptr(sw_inv), _ptr(dx),
+                                   C.c_int(_is_fp32(dx)), C.c_int(T), C.c_int(N), C.c_int(K), _ptr(ws),
+                                   C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()), _stream(stream)))
+
+
+def fp8_linear_wgrad(dy8t, x8t, sdy_inv, sx_inv, dw, accumulate=False, ws=None, stream=None):
+    N, T = dy8t.shape
+    K = x8t.shape[0]
+    _check(load().fp8_linear_wgrad(_ptr(dy8t), _ptr(x8t), _ptr(sdy_inv), _ptr(sx_inv), _ptr(dw),
+                                   C.c_int(_is_fp32(dw)), C.c_int(int(accumulate)), C.c_int(T), C.c_int(N),
+                                   C.c_int(K), _ptr(ws),
+                                   C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()), _stream(stream)))
+
+
+def fp8_attention_workspace_bytes(op, B, N, Hq, Hkv, d) -> int:
+    return int(load().fp8_attention_workspace_bytes(op, B, N, Hq, Hkv, d))
+
+
+def _scales(q_inv, k_inv, v_inv, do_inv, softmax_scale, p_scale, ds_scale, ds_amax):
+    return AttnScales(_ptr(q_inv).value, _ptr(k_inv).value, _ptr(v_inv).value, _ptr(do_inv).value,
+                      float(softmax_scale), float(p_scale), _ptr(ds_scale).value, _ptr(ds_amax).value)
+
+
+def fp8_attention_fwd(q8, k8, v8, q_inv, k_inv, v_inv, softmax_scale, causal, o, lse, ws, p_scale=448.0,
+                      stream=None):
+    B, N, Hq, d = q8.shape
+    Hkv = k8.shape[2]
+    sc = _scales(q_inv, k_inv, v_inv, None, softmax_scale, p_scale, None, None)
+    _check(load().fp8_attention_fwd(_ptr(q8), _ptr(k8), _ptr(v8), C.byref(sc), C.c_int(int(causal)), C.c_int(B),
+                                    C.c_int(N), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), _ptr(o), _ptr(lse),
+                                    _ptr(ws), C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+                                    _stream(stream)))
+
+
+def fp8_attention_bwd(q8, k8, v8, do8, o, lse, q_inv, k_inv, v_inv, do_inv, softmax_scale, ds_scale, causal,
+                      dq, dk, dv, ws, ds_amax=None, p_scale=448.0, stream=None):
+    B, N, Hq, d = q8.shape
+    Hkv = k8.shape[2]
+    sc = _scales(q_inv, k_inv, v_inv, do_inv, softmax_scale, p_scale, ds_scale, ds_amax)
+    _check(load().fp8_attention_bwd(_ptr(q8), _ptr(k8), _ptr(v8), _ptr(do8), _ptr(o), _ptr(lse), C.byref(sc),
+                                    C.c_int(int(causal)), C.c_int(B), C.c_int(N), C.c_int(Hq), C.c_int(Hkv),
+                                    C.c_int(d), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws),
+                                    C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
+                                    _stream(stream)))

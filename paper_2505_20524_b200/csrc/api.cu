@@ -1,0 +1,137 @@
+// Host-side state shared by every entry point: error text, the device status word, architecture check,
+// and the tensor-map encoder fetched from the driver at run time (the library does not link libcuda).
+#include <stdarg.h>
+#include <stdio.h>
+
+#include "common.cuh"
+
+namespace fp8dpa {
+
+static thread_local char g_err[512] = "no error";
+
+void set_error(const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+// One status word per device (each device that loads the module gets its own copy of the symbol).
+__device__ int g_device_status = 0;
+
+static const int kMaxDevices = 64;
+static int *g_status_ptr[kMaxDevices] = {nullptr};
+static int g_arch_ok[kMaxDevices] = {0};   // 0 unknown, 1 ok, -1 wrong arch
+static int g_sm_count[kMaxDevices] = {0};
+
+static int current_device()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
+int *device_status_ptr()
+{
+    int dev = current_device();
+    if (dev < 0) return nullptr;
+    if (!g_status_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) {
+            set_error("cudaGetSymbolAddress(status word) failed: %s", cudaGetErrorString(cudaGetLastError()));
+            return nullptr;
+        }
+        g_status_ptr[dev] = static_cast<int *>(p);
+    }
+    return g_status_ptr[dev];
+}
+
+int check_arch()
+{
+    int dev = current_device();
+    if (dev < 0) {
+        set_error("no current CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+        return FP8_ERR_CUDA;
+    }
+    if (g_arch_ok[dev] == 0) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            set_error("cudaDeviceGetAttribute failed: %s", cudaGetErrorString(cudaGetLastError()));
+            return FP8_ERR_CUDA;
+        }
+        g_arch_ok[dev] = (major == 10) ? 1 : -1;
+        g_sm_count[dev] = sms;
+    }
+    if (g_arch_ok[dev] < 0) {
+        set_error("this library only runs on compute capability 10.x (sm_100a); no fallback exists");
+        return FP8_ERR_ARCH;
+    }
+    return FP8_OK;
+}
+
+int sm_count()
+{
+    int dev = current_device();
+    return (dev >= 0 && g_sm_count[dev] > 0) ? g_sm_count[dev] : 148;
+}
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+static encode_tiled_fn g_encode = nullptr;
+
+static int load_encoder()
+{
+    if (g_encode) return FP8_OK;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
+        set_error("cuTensorMapEncodeTiled not available from the driver (%s)", cudaGetErrorString(e));
+        return FP8_ERR_CUDA;
+    }
+    g_encode = reinterpret_cast<encode_tiled_fn>(fn);
+    return FP8_OK;
+}
+
+int make_tmap_2d_u8(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint64_t pitch,
+                    uint32_t box_rows, uint32_t box_cols)
+{
+    int rc = load_encoder();
+    if (rc != FP8_OK) return rc;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {pitch};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled failed (CUresult %d) rows=%llu cols=%llu pitch=%llu box=%ux%u", (int)r,
+                  (unsigned long long)rows, (unsigned long long)cols, (unsigned long long)pitch, box_rows, box_cols);
+        return FP8_ERR_CUDA;
+    }
+    return FP8_OK;
+}
+
+}  // namespace fp8dpa
+
+extern "C" const char *fp8_last_error(void) { return fp8dpa::g_err; }
+
+extern "C" int fp8_device_status(int *status_out, void *stream)
+{
+    if (!status_out) {
+        fp8dpa::set_error("fp8_device_status: status_out is NULL");
+        return FP8_ERR_NULL;
+    }
+    int *p = fp8dpa::device_status_ptr();
+    if (!p) return FP8_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    FP8_CUDA_CHECK(cudaStreamSynchronize(s));
+    FP8_CUDA_CHECK(cudaMemcpy(status_out, p, sizeof(int), cudaMemcpyDeviceToHost));
+    FP8_CUDA_CHECK(cudaMemset(p, 0, sizeof(int)));
+    return FP8_OK;
+}

@@ -1,0 +1,307 @@
+// FP8 x FP8 -> FP32-accumulate GEMM on the 5th-generation tensor cores (tcgen05.mma.kind::f8f6f4).
+//
+//   C[M,N] (+)= sa_inv * sb_inv * A[M,K] . B[N,K]^T        A, B: FP8 codes, reduction index contiguous
+//
+// One persistent CTA per SM walks over 128 x BN output tiles.  Warp roles:
+//   warp 0    TMA producer: 128-byte-swizzled [128 x 128 B] / [BN x 128 B] boxes into a 4-stage ring
+//   warp 1    MMA issuer (one elected lane): 4 x (128 x BN x 32) MMAs per stage, accumulators in TMEM,
+//             two accumulator buffers so the epilogue of tile i overlaps the main loop of tile i+1
+//   warps 2-5 epilogue: tcgen05.ld -> descale -> BF16/FP32 -> 16-byte global stores
+// Every wait is bounded; on expiry the CTA records FP8_ERR_TIMEOUT and drains.
+#include "common.cuh"
+
+namespace fp8dpa {
+
+constexpr int G_BM = 128;
+constexpr int G_BK = 128;         // bytes = FP8 elements per stage row (one swizzle span)
+constexpr int G_STAGES = 4;
+constexpr int G_THREADS = 192;
+
+template <int BN>
+struct GemmSmem {
+    static constexpr int A_BYTES = G_BM * G_BK;
+    static constexpr int B_BYTES = BN * G_BK;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int BAR_OFFSET = G_STAGES * STAGE_BYTES;
+    // full[S], empty[S], tmem_full[2], tmem_empty[2], tmem base slot, abort flag
+    static constexpr int TOTAL = BAR_OFFSET + (2 * G_STAGES + 4) * 8 + 16;
+    static constexpr int DYN_BYTES = TOTAL + 1024;   // slack for manual 1024-byte alignment
+};
+
+struct GemmParams {
+    void *out;
+    const float *sa_inv, *sb_inv;
+    int M, N, K;
+    int out_is_fp32, accumulate;
+    uint32_t idesc;
+    int *status;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(G_THREADS, 1)
+gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                const GemmParams p)
+{
+    using L = GemmSmem<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_base = sbase + L::BAR_OFFSET;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (G_STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * G_STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * G_STAGES + 2 + b); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFFSET + (2 * G_STAGES + 4) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_m = (p.M + G_BM - 1) / G_BM, tiles_n = (p.N + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
+    const int k_blocks = (p.K + G_BK - 1) / G_BK;
+    constexpr uint32_t TMEM_COLS = 2 * BN;   // 256 or 512: a power of two >= 32
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < G_STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 4);   // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const WaitCtx ctx{p.status, abort_flag};
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % tiles_m) * G_BM, n0 = (tile / tiles_m) * BN;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctx)) { ok = false; break; }
+                    const uint32_t sa = sbase + stage * L::STAGE_BYTES, sb = sa + L::A_BYTES;
+                    mbar_expect_tx(full_bar(stage), L::STAGE_BYTES);
+                    tma_load_2d(sa, &tmap_a, full_bar(stage), kb * G_BK, m0);
+                    tma_load_2d(sb, &tmap_b, full_bar(stage), kb * G_BK, n0);
+                    if (++stage == G_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+                const int buf = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), acc_phase ^ 1u, ctx)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, ctx)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = sbase + stage * L::STAGE_BYTES, sb = sa + L::A_BYTES;
+                    const uint64_t da = umma_desc_k_sw128(sa), db = umma_desc_k_sw128(sb);
+#pragma unroll
+                    for (int k = 0; k < G_BK / 32; ++k) {
+                        // advance 32 bytes along the reduction index inside the swizzle span: +2 (16-byte units)
+                        umma_f8_ss(tmem_d, da + 2u * k, db + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
+                    if (++stage == G_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(tfull_bar(buf));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int quad = warp & 3;                     // TMEM lanes 32*quad .. 32*quad+31
+        const float descale = __ldg(p.sa_inv) * __ldg(p.sb_inv);
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
+            const int buf = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            const int m0 = (tile % tiles_m) * G_BM, n0 = (tile / tiles_m) * BN;
+            if (!mbar_wait(tfull_bar(buf), acc_phase, ctx)) { ok = false; break; }
+            tc_fence_after();
+            const int row = m0 + quad * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN);
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(taddr + (uint32_t)c, r);
+                tmem_ld_wait();
+                const int col = n0 + c;
+                if (row < p.M && col < p.N) {
+                    // N is a multiple of 16, so a 32-column chunk is either whole or half inside
+                    const int ncols = min(32, p.N - col);
+                    if (p.out_is_fp32) {
+                        float *dst = static_cast<float *>(p.out) + (size_t)row * p.N + col;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            if (j < ncols) {
+                                float4 v = make_float4(__uint_as_float(r[j]) * descale, __uint_as_float(r[j + 1]) * descale,
+                                                       __uint_as_float(r[j + 2]) * descale,
+                                                       __uint_as_float(r[j + 3]) * descale);
+                                if (p.accumulate) {
+                                    const float4 o = *reinterpret_cast<const float4 *>(dst + j);
+                                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                                }
+                                *reinterpret_cast<float4 *>(dst + j) = v;
+                            }
+                        }
+                    } else {
+                        uint16_t *dst = static_cast<uint16_t *>(p.out) + (size_t)row * p.N + col;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            if (j < ncols) {
+                                float v[8];
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(r[j + q]) * descale;
+                                if (p.accumulate) {
+                                    const uint4 o = *reinterpret_cast<const uint4 *>(dst + j);
+                                    v[0] += bf16_lo(o.x); v[1] += bf16_hi(o.x); v[2] += bf16_lo(o.y); v[3] += bf16_hi(o.y);
+                                    v[4] += bf16_lo(o.z); v[5] += bf16_hi(o.z); v[6] += bf16_lo(o.w); v[7] += bf16_hi(o.w);
+                                }
+                                *reinterpret_cast<uint4 *>(dst + j) =
+                                    make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                                               pack_bf16x2(v[6], v[7]));
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown (all roles fall through)
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait gave up: let copies that may still be in flight land before the CTA's memory is released
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+static int validate_gemm(const char *who, const void *a, const void *b, const float *sa, const float *sb, void *out,
+                         int M, int N, int K)
+{
+    if (!a || !b || !sa || !sb || !out) {
+        set_error("%s: NULL pointer", who);
+        return FP8_ERR_NULL;
+    }
+    if (M <= 0 || N <= 0 || K <= 0 || (K % 16) || (N % 16)) {
+        set_error("%s: unsupported shape (rows=%d cols=%d reduce=%d; cols and reduce must be positive multiples of 16)",
+                  who, M, N, K);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(a) || !aligned16(b) || !aligned16(out)) {
+        set_error("%s: tensor pointers must be 16-byte aligned", who);
+        return FP8_ERR_ALIGN;
+    }
+    return FP8_OK;
+}
+
+template <int BN>
+static int launch_gemm(const uint8_t *a, const uint8_t *b, const GemmParams &p, cudaStream_t st)
+{
+    CUtensorMap ta, tb;
+    int rc = make_tmap_2d_u8(&ta, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, G_BM, G_BK);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_2d_u8(&tb, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN, G_BK);
+    if (rc != FP8_OK) return rc;
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        GemmSmem<BN>::DYN_BYTES));
+    const int tiles = ((p.M + G_BM - 1) / G_BM) * ((p.N + BN - 1) / BN);
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    gemm_fp8_kernel<BN><<<grid, G_THREADS, GemmSmem<BN>::DYN_BYTES, st>>>(ta, tb, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+// C[M,N] (+)= sa_inv*sb_inv * A[M,K] . B[N,K]^T
+int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int fmt_b, const float *sa_inv,
+             const float *sb_inv, void *out, int out_is_fp32, int accumulate, int M, int N, int K, cudaStream_t st)
+{
+    int rc = validate_gemm(who, a, b, sa_inv, sb_inv, out, M, N, K);
+    if (rc != FP8_OK) return rc;
+    rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    GemmParams p;
+    p.out = out;
+    p.sa_inv = sa_inv;
+    p.sb_inv = sb_inv;
+    p.M = M; p.N = N; p.K = K;
+    p.out_is_fp32 = out_is_fp32;
+    p.accumulate = accumulate;
+    p.status = device_status_ptr();
+    if (!p.status) return FP8_ERR_CUDA;
+    // 128 x 256 tiles when that still fills the machine, 128 x 128 otherwise
+    const long tiles256 = (long)((M + 127) / 128) * ((N + 255) / 256);
+    if (N >= 256 && tiles256 >= sm_count()) {
+        p.idesc = umma_idesc_f8(fmt_a, fmt_b, G_BM, 256);
+        return launch_gemm<256>(a, b, p, st);
+    }
+    p.idesc = umma_idesc_f8(fmt_a, fmt_b, G_BM, 128);
+    return launch_gemm<128>(a, b, p, st);
+}
+
+}  // namespace fp8dpa
+
+using namespace fp8dpa;
+
+extern "C" int fp8_linear_fwd(const uint8_t *X8, const uint8_t *W8, const float *sX_inv, const float *sW_inv, void *Y,
+                              int out_is_fp32, int T, int N, int K, void *ws, size_t ws_bytes, void *stream)
+{
+    (void)ws; (void)ws_bytes;
+    return gemm_fp8("fp8_linear_fwd", X8, FP8_E4M3, W8, FP8_E4M3, sX_inv, sW_inv, Y, out_is_fp32, 0, T, N, K,
+                    static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int fp8_linear_dgrad(const uint8_t *dY8, const uint8_t *W8t, const float *sdY_inv, const float *sW_inv,
+                                void *dX, int out_is_fp32, int T, int N, int K, void *ws, size_t ws_bytes,
+                                void *stream)
+{
+    (void)ws; (void)ws_bytes;
+    // dX[T,K] = dY8[T,N] . W8t[K,N]^T : rows T, cols K, reduce N
+    return gemm_fp8("fp8_linear_dgrad", dY8, FP8_E5M2, W8t, FP8_E4M3, sdY_inv, sW_inv, dX, out_is_fp32, 0, T, K, N,
+                    static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int fp8_linear_wgrad(const uint8_t *dY8t, const uint8_t *X8t, const float *sdY_inv, const float *sX_inv,
+                                void *dW, int out_is_fp32, int accumulate, int T, int N, int K, void *ws,
+                                size_t ws_bytes, void *stream)
+{
+    (void)ws; (void)ws_bytes;
+    // dW[N,K] = dY8t[N,T] . X8t[K,T]^T : rows N, cols K, reduce T
+    return gemm_fp8("fp8_linear_wgrad", dY8t, FP8_E5M2, X8t, FP8_E4M3, sdY_inv, sX_inv, dW, out_is_fp32, accumulate,
+                    N, K, T, static_cast<cudaStream_t>(stream));
+}

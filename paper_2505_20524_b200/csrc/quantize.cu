@@ -1,0 +1,346 @@
+// Per-tensor scaling kernels: amax reduction, scale computation, saturating BF16 -> FP8 cast
+// (optionally with a transposed copy and a fused amax).  All are HBM streams: 128-bit loads and stores,
+// warp-shuffle + one atomic per CTA for the reduction, scales read from device memory.
+//
+// No fast-math on this file: the binary32 division and product below define the bit-exact result.
+#include <float.h>
+
+#include "common.cuh"
+
+namespace fp8dpa {
+
+// ---------------------------------------------------------------- amax
+__device__ __forceinline__ uint32_t absmax2(uint32_t m, uint32_t w) { return __vmaxu2(m, w & 0x7FFF7FFFu); }
+
+__device__ __forceinline__ void block_atomic_max_bf16(uint32_t m2, unsigned int *amax_bits)
+{
+    __shared__ uint32_t warp_max[32];
+    uint32_t m = max(m2 & 0xFFFFu, m2 >> 16);
+    m = __reduce_max_sync(0xffffffffu, m);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) warp_max[warp] = m;
+    __syncthreads();
+    if (warp == 0) {
+        const int nwarps = (blockDim.x + 31) >> 5;
+        m = lane < nwarps ? warp_max[lane] : 0u;
+        m = __reduce_max_sync(0xffffffffu, m);
+        // |x| as BF16 bits << 16 is the binary32 pattern of |x|; positive floats order like unsigned ints
+        if (lane == 0 && m != 0u) atomicMax(amax_bits, m << 16);
+    }
+}
+
+__global__ void __launch_bounds__(512) amax_kernel(const uint4 *__restrict__ x, size_t n_vec,
+                                                   const uint16_t *__restrict__ tail, int n_tail,
+                                                   unsigned int *__restrict__ amax_bits)
+{
+    uint32_t m = 0;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // four independent 16-byte loads in flight per thread
+    for (; i + 3 * stride < n_vec; i += 4 * stride) {
+        const uint4 a = __ldg(x + i), b = __ldg(x + i + stride), c = __ldg(x + i + 2 * stride),
+                    d = __ldg(x + i + 3 * stride);
+        m = absmax2(absmax2(absmax2(absmax2(m, a.x), a.y), a.z), a.w);
+        m = absmax2(absmax2(absmax2(absmax2(m, b.x), b.y), b.z), b.w);
+        m = absmax2(absmax2(absmax2(absmax2(m, c.x), c.y), c.z), c.w);
+        m = absmax2(absmax2(absmax2(absmax2(m, d.x), d.y), d.z), d.w);
+    }
+    for (; i < n_vec; i += stride) {
+        const uint4 a = __ldg(x + i);
+        m = absmax2(absmax2(absmax2(absmax2(m, a.x), a.y), a.z), a.w);
+    }
+    if (blockIdx.x == 0 && (int)threadIdx.x < n_tail) m = absmax2(m, (uint32_t)tail[threadIdx.x]);
+    block_atomic_max_bf16(m, amax_bits);
+}
+
+// ---------------------------------------------------------------- scale
+__global__ void scale_kernel(const float *__restrict__ amax, float fp8_max, int margin, float *__restrict__ scale,
+                             float *__restrict__ scale_inv)
+{
+    const float a = *amax;
+    float s;
+    if (!(a > 0.0f) || isinf(a)) {
+        s = 1.0f;
+    } else {
+        s = __fmul_rn(__fdiv_rn(fp8_max, a), ldexpf(1.0f, -margin));   // power-of-two factor: exact
+        if (isinf(s)) s = FLT_MAX;
+    }
+    *scale = s;
+    *scale_inv = __fdiv_rn(1.0f, s);
+}
+
+// ---------------------------------------------------------------- cast
+// 8 BF16 (one 16-byte word) -> 8 FP8 codes (two 32-bit words); each product is one binary32 multiply.
+template <int FMT>
+__device__ __forceinline__ uint2 cast8(const uint4 v, const float s)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint16_t h[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        h[i] = cvt_f32x2_to_fp8x2<FMT>(__fmul_rn(bf16_lo(w[i]), s), __fmul_rn(bf16_hi(w[i]), s));
+    return make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
+}
+
+template <int FMT, bool AMAX>
+__global__ void __launch_bounds__(256) cast_flat_kernel(const uint4 *__restrict__ x, size_t n16,
+                                                        const uint16_t *__restrict__ tail_in,
+                                                        uint8_t *__restrict__ tail_out, int n_tail,
+                                                        const float *__restrict__ scale_ptr,
+                                                        uint4 *__restrict__ out, unsigned int *__restrict__ amax_bits)
+{
+    const float s = __ldg(scale_ptr);
+    uint32_t m = 0;
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + stride < n16; i += 2 * stride) {
+        const uint4 a0 = __ldg(x + 2 * i), a1 = __ldg(x + 2 * i + 1);
+        const uint4 b0 = __ldg(x + 2 * (i + stride)), b1 = __ldg(x + 2 * (i + stride) + 1);
+        if (AMAX) {
+            m = absmax2(absmax2(absmax2(absmax2(m, a0.x), a0.y), a0.z), a0.w);
+            m = absmax2(absmax2(absmax2(absmax2(m, a1.x), a1.y), a1.z), a1.w);
+            m = absmax2(absmax2(absmax2(absmax2(m, b0.x), b0.y), b0.z), b0.w);
+            m = absmax2(absmax2(absmax2(absmax2(m, b1.x), b1.y), b1.z), b1.w);
+        }
+        const uint2 p0 = cast8<FMT>(a0, s), p1 = cast8<FMT>(a1, s);
+        const uint2 q0 = cast8<FMT>(b0, s), q1 = cast8<FMT>(b1, s);
+        out[i] = make_uint4(p0.x, p0.y, p1.x, p1.y);
+        out[i + stride] = make_uint4(q0.x, q0.y, q1.x, q1.y);
+    }
+    for (; i < n16; i += stride) {
+        const uint4 a0 = __ldg(x + 2 * i), a1 = __ldg(x + 2 * i + 1);
+        if (AMAX) {
+            m = absmax2(absmax2(absmax2(absmax2(m, a0.x), a0.y), a0.z), a0.w);
+            m = absmax2(absmax2(absmax2(absmax2(m, a1.x), a1.y), a1.z), a1.w);
+        }
+        const uint2 p0 = cast8<FMT>(a0, s), p1 = cast8<FMT>(a1, s);
+        out[i] = make_uint4(p0.x, p0.y, p1.x, p1.y);
+    }
+    if (blockIdx.x == 0 && (int)threadIdx.x < n_tail) {
+        const uint32_t w = tail_in[threadIdx.x];
+        if (AMAX) m = absmax2(m, w);
+        const float p = __fmul_rn(bf16_lo(w), s);
+        tail_out[threadIdx.x] = (uint8_t)(cvt_f32x2_to_fp8x2<FMT>(p, 0.0f) & 0xFF);
+    }
+    if (AMAX) block_atomic_max_bf16(m, amax_bits);
+}
+
+// Cast + transposed copy: one CTA per 128 x 128 tile.  Codes go straight to `out` (16-byte stores) and
+// into a padded shared tile, which is then read column-wise so that `out_t` also gets 16-byte stores with
+// two lanes covering each 32-byte sector.
+constexpr int TT = 128;          // tile edge
+constexpr int TPITCH = TT + 4;   // 33 words per row: column reads hit distinct banks
+
+template <int FMT, bool AMAX>
+__global__ void __launch_bounds__(256) cast_transpose_kernel(const uint16_t *__restrict__ x, int rows, int cols,
+                                                             const float *__restrict__ scale_ptr,
+                                                             uint8_t *__restrict__ out, uint8_t *__restrict__ out_t,
+                                                             unsigned int *__restrict__ amax_bits)
+{
+    __shared__ __align__(16) uint8_t tile[TT * TPITCH];
+    const float s = __ldg(scale_ptr);
+    const int r0 = blockIdx.y * TT, c0 = blockIdx.x * TT;
+    uint32_t m = 0;
+    // phase 1: 128 rows x 8 groups of 16 columns
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int idx = it * 256 + threadIdx.x;
+        const int r = idx >> 3, cg = idx & 7;
+        const int gr = r0 + r, gc = c0 + cg * 16;
+        if (gr < rows && gc < cols) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(x + (size_t)gr * cols + gc);
+            const uint4 a0 = __ldg(src), a1 = __ldg(src + 1);
+            if (AMAX) {
+                m = absmax2(absmax2(absmax2(absmax2(m, a0.x), a0.y), a0.z), a0.w);
+                m = absmax2(absmax2(absmax2(absmax2(m, a1.x), a1.y), a1.z), a1.w);
+            }
+            const uint2 p0 = cast8<FMT>(a0, s), p1 = cast8<FMT>(a1, s);
+            if (out) *reinterpret_cast<uint4 *>(out + (size_t)gr * cols + gc) = make_uint4(p0.x, p0.y, p1.x, p1.y);
+            uint32_t *t = reinterpret_cast<uint32_t *>(tile + r * TPITCH + cg * 16);
+            t[0] = p0.x; t[1] = p0.y; t[2] = p1.x; t[3] = p1.y;
+        }
+    }
+    __syncthreads();
+    // phase 2: 128 columns x 8 groups of 16 rows; lanes (2k, 2k+1) write the two halves of one 32-byte sector
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int idx = it * 256 + threadIdx.x;
+        const int half = idx & 1, c = (idx >> 1) & 127, rp = idx >> 8;   // rp: pair of row groups (0..3)
+        const int rg = rp * 2 + half;
+        const int gc = c0 + c, gr = r0 + rg * 16;
+        if (gc < cols && gr < rows) {
+            uint32_t w[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t v = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) v |= (uint32_t)tile[(rg * 16 + q * 4 + b) * TPITCH + c] << (8 * b);
+                w[q] = v;
+            }
+            *reinterpret_cast<uint4 *>(out_t + (size_t)gc * rows + gr) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+    if (AMAX) block_atomic_max_bf16(m, amax_bits);
+}
+
+static int validate_cast(const void *x, size_t rows, size_t cols, const float *scale, int fmt, uint8_t *out,
+                         uint8_t *out_t)
+{
+    if (!x || !scale || (!out && !out_t)) {
+        set_error("fp8_cast: NULL pointer (x=%p scale=%p out=%p out_t=%p)", x, (const void *)scale, (void *)out,
+                  (void *)out_t);
+        return FP8_ERR_NULL;
+    }
+    if (fmt != FP8_E4M3 && fmt != FP8_E5M2) {
+        set_error("fp8_cast: fmt %d is not FP8_E4M3 / FP8_E5M2", fmt);
+        return FP8_ERR_ENUM;
+    }
+    if (rows == 0 || cols == 0) {
+        set_error("fp8_cast: empty tensor (rows=%zu cols=%zu)", rows, cols);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(x) || !aligned16(out) || !aligned16(out_t)) {
+        set_error("fp8_cast: tensor pointers must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    if (out_t && (rows % 16 || cols % 16)) {
+        set_error("fp8_cast: transposed copy needs rows %% 16 == 0 and cols %% 16 == 0 (rows=%zu cols=%zu)", rows, cols);
+        return FP8_ERR_SHAPE;
+    }
+    if (!out_t && rows != 1 && cols % 16) {
+        set_error("fp8_cast: cols %% 16 != 0 for a 2-D tensor (cols=%zu)", cols);
+        return FP8_ERR_SHAPE;
+    }
+    if (rows > 0x7FFFFFFFull || cols > 0x7FFFFFFFull) {
+        set_error("fp8_cast: rows/cols beyond 2^31-1");
+        return FP8_ERR_SHAPE;
+    }
+    return FP8_OK;
+}
+
+template <int FMT, bool AMAX>
+static void launch_cast(const void *x, size_t rows, size_t cols, const float *scale, uint8_t *out, uint8_t *out_t,
+                        float *amax_out, cudaStream_t st)
+{
+    unsigned int *ab = reinterpret_cast<unsigned int *>(amax_out);
+    if (out_t) {
+        dim3 grid((unsigned)((cols + TT - 1) / TT), (unsigned)((rows + TT - 1) / TT));
+        cast_transpose_kernel<FMT, AMAX><<<grid, 256, 0, st>>>(static_cast<const uint16_t *>(x), (int)rows, (int)cols,
+                                                             scale, out, out_t, ab);
+    } else {
+        const size_t n = rows * cols, n16 = n / 16;
+        const int n_tail = (int)(n - n16 * 16);
+        size_t blocks = (n16 + 2 * 256 - 1) / (2 * 256);
+        const size_t cap = (size_t)sm_count() * 8;
+        if (blocks > cap) blocks = cap;
+        if (blocks == 0) blocks = 1;
+        cast_flat_kernel<FMT, AMAX><<<(unsigned)blocks, 256, 0, st>>>(
+            static_cast<const uint4 *>(x), n16, static_cast<const uint16_t *>(x) + n16 * 16, out + n16 * 16, n_tail,
+            scale, reinterpret_cast<uint4 *>(out), ab);
+    }
+}
+
+static int do_amax(const void *x, size_t n, float *amax, cudaStream_t st)
+{
+    FP8_CUDA_CHECK(cudaMemsetAsync(amax, 0, sizeof(float), st));
+    const size_t n_vec = n / 8;
+    const int n_tail = (int)(n - n_vec * 8);
+    size_t blocks = (n_vec + 4 * 512 - 1) / (4 * 512);
+    const size_t cap = (size_t)sm_count() * 4;
+    if (blocks > cap) blocks = cap;
+    if (blocks == 0) blocks = 1;
+    amax_kernel<<<(unsigned)blocks, 512, 0, st>>>(static_cast<const uint4 *>(x), n_vec,
+                                                 static_cast<const uint16_t *>(x) + n_vec * 8, n_tail,
+                                                 reinterpret_cast<unsigned int *>(amax));
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+static int do_cast(const void *x, size_t rows, size_t cols, const float *scale, int fmt, uint8_t *out, uint8_t *out_t,
+                   float *amax_out, cudaStream_t st)
+{
+    if (amax_out) FP8_CUDA_CHECK(cudaMemsetAsync(amax_out, 0, sizeof(float), st));
+    if (fmt == FP8_E4M3) {
+        if (amax_out) launch_cast<0, true>(x, rows, cols, scale, out, out_t, amax_out, st);
+        else launch_cast<0, false>(x, rows, cols, scale, out, out_t, amax_out, st);
+    } else {
+        if (amax_out) launch_cast<1, true>(x, rows, cols, scale, out, out_t, amax_out, st);
+        else launch_cast<1, false>(x, rows, cols, scale, out, out_t, amax_out, st);
+    }
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+}  // namespace fp8dpa
+
+using namespace fp8dpa;
+
+extern "C" int fp8_amax(const void *x_bf16, size_t n, float *amax, void *stream)
+{
+    if (!x_bf16 || !amax) {
+        set_error("fp8_amax: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if (n == 0) {
+        set_error("fp8_amax: n == 0");
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(x_bf16)) {
+        set_error("fp8_amax: x must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    return do_amax(x_bf16, n, amax, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int fp8_scale(const float *amax, int fmt, int margin, float *scale, float *scale_inv, void *stream)
+{
+    if (!amax || !scale || !scale_inv) {
+        set_error("fp8_scale: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if (fmt != FP8_E4M3 && fmt != FP8_E5M2) {
+        set_error("fp8_scale: fmt %d is not FP8_E4M3 / FP8_E5M2", fmt);
+        return FP8_ERR_ENUM;
+    }
+    if (margin < -64 || margin > 64) {
+        set_error("fp8_scale: margin %d outside [-64, 64]", margin);
+        return FP8_ERR_SHAPE;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    scale_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(amax, fmt == FP8_E4M3 ? 448.0f : 57344.0f, margin,
+                                                                scale, scale_inv);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+extern "C" int fp8_cast(const void *x_bf16, size_t rows, size_t cols, const float *scale, int fmt, uint8_t *out,
+                        uint8_t *out_t, float *amax_out, void *stream)
+{
+    int rc = validate_cast(x_bf16, rows, cols, scale, fmt, out, out_t);
+    if (rc != FP8_OK) return rc;
+    rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    return do_cast(x_bf16, rows, cols, scale, fmt, out, out_t, amax_out, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fmt, uint8_t *out, uint8_t *out_t,
+                            float *amax, float *scale, float *scale_inv, void *stream)
+{
+    if (!amax || !scale || !scale_inv) {
+        set_error("fp8_quantize: NULL amax/scale/scale_inv");
+        return FP8_ERR_NULL;
+    }
+    int rc = validate_cast(x_bf16, rows, cols, scale, fmt, out, out_t);
+    if (rc != FP8_OK) return rc;
+    rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = do_amax(x_bf16, rows * cols, amax, st);
+    if (rc != FP8_OK) return rc;
+    scale_kernel<<<1, 1, 0, st>>>(amax, fmt == FP8_E4M3 ? 448.0f : 57344.0f, 0, scale, scale_inv);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return do_cast(x_bf16, rows, cols, scale, fmt, out, out_t, nullptr, st);
+}

@@ -1,0 +1,104 @@
+"""GPU parity: FP8 linear forward / dgrad / wgrad against the double-accumulating oracle on identical codes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as o
+import paper_2505_20524_b200 as fp8
+from paper_2505_20524_b200 import synth
+from gpu_util import dev, host, scalar, gpu_quantize, bf16_host_to_f64, rel_err
+
+pytestmark = pytest.mark.gpu
+
+# max |gpu - ref| / sum_k |a_k||b_k| : FP32 accumulation (<= K * 2^-24) plus one BF16 rounding (2^-9 of |ref|)
+TOL_BF16 = 2e-2      # the stated bar; observed values are near 2^-9
+TOL_FP32 = 1e-4
+
+
+def run_three(x, w, dy, out_dtype, rows=None):
+    """Quantize on the GPU, run the three GEMMs, return GPU outputs and oracle inputs."""
+    T, K = x.shape
+    N = w.shape[0]
+    x8, x8t, _, _, sx = gpu_quantize(x, o.E4M3, True)
+    w8, w8t, _, _, sw = gpu_quantize(w, o.E4M3, True)
+    dy8, dy8t, _, _, sdy = gpu_quantize(dy, o.E5M2, True)
+    y = torch.empty((T, N), dtype=out_dtype, device="cuda")
+    dx = torch.empty((T, K), dtype=out_dtype, device="cuda")
+    dw = torch.empty((N, K), dtype=out_dtype, device="cuda")
+    fp8.fp8_linear_fwd(x8, w8, sx, sw, y)
+    fp8.fp8_linear_dgrad(dy8, w8t, sdy, sw, dx)
+    fp8.fp8_linear_wgrad(dy8t, x8t, sdy, sx, dw)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    # the oracle quantises the same BF16 bytes itself (bit-exactness of that step is tested elsewhere)
+    ox8, _, _, osx = o.quantize(x, o.E4M3)
+    ow8, _, _, osw = o.quantize(w, o.E4M3)
+    ody8, _, _, osdy = o.quantize(dy, o.E5M2)
+    assert np.array_equal(host(x8), ox8) and np.array_equal(host(dy8), ody8)
+    return (y, dx, dw), (ox8, ow8, ody8, osx, osw, osdy)
+
+
+def check(got_t, ref, mag, tol):
+    got = got_t.float().cpu().numpy().astype(np.float64)
+    err = rel_err(got, ref, mag)
+    assert err <= tol, err
+    return err
+
+
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("T,N,K", [(256, 768, 256), (256, 256, 256), (256, 1024, 256), (256, 256, 1024),
+                                   (128, 128, 128), (400, 272, 144), (16, 16, 16), (144, 528, 2064)])
+def test_three_gemms_match_oracle(T, N, K, out_dtype):
+    cfg_seed = T * 7 + N * 3 + K
+    cols = synth.choose_columns(K, 2, cfg_seed, 1)
+    x = synth.normal_bf16((T, K), cfg_seed, 0, 1.0, cols, 50.0)
+    w = synth.normal_bf16((N, K), cfg_seed, 1, synth.W_STD)
+    dy = synth.normal_bf16((T, N), cfg_seed, 2, synth.GRAD_STD)
+    (y, dx, dw), (x8, w8, dy8, sx, sw, sdy) = run_three(x, w, dy, out_dtype)
+    tol = TOL_BF16 if out_dtype == torch.bfloat16 else TOL_FP32
+    ref, mag = o.linear_fwd(x8, w8, sx, sw)
+    e1 = check(y, ref, mag, tol)
+    ref, mag = o.linear_dgrad(dy8, w8, sdy, sw)
+    e2 = check(dx, ref, mag, tol)
+    ref, mag = o.linear_wgrad(dy8, x8, sdy, sx)
+    e3 = check(dw, ref, mag, tol)
+    if out_dtype == torch.bfloat16:
+        assert max(e1, e2, e3) <= 2.0 ** -8          # what the arithmetic should give: one BF16 rounding
+
+
+def test_wgrad_accumulate_fp32():
+    T, N, K = 256, 128, 384
+    x = synth.normal_bf16((T, K), 1, 0, 1.0)
+    dy = synth.normal_bf16((T, N), 1, 2, synth.GRAD_STD)
+    x8, x8t, _, _, sx = gpu_quantize(x, o.E4M3, True)
+    dy8, dy8t, _, _, sdy = gpu_quantize(dy, o.E5M2, True)
+    prev = np.random.default_rng(0).normal(size=(N, K)).astype(np.float32) * 1e-3
+    dw = dev(prev.copy())
+    fp8.fp8_linear_wgrad(dy8t, x8t, sdy, sx, dw, accumulate=True)
+    ref, mag = o.linear_wgrad(host(dy8), host(x8), float(sdy.item()), float(sx.item()), prev=prev.astype(np.float64))
+    assert rel_err(host(dw).astype(np.float64), ref, mag + np.abs(prev)) <= TOL_FP32
+
+
+def test_exact_cases():
+    """All-ones operands and an identity weight give exactly representable results."""
+    K = 256
+    ones = torch.full((128, K), 0x38, dtype=torch.uint8, device="cuda")
+    y = torch.empty((128, 128), dtype=torch.float32, device="cuda")
+    fp8.fp8_linear_fwd(ones, ones[:128], scalar(0.5), scalar(3.0), y)
+    assert torch.all(y == K * 1.5)
+    eye = torch.where(torch.eye(K, device="cuda", dtype=torch.bool), 0x38, 0).to(torch.uint8)
+    x8 = dev(np.random.default_rng(1).integers(0, 0x7F, size=(128, K)).astype(np.uint8))
+    y = torch.empty((128, K), dtype=torch.float32, device="cuda")
+    fp8.fp8_linear_fwd(x8, eye, scalar(1.0), scalar(1.0), y)
+    assert np.array_equal(host(y).astype(np.float64), o.decode_array(host(x8), o.E4M3))
+
+
+def test_argument_validation():
+    a = torch.zeros((64, 64), dtype=torch.uint8, device="cuda")
+    y = torch.empty((64, 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_linear_fwd(a[:, :40].contiguous(), a[:, :40].contiguous(), scalar(1), scalar(1), y)
+    assert e.value.status == -3
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_linear_fwd(a, a, None, scalar(1), y)
+    assert e.value.status == -1

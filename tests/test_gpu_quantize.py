@@ -1,0 +1,110 @@
+"""GPU parity: amax -> scale -> cast must match the oracle bit for bit (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as o
+import paper_2505_20524_b200 as fp8
+from paper_2505_20524_b200 import synth
+from gpu_util import dev, host, scalar, gpu_quantize
+
+pytestmark = pytest.mark.gpu
+FMTS = [o.E4M3, o.E5M2]
+
+
+def bits(t):
+    return int(t.cpu().view(torch.int32).item()) & 0xFFFFFFFF
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_all_65536_bf16_patterns_scale_one(fmt):
+    x = np.arange(65536, dtype=np.uint16)
+    out = torch.empty(65536, dtype=torch.uint8, device="cuda")
+    fp8.fp8_cast(dev(x), scalar(1.0), fmt, out)
+    got = host(out)
+    exp = o.cast(x, 1.0, fmt)
+    vals = o.bf16_to_f32(x)
+    ok = ~np.isnan(vals)
+    assert np.array_equal(got[ok], exp[ok])
+    assert np.isnan(o.decode_array(got[~ok], fmt)).all()      # a NaN input gives a NaN code
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("n", [1, 7, 16, 1000, 4096 + 5, (1 << 20) + 3, 1 << 24])
+def test_flat_quantize_bit_exact(fmt, n):
+    x = synth.flat_tensor(n, seed=2 + n % 7)
+    q, _, a, s, si = gpu_quantize(x, fmt)
+    eq, ea, es, esi = o.quantize(x, fmt)
+    assert bits(a) == int(np.float32(ea).view(np.uint32))
+    assert bits(s) == int(np.float32(es).view(np.uint32))
+    assert bits(si) == int(np.float32(esi).view(np.uint32))
+    assert np.array_equal(host(q), eq)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("shape", [(16, 16), (256, 256), (48, 272), (400, 144), (1024, 768), (2048, 5632)])
+def test_cast_with_transposed_copy(fmt, shape):
+    cols = synth.choose_columns(shape[1], 2, 0, 1)
+    x = synth.normal_bf16(shape, 0, 3, 1.0, cols, 50.0)
+    q, qt, a, s, si = gpu_quantize(x, fmt, transpose=True)
+    eq, ea, es, esi = o.quantize(x, fmt)
+    assert bits(a) == int(np.float32(ea).view(np.uint32))
+    assert np.array_equal(host(q), eq)
+    assert np.array_equal(host(qt), eq.T)
+
+
+def test_amax_scale_cast_separately_and_fused_amax():
+    x = synth.normal_bf16((512, 384), 1, 4, 3.0)
+    xd = dev(x)
+    a, s, si, a2 = scalar(), scalar(), scalar(), scalar(123.0)
+    fp8.fp8_amax(xd, a)
+    assert float(a.item()) == float(o.amax(x))
+    for fmt in FMTS:
+        for margin in (0, 1, 3):
+            fp8.fp8_scale(a, fmt, margin, s, si)
+            es, esi = o.scale(o.amax(x), fmt, margin)
+            assert bits(s) == int(es.view(np.uint32)) and bits(si) == int(esi.view(np.uint32))
+        fp8.fp8_scale(a, fmt, 0, s, si)
+        out = torch.empty(x.shape, dtype=torch.uint8, device="cuda")
+        out_t = torch.empty(x.shape[::-1], dtype=torch.uint8, device="cuda")
+        fp8.fp8_cast(xd, s, fmt, out, None, a2)                       # delayed-scaling style: cast + amax
+        assert float(a2.item()) == float(o.amax(x))
+        es, _ = o.scale(o.amax(x), fmt)
+        assert np.array_equal(host(out), o.cast(x, es, fmt))
+        a2.fill_(7.0)
+        fp8.fp8_cast(xd, s, fmt, out, out_t, a2)
+        assert float(a2.item()) == float(o.amax(x))
+        assert np.array_equal(host(out_t), o.cast(x, es, fmt).T)
+
+
+def test_scale_guards():
+    s, si = scalar(), scalar()
+    for a, fmt in ((0.0, o.E4M3), (float("inf"), o.E5M2), (1e-40, o.E5M2), (200.0, o.E4M3)):
+        fp8.fp8_scale(scalar(a), fmt, 0, s, si)
+        es, esi = o.scale(np.float32(a), fmt)
+        assert bits(s) == int(es.view(np.uint32)) and bits(si) == int(esi.view(np.uint32))
+
+
+def test_saturating_cast_with_stale_scale():
+    x = synth.normal_bf16((64, 64), 5, 5, 100.0)
+    for fmt in FMTS:
+        out = torch.empty(x.shape, dtype=torch.uint8, device="cuda")
+        fp8.fp8_cast(dev(x), scalar(1000.0), fmt, out)
+        got = host(out)
+        assert np.array_equal(got, o.cast(x, 1000.0, fmt))
+        assert np.isfinite(o.decode_array(got, fmt)).all()
+
+
+def test_argument_validation_returns_errors_not_faults():
+    x = dev(synth.normal_bf16((32, 32), 0, 0, 1.0))
+    out = torch.empty((32, 32), dtype=torch.uint8, device="cuda")
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_cast(x, scalar(1.0), 5, out)
+    assert e.value.status == -4
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_cast(x, None, 0, out)
+    assert e.value.status == -1
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_cast(x.view(torch.int16).flatten()[1:].view(torch.bfloat16), scalar(1.0), 0, out)
+    assert e.value.status == -2
+    assert fp8.fp8_device_status() == 0
