@@ -1,0 +1,356 @@
+// FP8 attention forward (Appendix B, Eq. (P) with QK^T and PV on FP8 tensor cores).
+//
+// One CTA per (128-query tile, query head, batch); two CTAs share an SM so that one CTA's softmax overlaps
+// the other's MMAs.  Per 128-key block j (ascending):
+//   warp 0  TMA: K_j and V_j tiles ([128 keys x d bytes], swizzled) into a 2-stage ring; Q once
+//   warp 1  MMA: S = Q K_j^T (d/32 MMAs, 128x128, accumulator in TMEM columns 0..127), then
+//                O += P8 V_j (4 MMAs, 128 x d, TMEM columns 128..128+d) with V read in place as an
+//                MN-major operand (no transposed copy of V)
+//   warps 2-5  softmax, one row per thread: running max m, l += sum P~, P~ = 2^(c*S - m) scaled by c_P and
+//              rounded to E4M3, written to shared memory in the K-major 128-byte-swizzled operand layout;
+//              O in TMEM is rescaled by 2^(m_old - m_new) when a row maximum grows
+// Final: O = v_inv * acc / (c_P * l) as BF16, LSE = ln2 * (m + log2 l).
+#include <math.h>
+
+#include "common.cuh"
+
+namespace fp8dpa {
+
+constexpr int A_BM = 128;          // query rows per CTA
+constexpr int A_BN = 128;          // keys per block
+constexpr int A_KV_STAGES = 2;
+constexpr int A_THREADS = 192;
+constexpr int A_TMEM_COLS = 256;   // S: [0,128)  O: [128, 128+d)
+
+template <int D>
+struct AttnFwdSmem {
+    static constexpr int Q_BYTES = A_BM * D;
+    static constexpr int KV_BYTES = A_BN * D;             // one of K or V
+    static constexpr int STAGE_BYTES = 2 * KV_BYTES;      // K then V
+    static constexpr int P_BYTES = A_BM * A_BN;
+    static constexpr int Q_OFF = 0;
+    static constexpr int KV_OFF = Q_OFF + Q_BYTES;
+    static constexpr int P_OFF = KV_OFF + A_KV_STAGES * STAGE_BYTES;
+    static constexpr int BAR_OFF = P_OFF + P_BYTES;
+    // q_full, kv_full[2], kv_empty[2], s_full, p_full, pv_done
+    static constexpr int N_BARS = 1 + 2 * A_KV_STAGES + 3;
+    static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
+    static constexpr int DYN_BYTES = TOTAL + 1024;
+};
+
+struct AttnFwdParams {
+    uint16_t *O;         // [B,N,Hq,D] BF16
+    float *LSE;          // [B,Hq,N]
+    const float *q_inv, *k_inv, *v_inv;
+    float softmax_scale;
+    float log2_p_scale;
+    int causal;
+    int B, N, Hq, Hkv;
+    int *status;
+};
+
+__device__ __forceinline__ float fast_ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int D>
+__global__ void __launch_bounds__(A_THREADS, 2)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const AttnFwdParams p)
+{
+    using L = AttnFwdSmem<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::BAR_OFF;
+    const uint32_t q_full = bar0;
+    auto kv_full = [&](int s) { return bar0 + 8u * (1 + s); };
+    auto kv_empty = [&](int s) { return bar0 + 8u * (1 + A_KV_STAGES + s); };
+    const uint32_t s_full = bar0 + 8u * (1 + 2 * A_KV_STAGES);
+    const uint32_t p_full = s_full + 8u;
+    const uint32_t pv_done = s_full + 16u;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFF + L::N_BARS * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // heavy (late) query tiles first: with a causal mask tile q attends to q+1 key blocks
+    const int q_tile = (int)gridDim.x - 1 - (int)blockIdx.x;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int g = h / (p.Hq / p.Hkv);
+    const int q0 = q_tile * A_BM;
+    const int n_kv_all = (p.N + A_BN - 1) / A_BN;
+    const int n_kv = p.causal ? min(n_kv_all, q_tile + 1) : n_kv_all;
+
+    if (threadIdx.x == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < A_KV_STAGES; ++s) {
+            mbar_init(kv_full(s), 1);
+            mbar_init(kv_empty(s), 1);
+        }
+        mbar_init(s_full, 1);
+        mbar_init(p_full, 4);     // one arrival per softmax warp
+        mbar_init(pv_done, 1);
+        *abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), A_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 128u;
+    const WaitCtx ctx{p.status, abort_flag};
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            mbar_expect_tx(q_full, L::Q_BYTES);
+            tma_load_3d(sbase + L::Q_OFF, &tm_q, q_full, h * D, q0, b);
+            for (int j = 0; j < n_kv; ++j) {
+                const int st = j % A_KV_STAGES;
+                const uint32_t ph = (uint32_t)(j / A_KV_STAGES) & 1u;
+                if (!mbar_wait(kv_empty(st), ph ^ 1u, ctx)) break;
+                const uint32_t sk = sbase + L::KV_OFF + st * L::STAGE_BYTES, sv = sk + L::KV_BYTES;
+                mbar_expect_tx(kv_full(st), L::STAGE_BYTES);
+                tma_load_3d(sk, &tm_k, kv_full(st), g * D, j * A_BN, b);
+                tma_load_3d(sv, &tm_v, kv_full(st), g * D, j * A_BN, b);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            constexpr uint32_t idesc_s = umma_idesc_f8(0, 0, A_BM, A_BN, 0, 0);
+            constexpr uint32_t idesc_o = umma_idesc_f8(0, 0, A_BM, D, 0, 1);      // V is MN-major
+            const uint64_t dq = umma_desc(sbase + L::Q_OFF, D, 16);
+            const uint64_t dp = umma_desc(sbase + L::P_OFF, 128, 16);
+            bool ok = mbar_wait(q_full, 0, ctx);
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int st = j % A_KV_STAGES;
+                const uint32_t ph = (uint32_t)(j / A_KV_STAGES) & 1u;
+                if (!mbar_wait(kv_full(st), ph, ctx)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t sk = sbase + L::KV_OFF + st * L::STAGE_BYTES, sv = sk + L::KV_BYTES;
+                const uint64_t dk = umma_desc(sk, D, 16);
+                // S = Q K^T: reduction over d in steps of 32 bytes inside the swizzle span
+#pragma unroll
+                for (int k = 0; k < D / 32; ++k) umma_f8_ss(tmem_s, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
+                umma_commit(s_full);
+                if (!mbar_wait(p_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
+                tc_fence_after();
+                // O += P V: reduction over 128 keys in steps of 32; V advances 32 rows (32*D bytes) per step
+                const uint64_t dv = umma_desc(sv, D, 16);
+#pragma unroll
+                for (int k = 0; k < A_BN / 32; ++k)
+                    umma_f8_ss(tmem_o, dp + 2u * k, dv + (uint32_t)((32 * D) >> 4) * k, idesc_o, (j | k) != 0);
+                umma_commit(kv_empty(st));
+                umma_commit(pv_done);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax / correction / epilogue
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;                  // row inside the tile = TMEM lane
+        const int row = q0 + r;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const float c = p.softmax_scale * __ldg(p.q_inv) * __ldg(p.k_inv) * 1.4426950408889634f;
+        float m = -INFINITY, l = 0.0f;                   // running max of c*S; l = sum of c_P * P~
+        uint8_t *prow = smem + L::P_OFF + r * 128;
+        bool ok = true;
+        for (int j = 0; j < n_kv; ++j) {
+            const int k0 = j * A_BN;
+            // keys beyond the row (causal, only the diagonal block) or beyond N get -inf
+            const int limit = min(p.causal ? row : 0x7FFFFFFF, p.N - 1) - k0;   // last valid local column
+            const bool need_mask = (k0 + A_BN - 1 > q0 && p.causal) || (k0 + A_BN > p.N);
+            if (!mbar_wait(s_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
+            tc_fence_after();
+            // pass 1: row maximum
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int cc = 0; cc < A_BN; cc += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)cc, v);
+                tmem_ld_wait();
+                if (need_mask) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (cc + i <= limit) mx = fmaxf(mx, __uint_as_float(v[i]));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+                }
+            }
+            const float m_new = fmaxf(m, mx * c);
+            const float alpha = fast_ex2(m - m_new);     // 0 on the first block (m = -inf)
+            // the previous PV must have finished before O is rescaled or P is overwritten
+            if (j > 0) {
+                if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, ctx)) { ok = false; break; }
+                tc_fence_after();
+                if (__any_sync(0xffffffffu, m_new > m)) {
+#pragma unroll 1
+                    for (int cc = 0; cc < D; cc += 32) {
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(tmem_o + lane_addr + (uint32_t)cc, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+                        tmem_st_32x32b_x32(tmem_o + lane_addr + (uint32_t)cc, v);
+                    }
+                    tmem_st_wait();
+                }
+            }
+            // pass 2: P~ * c_P = 2^(c*S - m_new + log2 c_P), row sum, E4M3 codes into the operand layout
+            const float shift = m_new - p.log2_p_scale;
+            float lsum = 0.0f;
+#pragma unroll 1
+            for (int cc = 0; cc < A_BN; cc += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)cc, v);
+                tmem_ld_wait();
+                float e[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    e[i] = fast_ex2(fmaf(__uint_as_float(v[i]), c, -shift));
+                    if (need_mask && cc + i > limit) e[i] = 0.0f;
+                    lsum += e[i];
+                }
+                uint32_t w[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    w[i] = (uint32_t)cvt_f32x2_to_fp8x2<0>(e[4 * i], e[4 * i + 1]) |
+                           ((uint32_t)cvt_f32x2_to_fp8x2<0>(e[4 * i + 2], e[4 * i + 3]) << 16);
+                // two 16-byte chunks (keys cc..cc+15, cc+16..cc+31) at their swizzled positions
+                const int ch = cc >> 4;
+                *reinterpret_cast<uint4 *>(prow + (((ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(prow + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
+            l = l * alpha + lsum;
+            m = m_new;
+            tc_fence_before();
+            fence_proxy_async_smem();     // generic-proxy writes of P become visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);
+        }
+        if (ok && mbar_wait(pv_done, (uint32_t)(n_kv - 1) & 1u, ctx)) {
+            tc_fence_after();
+            const float inv = __ldg(p.v_inv) / l;        // l already carries c_P
+            uint16_t *orow = p.O + (((size_t)b * p.N + row) * p.Hq + h) * D;
+#pragma unroll 1
+            for (int cc = 0; cc < D; cc += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32b_x32(tmem_o + lane_addr + (uint32_t)cc, v);
+                tmem_ld_wait();
+                if (row < p.N) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 o;
+                        o.x = pack_bf16x2(__uint_as_float(v[i]) * inv, __uint_as_float(v[i + 1]) * inv);
+                        o.y = pack_bf16x2(__uint_as_float(v[i + 2]) * inv, __uint_as_float(v[i + 3]) * inv);
+                        o.z = pack_bf16x2(__uint_as_float(v[i + 4]) * inv, __uint_as_float(v[i + 5]) * inv);
+                        o.w = pack_bf16x2(__uint_as_float(v[i + 6]) * inv, __uint_as_float(v[i + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + cc + i) = o;
+                    }
+                }
+            }
+            if (row < p.N)
+                p.LSE[((size_t)b * p.Hq + h) * p.N + row] = (m + log2f(l) - p.log2_p_scale) * 0.69314718055994531f;
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, A_TMEM_COLS);
+    }
+}
+
+int validate_attn(const char *who, const void *q, const void *k, const void *v, const fp8_attn_scales *sc, int B, int N,
+                  int Hq, int Hkv, int d)
+{
+    if (!q || !k || !v || !sc || !sc->q_inv || !sc->k_inv || !sc->v_inv) {
+        set_error("%s: NULL pointer", who);
+        return FP8_ERR_NULL;
+    }
+    if (B <= 0 || N <= 0 || Hq <= 0 || Hkv <= 0 || (Hq % Hkv) || (d != 64 && d != 128) || (N % 16)) {
+        set_error("%s: unsupported shape B=%d N=%d Hq=%d Hkv=%d d=%d (d in {64,128}, N %% 16 == 0, Hq %% Hkv == 0)", who,
+                  B, N, Hq, Hkv, d);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v)) {
+        set_error("%s: tensor pointers must be 16-byte aligned", who);
+        return FP8_ERR_ALIGN;
+    }
+    if (!(sc->softmax_scale > 0.0f) || !(sc->p_scale > 0.0f)) {
+        set_error("%s: softmax_scale and p_scale must be positive", who);
+        return FP8_ERR_SHAPE;
+    }
+    return FP8_OK;
+}
+
+template <int D>
+static int launch_attn_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const AttnFwdParams &p,
+                           cudaStream_t st)
+{
+    CUtensorMap tq, tk, tv;
+    int rc = make_tmap_3d_u8(&tq, Q8, (uint64_t)p.Hq * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BM);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tk, K8, (uint64_t)p.Hkv * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BN);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tv, V8, (uint64_t)p.Hkv * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BN);
+    if (rc != FP8_OK) return rc;
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        AttnFwdSmem<D>::DYN_BYTES));
+    dim3 grid((unsigned)((p.N + A_BM - 1) / A_BM), (unsigned)p.Hq, (unsigned)p.B);
+    attn_fwd_kernel<D><<<grid, A_THREADS, AttnFwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+}  // namespace fp8dpa
+
+using namespace fp8dpa;
+
+extern "C" int fp8_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const fp8_attn_scales *sc,
+                                 int causal, int B, int N, int Hq, int Hkv, int d, void *O_bf16, float *LSE, void *ws,
+                                 size_t ws_bytes, void *stream)
+{
+    (void)ws; (void)ws_bytes;
+    int rc = validate_attn("fp8_attention_fwd", Q8, K8, V8, sc, B, N, Hq, Hkv, d);
+    if (rc != FP8_OK) return rc;
+    if (!O_bf16 || !LSE) {
+        set_error("fp8_attention_fwd: NULL output pointer");
+        return FP8_ERR_NULL;
+    }
+    if (!aligned16(O_bf16)) {
+        set_error("fp8_attention_fwd: O must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    AttnFwdParams p;
+    p.O = static_cast<uint16_t *>(O_bf16);
+    p.LSE = LSE;
+    p.q_inv = sc->q_inv; p.k_inv = sc->k_inv; p.v_inv = sc->v_inv;
+    p.softmax_scale = sc->softmax_scale;
+    p.log2_p_scale = log2f(sc->p_scale);
+    p.causal = causal ? 1 : 0;
+    p.B = B; p.N = N; p.Hq = Hq; p.Hkv = Hkv;
+    p.status = device_status_ptr();
+    if (!p.status) return FP8_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return d == 128 ? launch_attn_fwd<128>(Q8, K8, V8, p, st) : launch_attn_fwd<64>(Q8, K8, V8, p, st);
+}

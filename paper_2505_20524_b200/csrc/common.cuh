@@ -20,6 +20,9 @@ int sm_count();
 int make_tmap_2d_u8(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint64_t pitch,
                     uint32_t box_rows, uint32_t box_cols);
 
+int make_tmap_3d_u8(CUtensorMap *map, const void *base, uint64_t d0_cols, uint64_t d1_rows, uint64_t d2_batch,
+                    uint32_t box_cols, uint32_t box_rows);
+
 #define FP8_CUDA_CHECK(expr)                                                                        \
     do {                                                                                            \
         cudaError_t e_ = (expr);                                                                    \
@@ -169,12 +172,27 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t saddr)
     d |= (uint64_t)2 << 61;                       // SWIZZLE_128B
     return d;
 }
-// Instruction descriptor of tcgen05.mma.kind::f8f6f4: FP32 accumulate, both operands K-major.
-// fmt: 0 = E4M3, 1 = E5M2.
-__host__ __device__ constexpr uint32_t umma_idesc_f8(int fmt_a, int fmt_b, int M, int N)
+// General form.  swizzle_bytes: 128 or 64 (row length of the tile in bytes = swizzle span).
+//  K-major  (reduction index contiguous):   8 rows x span bytes per atom, SBO = 8*span between 8-row groups.
+//  MN-major (output index contiguous, `span` bytes of it per reduction row): 8 reduction rows x span bytes
+//            per atom, SBO = 8*span between groups of 8 reduction rows, LBO = distance to the next span-wide
+//            block of the output index (unused when the operand is one span wide).
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, int swizzle_bytes, uint32_t lbo_bytes)
 {
-    return (1u << 4) | ((uint32_t)fmt_a << 7) | ((uint32_t)fmt_b << 10) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((8u * swizzle_bytes) >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)(swizzle_bytes == 128 ? 2 : 4) << 61;   // SWIZZLE_128B = 2, SWIZZLE_64B = 4
+    return d;
+}
+// Instruction descriptor of tcgen05.mma.kind::f8f6f4 with FP32 accumulate.  fmt: 0 = E4M3, 1 = E5M2;
+// *_mn = 1 when that operand is MN-major (output index contiguous) instead of K-major.
+__host__ __device__ constexpr uint32_t umma_idesc_f8(int fmt_a, int fmt_b, int M, int N, int a_mn = 0, int b_mn = 0)
+{
+    return (1u << 4) | ((uint32_t)fmt_a << 7) | ((uint32_t)fmt_b << 10) | ((uint32_t)a_mn << 15) |
+           ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 // D[tmem] (+)= A[smem] * B[smem]; one thread issues.

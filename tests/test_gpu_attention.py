@@ -1,0 +1,70 @@
+"""GPU parity: FP8 attention forward / backward against the oracle on identical FP8 codes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as o
+import paper_2505_20524_b200 as fp8
+from paper_2505_20524_b200 import synth
+from gpu_util import dev, host, scalar, gpu_quantize, rel_err
+
+pytestmark = pytest.mark.gpu
+
+TOL_FWD = 2e-2     # max |gpu - ref| / sum_j P8_ij |V_jd| (normalised like O)
+TOL_BWD = 3e-2
+KV_BLOCK = 128     # the kernel takes keys in blocks of 128 with an exact running maximum
+
+
+def quantized_qkv(cfg, N, B, seed_shift=0):
+    q, k, v, do = synth.attention_inputs(cfg, seq=N, batch=B)
+    out = {}
+    for name, t, fmt in (("q", q, o.E4M3), ("k", k, o.E4M3), ("v", v, o.E4M3), ("do", do, o.E5M2)):
+        c, a, s, si = o.quantize(t, fmt)
+        out[name] = (c, float(si))
+    return out
+
+
+def run_fwd(qd, B, N, Hq, Hkv, d, causal, s):
+    q8, k8, v8 = dev(qd["q"][0]), dev(qd["k"][0]), dev(qd["v"][0])
+    O = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda")
+    LSE = torch.empty((B, Hq, N), dtype=torch.float32, device="cuda")
+    fp8.fp8_attention_fwd(q8, k8, v8, scalar(qd["q"][1]), scalar(qd["k"][1]), scalar(qd["v"][1]), s, causal,
+                          O, LSE, None)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    return O, LSE
+
+
+@pytest.mark.parametrize("name,B,N,causal", [("c1", 1, 256, True), ("c1", 2, 128, True), ("c1", 1, 400, True),
+                                             ("c1", 1, 256, False), ("c1", 1, 16, True), ("c1", 1, 208, False),
+                                             ("c3", 1, 384, True), ("c4", 1, 272, True), ("c4", 1, 256, False)])
+def test_forward_matches_oracle(name, B, N, causal):
+    cfg = synth.CONFIGS[name]
+    Hq, Hkv, d = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    if name != "c1":
+        Hq, Hkv = Hq // 4, Hkv // 4          # a few heads are enough at this size
+        cfg = synth.BlockConfig(**{**cfg.__dict__, "n_q_heads": Hq, "n_kv_heads": Hkv})
+    qd = quantized_qkv(cfg, N, B)
+    s = d ** -0.5
+    O, LSE = run_fwd(qd, B, N, Hq, Hkv, d, causal, s)
+    p = o.attn_params(B, N, Hq, Hkv, d, causal=causal, quant=True, kv_block=KV_BLOCK, max_mode=0, s=s,
+                      q_inv=qd["q"][1], k_inv=qd["k"][1], v_inv=qd["v"][1])
+    ref, lse, mag = o.attention_fwd(qd["q"][0], qd["k"][0], qd["v"][0], p)
+    got = O.float().cpu().numpy().astype(np.float64).transpose(0, 2, 1, 3).reshape(B * Hq, N, d)
+    err = rel_err(got, ref, mag)
+    assert err <= TOL_FWD, err
+    glse = LSE.cpu().numpy().astype(np.float64).reshape(B * Hq, N)
+    assert np.max(np.abs(glse - lse)) <= 1e-3 * max(1.0, np.abs(lse).max())
+
+
+def test_softmax_scale_parameter():
+    """s = 0.125 at d = 128 (the frozen-gain QK-norm setting of Appendix A) instead of 1/sqrt(d)."""
+    cfg = synth.BlockConfig(**{**synth.CONFIGS["c3"].__dict__, "n_q_heads": 2, "n_kv_heads": 2})
+    B, N, d = 1, 256, 128
+    qd = quantized_qkv(cfg, N, B)
+    O, LSE = run_fwd(qd, B, N, 2, 2, d, True, 0.125)
+    p = o.attn_params(B, N, 2, 2, d, causal=True, quant=True, kv_block=KV_BLOCK, s=0.125,
+                      q_inv=qd["q"][1], k_inv=qd["k"][1], v_inv=qd["v"][1])
+    ref, lse, mag = o.attention_fwd(qd["q"][0], qd["k"][0], qd["v"][0], p)
+    got = O.float().cpu().numpy().astype(np.float64).transpose(0, 2, 1, 3).reshape(B * 2, N, d)
+    assert rel_err(got, ref, mag) <= TOL_FWD
