@@ -68,3 +68,59 @@ def test_softmax_scale_parameter():
     ref, lse, mag = o.attention_fwd(qd["q"][0], qd["k"][0], qd["v"][0], p)
     got = O.float().cpu().numpy().astype(np.float64).transpose(0, 2, 1, 3).reshape(B * 2, N, d)
     assert rel_err(got, ref, mag) <= TOL_FWD
+
+
+def oracle_fwd_for_bwd(qd, p, B, N, Hq, d):
+    """Oracle forward; returns O as BF16 bits [B,N,Hq,d] and LSE float32 [B,Hq,N] (what a framework saves)."""
+    ref, lse, _ = o.attention_fwd(qd["q"][0], qd["k"][0], qd["v"][0], p)
+    O = ref.reshape(B, Hq, N, d).transpose(0, 2, 1, 3)
+    O_bits = synth.f32_to_bf16(O.astype(np.float32))
+    return O_bits, lse.reshape(B, Hq, N).astype(np.float32)
+
+
+def run_bwd(qd, O_bits, lse32, B, N, Hq, Hkv, d, causal, s, ds_scale):
+    q8, k8, v8, do8 = dev(qd["q"][0]), dev(qd["k"][0]), dev(qd["v"][0]), dev(qd["do"][0])
+    dQ = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda")
+    dK = torch.empty((B, N, Hkv, d), dtype=torch.bfloat16, device="cuda")
+    dV = torch.empty((B, N, Hkv, d), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(fp8.fp8_attention_workspace_bytes(1, B, N, Hq, Hkv, d), dtype=torch.uint8, device="cuda")
+    amax = scalar(-1.0)
+    fp8.fp8_attention_bwd(q8, k8, v8, do8, dev(O_bits), dev(lse32), scalar(qd["q"][1]), scalar(qd["k"][1]),
+                          scalar(qd["v"][1]), scalar(qd["do"][1]), s, scalar(ds_scale), causal, dQ, dK, dV, ws,
+                          ds_amax=amax)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    return dQ, dK, dV, float(amax.item())
+
+
+@pytest.mark.parametrize("name,B,N,causal", [("c1", 1, 256, True), ("c1", 2, 128, True), ("c1", 1, 400, True),
+                                             ("c1", 1, 256, False), ("c1", 1, 16, True),
+                                             ("c3", 1, 384, True), ("c4", 1, 272, True), ("c4", 1, 256, False)])
+def test_backward_matches_oracle(name, B, N, causal):
+    cfg = synth.CONFIGS[name]
+    Hq, Hkv, d = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    if name != "c1":
+        Hq, Hkv = Hq // 4, Hkv // 4
+        cfg = synth.BlockConfig(**{**cfg.__dict__, "n_q_heads": Hq, "n_kv_heads": Hkv})
+    G = Hq // Hkv
+    qd = quantized_qkv(cfg, N, B)
+    s = d ** -0.5
+    kw = dict(causal=causal, quant=True, kv_block=KV_BLOCK, max_mode=0, s=s, q_inv=qd["q"][1], k_inv=qd["k"][1],
+              v_inv=qd["v"][1], do_inv=qd["do"][1])
+    p = o.attn_params(B, N, Hq, Hkv, d, ds_scale=1.0, **kw)
+    O_bits, lse32 = oracle_fwd_for_bwd(qd, p, B, N, Hq, d)
+    Of = synth.bf16_to_f32(O_bits).astype(np.float64)
+    args = (qd["q"][0], qd["k"][0], qd["v"][0], qd["do"][0], Of, lse32.astype(np.float64))
+    # delayed-scaling style calibration of the dS scale: one oracle pass with scale 1 gives amax(dS)
+    cal = o.attention_bwd(*args, p)
+    ds_scale, _ = o.scale(np.float32(cal["amax_dS"]), o.E5M2)
+    p = o.attn_params(B, N, Hq, Hkv, d, ds_scale=float(ds_scale), **kw)
+    ref = o.attention_bwd(*args, p)
+    dQ, dK, dV, amax = run_bwd(qd, O_bits, lse32, B, N, Hq, Hkv, d, causal, s, float(ds_scale))
+    assert abs(amax - ref["amax_dS"]) <= 1e-3 * ref["amax_dS"]
+    gq = dQ.float().cpu().numpy().astype(np.float64).reshape(B, N, Hkv, G, d).transpose(0, 2, 3, 1, 4)
+    gq = gq.reshape(B * Hkv, G, N, d)
+    gk = dK.float().cpu().numpy().astype(np.float64).transpose(0, 2, 1, 3).reshape(B * Hkv, N, d)
+    gv = dV.float().cpu().numpy().astype(np.float64).transpose(0, 2, 1, 3).reshape(B * Hkv, N, d)
+    errs = {n_: rel_err(g_, ref[n_], ref["mag_" + n_]) for n_, g_ in (("dQ", gq), ("dK", gk), ("dV", gv))}
+    assert max(errs.values()) <= TOL_BWD, errs
