@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the FP8 transformer-block hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config c4|c3|c1]
+
+One step = one pass of the whole hot path over one block of synthetic input: JIT quantize of every
+activation / weight / gradient, the 12 FP8 GEMMs (forward, dgrad, wgrad of 4 projections), quantize of
+Q/K/V/dO and FP8 attention forward + backward.  `value` = (GEMM + causal-attention FLOPs) / time in TFLOP/s
+with inputs resident in HBM; `e2e` = the same with host->device copies of the BF16 inputs and device->host
+copies of every output inside the timed region.  With N > 1 (torchrun) every rank runs an independent replica
+(the path has no exchange step); the time is the max over ranks.
+
+`--impl reference` times the CPU oracle (as it stands) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "FP8 GEMM + FP8 attention TFLOP/s (fwd+bwd) on 1 B200, % of dense FP8 peak"
+UNIT = "TFLOP/s"
+FP8_NOMINAL_TFLOPS = 4500.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"], "hbm": d["hbm_gbs"],
+                "source": "measured"}
+    return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm": 6650.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------- clocks
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+            nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonHwPowerBrakeSlowdown: "hw_power_brake",
+        }
+        while not self._halt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+# ---------------------------------------------------------------------------------------------- oracle sample
+def oracle_sample(cfg, reps: int = 1):
+    """Runs the CPU oracle on a bounded sample of the workload; returns (flops, seconds, description)."""
+    import numpy as np
+    import oracle as o
+    from paper_2505_20524_b200 import synth
+
+    small = synth.BlockConfig(**{**cfg.__dict__})
+    flops, secs = 0.0, 0.0
+    desc = []
+    if cfg.has_linears:
+        T, N, K = cfg.linear_shapes()["qkv"]
+        Ts = 512                                      # token slice of the QKV projection
+        cols = synth.choose_columns(K, cfg.n_outlier_cols(K), cfg.seed, 100)
+        x = synth.normal_bf16((Ts, K), cfg.seed, 0, 1.0, cols, cfg.act_outlier_factor)
+        w = synth.normal_bf16((N, K), cfg.seed, 1, synth.W_STD)
+        dy = synth.normal_bf16((Ts, N), cfg.seed, 8, synth.GRAD_STD)
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            x8, _, _, sx = o.quantize(x, o.E4M3)
+            w8, _, _, sw = o.quantize(w, o.E4M3)
+            dy8, _, _, sdy = o.quantize(dy, o.E5M2)
+            rows = np.arange(128)
+            o.linear_fwd(x8, w8, sx, sw, rows=rows)
+            o.linear_dgrad(dy8, w8, sdy, sw, rows=rows)
+            o.linear_wgrad(dy8, x8, sdy, sx, rows=rows)
+        secs += time.perf_counter() - t0
+        flops += reps * 2.0 * 128 * (N * K + N * K + Ts * K)
+        desc.append(f"quantize + 128 output rows each of QKV fwd/dgrad/wgrad on a {Ts}-token slice")
+    Na = min(1024, cfg.seq)
+    q, k, v, do = synth.attention_inputs(small, seq=Na, batch=1)
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        q8, _, _, qi = o.quantize(q, o.E4M3)
+        k8, _, _, ki = o.quantize(k, o.E4M3)
+        v8, _, _, vi = o.quantize(v, o.E4M3)
+        do8, _, _, doi = o.quantize(do, o.E5M2)
+        G = cfg.n_q_heads // cfg.n_kv_heads
+        p = o.attn_params(1, Na, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, kv_block=128, q_inv=qi, k_inv=ki,
+                          v_inv=vi, do_inv=doi, ds_scale=4096.0)
+        heads = [(0, h) for h in range(G)]
+        O, lse, _ = o.attention_fwd(q8, k8, v8, p, heads=heads)
+        Of = np.zeros((1, Na, cfg.n_q_heads, cfg.head_dim))
+        Lf = np.zeros((1, cfg.n_q_heads, Na))
+        Of[0, :, :G] = O.transpose(1, 0, 2)
+        Lf[0, :G] = lse
+        o.attention_bwd(q8, k8, v8, do8, Of, Lf, p, kv_heads=[(0, 0)])
+    secs += time.perf_counter() - t0
+    flops += reps * 3.5 * 2.0 * G * Na * Na * cfg.head_dim
+    desc.append(f"attention fwd+bwd of one KV group ({G} heads) at seq {Na}")
+    return flops, secs, "; ".join(desc), o.num_threads()
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    for _ in range(args.warmup):
+        oracle_sample(cfg)
+    flops, secs = 0.0, 0.0
+    for _ in range(args.steps):
+        f, s, desc, cores = oracle_sample(cfg)
+        flops += f
+        secs += s
+    value = flops / secs / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name + " (bounded sample per step: " + desc + ")"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------- our arm
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2505_20524_b200 as fp8
+    from paper_2505_20524_b200.hotpath import BlockHotPath
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    fp8.binding.load()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    hp = BlockHotPath(cfg, dev)
+    host = hp.generate_host_inputs()
+    hp.allocate()
+    hp.calibrate_ds_scale()
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        hp.step()
+    torch.cuda.synchronize()
+
+    # ---- device-resident timing (inputs already in HBM)
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        hp.step(time_gemms=True)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop()
+    ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    ms_total = float(ms.item())
+    status = fp8.fp8_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status}: a bounded wait expired inside a kernel")
+
+    flops_step = hp.gemm_flops() + hp.attention_flops()
+    value = world * flops_step * args.steps / (ms_total / 1e3) / 1e12
+
+    # ---- dominant kernel: the FP8 GEMM; duration from the events recorded around each launch
+    gemm_ms = sum(a.elapsed_time(b) for evs in hp.gemm_events for a, b in evs)
+    n_gemm = sum(len(evs) for evs in hp.gemm_events)
+    gemm_tflops = hp.gemm_flops() * args.steps / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else None
+    peaks = measured_peaks()
+    fp8_peak = 2.0 * peaks["bf16_sustained"]          # FP8 = 2x the BF16 rate; kernel timed inside a long step
+    roofline = None
+    if gemm_tflops is not None:
+        roofline = {
+            "bound": "tensor", "kernel": "gemm_fp8_kernel", "achieved": gemm_tflops, "peak": fp8_peak,
+            "unit": "TFLOP/s", "frac": gemm_tflops / fp8_peak,
+            "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name),
+            "peak_source": f"2 x bf16_tflops_sustained ({peaks['source']})",
+            "launches": n_gemm, "avg_launch_ms": gemm_ms / max(n_gemm, 1),
+            "flops_per_launch": hp.gemm_flops() / 12.0,
+            "frac_of_nominal_4500": gemm_tflops / FP8_NOMINAL_TFLOPS,
+        }
+
+    # ---- end to end: pinned host inputs -> device, step, every output -> pinned host
+    ins, outs = hp.input_tensors(), hp.output_tensors()
+    h_in = [torch.from_numpy(host[n].view("int16")).view(torch.bfloat16).pin_memory() for n, _ in ins]
+    h_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for _, t in outs]
+    h2d = sum(t.numel() * t.element_size() for t in h_in)
+    d2h = sum(t.numel() * t.element_size() for t in h_out)
+
+    def e2e_step():
+        for (_, d), h in zip(ins, h_in):
+            d.copy_(h, non_blocking=True)
+        hp.step()
+        for (_, d), h in zip(outs, h_out):
+            h.copy_(d, non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_step()
+    torch.cuda.synchronize()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    ms2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(ms2, op=dist.ReduceOp.MAX)
+    e2e_value = world * flops_step * e2e_steps / (float(ms2.item()) / 1e3) / 1e12
+
+    cpu_baseline = None
+    if rank == 0 and world == 1:
+        f, s, desc, cores = oracle_sample(cfg, reps=3)
+        cpu_baseline = {"value": f / s / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                        "seconds": s}
+
+    if rank == 0:
+        c = cfg
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp8 (e4m3/e5m2 operands, f32 accumulate)", "data": "synthetic",
+            "config": {"workload": f"{c.name}: Llama-style block, tokens {c.tokens} ({c.batch}x{c.seq}), hidden "
+                                   f"{c.hidden}, heads {c.n_q_heads}/{c.n_kv_heads} x {c.head_dim}, ffn {c.ffn}"
+                                   f"{' gated' if c.gated else ''}; quantize + 12 GEMMs + causal attention fwd+bwd",
+                       "l2": "per-step working set (GBs) exceeds the 126 MB L2; no flush needed",
+                       "replicas": world},
+            "pct_of_nominal_fp8_peak": 100.0 * value / world / FP8_NOMINAL_TFLOPS,
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": hp.launches_per_step() * args.steps,
+            "roofline": roofline,
+            "cpu_baseline": cpu_baseline,
+            "breakdown": {"gemm_ms_per_step": gemm_ms / args.steps, "gemm_tflops": gemm_tflops,
+                          "gemm_tflop_per_step": hp.gemm_flops() / 1e12,
+                          "attention_tflop_per_step": hp.attention_flops() / 1e12,
+                          "quantize_gb_per_step": hp.quantize_bytes() / 1e9},
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes (read + write) per GEMM launch from the ncu capture summarised under profiles/ (null until one
+# exists for the workload).
+GEMM_DRAM_BYTES_PER_LAUNCH = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="c4", choices=["c1", "c3", "c4"])
+    args = ap.parse_args()
+    from paper_2505_20524_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,229 @@
+"""One pass of the whole FP8 hot path over a transformer block's tensors, as a sequence of C-ABI calls.
+
+A step is: just-in-time quantize (amax -> scale -> cast, with transposed copies) of every activation, weight
+and upstream gradient; forward, dgrad and wgrad GEMMs of the QKV, output, up(-gate) and down projections;
+quantize of Q, K, V, dO; FP8 attention forward and backward.  This module only owns device buffers (torch)
+and the order of calls; every computation runs in the CUDA library.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+from . import binding as fp8
+from . import synth
+
+LAYERS = ("qkv", "o", "up", "down")
+
+
+def _bits_to_dev(a: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def _f32(device, v=0.0):
+    return torch.full((1,), float(v), dtype=torch.float32, device=device)
+
+
+@dataclass
+class QTensor:
+    """A BF16 tensor with its FP8 copy (and transposed copy) and the three device scalars of its scaling."""
+    x: torch.Tensor
+    fmt: int
+    transpose: bool
+    q: torch.Tensor = None
+    qt: torch.Tensor = None
+    amax: torch.Tensor = None
+    scale: torch.Tensor = None
+    scale_inv: torch.Tensor = None
+
+    def __post_init__(self):
+        dev = self.x.device
+        self.q = torch.empty(self.x.shape, dtype=torch.uint8, device=dev)
+        if self.transpose:
+            rows, cols = self.x.numel() // self.x.shape[-1], self.x.shape[-1]
+            self.qt = torch.empty((cols, rows), dtype=torch.uint8, device=dev)
+        self.amax, self.scale, self.scale_inv = _f32(dev), _f32(dev), _f32(dev)
+
+    def quantize(self):
+        fp8.fp8_quantize(self.x, self.fmt, self.q, self.qt, self.amax, self.scale, self.scale_inv)
+
+    @property
+    def nbytes_in(self):
+        return self.x.numel() * 2
+
+
+@dataclass
+class Linear:
+    name: str
+    T: int
+    N: int
+    K: int
+    x: QTensor
+    w: QTensor
+    dy: QTensor
+    y: torch.Tensor = None
+    dx: torch.Tensor = None
+    dw: torch.Tensor = None
+
+    @property
+    def flops(self):            # forward + dgrad + wgrad
+        return 3 * 2.0 * self.T * self.N * self.K
+
+
+class BlockHotPath:
+    """Device buffers of one block configuration and the step that runs the hot path over them."""
+
+    KERNELS_PER_QUANTIZE = 3    # amax, scale, cast
+    KERNELS_PER_ATTN_BWD = 3    # prep, main, finish
+
+    def __init__(self, cfg: synth.BlockConfig, device="cuda", with_linears=None, with_attention=True,
+                 seq=None, batch=None):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.with_linears = cfg.has_linears if with_linears is None else with_linears
+        self.with_attention = with_attention
+        self.B = cfg.batch if batch is None else batch
+        self.N = cfg.seq if seq is None else seq
+        self.linears: list[Linear] = []
+        self.attn = None
+        self.host_inputs: dict[str, np.ndarray] = {}
+        self.gemm_events = []
+
+    # ------------------------------------------------------------------ inputs
+    def generate_host_inputs(self):
+        """Seeded BF16 inputs on the host (numpy uint16 bits), keyed by tensor name."""
+        h = {}
+        if self.with_linears:
+            for layer in LAYERS:
+                x, w, dy = synth.linear_inputs(self.cfg, layer)
+                h["x_" + layer], h["w_" + layer], h["dy_" + layer] = x, w, dy
+        if self.with_attention:
+            h["q"], h["k"], h["v"], h["do"] = synth.attention_inputs(self.cfg, seq=self.N, batch=self.B)
+        self.host_inputs = h
+        return h
+
+    def allocate(self, host_inputs=None):
+        h = self.host_inputs if host_inputs is None else host_inputs
+        dev = self.device
+        if self.with_linears:
+            for layer in LAYERS:
+                T, N, K = self.cfg.linear_shapes()[layer]
+                lin = Linear(layer, T, N, K,
+                             QTensor(_bits_to_dev(h["x_" + layer], dev), fp8.E4M3, True),
+                             QTensor(_bits_to_dev(h["w_" + layer], dev), fp8.E4M3, True),
+                             QTensor(_bits_to_dev(h["dy_" + layer], dev), fp8.E5M2, True))
+                lin.y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+                lin.dx = torch.empty((T, K), dtype=torch.bfloat16, device=dev)
+                lin.dw = torch.empty((N, K), dtype=torch.bfloat16, device=dev)
+                self.linears.append(lin)
+        if self.with_attention:
+            c = self.cfg
+            a = {n: QTensor(_bits_to_dev(h[n], dev), fp8.E5M2 if n == "do" else fp8.E4M3, False)
+                 for n in ("q", "k", "v", "do")}
+            B, N, Hq, Hkv, d = self.B, self.N, c.n_q_heads, c.n_kv_heads, c.head_dim
+            a["o"] = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device=dev)
+            a["lse"] = torch.empty((B, Hq, N), dtype=torch.float32, device=dev)
+            a["dq"] = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device=dev)
+            a["dk"] = torch.empty((B, N, Hkv, d), dtype=torch.bfloat16, device=dev)
+            a["dv"] = torch.empty((B, N, Hkv, d), dtype=torch.bfloat16, device=dev)
+            a["ws"] = torch.empty(fp8.fp8_attention_workspace_bytes(1, B, N, Hq, Hkv, d), dtype=torch.uint8,
+                                  device=dev)
+            a["ds_scale"] = _f32(dev, 1.0)
+            a["ds_amax"] = _f32(dev)
+            a["softmax_scale"] = float(d) ** -0.5
+            self.attn = a
+        return self
+
+    def input_tensors(self):
+        """(name, device BF16 tensor) of every input of a step, in a fixed order."""
+        out = []
+        for lin in self.linears:
+            out += [("x_" + lin.name, lin.x.x), ("w_" + lin.name, lin.w.x), ("dy_" + lin.name, lin.dy.x)]
+        if self.attn is not None:
+            out += [(n, self.attn[n].x) for n in ("q", "k", "v", "do")]
+        return out
+
+    def output_tensors(self):
+        out = []
+        for lin in self.linears:
+            out += [("y_" + lin.name, lin.y), ("dx_" + lin.name, lin.dx), ("dw_" + lin.name, lin.dw)]
+        if self.attn is not None:
+            out += [(n, self.attn[n]) for n in ("o", "lse", "dq", "dk", "dv")]
+        return out
+
+    # ------------------------------------------------------------------ work accounting
+    def gemm_flops(self):
+        return sum(l.flops for l in self.linears)
+
+    def attention_flops(self):
+        """Causal attention: forward 2*B*Hq*N^2*d (half of the dense 4*N^2*d), backward 2.5x that."""
+        if self.attn is None:
+            return 0.0
+        c = self.cfg
+        fwd = 2.0 * self.B * c.n_q_heads * self.N * self.N * c.head_dim
+        return 3.5 * fwd
+
+    def quantize_bytes(self):
+        """Algorithmic HBM bytes of the JIT quantize calls: 2 (amax read) + 2 (cast read) + 1 per FP8 copy."""
+        b = 0
+        for lin in self.linears:
+            for t in (lin.x, lin.w, lin.dy):
+                b += t.x.numel() * (4 + 1 + (1 if t.transpose else 0))
+        if self.attn is not None:
+            for n in ("q", "k", "v", "do"):
+                b += self.attn[n].x.numel() * 5
+        return b
+
+    def launches_per_step(self):
+        n = 0
+        for _ in self.linears:
+            n += 3 * self.KERNELS_PER_QUANTIZE + 3
+        if self.attn is not None:
+            n += 4 * self.KERNELS_PER_QUANTIZE + 1 + self.KERNELS_PER_ATTN_BWD
+        return n
+
+    # ------------------------------------------------------------------ the step
+    def calibrate_ds_scale(self):
+        """Delayed-scaling style: one backward with scale 1 gives amax(dS); scale = 57344 / amax."""
+        if self.attn is None:
+            return
+        a = self.attn
+        a["ds_scale"].fill_(1.0)
+        self.step()
+        tmp_scale_inv = _f32(self.device)
+        fp8.fp8_scale(a["ds_amax"], fp8.E5M2, 0, a["ds_scale"], tmp_scale_inv)
+        torch.cuda.synchronize(self.device)
+
+    def step(self, time_gemms: bool = False):
+        ev = []
+
+        def gemm(fn, *args, **kw):
+            if time_gemms:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn(*args, **kw)
+                e1.record()
+                ev.append((e0, e1))
+            else:
+                fn(*args, **kw)
+
+        for lin in self.linears:
+            lin.x.quantize()
+            lin.w.quantize()
+            lin.dy.quantize()
+            gemm(fp8.fp8_linear_fwd, lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
+            gemm(fp8.fp8_linear_dgrad, lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+            gemm(fp8.fp8_linear_wgrad, lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+        if self.attn is not None:
+            a = self.attn
+            for n in ("q", "k", "v", "do"):
+                a[n].quantize()
+            fp8.fp8_attention_fwd(a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv, a["v"].scale_inv,
+                                  a["softmax_scale"], True, a["o"], a["lse"], None)
+            fp8.fp8_attention_bwd(a["q"].q, a["k"].q, a["v"].q, a["do"].q, a["o"], a["lse"], a["q"].scale_inv,
+                                  a["k"].scale_inv, a["v"].scale_inv, a["do"].scale_inv, a["softmax_scale"],
+                                  a["ds_scale"], True, a["dq"], a["dk"], a["dv"], a["ws"], ds_amax=a["ds_amax"])
+        if time_gemms:
+            self.gemm_events.append(ev)

@@ -3,10 +3,10 @@
  * Holds none of the method's arithmetic: it only draws N(0, std) values from a counter-based
  * generator, applies the outlier edits the workload recipes ask for, and rounds to BF16 bits.
  *
- * element i of tensor `tid` under `seed`:
- *   u1, u2 = uniform(splitmix64(key + 2i)), uniform(splitmix64(key + 2i + 1)),
+ * elements 2j and 2j+1 of tensor `tid` under `seed` share one Box-Muller pair:
+ *   u1, u2 = uniform(splitmix64(key + 2j)), uniform(splitmix64(key + 2j + 1)),
  *   key    = splitmix64(seed * 0x9E3779B97F4A7C15 + tid)
- *   z      = sqrt(-2 ln u1) * cos(2 pi u2)                     (Box-Muller, double)
+ *   z      = sqrt(-2 ln u1) * cos(2 pi u2)  for element 2j,  ... * sin(2 pi u2)  for element 2j+1   (double)
  *   v      = z * std, times col_factor if the column is an outlier column,
  *            or replaced by +-elem_value with probability elem_prob (third draw)
  *   out    = BF16(round-to-nearest-even(float(v)))
@@ -42,13 +42,17 @@ void synth_fill_bf16(uint16_t *out, int64_t rows, int64_t cols, uint64_t seed, u
 {
     const uint64_t key = splitmix64(seed * 0x9E3779B97F4A7C15ull + tid);
     const uint64_t key2 = splitmix64(key ^ 0xD1B54A32D192ED03ull);
+    const int64_t n = rows * cols;
 #pragma omp parallel for schedule(static)
-    for (int64_t r = 0; r < rows; ++r) {
-        for (int64_t c = 0; c < cols; ++c) {
-            const uint64_t i = (uint64_t)(r * cols + c);
-            const double u1 = u01(splitmix64(key + 2 * i));
-            const double u2 = u01(splitmix64(key + 2 * i + 1));
-            double v = sqrt(-2.0 * log(u1)) * cos(6.283185307179586476925 * u2) * std;
+    for (int64_t ii = 0; ii < n; ++ii) {
+        {
+            const uint64_t i = (uint64_t)ii;
+            const int64_t c = ii % cols;
+            const uint64_t j = i >> 1;
+            const double u1 = u01(splitmix64(key + 2 * j));
+            const double u2 = u01(splitmix64(key + 2 * j + 1));
+            const double ang = 6.283185307179586476925 * u2;
+            double v = sqrt(-2.0 * log(u1)) * ((i & 1) ? sin(ang) : cos(ang)) * std;
             if (col_is_outlier && col_is_outlier[c]) v *= col_factor;
             if (elem_prob > 0.0) {
                 const uint64_t r3 = splitmix64(key2 + i);

@@ -41,7 +41,17 @@ def gpu_quantize(x_bits: np.ndarray, fmt: int, transpose: bool = False):
     return q, qt, a, s, si
 
 
-def rel_err(got: np.ndarray, ref: np.ndarray, mag: np.ndarray) -> float:
-    """max |got - ref| / mag, mag = the sum of |a||b| over the reduction (componentwise GEMM error)."""
+def rel_err(got: np.ndarray, ref: np.ndarray, mag: np.ndarray, floor_frac: float = 0.0) -> float:
+    """max |got - ref| / mag, mag = the sum of |a||b| over the reduction (componentwise GEMM error).
+
+    floor_frac > 0 floors the denominator at floor_frac * mean(mag).  The attention gradients need it:
+    dS = P o (dP - D) cancels to an exact zero on rows whose softmax is one-hot (the oracle's double
+    arithmetic gives 0, FP32 gives rounding noise ~1e-7 of the operands), so there mag is 0 and the plain
+    ratio would divide noise by zero; the floor turns the check into an absolute one at 1% of the
+    tensor's typical magnitude sum."""
     tiny = 1e-30
-    return float(np.max(np.abs(got - ref) / np.maximum(mag, tiny)))
+    den = np.maximum(mag, max(tiny, floor_frac * float(np.mean(mag))))
+    return float(np.max(np.abs(got - ref) / den))
+
+
+BWD_FLOOR = 1e-2
