@@ -37,7 +37,7 @@ class AttnParams(C.Structure):
                 ("max_mode", C.c_int32), ("pad_", C.c_int32),
                 ("s", C.c_double), ("c_P", C.c_double),
                 ("q_inv", C.c_double), ("k_inv", C.c_double), ("v_inv", C.c_double), ("do_inv", C.c_double),
-                ("ds_scale", C.c_double)]
+                ("ds_scale", C.c_double), ("flip_eps", C.c_double)]
 
 
 def _L():
@@ -195,12 +195,12 @@ def linear_wgrad(dy8, x8, sdy_inv, sx_inv, rows=None, cols=None, prev=None):
 
 # ---------------------------------------------------------------- attention
 def attn_params(B, N, Hq, Hkv, d, causal=True, quant=True, kv_block=0, max_mode=0, s=None, c_P=448.0,
-                q_inv=1.0, k_inv=1.0, v_inv=1.0, do_inv=1.0, ds_scale=1.0) -> AttnParams:
+                q_inv=1.0, k_inv=1.0, v_inv=1.0, do_inv=1.0, ds_scale=1.0, flip_eps=0.0) -> AttnParams:
     return AttnParams(B=B, N=N, Hq=Hq, Hkv=Hkv, d=d, causal=int(causal), quant=int(quant),
                       kv_block=kv_block, max_mode=max_mode, pad_=0,
                       s=float(d ** -0.5 if s is None else s), c_P=float(c_P),
                       q_inv=float(q_inv), k_inv=float(k_inv), v_inv=float(v_inv), do_inv=float(do_inv),
-                      ds_scale=float(ds_scale))
+                      ds_scale=float(ds_scale), flip_eps=float(flip_eps))
 
 
 def _pairs(sel, nb, nh):
@@ -209,10 +209,11 @@ def _pairs(sel, nb, nh):
     return _c(np.asarray(sel, dtype=np.int32).reshape(-1, 2), np.int32)
 
 
-def attention_fwd(q, k, v, p: AttnParams, heads=None, rows=None, real=False):
+def attention_fwd(q, k, v, p: AttnParams, heads=None, rows=None, real=False, with_slack=False):
     """O[pair,row,d], LSE[pair,row], mag for the (batch, query head) pairs and the query-row range given.
 
-    q, k, v: [B,N,H,d] uint8 E4M3 codes, or float64 values when real=True."""
+    q, k, v: [B,N,H,d] uint8 E4M3 codes, or float64 values when real=True.  with_slack adds a fourth
+    array: how far O may move through FP32-vs-double tie decisions of the P8 encode (needs p.flip_eps)."""
     dt = np.float64 if real else np.uint8
     q, k, v = _c(q, dt), _c(k, dt), _c(v, dt)
     bh = _pairs(heads, p.B, p.Hq)
@@ -220,18 +221,21 @@ def attention_fwd(q, k, v, p: AttnParams, heads=None, rows=None, real=False):
     O = np.empty((bh.shape[0], r1 - r0, p.d), dtype=np.float64)
     LSE = np.empty((bh.shape[0], r1 - r0), dtype=np.float64)
     mag = np.empty_like(O)
+    slack = np.zeros_like(O) if with_slack else None
     f = _L().oracle_attention_fwd_real if real else _L().oracle_attention_fwd
     f.restype = None
     f(_p(q), _p(k), _p(v), C.byref(p), _p(bh), C.c_int(bh.shape[0]), C.c_int(r0), C.c_int(r1),
-      _p(O), _p(LSE), _p(mag))
-    return O, LSE, mag
+      _p(O), _p(LSE), _p(mag), _p(slack))
+    return (O, LSE, mag, slack) if with_slack else (O, LSE, mag)
 
 
 def attention_bwd(q, k, v, do, O, LSE, p: AttnParams, kv_heads=None, q_rows=None, k_rows=None, real=False):
     """Gradients for the (batch, kv head) pairs given, over query rows x key rows.
 
     O: [B,N,Hq,d] float64 (the values handed to the backward, e.g. BF16-rounded), LSE: [B,Hq,N] float64.
-    Returns dict with dQ[pair,G,nq,d], dK/dV[pair,nk,d], mag_*, amax_dS."""
+    Returns dict with dQ[pair,G,nq,d], dK/dV[pair,nk,d], mag_* (error-metric denominators), slack_* (how far
+    each output may move through FP32-vs-double tie decisions of the two encodes; zero unless p.flip_eps > 0)
+    and amax_dS."""
     dt = np.float64 if real else np.uint8
     q, k, v, do = _c(q, dt), _c(k, dt), _c(v, dt), _c(do, dt)
     O = _c(O, np.float64)
@@ -247,12 +251,14 @@ def attention_bwd(q, k, v, do, O, LSE, p: AttnParams, kv_heads=None, q_rows=None
     }
     for key in ("dQ", "dK", "dV"):
         out["mag_" + key] = np.empty_like(out[key])
+        out["slack_" + key] = np.zeros_like(out[key])
     am = C.c_double()
     f = _L().oracle_attention_bwd_real if real else _L().oracle_attention_bwd
     f.restype = None
     f(_p(q), _p(k), _p(v), _p(do), _p(O), _p(LSE), C.byref(p), _p(bg), C.c_int(n),
       C.c_int(q0), C.c_int(q1), C.c_int(k0), C.c_int(k1),
       _p(out["dQ"]), _p(out["dK"]), _p(out["dV"]),
-      _p(out["mag_dQ"]), _p(out["mag_dK"]), _p(out["mag_dV"]), C.byref(am))
+      _p(out["mag_dQ"]), _p(out["mag_dK"]), _p(out["mag_dV"]), C.byref(am),
+      _p(out["slack_dQ"]), _p(out["slack_dK"]), _p(out["slack_dV"]))
     out["amax_dS"] = am.value
     return out

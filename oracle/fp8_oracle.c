@@ -246,6 +246,7 @@ typedef struct {
     double c_P;        /* quantisation scale of P~ = exp(x - m) in (0,1]; 448 = FP8Max/amax with amax = 1 */
     double q_inv, k_inv, v_inv, do_inv;  /* descales of Q8, K8, V8, dO8 */
     double ds_scale;   /* backward: quantisation scale of dS */
+    double flip_eps;   /* relative uncertainty of an FP32 evaluation (0 disables the slack outputs) */
 } oracle_attn_params;
 
 typedef struct {
@@ -279,6 +280,40 @@ static double score(const oracle_attn_params *p, const operand *Q, const operand
     return p->s * p->q_inv * p->k_inv * acc;
 }
 
+/* same sum over absolute values: the size against which an FP32 evaluation of x_ij is accurate */
+static double score_mag(const oracle_attn_params *p, const operand *Q, const operand *K,
+                        int b, int h, int g, int i, int j)
+{
+    double acc = 0.0;
+    for (int dd = 0; dd < p->d; ++dd)
+        acc += fabs(ld(Q, idx4(p, p->Hq, b, i, h, dd)) * ld(K, idx4(p, p->Hkv, b, j, g, dd)));
+    return p->s * p->q_inv * p->k_inv * acc;
+}
+
+/* Where a value about to be encoded lies within `band` of the rounding boundary between two neighbouring
+ * codes, a kernel that evaluates it in binary32 may legitimately pick the other code.  Returns the distance
+ * between the two candidate values in that case, else 0.  The sums of these distances (times the other
+ * operand's magnitude) are the `slack` outputs: the amount by which a correct FP32 implementation may
+ * differ from this double-precision one through such tie decisions alone. */
+static double flip_step(double y, double band, int fmt)
+{
+    if (!(band > 0.0)) return 0.0;
+    const double a = fabs(y);
+    const int top = (fmt == ORACLE_E4M3) ? 0x7E : 0x7B;
+    if (a > oracle_fp8_max(fmt) + band) return 0.0;
+    const int c = oracle_fp8_encode((float)a, fmt) & 0x7F;
+    const double v = oracle_fp8_decode((uint8_t)c, fmt);
+    if (c < top) {
+        const double up = oracle_fp8_decode((uint8_t)(c + 1), fmt);
+        if (0.5 * (v + up) - a <= band) return up - v;
+    }
+    if (c > 0) {
+        const double dn = oracle_fp8_decode((uint8_t)(c - 1), fmt);
+        if (a - 0.5 * (v + dn) <= band) return v - dn;
+    }
+    return 0.0;
+}
+
 static double quant_p(const oracle_attn_params *p, double pt)
 {
     /* P~ * c_P is formed as a binary32 product and rounded once to E4M3; returned still scaled by c_P */
@@ -294,9 +329,10 @@ static double quant_p(const oracle_attn_params *p, double pt)
  * Outputs: O[pair][row][d], LSE[pair][row], mag (sum of |P8||V| with the same normalisation; may be NULL). */
 static void attention_fwd_core(const operand *Q, const operand *K, const operand *V,
                                const oracle_attn_params *p, const int32_t *bh, int nbh, int r0, int r1,
-                               double *O, double *LSE, double *mag)
+                               double *O, double *LSE, double *mag, double *slack)
 {
     const int d = p->d, nr = r1 - r0, G = p->Hq / p->Hkv;
+    const int want_slack = slack != NULL && p->quant && p->flip_eps > 0.0;
     const double LOG2E = 1.4426950408889634074, LN2 = 0.69314718055994530942;
     const double cP = p->quant ? p->c_P : 1.0;
 #pragma omp parallel for collapse(2) schedule(dynamic, 8)
@@ -308,6 +344,7 @@ static void attention_fwd_core(const operand *Q, const operand *K, const operand
             double *x = (double *)malloc(sizeof(double) * (size_t)Bc);
             double *acc = (double *)calloc((size_t)d, sizeof(double));
             double *am = (double *)calloc((size_t)d, sizeof(double));
+            double *sl = (double *)calloc((size_t)d, sizeof(double));
             double m = -INFINITY, l = 0.0;
             for (int j0 = 0; j0 <= jlast; j0 += Bc) {
                 const int j1 = (j0 + Bc - 1 < jlast) ? j0 + Bc - 1 : jlast;
@@ -320,17 +357,24 @@ static void attention_fwd_core(const operand *Q, const operand *K, const operand
                 if (cand > m) {
                     double f = isinf(m) ? 0.0 : exp(m - cand);
                     l *= f;
-                    for (int dd = 0; dd < d; ++dd) { acc[dd] *= f; am[dd] *= f; }
+                    for (int dd = 0; dd < d; ++dd) { acc[dd] *= f; am[dd] *= f; sl[dd] *= f; }
                     m = cand;
                 }
                 for (int j = j0; j <= j1; ++j) {
                     double pt = exp(x[j - j0] - m);
                     l += pt;
                     double w = quant_p(p, pt);
+                    double step = 0.0;
+                    if (want_slack) {
+                        /* P~ inherits the absolute error of its exponent: eps * (1 + |terms of x|) */
+                        const double y = pt * p->c_P;
+                        step = flip_step(y, y * p->flip_eps * (1.0 + score_mag(p, Q, K, b, h, g, i, j)), ORACLE_E4M3);
+                    }
                     for (int dd = 0; dd < d; ++dd) {
                         double v = ld(V, idx4(p, p->Hkv, b, j, g, dd));
                         acc[dd] += w * v;
                         am[dd] += w * fabs(v);
+                        sl[dd] += step * fabs(v);
                     }
                 }
             }
@@ -338,34 +382,35 @@ static void attention_fwd_core(const operand *Q, const operand *K, const operand
             for (int dd = 0; dd < d; ++dd) {
                 O[o * d + dd] = p->v_inv * acc[dd] / (cP * l);
                 if (mag) mag[o * d + dd] = p->v_inv * am[dd] / (cP * l);
+                if (slack) slack[o * d + dd] = p->v_inv * sl[dd] / (cP * l);
             }
             LSE[o] = m + log(l);
-            free(x); free(acc); free(am);
+            free(x); free(acc); free(am); free(sl);
         }
     }
 }
 
 void oracle_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8,
                           const oracle_attn_params *p, const int32_t *bh, int nbh, int r0, int r1,
-                          double *O, double *LSE, double *mag)
+                          double *O, double *LSE, double *mag, double *slack)
 {
     operand Q, K, V;
     operand_init(&Q, Q8, NULL, ORACLE_E4M3);
     operand_init(&K, K8, NULL, ORACLE_E4M3);
     operand_init(&V, V8, NULL, ORACLE_E4M3);
-    attention_fwd_core(&Q, &K, &V, p, bh, nbh, r0, r1, O, LSE, mag);
+    attention_fwd_core(&Q, &K, &V, p, bh, nbh, r0, r1, O, LSE, mag, slack);
 }
 
 /* Same arithmetic on real-valued operands (used with quant = 0 for the finite-difference pin). */
 void oracle_attention_fwd_real(const double *Qd, const double *Kd, const double *Vd,
                                const oracle_attn_params *p, const int32_t *bh, int nbh, int r0, int r1,
-                               double *O, double *LSE, double *mag)
+                               double *O, double *LSE, double *mag, double *slack)
 {
     operand Q, K, V;
     operand_init(&Q, NULL, Qd, ORACLE_E4M3);
     operand_init(&K, NULL, Kd, ORACLE_E4M3);
     operand_init(&V, NULL, Vd, ORACLE_E4M3);
-    attention_fwd_core(&Q, &K, &V, p, bh, nbh, r0, r1, O, LSE, mag);
+    attention_fwd_core(&Q, &K, &V, p, bh, nbh, r0, r1, O, LSE, mag, slack);
 }
 
 /* Backward of O = PV through the softmax (the paper runs it in FP8 too but gives no formula; this is the
@@ -378,26 +423,37 @@ void oracle_attention_fwd_real(const double *Qd, const double *Kd, const double 
  * Covers query rows [q0,q1) x key rows [k0,k1) for the listed (batch, kv head) pairs: dQ is complete
  * when the key range holds every key the rows attend to, dK/dV when the query range holds every query
  * that attends to the keys.  O is [B,N,Hq,d] and LSE [B,Hq,N], given by the caller.
- * Outputs: dQ[pair][G][q1-q0][d], dK,dV[pair][k1-k0][d], their magnitude sums (nullable), amax of |dS|. */
+ * Outputs: dQ[pair][G][q1-q0][d], dK,dV[pair][k1-k0][d], amax of |dS|, and (nullable) the magnitude sums
+ * that serve as error-metric denominators: for dV the sum of |P8||dO|; for dQ and dK the sums of
+ * P(|dP| + |D|)|K| resp. P(|dP| + |D|)|Q|, i.e. the size of the terms *before* dP - D cancels (the
+ * componentwise condition of the formula: where softmax is nearly one-hot, dP - D is a difference of two
+ * nearly equal numbers and an FP32 evaluation is only accurate relative to those numbers). */
 static void attention_bwd_core(const operand *Q, const operand *K, const operand *V, const operand *dO,
                                const double *O, const double *LSE, const oracle_attn_params *p,
                                const int32_t *bg, int nbg, int q0, int q1, int k0, int k1,
                                double *dQ, double *dK, double *dV,
-                               double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS)
+                               double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS,
+                               double *slack_dQ, double *slack_dK, double *slack_dV)
 {
     const int d = p->d, G = p->Hq / p->Hkv, nq = q1 - q0, nk = k1 - k0;
     const double cP = p->quant ? p->c_P : 1.0;
+    const int want_slack = p->quant && p->flip_eps > 0.0 && slack_dQ && slack_dK && slack_dV;
     double amax = 0.0;
-    /* D_i for every (pair, head in group, row) */
+    /* D_i for every (pair, head in group, row), and the sum of the absolute terms of D_i */
     double *D = (double *)malloc(sizeof(double) * (size_t)nbg * G * nq);
+    double *Dm = (double *)malloc(sizeof(double) * (size_t)nbg * G * nq);
 #pragma omp parallel for collapse(2) schedule(static)
     for (int pi = 0; pi < nbg; ++pi)
         for (int r = 0; r < G * nq; ++r) {
             const int b = bg[2 * pi], g = bg[2 * pi + 1], h = g * G + r / nq, i = q0 + r % nq;
-            double acc = 0.0;
-            for (int dd = 0; dd < d; ++dd)
-                acc += p->do_inv * ld(dO, idx4(p, p->Hq, b, i, h, dd)) * O[idx4(p, p->Hq, b, i, h, dd)];
+            double acc = 0.0, accm = 0.0;
+            for (int dd = 0; dd < d; ++dd) {
+                const double t = p->do_inv * ld(dO, idx4(p, p->Hq, b, i, h, dd)) * O[idx4(p, p->Hq, b, i, h, dd)];
+                acc += t;
+                accm += fabs(t);
+            }
             D[((int64_t)pi * G + r / nq) * nq + r % nq] = acc;
+            Dm[((int64_t)pi * G + r / nq) * nq + r % nq] = accm;
         }
 
     /* row-local pass: dQ_i, and amax|dS| */
@@ -407,27 +463,41 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
             const int b = bg[2 * pi], g = bg[2 * pi + 1], hg = r / nq, h = g * G + hg, i = q0 + r % nq;
             const double lse = LSE[((int64_t)b * p->Hq + h) * p->N + i];
             const double Di = D[((int64_t)pi * G + hg) * nq + (i - q0)];
+            const double Dmi = Dm[((int64_t)pi * G + hg) * nq + (i - q0)];
             double *out = dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d;
             double *mout = mag_dQ ? mag_dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d : NULL;
-            for (int dd = 0; dd < d; ++dd) { out[dd] = 0.0; if (mout) mout[dd] = 0.0; }
+            double *sout = want_slack ? slack_dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d : NULL;
+            for (int dd = 0; dd < d; ++dd) { out[dd] = 0.0; if (mout) mout[dd] = 0.0; if (sout) sout[dd] = 0.0; }
             for (int j = k0; j < k1; ++j) {
                 if (p->causal && j > i) break;
                 double P = exp(score(p, Q, K, b, h, g, i, j) - lse);
-                double dP = 0.0;
-                for (int dd = 0; dd < d; ++dd)
-                    dP += ld(dO, idx4(p, p->Hq, b, i, h, dd)) * ld(V, idx4(p, p->Hkv, b, j, g, dd));
+                double dP = 0.0, dPm = 0.0;
+                for (int dd = 0; dd < d; ++dd) {
+                    const double t = ld(dO, idx4(p, p->Hq, b, i, h, dd)) * ld(V, idx4(p, p->Hkv, b, j, g, dd));
+                    dP += t;
+                    dPm += fabs(t);
+                }
                 dP *= p->do_inv * p->v_inv;
+                dPm *= p->do_inv * p->v_inv;
                 double dS = P * (dP - Di);
+                const double m_ds = P * (fabs(dP) + fabs(Di));   /* size of dS before the subtraction cancels */
                 if (fabs(dS) > amax) amax = fabs(dS);
-                double u = dS;
+                double u = dS, step = 0.0;
                 if (p->quant) {
                     volatile float prod = (float)dS * (float)p->ds_scale;
                     u = oracle_fp8_decode(oracle_fp8_encode(prod, ORACLE_E5M2), ORACLE_E5M2) / p->ds_scale;
                 }
+                if (want_slack) {
+                    /* uncertainty of dS: P * eps * (terms of dP and D) + |dS| * (relative uncertainty of P) */
+                    const double band = p->flip_eps * (P * (dPm + Dmi) +
+                                                       fabs(dS) * (1.0 + score_mag(p, Q, K, b, h, g, i, j)));
+                    step = flip_step(dS * p->ds_scale, band * p->ds_scale, ORACLE_E5M2) / p->ds_scale;
+                }
                 for (int dd = 0; dd < d; ++dd) {
                     double kv = ld(K, idx4(p, p->Hkv, b, j, g, dd));
                     out[dd] += p->s * p->k_inv * u * kv;
-                    if (mout) mout[dd] += p->s * p->k_inv * fabs(u) * fabs(kv);
+                    if (mout) mout[dd] += p->s * p->k_inv * m_ds * fabs(kv);
+                    if (sout) sout[dd] += p->s * p->k_inv * step * fabs(kv);
                 }
             }
         }
@@ -441,10 +511,13 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
             double *oV = dV + ((int64_t)pi * nk + (j - k0)) * d;
             double *mK = mag_dK ? mag_dK + ((int64_t)pi * nk + (j - k0)) * d : NULL;
             double *mV = mag_dV ? mag_dV + ((int64_t)pi * nk + (j - k0)) * d : NULL;
+            double *sK = want_slack ? slack_dK + ((int64_t)pi * nk + (j - k0)) * d : NULL;
+            double *sV = want_slack ? slack_dV + ((int64_t)pi * nk + (j - k0)) * d : NULL;
             for (int dd = 0; dd < d; ++dd) {
                 oK[dd] = 0.0; oV[dd] = 0.0;
                 if (mK) mK[dd] = 0.0;
                 if (mV) mV[dd] = 0.0;
+                if (sK) { sK[dd] = 0.0; sV[dd] = 0.0; }
             }
             for (int hg = 0; hg < G; ++hg) {
                 const int h = g * G + hg;
@@ -452,17 +525,29 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
                     if (p->causal && j > i) continue;
                     const double lse = LSE[((int64_t)b * p->Hq + h) * p->N + i];
                     const double Di = D[((int64_t)pi * G + hg) * nq + (i - q0)];
+                    const double Dmi = Dm[((int64_t)pi * G + hg) * nq + (i - q0)];
                     double P = exp(score(p, Q, K, b, h, g, i, j) - lse);
                     double w = quant_p(p, P) / cP;
-                    double dP = 0.0;
-                    for (int dd = 0; dd < d; ++dd)
-                        dP += ld(dO, idx4(p, p->Hq, b, i, h, dd)) * ld(V, idx4(p, p->Hkv, b, j, g, dd));
+                    double dP = 0.0, dPm = 0.0;
+                    for (int dd = 0; dd < d; ++dd) {
+                        const double t = ld(dO, idx4(p, p->Hq, b, i, h, dd)) * ld(V, idx4(p, p->Hkv, b, j, g, dd));
+                        dP += t;
+                        dPm += fabs(t);
+                    }
                     dP *= p->do_inv * p->v_inv;
+                    dPm *= p->do_inv * p->v_inv;
                     double dS = P * (dP - Di);
-                    double u = dS;
+                    const double m_ds = P * (fabs(dP) + fabs(Di));
+                    double u = dS, stepS = 0.0, stepP = 0.0;
                     if (p->quant) {
                         volatile float prod = (float)dS * (float)p->ds_scale;
                         u = oracle_fp8_decode(oracle_fp8_encode(prod, ORACLE_E5M2), ORACLE_E5M2) / p->ds_scale;
+                    }
+                    if (want_slack) {
+                        const double xm = 1.0 + score_mag(p, Q, K, b, h, g, i, j);
+                        const double band = p->flip_eps * (P * (dPm + Dmi) + fabs(dS) * xm);
+                        stepS = flip_step(dS * p->ds_scale, band * p->ds_scale, ORACLE_E5M2) / p->ds_scale;
+                        stepP = flip_step(P * p->c_P, P * p->c_P * p->flip_eps * xm, ORACLE_E4M3) / p->c_P;
                     }
                     for (int dd = 0; dd < d; ++dd) {
                         double dov = ld(dO, idx4(p, p->Hq, b, i, h, dd));
@@ -470,12 +555,17 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
                         oV[dd] += p->do_inv * w * dov;
                         oK[dd] += p->s * p->q_inv * u * qv;
                         if (mV) mV[dd] += p->do_inv * w * fabs(dov);
-                        if (mK) mK[dd] += p->s * p->q_inv * fabs(u) * fabs(qv);
+                        if (mK) mK[dd] += p->s * p->q_inv * m_ds * fabs(qv);
+                        if (sK) {
+                            sK[dd] += p->s * p->q_inv * stepS * fabs(qv);
+                            sV[dd] += p->do_inv * stepP * fabs(dov);
+                        }
                     }
                 }
             }
         }
     free(D);
+    free(Dm);
     if (amax_dS) *amax_dS = amax;
 }
 
@@ -483,7 +573,8 @@ void oracle_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V
                           const double *O, const double *LSE, const oracle_attn_params *p,
                           const int32_t *bg, int nbg, int q0, int q1, int k0, int k1,
                           double *dQ, double *dK, double *dV,
-                          double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS)
+                          double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS,
+                          double *slack_dQ, double *slack_dK, double *slack_dV)
 {
     operand Q, K, V, dO;
     operand_init(&Q, Q8, NULL, ORACLE_E4M3);
@@ -491,14 +582,15 @@ void oracle_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V
     operand_init(&V, V8, NULL, ORACLE_E4M3);
     operand_init(&dO, dO8, NULL, ORACLE_E5M2);
     attention_bwd_core(&Q, &K, &V, &dO, O, LSE, p, bg, nbg, q0, q1, k0, k1,
-                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS);
+                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS, slack_dQ, slack_dK, slack_dV);
 }
 
 void oracle_attention_bwd_real(const double *Qd, const double *Kd, const double *Vd, const double *dOd,
                                const double *O, const double *LSE, const oracle_attn_params *p,
                                const int32_t *bg, int nbg, int q0, int q1, int k0, int k1,
                                double *dQ, double *dK, double *dV,
-                               double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS)
+                               double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS,
+                               double *slack_dQ, double *slack_dK, double *slack_dV)
 {
     operand Q, K, V, dO;
     operand_init(&Q, NULL, Qd, ORACLE_E4M3);
@@ -506,7 +598,7 @@ void oracle_attention_bwd_real(const double *Qd, const double *Kd, const double 
     operand_init(&V, NULL, Vd, ORACLE_E4M3);
     operand_init(&dO, NULL, dOd, ORACLE_E5M2);
     attention_bwd_core(&Q, &K, &V, &dO, O, LSE, p, bg, nbg, q0, q1, k0, k1,
-                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS);
+                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS, slack_dQ, slack_dK, slack_dV);
 }
 
 int oracle_num_threads(void)

@@ -41,17 +41,26 @@ def gpu_quantize(x_bits: np.ndarray, fmt: int, transpose: bool = False):
     return q, qt, a, s, si
 
 
-def rel_err(got: np.ndarray, ref: np.ndarray, mag: np.ndarray, floor_frac: float = 0.0) -> float:
-    """max |got - ref| / mag, mag = the sum of |a||b| over the reduction (componentwise GEMM error).
+def rel_err(got: np.ndarray, ref: np.ndarray, mag: np.ndarray, slack=None, floor_frac: float = 0.0) -> float:
+    """max (|got - ref| - slack)+ / mag: componentwise error against the oracle's magnitude sums.
 
-    floor_frac > 0 floors the denominator at floor_frac * mean(mag).  The attention gradients need it:
-    dS = P o (dP - D) cancels to an exact zero on rows whose softmax is one-hot (the oracle's double
-    arithmetic gives 0, FP32 gives rounding noise ~1e-7 of the operands), so there mag is 0 and the plain
-    ratio would divide noise by zero; the floor turns the check into an absolute one at 1% of the
-    tensor's typical magnitude sum."""
+    mag: for GEMMs and the attention output, the sum of |a||b| over the reduction; for dQ and dK it is built
+    from P(|dP| + |D|), the size of dS before dP - D cancels (an FP32 evaluation of that difference is only
+    accurate relative to the two numbers being subtracted).
+    slack: the oracle's bound on how far an output may move because a value that is re-quantised to FP8
+    inside the kernel (P~, dS) lies within FP32 rounding noise of a tie between two codes; there both codes
+    are correct results, and the jump between them (6-25% of that term) is not an error.
+    floor_frac floors the denominator at floor_frac * mean(mag) so an output with all-zero operands cannot
+    divide by zero."""
     tiny = 1e-30
     den = np.maximum(mag, max(tiny, floor_frac * float(np.mean(mag))))
-    return float(np.max(np.abs(got - ref) / den))
+    diff = np.abs(got - ref)
+    if slack is not None:
+        diff = np.maximum(diff - slack, 0.0)
+    return float(np.max(diff / den))
 
 
-BWD_FLOOR = 1e-2
+BWD_FLOOR = 1e-6
+# relative uncertainty of the kernel's FP32 evaluation of a length-128 dot product and an exp2:
+# measured tcgen05 accumulation error is 2^-22 of the magnitude sum at K = 128; 8x margin
+FLIP_EPS = 2.0 ** -19

@@ -217,3 +217,27 @@ def test_softmax_scale_fold_identity():
     O2, _, _ = o.attention_fwd(q, k, v, p2)
     assert np.allclose(O1, O2, rtol=1e-12)
     assert abs(0.125 * 128 ** 0.5 - g2) < 1e-12
+
+
+def test_tie_slack_outputs():
+    """slack_* bound the effect of FP32-vs-double tie decisions: zero without flip_eps, monotone in it, and
+    with an absurdly large eps every term counts with the full gap between neighbouring codes."""
+    B, N, H, d = 1, 10, 1, 8
+    q, k, v = rand_codes((B, N, H, d), 60), rand_codes((B, N, H, d), 61), rand_codes((B, N, H, d), 62)
+    do = rand_codes((B, N, H, d), 63, 0x10, 0x30)
+    prev_f, prev_b = None, None
+    for eps in (0.0, 1e-6, 1e-2, 1e3):
+        p = o.attn_params(B, N, H, H, d, quant=True, s=0.4, ds_scale=64.0, flip_eps=eps)
+        O, LSE, mag, slack = o.attention_fwd(q, k, v, p, with_slack=True)
+        g = o.attention_bwd(q, k, v, do, O.reshape(B, N, H, d), LSE.reshape(B, H, N), p)
+        tot_b = sum(g["slack_" + n].sum() for n in ("dQ", "dK", "dV"))
+        if eps == 0.0:
+            assert slack.sum() == 0.0 and tot_b == 0.0
+        else:
+            assert slack.sum() >= prev_f and tot_b >= prev_b
+        prev_f, prev_b = slack.sum(), tot_b
+    assert (slack > 0).all()
+    # Q = 0: every P~ c_P is exactly 448 (the top code, no neighbour above, the one below is 32 away)
+    p = o.attn_params(B, N, H, H, d, quant=True, flip_eps=1e-6)
+    _, _, _, slack = o.attention_fwd(np.zeros_like(q), k, v, p, with_slack=True)
+    assert slack.sum() == 0.0
