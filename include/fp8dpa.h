@@ -135,6 +135,30 @@ FP8_API int fp8_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uint8_
                       int causal, int B, int N, int Hq, int Hkv, int d,
                       void *dQ_bf16, void *dK_bf16, void *dV_bf16, void *ws, size_t ws_bytes, void *stream);
 
+/* ---- attention backward without caller scratch -------------------------------------------------------
+ * (No counterpart in the paper: this is a packaging variant of fp8_attention_bwd, same arithmetic.)
+ *
+ * For callers that cannot allocate or pass device scratch - e.g. code that runs inside an already
+ * committed memory pool, a plugin that only ever receives its input and output buffers, or a launch thread
+ * that must not re-enter an allocator.  The scratch fp8_attention_bwd takes as `ws` is replaced by a fixed
+ * array of FP8_STATIC_SCRATCH_BYTES inside the library's device image; every GPU that loads the library
+ * holds that array until the process exits.  The call allocates nothing (no cudaMalloc / cudaFree, no
+ * allocating library routine).
+ *
+ * Limit: fp8_attention_workspace_bytes(1, B, N, Hq, Hkv, d), about B*N*Hq*(d+1)*4 bytes, must not exceed
+ * FP8_STATIC_SCRATCH_BYTES; larger problems return FP8_ERR_WORKSPACE and launch nothing.
+ * The first call on each device looks up the array's device address (with that device current); make that
+ * first call before any stream capture begins.
+ * All calls share the one array and it keeps the previous call's contents; each call clears what it needs
+ * to start from zero.  Two calls that overlap on the GPU (different streams, or different host threads)
+ * race on it: serialise them.  Inputs, outputs, scales and status codes are those of fp8_attention_bwd. */
+#define FP8_STATIC_SCRATCH_BYTES (32u << 20)
+
+FP8_API int fp8_attention_bwd_static(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const uint8_t *dO8,
+                             const void *O_bf16, const float *LSE, const fp8_attn_scales *sc,
+                             int causal, int B, int N, int Hq, int Hkv, int d,
+                             void *dQ_bf16, void *dK_bf16, void *dV_bf16, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

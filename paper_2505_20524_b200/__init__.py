@@ -6,6 +6,7 @@ attention behind a C ABI (``include/fp8dpa.h``), with a thin Python binding of t
 ``build``    compiles ``csrc/*.cu`` into ``csrc/libfp8dpa.so``
 """
 from . import binding  # noqa: F401
-from .binding import (E4M3, E5M2, Fp8Error, fp8_amax, fp8_attention_bwd, fp8_attention_fwd,  # noqa: F401
+from .binding import (E4M3, E5M2, Fp8Error, fp8_amax, fp8_attention_bwd, fp8_attention_bwd_static,  # noqa: F401
+                      fp8_attention_fwd,
                       fp8_attention_workspace_bytes, fp8_cast, fp8_device_status, fp8_last_error,
                       fp8_linear_dgrad, fp8_linear_fwd, fp8_linear_wgrad, fp8_quantize, fp8_scale)

@@ -21,7 +21,9 @@ _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_cast", "fp8_quantize",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_attention_workspace_bytes",
-           "fp8_attention_fwd", "fp8_attention_bwd"]
+           "fp8_attention_fwd", "fp8_attention_bwd", "fp8_attention_bwd_static"]
+
+STATIC_SCRATCH_BYTES = 32 << 20
 
 STATUS_NAMES = {0: "FP8_OK", -1: "FP8_ERR_NULL", -2: "FP8_ERR_ALIGN", -3: "FP8_ERR_SHAPE", -4: "FP8_ERR_ENUM",
                 -5: "FP8_ERR_WORKSPACE", -6: "FP8_ERR_CUDA", -7: "FP8_ERR_TIMEOUT", -8: "FP8_ERR_ARCH"}
@@ -169,3 +171,15 @@ def fp8_attention_bwd(q8, k8, v8, do8, o, lse, q_inv, k_inv, v_inv, do_inv, soft
                                     C.c_int(d), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(ws),
                                     C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
                                     _stream(stream)))
+
+
+def fp8_attention_bwd_static(q8, k8, v8, do8, o, lse, q_inv, k_inv, v_inv, do_inv, softmax_scale, ds_scale, causal,
+                             dq, dk, dv, ds_amax=None, p_scale=448.0, stream=None):
+    """fp8_attention_bwd for callers that cannot provide scratch: it uses the fixed array inside the library
+    (problems up to STATIC_SCRATCH_BYTES of scratch; calls must not overlap on the GPU)."""
+    B, N, Hq, d = q8.shape
+    Hkv = k8.shape[2]
+    sc = _scales(q_inv, k_inv, v_inv, do_inv, softmax_scale, p_scale, ds_scale, ds_amax)
+    _check(load().fp8_attention_bwd_static(_ptr(q8), _ptr(k8), _ptr(v8), _ptr(do8), _ptr(o), _ptr(lse),
+                                           C.byref(sc), C.c_int(int(causal)), C.c_int(B), C.c_int(N), C.c_int(Hq),
+                                           C.c_int(Hkv), C.c_int(d), _ptr(dq), _ptr(dk), _ptr(dv), _stream(stream)))
