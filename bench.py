@@ -177,6 +177,22 @@ def run_reference(args, cfg):
 
 
 # ---------------------------------------------------------------------------------------------- our arm
+def max_over_ranks(ms_local: float, world: int, device=None) -> float:
+    """Device time of the slowest rank (every rank gets the same number)."""
+    if world <= 1:
+        return float(ms_local)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tflops(world: int, flops_per_step: float, steps: int, ms_total: float) -> float:
+    """Whole-job throughput: every rank runs its own replica of the step (weak scaling)."""
+    return world * flops_per_step * steps / (ms_total / 1e3) / 1e12
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -221,16 +237,13 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
     barrier()
     clocks = sampler.stop()
-    ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms_total = float(ms.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
     status = fp8.fp8_device_status()
     if status != 0:
         raise SystemExit(f"device status {status}: a bounded wait expired inside a kernel")
 
     flops_step = hp.gemm_flops() + hp.attention_flops()
-    value = world * flops_step * args.steps / (ms_total / 1e3) / 1e12
+    value = job_tflops(world, flops_step, args.steps, ms_total)
 
     # ---- dominant kernel: the FP8 GEMM; duration from the events recorded around each launch
     gemm_ms = sum(a.elapsed_time(b) for evs in hp.gemm_events for a, b in evs)
@@ -274,10 +287,7 @@ def run_ours(args, cfg):
     e1.record()
     torch.cuda.synchronize()
     barrier()
-    ms2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(ms2, op=dist.ReduceOp.MAX)
-    e2e_value = world * flops_step * e2e_steps / (float(ms2.item()) / 1e3) / 1e12
+    e2e_value = job_tflops(world, flops_step, e2e_steps, max_over_ranks(e0.elapsed_time(e1), world, dev))
 
     cpu_baseline = None
     if rank == 0 and world == 1:

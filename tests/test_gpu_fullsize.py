@@ -1,0 +1,153 @@
+"""GPU parity at the full workload sizes, in the launch configuration bench.py times (BlockHotPath.step).
+
+The oracle cannot redo these sizes whole, so it computes sampled outputs one by one: output rows/columns of
+each GEMM (each a complete reduction), and for attention the query rows / key rows whose results depend only
+on data the oracle can afford (causality makes the first rows an N = rows problem, and the last key rows
+depend only on the last query rows)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as o
+import paper_2505_20524_b200 as fp8
+from paper_2505_20524_b200 import synth
+from paper_2505_20524_b200.hotpath import BlockHotPath
+from gpu_util import dev, host, scalar, rel_err, BWD_FLOOR, FLIP_EPS
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("log2n,fmts", [(27, (o.E4M3, o.E5M2)), (29, (o.E4M3,))])
+def test_quantize_sweep_sizes_bit_exact(log2n, fmts):
+    n = 1 << log2n
+    x = synth.flat_tensor(n)
+    xd = dev(x)
+    a, s, si = scalar(), scalar(), scalar()
+    ea = o.amax(x)
+    assert float(ea) == 200.0
+    for fmt in fmts:
+        q = torch.empty(n, dtype=torch.uint8, device="cuda")
+        fp8.fp8_quantize(xd, fmt, q, None, a, s, si)
+        es, esi = o.scale(ea, fmt)
+        assert float(a.item()) == float(ea) and float(s.item()) == float(es) and float(si.item()) == float(esi)
+        exp = o.cast(x.reshape(-1, 4096), es, fmt).reshape(-1)
+        assert np.array_equal(host(q), exp)
+        del q
+
+
+def _sample(n, k, seed):
+    """k indices of [0, n): tile edges, the ragged end and seeded picks."""
+    fixed = [0, 1, 127, 128, 255, 256, n // 2 - 1, n // 2, n - 129, n - 128, n - 2, n - 1]
+    rng = np.random.default_rng(seed)
+    idx = sorted(set([i for i in fixed if 0 <= i < n] + rng.integers(0, n, size=k).tolist()))
+    return np.array(idx[:max(k, len(fixed))], dtype=np.int64)
+
+
+@pytest.mark.parametrize("name", ["c3", "c4"])
+def test_block_gemms_sampled(name):
+    cfg = synth.CONFIGS[name]
+    hp = BlockHotPath(cfg, "cuda", with_attention=False)
+    h = hp.generate_host_inputs()
+    hp.allocate()
+    hp.step()
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    for lin in hp.linears:
+        x8, _, _, sx = o.quantize(h["x_" + lin.name], o.E4M3)
+        w8, _, _, sw = o.quantize(h["w_" + lin.name], o.E4M3)
+        dy8, _, _, sdy = o.quantize(h["dy_" + lin.name], o.E5M2)
+        assert np.array_equal(host(lin.x.q), x8) and np.array_equal(host(lin.w.qt), w8.T)
+        assert np.array_equal(host(lin.dy.qt), dy8.T)
+        T, N, K = lin.T, lin.N, lin.K
+        for out, fn, a8, b8, sa, sb, nr, nc in ((lin.y, o.linear_fwd, x8, w8, sx, sw, T, N),
+                                                (lin.dx, o.linear_dgrad, dy8, w8, sdy, sw, T, K),
+                                                (lin.dw, o.linear_wgrad, dy8, x8, sdy, sx, N, K)):
+            rows, cols = _sample(nr, 16, 1), _sample(nc, 48, 2)
+            ref, mag = fn(a8, b8, sa, sb, rows=rows, cols=cols)
+            got = out[torch.from_numpy(rows).cuda()][:, torch.from_numpy(cols).cuda()].float().cpu().numpy()
+            err = rel_err(got.astype(np.float64), ref, mag)
+            assert err <= 2.0 ** -8, (lin.name, fn.__name__, err)
+
+
+def _attention_case(name, kv_heads, head_rows):
+    cfg = synth.CONFIGS[name]
+    hp = BlockHotPath(cfg, "cuda", with_linears=False)
+    h = hp.generate_host_inputs()
+    hp.allocate()
+    a = hp.attn
+    B, N, Hq, Hkv, d = hp.B, hp.N, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    G = Hq // Hkv
+    q8, _, _, qi = o.quantize(h["q"], o.E4M3)
+    k8, _, _, ki = o.quantize(h["k"], o.E4M3)
+    v8, _, _, vi = o.quantize(h["v"], o.E4M3)
+    do8, _, _, doi = o.quantize(h["do"], o.E5M2)
+    lo, hi = (0, head_rows), (N - head_rows, N)
+    kw = dict(causal=True, quant=True, kv_block=128, max_mode=0, q_inv=qi, k_inv=ki, v_inv=vi, do_inv=doi,
+              flip_eps=FLIP_EPS)
+    p = o.attn_params(B, N, Hq, Hkv, d, ds_scale=1.0, **kw)
+    heads = [(b, g * G + j) for (b, g) in kv_heads for j in range(G)]
+    fwd = {}
+    for rng in (lo, hi):
+        fwd[rng] = o.attention_fwd(q8, k8, v8, p, heads=heads, rows=rng, with_slack=True)
+    # a dS scale from the oracle alone: power of two, 4x headroom over the amax seen on the sampled pairs
+    O_or = np.zeros((B, N, Hq, d))
+    L_or = np.zeros((B, Hq, N))
+    for rng in (lo, hi):
+        O_, lse_, _, _ = fwd[rng]
+        for n_, (b, hh) in enumerate(heads):
+            O_or[b, rng[0]:rng[1], hh] = synth.bf16_to_f32(synth.f32_to_bf16(O_[n_].astype(np.float32)))
+            L_or[b, hh, rng[0]:rng[1]] = lse_[n_].astype(np.float32)
+    cal = o.attention_bwd(q8, k8, v8, do8, O_or, L_or, p, kv_heads=kv_heads, q_rows=hi, k_rows=hi)
+    ds_scale = 2.0 ** np.floor(np.log2(57344.0 / (4.0 * cal["amax_dS"])))
+    a["ds_scale"].fill_(float(ds_scale))
+
+    hp.step()                                                 # the timed configuration: quantize + fwd + bwd
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    assert np.array_equal(host(a["q"].q), q8) and np.array_equal(host(a["do"].q), do8)
+    gO = a["o"].float().cpu().numpy().astype(np.float64)
+    gL = a["lse"].cpu().numpy().astype(np.float64)
+    for rng in (lo, hi):
+        O_, lse_, mag_, slack_ = fwd[rng]
+        for n_, (b, hh) in enumerate(heads):
+            e = rel_err(gO[b, rng[0]:rng[1], hh], O_[n_], mag_[n_], slack_[n_])
+            assert e <= 2e-2, ("O", rng, b, hh, e)
+            assert np.max(np.abs(gL[b, hh, rng[0]:rng[1]] - lse_[n_])) <= 1e-3 * max(1.0, np.abs(lse_[n_]).max())
+
+    # backward again on the oracle's O / LSE for the sampled (head, row) ranges, so both sides see equal inputs
+    Ot = a["o"].clone()
+    Lt = a["lse"].clone()
+    for rng in (lo, hi):
+        for (b, hh) in heads:
+            bits = synth.f32_to_bf16(O_or[b, rng[0]:rng[1], hh].astype(np.float32))
+            Ot[b, rng[0]:rng[1], hh] = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
+            Lt[b, hh, rng[0]:rng[1]] = torch.from_numpy(L_or[b, hh, rng[0]:rng[1]].astype(np.float32)).cuda()
+    fp8.fp8_attention_bwd(a["q"].q, a["k"].q, a["v"].q, a["do"].q, Ot, Lt, a["q"].scale_inv, a["k"].scale_inv,
+                          a["v"].scale_inv, a["do"].scale_inv, a["softmax_scale"], a["ds_scale"], True, a["dq"],
+                          a["dk"], a["dv"], a["ws"], ds_amax=a["ds_amax"])
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    p = o.attn_params(B, N, Hq, Hkv, d, ds_scale=float(ds_scale), **kw)
+    first = o.attention_bwd(q8, k8, v8, do8, O_or, L_or, p, kv_heads=kv_heads, q_rows=lo, k_rows=lo)
+    last = o.attention_bwd(q8, k8, v8, do8, O_or, L_or, p, kv_heads=kv_heads, q_rows=hi, k_rows=hi)
+    assert float(a["ds_amax"].item()) >= 0.999 * max(first["amax_dS"], last["amax_dS"])
+    gq = a["dq"].float().cpu().numpy().astype(np.float64)
+    gk = a["dk"].float().cpu().numpy().astype(np.float64)
+    gv = a["dv"].float().cpu().numpy().astype(np.float64)
+    for n_, (b, g) in enumerate(kv_heads):
+        for j in range(G):
+            e = rel_err(gq[b, lo[0]:lo[1], g * G + j], first["dQ"][n_, j], first["mag_dQ"][n_, j],
+                        first["slack_dQ"][n_, j], BWD_FLOOR)
+            assert e <= 3e-2, ("dQ", b, g, j, e)
+        for nm, got in (("dK", gk), ("dV", gv)):
+            e = rel_err(got[b, hi[0]:hi[1], g], last[nm][n_], last["mag_" + nm][n_], last["slack_" + nm][n_],
+                        BWD_FLOOR)
+            assert e <= 3e-2, (nm, b, g, e)
+
+
+def test_attention_8b_block_sampled():
+    _attention_case("c4", kv_heads=[(0, 0), (1, 7)], head_rows=256)
+
+
+def test_attention_long_context_sampled():
+    _attention_case("c5", kv_heads=[(0, 13)], head_rows=1024)
