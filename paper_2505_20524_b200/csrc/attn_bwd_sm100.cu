@@ -64,12 +64,6 @@ struct AttnBwdParams {
     int *status;
 };
 
-__device__ __forceinline__ float ex2_approx(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 __device__ __forceinline__ float e5m2_to_float(uint32_t code)
 {
     // an E5M2 code is the high byte of the binary16 value it denotes

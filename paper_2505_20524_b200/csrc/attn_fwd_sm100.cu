@@ -49,11 +49,36 @@ struct AttnFwdParams {
     int *status;
 };
 
-__device__ __forceinline__ float fast_ex2(float x)
+// One 32-column chunk of a score row -> 32 values of c_P * P~ = 2^(c*S - shift), their sum, and 32 E4M3 codes.
+// MASK: columns beyond `limit` (relative to the chunk start) contribute exactly 0.
+template <bool MASK>
+__device__ __forceinline__ float softmax_chunk(const uint32_t (&v)[32], float c, float neg_shift, int limit,
+                                               uint32_t (&w)[8])
 {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
+    const uint64_t c2 = pack_f32x2(c, c), s2 = pack_f32x2(neg_shift, neg_shift);
+    float e[32];
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        float a, b;
+        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, s2), a, b);
+        e[i] = ex2_approx(a);
+        e[i + 1] = ex2_approx(b);
+        if (MASK) {
+            if (i > limit) e[i] = 0.0f;
+            if (i + 1 > limit) e[i + 1] = 0.0f;
+        }
+    }
+    uint64_t acc0 = pack_f32x2(e[0], e[1]), acc1 = pack_f32x2(e[2], e[3]);
+#pragma unroll
+    for (int i = 4; i < 32; i += 4) {
+        acc0 = add_f32x2(acc0, pack_f32x2(e[i], e[i + 1]));
+        acc1 = add_f32x2(acc1, pack_f32x2(e[i + 2], e[i + 3]));
+    }
+    float s0, s1;
+    unpack_f32x2(add_f32x2(acc0, acc1), s0, s1);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[i] = cvt_f32x4_to_fp8x4<0>(e[4 * i], e[4 * i + 1], e[4 * i + 2], e[4 * i + 3]);
+    return s0 + s1;
 }
 
 template <int D>
@@ -172,65 +197,77 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const bool need_mask = (k0 + A_BN - 1 > q0 && p.causal) || (k0 + A_BN > p.N);
             if (!mbar_wait(s_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
             tc_fence_after();
-            // pass 1: row maximum
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int cc = 0; cc < A_BN; cc += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)cc, v);
+            // pass 1: row maximum (two chunk loads in flight per wait)
+            float mx = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t va[32], vb[32];
+                tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(half * 64), va);
+                tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(half * 64 + 32), vb);
                 tmem_ld_wait();
                 if (need_mask) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (cc + i <= limit) mx = fmaxf(mx, __uint_as_float(v[i]));
+                    for (int i = 0; i < 32; ++i) {
+                        if (half * 64 + i <= limit) mx = fmaxf(mx, __uint_as_float(va[i]));
+                        if (half * 64 + 32 + i <= limit) mx1 = fmaxf(mx1, __uint_as_float(vb[i]));
+                    }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
-                }
-            }
-            const float m_new = fmaxf(m, mx * c);
-            const float alpha = fast_ex2(m - m_new);     // 0 on the first block (m = -inf)
-            // the previous PV must have finished before O is rescaled or P is overwritten
-            if (j > 0) {
-                if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, ctx)) { ok = false; break; }
-                tc_fence_after();
-                if (__any_sync(0xffffffffu, m_new > m)) {
-#pragma unroll 1
-                    for (int cc = 0; cc < D; cc += 32) {
-                        uint32_t v[32];
-                        tmem_ld_32x32b_x32(tmem_o + lane_addr + (uint32_t)cc, v);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
-                        tmem_st_32x32b_x32(tmem_o + lane_addr + (uint32_t)cc, v);
+                    for (int i = 0; i < 32; i += 2) {
+                        mx = fmax3(mx, __uint_as_float(va[i]), __uint_as_float(va[i + 1]));
+                        mx1 = fmax3(mx1, __uint_as_float(vb[i]), __uint_as_float(vb[i + 1]));
                     }
-                    tmem_st_wait();
                 }
             }
-            // pass 2: P~ * c_P = 2^(c*S - m_new + log2 c_P), row sum, E4M3 codes into the operand layout
-            const float shift = m_new - p.log2_p_scale;
-            float lsum = 0.0f;
+            mx = fmaxf(mx, mx1);
+            const float m_new = fmaxf(m, mx * c);
+            const float alpha = ex2_approx(m - m_new);   // 0 on the first block (m = -inf)
+            // S_j was issued after P8_{j-1} V_{j-1} and the tensor pipe completes in issue order, so seeing S_j
+            // means the previous PV is done: O may be rescaled and the P tile overwritten
+            if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
+                const uint64_t a2 = pack_f32x2(alpha, alpha);
 #pragma unroll 1
-            for (int cc = 0; cc < A_BN; cc += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)cc, v);
-                tmem_ld_wait();
-                float e[32];
+                for (int cc = 0; cc < D; cc += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(tmem_o + lane_addr + (uint32_t)cc, v);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    e[i] = fast_ex2(fmaf(__uint_as_float(v[i]), c, -shift));
-                    if (need_mask && cc + i > limit) e[i] = 0.0f;
-                    lsum += e[i];
+                    for (int i = 0; i < 32; i += 2) {
+                        float a, b;
+                        unpack_f32x2(mul_f32x2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), a2), a, b);
+                        v[i] = __float_as_uint(a);
+                        v[i + 1] = __float_as_uint(b);
+                    }
+                    tmem_st_32x32b_x32(tmem_o + lane_addr + (uint32_t)cc, v);
                 }
-                uint32_t w[8];
+                tmem_st_wait();
+            }
+            // pass 2: P~ * c_P = 2^(c*S - m_new + log2 c_P), row sum, E4M3 codes into the operand layout;
+            // the load of chunk q+1 is in flight while chunk q is processed
+            const float neg_shift = p.log2_p_scale - m_new;
+            float lsum = 0.0f;
+            {
+                uint32_t va[32], vb[32], w[8];
+                tmem_ld_32x32b_x32(tmem_s + lane_addr, va);
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    w[i] = (uint32_t)cvt_f32x2_to_fp8x2<0>(e[4 * i], e[4 * i + 1]) |
-                           ((uint32_t)cvt_f32x2_to_fp8x2<0>(e[4 * i + 2], e[4 * i + 3]) << 16);
-                // two 16-byte chunks (keys cc..cc+15, cc+16..cc+31) at their swizzled positions
-                const int ch = cc >> 4;
-                *reinterpret_cast<uint4 *>(prow + (((ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                *reinterpret_cast<uint4 *>(prow + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                for (int q = 0; q < 4; ++q) {
+                    const int cc = q * 32;
+                    tmem_ld_wait();
+                    if (q < 3) {
+                        if (q & 1) tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(cc + 32), va);
+                        else tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(cc + 32), vb);
+                    }
+                    if (q & 1)
+                        lsum += need_mask ? softmax_chunk<true>(vb, c, neg_shift, limit - cc, w)
+                                          : softmax_chunk<false>(vb, c, neg_shift, 0, w);
+                    else
+                        lsum += need_mask ? softmax_chunk<true>(va, c, neg_shift, limit - cc, w)
+                                          : softmax_chunk<false>(va, c, neg_shift, 0, w);
+                    // two 16-byte chunks (keys cc..cc+15, cc+16..cc+31) at their swizzled positions
+                    const int ch = cc >> 4;
+                    *reinterpret_cast<uint4 *>(prow + (((ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(prow + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+                }
             }
             l = l * alpha + lsum;
             m = m_new;
