@@ -158,21 +158,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint64_t dq = umma_desc(sbase + L::Q_OFF, D, 16);
             const uint64_t dp = umma_desc(sbase + L::P_OFF, 128, 16);
             bool ok = mbar_wait(q_full, 0, ctx);
-            for (int j = 0; j < n_kv && ok; ++j) {
+            // S = Q K_j^T: reduction over d in steps of 32 bytes inside the swizzle span
+            auto issue_s = [&](int j) -> bool {
                 const int st = j % A_KV_STAGES;
                 const uint32_t ph = (uint32_t)(j / A_KV_STAGES) & 1u;
-                if (!mbar_wait(kv_full(st), ph, ctx)) { ok = false; break; }
+                if (!mbar_wait(kv_full(st), ph, ctx)) return false;
                 tc_fence_after();
-                const uint32_t sk = sbase + L::KV_OFF + st * L::STAGE_BYTES, sv = sk + L::KV_BYTES;
-                const uint64_t dk = umma_desc(sk, D, 16);
-                // S = Q K^T: reduction over d in steps of 32 bytes inside the swizzle span
+                const uint64_t dk = umma_desc(sbase + L::KV_OFF + st * L::STAGE_BYTES, D, 16);
 #pragma unroll
                 for (int k = 0; k < D / 32; ++k) umma_f8_ss(tmem_s, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
                 umma_commit(s_full);
+                return true;
+            };
+            if (ok) ok = issue_s(0);
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const int st = j % A_KV_STAGES;
+                // P8_j is in shared memory, which also means S_j has been read: the S columns are free
                 if (!mbar_wait(p_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
                 tc_fence_after();
+                // next scores first, so that the softmax of block j+1 can start while P8_j V_j runs
+                if (j + 1 < n_kv && !issue_s(j + 1)) { ok = false; break; }
                 // O += P V: reduction over 128 keys in steps of 32; V advances 32 rows (32*D bytes) per step
-                const uint64_t dv = umma_desc(sv, D, 16);
+                const uint64_t dv = umma_desc(sbase + L::KV_OFF + st * L::STAGE_BYTES + L::KV_BYTES, D, 16);
 #pragma unroll
                 for (int k = 0; k < A_BN / 32; ++k)
                     umma_f8_ss(tmem_o, dp + 2u * k, dv + (uint32_t)((32 * D) >> 4) * k, idesc_o, (j | k) != 0);
@@ -222,8 +229,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             mx = fmaxf(mx, mx1);
             const float m_new = fmaxf(m, mx * c);
             const float alpha = ex2_approx(m - m_new);   // 0 on the first block (m = -inf)
-            // S_j was issued after P8_{j-1} V_{j-1} and the tensor pipe completes in issue order, so seeing S_j
-            // means the previous PV is done: O may be rescaled and the P tile overwritten
+            // the previous PV (issued after S_j) must be done before O is rescaled or the P tile overwritten
+            if (j > 0) {
+                if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, ctx)) { ok = false; break; }
+                tc_fence_after();
+            }
             if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
                 const uint64_t a2 = pack_f32x2(alpha, alpha);
 #pragma unroll 1
