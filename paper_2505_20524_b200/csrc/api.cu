@@ -143,6 +143,28 @@ int make_tmap_3d_u8(CUtensorMap *map, const void *base, uint64_t d0_cols, uint64
     return FP8_OK;
 }
 
+// Rank-3 map over a [B, N, C] binary32 tensor without swizzle (used for bulk reduce-add of FP32 tiles).
+int make_tmap_3d_f32(CUtensorMap *map, const void *base, uint64_t d0_cols, uint64_t d1_rows, uint64_t d2_batch,
+                     uint32_t box_cols, uint32_t box_rows)
+{
+    int rc = load_encoder();
+    if (rc != FP8_OK) return rc;
+    cuuint64_t dims[3] = {d0_cols, d1_rows, d2_batch};
+    cuuint64_t strides[2] = {d0_cols * 4, d0_cols * d1_rows * 4};
+    cuuint32_t box[3] = {box_cols, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled (rank 3, f32) failed (CUresult %d) dims=%llu,%llu,%llu box=%u,%u", (int)r,
+                  (unsigned long long)d0_cols, (unsigned long long)d1_rows, (unsigned long long)d2_batch, box_cols,
+                  box_rows);
+        return FP8_ERR_CUDA;
+    }
+    return FP8_OK;
+}
+
 }  // namespace fp8dpa
 
 extern "C" const char *fp8_last_error(void) { return fp8dpa::g_err; }

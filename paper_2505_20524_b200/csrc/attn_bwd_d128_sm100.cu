@@ -1,0 +1,507 @@
+// FP8 attention backward for head_dim 128: software-pipelined, transposed formulation.
+//
+// One CTA per (128-key tile, KV head, batch) keeps K_j, V_j in shared memory and dK_j, dV_j in TMEM (256
+// columns).  It walks over 64-query sub-tiles t (and the query heads of the group).  With rows = keys:
+//   S^T  = K  Q_t^T   [128 x 64]     dP^T = V dO_t^T   [128 x 64]          (64 TMEM columns each)
+//   P~^T = 2^(c S^T - lse2_q),  P8^T = E4M3,  dS8^T = E5M2( P~^T o (a dP^T - db_q) )   (256 threads)
+//   dV  += P8^T dO_t      dK += dS8^T Q_t      dQ_t^T = K^T dS8^T  [128(d) x 64]  (64 TMEM columns)
+// The other 256 TMEM columns are four 64-column slots: S ping-pong (2), dP (1), dQ^T (1), so the scores of
+// sub-tile t+1 are in TMEM before the threads finish sub-tile t, and dP_{t+1}, dQ_t, dV_t, dK_t run on the
+// tensor pipe while the threads work on t+1.  dQ^T tiles leave through shared memory and one bulk
+// reduce-add (binary32 add in L2) per sub-tile into the FP32 accumulator.
+//
+// Warps: 0 = TMA producer, 1 = MMA issuer, 2-9 = element-wise (two threads per key row, 32 query columns
+// each), 10-13 = dQ drain.  Every wait is bounded.
+#include <cuda_fp16.h>
+#include <math.h>
+
+#include "common.cuh"
+
+namespace fp8dpa {
+
+namespace bwd128 {
+
+constexpr int D = 128;
+constexpr int KT = 128;            // keys per CTA
+constexpr int QT = 64;             // queries per sub-tile
+constexpr int STAGES = 3;          // (Q, dO, lse2, db) stages
+constexpr int THREADS = 14 * 32;
+constexpr int EW_WARPS = 8, DRAIN_WARPS = 4;
+constexpr int TMEM_COLS = 512;
+
+struct Smem {
+    static constexpr int K_OFF = 0;
+    static constexpr int V_OFF = K_OFF + KT * D;
+    static constexpr int QDO_OFF = V_OFF + KT * D;
+    static constexpr int Q_BYTES = QT * D;                       // 8 KB
+    static constexpr int VEC_BYTES = QT * 4;                     // 256 B
+    static constexpr int STAGE_BYTES = 2 * Q_BYTES + 2 * 1024;   // Q, dO, lse2 (padded to 1 KB), db (1 KB)
+    static constexpr int STAGE_TX = 2 * Q_BYTES + 2 * VEC_BYTES;
+    static constexpr int PDS_OFF = QDO_OFF + STAGES * STAGE_BYTES;
+    static constexpr int PDS_TILE = KT * QT;                     // 8 KB: [128 key rows x 64 B]
+    static constexpr int PDS_BUF = 2 * PDS_TILE;                 // P8^T then dS8^T
+    static constexpr int DQ_OFF = PDS_OFF + 2 * PDS_BUF;
+    static constexpr int DQ_BYTES = QT * D * 4;                  // 32 KB: [64 q x 128 d] FP32
+    static constexpr int BAR_OFF = DQ_OFF + DQ_BYTES;
+    // kv_full, qdo_full[3], qdo_empty[3], s_full[2], dp_full, pds_full, pds_free[2], dq_full, dq_empty, all_done
+    static constexpr int N_BARS = 1 + 2 * STAGES + 2 + 1 + 1 + 2 + 1 + 1 + 1;
+    static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
+    static constexpr int DYN_BYTES = TOTAL + 1024;
+};
+// TMEM columns
+constexpr uint32_t T_S0 = 0, T_S1 = 64, T_DP = 128, T_DQ = 192, T_DV = 256, T_DK = 384;
+
+struct Params {
+    const float *lse2;     // [B,Hq,Npad]  LSE*log2(e) - log2(c_P); +inf in the padding
+    const float *db;       // [B,Hq,Npad]  D * ds_scale / c_P; 0 in the padding
+    uint16_t *dK, *dV;     // [B,N,Hkv,D] BF16
+    const float *q_inv, *k_inv, *v_inv, *do_inv, *ds_scale;
+    float *ds_amax;
+    float softmax_scale, p_scale;
+    int causal;
+    int B, N, Npad, Hq, Hkv;
+    int *status;
+};
+
+__device__ __forceinline__ float e5m2_to_f32(uint32_t code)
+{
+    return __half2float(__ushort_as_half((unsigned short)(code << 8)));
+}
+
+// ---------------------------------------------------------------- prep
+// One warp per (b, i, h) with i < Npad: D_i = do_inv * sum_d dec(dO8) * O, then
+// lse2 = LSE*log2e - log2(c_P), db = D * ds_scale / c_P; rows i >= N get (+inf, 0); the dQ accumulator row
+// is zeroed.
+__global__ void __launch_bounds__(256) prep_kernel(const uint8_t *__restrict__ dO8, const uint16_t *__restrict__ O,
+                                                   const float *__restrict__ LSE, const float *__restrict__ do_inv,
+                                                   const float *__restrict__ ds_scale, float p_scale,
+                                                   float log2_p_scale, float *__restrict__ lse2,
+                                                   float *__restrict__ db, float *__restrict__ dQacc, int B, int N,
+                                                   int Npad, int Hq)
+{
+    const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (b*Npad + i)*Hq + h
+    const int lane = threadIdx.x & 31;
+    if (w >= (long)B * Npad * Hq) return;
+    const int h = (int)(w % Hq);
+    const long bi = w / Hq;
+    const int i = (int)(bi % Npad), b = (int)(bi / Npad);
+    const size_t vi = ((size_t)b * Hq + h) * Npad + i;
+    if (i >= N) {
+        if (lane == 0) {
+            lse2[vi] = INFINITY;
+            db[vi] = 0.0f;
+        }
+        return;
+    }
+    const size_t row = ((size_t)b * N + i) * Hq + h;
+    const uint32_t c4 = *reinterpret_cast<const uint32_t *>(dO8 + row * D + lane * 4);
+    const uint2 o4 = *reinterpret_cast<const uint2 *>(O + row * D + lane * 4);
+    float acc = e5m2_to_f32(c4 & 0xFF) * bf16_lo(o4.x) + e5m2_to_f32((c4 >> 8) & 0xFF) * bf16_hi(o4.x) +
+                e5m2_to_f32((c4 >> 16) & 0xFF) * bf16_lo(o4.y) + e5m2_to_f32(c4 >> 24) * bf16_hi(o4.y);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    *reinterpret_cast<float4 *>(dQacc + row * D + lane * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (lane == 0) {
+        lse2[vi] = __ldg(LSE + ((size_t)b * Hq + h) * N + i) * 1.4426950408889634f - log2_p_scale;
+        db[vi] = acc * __ldg(do_inv) * __ldg(ds_scale) / p_scale;
+    }
+}
+
+__global__ void __launch_bounds__(256) finish_kernel(const float4 *__restrict__ acc, uint2 *__restrict__ dQ, size_t n4,
+                                                     const float *__restrict__ k_inv,
+                                                     const float *__restrict__ ds_scale, float softmax_scale)
+{
+    const float f = softmax_scale * __ldg(k_inv) / __ldg(ds_scale);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        const float4 v = acc[i];
+        dQ[i] = make_uint2(pack_bf16x2(v.x * f, v.y * f), pack_bf16x2(v.z * f, v.w * f));
+    }
+}
+
+// ---------------------------------------------------------------- main
+__global__ void __launch_bounds__(THREADS, 1)
+main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+            const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+            const __grid_constant__ CUtensorMap tm_dq, const Params p)
+{
+    using L = Smem;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::BAR_OFF;
+    const uint32_t kv_full = bar0;
+    auto qdo_full = [&](int s) { return bar0 + 8u * (1 + s); };
+    auto qdo_empty = [&](int s) { return bar0 + 8u * (1 + STAGES + s); };
+    auto s_full = [&](int s) { return bar0 + 8u * (1 + 2 * STAGES + s); };
+    const uint32_t dp_full = bar0 + 8u * (3 + 2 * STAGES);
+    const uint32_t pds_full = dp_full + 8u;
+    auto pds_free = [&](int s) { return dp_full + 16u + 8u * s; };
+    const uint32_t dq_full = dp_full + 32u, dq_empty = dp_full + 40u, all_done = dp_full + 48u;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFF + L::N_BARS * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k_tile = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    const int G = p.Hq / p.Hkv;
+    const int k0 = k_tile * KT;
+    const int n_sub = p.Npad / QT;
+    const int i_first = p.causal ? (k0 / QT) : 0;         // first 64-query sub-tile that sees these keys
+    const int per_head = n_sub - i_first;
+    const int n_iter = per_head * G;
+    auto head_of = [&](int t) { return g * G + t / per_head; };
+    auto q0_of = [&](int t) { return (i_first + t % per_head) * QT; };
+
+    if (threadIdx.x == 0) {
+        mbar_init(kv_full, 1);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(qdo_full(s), 1);
+            mbar_init(qdo_empty(s), 1);
+        }
+        mbar_init(s_full(0), 1);
+        mbar_init(s_full(1), 1);
+        mbar_init(dp_full, 1);
+        mbar_init(pds_full, EW_WARPS);
+        mbar_init(pds_free(0), 1);
+        mbar_init(pds_free(1), 1);
+        mbar_init(dq_full, 1);
+        mbar_init(dq_empty, DRAIN_WARPS);
+        mbar_init(all_done, 1);
+        *abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_do);
+        tma_prefetch_desc(&tm_dq);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const WaitCtx ctx{p.status, abort_flag};
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            mbar_expect_tx(kv_full, 2 * KT * D);
+            tma_load_3d(sbase + L::K_OFF, &tm_k, kv_full, g * D, k0, b);
+            tma_load_3d(sbase + L::V_OFF, &tm_v, kv_full, g * D, k0, b);
+            for (int t = 0; t < n_iter; ++t) {
+                const int st = t % STAGES;
+                const uint32_t ph = (uint32_t)(t / STAGES) & 1u;
+                const int h = head_of(t), q0 = q0_of(t);
+                if (!mbar_wait(qdo_empty(st), ph ^ 1u, ctx)) break;
+                const uint32_t sq = sbase + L::QDO_OFF + st * L::STAGE_BYTES, sdo = sq + L::Q_BYTES;
+                const uint32_t sl = sdo + L::Q_BYTES, sd = sl + 1024;
+                const size_t vi = ((size_t)b * p.Hq + h) * p.Npad + q0;
+                mbar_expect_tx(qdo_full(st), L::STAGE_TX);
+                tma_load_3d(sq, &tm_q, qdo_full(st), h * D, q0, b);
+                tma_load_3d(sdo, &tm_do, qdo_full(st), h * D, q0, b);
+                bulk_load_1d(sl, p.lse2 + vi, L::VEC_BYTES, qdo_full(st));
+                bulk_load_1d(sd, p.db + vi, L::VEC_BYTES, qdo_full(st));
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            constexpr uint32_t E4 = 0, E5 = 1;
+            constexpr uint32_t id_s = umma_idesc_f8(E4, E4, 128, QT, 0, 0);      // K (K-major) x Q (K-major)
+            constexpr uint32_t id_dp = umma_idesc_f8(E4, E5, 128, QT, 0, 0);     // V x dO
+            constexpr uint32_t id_dv = umma_idesc_f8(E4, E5, 128, D, 0, 1);      // P8^T (K-major) x dO (MN)
+            constexpr uint32_t id_dk = umma_idesc_f8(E5, E4, 128, D, 0, 1);      // dS8^T (K-major) x Q (MN)
+            constexpr uint32_t id_dq = umma_idesc_f8(E4, E5, 128, QT, 1, 1);     // K^T (MN) x dS8^T (MN)
+            const uint64_t d_k = umma_desc(sbase + L::K_OFF, 128, 16);
+            const uint64_t d_v = umma_desc(sbase + L::V_OFF, 128, 16);
+            constexpr uint32_t ROWS32_128 = (32 * 128) >> 4;   // 32 rows of a 128-byte-row tile
+            constexpr uint32_t ROWS32_64 = (32 * 64) >> 4;     // 32 rows of a 64-byte-row tile
+            auto stage_q = [&](int t) { return sbase + L::QDO_OFF + (t % STAGES) * L::STAGE_BYTES; };
+            auto wait_stage = [&](int t) {
+                return mbar_wait(qdo_full(t % STAGES), (uint32_t)(t / STAGES) & 1u, ctx);
+            };
+            auto issue_s = [&](int t) {     // S^T_t = K Q_t^T into slot t & 1
+                const uint64_t d_q = umma_desc(stage_q(t), 128, 16);
+                const uint32_t dst = tmem_base + ((t & 1) ? T_S1 : T_S0);
+#pragma unroll
+                for (int k = 0; k < D / 32; ++k) umma_f8_ss(dst, d_k + 2u * k, d_q + 2u * k, id_s, k != 0);
+                umma_commit(s_full(t & 1));
+            };
+            auto issue_dp = [&](int t) {    // dP^T_t = V dO_t^T
+                const uint64_t d_do = umma_desc(stage_q(t) + L::Q_BYTES, 128, 16);
+#pragma unroll
+                for (int k = 0; k < D / 32; ++k) umma_f8_ss(tmem_base + T_DP, d_v + 2u * k, d_do + 2u * k, id_dp, k != 0);
+                umma_commit(dp_full);
+            };
+            bool ok = mbar_wait(kv_full, 0, ctx);
+            if (ok) ok = wait_stage(0);
+            if (ok) {
+                tc_fence_after();
+                issue_s(0);
+                issue_dp(0);
+            }
+            if (ok && n_iter > 1) {
+                ok = wait_stage(1);
+                if (ok) {
+                    tc_fence_after();
+                    issue_s(1);
+                }
+            }
+            for (int t = 0; t < n_iter && ok; ++t) {
+                const int pb = t & 1;
+                // P8^T_t and dS8^T_t are in shared memory; S_t and dP_t have been read
+                if (!mbar_wait(pds_full, (uint32_t)t & 1u, ctx)) { ok = false; break; }
+                tc_fence_after();
+                if (t + 1 < n_iter) issue_dp(t + 1);      // its stage was waited for when S_{t+1} was issued
+                const uint32_t sp = sbase + L::PDS_OFF + pb * L::PDS_BUF, sds = sp + L::PDS_TILE;
+                const uint64_t d_p = umma_desc(sp, 64, 16), d_ds = umma_desc(sds, 64, 16);
+                const uint64_t d_q = umma_desc(stage_q(t), 128, 16), d_do = umma_desc(stage_q(t) + L::Q_BYTES, 128, 16);
+                // dQ^T_t = K^T dS8^T_t: reduction over the 128 keys, 32 rows of either tile per step
+                if (t > 0 && !mbar_wait(dq_empty, (uint32_t)(t - 1) & 1u, ctx)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < KT / 32; ++k)
+                    umma_f8_ss(tmem_base + T_DQ, d_k + ROWS32_128 * k, d_ds + ROWS32_64 * k, id_dq, k != 0);
+                umma_commit(dq_full);
+                if (t + 2 < n_iter) {
+                    if (!wait_stage(t + 2)) { ok = false; break; }
+                    tc_fence_after();
+                    issue_s(t + 2);                        // slot t & 1: S_t has been read
+                }
+                // dV += P8^T dO_t, dK += dS8^T Q_t: reduction over the 64 queries, 32 per step
+#pragma unroll
+                for (int k = 0; k < QT / 32; ++k)
+                    umma_f8_ss(tmem_base + T_DV, d_p + 2u * k, d_do + ROWS32_128 * k, id_dv, (t | k) != 0);
+#pragma unroll
+                for (int k = 0; k < QT / 32; ++k)
+                    umma_f8_ss(tmem_base + T_DK, d_ds + 2u * k, d_q + ROWS32_128 * k, id_dk, (t | k) != 0);
+                umma_commit(qdo_empty(t % STAGES));
+                umma_commit(pds_free(pb));
+            }
+            if (ok) umma_commit(all_done);
+        }
+    } else if (warp < 2 + EW_WARPS) {
+        // ------------------------------------------------------------ element-wise: P8^T, dS8^T
+        const int ew = warp - 2;
+        const int quad = warp & 3;                      // TMEM lanes 32*quad..: rows (keys) of this warp
+        const int half = ew >> 2;                       // query columns [32*half, 32*half + 32)
+        const int r = quad * 32 + lane;                 // key row inside the tile
+        const int key = k0 + r;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const float c = p.softmax_scale * __ldg(p.q_inv) * __ldg(p.k_inv) * 1.4426950408889634f;
+        const float dss = __ldg(p.ds_scale);
+        const float a_dp = __ldg(p.do_inv) * __ldg(p.v_inv) * dss / p.p_scale;
+        const uint64_t c2 = pack_f32x2(c, c), a2 = pack_f32x2(a_dp, a_dp);
+        const int sw = (r >> 1) & 3;                    // 64-byte swizzle: 16-byte chunk index ^ ((row >> 1) & 3)
+        const int ch0 = half * 2;
+        float amax = 0.0f;
+        bool ok = true;
+        for (int t = 0; t < n_iter; ++t) {
+            const int q0 = q0_of(t), st = t % STAGES, pb = t & 1;
+            const int qbase = q0 + half * 32;           // first query column of this thread
+            // valid iff key <= query (causal) and key < N; queries >= N carry lse2 = +inf
+            const bool need_mask = (p.causal && q0 < k0 + KT - 1) || (k0 + KT > p.N);
+            const int first_ok = (key < p.N) ? (p.causal ? key - qbase : 0) : 64;   // columns >= first_ok are valid
+            const float *vec = reinterpret_cast<const float *>(smem + L::QDO_OFF + st * L::STAGE_BYTES + 2 * L::Q_BYTES);
+            const float *lse2 = vec + half * 32, *dbv = vec + 256 + half * 32;
+            if (!mbar_wait_warp(qdo_full(st), (uint32_t)(t / STAGES) & 1u, ctx)) { ok = false; break; }
+            if (!mbar_wait_warp(s_full(pb), (uint32_t)(t >> 1) & 1u, ctx)) { ok = false; break; }
+            tc_fence_after();
+            uint32_t sv[32];
+            tmem_ld_32x32b_x32(tmem_base + (pb ? T_S1 : T_S0) + lane_addr + (uint32_t)(half * 32), sv);
+            tmem_ld_wait();
+            float pe[32];
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+                const float2 l2 = *reinterpret_cast<const float2 *>(lse2 + i);
+                float x0, x1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2,
+                                       pack_f32x2(-l2.x, -l2.y)), x0, x1);
+                pe[i] = ex2_approx(x0);                 // c_P * P
+                pe[i + 1] = ex2_approx(x1);
+            }
+            if (need_mask) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i < first_ok) pe[i] = 0.0f;
+            }
+            uint32_t w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w[i] = cvt_f32x4_to_fp8x4<0>(pe[4 * i], pe[4 * i + 1], pe[4 * i + 2], pe[4 * i + 3]);
+            // the P8/dS8 buffer pb was last read by the MMAs of sub-tile t-2
+            if (t >= 2 && !mbar_wait_warp(pds_free(pb), (uint32_t)((t >> 1) - 1) & 1u, ctx)) { ok = false; break; }
+            uint8_t *prow = smem + L::PDS_OFF + pb * L::PDS_BUF + r * 64;
+            uint8_t *dsrow = prow + L::PDS_TILE;
+            *reinterpret_cast<uint4 *>(prow + ((ch0 ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4 *>(prow + (((ch0 + 1) ^ sw) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+            if (!mbar_wait_warp(dp_full, (uint32_t)t & 1u, ctx)) { ok = false; break; }
+            tc_fence_after();
+            tmem_ld_32x32b_x32(tmem_base + T_DP + lane_addr + (uint32_t)(half * 32), sv);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+                const float2 d2 = *reinterpret_cast<const float2 *>(dbv + i);
+                float y0, y1;
+                unpack_f32x2(mul_f32x2(pack_f32x2(pe[i], pe[i + 1]),
+                                       fma_f32x2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), a2,
+                                                 pack_f32x2(-d2.x, -d2.y))), y0, y1);
+                pe[i] = y0;                              // ds_scale * dS
+                pe[i + 1] = y1;
+                amax = fmaxf(fmaxf(amax, fabsf(y0)), fabsf(y1));
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w[i] = cvt_f32x4_to_fp8x4<1>(pe[4 * i], pe[4 * i + 1], pe[4 * i + 2], pe[4 * i + 3]);
+            *reinterpret_cast<uint4 *>(dsrow + ((ch0 ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4 *>(dsrow + (((ch0 + 1) ^ sw) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+            tc_fence_before();
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pds_full);
+        }
+        // ---- epilogue: warps with half == 0 write dV, the others dK (TMEM lane = key)
+        if (ok && mbar_wait_warp(all_done, 0, ctx)) {
+            tc_fence_after();
+            const float f = half == 0 ? __ldg(p.do_inv) / p.p_scale : p.softmax_scale * __ldg(p.q_inv) / dss;
+            uint16_t *dst = (half == 0 ? p.dV : p.dK) + (((size_t)b * p.N + key) * p.Hkv + g) * D;
+            const uint32_t tcol = half == 0 ? T_DV : T_DK;
+#pragma unroll 1
+            for (int cc = 0; cc < D; cc += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32b_x32(tmem_base + tcol + lane_addr + (uint32_t)cc, v);
+                tmem_ld_wait();
+                if (key < p.N) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 o;
+                        o.x = pack_bf16x2(__uint_as_float(v[i]) * f, __uint_as_float(v[i + 1]) * f);
+                        o.y = pack_bf16x2(__uint_as_float(v[i + 2]) * f, __uint_as_float(v[i + 3]) * f);
+                        o.z = pack_bf16x2(__uint_as_float(v[i + 4]) * f, __uint_as_float(v[i + 5]) * f);
+                        o.w = pack_bf16x2(__uint_as_float(v[i + 6]) * f, __uint_as_float(v[i + 7]) * f);
+                        *reinterpret_cast<uint4 *>(dst + cc + i) = o;
+                    }
+                }
+            }
+            if (p.ds_amax) {
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+                // the kernel tracked ds_scale * |dS|; non-negative floats order like unsigned integers
+                if (lane == 0) atomicMax(reinterpret_cast<unsigned int *>(p.ds_amax), __float_as_uint(amax / dss));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ dQ drain (4 warps)
+        const int quad = warp & 3;                      // TMEM lane = d index
+        const int dd = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        float *dq_s = reinterpret_cast<float *>(smem + L::DQ_OFF);
+        const bool issuer = (warp == 2 + EW_WARPS) && lane == 0;
+        for (int t = 0; t < n_iter; ++t) {
+            const int h = head_of(t), q0 = q0_of(t);
+            const bool got = mbar_wait_warp(dq_full, (uint32_t)t & 1u, ctx);
+            uint32_t va[32], vb[32];
+            if (got) {
+                tc_fence_after();
+                tmem_ld_32x32b_x32(tmem_base + T_DQ + lane_addr, va);
+                tmem_ld_32x32b_x32(tmem_base + T_DQ + lane_addr + 32u, vb);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(dq_empty);   // the dQ^T slot may be overwritten
+            }
+            // the previous bulk reduce must have finished reading the staging tile
+            if (issuer) bulk_wait_group_read0();
+            if (named_barrier_or(1, DRAIN_WARPS * 32, !got)) break;   // all four warps leave together
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                dq_s[i * D + dd] = __uint_as_float(va[i]);
+                dq_s[(i + 32) * D + dd] = __uint_as_float(vb[i]);
+            }
+            fence_proxy_async_smem();
+            named_barrier_sync(1, DRAIN_WARPS * 32);
+            if (issuer) {
+                tma_reduce_add_3d(&tm_dq, sbase + L::DQ_OFF, h * D, q0, b);
+                bulk_commit_group();
+            }
+        }
+        if (issuer) bulk_wait_group0();                 // all reduce-adds complete before the CTA exits
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace bwd128
+
+size_t attn_bwd_d128_ws_bytes(int B, int N, int Hq)
+{
+    const size_t Npad = ((size_t)N + bwd128::QT - 1) / bwd128::QT * bwd128::QT;
+    const size_t vec = (((size_t)B * Hq * Npad * sizeof(float)) + 255) & ~(size_t)255;
+    return 2 * vec + (size_t)B * N * Hq * bwd128::D * sizeof(float);
+}
+
+int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const uint8_t *dO8,
+                         const uint16_t *O, const float *LSE, const fp8_attn_scales *sc, int causal, int B, int N,
+                         int Hq, int Hkv, uint16_t *dQ, uint16_t *dK, uint16_t *dV, void *ws, int *status,
+                         cudaStream_t st)
+{
+    using namespace bwd128;
+    const int Npad = (N + QT - 1) / QT * QT;
+    const size_t vec = (((size_t)B * Hq * Npad * sizeof(float)) + 255) & ~(size_t)255;
+    float *lse2 = static_cast<float *>(ws);
+    float *db = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + vec);
+    float *dQacc = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + 2 * vec);
+    CUtensorMap tq, tk, tv, tdo, tdq;
+    int rc = make_tmap_3d_u8(&tq, Q8, (uint64_t)Hq * D, (uint64_t)N, (uint64_t)B, D, QT);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tk, K8, (uint64_t)Hkv * D, (uint64_t)N, (uint64_t)B, D, KT);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tv, V8, (uint64_t)Hkv * D, (uint64_t)N, (uint64_t)B, D, KT);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tdo, dO8, (uint64_t)Hq * D, (uint64_t)N, (uint64_t)B, D, QT);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_f32(&tdq, dQacc, (uint64_t)Hq * D, (uint64_t)N, (uint64_t)B, D, QT);
+    if (rc != FP8_OK) return rc;
+    if (sc->ds_amax) FP8_CUDA_CHECK(cudaMemsetAsync(sc->ds_amax, 0, sizeof(float), st));
+    const float log2_p = log2f(sc->p_scale);
+    const long warps = (long)B * Npad * Hq;
+    prep_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(dO8, O, LSE, sc->do_inv, sc->ds_scale, sc->p_scale, log2_p,
+                                                            lse2, db, dQacc, B, N, Npad, Hq);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    Params p;
+    p.lse2 = lse2; p.db = db;
+    p.dK = dK; p.dV = dV;
+    p.q_inv = sc->q_inv; p.k_inv = sc->k_inv; p.v_inv = sc->v_inv; p.do_inv = sc->do_inv;
+    p.ds_scale = sc->ds_scale;
+    p.ds_amax = sc->ds_amax;
+    p.softmax_scale = sc->softmax_scale;
+    p.p_scale = sc->p_scale;
+    p.causal = causal ? 1 : 0;
+    p.B = B; p.N = N; p.Npad = Npad; p.Hq = Hq; p.Hkv = Hkv;
+    p.status = status;
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::DYN_BYTES));
+    dim3 grid((unsigned)((N + KT - 1) / KT), (unsigned)Hkv, (unsigned)B);
+    main_kernel<<<grid, THREADS, Smem::DYN_BYTES, st>>>(tq, tk, tv, tdo, tdq, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    const size_t n4 = (size_t)B * N * Hq * D / 4;
+    size_t blocks = (n4 + 255) / 256;
+    const size_t cap = (size_t)sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    finish_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4 *>(dQacc),
+                                                   reinterpret_cast<uint2 *>(dQ), n4, sc->k_inv, sc->ds_scale,
+                                                   sc->softmax_scale);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+}  // namespace fp8dpa

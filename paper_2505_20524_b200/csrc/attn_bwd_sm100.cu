@@ -4,7 +4,8 @@
 //   dV_j = sum_i P8_ij dO_i                     dP_ij = dO_i . V_j
 //   dS   = P o (dP - D)   -> E5M2 (dS8)         dQ_i  = s sum_j dS8_ij K_j       dK_j = s sum_i dS8_ij Q_i
 //
-// Three launches on the caller's stream:
+// This file holds the simple (un-pipelined) form, used for head_dim 64; head_dim 128 runs the pipelined kernel
+// of attn_bwd_d128_sm100.cu.  Three launches on the caller's stream:
 //   1. prep:    D (FP32) from dO8 and O, and zeroing of the FP32 dQ accumulator (both live in the workspace)
 //   2. main:    one CTA per (128-key tile, KV head, batch); it keeps K_j, V_j in shared memory, walks over
 //               the query tiles (and the query heads of the group) that see these keys, and per tile pair runs
@@ -21,6 +22,11 @@
 
 namespace fp8dpa {
 
+size_t attn_bwd_d128_ws_bytes(int B, int N, int Hq);
+int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const uint8_t *dO8,
+                         const uint16_t *O, const float *LSE, const fp8_attn_scales *sc, int causal, int B, int N,
+                         int Hq, int Hkv, uint16_t *dQ, uint16_t *dK, uint16_t *dV, void *ws, int *status,
+                         cudaStream_t st);
 int validate_attn(const char *who, const void *q, const void *k, const void *v, const fp8_attn_scales *sc, int B, int N,
                   int Hq, int Hkv, int d);
 
@@ -371,6 +377,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
 static size_t bwd_ws_bytes(int B, int N, int Hq, int d)
 {
+    if (d == 128) return attn_bwd_d128_ws_bytes(B, N, Hq);
     const size_t acc = (size_t)B * N * Hq * d * sizeof(float);
     const size_t dsum = (((size_t)B * Hq * N * sizeof(float)) + 255) & ~(size_t)255;
     return acc + dsum;
@@ -464,6 +471,7 @@ extern "C" int fp8_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uin
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint16_t *O = static_cast<const uint16_t *>(O_bf16);
     uint16_t *dQ = static_cast<uint16_t *>(dQ_bf16);
-    return d == 128 ? launch_attn_bwd<128>(Q8, K8, V8, dO8, O, dQ, p, dsum, st)
-                    : launch_attn_bwd<64>(Q8, K8, V8, dO8, O, dQ, p, dsum, st);
+    if (d == 128)
+        return launch_attn_bwd_d128(Q8, K8, V8, dO8, O, LSE, sc, causal, B, N, Hq, Hkv, dQ, p.dK, p.dV, ws, p.status, st);
+    return launch_attn_bwd<64>(Q8, K8, V8, dO8, O, dQ, p, dsum, st);
 }
