@@ -24,7 +24,7 @@ namespace bwd128 {
 constexpr int D = 128;
 constexpr int KT = 128;            // keys per CTA
 constexpr int QT = 64;             // queries per sub-tile
-constexpr int STAGES = 3;          // (Q, dO, lse2, db) stages
+constexpr int STAGES = 6;          // (Q, dO, lse2, db) stages: a TMA load takes several sub-tile periods to land
 constexpr int THREADS = 14 * 32;
 constexpr int EW_WARPS = 8, DRAIN_WARPS = 4;
 constexpr int TMEM_COLS = 512;
