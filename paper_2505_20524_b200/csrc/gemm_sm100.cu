@@ -37,6 +37,25 @@ struct GemmParams {
     int *status;
 };
 
+// Tile order: bands of G_BAND tiles along the longer output dimension; inside a band the index along the
+// shorter dimension advances slowest.  The CTAs that run at the same time then share one band of one operand
+// (a few MB) and a handful of panels of the other, and both stay in L2 however long the matrix is.
+constexpr int G_BAND = 16;
+__device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
+{
+    const int per_band = G_BAND * n_short;
+    const int band = tile / per_band, within = tile - band * per_band;
+    const int len = min(G_BAND, n_long - band * G_BAND);     // the last band may be short
+    i_short = within / len;
+    i_long = band * G_BAND + (within - i_short * len);
+}
+template <int BN>
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int &tm, int &tn)
+{
+    if (tiles_m * G_BM >= tiles_n * BN) band_coords(tile, tiles_m, tiles_n, tm, tn);
+    else band_coords(tile, tiles_n, tiles_m, tn, tm);
+}
+
 template <int BN>
 __global__ void __launch_bounds__(G_THREADS, 1)
 gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
@@ -91,7 +110,9 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % tiles_m) * G_BM, n0 = (tile / tiles_m) * BN;
+                int tm, tn;
+                tile_coords<BN>(tile, tiles_m, tiles_n, tm, tn);
+                const int m0 = tm * G_BM, n0 = tn * BN;
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctx)) { ok = false; break; }
                     const uint32_t sa = sbase + stage * L::STAGE_BYTES, sb = sa + L::A_BYTES;
@@ -140,7 +161,9 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int m0 = (tile % tiles_m) * G_BM, n0 = (tile / tiles_m) * BN;
+            int tm, tn;
+            tile_coords<BN>(tile, tiles_m, tiles_n, tm, tn);
+            const int m0 = tm * G_BM, n0 = tn * BN;
             if (!mbar_wait(tfull_bar(buf), acc_phase, ctx)) { ok = false; break; }
             tc_fence_after();
             const int row = m0 + quad * 32 + lane;
