@@ -81,6 +81,16 @@ FP8_API int fp8_cast(const void *x_bf16, size_t rows, size_t cols, const float *
 FP8_API int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fmt, uint8_t *out, uint8_t *out_t,
                  float *amax, float *scale, float *scale_inv, void *stream);
 
+/* Delayed scaling (Appendix E): H holds the last `len` abs-max values of one tensor (the paper trains with
+ * len = 1024, margin 0); rho = FP8Max / (2^margin * max H); after a step, H <- {amax} u H minus its oldest
+ * entry, "to use in the next iteration".  This call does that update on the device: history[*head] = *amax_new,
+ * *head = (*head + 1) % len, then *scale / *scale_inv from the maximum of the updated history (guards as in
+ * fp8_scale; an all-zero history gives 1).  history: `len` floats, zero-initialised by the caller; head: device
+ * int, initially 0, the position of the oldest entry.  A training step then needs a single pass per tensor:
+ * fp8_cast(x, scale, ..., amax_out = amax_new) followed by fp8_scale_update for the next step. */
+FP8_API int fp8_scale_update(float *history, int len, int *head, const float *amax_new, int fmt, int margin,
+                     float *scale, float *scale_inv, void *stream);
+
 /* ---- linear layers --------------------------------------------------------------------------------
  * Appendix E: GEMM(X,Y) = 1/(rho_X rho_Y) * FP8GEMM(FP8cast(rho_X X), FP8cast(rho_Y Y)), BF16 result;
  * Table "Comparison between FP8 methods": Linear_W(X) = XW for the FFN, QKV and output projections.

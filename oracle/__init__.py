@@ -123,6 +123,20 @@ def scale(amax_value, fmt: int, margin: int = 0):
     return np.float32(s.value), np.float32(si.value)
 
 
+def scale_update(history: np.ndarray, head: int, amax_new, fmt: int, margin: int = 0):
+    """Delayed scaling: push amax_new into the FIFO `history` (float32, modified in place; `head` = position of
+    the oldest entry) and return (new_head, scale, scale_inv) computed from the updated history."""
+    assert history.dtype == np.float32 and history.flags["C_CONTIGUOUS"]
+    h = C.c_int(int(head))
+    s = C.c_float()
+    si = C.c_float()
+    f = _L().oracle_scale_update
+    f.restype = None
+    f(_p(history), C.c_int(history.size), C.byref(h), C.c_float(float(amax_new)), C.c_int(fmt), C.c_int(margin),
+      C.byref(s), C.byref(si))
+    return h.value, np.float32(s.value), np.float32(si.value)
+
+
 def cast(x_bf16: np.ndarray, scale_value, fmt: int, transpose: bool = False):
     x = _c(x_bf16, np.uint16)
     if x.ndim == 1:

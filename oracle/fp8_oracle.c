@@ -142,6 +142,25 @@ void oracle_scale(float amax, int fmt, int margin, float *scale, float *scale_in
 }
 
 /* ------------------------------------------------------------------------------------------------
+ * Delayed scaling (Appendix E): H = {h_1..h_l} holds the last l abs-max values of a tensor,
+ * rho = FP8Max / (2^m max H), and after a step H <- {amax(X)} u {h_t}_{t=2..l}, "to use in the next
+ * iteration".  Reading of the set notation: a FIFO, the dropped h_1 is the oldest entry; the new scale is
+ * computed from the history *after* the insertion and is the one the next step casts with.  `head` is
+ * the position of the oldest entry.  Entries that were never written are 0 and an all-zero history
+ * gives scale 1 (same guard as oracle_scale).
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_scale_update(float *history, int len, int *head, float amax_new, int fmt, int margin,
+                         float *scale, float *scale_inv)
+{
+    history[*head] = amax_new;
+    *head = (*head + 1) % len;
+    float mx = 0.0f;
+    for (int i = 0; i < len; ++i)
+        if (history[i] > mx || isnan(history[i])) mx = history[i];
+    oracle_scale(mx, fmt, margin, scale, scale_inv);
+}
+
+/* ------------------------------------------------------------------------------------------------
  * cast: FP8cast(rho * X) of Appendix E.  Reading of the precision (paper silent): the BF16 value is
  * widened exactly to binary32, multiplied by the scale in binary32 (round-to-nearest), and the product
  * is rounded once more to FP8 by oracle_fp8_encode.  out_t, if not NULL, is the same codes laid out

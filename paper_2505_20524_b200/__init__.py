@@ -9,4 +9,5 @@ from . import binding  # noqa: F401
 from .binding import (E4M3, E5M2, Fp8Error, fp8_amax, fp8_attention_bwd, fp8_attention_bwd_static,  # noqa: F401
                       fp8_attention_fwd,
                       fp8_attention_workspace_bytes, fp8_cast, fp8_device_status, fp8_last_error,
-                      fp8_linear_dgrad, fp8_linear_fwd, fp8_linear_wgrad, fp8_quantize, fp8_scale)
+                      fp8_linear_dgrad, fp8_linear_fwd, fp8_linear_wgrad, fp8_quantize, fp8_scale,
+                      fp8_scale_update)

@@ -19,7 +19,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
-SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_cast", "fp8_quantize",
+SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
+           "fp8_quantize",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
@@ -89,6 +90,13 @@ def fp8_amax(x, amax, stream=None):
 
 def fp8_scale(amax, fmt, margin, scale, scale_inv, stream=None):
     _check(load().fp8_scale(_ptr(amax), C.c_int(fmt), C.c_int(margin), _ptr(scale), _ptr(scale_inv), _stream(stream)))
+
+
+def fp8_scale_update(history, head, amax_new, fmt, margin, scale, scale_inv, stream=None):
+    """Delayed scaling: push *amax_new into the FIFO `history` (float32 CUDA tensor, `head` an int32 CUDA scalar)
+    and recompute scale / scale_inv from the updated history."""
+    _check(load().fp8_scale_update(_ptr(history), C.c_int(history.numel()), _ptr(head), _ptr(amax_new), C.c_int(fmt),
+                                   C.c_int(margin), _ptr(scale), _ptr(scale_inv), _stream(stream)))
 
 
 def _rows_cols(x):

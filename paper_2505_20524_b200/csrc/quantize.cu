@@ -69,6 +69,46 @@ __global__ void scale_kernel(const float *__restrict__ amax, float fp8_max, int 
     *scale_inv = __fdiv_rn(1.0f, s);
 }
 
+// ---------------------------------------------------------------- delayed scaling: history ring update
+// One CTA: insert the new amax at the position of the oldest entry, then scale = FP8Max / (2^m max H).
+__global__ void __launch_bounds__(256) scale_update_kernel(float *__restrict__ history, int len, int *__restrict__ head,
+                                                           const float *__restrict__ amax_new, float fp8_max,
+                                                           int margin, float *__restrict__ scale,
+                                                           float *__restrict__ scale_inv)
+{
+    __shared__ float warp_max[8];
+    __shared__ int s_nan;
+    if (threadIdx.x == 0) {
+        const int h = *head;
+        history[h] = *amax_new;
+        *head = (h + 1) % len;
+        s_nan = 0;
+    }
+    __syncthreads();
+    float m = 0.0f;
+    for (int i = threadIdx.x; i < len; i += blockDim.x) {
+        const float v = history[i];
+        if (v != v) s_nan = 1;
+        m = fmaxf(m, v);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) m = fmaxf(m, warp_max[w]);
+        float s;
+        if (s_nan || !(m > 0.0f) || isinf(m)) {
+            s = 1.0f;
+        } else {
+            s = __fmul_rn(__fdiv_rn(fp8_max, m), ldexpf(1.0f, -margin));
+            if (isinf(s)) s = FLT_MAX;
+        }
+        *scale = s;
+        *scale_inv = __fdiv_rn(1.0f, s);
+    }
+}
+
 // ---------------------------------------------------------------- cast
 // 8 BF16 (one 16-byte word) -> 8 FP8 codes (two 32-bit words); each product is one binary32 multiply.
 template <int FMT>
@@ -343,4 +383,27 @@ extern "C" int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fm
     scale_kernel<<<1, 1, 0, st>>>(amax, fmt == FP8_E4M3 ? 448.0f : 57344.0f, 0, scale, scale_inv);
     FP8_CUDA_CHECK(cudaGetLastError());
     return do_cast(x_bf16, rows, cols, scale, fmt, out, out_t, nullptr, st);
+}
+
+extern "C" int fp8_scale_update(float *history, int len, int *head, const float *amax_new, int fmt, int margin,
+                                float *scale, float *scale_inv, void *stream)
+{
+    if (!history || !head || !amax_new || !scale || !scale_inv) {
+        set_error("fp8_scale_update: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if (fmt != FP8_E4M3 && fmt != FP8_E5M2) {
+        set_error("fp8_scale_update: fmt %d is not FP8_E4M3 / FP8_E5M2", fmt);
+        return FP8_ERR_ENUM;
+    }
+    if (len <= 0 || len > (1 << 20) || margin < -64 || margin > 64) {
+        set_error("fp8_scale_update: len %d must be in [1, 2^20] and margin %d in [-64, 64]", len, margin);
+        return FP8_ERR_SHAPE;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    scale_update_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        history, len, head, amax_new, fmt == FP8_E4M3 ? 448.0f : 57344.0f, margin, scale, scale_inv);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
 }

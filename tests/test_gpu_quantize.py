@@ -108,3 +108,41 @@ def test_argument_validation_returns_errors_not_faults():
         fp8.fp8_cast(x.view(torch.int16).flatten()[1:].view(torch.bfloat16), scalar(1.0), 0, out)
     assert e.value.status == -2
     assert fp8.fp8_device_status() == 0
+
+
+def test_delayed_scaling_ring_matches_oracle():
+    """fp8_scale_update against the oracle over more steps than the history holds (l = 1024 as in Appendix E)."""
+    l, steps = 1024, 2200
+    rng = np.random.default_rng(3)
+    amaxes = np.abs(rng.normal(size=steps)).astype(np.float32) * np.where(rng.random(steps) < 0.01, 40.0, 1.0).astype(np.float32)
+    hist_d = torch.zeros(l, dtype=torch.float32, device="cuda")
+    head_d = torch.zeros(1, dtype=torch.int32, device="cuda")
+    a_d = torch.from_numpy(amaxes).cuda()
+    s, si = scalar(), scalar()
+    hist = np.zeros(l, dtype=np.float32)
+    head = 0
+    for t in range(steps):
+        fp8.fp8_scale_update(hist_d, head_d, a_d[t:t + 1], o.E4M3, 0, s, si)
+        head, es, esi = o.scale_update(hist, head, amaxes[t], o.E4M3)
+        if t % 97 == 0 or t == steps - 1:
+            assert bits(s) == int(es.view(np.uint32)) and bits(si) == int(esi.view(np.uint32)), t
+            assert int(head_d.item()) == head
+            assert np.array_equal(hist_d.cpu().numpy(), hist)
+
+
+def test_delayed_scaling_step_is_one_pass():
+    """cast with last step's scale + fused amax, then the ring update: equals the oracle's chain bit for bit."""
+    l = 16
+    hist_d = torch.zeros(l, dtype=torch.float32, device="cuda")
+    head_d = torch.zeros(1, dtype=torch.int32, device="cuda")
+    s, si, a = scalar(1.0), scalar(1.0), scalar()
+    hist = np.zeros(l, dtype=np.float32)
+    head, es = 0, np.float32(1.0)
+    for step in range(5):
+        x = synth.normal_bf16((256, 128), 10 + step, 1, 1.0 + step)
+        out = torch.empty(x.shape, dtype=torch.uint8, device="cuda")
+        fp8.fp8_cast(dev(x), s, o.E4M3, out, None, a)                 # scale from the history so far
+        assert np.array_equal(host(out), o.cast(x, es, o.E4M3))
+        fp8.fp8_scale_update(hist_d, head_d, a, o.E4M3, 0, s, si)
+        head, es, _ = o.scale_update(hist, head, o.amax(x), o.E4M3)
+        assert bits(s) == int(es.view(np.uint32))

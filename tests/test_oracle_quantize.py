@@ -115,3 +115,23 @@ def test_larger_outlier_quantises_the_rest_less_accurately(fmt):
             assert ncodes <= prev_codes
             assert err >= prev_err * 0.999
         prev_codes, prev_err = ncodes, err
+
+
+def test_delayed_scaling_history_is_a_fifo_of_the_last_l_amaxes():
+    """Appendix E: rho = FP8Max / (2^m max H), H <- {amax} u {h_t}_{t=2..l} (the oldest entry leaves)."""
+    l = 5
+    hist = np.zeros(l, dtype=np.float32)
+    head = 0
+    seq = [3.0, 1.0, 7.0, 2.0, 2.0, 1.0, 1.0, 0.5, 0.5, 0.5, 0.25, 0.25]
+    for t, a in enumerate(seq):
+        head, s, si = o.scale_update(hist, head, a, o.E4M3)
+        window = seq[max(0, t + 1 - l):t + 1]                     # the last l values, independent bookkeeping
+        es, esi = o.scale(np.float32(max(window)), o.E4M3)
+        assert (s, si) == (es, esi), (t, window)
+        assert sorted(hist[hist > 0].tolist()) == sorted(window)
+        assert head == (t + 1) % l
+    # 7.0 dominated from step 2 until it left the window at step 7
+    assert o.scale_update(np.zeros(4, dtype=np.float32), 0, 0.0, o.E5M2)[1:] == (1.0, 1.0)   # empty history
+    h2 = np.zeros(3, dtype=np.float32)
+    _, s2, _ = o.scale_update(h2, 0, 2.0, o.E5M2, margin=1)
+    assert s2 == np.float32(57344.0 / 2.0 / 2.0)
