@@ -1,0 +1,279 @@
+// FP8 GEMM on CTA pairs (tcgen05.mma.cta_group::2): C[M,N] (+)= sa_inv*sb_inv * A[M,K] . B[N,K]^T
+//
+// Two CTAs of a cluster (ranks 0 and 1, neighbouring SMs) compute one 256 x 256 tile.  Each CTA loads its own
+// 128 rows of A and its own 128 rows of B per stage (32 KB instead of the 48 KB a lone CTA needs for a
+// 128 x 256 tile: the main loop is bound by the L2 -> shared-memory feed, so this is where the time goes); the
+// MMA of shape 256 x 256 x 32 is issued by one thread of the even CTA, reads both CTAs' shared memory and writes
+// 128 accumulator rows into each CTA's TMEM.  Accumulators are double-buffered (2 x 256 columns), so the epilogue
+// of tile i overlaps the main loop of tile i+1.
+//
+// Barrier protocol (per CTA, same offsets in both):
+//   full[s]   used in the even CTA only: its producer posts the byte count of both CTAs' loads; every load of the
+//             pair credits the even CTA's barrier
+//   empty[s]  one arrival per phase: the multicast commit of the MMAs that read stage s (lands in both CTAs)
+//   tfull[b]  multicast commit after the last MMA of a tile (lands in both CTAs)
+//   tempty[b] used in the even CTA only: 8 arrivals (4 epilogue warps of each CTA; the odd CTA arrives remotely)
+// Every wait is bounded; a cluster barrier before exit keeps either CTA alive while its peer can still reach it.
+#include "common.cuh"
+
+namespace fp8dpa {
+
+namespace g2 {
+
+constexpr int BM = 128;            // rows per CTA (256 per pair)
+constexpr int BN = 256;            // columns per pair; each CTA stages 128 rows of B
+constexpr int BK = 128;
+constexpr int STAGES = 6;
+constexpr int THREADS = 192;
+constexpr int A_BYTES = BM * BK, B_BYTES = (BN / 2) * BK;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;              // 32 KB per CTA
+constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+constexpr int N_BARS = 2 * STAGES + 4;
+constexpr int DYN_BYTES = BAR_OFFSET + N_BARS * 8 + 16 + 1024;
+constexpr uint32_t TMEM_COLS = 512;
+
+struct Params {
+    void *out;
+    const float *sa_inv, *sb_inv;
+    int M, N, K;
+    int out_is_fp32, accumulate;
+    uint32_t idesc;
+    int num_pairs;
+    int *status;
+};
+
+constexpr int BAND = 16;
+__device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
+{
+    const int per_band = BAND * n_short;
+    const int band = tile / per_band, within = tile - band * per_band;
+    const int len = min(BAND, n_long - band * BAND);
+    i_short = within / len;
+    i_long = band * BAND + (within - i_short * len);
+}
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int &tm, int &tn)
+{
+    if (tiles_m >= tiles_n) band_coords(tile, tiles_m, tiles_n, tm, tn);
+    else band_coords(tile, tiles_n, tiles_m, tn, tm);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_base = sbase + BAR_OFFSET;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+    auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + BAR_OFFSET + N_BARS * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();            // 0 = even CTA (issues the MMAs), 1 = its peer
+    const int pair = blockIdx.x >> 1;
+    const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
+    const int k_blocks = (p.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 8);
+        }
+        *abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                  // both CTAs' barriers exist before anyone signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const WaitCtx ctx{p.status, abort_flag};
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (both CTAs)
+        if (elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs) {
+                int tm, tn;
+                tile_coords(tile, tiles_m, tiles_n, tm, tn);
+                const int m0 = tm * 2 * BM + (int)rank * BM, n0 = tn * BN + (int)rank * (BN / 2);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctx)) { ok = false; break; }
+                    const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+                    tma_load_2d_pair(sa, &tmap_a, full_bar(stage), kb * BK, m0);
+                    tma_load_2d_pair(sb, &tmap_b, full_bar(stage), kb * BK, n0);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (even CTA only)
+        if (rank == 0 && elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs, ++it) {
+                const int buf = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), acc_phase ^ 1u, ctx)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, ctx)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    const uint64_t da = umma_desc_k_sw128(sa), db = umma_desc_k_sw128(sb);
+#pragma unroll
+                    for (int k = 0; k < BK / 32; ++k)
+                        umma_f8_ss_pair(tmem_d, da + 2u * k, db + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit_pair(empty_bar(stage), 3);      // frees the stage in both CTAs
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit_pair(tfull_bar(buf), 3);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5 of both CTAs)
+        const int quad = warp & 3;
+        const float descale = __ldg(p.sa_inv) * __ldg(p.sb_inv);
+        bool ok = true;
+        int it = 0;
+        for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs, ++it) {
+            const int buf = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            int tm, tn;
+            tile_coords(tile, tiles_m, tiles_n, tm, tn);
+            const int m0 = tm * 2 * BM + (int)rank * BM, n0 = tn * BN;
+            if (!mbar_wait_warp(tfull_bar(buf), acc_phase, ctx)) { ok = false; break; }
+            tc_fence_after();
+            const int row = m0 + quad * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN);
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(taddr + (uint32_t)c, r);
+                tmem_ld_wait();
+                const int col = n0 + c;
+                if (row < p.M && col < p.N) {
+                    const int ncols = min(32, p.N - col);
+                    if (p.out_is_fp32) {
+                        float *dst = static_cast<float *>(p.out) + (size_t)row * p.N + col;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            if (j < ncols) {
+                                float4 v = make_float4(__uint_as_float(r[j]) * descale, __uint_as_float(r[j + 1]) * descale,
+                                                       __uint_as_float(r[j + 2]) * descale,
+                                                       __uint_as_float(r[j + 3]) * descale);
+                                if (p.accumulate) {
+                                    const float4 o = *reinterpret_cast<const float4 *>(dst + j);
+                                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                                }
+                                *reinterpret_cast<float4 *>(dst + j) = v;
+                            }
+                        }
+                    } else {
+                        uint16_t *dst = static_cast<uint16_t *>(p.out) + (size_t)row * p.N + col;
+#pragma unroll
+                        for (int j = 0; j < 32; j += 8) {
+                            if (j < ncols) {
+                                float v[8];
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(r[j + q]) * descale;
+                                if (p.accumulate) {
+                                    const uint4 o = *reinterpret_cast<const uint4 *>(dst + j);
+                                    v[0] += bf16_lo(o.x); v[1] += bf16_hi(o.x); v[2] += bf16_lo(o.y); v[3] += bf16_hi(o.y);
+                                    v[4] += bf16_lo(o.z); v[5] += bf16_hi(o.z); v[6] += bf16_lo(o.w); v[7] += bf16_hi(o.w);
+                                }
+                                *reinterpret_cast<uint4 *>(dst + j) =
+                                    make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                                               pack_bf16x2(v[6], v[7]));
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_pair_leader(tempty_bar(buf));   // the even CTA's barrier, from either CTA
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+        __syncthreads();
+    }
+    cluster_sync_all();             // neither CTA leaves (or frees TMEM) while its peer may still touch it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace g2
+
+// Returns FP8_OK after launching, or a negative status.  `max_pairs` = 0 lets the runtime size the grid.
+int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, void *out,
+                     int out_is_fp32, int accumulate, int M, int N, int K, uint32_t idesc, int *status,
+                     cudaStream_t st)
+{
+    using namespace g2;
+    CUtensorMap ta, tb;
+    int rc = make_tmap_2d_u8(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM, BK);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_2d_u8(&tb, b, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
+    if (rc != FP8_OK) return rc;
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
+    static int max_clusters = -1;
+    if (max_clusters < 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * 74, 1, 1);
+        cfg.blockDim = dim3(THREADS, 1, 1);
+        cfg.dynamicSmemBytes = DYN_BYTES;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            n = sm_count() / 2;
+        }
+        max_clusters = n;
+    }
+    const int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
+    Params p;
+    p.out = out; p.sa_inv = sa_inv; p.sb_inv = sb_inv;
+    p.M = M; p.N = N; p.K = K;
+    p.out_is_fp32 = out_is_fp32; p.accumulate = accumulate;
+    p.idesc = idesc;
+    p.num_pairs = tiles < max_clusters ? tiles : max_clusters;
+    p.status = status;
+    kernel<<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+}  // namespace fp8dpa

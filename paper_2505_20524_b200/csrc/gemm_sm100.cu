@@ -8,6 +8,8 @@
 //             (MT = 1: two accumulator buffers, so the epilogue of tile i overlaps the main loop of tile i+1)
 //   warps 2.. epilogue (4 per accumulator): tcgen05.ld -> descale -> BF16/FP32 -> 16-byte global stores
 // Every wait is bounded; on expiry the CTA records FP8_ERR_TIMEOUT and drains.
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace fp8dpa {
@@ -250,6 +252,17 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     }
 }
 
+int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, void *out,
+                     int out_is_fp32, int accumulate, int M, int N, int K, uint32_t idesc, int *status,
+                     cudaStream_t st);
+
+// FP8DPA_GEMM=1cta|2cta forces one kernel family (for A/B measurements); default: chosen per shape.
+static int gemm_family_override()
+{
+    const char *e = getenv("FP8DPA_GEMM");
+    return !e ? 0 : (e[0] == '1' ? 1 : (e[0] == '2' ? 2 : 0));
+}
+
 static int validate_gemm(const char *who, const void *a, const void *b, const float *sa, const float *sb, void *out,
                          int M, int N, int K)
 {
@@ -304,6 +317,17 @@ int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int
     p.accumulate = accumulate;
     p.status = device_status_ptr();
     if (!p.status) return FP8_ERR_CUDA;
+    // CTA pairs (256 x 256 per pair, 32 KB per CTA and stage) whenever the matrix is large enough to give every
+    // pair at least two tiles: same wave quantisation as 128 x 256 tiles on single CTAs, two thirds of the L2
+    // traffic, and the epilogue still overlaps the next main loop.
+    {
+        const long pair_tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
+        const int fam = gemm_family_override();
+        if (fam != 1 && M >= 256 && N >= 256 && (fam == 2 || pair_tiles >= sm_count())) {
+            return launch_gemm_2cta(a, b, sa_inv, sb_inv, out, out_is_fp32, accumulate, M, N, K,
+                                    umma_idesc_f8(fmt_a, fmt_b, 256, 256), p.status, st);
+        }
+    }
     // Tile choice.  The 256 x 256 tile needs 2/3 of the L2 traffic of 128 x 256 but cannot overlap its epilogue
     // with the next main loop (its two accumulators fill TMEM), so it only wins for long reductions (measured:
     // +3% at K = 8192, -15% at K = 2048) and when it still fills the SMs in whole waves.

@@ -66,6 +66,31 @@ def test_three_gemms_match_oracle(T, N, K, out_dtype):
         assert max(e1, e2, e3) <= 2.0 ** -8          # what the arithmetic should give: one BF16 rounding
 
 
+@pytest.mark.parametrize("family", ["1cta", "2cta"])
+@pytest.mark.parametrize("T,N,K", [(256, 256, 128), (400, 528, 144), (1024, 768, 2064), (272, 1040, 256)])
+def test_both_kernel_families_on_ragged_shapes(family, T, N, K, monkeypatch):
+    """FP8DPA_GEMM forces the single-CTA or the CTA-pair kernel; both must agree with the oracle on tiles that
+    hang over the matrix edge (the pair kernel is otherwise only chosen for large matrices)."""
+    monkeypatch.setenv("FP8DPA_GEMM", family)
+    x = synth.normal_bf16((T, K), T + N, 0, 1.0, [1, K - 2], 50.0)
+    w = synth.normal_bf16((N, K), T + N, 1, synth.W_STD)
+    dy = synth.normal_bf16((T, N), T + N, 2, synth.GRAD_STD)
+    for out_dtype, tol in ((torch.bfloat16, 2.0 ** -8), (torch.float32, TOL_FP32)):
+        (y, dx, dw), (x8, w8, dy8, sx, sw, sdy) = run_three(x, w, dy, out_dtype)
+        check(y, *o.linear_fwd(x8, w8, sx, sw), tol)
+        check(dx, *o.linear_dgrad(dy8, w8, sdy, sw), tol)
+        check(dw, *o.linear_wgrad(dy8, x8, sdy, sx), tol)
+    if family == "2cta":                       # accumulate path of the pair kernel's epilogue
+        prev = np.random.default_rng(1).normal(size=(N, K)).astype(np.float32) * 1e-3
+        dwa = dev(prev.copy())
+        x8d, x8t, _, _, sxd = gpu_quantize(x, o.E4M3, True)
+        dy8d, dy8t, _, _, sdyd = gpu_quantize(dy, o.E5M2, True)
+        fp8.fp8_linear_wgrad(dy8t, x8t, sdyd, sxd, dwa, accumulate=True)
+        ref, mag = o.linear_wgrad(host(dy8d), host(x8d), float(sdyd.item()), float(sxd.item()),
+                                  prev=prev.astype(np.float64))
+        assert rel_err(host(dwa).astype(np.float64), ref, mag + np.abs(prev)) <= TOL_FP32
+
+
 def test_wgrad_accumulate_fp32():
     T, N, K = 256, 128, 384
     x = synth.normal_bf16((T, K), 1, 0, 1.0)
