@@ -292,7 +292,7 @@ def run_ours(args, cfg):
     cpu_baseline = None
     if rank == 0 and world == 1:
         f, s, desc, cores = oracle_sample(cfg, reps=1)
-        reps = int(min(8, max(1, round(12.0 / max(s, 1e-3)))))      # aim at 10-30 s of CPU work
+        reps = int(min(16, max(1, round(15.0 / max(s, 1e-3)))))      # aim at 10-30 s of CPU work
         if reps > 1:
             f, s, desc, cores = oracle_sample(cfg, reps=reps)
         cpu_baseline = {"value": f / s / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",

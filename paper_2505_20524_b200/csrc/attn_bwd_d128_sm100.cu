@@ -72,7 +72,7 @@ __device__ __forceinline__ float e5m2_to_f32(uint32_t code)
 // One warp per (b, i, h) with i < Npad: D_i = do_inv * sum_d dec(dO8) * O, then
 // lse2 = LSE*log2e - log2(c_P), db = D * ds_scale / c_P; rows i >= N get (+inf, 0); the dQ accumulator row
 // is zeroed.
-__global__ void __launch_bounds__(256) prep_kernel(const uint8_t *__restrict__ dO8, const uint16_t *__restrict__ O,
+__global__ void __launch_bounds__(256) attn_bwd_d128_prep_kernel(const uint8_t *__restrict__ dO8, const uint16_t *__restrict__ O,
                                                    const float *__restrict__ LSE, const float *__restrict__ do_inv,
                                                    const float *__restrict__ ds_scale, float p_scale,
                                                    float log2_p_scale, float *__restrict__ lse2,
@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(256) prep_kernel(const uint8_t *__restrict__ d
     }
 }
 
-__global__ void __launch_bounds__(256) finish_kernel(const float4 *__restrict__ acc, uint2 *__restrict__ dQ, size_t n4,
+__global__ void __launch_bounds__(256) attn_bwd_d128_finish_kernel(const float4 *__restrict__ acc, uint2 *__restrict__ dQ, size_t n4,
                                                      const float *__restrict__ k_inv,
                                                      const float *__restrict__ ds_scale, float softmax_scale)
 {
@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(256) finish_kernel(const float4 *__restrict__ 
 
 // ---------------------------------------------------------------- main
 __global__ void __launch_bounds__(THREADS, 1)
-main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
             const __grid_constant__ CUtensorMap tm_dq, const Params p)
 {
@@ -141,7 +141,9 @@ main_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CU
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int k_tile = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    // KV head fastest: the CTAs that run at the same time then add their dQ tiles into different rows of a small,
+    // L2-resident band of the accumulator instead of contending for the same rows
+    const int g = blockIdx.x, k_tile = blockIdx.y, b = blockIdx.z;
     const int G = p.Hq / p.Hkv;
     const int k0 = k_tile * KT;
     const int n_sub = p.Npad / QT;
@@ -475,7 +477,7 @@ int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8
     if (sc->ds_amax) FP8_CUDA_CHECK(cudaMemsetAsync(sc->ds_amax, 0, sizeof(float), st));
     const float log2_p = log2f(sc->p_scale);
     const long warps = (long)B * Npad * Hq;
-    prep_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(dO8, O, LSE, sc->do_inv, sc->ds_scale, sc->p_scale, log2_p,
+    attn_bwd_d128_prep_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(dO8, O, LSE, sc->do_inv, sc->ds_scale, sc->p_scale, log2_p,
                                                             lse2, db, dQacc, B, N, Npad, Hq);
     FP8_CUDA_CHECK(cudaGetLastError());
     Params p;
@@ -489,15 +491,15 @@ int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8
     p.causal = causal ? 1 : 0;
     p.B = B; p.N = N; p.Npad = Npad; p.Hq = Hq; p.Hkv = Hkv;
     p.status = status;
-    FP8_CUDA_CHECK(cudaFuncSetAttribute(main_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::DYN_BYTES));
-    dim3 grid((unsigned)((N + KT - 1) / KT), (unsigned)Hkv, (unsigned)B);
-    main_kernel<<<grid, THREADS, Smem::DYN_BYTES, st>>>(tq, tk, tv, tdo, tdq, p);
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_d128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::DYN_BYTES));
+    dim3 grid((unsigned)Hkv, (unsigned)((N + KT - 1) / KT), (unsigned)B);
+    attn_bwd_d128_kernel<<<grid, THREADS, Smem::DYN_BYTES, st>>>(tq, tk, tv, tdo, tdq, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     const size_t n4 = (size_t)B * N * Hq * D / 4;
     size_t blocks = (n4 + 255) / 256;
     const size_t cap = (size_t)sm_count() * 8;
     if (blocks > cap) blocks = cap;
-    finish_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4 *>(dQacc),
+    attn_bwd_d128_finish_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4 *>(dQacc),
                                                    reinterpret_cast<uint2 *>(dQ), n4, sc->k_inv, sc->ds_scale,
                                                    sc->softmax_scale);
     FP8_CUDA_CHECK(cudaGetLastError());

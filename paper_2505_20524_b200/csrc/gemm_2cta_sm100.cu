@@ -58,7 +58,7 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
-kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p)
+gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -244,7 +244,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     if (rc != FP8_OK) return rc;
     rc = make_tmap_2d_u8(&tb, b, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
     if (rc != FP8_OK) return rc;
-    FP8_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
     static int max_clusters = -1;
     if (max_clusters < 0) {
         cudaLaunchConfig_t cfg = {};
@@ -257,7 +257,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_fp8_pair_kernel, &cfg) != cudaSuccess || n <= 0) {
             (void)cudaGetLastError();
             n = sm_count() / 2;
         }
@@ -271,7 +271,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     p.idesc = idesc;
     p.num_pairs = tiles < max_clusters ? tiles : max_clusters;
     p.status = status;
-    kernel<<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
+    gemm_fp8_pair_kernel<<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }
