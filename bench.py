@@ -254,7 +254,7 @@ def run_ours(args, cfg):
     roofline = None
     if gemm_tflops is not None:
         roofline = {
-            "bound": "tensor", "kernel": "gemm_fp8_kernel", "achieved": gemm_tflops, "peak": fp8_peak,
+            "bound": "tensor", "kernel": "gemm_fp8_pair_kernel", "achieved": gemm_tflops, "peak": fp8_peak,
             "unit": "TFLOP/s", "frac": gemm_tflops / fp8_peak,
             "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name),
             "peak_source": f"2 x bf16_tflops_sustained ({peaks['source']})",
@@ -326,9 +326,9 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) per GEMM launch from the ncu capture summarised under profiles/ (null until one
-# exists for the workload).
-GEMM_DRAM_BYTES_PER_LAUNCH = {}
+# DRAM bytes (read + write) per GEMM launch, averaged over the 12 launches of one step, from the single-pass ncu
+# capture summarised in profiles/gemm_fp8_pair_kernel.md (null for workloads without a capture).
+GEMM_DRAM_BYTES_PER_LAUNCH = {"c4": 416.15e6}
 
 
 def main():
