@@ -91,6 +91,21 @@ FP8_API int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fmt, 
 FP8_API int fp8_scale_update(float *history, int len, int *head, const float *amax_new, int fmt, int margin,
                      float *scale, float *scale_inv, void *stream);
 
+/* Gated activation fused with the cast (Appendix B: FFN with activation phi; SwiGLU in the Llama-style
+ * workloads).  gate_up is the [T, 2F] BF16 output of the fused first FFN projection, gate = columns [0,F),
+ * up = columns [F,2F).  h = silu(gate) * up is formed in FP32, rounded to BF16 (never written to memory), and
+ * then treated exactly like the input of fp8_cast: out[t,f] = sat_rne_fmt(float(h) * *scale), out_t the same
+ * codes as [F,T] (nullable), *amax_out = amax(h) (nullable).  out and out_t may both be NULL when only the amax
+ * is wanted (first pass of just-in-time scaling).  F % 16 == 0, T % 16 == 0 when out_t is given.
+ * silu uses expf, so a code can differ from a double-precision evaluation where h lies within an ulp of a
+ * rounding boundary. */
+FP8_API int fp8_swiglu_cast(const void *gate_up_bf16, size_t T, size_t F, const float *scale, int fmt,
+                    uint8_t *out, uint8_t *out_t, float *amax_out, void *stream);
+
+/* Kurtosis monitor (Section 4): *out = mean over rows of mu[x^4] / mu[x^2]^2 of a [rows, cols] BF16 tensor
+ * (un-centred; rows are token vectors).  *out is overwritten.  cols % 8 == 0. */
+FP8_API int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *out, void *stream);
+
 /* ---- linear layers --------------------------------------------------------------------------------
  * Appendix E: GEMM(X,Y) = 1/(rho_X rho_Y) * FP8GEMM(FP8cast(rho_X X), FP8cast(rho_Y Y)), BF16 result;
  * Table "Comparison between FP8 methods": Linear_W(X) = XW for the FFN, QKV and output projections.

@@ -137,6 +137,26 @@ def scale_update(history: np.ndarray, head: int, amax_new, fmt: int, margin: int
     return h.value, np.float32(s.value), np.float32(si.value)
 
 
+def kurtosis(x_bf16: np.ndarray) -> float:
+    """Mean over rows of mu[x^4] / mu[x^2]^2 (un-centred), x = rows of a [rows, cols] BF16 tensor."""
+    x = _c(x_bf16, np.uint16)
+    x2 = x.reshape(-1, x.shape[-1])
+    f = _L().oracle_kurtosis_bf16
+    f.restype = C.c_double
+    return float(f(_p(x2), C.c_size_t(x2.shape[0]), C.c_size_t(x2.shape[1])))
+
+
+def swiglu(gate_up_bf16: np.ndarray) -> np.ndarray:
+    """h = silu(gate) * up as BF16 bits; gate / up are the first / second half of the last axis."""
+    x = _c(gate_up_bf16, np.uint16)
+    T, F2 = x.shape
+    out = np.empty((T, F2 // 2), dtype=np.uint16)
+    f = _L().oracle_swiglu_bf16
+    f.restype = None
+    f(_p(x), C.c_size_t(T), C.c_size_t(F2 // 2), _p(out))
+    return out
+
+
 def cast(x_bf16: np.ndarray, scale_value, fmt: int, transpose: bool = False):
     x = _c(x_bf16, np.uint16)
     if x.ndim == 1:

@@ -181,6 +181,56 @@ void oracle_cast_bf16(const uint16_t *x, size_t rows, size_t cols, float scale, 
 }
 
 /* ------------------------------------------------------------------------------------------------
+ * Kurtosis monitor (Section 4, "Long-term outlier dynamics"): kurt(x) = mu[x^4] / sigma^2[x]^2 for one token
+ * vector x, without centring, averaged over the tokens of the tensor.  Reading of the printed formula
+ * (its denominator is typeset as the variance of x^2): the un-centred second moment of x, squared, i.e.
+ * mu[x^4] / mu[x^2]^2 - the only reading under which "maximised when few elements are extremely large"
+ * holds (a one-hot vector of length D gives D, a constant vector 1, a Gaussian about 3).
+ * A row of zeros contributes 0.
+ * ---------------------------------------------------------------------------------------------- */
+double oracle_kurtosis_bf16(const uint16_t *x, size_t rows, size_t cols)
+{
+    double total = 0.0;
+#pragma omp parallel for reduction(+ : total) schedule(static)
+    for (long r = 0; r < (long)rows; ++r) {
+        double s2 = 0.0, s4 = 0.0;
+        for (size_t c = 0; c < cols; ++c) {
+            double v = (double)bf16_bits_to_float(x[(size_t)r * cols + c]);
+            s2 += v * v;
+            s4 += v * v * v * v;
+        }
+        if (s2 > 0.0) total += (s4 / (double)cols) / ((s2 / (double)cols) * (s2 / (double)cols));
+    }
+    return total / (double)rows;
+}
+
+static uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x40);   /* NaN stays NaN */
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Gated activation feeding the second FFN projection (Appendix B: FFN with activation phi; the Llama-style
+ * workloads use SwiGLU): h = silu(gate) * up, silu(g) = g / (1 + exp(-g)), gate = columns [0,F) and
+ * up = columns [F,2F) of the fused first-projection output.  h is rounded to BF16 (what a BF16 framework
+ * would hold) and that tensor is what amax and the cast see, so the rest equals oracle_cast_bf16.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_swiglu_bf16(const uint16_t *gate_up, size_t T, size_t F, uint16_t *h)
+{
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < (long)T; ++t)
+        for (size_t f = 0; f < F; ++f) {
+            double g = (double)bf16_bits_to_float(gate_up[(size_t)t * 2 * F + f]);
+            double u = (double)bf16_bits_to_float(gate_up[(size_t)t * 2 * F + F + f]);
+            h[(size_t)t * F + f] = f32_to_bf16_rne((float)(g / (1.0 + exp(-g)) * u));
+        }
+}
+
+/* ------------------------------------------------------------------------------------------------
  * FP8 GEMM with descale (Appendix E): ref[i,j] = sa_inv*sb_inv * sum_k dec(A[i,k]) * dec(B[j,k]),
  * accumulated in double, on a list of output rows and columns.  A and B are addressed through
  * (row stride, reduction stride) so that the three linear products are this one routine on three

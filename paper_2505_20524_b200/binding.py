@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
-           "fp8_quantize",
+           "fp8_quantize", "fp8_swiglu_cast", "fp8_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
@@ -115,6 +115,18 @@ def fp8_quantize(x, fmt, out, out_t, amax, scale, scale_inv, stream=None):
     rows, cols = _rows_cols(x)
     _check(load().fp8_quantize(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), C.c_int(fmt), _ptr(out), _ptr(out_t),
                                _ptr(amax), _ptr(scale), _ptr(scale_inv), _stream(stream)))
+
+
+def fp8_swiglu_cast(gate_up, scale, fmt, out, out_t=None, amax_out=None, stream=None):
+    """h = silu(gate) * up fused with the cast; gate_up is [T, 2F] BF16.  out / out_t may be None (amax only)."""
+    T, F2 = gate_up.shape
+    _check(load().fp8_swiglu_cast(_ptr(gate_up), C.c_size_t(T), C.c_size_t(F2 // 2), _ptr(scale), C.c_int(fmt),
+                                  _ptr(out), _ptr(out_t), _ptr(amax_out), _stream(stream)))
+
+
+def fp8_kurtosis(x, out, stream=None):
+    rows, cols = _rows_cols(x)
+    _check(load().fp8_kurtosis(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), _ptr(out), _stream(stream)))
 
 
 def _is_fp32(t):

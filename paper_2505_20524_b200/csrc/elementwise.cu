@@ -1,0 +1,219 @@
+// Element-wise companions of the quantize path: the gated activation fused with the cast, and the kurtosis
+// monitor.  Both are HBM streams (16-byte loads and stores).  The sigmoid uses the hardware exp2 and reciprocal
+// approximations (relative error near 2^-22): h is rounded to BF16 straight after, so the approximation shows
+// only where the exact value sits within that distance of a BF16 rounding boundary.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace fp8dpa {
+
+__device__ __forceinline__ uint32_t absmax2e(uint32_t m, uint32_t w) { return __vmaxu2(m, w & 0x7FFF7FFFu); }
+
+__device__ __forceinline__ void block_max_bf16_to(uint32_t m2, unsigned int *amax_bits)
+{
+    __shared__ uint32_t warp_max[32];
+    uint32_t m = max(m2 & 0xFFFFu, m2 >> 16);
+    m = __reduce_max_sync(0xffffffffu, m);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) warp_max[warp] = m;
+    __syncthreads();
+    if (warp == 0) {
+        const int nwarps = (blockDim.x + 31) >> 5;
+        m = lane < nwarps ? warp_max[lane] : 0u;
+        m = __reduce_max_sync(0xffffffffu, m);
+        if (lane == 0 && m != 0u) atomicMax(amax_bits, m << 16);
+    }
+}
+
+__device__ __forceinline__ float silu_mul(float g, float u)
+{
+    float r;
+    const float e = ex2_approx(-1.4426950408889634f * g);     // exp(-g); +inf for very negative g gives r = 0
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(1.0f + e));
+    return g * r * u;
+}
+
+// 8 gate + 8 up BF16 -> 8 BF16 values of h (packed two per word)
+__device__ __forceinline__ uint4 swiglu8(const uint4 g, const uint4 u)
+{
+    const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, uw[4] = {u.x, u.y, u.z, u.w};
+    uint32_t h[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        h[i] = pack_bf16x2(silu_mul(bf16_lo(gw[i]), bf16_lo(uw[i])), silu_mul(bf16_hi(gw[i]), bf16_hi(uw[i])));
+    return make_uint4(h[0], h[1], h[2], h[3]);
+}
+
+template <int FMT>
+__device__ __forceinline__ uint2 cast8e(const uint4 v, const float s)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint16_t h[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        h[i] = cvt_f32x2_to_fp8x2<FMT>(__fmul_rn(bf16_lo(w[i]), s), __fmul_rn(bf16_hi(w[i]), s));
+    return make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
+}
+
+constexpr int ST = 128;          // tile edge
+constexpr int SPITCH = ST + 4;   // padded row of the staging tile
+
+// One CTA per 128 x 128 tile of h.  Phase 1 computes h, its amax, the codes (row-major store + staging tile);
+// phase 2 writes the transposed copy from the staging tile.
+template <int FMT>
+__global__ void __launch_bounds__(256) swiglu_cast_kernel(const uint16_t *__restrict__ gate_up, int T, int F,
+                                                          const float *__restrict__ scale_ptr,
+                                                          uint8_t *__restrict__ out, uint8_t *__restrict__ out_t,
+                                                          unsigned int *__restrict__ amax_bits)
+{
+    __shared__ __align__(16) uint8_t tile[ST * SPITCH];
+    const bool want_codes = out != nullptr || out_t != nullptr;
+    const float s = want_codes ? __ldg(scale_ptr) : 1.0f;
+    const int r0 = blockIdx.y * ST, c0 = blockIdx.x * ST;
+    uint32_t m = 0;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int idx = it * 256 + threadIdx.x;
+        const int r = idx >> 3, cg = idx & 7;
+        const int gr = r0 + r, gc = c0 + cg * 16;
+        if (gr < T && gc < F) {
+            const uint4 *pg = reinterpret_cast<const uint4 *>(gate_up + (size_t)gr * 2 * F + gc);
+            const uint4 *pu = reinterpret_cast<const uint4 *>(gate_up + (size_t)gr * 2 * F + F + gc);
+            const uint4 h0 = swiglu8(__ldg(pg), __ldg(pu)), h1 = swiglu8(__ldg(pg + 1), __ldg(pu + 1));
+            if (amax_bits) {
+                m = absmax2e(absmax2e(absmax2e(absmax2e(m, h0.x), h0.y), h0.z), h0.w);
+                m = absmax2e(absmax2e(absmax2e(absmax2e(m, h1.x), h1.y), h1.z), h1.w);
+            }
+            if (want_codes) {
+                const uint2 p0 = cast8e<FMT>(h0, s), p1 = cast8e<FMT>(h1, s);
+                if (out) *reinterpret_cast<uint4 *>(out + (size_t)gr * F + gc) = make_uint4(p0.x, p0.y, p1.x, p1.y);
+                if (out_t) {
+                    uint32_t *t = reinterpret_cast<uint32_t *>(tile + r * SPITCH + cg * 16);
+                    t[0] = p0.x; t[1] = p0.y; t[2] = p1.x; t[3] = p1.y;
+                }
+            }
+        }
+    }
+    if (out_t) {
+        __syncthreads();
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int idx = it * 256 + threadIdx.x;
+            const int half = idx & 1, c = (idx >> 1) & 127, rp = idx >> 8;
+            const int rg = rp * 2 + half;
+            const int gc = c0 + c, gr = r0 + rg * 16;
+            if (gc < F && gr < T) {
+                uint32_t w[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t v = 0;
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) v |= (uint32_t)tile[(rg * 16 + q * 4 + b) * SPITCH + c] << (8 * b);
+                    w[q] = v;
+                }
+                *reinterpret_cast<uint4 *>(out_t + (size_t)gc * T + gr) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+    }
+    if (amax_bits) block_max_bf16_to(m, amax_bits);
+}
+
+// One CTA per row: sums of x^2 and x^4, then kurt = mean(x^4) / mean(x^2)^2 added (scaled by 1/rows) to *out.
+__global__ void __launch_bounds__(256) kurtosis_kernel(const uint16_t *__restrict__ x, int cols, float inv_rows,
+                                                       float *__restrict__ out)
+{
+    __shared__ float red2[8], red4[8];
+    const uint4 *row = reinterpret_cast<const uint4 *>(x + (size_t)blockIdx.x * cols);
+    float s2 = 0.0f, s4 = 0.0f;
+    for (int i = threadIdx.x; i < cols / 8; i += blockDim.x) {
+        const uint4 v = __ldg(row + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float a = bf16_lo(w[k]), b = bf16_hi(w[k]);
+            const float a2 = a * a, b2 = b * b;
+            s2 += a2 + b2;
+            s4 += a2 * a2 + b2 * b2;
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        s2 += __shfl_xor_sync(0xffffffffu, s2, off);
+        s4 += __shfl_xor_sync(0xffffffffu, s4, off);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        red2[threadIdx.x >> 5] = s2;
+        red4[threadIdx.x >> 5] = s4;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t2 = 0.0f, t4 = 0.0f;
+        for (int w = 0; w < 8; ++w) { t2 += red2[w]; t4 += red4[w]; }
+        if (t2 > 0.0f) {
+            const float m2 = t2 / (float)cols, m4 = t4 / (float)cols;
+            atomicAdd(out, m4 / (m2 * m2) * inv_rows);
+        }
+    }
+}
+
+}  // namespace fp8dpa
+
+using namespace fp8dpa;
+
+extern "C" int fp8_swiglu_cast(const void *gate_up_bf16, size_t T, size_t F, const float *scale, int fmt, uint8_t *out,
+                               uint8_t *out_t, float *amax_out, void *stream)
+{
+    const bool want_codes = out || out_t;
+    if (!gate_up_bf16 || (want_codes && !scale) || (!want_codes && !amax_out)) {
+        set_error("fp8_swiglu_cast: NULL pointer (need gate_up, and either outputs with a scale or amax_out)");
+        return FP8_ERR_NULL;
+    }
+    if (fmt != FP8_E4M3 && fmt != FP8_E5M2) {
+        set_error("fp8_swiglu_cast: fmt %d is not FP8_E4M3 / FP8_E5M2", fmt);
+        return FP8_ERR_ENUM;
+    }
+    if (T == 0 || F == 0 || (F % 16) || (out_t && (T % 16)) || T > 0x7FFFFFFFull || F > 0x3FFFFFFFull) {
+        set_error("fp8_swiglu_cast: unsupported shape T=%zu F=%zu (F %% 16 == 0; T %% 16 == 0 with a transposed copy)", T, F);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(gate_up_bf16) || !aligned16(out) || !aligned16(out_t)) {
+        set_error("fp8_swiglu_cast: tensor pointers must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (amax_out) FP8_CUDA_CHECK(cudaMemsetAsync(amax_out, 0, sizeof(float), st));
+    dim3 grid((unsigned)((F + ST - 1) / ST), (unsigned)((T + ST - 1) / ST));
+    const uint16_t *x = static_cast<const uint16_t *>(gate_up_bf16);
+    unsigned int *ab = reinterpret_cast<unsigned int *>(amax_out);
+    if (fmt == FP8_E4M3) swiglu_cast_kernel<0><<<grid, 256, 0, st>>>(x, (int)T, (int)F, scale, out, out_t, ab);
+    else swiglu_cast_kernel<1><<<grid, 256, 0, st>>>(x, (int)T, (int)F, scale, out, out_t, ab);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+extern "C" int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *out, void *stream)
+{
+    if (!x_bf16 || !out) {
+        set_error("fp8_kurtosis: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if (rows == 0 || cols == 0 || (cols % 8) || rows > 0x7FFFFFFFull || cols > 0x7FFFFFFFull) {
+        set_error("fp8_kurtosis: unsupported shape rows=%zu cols=%zu (cols %% 8 == 0)", rows, cols);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(x_bf16)) {
+        set_error("fp8_kurtosis: x must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    FP8_CUDA_CHECK(cudaMemsetAsync(out, 0, sizeof(float), st));
+    kurtosis_kernel<<<(unsigned)rows, 256, 0, st>>>(static_cast<const uint16_t *>(x_bf16), (int)cols,
+                                                   1.0f / (float)rows, out);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
