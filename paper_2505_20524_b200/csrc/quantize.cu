@@ -54,19 +54,39 @@ __global__ void __launch_bounds__(512) amax_kernel(const uint4 *__restrict__ x, 
 }
 
 // ---------------------------------------------------------------- scale
+__device__ __forceinline__ float scale_from_amax(float a, float fp8_max, int margin)
+{
+    if (!(a > 0.0f) || isinf(a)) return 1.0f;
+    const float s = __fmul_rn(__fdiv_rn(fp8_max, a), ldexpf(1.0f, -margin));   // power-of-two factor: exact
+    return isinf(s) ? FLT_MAX : s;
+}
+
 __global__ void scale_kernel(const float *__restrict__ amax, float fp8_max, int margin, float *__restrict__ scale,
                              float *__restrict__ scale_inv)
 {
-    const float a = *amax;
-    float s;
-    if (!(a > 0.0f) || isinf(a)) {
-        s = 1.0f;
-    } else {
-        s = __fmul_rn(__fdiv_rn(fp8_max, a), ldexpf(1.0f, -margin));   // power-of-two factor: exact
-        if (isinf(s)) s = FLT_MAX;
-    }
+    const float s = scale_from_amax(*amax, fp8_max, margin);
     *scale = s;
     *scale_inv = __fdiv_rn(1.0f, s);
+}
+
+// Where a cast takes its scale from.  Caller-supplied: `scale` is read.  Just-in-time (`amax` non-NULL): every
+// thread derives the scale from the amax that the preceding pass left in memory (the arithmetic of scale_kernel)
+// and the first thread of the grid publishes scale and 1/scale; no separate one-thread launch in between.
+struct ScaleSrc {
+    const float *scale;
+    const float *amax;
+    float fp8_max;
+    float *scale_out, *scale_inv_out;
+};
+__device__ __forceinline__ float resolve_scale(const ScaleSrc &src, bool first_thread)
+{
+    if (!src.amax) return __ldg(src.scale);
+    const float s = scale_from_amax(__ldg(src.amax), src.fp8_max, 0);
+    if (first_thread) {
+        *src.scale_out = s;
+        *src.scale_inv_out = __fdiv_rn(1.0f, s);
+    }
+    return s;
 }
 
 // ---------------------------------------------------------------- delayed scaling: history ring update
@@ -126,16 +146,22 @@ template <int FMT, bool AMAX>
 __global__ void __launch_bounds__(256) cast_flat_kernel(const uint4 *__restrict__ x, size_t n16,
                                                         const uint16_t *__restrict__ tail_in,
                                                         uint8_t *__restrict__ tail_out, int n_tail,
-                                                        const float *__restrict__ scale_ptr,
+                                                        const ScaleSrc scale_src,
                                                         uint4 *__restrict__ out, unsigned int *__restrict__ amax_bits)
 {
-    const float s = __ldg(scale_ptr);
+    const float s = resolve_scale(scale_src, blockIdx.x == 0 && threadIdx.x == 0);
     uint32_t m = 0;
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // Back to front: the amax pass that precedes a just-in-time cast walked the tensor front to back, so its
+    // tail is what the L2 still holds.
+    if (n16 > 0) {
+        x += 2 * (n16 - 1);
+        out += n16 - 1;
+    }
     for (; i + stride < n16; i += 2 * stride) {
-        const uint4 a0 = __ldg(x + 2 * i), a1 = __ldg(x + 2 * i + 1);
-        const uint4 b0 = __ldg(x + 2 * (i + stride)), b1 = __ldg(x + 2 * (i + stride) + 1);
+        const uint4 a0 = __ldg(x - 2 * i), a1 = __ldg(x - 2 * i + 1);
+        const uint4 b0 = __ldg(x - 2 * (i + stride)), b1 = __ldg(x - 2 * (i + stride) + 1);
         if (AMAX) {
             m = absmax2(absmax2(absmax2(absmax2(m, a0.x), a0.y), a0.z), a0.w);
             m = absmax2(absmax2(absmax2(absmax2(m, a1.x), a1.y), a1.z), a1.w);
@@ -144,17 +170,17 @@ __global__ void __launch_bounds__(256) cast_flat_kernel(const uint4 *__restrict_
         }
         const uint2 p0 = cast8<FMT>(a0, s), p1 = cast8<FMT>(a1, s);
         const uint2 q0 = cast8<FMT>(b0, s), q1 = cast8<FMT>(b1, s);
-        out[i] = make_uint4(p0.x, p0.y, p1.x, p1.y);
-        out[i + stride] = make_uint4(q0.x, q0.y, q1.x, q1.y);
+        *(out - i) = make_uint4(p0.x, p0.y, p1.x, p1.y);
+        *(out - (i + stride)) = make_uint4(q0.x, q0.y, q1.x, q1.y);
     }
     for (; i < n16; i += stride) {
-        const uint4 a0 = __ldg(x + 2 * i), a1 = __ldg(x + 2 * i + 1);
+        const uint4 a0 = __ldg(x - 2 * i), a1 = __ldg(x - 2 * i + 1);
         if (AMAX) {
             m = absmax2(absmax2(absmax2(absmax2(m, a0.x), a0.y), a0.z), a0.w);
             m = absmax2(absmax2(absmax2(absmax2(m, a1.x), a1.y), a1.z), a1.w);
         }
         const uint2 p0 = cast8<FMT>(a0, s), p1 = cast8<FMT>(a1, s);
-        out[i] = make_uint4(p0.x, p0.y, p1.x, p1.y);
+        *(out - i) = make_uint4(p0.x, p0.y, p1.x, p1.y);
     }
     if (blockIdx.x == 0 && (int)threadIdx.x < n_tail) {
         const uint32_t w = tail_in[threadIdx.x];
@@ -173,13 +199,15 @@ constexpr int TPITCH = TT + 4;   // 33 words per row: column reads hit distinct 
 
 template <int FMT, bool AMAX>
 __global__ void __launch_bounds__(256) cast_transpose_kernel(const uint16_t *__restrict__ x, int rows, int cols,
-                                                             const float *__restrict__ scale_ptr,
+                                                             const ScaleSrc scale_src,
                                                              uint8_t *__restrict__ out, uint8_t *__restrict__ out_t,
                                                              unsigned int *__restrict__ amax_bits)
 {
     __shared__ __align__(16) uint8_t tile[TT * TPITCH];
-    const float s = __ldg(scale_ptr);
-    const int r0 = blockIdx.y * TT, c0 = blockIdx.x * TT;
+    const float s = resolve_scale(scale_src, blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0);
+    // tiles are taken back to front (last rows first): after the amax pass of a just-in-time cast the tail of
+    // the tensor is what the L2 still holds
+    const int r0 = (int)(gridDim.y - 1 - blockIdx.y) * TT, c0 = (int)(gridDim.x - 1 - blockIdx.x) * TT;
     uint32_t m = 0;
     // phase 1: 128 rows x 8 groups of 16 columns
 #pragma unroll
@@ -259,7 +287,7 @@ static int validate_cast(const void *x, size_t rows, size_t cols, const float *s
 }
 
 template <int FMT, bool AMAX>
-static void launch_cast(const void *x, size_t rows, size_t cols, const float *scale, uint8_t *out, uint8_t *out_t,
+static void launch_cast(const void *x, size_t rows, size_t cols, const ScaleSrc &scale, uint8_t *out, uint8_t *out_t,
                         float *amax_out, cudaStream_t st)
 {
     unsigned int *ab = reinterpret_cast<unsigned int *>(amax_out);
@@ -296,8 +324,8 @@ static int do_amax(const void *x, size_t n, float *amax, cudaStream_t st)
     return FP8_OK;
 }
 
-static int do_cast(const void *x, size_t rows, size_t cols, const float *scale, int fmt, uint8_t *out, uint8_t *out_t,
-                   float *amax_out, cudaStream_t st)
+static int do_cast(const void *x, size_t rows, size_t cols, const ScaleSrc &scale, int fmt, uint8_t *out,
+                   uint8_t *out_t, float *amax_out, cudaStream_t st)
 {
     if (amax_out) FP8_CUDA_CHECK(cudaMemsetAsync(amax_out, 0, sizeof(float), st));
     if (fmt == FP8_E4M3) {
@@ -363,7 +391,8 @@ extern "C" int fp8_cast(const void *x_bf16, size_t rows, size_t cols, const floa
     if (rc != FP8_OK) return rc;
     rc = check_arch();
     if (rc != FP8_OK) return rc;
-    return do_cast(x_bf16, rows, cols, scale, fmt, out, out_t, amax_out, static_cast<cudaStream_t>(stream));
+    const ScaleSrc src{scale, nullptr, 0.0f, nullptr, nullptr};
+    return do_cast(x_bf16, rows, cols, src, fmt, out, out_t, amax_out, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fmt, uint8_t *out, uint8_t *out_t,
@@ -380,9 +409,8 @@ extern "C" int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fm
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     rc = do_amax(x_bf16, rows * cols, amax, st);
     if (rc != FP8_OK) return rc;
-    scale_kernel<<<1, 1, 0, st>>>(amax, fmt == FP8_E4M3 ? 448.0f : 57344.0f, 0, scale, scale_inv);
-    FP8_CUDA_CHECK(cudaGetLastError());
-    return do_cast(x_bf16, rows, cols, scale, fmt, out, out_t, nullptr, st);
+    const ScaleSrc src{nullptr, amax, fmt == FP8_E4M3 ? 448.0f : 57344.0f, scale, scale_inv};
+    return do_cast(x_bf16, rows, cols, src, fmt, out, out_t, nullptr, st);
 }
 
 extern "C" int fp8_scale_update(float *history, int len, int *head, const float *amax_new, int fmt, int margin,

@@ -75,7 +75,7 @@ class Linear:
 class BlockHotPath:
     """Device buffers of one block configuration and the step that runs the hot path over them."""
 
-    KERNELS_PER_QUANTIZE = 3    # amax, scale, cast
+    KERNELS_PER_QUANTIZE = 2      # amax, cast (the cast derives the scale itself)
     KERNELS_PER_ATTN_BWD = 3    # prep, main, finish
 
     def __init__(self, cfg: synth.BlockConfig, device="cuda", with_linears=None, with_attention=True,
