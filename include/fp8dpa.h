@@ -97,10 +97,20 @@ FP8_API int fp8_scale_update(float *history, int len, int *head, const float *am
  * then treated exactly like the input of fp8_cast: out[t,f] = sat_rne_fmt(float(h) * *scale), out_t the same
  * codes as [F,T] (nullable), *amax_out = amax(h) (nullable).  out and out_t may both be NULL when only the amax
  * is wanted (first pass of just-in-time scaling).  F % 16 == 0, T % 16 == 0 when out_t is given.
- * silu uses expf, so a code can differ from a double-precision evaluation where h lies within an ulp of a
- * rounding boundary. */
+ * The sigmoid uses the hardware exp2 / reciprocal approximations (relative error near 2^-22), so a code can
+ * differ from a double-precision evaluation where h lies that close to a BF16 rounding boundary. */
 FP8_API int fp8_swiglu_cast(const void *gate_up_bf16, size_t T, size_t F, const float *scale, int fmt,
                     uint8_t *out, uint8_t *out_t, float *amax_out, void *stream);
+
+/* The un-gated FFN activations of the other architecture families (Appendix B, architecture table), fused with
+ * the cast in the same way: x is the [T,F] BF16 output of the first FFN projection, h = act(x) rounded to BF16,
+ * then out / out_t / amax_out as in fp8_swiglu_cast.
+ *   FP8_ACT_GELU   h = 0.5 x (1 + erf(x / sqrt 2))                                   (exact form)
+ *   FP8_ACT_XIELU  h = a_p x^2 + 0.5 x (x > 0);  a_n (e^x - 1) - a_n x + 0.5 x (x <= 0)   (Appendix B, Eq. (xIELU))
+ * act_params: device pointer to {a_p, a_n} (the per-layer trainable scalars) for xIELU, ignored for GeLU. */
+enum { FP8_ACT_GELU = 1, FP8_ACT_XIELU = 2 };
+FP8_API int fp8_act_cast(const void *x_bf16, size_t T, size_t F, int act, const float *act_params, const float *scale,
+                 int fmt, uint8_t *out, uint8_t *out_t, float *amax_out, void *stream);
 
 /* Kurtosis monitor (Section 4): *out = mean over rows of mu[x^4] / mu[x^2]^2 of a [rows, cols] BF16 tensor
  * (un-centred; rows are token vectors).  *out is overwritten.  cols % 8 == 0. */

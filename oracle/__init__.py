@@ -157,6 +157,19 @@ def swiglu(gate_up_bf16: np.ndarray) -> np.ndarray:
     return out
 
 
+GELU, XIELU = 1, 2
+
+
+def activation(x_bf16: np.ndarray, act: int, alpha_p: float = 0.0, alpha_n: float = 0.0) -> np.ndarray:
+    """GeLU (exact erf form) or xIELU of a BF16 tensor, rounded to BF16 (Appendix B)."""
+    x = _c(x_bf16, np.uint16)
+    out = np.empty_like(x)
+    f = _L().oracle_activation_bf16
+    f.restype = None
+    f(_p(x), C.c_size_t(x.size), C.c_int(act), C.c_double(alpha_p), C.c_double(alpha_n), _p(out))
+    return out
+
+
 def cast(x_bf16: np.ndarray, scale_value, fmt: int, transpose: bool = False):
     x = _c(x_bf16, np.uint16)
     if x.ndim == 1:

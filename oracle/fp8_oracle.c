@@ -231,6 +231,24 @@ void oracle_swiglu_bf16(const uint16_t *gate_up, size_t T, size_t F, uint16_t *h
 }
 
 /* ------------------------------------------------------------------------------------------------
+ * Element-wise FFN activations of the other architecture families (Appendix B, architecture table):
+ *   act 1  GeLU(x)  = x * Phi(x) = 0.5 x (1 + erf(x / sqrt 2))     (exact form; the paper names no approximation)
+ *   act 2  xIELU(x) = alpha_p x^2 + 0.5 x                          for x > 0      (Appendix B, Eq. (xIELU))
+ *                     alpha_n (e^x - 1) - alpha_n x + 0.5 x        for x <= 0
+ * x is the [T,F] BF16 output of the first FFN projection; h is rounded to BF16 like oracle_swiglu_bf16.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_activation_bf16(const uint16_t *x, size_t n, int act, double alpha_p, double alpha_n, uint16_t *h)
+{
+#pragma omp parallel for schedule(static)
+    for (long i = 0; i < (long)n; ++i) {
+        double v = (double)bf16_bits_to_float(x[i]), r;
+        if (act == 1) r = 0.5 * v * (1.0 + erf(v * 0.70710678118654752440));
+        else r = v > 0.0 ? alpha_p * v * v + 0.5 * v : alpha_n * expm1(v) - alpha_n * v + 0.5 * v;
+        h[i] = f32_to_bf16_rne((float)r);
+    }
+}
+
+/* ------------------------------------------------------------------------------------------------
  * FP8 GEMM with descale (Appendix E): ref[i,j] = sa_inv*sb_inv * sum_k dec(A[i,k]) * dec(B[j,k]),
  * accumulated in double, on a list of output rows and columns.  A and B are addressed through
  * (row stride, reduction stride) so that the three linear products are this one routine on three

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
-           "fp8_quantize", "fp8_swiglu_cast", "fp8_kurtosis",
+           "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
@@ -115,6 +115,16 @@ def fp8_quantize(x, fmt, out, out_t, amax, scale, scale_inv, stream=None):
     rows, cols = _rows_cols(x)
     _check(load().fp8_quantize(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), C.c_int(fmt), _ptr(out), _ptr(out_t),
                                _ptr(amax), _ptr(scale), _ptr(scale_inv), _stream(stream)))
+
+
+ACT_GELU, ACT_XIELU = 1, 2
+
+
+def fp8_act_cast(x, act, act_params, scale, fmt, out, out_t=None, amax_out=None, stream=None):
+    """h = GeLU(x) or xIELU(x; a_p, a_n) fused with the cast; x is [T, F] BF16, act_params a device float[2] or None."""
+    T, F = x.shape
+    _check(load().fp8_act_cast(_ptr(x), C.c_size_t(T), C.c_size_t(F), C.c_int(act), _ptr(act_params), _ptr(scale),
+                               C.c_int(fmt), _ptr(out), _ptr(out_t), _ptr(amax_out), _stream(stream)))
 
 
 def fp8_swiglu_cast(gate_up, scale, fmt, out, out_t=None, amax_out=None, stream=None):

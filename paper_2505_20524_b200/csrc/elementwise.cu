@@ -34,14 +34,62 @@ __device__ __forceinline__ float silu_mul(float g, float u)
     return g * r * u;
 }
 
-// 8 gate + 8 up BF16 -> 8 BF16 values of h (packed two per word)
-__device__ __forceinline__ uint4 swiglu8(const uint4 g, const uint4 u)
+// 0.5 * erfc(y) for y >= 0 as 0.5 * t * exp(Q(t) - y^2), t = 1 / (1 + y/2): Q is a degree-9 least-squares fit of
+// log(erfcx(y) / t) on Chebyshev nodes of t in [0.2, 1] (y in [0, 8]); evaluated in binary32 the relative error
+// stays below 2e-6 up to y = 4 and 6e-6 up to y = 8, past which the result is below 1e-29.
+__device__ __forceinline__ float half_erfc_pos(float y)
+{
+    float t;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.5f, y, 1.0f)));
+    float q = 1.227935892e-01f;
+    q = fmaf(q, t, -5.583772951e-01f);
+    q = fmaf(q, t, 8.634607687e-01f);
+    q = fmaf(q, t, -2.980391946e-01f);
+    q = fmaf(q, t, -4.172309384e-01f);
+    q = fmaf(q, t, 1.850209772e-01f);
+    q = fmaf(q, t, -2.980059381e-02f);
+    q = fmaf(q, t, 4.005914557e-01f);
+    q = fmaf(q, t, 9.969420963e-01f);
+    q = fmaf(q, t, -1.265360832e+00f);
+    return 0.5f * t * ex2_approx(1.4426950408889634f * fmaf(-y, y, q));
+}
+
+// activations: 0 = SiLU(gate) * up (two inputs), 1 = GeLU (exact form), 2 = xIELU with (a_p, a_n)
+constexpr int ACT_SWIGLU = 0;
+template <int ACT>
+__device__ __forceinline__ float act1(float x, float u, float a_p, float a_n)
+{
+    if (ACT == ACT_SWIGLU) return silu_mul(x, u);
+    if (ACT == FP8_ACT_GELU) {
+        // x * Phi(x), Phi(x) = erfc(-x / sqrt 2) / 2; from the tail side, so that the left tail keeps its relative accuracy
+        const float e = half_erfc_pos(fabsf(x) * 0.70710678118654752440f);
+        return x * (x < 0.0f ? e : 1.0f - e);
+    }
+    // xIELU, x <= 0: a_n (e^x - 1 - x) + x / 2.  e^x - 1 - x from its series near 0 (|x| < 1/4, next term below 2e-9
+    // of the first), from the hardware exp2 elsewhere.
+    const float pos = fmaf(a_p * x, x, 0.5f * x);
+    float ser = 1.0f / 5040.0f;
+    ser = fmaf(ser, x, 1.0f / 720.0f);
+    ser = fmaf(ser, x, 1.0f / 120.0f);
+    ser = fmaf(ser, x, 1.0f / 24.0f);
+    ser = fmaf(ser, x, 1.0f / 6.0f);
+    ser = fmaf(ser, x, 0.5f);
+    ser = ser * x * x;
+    const float big = ex2_approx(1.4426950408889634f * x) - 1.0f - x;
+    const float neg = fmaf(a_n, x > -0.25f ? ser : big, 0.5f * x);
+    return x > 0.0f ? pos : neg;
+}
+
+// 8 inputs (+ 8 up values for the gated form) -> 8 BF16 values of h (packed two per word)
+template <int ACT>
+__device__ __forceinline__ uint4 act8(const uint4 g, const uint4 u, float a_p, float a_n)
 {
     const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, uw[4] = {u.x, u.y, u.z, u.w};
     uint32_t h[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
-        h[i] = pack_bf16x2(silu_mul(bf16_lo(gw[i]), bf16_lo(uw[i])), silu_mul(bf16_hi(gw[i]), bf16_hi(uw[i])));
+        h[i] = pack_bf16x2(act1<ACT>(bf16_lo(gw[i]), bf16_lo(uw[i]), a_p, a_n),
+                           act1<ACT>(bf16_hi(gw[i]), bf16_hi(uw[i]), a_p, a_n));
     return make_uint4(h[0], h[1], h[2], h[3]);
 }
 
@@ -61,12 +109,17 @@ constexpr int SPITCH = ST + 4;   // padded row of the staging tile
 
 // One CTA per 128 x 128 tile of h.  Phase 1 computes h, its amax, the codes (row-major store + staging tile);
 // phase 2 writes the transposed copy from the staging tile.
-template <int FMT>
-__global__ void __launch_bounds__(256) swiglu_cast_kernel(const uint16_t *__restrict__ gate_up, int T, int F,
-                                                          const float *__restrict__ scale_ptr,
-                                                          uint8_t *__restrict__ out, uint8_t *__restrict__ out_t,
-                                                          unsigned int *__restrict__ amax_bits)
+template <int FMT, int ACT>
+__global__ void __launch_bounds__(256) act_cast_kernel(const uint16_t *__restrict__ gate_up, int T, int F,
+                                                       const float *__restrict__ act_params,
+                                                       const float *__restrict__ scale_ptr,
+                                                       uint8_t *__restrict__ out, uint8_t *__restrict__ out_t,
+                                                       unsigned int *__restrict__ amax_bits)
 {
+    constexpr bool GATED = ACT == ACT_SWIGLU;
+    const int pitch = GATED ? 2 * F : F;              // input row length
+    const float a_p = ACT == FP8_ACT_XIELU ? __ldg(act_params) : 0.0f;
+    const float a_n = ACT == FP8_ACT_XIELU ? __ldg(act_params + 1) : 0.0f;
     __shared__ __align__(16) uint8_t tile[ST * SPITCH];
     const bool want_codes = out != nullptr || out_t != nullptr;
     const float s = want_codes ? __ldg(scale_ptr) : 1.0f;
@@ -78,9 +131,11 @@ __global__ void __launch_bounds__(256) swiglu_cast_kernel(const uint16_t *__rest
         const int r = idx >> 3, cg = idx & 7;
         const int gr = r0 + r, gc = c0 + cg * 16;
         if (gr < T && gc < F) {
-            const uint4 *pg = reinterpret_cast<const uint4 *>(gate_up + (size_t)gr * 2 * F + gc);
-            const uint4 *pu = reinterpret_cast<const uint4 *>(gate_up + (size_t)gr * 2 * F + F + gc);
-            const uint4 h0 = swiglu8(__ldg(pg), __ldg(pu)), h1 = swiglu8(__ldg(pg + 1), __ldg(pu + 1));
+            const uint4 *pg = reinterpret_cast<const uint4 *>(gate_up + (size_t)gr * pitch + gc);
+            const uint4 *pu = reinterpret_cast<const uint4 *>(gate_up + (size_t)gr * pitch + F + gc);
+            const uint4 g0 = __ldg(pg), g1 = __ldg(pg + 1);
+            const uint4 u0 = GATED ? __ldg(pu) : g0, u1 = GATED ? __ldg(pu + 1) : g1;
+            const uint4 h0 = act8<ACT>(g0, u0, a_p, a_n), h1 = act8<ACT>(g1, u1, a_p, a_n);
             if (amax_bits) {
                 m = absmax2e(absmax2e(absmax2e(absmax2e(m, h0.x), h0.y), h0.z), h0.w);
                 m = absmax2e(absmax2e(absmax2e(absmax2e(m, h1.x), h1.y), h1.z), h1.w);
@@ -161,24 +216,24 @@ __global__ void __launch_bounds__(256) kurtosis_kernel(const uint16_t *__restric
 
 using namespace fp8dpa;
 
-extern "C" int fp8_swiglu_cast(const void *gate_up_bf16, size_t T, size_t F, const float *scale, int fmt, uint8_t *out,
-                               uint8_t *out_t, float *amax_out, void *stream)
+static int act_cast(const char *who, const void *x, size_t T, size_t F, int act, const float *act_params,
+                    const float *scale, int fmt, uint8_t *out, uint8_t *out_t, float *amax_out, void *stream)
 {
     const bool want_codes = out || out_t;
-    if (!gate_up_bf16 || (want_codes && !scale) || (!want_codes && !amax_out)) {
-        set_error("fp8_swiglu_cast: NULL pointer (need gate_up, and either outputs with a scale or amax_out)");
+    if (!x || (want_codes && !scale) || (!want_codes && !amax_out) || (act == FP8_ACT_XIELU && !act_params)) {
+        set_error("%s: NULL pointer (need the input, either outputs with a scale or amax_out, and act_params for xIELU)", who);
         return FP8_ERR_NULL;
     }
-    if (fmt != FP8_E4M3 && fmt != FP8_E5M2) {
-        set_error("fp8_swiglu_cast: fmt %d is not FP8_E4M3 / FP8_E5M2", fmt);
+    if ((fmt != FP8_E4M3 && fmt != FP8_E5M2) || act < 0 || act > FP8_ACT_XIELU) {
+        set_error("%s: fmt %d / act %d is not a known enum value", who, fmt, act);
         return FP8_ERR_ENUM;
     }
     if (T == 0 || F == 0 || (F % 16) || (out_t && (T % 16)) || T > 0x7FFFFFFFull || F > 0x3FFFFFFFull) {
-        set_error("fp8_swiglu_cast: unsupported shape T=%zu F=%zu (F %% 16 == 0; T %% 16 == 0 with a transposed copy)", T, F);
+        set_error("%s: unsupported shape T=%zu F=%zu (F %% 16 == 0; T %% 16 == 0 with a transposed copy)", who, T, F);
         return FP8_ERR_SHAPE;
     }
-    if (!aligned16(gate_up_bf16) || !aligned16(out) || !aligned16(out_t)) {
-        set_error("fp8_swiglu_cast: tensor pointers must be 16-byte aligned");
+    if (!aligned16(x) || !aligned16(out) || !aligned16(out_t)) {
+        set_error("%s: tensor pointers must be 16-byte aligned", who);
         return FP8_ERR_ALIGN;
     }
     int rc = check_arch();
@@ -186,12 +241,38 @@ extern "C" int fp8_swiglu_cast(const void *gate_up_bf16, size_t T, size_t F, con
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (amax_out) FP8_CUDA_CHECK(cudaMemsetAsync(amax_out, 0, sizeof(float), st));
     dim3 grid((unsigned)((F + ST - 1) / ST), (unsigned)((T + ST - 1) / ST));
-    const uint16_t *x = static_cast<const uint16_t *>(gate_up_bf16);
+    const uint16_t *xp = static_cast<const uint16_t *>(x);
     unsigned int *ab = reinterpret_cast<unsigned int *>(amax_out);
-    if (fmt == FP8_E4M3) swiglu_cast_kernel<0><<<grid, 256, 0, st>>>(x, (int)T, (int)F, scale, out, out_t, ab);
-    else swiglu_cast_kernel<1><<<grid, 256, 0, st>>>(x, (int)T, (int)F, scale, out, out_t, ab);
+#define FP8DPA_LAUNCH_ACT(FMT, ACT) \
+    act_cast_kernel<FMT, ACT><<<grid, 256, 0, st>>>(xp, (int)T, (int)F, act_params, scale, out, out_t, ab)
+    if (fmt == FP8_E4M3) {
+        if (act == ACT_SWIGLU) FP8DPA_LAUNCH_ACT(0, ACT_SWIGLU);
+        else if (act == FP8_ACT_GELU) FP8DPA_LAUNCH_ACT(0, FP8_ACT_GELU);
+        else FP8DPA_LAUNCH_ACT(0, FP8_ACT_XIELU);
+    } else {
+        if (act == ACT_SWIGLU) FP8DPA_LAUNCH_ACT(1, ACT_SWIGLU);
+        else if (act == FP8_ACT_GELU) FP8DPA_LAUNCH_ACT(1, FP8_ACT_GELU);
+        else FP8DPA_LAUNCH_ACT(1, FP8_ACT_XIELU);
+    }
+#undef FP8DPA_LAUNCH_ACT
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
+}
+
+extern "C" int fp8_swiglu_cast(const void *gate_up_bf16, size_t T, size_t F, const float *scale, int fmt, uint8_t *out,
+                               uint8_t *out_t, float *amax_out, void *stream)
+{
+    return act_cast("fp8_swiglu_cast", gate_up_bf16, T, F, ACT_SWIGLU, nullptr, scale, fmt, out, out_t, amax_out, stream);
+}
+
+extern "C" int fp8_act_cast(const void *x_bf16, size_t T, size_t F, int act, const float *act_params, const float *scale,
+                            int fmt, uint8_t *out, uint8_t *out_t, float *amax_out, void *stream)
+{
+    if (act != FP8_ACT_GELU && act != FP8_ACT_XIELU) {
+        set_error("fp8_act_cast: act %d is not FP8_ACT_GELU / FP8_ACT_XIELU", act);
+        return FP8_ERR_ENUM;
+    }
+    return act_cast("fp8_act_cast", x_bf16, T, F, act, act_params, scale, fmt, out, out_t, amax_out, stream);
 }
 
 extern "C" int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *out, void *stream)

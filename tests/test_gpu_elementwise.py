@@ -72,3 +72,41 @@ def test_swiglu_argument_validation():
     with pytest.raises(fp8.Fp8Error) as e:
         fp8.fp8_kurtosis(x[:, :60].contiguous(), scalar())
     assert e.value.status == -3
+
+
+@pytest.mark.parametrize("fmt", [o.E4M3, o.E5M2])
+@pytest.mark.parametrize("act", [o.GELU, o.XIELU])
+@pytest.mark.parametrize("T,F", [(256, 1024), (144, 272), (512, 8192)])
+def test_act_cast_matches_oracle(fmt, act, T, F):
+    c = synth.choose_columns(F, max(2, F // 100), 3, 9)
+    xb = synth.normal_bf16((T, F), 9, 3, 1.0, c, 8.0)
+    ap, an = 0.8125, 1.3125
+    h = o.activation(xb, act, ap, an)
+    x = dev(xb)
+    params = torch.tensor([ap, an], dtype=torch.float32, device="cuda") if act == o.XIELU else None
+    a = scalar()
+    fp8.fp8_act_cast(x, act, params, None, fmt, None, None, a)                # amax of h only
+    ea = o.amax(h)
+    assert abs(float(a.item()) - float(ea)) <= 2.0 ** -7 * float(ea)
+    s, si = scalar(), scalar()
+    fp8.fp8_scale(a, fmt, 0, s, si)
+    out = torch.empty((T, F), dtype=torch.uint8, device="cuda")
+    out_t = torch.empty((F, T), dtype=torch.uint8, device="cuda")
+    fp8.fp8_act_cast(x, act, params, s, fmt, out, out_t, None)
+    got = host(out)
+    exp = o.cast(h, float(s.item()), fmt)
+    diff = got != exp
+    assert diff.mean() <= 2e-3, diff.mean()            # FP32 erf / expm1 against double, seen through BF16 rounding
+    assert neighbours(got[diff], exp[diff], fmt).all()
+    assert np.array_equal(host(out_t), got.T)
+
+
+def test_act_cast_argument_validation():
+    x = dev(synth.normal_bf16((32, 64), 0, 0, 1.0))
+    out = torch.empty((32, 64), dtype=torch.uint8, device="cuda")
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_act_cast(x, fp8.ACT_XIELU, None, scalar(1), 0, out)           # xIELU needs its two scalars
+    assert e.value.status == -1
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_act_cast(x, 7, None, scalar(1), 0, out)
+    assert e.value.status == -4
