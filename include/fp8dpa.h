@@ -112,6 +112,30 @@ enum { FP8_ACT_GELU = 1, FP8_ACT_XIELU = 2 };
 FP8_API int fp8_act_cast(const void *x_bf16, size_t T, size_t F, int act, const float *act_params, const float *scale,
                  int fmt, uint8_t *out, uint8_t *out_t, float *amax_out, void *stream);
 
+/* Post-normalisation and residual connection of the block (Section 3; Appendix B: X^ = X + (N_post o GQA)(X),
+ * block(X) = X^ + (N_post o FFN)(X^)), fused with the amax of the result, which is the operand of the next FP8
+ * GEMM since these architectures have no pre-normalisation:
+ *   FP8_NORM_RMS         out = x + gamma (.) y / sqrt(mean(y^2) + eps)      (eps = 0 is the paper's N_gamma)
+ *   FP8_NORM_LAYERSCALE  out = x + gamma (.) y
+ * x, y, out: [T,D] BF16 device tensors (out may alias x); gamma: D binary32 on the device; *amax_out (nullable) is
+ * overwritten with amax(out).  D % 8 == 0, D <= 16384. */
+enum { FP8_NORM_RMS = 0, FP8_NORM_LAYERSCALE = 1 };
+FP8_API int fp8_postnorm_residual(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D,
+                          int mode, float eps, void *out_bf16, float *amax_out, void *stream);
+
+/* QK entropy regulariser and rotary embedding of per-head query / key vectors (Section 3; Appendix B:
+ * attnhead = selfattn(N_QK(X W_Q), N_QK(X W_K), X W_V) with rotary position embeddings), fused with the amax that
+ * the FP8 cast of Q / K needs.  x, out: [T,H,d] BF16 (out may alias x), d in {64, 128}.
+ *   FP8_QK_RMS   v / sqrt(mean(v^2) + eps) over the d entries of a head (unit gain: a frozen gain is folded into
+ *                the softmax scale, Section 3.1)        FP8_QK_TANH  tanh(alpha v)        FP8_QK_NONE  v
+ * then, if cos_table != NULL, the pairs (i, i + d/2) are rotated by the angle of position t mod seq_len:
+ * out[i] = v[i] c - v[i+d/2] s, out[i+d/2] = v[i+d/2] c + v[i] s with c, s = cos/sin_table[pos, i]
+ * ([seq_len, d/2] binary32 on the device, supplied by the caller).  *amax_out (nullable) = amax(out). */
+enum { FP8_QK_RMS = 0, FP8_QK_TANH = 1, FP8_QK_NONE = 2 };
+FP8_API int fp8_qk_norm_rope(const void *x_bf16, size_t T, size_t H, size_t d, int mode, float alpha, float eps,
+                     const float *cos_table, const float *sin_table, size_t seq_len, void *out_bf16,
+                     float *amax_out, void *stream);
+
 /* Kurtosis monitor (Section 4): *out = mean over rows of mu[x^4] / mu[x^2]^2 of a [rows, cols] BF16 tensor
  * (un-centred; rows are token vectors).  *out is overwritten.  cols % 8 == 0. */
 FP8_API int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *out, void *stream);

@@ -158,6 +158,34 @@ def swiglu(gate_up_bf16: np.ndarray) -> np.ndarray:
 
 
 GELU, XIELU = 1, 2
+NORM_RMS, NORM_LAYERSCALE = 0, 1
+QK_RMS, QK_TANH, QK_NONE = 0, 1, 2
+
+
+def postnorm_residual(x_bf16, y_bf16, gamma, mode: int = NORM_RMS, eps: float = 0.0) -> np.ndarray:
+    """x + gamma * y / rms(y) (mode 0) or x + gamma * y (mode 1), rounded to BF16 (Section 3, Appendix B)."""
+    x, y = _c(x_bf16, np.uint16), _c(y_bf16, np.uint16)
+    g = _c(gamma, np.float32)
+    T, D = x.shape
+    out = np.empty_like(x)
+    f = _L().oracle_postnorm_residual_bf16
+    f.restype = None
+    f(_p(x), _p(y), _p(g), C.c_size_t(T), C.c_size_t(D), C.c_int(mode), C.c_double(eps), _p(out))
+    return out
+
+
+def qk_norm_rope(x_bf16, mode: int, alpha: float, eps: float, cos=None, sin=None, seq_len: int = 1) -> np.ndarray:
+    """QK regulariser (per-head RMS norm / tanh(alpha x) / none) then rotary embedding on [T,H,d] BF16."""
+    x = _c(x_bf16, np.uint16)
+    T, H, d = x.shape
+    out = np.empty_like(x)
+    c = _c(cos, np.float32) if cos is not None else None
+    s_ = _c(sin, np.float32) if sin is not None else None
+    f = _L().oracle_qk_norm_rope_bf16
+    f.restype = None
+    f(_p(x), C.c_size_t(T), C.c_size_t(H), C.c_size_t(d), C.c_int(mode), C.c_double(alpha), C.c_double(eps),
+      _p(c) if c is not None else None, _p(s_) if s_ is not None else None, C.c_size_t(seq_len), _p(out))
+    return out
 
 
 def activation(x_bf16: np.ndarray, act: int, alpha_p: float = 0.0, alpha_n: float = 0.0) -> np.ndarray:

@@ -249,6 +249,76 @@ void oracle_activation_bf16(const uint16_t *x, size_t n, int act, double alpha_p
 }
 
 /* ------------------------------------------------------------------------------------------------
+ * Post-normalisation + residual (Section 3; Appendix B: block(X) = X^ + (N_post o FFN)(X^), X^ = X + (N_post o GQA)(X)):
+ *   mode 0  RMSNorm     out = x + gamma (.) y / rms(y),  rms(y) = sqrt(mean(y^2) + eps)   (the paper's N_gamma has eps = 0)
+ *   mode 1  LayerScale  out = x + gamma (.) y
+ * x (residual stream), y (branch output): [T,D] BF16; gamma: D binary32; out rounded to BF16.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_postnorm_residual_bf16(const uint16_t *x, const uint16_t *y, const float *gamma, size_t T, size_t D,
+                                   int mode, double eps, uint16_t *out)
+{
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < (long)T; ++t) {
+        double ss = 0.0;
+        for (size_t d = 0; d < D; ++d) {
+            double v = (double)bf16_bits_to_float(y[(size_t)t * D + d]);
+            ss += v * v;
+        }
+        double rinv = mode == 0 ? 1.0 / sqrt(ss / (double)D + eps) : 1.0;
+        for (size_t d = 0; d < D; ++d) {
+            double r = (double)bf16_bits_to_float(x[(size_t)t * D + d]) +
+                       (double)gamma[d] * (double)bf16_bits_to_float(y[(size_t)t * D + d]) * rinv;
+            out[(size_t)t * D + d] = f32_to_bf16_rne((float)r);
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * QK entropy regulariser + rotary embedding on a [T, H, d] BF16 tensor of per-head vectors (Section 3, Appendix B:
+ * attnhead = selfattn(N_QK(X W_Q), N_QK(X W_K), X W_V), "standard" GQA with rotary position embeddings):
+ *   mode 0  N(v) = v / rms(v)  over the d entries of one head (frozen unit gain: the gain lives in the softmax scale)
+ *   mode 1  tanh(alpha v) element-wise
+ *   mode 2  identity
+ * then rotation of the pairs (i, i + d/2) by the angle of position pos = t mod seq_len:
+ *   out[i]       = v[i] cos[pos,i] - v[i+d/2] sin[pos,i]
+ *   out[i+d/2]   = v[i+d/2] cos[pos,i] + v[i] sin[pos,i]         cos, sin: [seq_len, d/2] binary32 tables (inputs)
+ * rounded to BF16.  cos == NULL skips the rotation.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_qk_norm_rope_bf16(const uint16_t *x, size_t T, size_t H, size_t d, int mode, double alpha, double eps,
+                              const float *cos_t, const float *sin_t, size_t seq_len, uint16_t *out)
+{
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < (long)T; ++t) {
+        double v[1024];
+        for (size_t h = 0; h < H; ++h) {
+            const uint16_t *px = x + ((size_t)t * H + h) * d;
+            uint16_t *po = out + ((size_t)t * H + h) * d;
+            double ss = 0.0;
+            for (size_t i = 0; i < d; ++i) {
+                v[i] = (double)bf16_bits_to_float(px[i]);
+                ss += v[i] * v[i];
+            }
+            if (mode == 0) {
+                double rinv = 1.0 / sqrt(ss / (double)d + eps);
+                for (size_t i = 0; i < d; ++i) v[i] *= rinv;
+            } else if (mode == 1) {
+                for (size_t i = 0; i < d; ++i) v[i] = tanh(alpha * v[i]);
+            }
+            if (cos_t) {
+                size_t pos = (size_t)t % seq_len, hd = d / 2;
+                for (size_t i = 0; i < hd; ++i) {
+                    double c = (double)cos_t[pos * hd + i], sn = (double)sin_t[pos * hd + i];
+                    double a = v[i], b = v[i + hd];
+                    v[i] = a * c - b * sn;
+                    v[i + hd] = b * c + a * sn;
+                }
+            }
+            for (size_t i = 0; i < d; ++i) po[i] = f32_to_bf16_rne((float)v[i]);
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------------
  * FP8 GEMM with descale (Appendix E): ref[i,j] = sa_inv*sb_inv * sum_k dec(A[i,k]) * dec(B[j,k]),
  * accumulated in double, on a list of output rows and columns.  A and B are addressed through
  * (row stride, reduction stride) so that the three linear products are this one routine on three

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
-           "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_kurtosis",
+           "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_qk_norm_rope", "fp8_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
@@ -118,6 +118,23 @@ def fp8_quantize(x, fmt, out, out_t, amax, scale, scale_inv, stream=None):
 
 
 ACT_GELU, ACT_XIELU = 1, 2
+NORM_RMS, NORM_LAYERSCALE = 0, 1
+QK_RMS, QK_TANH, QK_NONE = 0, 1, 2
+
+
+def fp8_postnorm_residual(x, y, gamma, mode, eps, out, amax_out=None, stream=None):
+    """out = x + gamma * y / rms(y) (NORM_RMS) or x + gamma * y (NORM_LAYERSCALE); [T, D] BF16, amax of out optional."""
+    T, D = x.shape
+    _check(load().fp8_postnorm_residual(_ptr(x), _ptr(y), _ptr(gamma), C.c_size_t(T), C.c_size_t(D), C.c_int(mode),
+                                        C.c_float(eps), _ptr(out), _ptr(amax_out), _stream(stream)))
+
+
+def fp8_qk_norm_rope(x, mode, alpha, eps, cos_table, sin_table, seq_len, out, amax_out=None, stream=None):
+    """QK regulariser (per-head RMS norm / tanh(alpha x) / none) + rotary embedding on [T, H, d] BF16."""
+    T, H, d = x.shape
+    _check(load().fp8_qk_norm_rope(_ptr(x), C.c_size_t(T), C.c_size_t(H), C.c_size_t(d), C.c_int(mode),
+                                   C.c_float(alpha), C.c_float(eps), _ptr(cos_table), _ptr(sin_table),
+                                   C.c_size_t(seq_len), _ptr(out), _ptr(amax_out), _stream(stream)))
 
 
 def fp8_act_cast(x, act, act_params, scale, fmt, out, out_t=None, amax_out=None, stream=None):

@@ -212,6 +212,161 @@ __global__ void __launch_bounds__(256) kurtosis_kernel(const uint16_t *__restric
     }
 }
 
+// Post-norm + residual, one CTA per token row.  The row of y stays in registers between the sum of squares and the
+// update: KG 16-byte groups per thread at 256 threads (KG = 1, 2, 4, 8 for up to 2048 ... 16384 columns, chosen at
+// launch so that short rows do not pay for the registers of long ones).
+template <int MODE, int KG>
+__global__ void __launch_bounds__(256) postnorm_residual_kernel(const uint16_t *__restrict__ x,
+                                                                const uint16_t *__restrict__ y,
+                                                                const float *__restrict__ gamma, int D, float eps,
+                                                                uint16_t *__restrict__ out,
+                                                                unsigned int *__restrict__ amax_bits)
+{
+    __shared__ float red[8];
+    const size_t base = (size_t)blockIdx.x * D;
+    const uint4 *py = reinterpret_cast<const uint4 *>(y + base);
+    const uint4 *px = reinterpret_cast<const uint4 *>(x + base);
+    uint4 *po = reinterpret_cast<uint4 *>(out + base);
+    const int n8 = D / 8;
+    uint4 yv[KG], xv8[KG];
+    float ss = 0.0f;
+#pragma unroll
+    for (int k = 0; k < KG; ++k) {
+        const int i = k * 256 + threadIdx.x;
+        if (i < n8) {
+            yv[k] = __ldg(py + i);
+            xv8[k] = __ldg(px + i);       // in flight during the reduction
+            const uint32_t w[4] = {yv[k].x, yv[k].y, yv[k].z, yv[k].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float a = bf16_lo(w[q]), b = bf16_hi(w[q]);
+                ss = fmaf(a, a, fmaf(b, b, ss));
+            }
+        }
+    }
+    float rinv = 1.0f;
+    if (MODE == FP8_NORM_RMS) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        float tot = 0.0f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) tot += red[w];
+        rinv = 1.0f / sqrtf(tot / (float)D + eps);
+    }
+    uint32_t m = 0;
+#pragma unroll
+    for (int k = 0; k < KG; ++k) {
+        const int i = k * 256 + threadIdx.x;
+        if (i < n8) {
+            const uint4 xv = xv8[k];
+            const float4 g0 = __ldg(reinterpret_cast<const float4 *>(gamma) + 2 * i);
+            const float4 g1 = __ldg(reinterpret_cast<const float4 *>(gamma) + 2 * i + 1);
+            const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+            const uint32_t yw[4] = {yv[k].x, yv[k].y, yv[k].z, yv[k].w}, xw[4] = {xv.x, xv.y, xv.z, xv.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float lo = fmaf(g[2 * q] * rinv, bf16_lo(yw[q]), bf16_lo(xw[q]));
+                const float hi = fmaf(g[2 * q + 1] * rinv, bf16_hi(yw[q]), bf16_hi(xw[q]));
+                o[q] = pack_bf16x2(lo, hi);
+                m = absmax2e(m, o[q]);
+            }
+            po[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
+    if (amax_bits) block_max_bf16_to(m, amax_bits);
+}
+
+// QK regulariser + rotary embedding.  A (token, head) vector is handled by D/16 adjacent lanes: lane j of the group
+// holds elements [8j, 8j+8) of the first half and the same of the second half (two 16-byte loads), so the rotation
+// partner i + D/2 of every element lives in the same lane and the sum of squares needs log2(D/16) shuffles.
+// A lane group takes QK_HC consecutive heads of one token, so the 16 cos/sin values of its position are read once
+// per QK_HC vectors.
+constexpr int QK_HC = 8;
+template <int D, int MODE>
+__global__ void __launch_bounds__(256) qk_norm_rope_kernel(const uint16_t *__restrict__ x, size_t n_tok, int H,
+                                                           float alpha, float eps, const float *__restrict__ cos_t,
+                                                           const float *__restrict__ sin_t, int seq_len,
+                                                           uint16_t *__restrict__ out,
+                                                           unsigned int *__restrict__ amax_bits)
+{
+    constexpr int LPV = D / 16;             // lanes per vector: 8 (d = 128) or 4 (d = 64)
+    constexpr int GPB = 256 / LPV;          // lane groups per CTA
+    const int j = threadIdx.x % LPV;
+    const int chunks = (H + QK_HC - 1) / QK_HC;
+    const size_t n_items = n_tok * (size_t)chunks;            // (token, chunk of heads)
+    uint32_t m = 0;
+    // The trip counts are uniform over the CTA (the shuffles below name every lane of the warp): a lane group past
+    // the end re-reads the last vector and stores nothing.
+    for (size_t base = (size_t)blockIdx.x * GPB; base < n_items; base += (size_t)gridDim.x * GPB) {
+        const size_t item_raw = base + threadIdx.x / LPV;
+        const bool item_valid = item_raw < n_items;
+        const size_t item = item_valid ? item_raw : n_items - 1;
+        const size_t tok = item / (size_t)chunks;
+        const int h0 = (int)(item % (size_t)chunks) * QK_HC;
+        float c[8], sn[8];
+        if (cos_t) {
+            const size_t pos = tok % (size_t)seq_len;
+            const float4 *pc = reinterpret_cast<const float4 *>(cos_t + pos * (D / 2) + j * 8);
+            const float4 *ps = reinterpret_cast<const float4 *>(sin_t + pos * (D / 2) + j * 8);
+            const float4 c0 = __ldg(pc), c1 = __ldg(pc + 1), s0 = __ldg(ps), s1 = __ldg(ps + 1);
+            c[0] = c0.x; c[1] = c0.y; c[2] = c0.z; c[3] = c0.w; c[4] = c1.x; c[5] = c1.y; c[6] = c1.z; c[7] = c1.w;
+            sn[0] = s0.x; sn[1] = s0.y; sn[2] = s0.z; sn[3] = s0.w; sn[4] = s1.x; sn[5] = s1.y; sn[6] = s1.z; sn[7] = s1.w;
+        }
+#pragma unroll 2
+        for (int hh = 0; hh < QK_HC; ++hh) {
+            const bool valid = item_valid && h0 + hh < H;
+            const size_t v = tok * (size_t)H + (size_t)min(h0 + hh, H - 1);
+            const uint16_t *px = x + v * D + j * 8;
+            const uint4 wa = __ldg(reinterpret_cast<const uint4 *>(px));
+            const uint4 wb = __ldg(reinterpret_cast<const uint4 *>(px + D / 2));
+            const uint32_t ua[4] = {wa.x, wa.y, wa.z, wa.w}, ub[4] = {wb.x, wb.y, wb.z, wb.w};
+            float a[8], b[8];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                a[2 * q] = bf16_lo(ua[q]); a[2 * q + 1] = bf16_hi(ua[q]);
+                b[2 * q] = bf16_lo(ub[q]); b[2 * q + 1] = bf16_hi(ub[q]);
+            }
+            if (MODE == FP8_QK_RMS) {
+                float ss = 0.0f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ss = fmaf(a[e], a[e], fmaf(b[e], b[e], ss));
+#pragma unroll
+                for (int off = LPV / 2; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+                const float rinv = 1.0f / sqrtf(ss / (float)D + eps);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { a[e] *= rinv; b[e] *= rinv; }
+            } else if (MODE == FP8_QK_TANH) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { a[e] = tanhf(alpha * a[e]); b[e] = tanhf(alpha * b[e]); }
+            }
+            if (cos_t) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float ra = a[e] * c[e] - b[e] * sn[e], rb = b[e] * c[e] + a[e] * sn[e];
+                    a[e] = ra;
+                    b[e] = rb;
+                }
+            }
+            uint32_t oa[4], ob[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                oa[q] = pack_bf16x2(a[2 * q], a[2 * q + 1]);
+                ob[q] = pack_bf16x2(b[2 * q], b[2 * q + 1]);
+                if (valid) m = absmax2e(absmax2e(m, oa[q]), ob[q]);
+            }
+            if (valid) {
+                uint16_t *po = out + v * D + j * 8;
+                *reinterpret_cast<uint4 *>(po) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
+                *reinterpret_cast<uint4 *>(po + D / 2) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+            }
+        }
+    }
+    if (amax_bits) block_max_bf16_to(m, amax_bits);
+}
+
 }  // namespace fp8dpa
 
 using namespace fp8dpa;
@@ -295,6 +450,99 @@ extern "C" int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float 
     FP8_CUDA_CHECK(cudaMemsetAsync(out, 0, sizeof(float), st));
     kurtosis_kernel<<<(unsigned)rows, 256, 0, st>>>(static_cast<const uint16_t *>(x_bf16), (int)cols,
                                                    1.0f / (float)rows, out);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+extern "C" int fp8_postnorm_residual(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D,
+                                     int mode, float eps, void *out_bf16, float *amax_out, void *stream)
+{
+    if (!x_bf16 || !y_bf16 || !gamma || !out_bf16) {
+        set_error("fp8_postnorm_residual: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if (mode != FP8_NORM_RMS && mode != FP8_NORM_LAYERSCALE) {
+        set_error("fp8_postnorm_residual: mode %d is not FP8_NORM_RMS / FP8_NORM_LAYERSCALE", mode);
+        return FP8_ERR_ENUM;
+    }
+    if (T == 0 || D == 0 || (D % 8) || D > 16384 || T > 0x7FFFFFFFull || !(eps >= 0.0f)) {
+        set_error("fp8_postnorm_residual: unsupported shape T=%zu D=%zu (D %% 8 == 0, D <= 16384) or eps < 0", T, D);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(x_bf16) || !aligned16(y_bf16) || !aligned16(gamma) || !aligned16(out_bf16)) {
+        set_error("fp8_postnorm_residual: pointers must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (amax_out) FP8_CUDA_CHECK(cudaMemsetAsync(amax_out, 0, sizeof(float), st));
+    const uint16_t *x = static_cast<const uint16_t *>(x_bf16), *y = static_cast<const uint16_t *>(y_bf16);
+    uint16_t *o = static_cast<uint16_t *>(out_bf16);
+    unsigned int *ab = reinterpret_cast<unsigned int *>(amax_out);
+#define FP8DPA_LAUNCH_PN(MM, KG) \
+    postnorm_residual_kernel<MM, KG><<<(unsigned)T, 256, 0, st>>>(x, y, gamma, (int)D, eps, o, ab)
+#define FP8DPA_LAUNCH_PN_KG(MM) \
+    do { \
+        if (D <= 2048) FP8DPA_LAUNCH_PN(MM, 1); \
+        else if (D <= 4096) FP8DPA_LAUNCH_PN(MM, 2); \
+        else if (D <= 8192) FP8DPA_LAUNCH_PN(MM, 4); \
+        else FP8DPA_LAUNCH_PN(MM, 8); \
+    } while (0)
+    if (mode == FP8_NORM_RMS) FP8DPA_LAUNCH_PN_KG(FP8_NORM_RMS);
+    else FP8DPA_LAUNCH_PN_KG(FP8_NORM_LAYERSCALE);
+#undef FP8DPA_LAUNCH_PN_KG
+#undef FP8DPA_LAUNCH_PN
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+extern "C" int fp8_qk_norm_rope(const void *x_bf16, size_t T, size_t H, size_t d, int mode, float alpha, float eps,
+                                const float *cos_table, const float *sin_table, size_t seq_len, void *out_bf16,
+                                float *amax_out, void *stream)
+{
+    if (!x_bf16 || !out_bf16 || ((cos_table == nullptr) != (sin_table == nullptr))) {
+        set_error("fp8_qk_norm_rope: NULL pointer (cos and sin tables come together)");
+        return FP8_ERR_NULL;
+    }
+    if (mode < FP8_QK_RMS || mode > FP8_QK_NONE) {
+        set_error("fp8_qk_norm_rope: mode %d is not FP8_QK_RMS / FP8_QK_TANH / FP8_QK_NONE", mode);
+        return FP8_ERR_ENUM;
+    }
+    if (T == 0 || H == 0 || (d != 64 && d != 128) || (cos_table && seq_len == 0) || H > 65535 || !(eps >= 0.0f) ||
+        seq_len > 0x7FFFFFFFull) {
+        set_error("fp8_qk_norm_rope: unsupported shape T=%zu H=%zu d=%zu seq_len=%zu (d in {64,128})", T, H, d, seq_len);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(x_bf16) || !aligned16(out_bf16) || !aligned16(cos_table) || !aligned16(sin_table)) {
+        set_error("fp8_qk_norm_rope: pointers must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (amax_out) FP8_CUDA_CHECK(cudaMemsetAsync(amax_out, 0, sizeof(float), st));
+    const size_t gpb = 256 / (d / 16);          // lane groups per CTA, each taking QK_HC heads of one token
+    const size_t n_items = T * ((H + QK_HC - 1) / QK_HC);
+    size_t blocks = (n_items + gpb - 1) / gpb;
+    const size_t cap = (size_t)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    const uint16_t *x = static_cast<const uint16_t *>(x_bf16);
+    uint16_t *o = static_cast<uint16_t *>(out_bf16);
+    unsigned int *ab = reinterpret_cast<unsigned int *>(amax_out);
+#define FP8DPA_LAUNCH_QK(DD, MM) \
+    qk_norm_rope_kernel<DD, MM><<<(unsigned)blocks, 256, 0, st>>>(x, T, (int)H, alpha, eps, cos_table, sin_table, \
+                                                                 (int)(seq_len ? seq_len : 1), o, ab)
+    if (d == 128) {
+        if (mode == FP8_QK_RMS) FP8DPA_LAUNCH_QK(128, FP8_QK_RMS);
+        else if (mode == FP8_QK_TANH) FP8DPA_LAUNCH_QK(128, FP8_QK_TANH);
+        else FP8DPA_LAUNCH_QK(128, FP8_QK_NONE);
+    } else {
+        if (mode == FP8_QK_RMS) FP8DPA_LAUNCH_QK(64, FP8_QK_RMS);
+        else if (mode == FP8_QK_TANH) FP8DPA_LAUNCH_QK(64, FP8_QK_TANH);
+        else FP8DPA_LAUNCH_QK(64, FP8_QK_NONE);
+    }
+#undef FP8DPA_LAUNCH_QK
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }

@@ -110,3 +110,70 @@ def test_act_cast_argument_validation():
     with pytest.raises(fp8.Fp8Error) as e:
         fp8.fp8_act_cast(x, 7, None, scalar(1), 0, out)
     assert e.value.status == -4
+
+
+def bf16_close(got_bits, exp_bits, max_frac=2e-3):
+    """Equal BF16 tensors except for at most `max_frac` of elements that differ by one BF16 step."""
+    g = got_bits.astype(np.int32).ravel()
+    e = exp_bits.astype(np.int32).ravel()
+    diff = g != e
+    assert diff.mean() <= max_frac, diff.mean()
+    # sign-magnitude ordering: one step apart (or +0 / -0)
+    key = lambda b: np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+    assert np.all(np.abs(key(g[diff]) - key(e[diff])) <= 1)
+
+
+@pytest.mark.parametrize("mode,eps", [(o.NORM_RMS, 0.0), (o.NORM_RMS, 1e-5), (o.NORM_LAYERSCALE, 0.0)])
+@pytest.mark.parametrize("T,D", [(64, 2048), (100, 4096), (7, 264), (16, 16384)])
+def test_postnorm_residual_matches_oracle(mode, eps, T, D):
+    c = synth.choose_columns(D, max(1, D // 200), 4, 1)
+    xb = synth.normal_bf16((T, D), 10, 1, 1.0, c, 20.0)
+    yb = synth.normal_bf16((T, D), 10, 2, 0.02, c, 20.0)
+    gamma = (np.full(D, 1.0 / np.sqrt(32.0)) * (1.0 + 0.01 * np.arange(D) / D)).astype(np.float32)
+    exp = o.postnorm_residual(xb, yb, gamma, mode, eps)
+    out = torch.empty((T, D), dtype=torch.int16, device="cuda")
+    a = scalar(-1.0)
+    fp8.fp8_postnorm_residual(dev(xb), dev(yb), torch.from_numpy(gamma).cuda(), mode, eps, out, a)
+    got = host(out).view(np.uint16)
+    bf16_close(got, exp)
+    assert float(a.item()) == float(o.amax(got))            # amax of what was written
+    # in place on the residual stream
+    xio = dev(xb)
+    fp8.fp8_postnorm_residual(xio, dev(yb), torch.from_numpy(gamma).cuda(), mode, eps, xio, None)
+    assert np.array_equal(host(xio).view(np.uint16), got)
+
+
+@pytest.mark.parametrize("mode", [o.QK_RMS, o.QK_TANH, o.QK_NONE])
+@pytest.mark.parametrize("rope", [True, False])
+@pytest.mark.parametrize("T,H,d,N", [(256, 8, 128, 64), (96, 4, 64, 32), (33, 3, 128, 11)])
+def test_qk_norm_rope_matches_oracle(mode, rope, T, H, d, N):
+    xb = synth.normal_bf16((T, H * d), 12, 3, 1.5).reshape(T, H, d)
+    inv = 10000.0 ** (-np.arange(d // 2) * 2.0 / d)
+    ang = np.arange(N)[:, None] * inv[None]
+    cos, sin = np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)
+    exp = o.qk_norm_rope(xb, mode, 0.5, 1e-6, cos if rope else None, sin if rope else None, N)
+    out = torch.empty((T, H, d), dtype=torch.int16, device="cuda")
+    a = scalar(-1.0)
+    fp8.fp8_qk_norm_rope(dev(xb), mode, 0.5, 1e-6, torch.from_numpy(cos).cuda() if rope else None,
+                         torch.from_numpy(sin).cuda() if rope else None, N, out, a)
+    got = host(out).view(np.uint16)
+    bf16_close(got, exp, 4e-3 if mode == o.QK_TANH else 2e-3)
+    assert float(a.item()) == float(o.amax(got))
+
+
+def test_glue_argument_validation():
+    x = dev(synth.normal_bf16((8, 64), 0, 0, 1.0))
+    g = torch.ones(64, device="cuda")
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_postnorm_residual(x, x, g, 5, 0.0, x)
+    assert e.value.status == -4
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_postnorm_residual(x[:, :60].contiguous(), x[:, :60].contiguous(), g, 0, 0.0, x)
+    assert e.value.status == -3
+    q = x.view(8, 1, 64)
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_qk_norm_rope(q, 0, 0.0, 0.0, g, None, 4, q)           # cos without sin
+    assert e.value.status == -1
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_qk_norm_rope(x.view(8, 2, 32), 0, 0.0, 0.0, None, None, 1, x.view(8, 2, 32))
+    assert e.value.status == -3

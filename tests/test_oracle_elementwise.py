@@ -82,3 +82,63 @@ def test_xielu_values_and_limits():
     # alpha_p = alpha_n = 0 is x / 2
     z = synth.bf16_to_f32(o.activation(bf16(x), o.XIELU, 0.0, 0.0))[0]
     assert np.array_equal(z, x[0] * 0.5)
+
+
+def test_postnorm_residual_closed_forms():
+    D = 64
+    x = np.arange(D, dtype=np.float64)[None] * 0.25
+    g = np.full(D, 0.5, dtype=np.float32)
+    # constant branch output: y / rms(y) = sign(y)
+    out = synth.bf16_to_f32(o.postnorm_residual(bf16(x), bf16(np.full((1, D), -3.0)), g))
+    assert np.array_equal(out, x - 0.5)
+    # one non-zero entry a: rms = |a| / sqrt(D), so that entry becomes sqrt(D) = 8
+    y = np.zeros((1, D)); y[0, 5] = 0.75
+    out = synth.bf16_to_f32(o.postnorm_residual(bf16(x), bf16(y), g))
+    exp = x.copy(); exp[0, 5] += 0.5 * 8.0
+    assert np.array_equal(out, exp)
+    # scale invariance in y (powers of two are exact), and eps breaks it the right way
+    yy = synth.normal_bf16((8, D), 3, 4, 1.0)
+    xx = synth.normal_bf16((8, D), 3, 5, 1.0)
+    y4 = bf16(4.0 * synth.bf16_to_f32(yy))
+    assert np.array_equal(o.postnorm_residual(xx, yy, g), o.postnorm_residual(xx, y4, g))
+    big_eps = synth.bf16_to_f32(o.postnorm_residual(xx, yy, g, o.NORM_RMS, 1e6))
+    assert np.allclose(big_eps, synth.bf16_to_f32(xx), atol=0.01)          # y / sqrt(1e6) vanishes
+    # LayerScale: x + gamma * y, exact on these values
+    out = synth.bf16_to_f32(o.postnorm_residual(bf16(x), bf16(np.full((1, D), 2.0)), g, o.NORM_LAYERSCALE))
+    assert np.array_equal(out, x + 1.0)
+    # against numpy on random data
+    xf, yf = synth.bf16_to_f32(xx).astype(np.float64), synth.bf16_to_f32(yy).astype(np.float64)
+    ref = xf + 0.5 * yf / np.sqrt((yf ** 2).mean(axis=1, keepdims=True) + 1e-5)
+    got = synth.bf16_to_f32(o.postnorm_residual(xx, yy, g, o.NORM_RMS, 1e-5))
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-30)
+
+
+def test_qk_norm_rope_closed_forms():
+    T, H, d, N = 6, 2, 64, 3
+    q = synth.normal_bf16((T, H * d), 5, 6, 2.0).reshape(T, H, d)
+    qf = synth.bf16_to_f32(q).astype(np.float64)
+    # RMS norm without rotation: unit mean square per head
+    out = synth.bf16_to_f32(o.qk_norm_rope(q, o.QK_RMS, 0.0, 0.0)).astype(np.float64)
+    assert np.allclose((out ** 2).mean(axis=2), 1.0, atol=5e-3)
+    assert np.all(np.abs(out - qf / np.sqrt((qf ** 2).mean(axis=2, keepdims=True))) <= 2.0 ** -8 * np.abs(out) + 1e-30)
+    # tanh regulariser: values
+    v = np.zeros((1, 1, d)); v[0, 0, :4] = [2.0, -2.0, 0.0, 1.0]
+    out = synth.bf16_to_f32(o.qk_norm_rope(bf16(v), o.QK_TANH, 0.5, 0.0))[0, 0]
+    assert abs(out[0] - 0.761594) < 3e-3 and out[1] == -out[0] and out[2] == 0.0 and abs(out[3] - 0.462117) < 2e-3
+    # quarter turn at every frequency: (a, b) -> (-b, a); identity at angle 0; position = t mod seq_len
+    cos = np.zeros((N, d // 2), dtype=np.float32); sin = np.zeros((N, d // 2), dtype=np.float32)
+    cos[0] = 1.0                              # position 0: no rotation
+    sin[1] = 1.0                              # position 1: 90 degrees
+    cos[2] = -1.0                             # position 2: 180 degrees
+    out = synth.bf16_to_f32(o.qk_norm_rope(q, o.QK_NONE, 0.0, 0.0, cos, sin, N))
+    f = synth.bf16_to_f32(q)
+    for t in range(T):
+        a, b = f[t, :, :d // 2], f[t, :, d // 2:]
+        exp = {0: (a, b), 1: (-b, a), 2: (-a, -b)}[t % N]
+        assert np.array_equal(out[t, :, :d // 2], exp[0]) and np.array_equal(out[t, :, d // 2:], exp[1])
+    # a rotation keeps the length of every pair
+    th = np.linspace(0.1, 3.0, N * d // 2).reshape(N, d // 2)
+    out = synth.bf16_to_f32(o.qk_norm_rope(q, o.QK_NONE, 0.0, 0.0, np.cos(th), np.sin(th), N)).astype(np.float64)
+    n_in = qf[:, :, :d // 2] ** 2 + qf[:, :, d // 2:] ** 2
+    n_out = out[:, :, :d // 2] ** 2 + out[:, :, d // 2:] ** 2
+    assert np.allclose(n_in, n_out, rtol=2e-2, atol=1e-6)
