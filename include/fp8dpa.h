@@ -162,6 +162,19 @@ FP8_API int fp8_linear_wgrad(const uint8_t *dY8t, const uint8_t *X8t, const floa
                      void *dW, int out_is_fp32, int accumulate, int T, int N, int K,
                      void *ws, size_t ws_bytes, void *stream);
 
+/* Producer forms for delayed scaling (Appendix E: rho comes from the amax history, so the producer of a tensor can
+ * emit FP8 in its own epilogue, "a single pass on the data", Section 2).  Same products as fp8_linear_fwd /
+ * fp8_linear_dgrad; the result is rounded to BF16 (the tensor an unfused chain would store), its amax is written to
+ * *y_amax (nullable; overwritten; feed it to fp8_scale_update for the next step), and the codes
+ * sat_rne_fmt(float(bf16 result) * *y_scale) go to Y8 [T,N] (dX8 [T,K]).  The codes and the amax are bit-identical
+ * to fp8_linear_fwd (BF16 output) followed by fp8_cast with the same scale. */
+FP8_API int fp8_linear_fwd_q(const uint8_t *X8, const uint8_t *W8, const float *sX_inv, const float *sW_inv,
+                     const float *y_scale, int y_fmt, uint8_t *Y8, float *y_amax, int T, int N, int K,
+                     void *stream);
+FP8_API int fp8_linear_dgrad_q(const uint8_t *dY8, const uint8_t *W8t, const float *sdY_inv, const float *sW_inv,
+                       const float *dx_scale, int dx_fmt, uint8_t *dX8, float *dx_amax, int T, int N, int K,
+                       void *stream);
+
 /* ---- attention ------------------------------------------------------------------------------------
  * Appendix B, Eq. (P): P = Softmax(s Q K^T + M), output P V, grouped-query heads; Appendix E table: both
  * products in FP8, forward and backward.  Tensors are [B, N, H, d] row-major; query head h reads KV head
@@ -188,6 +201,14 @@ FP8_API size_t fp8_attention_workspace_bytes(int op, int B, int N, int Hq, int H
 FP8_API int fp8_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const fp8_attn_scales *sc,
                       int causal, int B, int N, int Hq, int Hkv, int d,
                       void *O_bf16, float *LSE, void *ws, size_t ws_bytes, void *stream);
+
+/* Producer form of the forward for delayed scaling (Appendix E; "a single pass", Section 2): besides O (BF16, still
+ * needed by the backward) and LSE it writes O8[B,N,Hq,d] = sat_rne_e4m3(float(O) * *o_scale), the operand of the
+ * output projection, and *o_amax = amax(O) (nullable, overwritten).  Bit-identical to fp8_attention_fwd followed by
+ * fp8_cast(O, o_scale, FP8_E4M3, amax_out). */
+FP8_API int fp8_attention_fwd_q(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const fp8_attn_scales *sc,
+                        int causal, int B, int N, int Hq, int Hkv, int d, void *O_bf16, float *LSE,
+                        const float *o_scale, uint8_t *O8, float *o_amax, void *stream);
 
 FP8_API int fp8_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const uint8_t *dO8,
                       const void *O_bf16, const float *LSE, const fp8_attn_scales *sc,

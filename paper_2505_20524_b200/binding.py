@@ -21,8 +21,8 @@ _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_qk_norm_rope", "fp8_kurtosis",
-           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_attention_workspace_bytes",
-           "fp8_attention_fwd", "fp8_attention_bwd", "fp8_attention_bwd_static"]
+           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_attention_workspace_bytes",
+           "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -171,6 +171,23 @@ def fp8_linear_fwd(x8, w8, sx_inv, sw_inv, y, ws=None, stream=None):
                                  C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()), _stream(stream)))
 
 
+def fp8_linear_fwd_q(x8, w8, sx_inv, sw_inv, y_scale, y_fmt, y8, y_amax=None, stream=None):
+    """Forward product emitting FP8 codes of the BF16-rounded result under a caller (delayed) scale, plus its amax."""
+    T, K = x8.shape
+    N = w8.shape[0]
+    _check(load().fp8_linear_fwd_q(_ptr(x8), _ptr(w8), _ptr(sx_inv), _ptr(sw_inv), _ptr(y_scale), C.c_int(y_fmt),
+                                   _ptr(y8), _ptr(y_amax), C.c_int(T), C.c_int(N), C.c_int(K), _stream(stream)))
+
+
+def fp8_linear_dgrad_q(dy8, w8t, sdy_inv, sw_inv, dx_scale, dx_fmt, dx8, dx_amax=None, stream=None):
+    """Data-gradient product emitting FP8 codes of the BF16-rounded result under a caller scale, plus its amax."""
+    T, N = dy8.shape
+    K = w8t.shape[0]
+    _check(load().fp8_linear_dgrad_q(_ptr(dy8), _ptr(w8t), _ptr(sdy_inv), _ptr(sw_inv), _ptr(dx_scale),
+                                     C.c_int(dx_fmt), _ptr(dx8), _ptr(dx_amax), C.c_int(T), C.c_int(N), C.c_int(K),
+                                     _stream(stream)))
+
+
 def fp8_linear_dgrad(dy8, w8t, sdy_inv, sw_inv, dx, ws=None, stream=None):
     T, N = dy8.shape
     K = w8t.shape[0]
@@ -206,6 +223,17 @@ def fp8_attention_fwd(q8, k8, v8, q_inv, k_inv, v_inv, softmax_scale, causal, o,
                                     C.c_int(N), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), _ptr(o), _ptr(lse),
                                     _ptr(ws), C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
                                     _stream(stream)))
+
+
+def fp8_attention_fwd_q(q8, k8, v8, q_inv, k_inv, v_inv, softmax_scale, causal, o, lse, o_scale, o8, o_amax=None,
+                        p_scale=448.0, stream=None):
+    """Forward that also emits E4M3 codes of O under a caller (delayed) scale and amax(O)."""
+    B, N, Hq, d = q8.shape
+    Hkv = k8.shape[2]
+    sc = _scales(q_inv, k_inv, v_inv, None, softmax_scale, p_scale, None, None)
+    _check(load().fp8_attention_fwd_q(_ptr(q8), _ptr(k8), _ptr(v8), C.byref(sc), C.c_int(int(causal)), C.c_int(B),
+                                      C.c_int(N), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), _ptr(o), _ptr(lse),
+                                      _ptr(o_scale), _ptr(o8), _ptr(o_amax), _stream(stream)))
 
 
 def fp8_attention_bwd(q8, k8, v8, do8, o, lse, q_inv, k_inv, v_inv, do_inv, softmax_scale, ds_scale, causal,

@@ -47,6 +47,10 @@ struct AttnFwdParams {
     int causal;
     int B, N, Hq, Hkv;
     int *status;
+    // producer form (delayed scaling): also emit E4M3 codes of the BF16 output under *o_scale, and its amax
+    const float *o_scale;
+    uint8_t *O8;                 // [B,N,Hq,D]
+    unsigned int *o_amax_bits;   // nullable
 };
 
 // One 32-column chunk of a score row -> 32 values of c_P * P~ = 2^(c*S - shift), their sum, and 32 E4M3 codes.
@@ -290,6 +294,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             tc_fence_after();
             const float inv = __ldg(p.v_inv) / l;        // l already carries c_P
             uint16_t *orow = p.O + (((size_t)b * p.N + row) * p.Hq + h) * D;
+            uint8_t *o8row = p.O8 + (((size_t)b * p.N + row) * p.Hq + h) * D;
+            const float o_scale = p.o_scale ? __ldg(p.o_scale) : 1.0f;
+            uint32_t amax2 = 0;
 #pragma unroll 1
             for (int cc = 0; cc < D; cc += 32) {
                 uint32_t v[32];
@@ -304,8 +311,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         o.z = pack_bf16x2(__uint_as_float(v[i + 4]) * inv, __uint_as_float(v[i + 5]) * inv);
                         o.w = pack_bf16x2(__uint_as_float(v[i + 6]) * inv, __uint_as_float(v[i + 7]) * inv);
                         *reinterpret_cast<uint4 *>(orow + cc + i) = o;
+                        if (p.o_scale) {
+                            // the codes an unfused cast of the BF16 output would give
+                            amax2 = __vmaxu2(__vmaxu2(__vmaxu2(__vmaxu2(amax2, o.x & 0x7FFF7FFFu), o.y & 0x7FFF7FFFu),
+                                                      o.z & 0x7FFF7FFFu), o.w & 0x7FFF7FFFu);
+                            const uint32_t c0 = cvt_f32x4_to_fp8x4<0>(
+                                __fmul_rn(bf16_lo(o.x), o_scale), __fmul_rn(bf16_hi(o.x), o_scale),
+                                __fmul_rn(bf16_lo(o.y), o_scale), __fmul_rn(bf16_hi(o.y), o_scale));
+                            const uint32_t c1 = cvt_f32x4_to_fp8x4<0>(
+                                __fmul_rn(bf16_lo(o.z), o_scale), __fmul_rn(bf16_hi(o.z), o_scale),
+                                __fmul_rn(bf16_lo(o.w), o_scale), __fmul_rn(bf16_hi(o.w), o_scale));
+                            *reinterpret_cast<uint2 *>(o8row + cc + i) = make_uint2(c0, c1);
+                        }
                     }
                 }
+            }
+            if (p.o_scale && p.o_amax_bits) {
+                uint32_t mm = row < p.N ? max(amax2 & 0xFFFFu, amax2 >> 16) : 0u;
+                mm = __reduce_max_sync(0xffffffffu, mm);
+                if (lane == 0 && mm != 0u) atomicMax(p.o_amax_bits, mm << 16);
             }
             if (row < p.N)
                 p.LSE[((size_t)b * p.Hq + h) * p.N + row] = (m + log2f(l) - p.log2_p_scale) * 0.69314718055994531f;
@@ -371,19 +395,18 @@ static int launch_attn_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *
 
 using namespace fp8dpa;
 
-extern "C" int fp8_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const fp8_attn_scales *sc,
-                                 int causal, int B, int N, int Hq, int Hkv, int d, void *O_bf16, float *LSE, void *ws,
-                                 size_t ws_bytes, void *stream)
+static int attention_fwd_common(const char *who, const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8,
+                                const fp8_attn_scales *sc, int causal, int B, int N, int Hq, int Hkv, int d, void *O_bf16,
+                                float *LSE, const float *o_scale, uint8_t *O8, float *o_amax, void *stream)
 {
-    (void)ws; (void)ws_bytes;
-    int rc = validate_attn("fp8_attention_fwd", Q8, K8, V8, sc, B, N, Hq, Hkv, d);
+    int rc = validate_attn(who, Q8, K8, V8, sc, B, N, Hq, Hkv, d);
     if (rc != FP8_OK) return rc;
     if (!O_bf16 || !LSE) {
-        set_error("fp8_attention_fwd: NULL output pointer");
+        set_error("%s: NULL output pointer", who);
         return FP8_ERR_NULL;
     }
-    if (!aligned16(O_bf16)) {
-        set_error("fp8_attention_fwd: O must be 16-byte aligned");
+    if (!aligned16(O_bf16) || !aligned16(O8)) {
+        set_error("%s: O must be 16-byte aligned", who);
         return FP8_ERR_ALIGN;
     }
     rc = check_arch();
@@ -398,6 +421,31 @@ extern "C" int fp8_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uin
     p.B = B; p.N = N; p.Hq = Hq; p.Hkv = Hkv;
     p.status = device_status_ptr();
     if (!p.status) return FP8_ERR_CUDA;
+    p.o_scale = o_scale;
+    p.O8 = O8;
+    p.o_amax_bits = reinterpret_cast<unsigned int *>(o_amax);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (o_scale && o_amax) FP8_CUDA_CHECK(cudaMemsetAsync(o_amax, 0, sizeof(float), st));
     return d == 128 ? launch_attn_fwd<128>(Q8, K8, V8, p, st) : launch_attn_fwd<64>(Q8, K8, V8, p, st);
+}
+
+extern "C" int fp8_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const fp8_attn_scales *sc,
+                                 int causal, int B, int N, int Hq, int Hkv, int d, void *O_bf16, float *LSE, void *ws,
+                                 size_t ws_bytes, void *stream)
+{
+    (void)ws; (void)ws_bytes;
+    return attention_fwd_common("fp8_attention_fwd", Q8, K8, V8, sc, causal, B, N, Hq, Hkv, d, O_bf16, LSE, nullptr,
+                                nullptr, nullptr, stream);
+}
+
+extern "C" int fp8_attention_fwd_q(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const fp8_attn_scales *sc,
+                                   int causal, int B, int N, int Hq, int Hkv, int d, void *O_bf16, float *LSE,
+                                   const float *o_scale, uint8_t *O8, float *o_amax, void *stream)
+{
+    if (!o_scale || !O8) {
+        set_error("fp8_attention_fwd_q: NULL o_scale / O8");
+        return FP8_ERR_NULL;
+    }
+    return attention_fwd_common("fp8_attention_fwd_q", Q8, K8, V8, sc, causal, B, N, Hq, Hkv, d, O_bf16, LSE, o_scale, O8,
+                                o_amax, stream);
 }

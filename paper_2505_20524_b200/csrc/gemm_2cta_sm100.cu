@@ -15,6 +15,7 @@
 //   tempty[b] used in the even CTA only: 8 arrivals (4 epilogue warps of each CTA; the odd CTA arrives remotely)
 // Every wait is bounded; a cluster barrier before exit keeps either CTA alive while its peer can still reach it.
 #include "common.cuh"
+#include "gemm_epilogue.cuh"
 
 namespace fp8dpa {
 
@@ -33,10 +34,9 @@ constexpr int DYN_BYTES = BAR_OFFSET + N_BARS * 8 + 16 + 1024;
 constexpr uint32_t TMEM_COLS = 512;
 
 struct Params {
-    void *out;
+    GemmOut o;
     const float *sa_inv, *sb_inv;
     int M, N, K;
-    int out_is_fp32, accumulate;
     uint32_t idesc;
     int num_pairs;
     int *status;
@@ -154,6 +154,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         // ------------------------------------------------------------ epilogue (warps 2..5 of both CTAs)
         const int quad = warp & 3;
         const float descale = __ldg(p.sa_inv) * __ldg(p.sb_inv);
+        const float q_scale = p.o.q_scale ? __ldg(p.o.q_scale) : 1.0f;
+        uint32_t amax2 = 0;
         bool ok = true;
         int it = 0;
         for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs, ++it) {
@@ -172,48 +174,14 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                 tmem_ld_32x32b_x32(taddr + (uint32_t)c, r);
                 tmem_ld_wait();
                 const int col = n0 + c;
-                if (row < p.M && col < p.N) {
-                    const int ncols = min(32, p.N - col);
-                    if (p.out_is_fp32) {
-                        float *dst = static_cast<float *>(p.out) + (size_t)row * p.N + col;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            if (j < ncols) {
-                                float4 v = make_float4(__uint_as_float(r[j]) * descale, __uint_as_float(r[j + 1]) * descale,
-                                                       __uint_as_float(r[j + 2]) * descale,
-                                                       __uint_as_float(r[j + 3]) * descale);
-                                if (p.accumulate) {
-                                    const float4 o = *reinterpret_cast<const float4 *>(dst + j);
-                                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-                                }
-                                *reinterpret_cast<float4 *>(dst + j) = v;
-                            }
-                        }
-                    } else {
-                        uint16_t *dst = static_cast<uint16_t *>(p.out) + (size_t)row * p.N + col;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            if (j < ncols) {
-                                float v[8];
-#pragma unroll
-                                for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(r[j + q]) * descale;
-                                if (p.accumulate) {
-                                    const uint4 o = *reinterpret_cast<const uint4 *>(dst + j);
-                                    v[0] += bf16_lo(o.x); v[1] += bf16_hi(o.x); v[2] += bf16_lo(o.y); v[3] += bf16_hi(o.y);
-                                    v[4] += bf16_lo(o.z); v[5] += bf16_hi(o.z); v[6] += bf16_lo(o.w); v[7] += bf16_hi(o.w);
-                                }
-                                *reinterpret_cast<uint4 *>(dst + j) =
-                                    make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
-                                               pack_bf16x2(v[6], v[7]));
-                            }
-                        }
-                    }
-                }
+                if (row < p.M && col < p.N)
+                    gemm_store_chunk(r, descale, p.o, q_scale, p.N, row, col, min(32, p.N - col), amax2);
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_pair_leader(tempty_bar(buf));   // the even CTA's barrier, from either CTA
         }
+        gemm_publish_amax(p.o, amax2);
     }
 
     // ---------------------------------------------------------------- teardown
@@ -234,9 +202,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 }  // namespace g2
 
 // Returns FP8_OK after launching, or a negative status.  `max_pairs` = 0 lets the runtime size the grid.
-int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, void *out,
-                     int out_is_fp32, int accumulate, int M, int N, int K, uint32_t idesc, int *status,
-                     cudaStream_t st)
+int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, const GemmOut &o,
+                     int M, int N, int K, uint32_t idesc, int *status, cudaStream_t st)
 {
     using namespace g2;
     CUtensorMap ta, tb;
@@ -265,9 +232,8 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     }
     const int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
     Params p;
-    p.out = out; p.sa_inv = sa_inv; p.sb_inv = sb_inv;
+    p.o = o; p.sa_inv = sa_inv; p.sb_inv = sb_inv;
     p.M = M; p.N = N; p.K = K;
-    p.out_is_fp32 = out_is_fp32; p.accumulate = accumulate;
     p.idesc = idesc;
     p.num_pairs = tiles < max_clusters ? tiles : max_clusters;
     p.status = status;

@@ -11,6 +11,7 @@
 #include <stdlib.h>
 
 #include "common.cuh"
+#include "gemm_epilogue.cuh"
 
 namespace fp8dpa {
 
@@ -40,10 +41,9 @@ struct GemmCfg {
 };
 
 struct GemmParams {
-    void *out;
+    GemmOut o;
     const float *sa_inv, *sb_inv;
     int M, N, K;
-    int out_is_fp32, accumulate;
     uint32_t idesc;
     int *status;
 };
@@ -174,6 +174,8 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         const int quad = warp & 3;                     // TMEM lanes 32*quad .. 32*quad+31
         const int mt = e >> 2;                         // which 128-row accumulator (MT = 2 only)
         const float descale = __ldg(p.sa_inv) * __ldg(p.sb_inv);
+        const float q_scale = p.o.q_scale ? __ldg(p.o.q_scale) : 1.0f;
+        uint32_t amax2 = 0;
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++it) {
@@ -194,47 +196,14 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 const int col = n0 + c;
                 if (row < p.M && col < p.N) {
                     // N is a multiple of 16, so a 32-column chunk is either whole or half inside
-                    const int ncols = min(32, p.N - col);
-                    if (p.out_is_fp32) {
-                        float *dst = static_cast<float *>(p.out) + (size_t)row * p.N + col;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            if (j < ncols) {
-                                float4 v = make_float4(__uint_as_float(r[j]) * descale, __uint_as_float(r[j + 1]) * descale,
-                                                       __uint_as_float(r[j + 2]) * descale,
-                                                       __uint_as_float(r[j + 3]) * descale);
-                                if (p.accumulate) {
-                                    const float4 o = *reinterpret_cast<const float4 *>(dst + j);
-                                    v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-                                }
-                                *reinterpret_cast<float4 *>(dst + j) = v;
-                            }
-                        }
-                    } else {
-                        uint16_t *dst = static_cast<uint16_t *>(p.out) + (size_t)row * p.N + col;
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            if (j < ncols) {
-                                float v[8];
-#pragma unroll
-                                for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(r[j + q]) * descale;
-                                if (p.accumulate) {
-                                    const uint4 o = *reinterpret_cast<const uint4 *>(dst + j);
-                                    v[0] += bf16_lo(o.x); v[1] += bf16_hi(o.x); v[2] += bf16_lo(o.y); v[3] += bf16_hi(o.y);
-                                    v[4] += bf16_lo(o.z); v[5] += bf16_hi(o.z); v[6] += bf16_lo(o.w); v[7] += bf16_hi(o.w);
-                                }
-                                *reinterpret_cast<uint4 *>(dst + j) =
-                                    make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
-                                               pack_bf16x2(v[6], v[7]));
-                            }
-                        }
-                    }
+                    gemm_store_chunk(r, descale, p.o, q_scale, p.N, row, col, min(32, p.N - col), amax2);
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
         }
+        gemm_publish_amax(p.o, amax2);
     }
 
     // ---------------------------------------------------------------- teardown (all roles fall through)
@@ -252,9 +221,8 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     }
 }
 
-int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, void *out,
-                     int out_is_fp32, int accumulate, int M, int N, int K, uint32_t idesc, int *status,
-                     cudaStream_t st);
+int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, const GemmOut &o,
+                     int M, int N, int K, uint32_t idesc, int *status, cudaStream_t st);
 
 // FP8DPA_GEMM=1cta|2cta forces one kernel family (for A/B measurements); default: chosen per shape.
 static int gemm_family_override()
@@ -302,19 +270,22 @@ static int launch_gemm(const uint8_t *a, const uint8_t *b, const GemmParams &p, 
 
 // C[M,N] (+)= sa_inv*sb_inv * A[M,K] . B[N,K]^T
 int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int fmt_b, const float *sa_inv,
-             const float *sb_inv, void *out, int out_is_fp32, int accumulate, int M, int N, int K, cudaStream_t st)
+             const float *sb_inv, const GemmOut &o, int M, int N, int K, cudaStream_t st)
 {
-    int rc = validate_gemm(who, a, b, sa_inv, sb_inv, out, M, N, K);
+    int rc = validate_gemm(who, a, b, sa_inv, sb_inv, o.out, M, N, K);
     if (rc != FP8_OK) return rc;
+    if (o.q_scale && o.q_fmt != FP8_E4M3 && o.q_fmt != FP8_E5M2) {
+        set_error("%s: output format %d is not FP8_E4M3 / FP8_E5M2", who, o.q_fmt);
+        return FP8_ERR_ENUM;
+    }
     rc = check_arch();
     if (rc != FP8_OK) return rc;
+    if (o.q_scale && o.amax_bits) FP8_CUDA_CHECK(cudaMemsetAsync(o.amax_bits, 0, sizeof(float), st));
     GemmParams p;
-    p.out = out;
+    p.o = o;
     p.sa_inv = sa_inv;
     p.sb_inv = sb_inv;
     p.M = M; p.N = N; p.K = K;
-    p.out_is_fp32 = out_is_fp32;
-    p.accumulate = accumulate;
     p.status = device_status_ptr();
     if (!p.status) return FP8_ERR_CUDA;
     // CTA pairs (256 x 256 per pair, 32 KB per CTA and stage) whenever the matrix is large enough to give every
@@ -324,8 +295,8 @@ int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int
         const long pair_tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
         const int fam = gemm_family_override();
         if (fam != 1 && M >= 256 && N >= 256 && (fam == 2 || pair_tiles >= sm_count())) {
-            return launch_gemm_2cta(a, b, sa_inv, sb_inv, out, out_is_fp32, accumulate, M, N, K,
-                                    umma_idesc_f8(fmt_a, fmt_b, 256, 256), p.status, st);
+            return launch_gemm_2cta(a, b, sa_inv, sb_inv, o, M, N, K, umma_idesc_f8(fmt_a, fmt_b, 256, 256), p.status,
+                                    st);
         }
     }
     // Tile choice.  The 256 x 256 tile needs 2/3 of the L2 traffic of 128 x 256 but cannot overlap its epilogue
@@ -355,7 +326,8 @@ extern "C" int fp8_linear_fwd(const uint8_t *X8, const uint8_t *W8, const float 
                               int out_is_fp32, int T, int N, int K, void *ws, size_t ws_bytes, void *stream)
 {
     (void)ws; (void)ws_bytes;
-    return gemm_fp8("fp8_linear_fwd", X8, FP8_E4M3, W8, FP8_E4M3, sX_inv, sW_inv, Y, out_is_fp32, 0, T, N, K,
+    const GemmOut o{Y, out_is_fp32, 0, nullptr, 0, nullptr};
+    return gemm_fp8("fp8_linear_fwd", X8, FP8_E4M3, W8, FP8_E4M3, sX_inv, sW_inv, o, T, N, K,
                     static_cast<cudaStream_t>(stream));
 }
 
@@ -365,7 +337,8 @@ extern "C" int fp8_linear_dgrad(const uint8_t *dY8, const uint8_t *W8t, const fl
 {
     (void)ws; (void)ws_bytes;
     // dX[T,K] = dY8[T,N] . W8t[K,N]^T : rows T, cols K, reduce N
-    return gemm_fp8("fp8_linear_dgrad", dY8, FP8_E5M2, W8t, FP8_E4M3, sdY_inv, sW_inv, dX, out_is_fp32, 0, T, K, N,
+    const GemmOut o{dX, out_is_fp32, 0, nullptr, 0, nullptr};
+    return gemm_fp8("fp8_linear_dgrad", dY8, FP8_E5M2, W8t, FP8_E4M3, sdY_inv, sW_inv, o, T, K, N,
                     static_cast<cudaStream_t>(stream));
 }
 
@@ -375,6 +348,33 @@ extern "C" int fp8_linear_wgrad(const uint8_t *dY8t, const uint8_t *X8t, const f
 {
     (void)ws; (void)ws_bytes;
     // dW[N,K] = dY8t[N,T] . X8t[K,T]^T : rows N, cols K, reduce T
-    return gemm_fp8("fp8_linear_wgrad", dY8t, FP8_E5M2, X8t, FP8_E4M3, sdY_inv, sX_inv, dW, out_is_fp32, accumulate,
-                    N, K, T, static_cast<cudaStream_t>(stream));
+    const GemmOut o{dW, out_is_fp32, accumulate, nullptr, 0, nullptr};
+    return gemm_fp8("fp8_linear_wgrad", dY8t, FP8_E5M2, X8t, FP8_E4M3, sdY_inv, sX_inv, o, N, K, T,
+                    static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int fp8_linear_fwd_q(const uint8_t *X8, const uint8_t *W8, const float *sX_inv, const float *sW_inv,
+                                const float *y_scale, int y_fmt, uint8_t *Y8, float *y_amax, int T, int N, int K,
+                                void *stream)
+{
+    if (!y_scale) {
+        set_error("fp8_linear_fwd_q: NULL y_scale");
+        return FP8_ERR_NULL;
+    }
+    const GemmOut o{Y8, 0, 0, y_scale, y_fmt, reinterpret_cast<unsigned int *>(y_amax)};
+    return gemm_fp8("fp8_linear_fwd_q", X8, FP8_E4M3, W8, FP8_E4M3, sX_inv, sW_inv, o, T, N, K,
+                    static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int fp8_linear_dgrad_q(const uint8_t *dY8, const uint8_t *W8t, const float *sdY_inv, const float *sW_inv,
+                                  const float *dx_scale, int dx_fmt, uint8_t *dX8, float *dx_amax, int T, int N, int K,
+                                  void *stream)
+{
+    if (!dx_scale) {
+        set_error("fp8_linear_dgrad_q: NULL dx_scale");
+        return FP8_ERR_NULL;
+    }
+    const GemmOut o{dX8, 0, 0, dx_scale, dx_fmt, reinterpret_cast<unsigned int *>(dx_amax)};
+    return gemm_fp8("fp8_linear_dgrad_q", dY8, FP8_E5M2, W8t, FP8_E4M3, sdY_inv, sW_inv, o, T, K, N,
+                    static_cast<cudaStream_t>(stream));
 }

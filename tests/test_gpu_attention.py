@@ -128,3 +128,34 @@ def test_backward_matches_oracle(name, B, N, causal):
     assert max(errs.values()) <= TOL_BWD, errs
     for n_ in ("dQ", "dK", "dV"):
         assert ref["slack_" + n_].sum() <= 1e-2 * ref["mag_" + n_].sum()
+
+
+@pytest.mark.parametrize("name,B,N,causal", [("c1", 1, 400, True), ("c4", 1, 272, True), ("c1", 2, 128, False)])
+def test_forward_fp8_output_equals_unfused_chain(name, B, N, causal):
+    """Producer form: O and LSE unchanged, O8 and amax bit-identical to fp8_cast of the BF16 output."""
+    cfg = synth.CONFIGS[name]
+    Hq, Hkv, d = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    if name != "c1":
+        Hq, Hkv = Hq // 4, Hkv // 4
+        cfg = synth.BlockConfig(**{**cfg.__dict__, "n_q_heads": Hq, "n_kv_heads": Hkv})
+    qd = quantized_qkv(cfg, N, B)
+    s = d ** -0.5
+    O, LSE = run_fwd(qd, B, N, Hq, Hkv, d, causal, s)
+    a_now = scalar()
+    fp8.fp8_amax(O, a_now)
+    o_scale, o_inv = scalar(), scalar()
+    fp8.fp8_scale(scalar(float(a_now.item()) * 1.5), o.E4M3, 0, o_scale, o_inv)      # a "history" scale
+    ref8 = torch.empty((B, N, Hq, d), dtype=torch.uint8, device="cuda")
+    fp8.fp8_cast(O.view(B * N, Hq * d), o_scale, o.E4M3, ref8.view(B * N, Hq * d))
+    q8, k8, v8 = dev(qd["q"][0]), dev(qd["k"][0]), dev(qd["v"][0])
+    O2 = torch.empty_like(O)
+    LSE2 = torch.empty_like(LSE)
+    O8 = torch.full((B, N, Hq, d), 0x55, dtype=torch.uint8, device="cuda")
+    a = scalar(-2.0)
+    fp8.fp8_attention_fwd_q(q8, k8, v8, scalar(qd["q"][1]), scalar(qd["k"][1]), scalar(qd["v"][1]), s, causal,
+                            O2, LSE2, o_scale, O8, a)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    assert torch.equal(O2.view(torch.int16), O.view(torch.int16)) and torch.equal(LSE2, LSE)
+    assert torch.equal(O8, ref8)
+    assert float(a.item()) == float(a_now.item())

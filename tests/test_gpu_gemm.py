@@ -127,3 +127,63 @@ def test_argument_validation():
     with pytest.raises(fp8.Fp8Error) as e:
         fp8.fp8_linear_fwd(a, a, None, scalar(1), y)
     assert e.value.status == -1
+
+
+@pytest.mark.parametrize("family", ["1cta", "2cta"])
+@pytest.mark.parametrize("T,N,K", [(256, 768, 256), (400, 528, 144), (1024, 1040, 2064), (16, 16, 16)])
+def test_fp8_output_epilogue(family, T, N, K, monkeypatch):
+    """Producer form (delayed scaling): codes and amax equal the unfused chain bit for bit, and decode close to the oracle."""
+    monkeypatch.setenv("FP8DPA_GEMM", family)
+    seed = T + N + K
+    cols = synth.choose_columns(K, 2, seed, 1)
+    x = synth.normal_bf16((T, K), seed, 0, 1.0, cols, 50.0)
+    w = synth.normal_bf16((N, K), seed, 1, synth.W_STD)
+    dy = synth.normal_bf16((T, N), seed, 2, synth.GRAD_STD)
+    x8, _, _, _, sx = gpu_quantize(x, o.E4M3, True)
+    w8, w8t, _, _, sw = gpu_quantize(w, o.E4M3, True)
+    dy8, _, _, _, sdy = gpu_quantize(dy, o.E5M2, True)
+    for name, fmt in (("fwd", o.E4M3), ("dgrad", o.E5M2)):
+        rows, cols_out = (T, N) if name == "fwd" else (T, K)
+        ybf = torch.empty((rows, cols_out), dtype=torch.bfloat16, device="cuda")
+        if name == "fwd":
+            fp8.fp8_linear_fwd(x8, w8, sx, sw, ybf)
+        else:
+            fp8.fp8_linear_dgrad(dy8, w8t, sdy, sw, ybf)
+        # a "delayed" scale: from a slightly larger amax than this step's (history maximum), not from this tensor
+        a_now = scalar()
+        fp8.fp8_amax(ybf, a_now)
+        hist = scalar(float(a_now.item()) * 1.25)
+        s, si = scalar(), scalar()
+        fp8.fp8_scale(hist, fmt, 0, s, si)
+        ref8 = torch.empty((rows, cols_out), dtype=torch.uint8, device="cuda")
+        fp8.fp8_cast(ybf, s, fmt, ref8)
+        got8 = torch.full((rows, cols_out), 0x55, dtype=torch.uint8, device="cuda")
+        a = scalar(-3.0)
+        if name == "fwd":
+            fp8.fp8_linear_fwd_q(x8, w8, sx, sw, s, fmt, got8, a)
+        else:
+            fp8.fp8_linear_dgrad_q(dy8, w8t, sdy, sw, s, fmt, got8, a)
+        torch.cuda.synchronize()
+        assert fp8.fp8_device_status() == 0
+        assert torch.equal(got8, ref8)                                   # same accumulators, same roundings
+        assert float(a.item()) == float(a_now.item())
+        # against the oracle: decode / scale within the GEMM tolerance plus half a quantisation step of the format
+        ox8, _, _, osx = o.quantize(x, o.E4M3)
+        ow8, _, _, osw = o.quantize(w, o.E4M3)
+        ody8, _, _, osdy = o.quantize(dy, o.E5M2)
+        ref, mag = o.linear_fwd(ox8, ow8, osx, osw) if name == "fwd" else o.linear_dgrad(ody8, ow8, osdy, osw)
+        dec = o.decode_array(host(got8), fmt).astype(np.float64) * float(si.item())
+        step = np.maximum(np.abs(ref) * (2.0 ** -3 if fmt == o.E4M3 else 2.0 ** -2),
+                          (2.0 ** -9 if fmt == o.E4M3 else 2.0 ** -16) * float(si.item()))
+        assert np.all(np.abs(dec - ref) <= TOL_BF16 * mag + 0.5 * step + 2.0 ** -8 * np.abs(ref))
+
+
+def test_fp8_output_argument_validation():
+    x8 = torch.zeros((32, 32), dtype=torch.uint8, device="cuda")
+    s = scalar(1.0)
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_linear_fwd_q(x8, x8, s, s, None, 0, x8)
+    assert e.value.status == -1
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_linear_fwd_q(x8, x8, s, s, s, 3, x8)
+    assert e.value.status == -4
