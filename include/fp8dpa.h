@@ -175,6 +175,23 @@ FP8_API int fp8_linear_dgrad_q(const uint8_t *dY8, const uint8_t *W8t, const flo
                        const float *dx_scale, int dx_fmt, uint8_t *dX8, float *dx_amax, int T, int N, int K,
                        void *stream);
 
+/* ---- fine-grained ("blockwise") scaling: the comparison recipe -------------------------------------
+ * Section 2 (several scaling factors per tensor, one per block) and Appendix E ("Fine-grained scaling recipes",
+ * throughput table): activations are quantised in 1 x 128 blocks, weights in 128 x 128 blocks, every block
+ * just-in-time with its own rho_b = FP8Max / amax(block); the product then sums, over K-blocks of 128, FP8 partial
+ * products that each carry their own descale.  Kept beside the tensor-wise path to measure what the finer recipe
+ * costs on this hardware.
+ *
+ * fp8_quantize_blockwise: x [rows, cols] BF16 -> out [rows, cols] codes, one pass.  block_rows = 1: 1 x 128 blocks,
+ * scale_inv laid out K-block-major, [cols/128][rows] (the order the product reads it in).  block_rows = 128:
+ * 128 x 128 blocks, scale_inv [ceil(rows/128)][cols/128].  cols % 128 == 0.  Inputs are finite.
+ * fp8_linear_fwd_blockwise: Y[t,n] = sum_kb sx_inv[kb][t] * sw_inv[n/128][kb] * sum_{k in kb} X8[t,k] W8[n,k], BF16
+ * result; X8 [T,K], W8 [N,K] in E4M3; K % 128 == 0, N % 16 == 0. */
+FP8_API int fp8_quantize_blockwise(const void *x_bf16, size_t rows, size_t cols, int block_rows, int fmt,
+                           uint8_t *out, float *scale_inv, void *stream);
+FP8_API int fp8_linear_fwd_blockwise(const uint8_t *X8, const uint8_t *W8, const float *sx_inv, const float *sw_inv,
+                             void *Y_bf16, int T, int N, int K, void *stream);
+
 /* ---- attention ------------------------------------------------------------------------------------
  * Appendix B, Eq. (P): P = Softmax(s Q K^T + M), output P V, grouped-query heads; Appendix E table: both
  * products in FP8, forward and backward.  Tensors are [B, N, H, d] row-major; query head h reads KV head

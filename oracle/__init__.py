@@ -268,6 +268,36 @@ def linear_wgrad(dy8, x8, sdy_inv, sx_inv, rows=None, cols=None, prev=None):
     return _linear("oracle_linear_wgrad", dy8, x8, sdy_inv, sx_inv, T, N, K, N, K, rows, cols, prev)
 
 
+def quantize_blockwise(x_bf16, br: int, bc: int, fmt: int):
+    """Block-by-block just-in-time quantisation; returns (codes [R,C], scale_inv [ceil(R/br), ceil(C/bc)])."""
+    x = _c(x_bf16, np.uint16)
+    R, Cc = x.shape
+    codes = np.empty((R, Cc), dtype=np.uint8)
+    si = np.empty(((R + br - 1) // br, (Cc + bc - 1) // bc), dtype=np.float32)
+    f = _L().oracle_quantize_blockwise
+    f.restype = None
+    f(_p(x), C.c_size_t(R), C.c_size_t(Cc), C.c_size_t(br), C.c_size_t(bc), C.c_int(fmt), _p(codes), _p(si))
+    return codes, si
+
+
+def linear_fwd_blockwise(x8, w8, sx_inv, sw_inv, bk=128, bn=128, rows=None, cols=None):
+    """Y with one descale per (row, K-block) of X and per (bn x bk) block of W; returns (ref, mag) on rows x cols."""
+    x8, w8 = _c(x8, np.uint8), _c(w8, np.uint8)
+    T, K = x8.shape
+    N = w8.shape[0]
+    sx, sw = _c(sx_inv, np.float32), _c(sw_inv, np.float32)
+    assert sx.shape == (T, (K + bk - 1) // bk) and sw.shape == ((N + bn - 1) // bn, (K + bk - 1) // bk)
+    r = np.arange(T, dtype=np.int64) if rows is None else _c(rows, np.int64)
+    c = np.arange(N, dtype=np.int64) if cols is None else _c(cols, np.int64)
+    ref = np.empty((r.size, c.size), dtype=np.float64)
+    mag = np.empty_like(ref)
+    f = _L().oracle_linear_fwd_blockwise
+    f.restype = None
+    f(_p(x8), _p(w8), _p(sx), _p(sw), C.c_int64(T), C.c_int64(N), C.c_int64(K), C.c_int64(bk), C.c_int64(bn),
+      _p(r), C.c_int64(r.size), _p(c), C.c_int64(c.size), _p(ref), _p(mag))
+    return ref, mag
+
+
 # ---------------------------------------------------------------- attention
 def attn_params(B, N, Hq, Hkv, d, causal=True, quant=True, kv_block=0, max_mode=0, s=None, c_P=448.0,
                 q_inv=1.0, k_inv=1.0, v_inv=1.0, do_inv=1.0, ds_scale=1.0, flip_eps=0.0) -> AttnParams:

@@ -767,3 +767,70 @@ int oracle_num_threads(void)
     return 1;
 #endif
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Fine-grained ("blockwise") scaling, the recipe the paper measures against (Section 2: several scaling factors per
+ * tensor, different blocks with different factors; Appendix E, "Fine-grained scaling recipes"): a [R,C] tensor is cut
+ * into blocks of br x bc elements (1 x 128 for activations, 128 x 128 for weights in the recipe measured there) and
+ * every block is quantised like a tensor of its own: rho_b = FP8Max / amax(block), codes = FP8cast(rho_b * x).
+ * scale_inv[rb * ncb + cb] = 1 / rho_b with ncb = ceil(C / bc).  Edge blocks are short.
+ * ---------------------------------------------------------------------------------------------- */
+void oracle_quantize_blockwise(const uint16_t *x, size_t R, size_t C, size_t br, size_t bc, int fmt, uint8_t *codes,
+                               float *scale_inv)
+{
+    size_t nrb = (R + br - 1) / br, ncb = (C + bc - 1) / bc;
+#pragma omp parallel for schedule(static)
+    for (long b = 0; b < (long)(nrb * ncb); ++b) {
+        size_t rb = (size_t)b / ncb, cb = (size_t)b % ncb;
+        size_t r1 = (rb + 1) * br < R ? (rb + 1) * br : R, c1 = (cb + 1) * bc < C ? (cb + 1) * bc : C;
+        float amax = 0.0f;
+        for (size_t r = rb * br; r < r1; ++r)
+            for (size_t c = cb * bc; c < c1; ++c) {
+                float v = fabsf(bf16_bits_to_float(x[r * C + c]));
+                if (v > amax) amax = v;            /* NaN never compares greater: same reading as oracle_amax_bf16 */
+            }
+        float s, si;
+        oracle_scale(amax, fmt, 0, &s, &si);
+        scale_inv[b] = si;
+        for (size_t r = rb * br; r < r1; ++r)
+            for (size_t c = cb * bc; c < c1; ++c) {
+                volatile float p = bf16_bits_to_float(x[r * C + c]) * s;
+                codes[r * C + c] = oracle_fp8_encode(p, fmt);
+            }
+    }
+}
+
+/* Y[t,n] = sum over K-blocks kb of sx_inv[t,kb] * sw_inv[n/bn,kb] * sum_{k in kb} dec(X8[t,k]) dec(W8[n,k]):
+ * every K-block of 128 is an FP8 product of its own, descaled by its two factors and added in high precision
+ * (the "promotion" that makes this recipe slower).  sx_inv: [T, K/bk]; sw_inv: [ceil(N/bn), K/bk].
+ * mag is the same sum over absolute values. */
+void oracle_linear_fwd_blockwise(const uint8_t *X8, const uint8_t *W8, const float *sx_inv, const float *sw_inv,
+                                 int64_t T, int64_t N, int64_t K, int64_t bk, int64_t bn,
+                                 const int64_t *rows, int64_t nrows, const int64_t *cols, int64_t ncols,
+                                 double *ref, double *mag)
+{
+    double tab[256];
+    oracle_fp8_decode_table(ORACLE_E4M3, tab);
+    int64_t nkb = (K + bk - 1) / bk;
+    (void)T; (void)N;
+#pragma omp parallel for schedule(static)
+    for (long i = 0; i < (long)nrows; ++i)
+        for (int64_t j = 0; j < ncols; ++j) {
+            int64_t t = rows[i], n = cols[j];
+            double acc = 0.0, am = 0.0;
+            for (int64_t kb = 0; kb < nkb; ++kb) {
+                double part = 0.0, pm = 0.0;
+                int64_t k1 = (kb + 1) * bk < K ? (kb + 1) * bk : K;
+                for (int64_t k = kb * bk; k < k1; ++k) {
+                    double a = tab[X8[t * K + k]], b = tab[W8[n * K + k]];
+                    part += a * b;
+                    pm += fabs(a * b);
+                }
+                double sc = (double)sx_inv[t * nkb + kb] * (double)sw_inv[(n / bn) * nkb + kb];
+                acc += sc * part;
+                am += sc * pm;
+            }
+            ref[i * ncols + j] = acc;
+            mag[i * ncols + j] = am;
+        }
+}

@@ -21,7 +21,7 @@ _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_qk_norm_rope", "fp8_kurtosis",
-           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_attention_workspace_bytes",
+           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
 STATIC_SCRATCH_BYTES = 32 << 20
@@ -186,6 +186,20 @@ def fp8_linear_dgrad_q(dy8, w8t, sdy_inv, sw_inv, dx_scale, dx_fmt, dx8, dx_amax
     _check(load().fp8_linear_dgrad_q(_ptr(dy8), _ptr(w8t), _ptr(sdy_inv), _ptr(sw_inv), _ptr(dx_scale),
                                      C.c_int(dx_fmt), _ptr(dx8), _ptr(dx_amax), C.c_int(T), C.c_int(N), C.c_int(K),
                                      _stream(stream)))
+
+
+def fp8_quantize_blockwise(x, block_rows, fmt, out, scale_inv, stream=None):
+    """Block-by-block quantisation: 1 x 128 (scale_inv [cols/128, rows]) or 128 x 128 (scale_inv [rows/128, cols/128])."""
+    rows, cols = x.shape
+    _check(load().fp8_quantize_blockwise(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), C.c_int(block_rows), C.c_int(fmt),
+                                         _ptr(out), _ptr(scale_inv), _stream(stream)))
+
+
+def fp8_linear_fwd_blockwise(x8, w8, sx_inv, sw_inv, y, stream=None):
+    T, K = x8.shape
+    N = w8.shape[0]
+    _check(load().fp8_linear_fwd_blockwise(_ptr(x8), _ptr(w8), _ptr(sx_inv), _ptr(sw_inv), _ptr(y), C.c_int(T),
+                                           C.c_int(N), C.c_int(K), _stream(stream)))
 
 
 def fp8_linear_dgrad(dy8, w8t, sdy_inv, sw_inv, dx, ws=None, stream=None):

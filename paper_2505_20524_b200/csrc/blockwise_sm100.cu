@@ -1,0 +1,384 @@
+// Fine-grained ("blockwise") FP8 scaling: the recipe the paper measures its tensor-wise recipe against (Section 2;
+// Appendix E, "Fine-grained scaling recipes").  Activations carry one scale per 1 x 128 block, weights one per
+// 128 x 128 block; the GEMM is then a sum over K-blocks of 128 of FP8 products that each need their own descale, so
+// every K-block's partial accumulator leaves the tensor core and is folded into an FP32 running sum on the CUDA
+// cores ("promotion").  That extra work per K-block is the overhead the paper reports for this recipe.
+//
+// Kernels: two single-pass quantisers (a block is small enough to stay on chip between its amax and its cast) and
+//   gemm_blockwise_kernel: persistent, one CTA per SM, tile 128 x 128, K-block = one 128-byte swizzle span
+//     warp 0  TMA: A (128 rows x 128 B) and B (128 rows x 128 B) per K-block, 6 stages
+//     warp 1  MMA: 4 x tcgen05.mma (M128 N128 K32) per K-block into one of two 128-column TMEM buffers, the first
+//             one overwriting; commit frees the stage and publishes the partial
+//     warps 2-9  promotion: two threads per output row (warps w and w+4 share a TMEM lane group and take 64 columns
+//             each); acc[64] (registers) += partial[c] * sx_inv[kb,row] * sw_inv[tile,kb], the TMEM load of the next
+//             32 columns in flight during the FMAs; after the last K-block the row is written as BF16
+#include <float.h>
+
+#include "common.cuh"
+
+namespace fp8dpa {
+namespace bw {
+
+__device__ __forceinline__ float block_scale_from_amax(float a, float fp8_max)
+{
+    if (!(a > 0.0f) || isinf(a)) return 1.0f;
+    const float s = __fdiv_rn(fp8_max, a);
+    return isinf(s) ? FLT_MAX : s;
+}
+
+template <int FMT>
+__device__ __forceinline__ uint2 cast8(const uint4 v, const float s)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint16_t h[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        h[i] = cvt_f32x2_to_fp8x2<FMT>(__fmul_rn(bf16_lo(w[i]), s), __fmul_rn(bf16_hi(w[i]), s));
+    return make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
+}
+__device__ __forceinline__ uint32_t amax8(uint32_t m, const uint4 v)
+{
+    return __vmaxu2(__vmaxu2(__vmaxu2(__vmaxu2(m, v.x & 0x7FFF7FFFu), v.y & 0x7FFF7FFFu), v.z & 0x7FFF7FFFu),
+                    v.w & 0x7FFF7FFFu);
+}
+
+// 1 x 128 blocks: 16 lanes per block (16-byte loads), two blocks per warp and sweep.  scale_inv is written
+// K-block-major, [C/128][R], which is the order the GEMM's promotion warps read it in (one row per lane).
+template <int FMT>
+__global__ void __launch_bounds__(256) quantize_1x128_kernel(const uint16_t *__restrict__ x, size_t R, int C,
+                                                             uint8_t *__restrict__ out, float *__restrict__ scale_inv)
+{
+    const int ncb = C / 128;
+    const size_t n_blocks = R * (size_t)ncb;
+    const int j = threadIdx.x & 15;
+    // uniform trip count: the shuffles name every lane
+    for (size_t base = (size_t)blockIdx.x * 16; base < n_blocks; base += (size_t)gridDim.x * 16) {
+        const size_t b_raw = base + (threadIdx.x >> 4);
+        const bool valid = b_raw < n_blocks;
+        const size_t b = valid ? b_raw : n_blocks - 1;
+        const size_t r = b / ncb;
+        const int cb = (int)(b % ncb);
+        const size_t off = r * (size_t)C + (size_t)cb * 128 + j * 8;
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + off));
+        uint32_t m2 = amax8(0u, v);
+        uint32_t m = max(m2 & 0xFFFFu, m2 >> 16);
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+        const float s = block_scale_from_amax(__uint_as_float(m << 16), FMT == 0 ? 448.0f : 57344.0f);
+        if (valid) {
+            *reinterpret_cast<uint2 *>(out + off) = cast8<FMT>(v, s);
+            if (j == 0) scale_inv[(size_t)cb * R + r] = __fdiv_rn(1.0f, s);
+        }
+    }
+}
+
+// 128 x 128 blocks: one CTA per block, 8 groups of 8 elements per thread held in registers.  scale_inv: [R/128][C/128].
+template <int FMT>
+__global__ void __launch_bounds__(256) quantize_128x128_kernel(const uint16_t *__restrict__ x, int R, int C,
+                                                               uint8_t *__restrict__ out, float *__restrict__ scale_inv)
+{
+    __shared__ uint32_t warp_max[8];
+    const int r0 = blockIdx.y * 128, c0 = blockIdx.x * 128;
+    uint4 v[8];
+    uint32_t m2 = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int idx = k * 256 + threadIdx.x;
+        const int r = r0 + (idx >> 4), c = c0 + (idx & 15) * 8;
+        v[k] = make_uint4(0, 0, 0, 0);
+        if (r < R) v[k] = __ldg(reinterpret_cast<const uint4 *>(x + (size_t)r * C + c));
+        m2 = amax8(m2, v[k]);
+    }
+    uint32_t m = max(m2 & 0xFFFFu, m2 >> 16);
+    m = __reduce_max_sync(0xffffffffu, m);
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = max(m, warp_max[w]);
+    const float s = block_scale_from_amax(__uint_as_float(m << 16), FMT == 0 ? 448.0f : 57344.0f);
+    if (threadIdx.x == 0) scale_inv[(size_t)blockIdx.y * gridDim.x + blockIdx.x] = __fdiv_rn(1.0f, s);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int idx = k * 256 + threadIdx.x;
+        const int r = r0 + (idx >> 4), c = c0 + (idx & 15) * 8;
+        if (r < R) *reinterpret_cast<uint2 *>(out + (size_t)r * C + c) = cast8<FMT>(v[k], s);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ GEMM
+constexpr int BM = 128, BN = 128, BK = 128;
+constexpr int STAGES = 6;
+constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int BAR_OFFSET = STAGES * STAGE_BYTES;
+// full[S], empty[S], part_full[2], part_empty[2], tmem slot, abort flag
+constexpr int TOTAL = BAR_OFFSET + (2 * STAGES + 4) * 8 + 16;
+constexpr int DYN_BYTES = TOTAL + 1024;
+constexpr int THREADS = 320;
+constexpr uint32_t TMEM_COLS = 256;
+
+// Tile order: bands of BAND tiles along the longer output dimension, the index along the shorter one advancing
+// slowest inside a band, so that the CTAs running at one time share a few operand panels that stay in L2.
+constexpr int BAND = 16;
+__device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
+{
+    const int per_band = BAND * n_short;
+    const int band = tile / per_band, within = tile - band * per_band;
+    const int len = min(BAND, n_long - band * BAND);
+    i_short = within / len;
+    i_long = band * BAND + (within - i_short * len);
+}
+
+struct Params {
+    uint16_t *out;                 // [M,N] BF16
+    const float *sx_inv;           // [K/128][M]
+    const float *sw_inv;           // [ceil(N/128)][K/128]
+    int M, N, K;
+    int *status;
+};
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const Params p)
+{
+    constexpr int S = STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_base = sbase + BAR_OFFSET;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (S + s); };
+    auto pfull_bar = [&](int b) { return bar_base + 8u * (2 * S + b); };
+    auto pempty_bar = [&](int b) { return bar_base + 8u * (2 * S + 2 + b); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + BAR_OFFSET + (2 * S + 4) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
+    const int k_blocks = p.K / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(pfull_bar(b), 1);
+            mbar_init(pempty_bar(b), 8);              // one arrival per promotion warp
+        }
+        *abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_desc(&tmap_a);
+        tma_prefetch_desc(&tmap_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const WaitCtx ctx{p.status, abort_flag};
+    auto coords = [&](int tile, int &tm, int &tn) {
+        if (tiles_m >= tiles_n) band_coords(tile, tiles_m, tiles_n, tm, tn);
+        else band_coords(tile, tiles_n, tiles_m, tn, tm);
+    };
+
+    if (warp == 0) {
+        if (elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                int tm, tn;
+                coords(tile, tm, tn);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctx)) { ok = false; break; }
+                    const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+                    tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BK, tm * BM);
+                    tma_load_2d(sb, &tmap_b, full_bar(stage), kb * BK, tn * BN);
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (elect_one()) {
+            constexpr uint32_t idesc = umma_idesc_f8(0, 0, BM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            uint32_t n = 0;                           // K-blocks issued so far (over all tiles): partial buffer n & 1
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                for (int kb = 0; kb < k_blocks; ++kb, ++n) {
+                    const int buf = (int)(n & 1u);
+                    if (!mbar_wait(pempty_bar(buf), ((n >> 1) & 1u) ^ 1u, ctx)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(stage), phase, ctx)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
+                    const uint64_t da = umma_desc_k_sw128(sa), db = umma_desc_k_sw128(sb);
+#pragma unroll
+                    for (int k = 0; k < BK / 32; ++k)
+                        umma_f8_ss(tmem_base + (uint32_t)(buf * BN), da + 2u * k, db + 2u * k, idesc, k != 0 ? 1u : 0u);
+                    umma_commit(empty_bar(stage));
+                    umma_commit(pfull_bar(buf));
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else {
+        const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;              // which 64 of the tile's 128 columns
+        constexpr int HC = BN / 2;
+        const uint32_t lane_addr = ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * HC);
+        bool ok = true;
+        uint32_t n = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            int tm, tn;
+            coords(tile, tm, tn);
+            const int row = tm * BM + quad * 32 + lane;
+            const int n0 = tn * BN + half * HC;
+            const float *sx = p.sx_inv + (row < p.M ? row : 0);
+            const float *sw = p.sw_inv + (size_t)tn * k_blocks;
+            float acc[HC];
+#pragma unroll
+            for (int c = 0; c < HC; ++c) acc[c] = 0.0f;
+            // the two descale factors of a K-block are fetched PF K-blocks ahead: a global load per K-block on the
+            // critical path would cost more than the K-block's MMAs
+            constexpr int PF = 4;
+            float sxq[PF], swq[PF];
+#pragma unroll
+            for (int i = 0; i < PF; ++i) {
+                sxq[i] = i < k_blocks ? __ldg(sx + (size_t)i * p.M) : 0.0f;
+                swq[i] = i < k_blocks ? __ldg(sw + i) : 0.0f;
+            }
+            for (int kb = 0; kb < k_blocks; ++kb, ++n) {
+                const int buf = (int)(n & 1u);
+                const float sc = sxq[0] * swq[0];
+#pragma unroll
+                for (int i = 0; i + 1 < PF; ++i) { sxq[i] = sxq[i + 1]; swq[i] = swq[i + 1]; }
+                sxq[PF - 1] = kb + PF < k_blocks ? __ldg(sx + (size_t)(kb + PF) * p.M) : 0.0f;
+                swq[PF - 1] = kb + PF < k_blocks ? __ldg(sw + kb + PF) : 0.0f;
+                if (!mbar_wait_warp(pfull_bar(buf), (n >> 1) & 1u, ctx)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(buf * BN);
+                uint32_t r0[32], r1[32];
+                tmem_ld_32x32b_x32(taddr, r0);
+                tmem_ld_wait();
+                tmem_ld_32x32b_x32(taddr + 32u, r1);           // in flight during the first 32 FMAs
+#pragma unroll
+                for (int i = 0; i < 32; ++i) acc[i] = fmaf(__uint_as_float(r0[i]), sc, acc[i]);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pempty_bar(buf));   // the partial is in registers: the buffer is free
+#pragma unroll
+                for (int i = 0; i < 32; ++i) acc[32 + i] = fmaf(__uint_as_float(r1[i]), sc, acc[32 + i]);
+            }
+            if (ok && row < p.M) {
+                uint16_t *dst = p.out + (size_t)row * p.N + n0;
+#pragma unroll
+                for (int c = 0; c < HC; c += 8) {
+                    if (n0 + c < p.N)      // N % 16 == 0: groups of 8 are whole
+                        *reinterpret_cast<uint4 *>(dst + c) =
+                            make_uint4(pack_bf16x2(acc[c], acc[c + 1]), pack_bf16x2(acc[c + 2], acc[c + 3]),
+                                       pack_bf16x2(acc[c + 4], acc[c + 5]), pack_bf16x2(acc[c + 6], acc[c + 7]));
+                }
+            }
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace bw
+}  // namespace fp8dpa
+
+using namespace fp8dpa;
+
+extern "C" int fp8_quantize_blockwise(const void *x_bf16, size_t rows, size_t cols, int block_rows, int fmt,
+                                      uint8_t *out, float *scale_inv, void *stream)
+{
+    if (!x_bf16 || !out || !scale_inv) {
+        set_error("fp8_quantize_blockwise: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if ((fmt != FP8_E4M3 && fmt != FP8_E5M2) || (block_rows != 1 && block_rows != 128)) {
+        set_error("fp8_quantize_blockwise: fmt %d / block_rows %d not supported (E4M3 or E5M2; 1 or 128)", fmt, block_rows);
+        return FP8_ERR_ENUM;
+    }
+    if (rows == 0 || cols == 0 || (cols % 128) || rows > 0x7FFFFFFFull || cols > 0x7FFFFFFFull) {
+        set_error("fp8_quantize_blockwise: unsupported shape rows=%zu cols=%zu (cols %% 128 == 0)", rows, cols);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(x_bf16) || !aligned16(out)) {
+        set_error("fp8_quantize_blockwise: tensor pointers must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint16_t *x = static_cast<const uint16_t *>(x_bf16);
+    if (block_rows == 1) {
+        const size_t n_blocks = rows * (cols / 128);
+        size_t blocks = (n_blocks + 15) / 16;
+        const size_t cap = (size_t)sm_count() * 16;
+        if (blocks > cap) blocks = cap;
+        if (fmt == FP8_E4M3) bw::quantize_1x128_kernel<0><<<(unsigned)blocks, 256, 0, st>>>(x, rows, (int)cols, out, scale_inv);
+        else bw::quantize_1x128_kernel<1><<<(unsigned)blocks, 256, 0, st>>>(x, rows, (int)cols, out, scale_inv);
+    } else {
+        dim3 grid((unsigned)(cols / 128), (unsigned)((rows + 127) / 128));
+        if (fmt == FP8_E4M3) bw::quantize_128x128_kernel<0><<<grid, 256, 0, st>>>(x, (int)rows, (int)cols, out, scale_inv);
+        else bw::quantize_128x128_kernel<1><<<grid, 256, 0, st>>>(x, (int)rows, (int)cols, out, scale_inv);
+    }
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+extern "C" int fp8_linear_fwd_blockwise(const uint8_t *X8, const uint8_t *W8, const float *sx_inv, const float *sw_inv,
+                                        void *Y_bf16, int T, int N, int K, void *stream)
+{
+    if (!X8 || !W8 || !sx_inv || !sw_inv || !Y_bf16) {
+        set_error("fp8_linear_fwd_blockwise: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if (T <= 0 || N <= 0 || K <= 0 || (K % 128) || (N % 16)) {
+        set_error("fp8_linear_fwd_blockwise: unsupported shape T=%d N=%d K=%d (K %% 128 == 0, N %% 16 == 0)", T, N, K);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(X8) || !aligned16(W8) || !aligned16(Y_bf16)) {
+        set_error("fp8_linear_fwd_blockwise: tensor pointers must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    CUtensorMap ta, tb;
+    rc = make_tmap_2d_u8(&ta, X8, (uint64_t)T, (uint64_t)K, (uint64_t)K, bw::BM, bw::BK);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_2d_u8(&tb, W8, (uint64_t)N, (uint64_t)K, (uint64_t)K, bw::BN, bw::BK);
+    if (rc != FP8_OK) return rc;
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(bw::gemm_blockwise_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        bw::DYN_BYTES));
+    bw::Params p;
+    p.out = static_cast<uint16_t *>(Y_bf16);
+    p.sx_inv = sx_inv; p.sw_inv = sw_inv;
+    p.M = T; p.N = N; p.K = K;
+    p.status = device_status_ptr();
+    if (!p.status) return FP8_ERR_CUDA;
+    const int tiles = ((T + bw::BM - 1) / bw::BM) * ((N + bw::BN - 1) / bw::BN);
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    bw::gemm_blockwise_kernel<<<grid, bw::THREADS, bw::DYN_BYTES, static_cast<cudaStream_t>(stream)>>>(ta, tb, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
