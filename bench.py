@@ -270,12 +270,11 @@ def run_ours(args, cfg):
     h2d = sum(t.numel() * t.element_size() for t in h_in)
     d2h = sum(t.numel() * t.element_size() for t in h_out)
 
+    hin = {n: h for (n, _), h in zip(ins, h_in)}
+    hout = {n: h for (n, _), h in zip(outs, h_out)}
+
     def e2e_step():
-        for (_, d), h in zip(ins, h_in):
-            d.copy_(h, non_blocking=True)
-        hp.step()
-        for (_, d), h in zip(outs, h_out):
-            h.copy_(d, non_blocking=True)
+        hp.step_host(hin, hout)      # uploads, kernels and downloads pipelined over three streams
 
     e2e_steps = max(1, min(args.steps, 5))
     e2e_step()

@@ -153,6 +153,68 @@ class BlockHotPath:
             out += [(n, self.attn[n]) for n in ("o", "lse", "dq", "dk", "dv")]
         return out
 
+    # ------------------------------------------------------------------ host-to-host step
+    def step_host(self, h_in: dict, h_out: dict):
+        """One step on pinned host buffers: inputs go up, every output comes back.
+
+        Three streams: uploads, the kernels (the caller's current stream), downloads.  The copy engines run both
+        directions at once and under the kernels, so the step costs about max(upload, download) instead of their
+        sum.  h_in / h_out map the names of input_tensors() / output_tensors() to pinned host tensors.  On return
+        the current stream has waited for the last download.
+        """
+        main = torch.cuda.current_stream(self.device)
+        if not hasattr(self, "_up"):
+            self._up, self._down = torch.cuda.Stream(self.device), torch.cuda.Stream(self.device)
+        up, down = self._up, self._down
+        up.wait_stream(main)          # the previous step's kernels have read the device inputs
+        down.wait_stream(main)
+        groups = []                   # (inputs, kernels, outputs) per independent piece of the step
+        for lin in self.linears:
+            ins = [("x_" + lin.name, lin.x.x), ("w_" + lin.name, lin.w.x), ("dy_" + lin.name, lin.dy.x)]
+            outs = [("y_" + lin.name, lin.y), ("dx_" + lin.name, lin.dx), ("dw_" + lin.name, lin.dw)]
+            groups.append((ins, lambda lin=lin: self._run_linear(lin), outs))
+        if self.attn is not None:
+            a = self.attn
+            ins = [(n, a[n].x) for n in ("q", "k", "v", "do")]
+            outs = [(n, a[n]) for n in ("o", "lse", "dq", "dk", "dv")]
+            groups.append((ins, self._run_attention, outs))
+        ready = []
+        with torch.cuda.stream(up):
+            for ins, _, _ in groups:
+                for name, d in ins:
+                    d.copy_(h_in[name], non_blocking=True)
+                e = torch.cuda.Event()
+                e.record(up)
+                ready.append(e)
+        for (ins, run, outs), e in zip(groups, ready):
+            main.wait_event(e)
+            run()
+            done = torch.cuda.Event()
+            done.record(main)
+            with torch.cuda.stream(down):
+                down.wait_event(done)
+                for name, d in outs:
+                    h_out[name].copy_(d, non_blocking=True)
+        main.wait_stream(down)
+
+    def _run_linear(self, lin):
+        lin.x.quantize()
+        lin.w.quantize()
+        lin.dy.quantize()
+        fp8.fp8_linear_fwd(lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
+        fp8.fp8_linear_dgrad(lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+        fp8.fp8_linear_wgrad(lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+
+    def _run_attention(self):
+        a = self.attn
+        for n in ("q", "k", "v", "do"):
+            a[n].quantize()
+        fp8.fp8_attention_fwd(a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv, a["v"].scale_inv,
+                              a["softmax_scale"], True, a["o"], a["lse"], None)
+        fp8.fp8_attention_bwd(a["q"].q, a["k"].q, a["v"].q, a["do"].q, a["o"], a["lse"], a["q"].scale_inv,
+                              a["k"].scale_inv, a["v"].scale_inv, a["do"].scale_inv, a["softmax_scale"],
+                              a["ds_scale"], True, a["dq"], a["dk"], a["dv"], a["ws"], ds_amax=a["ds_amax"])
+
     # ------------------------------------------------------------------ work accounting
     def gemm_flops(self):
         return sum(l.flops for l in self.linears)

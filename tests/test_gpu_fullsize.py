@@ -151,3 +151,27 @@ def test_attention_8b_block_sampled():
 
 def test_attention_long_context_sampled():
     _attention_case("c5", kv_heads=[(0, 13)], head_rows=1024)
+
+
+def test_host_to_host_step_equals_device_step():
+    """The pipelined host-to-host step (uploads / kernels / downloads on three streams) returns the bits of step()."""
+    cfg = synth.CONFIGS["c1"]
+    hp = BlockHotPath(cfg, "cuda")
+    h = hp.generate_host_inputs()
+    hp.allocate()
+    hp.calibrate_ds_scale()
+    hp.step()
+    torch.cuda.synchronize()
+    ref = {n: t.clone() for n, t in hp.output_tensors()}
+    hin = {n: torch.from_numpy(h[n].view("int16")).view(torch.bfloat16).reshape(t.shape).pin_memory()
+           for n, t in hp.input_tensors()}
+    hout = {n: torch.empty(t.shape, dtype=t.dtype).pin_memory() for n, t in hp.output_tensors()}
+    for n, t in hp.input_tensors():
+        t.zero_()                                   # the device copies must come from the host buffers
+    for _ in range(3):                              # back-to-back steps reuse the device buffers
+        hp.step_host(hin, hout)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    for n, t in ref.items():
+        a, b = hout[n], t.cpu()
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), n
