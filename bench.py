@@ -330,6 +330,152 @@ def run_ours(args, cfg):
 GEMM_DRAM_BYTES_PER_LAUNCH = {"c4": 416.15e6}
 
 
+# ---------------------------------------------------------------------------------------------- per-kernel report
+def run_report(args):
+    """`--report`: every kernel of the library timed alone (CUDA events on the launching stream, 3 warm-ups, median of
+    `--steps` launches, a 256 MB fill between launches so that nothing is L2-resident from the previous one).  Prints
+    one JSON line {"report": [...]}; the default bench line is not affected."""
+    import numpy as np
+    import torch
+
+    import paper_2505_20524_b200 as fp8
+    from paper_2505_20524_b200 import synth
+
+    torch.cuda.set_device(0)
+    fp8.binding.load()
+    peaks = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    rows = []
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for i, (a, b) in enumerate(ev):
+            flush.fill_(i & 0xFF)
+            a.record()
+            fn()
+            b.record()
+        torch.cuda.synchronize()
+        return float(np.median([a.elapsed_time(b) for a, b in ev]))
+
+    def add(kernel, shape, ms, flops=None, nbytes=None):
+        r = {"kernel": kernel, "shape": shape, "ms": round(ms, 4)}
+        if flops is not None:
+            r["tflops"] = round(flops / ms / 1e9, 1)
+            r["frac_of_2x_bf16_burst"] = round(flops / ms / 1e9 / (2 * peaks["bf16_burst"]), 3)
+        if nbytes is not None:
+            r["gbs"] = round(nbytes / ms / 1e6, 0)
+            r["frac_of_hbm"] = round(nbytes / ms / 1e6 / peaks["hbm"], 3)
+        rows.append(r)
+
+    def f32(v=0.0):
+        return torch.full((1,), float(v), dtype=torch.float32, device="cuda")
+
+    def bf16(*shape, std=1.0):
+        return (std * torch.randn(shape, device="cuda")).to(torch.bfloat16)
+
+    def codes(*shape):
+        return torch.randint(0x20, 0x48, shape, dtype=torch.uint8, device="cuda")
+
+    # ---- quantize family (HBM): the flat sweep of workload c2 and the block tensors of c4
+    for n in (1 << 24, 1 << 27, 1 << 29):
+        x = bf16(n)
+        q = torch.empty(n, dtype=torch.uint8, device="cuda")
+        a, sc, si = f32(), f32(1.0), f32(1.0)
+        add("fp8_amax", f"{n}", timed(lambda: fp8.fp8_amax(x, a)), nbytes=2 * n)
+        add("fp8_cast e4m3", f"{n}", timed(lambda: fp8.fp8_cast(x, sc, fp8.E4M3, q)), nbytes=3 * n)
+        add("fp8_quantize e4m3 (amax + cast)", f"{n}", timed(lambda: fp8.fp8_quantize(x, fp8.E4M3, q, None, a, sc, si)),
+            nbytes=5 * n)
+        del x, q
+    c4 = synth.CONFIGS["c4"]
+    T, H, F = c4.tokens, c4.hidden, c4.ffn
+    x = bf16(T, 2 * F)
+    q, qt = torch.empty((T, 2 * F), dtype=torch.uint8, device="cuda"), torch.empty((2 * F, T), dtype=torch.uint8, device="cuda")
+    a, sc, si = f32(), f32(1.0), f32(1.0)
+    add("fp8_quantize e5m2 + transposed copy", f"{T}x{2 * F}",
+        timed(lambda: fp8.fp8_quantize(x, fp8.E5M2, q, qt, a, sc, si)), nbytes=6 * T * 2 * F)
+    h8, h8t = torch.empty((T, F), dtype=torch.uint8, device="cuda"), torch.empty((F, T), dtype=torch.uint8, device="cuda")
+    add("fp8_swiglu_cast (amax pass)", f"{T}x{F}", timed(lambda: fp8.fp8_swiglu_cast(x, None, 0, None, None, a)),
+        nbytes=4 * T * F)
+    add("fp8_swiglu_cast (cast + transposed copy)", f"{T}x{F}", timed(lambda: fp8.fp8_swiglu_cast(x, sc, 0, h8, h8t, None)),
+        nbytes=6 * T * F)
+    xa = x[:, :F].contiguous()
+    par = torch.tensor([0.8, 1.3], device="cuda")
+    for act, name in ((fp8.ACT_GELU, "gelu"), (fp8.ACT_XIELU, "xielu")):
+        add(f"fp8_act_cast {name} (amax pass)", f"{T}x{F}", timed(lambda: fp8.fp8_act_cast(xa, act, par, None, 0, None, None, a)),
+            nbytes=2 * T * F)
+        add(f"fp8_act_cast {name} (cast + transposed copy)", f"{T}x{F}",
+            timed(lambda: fp8.fp8_act_cast(xa, act, par, sc, 0, h8, h8t, None)), nbytes=4 * T * F)
+    add("fp8_kurtosis", f"{T}x{2 * F}", timed(lambda: fp8.fp8_kurtosis(x, a)), nbytes=2 * T * 2 * F)
+    del x, q, qt, h8, h8t, xa
+    r, y, g = bf16(2 * T, H), bf16(2 * T, H, std=0.02), torch.ones(H, device="cuda")
+    o_ = torch.empty_like(r)
+    for mode, name in ((fp8.NORM_RMS, "rmsnorm"), (fp8.NORM_LAYERSCALE, "layerscale")):
+        add(f"fp8_postnorm_residual {name}", f"{2 * T}x{H}", timed(lambda: fp8.fp8_postnorm_residual(r, y, g, mode, 1e-5, o_, a)),
+            nbytes=6 * 2 * T * H)
+    qk = bf16(2 * T, c4.n_q_heads, c4.head_dim)
+    qo = torch.empty_like(qk)
+    cos, sin = torch.rand((c4.seq, c4.head_dim // 2), device="cuda"), torch.rand((c4.seq, c4.head_dim // 2), device="cuda")
+    for mode, name in ((fp8.QK_RMS, "rms"), (fp8.QK_TANH, "tanh"), (fp8.QK_NONE, "none")):
+        add(f"fp8_qk_norm_rope {name} + rotary", f"{2 * T}x{c4.n_q_heads}x{c4.head_dim}",
+            timed(lambda: fp8.fp8_qk_norm_rope(qk, mode, 0.5, 1e-6, cos, sin, c4.seq, qo, a)), nbytes=4 * qk.numel())
+    del r, y, o_, qk, qo
+
+    # ---- GEMMs of c3 and c4: forward / dgrad / wgrad, the producer form and the blockwise recipe
+    for cname in ("c3", "c4"):
+        cfg = synth.CONFIGS[cname]
+        for layer, (Tt, N, K) in cfg.linear_shapes().items():
+            x8, w8, dy8 = codes(Tt, K), codes(N, K), codes(Tt, N)
+            x8t, w8t, dy8t = codes(K, Tt), codes(K, N), codes(N, Tt)
+            s1, s2 = f32(1e-2), f32(1e-2)
+            yb, dxb, dwb = (torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in ((Tt, N), (Tt, K), (N, K)))
+            fl = 2.0 * Tt * N * K
+            add("fp8_linear_fwd", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_fwd(x8, w8, s1, s2, yb)), flops=fl)
+            add("fp8_linear_dgrad", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_dgrad(dy8, w8t, s1, s2, dxb)), flops=fl)
+            add("fp8_linear_wgrad", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_wgrad(dy8t, x8t, s1, s2, dwb)), flops=fl)
+            if cname == "c4":
+                y8 = torch.empty((Tt, N), dtype=torch.uint8, device="cuda")
+                add("fp8_linear_fwd_q (fp8 epilogue + amax)", f"{cname} {layer} {Tt}x{N}x{K}",
+                    timed(lambda: fp8.fp8_linear_fwd_q(x8, w8, s1, s2, sc, fp8.E4M3, y8, a)), flops=fl)
+                sx = torch.full((K // 128, Tt), 1e-2, device="cuda")
+                sw = torch.full(((N + 127) // 128, K // 128), 1e-2, device="cuda")
+                add("fp8_linear_fwd_blockwise", f"{cname} {layer} {Tt}x{N}x{K}",
+                    timed(lambda: fp8.fp8_linear_fwd_blockwise(x8, w8, sx, sw, yb)), flops=fl)
+                xb = bf16(Tt, K)
+                add("fp8_quantize_blockwise 1x128", f"{Tt}x{K}", timed(lambda: fp8.fp8_quantize_blockwise(xb, 1, 0, x8, sx)),
+                    nbytes=3 * Tt * K)
+                del xb, y8, sx, sw
+            del x8, w8, dy8, x8t, w8t, dy8t, yb, dxb, dwb
+
+    # ---- attention of c3, c4, c5 (causal)
+    for cname in ("c3", "c4", "c5"):
+        cfg = synth.CONFIGS[cname]
+        B, N, Hq, Hkv, d = cfg.batch, cfg.seq, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+        sgn = torch.randint(0, 2, (B, N, Hq, d), dtype=torch.uint8, device="cuda") << 7
+        q8 = codes(B, N, Hq, d) | sgn
+        k8 = codes(B, N, Hkv, d) | (torch.randint(0, 2, (B, N, Hkv, d), dtype=torch.uint8, device="cuda") << 7)
+        v8 = codes(B, N, Hkv, d)
+        do8 = torch.randint(0x20, 0x40, (B, N, Hq, d), dtype=torch.uint8, device="cuda") | sgn
+        O = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda")
+        LSE = torch.empty((B, Hq, N), dtype=torch.float32, device="cuda")
+        dq, dk, dv = torch.empty_like(O), torch.empty((B, N, Hkv, d), dtype=torch.bfloat16, device="cuda"), None
+        dv = torch.empty_like(dk)
+        ws = torch.empty(fp8.fp8_attention_workspace_bytes(1, B, N, Hq, Hkv, d), dtype=torch.uint8, device="cuda")
+        s1, dss, s = f32(0.05), f32(64.0), d ** -0.5
+        fl = 2.0 * B * Hq * N * N * d
+        shape = f"{cname} B{B} N{N} H{Hq}/{Hkv} d{d}"
+        add("fp8_attention_fwd", shape, timed(lambda: fp8.fp8_attention_fwd(q8, k8, v8, s1, s1, s1, s, True, O, LSE, None)), flops=fl)
+        add("fp8_attention_bwd", shape,
+            timed(lambda: fp8.fp8_attention_bwd(q8, k8, v8, do8, O, LSE, s1, s1, s1, s1, s, dss, True, dq, dk, dv, ws)),
+            flops=2.5 * fl)
+        del q8, k8, v8, do8, O, LSE, dq, dk, dv, ws
+    status = fp8.fp8_device_status()
+    print(json.dumps({"report": rows, "device_status": status, "steps": args.steps,
+                      "peaks": {"hbm_gbs": peaks["hbm"], "bf16_tflops_burst": peaks["bf16_burst"], "source": peaks["source"]}}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -337,7 +483,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c4", choices=["c1", "c3", "c4", "c5"])
+    ap.add_argument("--report", action="store_true", help="time every kernel of the library alone and print a table")
     args = ap.parse_args()
+    if args.report:
+        return run_report(args)
     from paper_2505_20524_b200 import synth
     cfg = synth.CONFIGS[args.config]
     if args.impl == "reference":
