@@ -42,8 +42,10 @@ __device__ __forceinline__ uint32_t amax8(uint32_t m, const uint4 v)
                     v.w & 0x7FFF7FFFu);
 }
 
-// 1 x 128 blocks: 16 lanes per block (16-byte loads), two blocks per warp and sweep.  scale_inv is written
-// K-block-major, [C/128][R], which is the order the GEMM's promotion warps read it in (one row per lane).
+// 1 x 128 blocks: 16 lanes per block (16-byte loads), two blocks per warp; every thread takes BU blocks per sweep so
+// that BU loads are in flight before the first shuffle.  scale_inv is written K-block-major, [C/128][R], which is the
+// order the GEMM's promotion warps read it in (one row per lane).
+constexpr int BU = 4;
 template <int FMT>
 __global__ void __launch_bounds__(256) quantize_1x128_kernel(const uint16_t *__restrict__ x, size_t R, int C,
                                                              uint8_t *__restrict__ out, float *__restrict__ scale_inv)
@@ -52,22 +54,32 @@ __global__ void __launch_bounds__(256) quantize_1x128_kernel(const uint16_t *__r
     const size_t n_blocks = R * (size_t)ncb;
     const int j = threadIdx.x & 15;
     // uniform trip count: the shuffles name every lane
-    for (size_t base = (size_t)blockIdx.x * 16; base < n_blocks; base += (size_t)gridDim.x * 16) {
-        const size_t b_raw = base + (threadIdx.x >> 4);
-        const bool valid = b_raw < n_blocks;
-        const size_t b = valid ? b_raw : n_blocks - 1;
-        const size_t r = b / ncb;
-        const int cb = (int)(b % ncb);
-        const size_t off = r * (size_t)C + (size_t)cb * 128 + j * 8;
-        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(x + off));
-        uint32_t m2 = amax8(0u, v);
-        uint32_t m = max(m2 & 0xFFFFu, m2 >> 16);
+    for (size_t base = (size_t)blockIdx.x * (16 * BU); base < n_blocks; base += (size_t)gridDim.x * (16 * BU)) {
+        uint4 v[BU];
+        size_t off[BU], sidx[BU];
+        bool valid[BU];
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
-        const float s = block_scale_from_amax(__uint_as_float(m << 16), FMT == 0 ? 448.0f : 57344.0f);
-        if (valid) {
-            *reinterpret_cast<uint2 *>(out + off) = cast8<FMT>(v, s);
-            if (j == 0) scale_inv[(size_t)cb * R + r] = __fdiv_rn(1.0f, s);
+        for (int u = 0; u < BU; ++u) {
+            const size_t b_raw = base + (size_t)u * 16 + (threadIdx.x >> 4);
+            valid[u] = b_raw < n_blocks;
+            const size_t b = valid[u] ? b_raw : n_blocks - 1;
+            const size_t r = b / ncb;
+            const int cb = (int)(b % ncb);
+            off[u] = r * (size_t)C + (size_t)cb * 128 + j * 8;
+            sidx[u] = (size_t)cb * R + r;
+            v[u] = __ldg(reinterpret_cast<const uint4 *>(x + off[u]));
+        }
+#pragma unroll
+        for (int u = 0; u < BU; ++u) {
+            const uint32_t m2 = amax8(0u, v[u]);
+            uint32_t m = max(m2 & 0xFFFFu, m2 >> 16);
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+            const float s = block_scale_from_amax(__uint_as_float(m << 16), FMT == 0 ? 448.0f : 57344.0f);
+            if (valid[u]) {
+                *reinterpret_cast<uint2 *>(out + off[u]) = cast8<FMT>(v[u], s);
+                if (j == 0) scale_inv[sidx[u]] = __fdiv_rn(1.0f, s);
+            }
         }
     }
 }
@@ -332,7 +344,7 @@ extern "C" int fp8_quantize_blockwise(const void *x_bf16, size_t rows, size_t co
     const uint16_t *x = static_cast<const uint16_t *>(x_bf16);
     if (block_rows == 1) {
         const size_t n_blocks = rows * (cols / 128);
-        size_t blocks = (n_blocks + 15) / 16;
+        size_t blocks = (n_blocks + 16 * bw::BU - 1) / (16 * bw::BU);
         const size_t cap = (size_t)sm_count() * 16;
         if (blocks > cap) blocks = cap;
         if (fmt == FP8_E4M3) bw::quantize_1x128_kernel<0><<<(unsigned)blocks, 256, 0, st>>>(x, rows, (int)cols, out, scale_inv);
