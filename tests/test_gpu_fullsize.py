@@ -175,3 +175,77 @@ def test_host_to_host_step_equals_device_step():
     for n, t in ref.items():
         a, b = hout[n], t.cpu()
         assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), n
+
+
+def test_glue_and_producer_forms_at_c4_sizes():
+    """The (f)-row entry points at the 8B-class block's sizes, in the launch configurations bench.py --report times."""
+    from gpu_util import dev, scalar
+    cfg = synth.CONFIGS["c4"]
+    T, H, F = cfg.tokens, cfg.hidden, cfg.ffn
+    # gated activation + cast on the [T, 2F] output of the up projection: sampled rows against the oracle
+    cols = synth.choose_columns(2 * F, cfg.n_outlier_cols(2 * F), 4, 77)
+    gu = synth.normal_bf16((T, 2 * F), 4, 77, 1.0, cols, 8.0)
+    a, s, si = scalar(), scalar(), scalar()
+    x = dev(gu)
+    fp8.fp8_swiglu_cast(x, None, o.E4M3, None, None, a)
+    fp8.fp8_scale(a, o.E4M3, 0, s, si)
+    out = torch.empty((T, F), dtype=torch.uint8, device="cuda")
+    out_t = torch.empty((F, T), dtype=torch.uint8, device="cuda")
+    fp8.fp8_swiglu_cast(x, s, o.E4M3, out, out_t, None)
+    rows = _sample(T, 64, 5)
+    h = o.swiglu(np.ascontiguousarray(gu[rows]))
+    exp = o.cast(h, float(s.item()), o.E4M3)
+    got = host(out)[rows]
+    assert (got != exp).mean() <= 2e-3
+    assert np.array_equal(host(out_t)[:, rows], got.T)
+    assert abs(float(a.item()) - float(o.amax(o.swiglu(gu)))) <= 2.0 ** -7 * float(a.item())
+    del x, out, out_t
+    # post-norm + residual on the residual stream [T, H]
+    xb, yb = synth.normal_bf16((T, H), 4, 78, 1.0), synth.normal_bf16((T, H), 4, 79, 0.05)
+    g = np.full(H, 1.0 / np.sqrt(32.0), dtype=np.float32)
+    res = torch.empty((T, H), dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_postnorm_residual(dev(xb), dev(yb), torch.from_numpy(g).cuda(), o.NORM_RMS, 1e-5, res, a)
+    exp = o.postnorm_residual(xb[rows], yb[rows], g, o.NORM_RMS, 1e-5)
+    got = host(res)[rows]
+    d = got.astype(np.int32) != exp.astype(np.int32)
+    assert d.mean() <= 2e-3
+    assert float(a.item()) == float(o.amax(host(res)))
+    # producer form of the largest GEMM (up projection): bit-identical to the unfused chain
+    Tt, N, K = cfg.linear_shapes()["up"]
+    x8 = torch.randint(0x20, 0x48, (Tt, K), dtype=torch.uint8, device="cuda")
+    w8 = torch.randint(0x20, 0x48, (N, K), dtype=torch.uint8, device="cuda") | 0x80
+    s1 = scalar(2.0 ** -7)
+    ybf = torch.empty((Tt, N), dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_linear_fwd(x8, w8, s1, s1, ybf)
+    fp8.fp8_amax(ybf, a)
+    fp8.fp8_scale(scalar(float(a.item()) * 1.3), o.E4M3, 0, s, si)
+    ref8 = torch.empty((Tt, N), dtype=torch.uint8, device="cuda")
+    fp8.fp8_cast(ybf, s, o.E4M3, ref8)
+    got8 = torch.empty_like(ref8)
+    a2 = scalar()
+    fp8.fp8_linear_fwd_q(x8, w8, s1, s1, s, o.E4M3, got8, a2)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    assert torch.equal(got8, ref8) and float(a2.item()) == float(a.item())
+    del ybf, ref8, got8
+    # blockwise recipe at the QKV projection's size: sampled rows against the oracle
+    Tt, N, K = cfg.linear_shapes()["qkv"]
+    xq = synth.normal_bf16((Tt, K), 4, 80, 1.0, synth.choose_columns(K, 21, 4, 80), 30.0)
+    wq = synth.normal_bf16((N, K), 4, 81, synth.W_STD)
+    x8 = torch.empty((Tt, K), dtype=torch.uint8, device="cuda")
+    w8 = torch.empty((N, K), dtype=torch.uint8, device="cuda")
+    sx = torch.empty((K // 128, Tt), device="cuda")
+    sw = torch.empty((N // 128, K // 128), device="cuda")
+    fp8.fp8_quantize_blockwise(dev(xq), 1, o.E4M3, x8, sx)
+    fp8.fp8_quantize_blockwise(dev(wq), 128, o.E4M3, w8, sw)
+    y = torch.empty((Tt, N), dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_linear_fwd_blockwise(x8, w8, sx, sw, y)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    rows = _sample(Tt, 16, 6)
+    ox8, osx = o.quantize_blockwise(np.ascontiguousarray(xq[rows]), 1, 128, o.E4M3)
+    ow8, osw = o.quantize_blockwise(wq, 128, 128, o.E4M3)
+    assert np.array_equal(host(x8)[rows], ox8) and np.array_equal(host(w8), ow8)
+    ref, mag = o.linear_fwd_blockwise(ox8, ow8, osx, osw)
+    got = y.float().cpu().numpy().astype(np.float64)[rows]
+    assert rel_err(got, ref, mag) <= 2.0 ** -8
