@@ -288,13 +288,14 @@ int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int
     p.M = M; p.N = N; p.K = K;
     p.status = device_status_ptr();
     if (!p.status) return FP8_ERR_CUDA;
-    // CTA pairs (256 x 256 per pair, 32 KB per CTA and stage) whenever the matrix is large enough to give every
-    // pair at least two tiles: same wave quantisation as 128 x 256 tiles on single CTAs, two thirds of the L2
-    // traffic, and the epilogue still overlaps the next main loop.
+    // CTA pairs (256 x 256 per pair, 32 KB per CTA and stage) whenever the matrix gives most pairs a tile: two
+    // thirds of the L2 traffic of 128 x 256 tiles on single CTAs, and the epilogue still overlaps the next main loop.
     {
         const long pair_tiles = (long)((M + 255) / 256) * ((N + 255) / 256);
         const int fam = gemm_family_override();
-        if (fam != 1 && M >= 256 && N >= 256 && (fam == 2 || pair_tiles >= sm_count())) {
+        // (measured: from about three quarters of a wave of pairs upwards the pair kernel wins, e.g. 2048 x 2048 x
+        // 8192 with 64 pair tiles: 27 us against 36 us; below that the smaller single-CTA tiles fill more SMs)
+        if (fam != 1 && M >= 256 && N >= 256 && (fam == 2 || pair_tiles >= (3 * (sm_count() / 2)) / 4)) {
             return launch_gemm_2cta(a, b, sa_inv, sb_inv, o, M, N, K, umma_idesc_f8(fmt_a, fmt_b, 256, 256), p.status,
                                     st);
         }
