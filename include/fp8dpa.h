@@ -162,6 +162,15 @@ FP8_API int fp8_linear_wgrad(const uint8_t *dY8t, const uint8_t *X8t, const floa
                      void *dW, int out_is_fp32, int accumulate, int T, int N, int K,
                      void *ws, size_t ws_bytes, void *stream);
 
+/* The two gradients with every operand read in place, exactly as the forward product stores it: W8 [N,K],
+ * dY8 [T,N], X8 [T,K], row-major.  tcgen05 takes FP8 operands with either the reduction index or the output index
+ * contiguous, so no transposed FP8 copy has to be written by the cast (fp8_cast / fp8_quantize with out_t = NULL).
+ * Same arithmetic and outputs as fp8_linear_dgrad / fp8_linear_wgrad.  T, N, K multiples of 16. */
+FP8_API int fp8_linear_dgrad_rm(const uint8_t *dY8, const uint8_t *W8, const float *sdY_inv, const float *sW_inv,
+                        void *dX, int out_is_fp32, int T, int N, int K, void *stream);
+FP8_API int fp8_linear_wgrad_rm(const uint8_t *dY8, const uint8_t *X8, const float *sdY_inv, const float *sX_inv,
+                        void *dW, int out_is_fp32, int accumulate, int T, int N, int K, void *stream);
+
 /* Producer forms for delayed scaling (Appendix E: rho comes from the amax history, so the producer of a tensor can
  * emit FP8 in its own epilogue, "a single pass on the data", Section 2).  Same products as fp8_linear_fwd /
  * fp8_linear_dgrad; the result is rounded to BF16 (the tensor an unfused chain would store), its amax is written to

@@ -21,7 +21,7 @@ _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_qk_norm_rope", "fp8_kurtosis",
-           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
+           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
 STATIC_SCRATCH_BYTES = 32 << 20
@@ -186,6 +186,23 @@ def fp8_linear_dgrad_q(dy8, w8t, sdy_inv, sw_inv, dx_scale, dx_fmt, dx8, dx_amax
     _check(load().fp8_linear_dgrad_q(_ptr(dy8), _ptr(w8t), _ptr(sdy_inv), _ptr(sw_inv), _ptr(dx_scale),
                                      C.c_int(dx_fmt), _ptr(dx8), _ptr(dx_amax), C.c_int(T), C.c_int(N), C.c_int(K),
                                      _stream(stream)))
+
+
+def fp8_linear_dgrad_rm(dy8, w8, sdy_inv, sw_inv, dx, stream=None):
+    """dX = dY8 . W8 with W8 [N, K] read in place (no transposed copy)."""
+    T, N = dy8.shape
+    K = w8.shape[1]
+    _check(load().fp8_linear_dgrad_rm(_ptr(dy8), _ptr(w8), _ptr(sdy_inv), _ptr(sw_inv), _ptr(dx),
+                                      C.c_int(_is_fp32(dx)), C.c_int(T), C.c_int(N), C.c_int(K), _stream(stream)))
+
+
+def fp8_linear_wgrad_rm(dy8, x8, sdy_inv, sx_inv, dw, accumulate=False, stream=None):
+    """dW (+)= dY8^T . X8 with dY8 [T, N] and X8 [T, K] read in place (no transposed copies)."""
+    T, N = dy8.shape
+    K = x8.shape[1]
+    _check(load().fp8_linear_wgrad_rm(_ptr(dy8), _ptr(x8), _ptr(sdy_inv), _ptr(sx_inv), _ptr(dw),
+                                      C.c_int(_is_fp32(dw)), C.c_int(int(accumulate)), C.c_int(T), C.c_int(N),
+                                      C.c_int(K), _stream(stream)))
 
 
 def fp8_quantize_blockwise(x, block_rows, fmt, out, scale_inv, stream=None):

@@ -37,6 +37,7 @@ struct Params {
     GemmOut o;
     const float *sa_inv, *sb_inv;
     int M, N, K;
+    int a_mn, b_mn;                // operand stored with the output index contiguous ([K, M] / [K, N] in memory)
     uint32_t idesc;
     int num_pairs;
     int *status;
@@ -117,8 +118,12 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctx)) { ok = false; break; }
                     const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
                     if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
-                    tma_load_2d_pair(sa, &tmap_a, full_bar(stage), kb * BK, m0);
-                    tma_load_2d_pair(sb, &tmap_b, full_bar(stage), kb * BK, n0);
+                    // K-major tile: 128 rows of the output index x 128 reduction bytes; MN-major tile: 128 reduction
+                    // rows x 128 bytes of the output index (the matrix as it lies in memory, no transposed copy)
+                    if (p.a_mn) tma_load_2d_pair(sa, &tmap_a, full_bar(stage), m0, kb * BK);
+                    else tma_load_2d_pair(sa, &tmap_a, full_bar(stage), kb * BK, m0);
+                    if (p.b_mn) tma_load_2d_pair(sb, &tmap_b, full_bar(stage), n0, kb * BK);
+                    else tma_load_2d_pair(sb, &tmap_b, full_bar(stage), kb * BK, n0);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -140,10 +145,14 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                     if (!mbar_wait(full_bar(stage), phase, ctx)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    const uint64_t da = umma_desc_k_sw128(sa), db = umma_desc_k_sw128(sb);
+                    // 32 reduction elements per MMA: +32 bytes inside the swizzle span (K-major) or +32 rows of 128
+                    // bytes (MN-major), in 16-byte units
+                    const uint64_t da = p.a_mn ? umma_desc(sa, 128, 16) : umma_desc_k_sw128(sa);
+                    const uint64_t db = p.b_mn ? umma_desc(sb, 128, 16) : umma_desc_k_sw128(sb);
+                    const uint32_t step_a = p.a_mn ? (32u * 128u) >> 4 : 2u, step_b = p.b_mn ? (32u * 128u) >> 4 : 2u;
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
-                        umma_f8_ss_pair(tmem_d, da + 2u * k, db + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_f8_ss_pair(tmem_d, da + step_a * k, db + step_b * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
                     umma_commit_pair(empty_bar(stage), 3);      // frees the stage in both CTAs
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -203,13 +212,16 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 
 // Returns FP8_OK after launching, or a negative status.  `max_pairs` = 0 lets the runtime size the grid.
 int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, const GemmOut &o,
-                     int M, int N, int K, uint32_t idesc, int *status, cudaStream_t st)
+                     int M, int N, int K, int a_mn, int b_mn, uint32_t idesc, int *status, cudaStream_t st)
 {
     using namespace g2;
     CUtensorMap ta, tb;
-    int rc = make_tmap_2d_u8(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM, BK);
+    // an MN-major operand is the [K, M] (or [K, N]) matrix as stored: box = 128 reduction rows x 128 bytes
+    int rc = a_mn ? make_tmap_2d_u8(&ta, a, (uint64_t)K, (uint64_t)M, (uint64_t)M, BK, BM)
+                  : make_tmap_2d_u8(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM, BK);
     if (rc != FP8_OK) return rc;
-    rc = make_tmap_2d_u8(&tb, b, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
+    rc = b_mn ? make_tmap_2d_u8(&tb, b, (uint64_t)K, (uint64_t)N, (uint64_t)N, BK, BN / 2)
+              : make_tmap_2d_u8(&tb, b, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
     if (rc != FP8_OK) return rc;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
     static int max_clusters = -1;
@@ -234,6 +246,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     Params p;
     p.o = o; p.sa_inv = sa_inv; p.sb_inv = sb_inv;
     p.M = M; p.N = N; p.K = K;
+    p.a_mn = a_mn; p.b_mn = b_mn;
     p.idesc = idesc;
     p.num_pairs = tiles < max_clusters ? tiles : max_clusters;
     p.status = status;

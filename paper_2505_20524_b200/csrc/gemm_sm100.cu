@@ -44,6 +44,7 @@ struct GemmParams {
     GemmOut o;
     const float *sa_inv, *sb_inv;
     int M, N, K;
+    int a_mn, b_mn;                // operand stored with the output index contiguous (BN = 128, MT = 1 only)
     uint32_t idesc;
     int *status;
 };
@@ -129,9 +130,12 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                     const uint32_t sa = sbase + stage * L::STAGE_BYTES, sb = sa + MT * L::A_BYTES;
                     mbar_expect_tx(full_bar(stage), L::STAGE_BYTES);
 #pragma unroll
-                    for (int mt = 0; mt < MT; ++mt)
-                        tma_load_2d(sa + mt * L::A_BYTES, &tmap_a, full_bar(stage), kb * G_BK, m0 + mt * G_BM);
-                    tma_load_2d(sb, &tmap_b, full_bar(stage), kb * G_BK, n0);
+                    for (int mt = 0; mt < MT; ++mt) {
+                        if (p.a_mn) tma_load_2d(sa + mt * L::A_BYTES, &tmap_a, full_bar(stage), m0 + mt * G_BM, kb * G_BK);
+                        else tma_load_2d(sa + mt * L::A_BYTES, &tmap_a, full_bar(stage), kb * G_BK, m0 + mt * G_BM);
+                    }
+                    if (p.b_mn) tma_load_2d(sb, &tmap_b, full_bar(stage), n0, kb * G_BK);
+                    else tma_load_2d(sb, &tmap_b, full_bar(stage), kb * G_BK, n0);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -153,14 +157,19 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                     if (!mbar_wait(full_bar(stage), phase, ctx)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = sbase + stage * L::STAGE_BYTES, sb = sa + MT * L::A_BYTES;
-                    const uint64_t db = umma_desc_k_sw128(sb);
+                    const uint64_t db = p.b_mn ? umma_desc(sb, 128, 16) : umma_desc_k_sw128(sb);
+                    // 32 reduction elements per MMA: +32 bytes inside the swizzle span (K-major: +2 in 16-byte units)
+                    // or +32 rows of 128 bytes (MN-major)
+                    const uint32_t step_a = p.a_mn ? (32u * 128u) >> 4 : 2u, step_b = p.b_mn ? (32u * 128u) >> 4 : 2u;
 #pragma unroll
                     for (int k = 0; k < G_BK / 32; ++k) {
-                        // advance 32 bytes along the reduction index inside the swizzle span: +2 (16-byte units)
 #pragma unroll
-                        for (int mt = 0; mt < MT; ++mt)
-                            umma_f8_ss(tmem_d + (uint32_t)(mt * BN), umma_desc_k_sw128(sa + mt * L::A_BYTES) + 2u * k,
-                                       db + 2u * k, p.idesc, (kb | k) != 0 ? 1u : 0u);
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const uint32_t sam = sa + mt * L::A_BYTES;
+                            const uint64_t da = p.a_mn ? umma_desc(sam, 128, 16) : umma_desc_k_sw128(sam);
+                            umma_f8_ss(tmem_d + (uint32_t)(mt * BN), da + step_a * k, db + step_b * k, p.idesc,
+                                       (kb | k) != 0 ? 1u : 0u);
+                        }
                     }
                     umma_commit(empty_bar(stage));   // frees the stage once these MMAs have read it
                     if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -222,7 +231,7 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 }
 
 int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, const GemmOut &o,
-                     int M, int N, int K, uint32_t idesc, int *status, cudaStream_t st);
+                     int M, int N, int K, int a_mn, int b_mn, uint32_t idesc, int *status, cudaStream_t st);
 
 // FP8DPA_GEMM=1cta|2cta forces one kernel family (for A/B measurements); default: chosen per shape.
 static int gemm_family_override()
@@ -255,9 +264,12 @@ static int launch_gemm(const uint8_t *a, const uint8_t *b, const GemmParams &p, 
 {
     using L = GemmCfg<BN, MT>;
     CUtensorMap ta, tb;
-    int rc = make_tmap_2d_u8(&ta, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, G_BM, G_BK);
+    // an MN-major operand is the [K, M] (or [K, N]) matrix as stored: box = 128 reduction rows x 128 bytes
+    int rc = p.a_mn ? make_tmap_2d_u8(&ta, a, (uint64_t)p.K, (uint64_t)p.M, (uint64_t)p.M, G_BK, G_BM)
+                    : make_tmap_2d_u8(&ta, a, (uint64_t)p.M, (uint64_t)p.K, (uint64_t)p.K, G_BM, G_BK);
     if (rc != FP8_OK) return rc;
-    rc = make_tmap_2d_u8(&tb, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN, G_BK);
+    rc = p.b_mn ? make_tmap_2d_u8(&tb, b, (uint64_t)p.K, (uint64_t)p.N, (uint64_t)p.N, G_BK, BN)
+                : make_tmap_2d_u8(&tb, b, (uint64_t)p.N, (uint64_t)p.K, (uint64_t)p.K, BN, G_BK);
     if (rc != FP8_OK) return rc;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_kernel<BN, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         L::DYN_BYTES));
@@ -269,8 +281,10 @@ static int launch_gemm(const uint8_t *a, const uint8_t *b, const GemmParams &p, 
 }
 
 // C[M,N] (+)= sa_inv*sb_inv * A[M,K] . B[N,K]^T
+// a_mn / b_mn: that operand is given as the [K, M] (or [K, N]) matrix, i.e. the way the other two products of a
+// linear layer store it, and is read in place as an MN-major UMMA operand: no transposed copy exists anywhere.
 int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int fmt_b, const float *sa_inv,
-             const float *sb_inv, const GemmOut &o, int M, int N, int K, cudaStream_t st)
+             const float *sb_inv, const GemmOut &o, int M, int N, int K, cudaStream_t st, int a_mn = 0, int b_mn = 0)
 {
     int rc = validate_gemm(who, a, b, sa_inv, sb_inv, o.out, M, N, K);
     if (rc != FP8_OK) return rc;
@@ -281,7 +295,13 @@ int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int
     rc = check_arch();
     if (rc != FP8_OK) return rc;
     if (o.q_scale && o.amax_bits) FP8_CUDA_CHECK(cudaMemsetAsync(o.amax_bits, 0, sizeof(float), st));
+    if ((a_mn && (M % 16)) || (b_mn && (N % 16))) {
+        set_error("%s: an operand read in place needs its contiguous extent to be a multiple of 16 (rows=%d cols=%d)", who,
+                  M, N);
+        return FP8_ERR_SHAPE;
+    }
     GemmParams p;
+    p.a_mn = a_mn; p.b_mn = b_mn;
     p.o = o;
     p.sa_inv = sa_inv;
     p.sb_inv = sb_inv;
@@ -296,8 +316,8 @@ int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int
         // (measured: from about three quarters of a wave of pairs upwards the pair kernel wins, e.g. 2048 x 2048 x
         // 8192 with 64 pair tiles: 27 us against 36 us; below that the smaller single-CTA tiles fill more SMs)
         if (fam != 1 && M >= 256 && N >= 256 && (fam == 2 || pair_tiles >= (3 * (sm_count() / 2)) / 4)) {
-            return launch_gemm_2cta(a, b, sa_inv, sb_inv, o, M, N, K, umma_idesc_f8(fmt_a, fmt_b, 256, 256), p.status,
-                                    st);
+            return launch_gemm_2cta(a, b, sa_inv, sb_inv, o, M, N, K, a_mn, b_mn,
+                                    umma_idesc_f8(fmt_a, fmt_b, 256, 256, a_mn, b_mn), p.status, st);
         }
     }
     // Tile choice.  The 256 x 256 tile needs 2/3 of the L2 traffic of 128 x 256 but cannot overlap its epilogue
@@ -307,6 +327,11 @@ int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int
     auto waves = [&](long tiles) { return (double)((tiles + sms - 1) / sms); };
     const long t256 = (long)((M + 255) / 256) * ((N + 255) / 256);
     const long t128x256 = (long)((M + 127) / 128) * ((N + 255) / 256);
+    if (a_mn || b_mn) {
+        // operands read in place: one 128-byte swizzle span per operand tile, i.e. the 128 x 128 tile
+        p.idesc = umma_idesc_f8(fmt_a, fmt_b, G_BM, 128, a_mn, b_mn);
+        return launch_gemm<128, 1>(a, b, p, st);
+    }
     if (N >= 256 && M >= 256 && K >= 8192 && 2.0 * waves(t256) <= 1.02 * waves(t128x256)) {
         p.idesc = umma_idesc_f8(fmt_a, fmt_b, G_BM, 256);
         return launch_gemm<256, 2>(a, b, p, st);
@@ -378,4 +403,24 @@ extern "C" int fp8_linear_dgrad_q(const uint8_t *dY8, const uint8_t *W8t, const 
     const GemmOut o{dX8, 0, 0, dx_scale, dx_fmt, reinterpret_cast<unsigned int *>(dx_amax)};
     return gemm_fp8("fp8_linear_dgrad_q", dY8, FP8_E5M2, W8t, FP8_E4M3, sdY_inv, sW_inv, o, T, K, N,
                     static_cast<cudaStream_t>(stream));
+}
+
+// The same two gradients with every operand read in place, as stored for the forward product: W8 [N,K], dY8 [T,N],
+// X8 [T,K].  No transposed FP8 copies are needed (tcgen05 takes FP8 operands with either index contiguous).
+extern "C" int fp8_linear_dgrad_rm(const uint8_t *dY8, const uint8_t *W8, const float *sdY_inv, const float *sW_inv,
+                                   void *dX, int out_is_fp32, int T, int N, int K, void *stream)
+{
+    // dX[T,K] = dY8[T,N] . W8[N,K] : rows T, cols K, reduce N; B = W8 is [reduce, cols] in memory
+    const GemmOut o{dX, out_is_fp32, 0, nullptr, 0, nullptr};
+    return gemm_fp8("fp8_linear_dgrad_rm", dY8, FP8_E5M2, W8, FP8_E4M3, sdY_inv, sW_inv, o, T, K, N,
+                    static_cast<cudaStream_t>(stream), 0, 1);
+}
+
+extern "C" int fp8_linear_wgrad_rm(const uint8_t *dY8, const uint8_t *X8, const float *sdY_inv, const float *sX_inv,
+                                   void *dW, int out_is_fp32, int accumulate, int T, int N, int K, void *stream)
+{
+    // dW[N,K] = dY8[T,N]^T . X8[T,K] : rows N, cols K, reduce T; both operands are [reduce, output] in memory
+    const GemmOut o{dW, out_is_fp32, accumulate, nullptr, 0, nullptr};
+    return gemm_fp8("fp8_linear_wgrad_rm", dY8, FP8_E5M2, X8, FP8_E4M3, sdY_inv, sX_inv, o, N, K, T,
+                    static_cast<cudaStream_t>(stream), 1, 1);
 }

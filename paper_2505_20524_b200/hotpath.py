@@ -1,6 +1,7 @@
 """One pass of the whole FP8 hot path over a transformer block's tensors, as a sequence of C-ABI calls.
 
-A step is: just-in-time quantize (amax -> scale -> cast, with transposed copies) of every activation, weight
+A step is: just-in-time quantize (amax -> scale -> cast; no transposed copies: the gradient products read the
+row-major FP8 tensors in place) of every activation, weight
 and upstream gradient; forward, dgrad and wgrad GEMMs of the QKV, output, up(-gate) and down projections;
 quantize of Q, K, V, dO; FP8 attention forward and backward.  This module only owns device buffers (torch)
 and the order of calls; every computation runs in the CUDA library.
@@ -79,9 +80,12 @@ class BlockHotPath:
     KERNELS_PER_ATTN_BWD = 3    # prep, main, finish
 
     def __init__(self, cfg: synth.BlockConfig, device="cuda", with_linears=None, with_attention=True,
-                 seq=None, batch=None):
+                 seq=None, batch=None, transposed_copies=False):
+        # transposed_copies: also write [cols, rows] FP8 copies in the cast and run dgrad / wgrad on them (the
+        # form a K-major-only tensor core needs); off by default, tcgen05 reads the operands in place
         self.cfg = cfg
         self.device = torch.device(device)
+        self.transposed_copies = transposed_copies
         self.with_linears = cfg.has_linears if with_linears is None else with_linears
         self.with_attention = with_attention
         self.B = cfg.batch if batch is None else batch
@@ -111,9 +115,9 @@ class BlockHotPath:
             for layer in LAYERS:
                 T, N, K = self.cfg.linear_shapes()[layer]
                 lin = Linear(layer, T, N, K,
-                             QTensor(_bits_to_dev(h["x_" + layer], dev), fp8.E4M3, True),
-                             QTensor(_bits_to_dev(h["w_" + layer], dev), fp8.E4M3, True),
-                             QTensor(_bits_to_dev(h["dy_" + layer], dev), fp8.E5M2, True))
+                             QTensor(_bits_to_dev(h["x_" + layer], dev), fp8.E4M3, self.transposed_copies),
+                             QTensor(_bits_to_dev(h["w_" + layer], dev), fp8.E4M3, self.transposed_copies),
+                             QTensor(_bits_to_dev(h["dy_" + layer], dev), fp8.E5M2, self.transposed_copies))
                 lin.y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
                 lin.dx = torch.empty((T, K), dtype=torch.bfloat16, device=dev)
                 lin.dw = torch.empty((N, K), dtype=torch.bfloat16, device=dev)
@@ -202,8 +206,12 @@ class BlockHotPath:
         lin.w.quantize()
         lin.dy.quantize()
         fp8.fp8_linear_fwd(lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
-        fp8.fp8_linear_dgrad(lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
-        fp8.fp8_linear_wgrad(lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+        if self.transposed_copies:
+            fp8.fp8_linear_dgrad(lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+            fp8.fp8_linear_wgrad(lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+        else:
+            fp8.fp8_linear_dgrad_rm(lin.dy.q, lin.w.q, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+            fp8.fp8_linear_wgrad_rm(lin.dy.q, lin.x.q, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
 
     def _run_attention(self):
         a = self.attn
@@ -276,8 +284,12 @@ class BlockHotPath:
             lin.w.quantize()
             lin.dy.quantize()
             gemm(fp8.fp8_linear_fwd, lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
-            gemm(fp8.fp8_linear_dgrad, lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
-            gemm(fp8.fp8_linear_wgrad, lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+            if self.transposed_copies:
+                gemm(fp8.fp8_linear_dgrad, lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+                gemm(fp8.fp8_linear_wgrad, lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+            else:
+                gemm(fp8.fp8_linear_dgrad_rm, lin.dy.q, lin.w.q, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+                gemm(fp8.fp8_linear_wgrad_rm, lin.dy.q, lin.x.q, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
         if self.attn is not None:
             a = self.attn
             for n in ("q", "k", "v", "do"):

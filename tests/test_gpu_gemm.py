@@ -187,3 +187,44 @@ def test_fp8_output_argument_validation():
     with pytest.raises(fp8.Fp8Error) as e:
         fp8.fp8_linear_fwd_q(x8, x8, s, s, s, 3, x8)
     assert e.value.status == -4
+
+
+@pytest.mark.parametrize("family", ["1cta", "2cta"])
+@pytest.mark.parametrize("T,N,K", [(256, 768, 256), (400, 528, 144), (1024, 1040, 2064), (16, 16, 16), (512, 256, 1024)])
+def test_gradients_with_operands_read_in_place(family, T, N, K, monkeypatch):
+    """dgrad / wgrad on the row-major FP8 tensors of the forward (MN-major UMMA operands) against the oracle and
+    against the transposed-copy path."""
+    monkeypatch.setenv("FP8DPA_GEMM", family)
+    seed = 3 * T + N + K
+    cols = synth.choose_columns(K, 2, seed, 1)
+    x = synth.normal_bf16((T, K), seed, 0, 1.0, cols, 50.0)
+    w = synth.normal_bf16((N, K), seed, 1, synth.W_STD)
+    dy = synth.normal_bf16((T, N), seed, 2, synth.GRAD_STD)
+    x8, x8t, _, _, sx = gpu_quantize(x, o.E4M3, True)
+    w8, w8t, _, _, sw = gpu_quantize(w, o.E4M3, True)
+    dy8, dy8t, _, _, sdy = gpu_quantize(dy, o.E5M2, True)
+    for dt, tol in ((torch.bfloat16, 2.0 ** -8), (torch.float32, TOL_FP32)):
+        dx = torch.empty((T, K), dtype=dt, device="cuda")
+        dw = torch.empty((N, K), dtype=dt, device="cuda")
+        fp8.fp8_linear_dgrad_rm(dy8, w8, sdy, sw, dx)
+        fp8.fp8_linear_wgrad_rm(dy8, x8, sdy, sx, dw)
+        dx2, dw2 = torch.empty_like(dx), torch.empty_like(dw)
+        fp8.fp8_linear_dgrad(dy8, w8t, sdy, sw, dx2)
+        fp8.fp8_linear_wgrad(dy8t, x8t, sdy, sx, dw2)
+        torch.cuda.synchronize()
+        assert fp8.fp8_device_status() == 0
+        ox8, _, _, osx = o.quantize(x, o.E4M3)
+        ow8, _, _, osw = o.quantize(w, o.E4M3)
+        ody8, _, _, osdy = o.quantize(dy, o.E5M2)
+        ref, mag = o.linear_dgrad(ody8, ow8, osdy, osw)
+        check(dx, ref, mag, tol)
+        ref, mag = o.linear_wgrad(ody8, ox8, osdy, osx)
+        check(dw, ref, mag, tol)
+        # the same products in the same order of reduction: the two operand forms agree to FP32 accumulation noise
+        assert (dx.float() - dx2.float()).abs().max().item() <= 2.0 ** -7 * dx2.float().abs().max().item() + 1e-30
+        assert (dw.float() - dw2.float()).abs().max().item() <= 2.0 ** -7 * dw2.float().abs().max().item() + 1e-30
+    # accumulate into FP32 weight gradients
+    acc = torch.full((N, K), 0.5, dtype=torch.float32, device="cuda")
+    fp8.fp8_linear_wgrad_rm(dy8, x8, sdy, sx, acc, accumulate=True)
+    ref, mag = o.linear_wgrad(ody8, ox8, osdy, osx, prev=np.full((N, K), 0.5))
+    check(acc, ref, mag + 0.5, TOL_FP32)
