@@ -69,7 +69,7 @@ __device__ __forceinline__ float e5m2_to_f32(uint32_t code)
 }
 
 // ---------------------------------------------------------------- prep
-// One warp per (b, i, h) with i < Npad: D_i = do_inv * sum_d dec(dO8) * O, then
+// Eight lanes per (b, i, h) with i < Npad (16-byte loads): D_i = do_inv * sum_d dec(dO8) * O, then
 // lse2 = LSE*log2e - log2(c_P), db = D * ds_scale / c_P; rows i >= N get (+inf, 0); the dQ accumulator row
 // is zeroed.
 __global__ void __launch_bounds__(256) attn_bwd_d128_prep_kernel(const uint8_t *__restrict__ dO8, const uint16_t *__restrict__ O,
@@ -79,40 +79,67 @@ __global__ void __launch_bounds__(256) attn_bwd_d128_prep_kernel(const uint8_t *
                                                    float *__restrict__ db, float *__restrict__ dQacc, int B, int N,
                                                    int Npad, int Hq)
 {
-    const long w = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (b*Npad + i)*Hq + h
-    const int lane = threadIdx.x & 31;
-    if (w >= (long)B * Npad * Hq) return;
-    const int h = (int)(w % Hq);
-    const long bi = w / Hq;
-    const int i = (int)(bi % Npad), b = (int)(bi / Npad);
-    const size_t vi = ((size_t)b * Hq + h) * Npad + i;
-    if (i >= N) {
-        if (lane == 0) {
-            lse2[vi] = INFINITY;
-            db[vi] = 0.0f;
-        }
-        return;
-    }
-    const size_t row = ((size_t)b * N + i) * Hq + h;
-    const uint32_t c4 = *reinterpret_cast<const uint32_t *>(dO8 + row * D + lane * 4);
-    const uint2 o4 = *reinterpret_cast<const uint2 *>(O + row * D + lane * 4);
-    float acc = e5m2_to_f32(c4 & 0xFF) * bf16_lo(o4.x) + e5m2_to_f32((c4 >> 8) & 0xFF) * bf16_hi(o4.x) +
-                e5m2_to_f32((c4 >> 16) & 0xFF) * bf16_lo(o4.y) + e5m2_to_f32(c4 >> 24) * bf16_hi(o4.y);
+    const long n_rows = (long)B * Npad * Hq;
+    const int j = threadIdx.x & 7;
+    const float scale = __ldg(do_inv) * __ldg(ds_scale) / p_scale;
+    // the trip count is uniform over the CTA: the shuffles below name every lane
+    for (long base = (long)blockIdx.x * 32; base < n_rows; base += (long)gridDim.x * 32) {
+        const long w_raw = base + (threadIdx.x >> 3);            // (b*Npad + i)*Hq + h
+        const bool in_range = w_raw < n_rows;
+        const long w = in_range ? w_raw : n_rows - 1;
+        const int h = (int)(w % Hq);
+        const long bi = w / Hq;
+        const int i = (int)(bi % Npad), b = (int)(bi / Npad);
+        const size_t vi = ((size_t)b * Hq + h) * Npad + i;
+        const bool real = i < N;
+        const size_t row = ((size_t)b * N + (real ? i : 0)) * Hq + h;
+        float acc = 0.0f;
+        if (real) {
+            const uint4 c = __ldg(reinterpret_cast<const uint4 *>(dO8 + row * D + j * 16));
+            const uint4 o0 = __ldg(reinterpret_cast<const uint4 *>(O + row * D + j * 16));
+            const uint4 o1 = __ldg(reinterpret_cast<const uint4 *>(O + row * D + j * 16 + 8));
+            const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
+            const uint32_t ow[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    *reinterpret_cast<float4 *>(dQacc + row * D + lane * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (lane == 0) {
-        lse2[vi] = __ldg(LSE + ((size_t)b * Hq + h) * N + i) * 1.4426950408889634f - log2_p_scale;
-        db[vi] = acc * __ldg(do_inv) * __ldg(ds_scale) / p_scale;
+            for (int q = 0; q < 4; ++q) {
+                acc = fmaf(e5m2_to_f32(cw[q] & 0xFF), bf16_lo(ow[2 * q]), acc);
+                acc = fmaf(e5m2_to_f32((cw[q] >> 8) & 0xFF), bf16_hi(ow[2 * q]), acc);
+                acc = fmaf(e5m2_to_f32((cw[q] >> 16) & 0xFF), bf16_lo(ow[2 * q + 1]), acc);
+                acc = fmaf(e5m2_to_f32(cw[q] >> 24), bf16_hi(ow[2 * q + 1]), acc);
+            }
+        }
+#pragma unroll
+        for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        if (!in_range) continue;
+        if (real) {
+            float4 *z = reinterpret_cast<float4 *>(dQacc + row * D + j * 16);
+            const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+            z[0] = zero; z[1] = zero; z[2] = zero; z[3] = zero;
+        }
+        if (j == 0) {
+            lse2[vi] = real ? __ldg(LSE + ((size_t)b * Hq + h) * N + i) * 1.4426950408889634f - log2_p_scale : INFINITY;
+            db[vi] = real ? acc * scale : 0.0f;
+        }
     }
 }
 
+// dQ = s * k_inv / ds_scale * accumulator, BF16; four 16-byte loads in flight per thread
 __global__ void __launch_bounds__(256) attn_bwd_d128_finish_kernel(const float4 *__restrict__ acc, uint2 *__restrict__ dQ, size_t n4,
                                                      const float *__restrict__ k_inv,
                                                      const float *__restrict__ ds_scale, float softmax_scale)
 {
     const float f = softmax_scale * __ldg(k_inv) / __ldg(ds_scale);
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n4; i += 4 * stride) {
+        const float4 v0 = __ldcs(acc + i), v1 = __ldcs(acc + i + stride), v2 = __ldcs(acc + i + 2 * stride),
+                     v3 = __ldcs(acc + i + 3 * stride);
+        dQ[i] = make_uint2(pack_bf16x2(v0.x * f, v0.y * f), pack_bf16x2(v0.z * f, v0.w * f));
+        dQ[i + stride] = make_uint2(pack_bf16x2(v1.x * f, v1.y * f), pack_bf16x2(v1.z * f, v1.w * f));
+        dQ[i + 2 * stride] = make_uint2(pack_bf16x2(v2.x * f, v2.y * f), pack_bf16x2(v2.z * f, v2.w * f));
+        dQ[i + 3 * stride] = make_uint2(pack_bf16x2(v3.x * f, v3.y * f), pack_bf16x2(v3.z * f, v3.w * f));
+    }
+    for (; i < n4; i += stride) {
         const float4 v = acc[i];
         dQ[i] = make_uint2(pack_bf16x2(v.x * f, v.y * f), pack_bf16x2(v.z * f, v.w * f));
     }
@@ -476,8 +503,10 @@ int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8
     if (rc != FP8_OK) return rc;
     if (sc->ds_amax) FP8_CUDA_CHECK(cudaMemsetAsync(sc->ds_amax, 0, sizeof(float), st));
     const float log2_p = log2f(sc->p_scale);
-    const long warps = (long)B * Npad * Hq;
-    attn_bwd_d128_prep_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, st>>>(dO8, O, LSE, sc->do_inv, sc->ds_scale, sc->p_scale, log2_p,
+    const long prep_rows = (long)B * Npad * Hq;
+    long prep_blocks = (prep_rows + 31) / 32;                   // 32 rows per CTA and sweep
+    if (prep_blocks > (long)sm_count() * 16) prep_blocks = (long)sm_count() * 16;
+    attn_bwd_d128_prep_kernel<<<(unsigned)prep_blocks, 256, 0, st>>>(dO8, O, LSE, sc->do_inv, sc->ds_scale, sc->p_scale, log2_p,
                                                             lse2, db, dQacc, B, N, Npad, Hq);
     FP8_CUDA_CHECK(cudaGetLastError());
     Params p;
