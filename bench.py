@@ -434,6 +434,10 @@ def run_report(args):
             add("fp8_linear_fwd", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_fwd(x8, w8, s1, s2, yb)), flops=fl)
             add("fp8_linear_dgrad", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_dgrad(dy8, w8t, s1, s2, dxb)), flops=fl)
             add("fp8_linear_wgrad", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_wgrad(dy8t, x8t, s1, s2, dwb)), flops=fl)
+            add("fp8_linear_dgrad_rm (W8 read in place)", f"{cname} {layer} {Tt}x{N}x{K}",
+                timed(lambda: fp8.fp8_linear_dgrad_rm(dy8, w8, s1, s2, dxb)), flops=fl)
+            add("fp8_linear_wgrad_rm (dY8, X8 read in place)", f"{cname} {layer} {Tt}x{N}x{K}",
+                timed(lambda: fp8.fp8_linear_wgrad_rm(dy8, x8, s1, s2, dwb)), flops=fl)
             if cname == "c4":
                 y8 = torch.empty((Tt, N), dtype=torch.uint8, device="cuda")
                 add("fp8_linear_fwd_q (fp8 epilogue + amax)", f"{cname} {layer} {Tt}x{N}x{K}",
