@@ -452,6 +452,22 @@ def run_report(args):
                 del xb, y8, sx, sw
             del x8, w8, dy8, x8t, w8t, dy8t, yb, dxb, dwb
 
+    # ---- grouped (mixture-of-experts) forward product: 8 experts, 2 active, c3-sized FFN
+    c3 = synth.CONFIGS["c3"]
+    E, Tr = 8, 2 * c3.tokens                                   # every token is routed to 2 experts
+    rng = np.random.default_rng(1)
+    wts = np.maximum(1e-3, 1 + 0.3 * rng.standard_normal(E))
+    sizes = np.floor(wts / wts.sum() * Tr).astype(int)
+    sizes[-1] += Tr - sizes.sum()
+    offs = torch.from_numpy(np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)).cuda()
+    Ng, Kg = 2 * c3.ffn, c3.hidden
+    x8, w8 = codes(Tr, Kg), codes(E, Ng, Kg)
+    yb = torch.empty((Tr, Ng), dtype=torch.bfloat16, device="cuda")
+    s1, swg = f32(1e-2), torch.full((E,), 1e-2, device="cuda")
+    add("fp8_grouped_linear_fwd (8 experts, uneven)", f"{Tr} rows x {Ng} x {Kg}",
+        timed(lambda: fp8.fp8_grouped_linear_fwd(x8, w8, s1, swg, offs, yb)), flops=2.0 * Tr * Ng * Kg)
+    del x8, w8, yb
+
     # ---- attention of c3, c4, c5 (causal)
     for cname in ("c3", "c4", "c5"):
         cfg = synth.CONFIGS[cname]

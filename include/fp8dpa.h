@@ -171,6 +171,16 @@ FP8_API int fp8_linear_dgrad_rm(const uint8_t *dY8, const uint8_t *W8, const flo
 FP8_API int fp8_linear_wgrad_rm(const uint8_t *dY8, const uint8_t *X8, const float *sdY_inv, const float *sX_inv,
                         void *dW, int out_is_fp32, int accumulate, int T, int N, int K, void *stream);
 
+/* Grouped forward product for a mixture-of-experts FFN (Appendix D: sparse FFNs, 8 experts of which 2 are
+ * active per token): X8 [T,K] holds the routed token copies sorted by expert; expert g owns the rows
+ * [group_offsets[g], group_offsets[g+1]) (device int32 array of n_groups + 1 ascending entries, the router's output,
+ * group_offsets[0] = 0, group_offsets[n_groups] <= T), the weights W8[g] ([N,K] each, stored back to back) and the
+ * descale sW_inv[g].  Y[t, :] = sX_inv * sW_inv[g(t)] * X8[t, :] . W8[g(t)]^T, one launch for all experts; rows
+ * past group_offsets[n_groups] are left untouched.  n_groups <= 256. */
+FP8_API int fp8_grouped_linear_fwd(const uint8_t *X8, const uint8_t *W8, const float *sX_inv, const float *sW_inv,
+                           const int *group_offsets, int n_groups, void *Y, int out_is_fp32, int T, int N, int K,
+                           void *stream);
+
 /* Producer forms for delayed scaling (Appendix E: rho comes from the amax history, so the producer of a tensor can
  * emit FP8 in its own epilogue, "a single pass on the data", Section 2).  Same products as fp8_linear_fwd /
  * fp8_linear_dgrad; the result is rounded to BF16 (the tensor an unfused chain would store), its amax is written to

@@ -41,7 +41,13 @@ struct Params {
     uint32_t idesc;
     int num_pairs;
     int *status;
+    // grouped form (mixture-of-experts FFN: the rows of A are sorted by expert, every expert has its own B):
+    // group g owns rows [group_offsets[g], group_offsets[g+1]) of A and C, rows [g*N, (g+1)*N) of B and the
+    // descale sb_inv[g]; the offsets live on the device (they come out of the router)
+    const int *group_offsets;
+    int n_groups;
 };
+constexpr int MAX_GROUPS = 256;
 
 constexpr int BAND = 16;
 __device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
@@ -58,9 +64,29 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
     else band_coords(tile, tiles_n, tiles_m, tn, tm);
 }
 
+// Tile -> (group, row offset of the group, rows of the group, tile coordinates inside the group) for the grouped form:
+// tile_start[g] = first tile of group g (tiles of a group: ceil(rows / 256) x tiles_n, row tile fastest).
+struct GroupTile { int g, row0, rows, tm, tn; };
+__device__ __forceinline__ GroupTile group_tile(const int *tile_start, const int *offs, int n_groups, int tiles_n, int tile)
+{
+    int g = 0;
+    while (g + 1 < n_groups && tile >= tile_start[g + 1]) ++g;
+    const int local = tile - tile_start[g];
+    const int rows = offs[g + 1] - offs[g];
+    const int tiles_m = (rows + 2 * BM - 1) / (2 * BM);
+    GroupTile t;
+    t.g = g; t.row0 = offs[g]; t.rows = rows;
+    t.tn = local / tiles_m;
+    t.tm = local - t.tn * tiles_m;
+    return t;
+}
+
+template <bool GROUPED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p)
 {
+    __shared__ int g_tile_start[GROUPED ? MAX_GROUPS + 1 : 1];
+    __shared__ int g_offs[GROUPED ? MAX_GROUPS + 1 : 1];
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
@@ -76,8 +102,24 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const uint32_t rank = cluster_ctarank();            // 0 = even CTA (issues the MMAs), 1 = its peer
     const int pair = blockIdx.x >> 1;
     const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
-    const int num_tiles = tiles_m * tiles_n;
+    int num_tiles = tiles_m * tiles_n;
     const int k_blocks = (p.K + BK - 1) / BK;
+    if (GROUPED) {
+        // every CTA builds the same tile table from the device-side offsets
+        if (threadIdx.x == 0) {
+            int acc = 0;
+            for (int g = 0; g < p.n_groups; ++g) {
+                const int o0 = __ldg(p.group_offsets + g), o1 = __ldg(p.group_offsets + g + 1);
+                g_offs[g] = o0;
+                g_tile_start[g] = acc;
+                acc += ((max(o1 - o0, 0) + 2 * BM - 1) / (2 * BM)) * tiles_n;
+            }
+            g_offs[p.n_groups] = __ldg(p.group_offsets + p.n_groups);
+            g_tile_start[p.n_groups] = acc;
+        }
+        __syncthreads();
+        num_tiles = g_tile_start[p.n_groups];
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -111,9 +153,16 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs) {
-                int tm, tn;
-                tile_coords(tile, tiles_m, tiles_n, tm, tn);
-                const int m0 = tm * 2 * BM + (int)rank * BM, n0 = tn * BN + (int)rank * (BN / 2);
+                int tm, tn, m_base = 0, n_base = 0;
+                if (GROUPED) {
+                    const GroupTile gt = group_tile(g_tile_start, g_offs, p.n_groups, tiles_n, tile);
+                    tm = gt.tm; tn = gt.tn;
+                    m_base = gt.row0;              // rows of A: the group's slice of the sorted token matrix
+                    n_base = gt.g * p.N;           // rows of B: the group's weight matrix
+                } else {
+                    tile_coords(tile, tiles_m, tiles_n, tm, tn);
+                }
+                const int m0 = m_base + tm * 2 * BM + (int)rank * BM, n0 = n_base + tn * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctx)) { ok = false; break; }
                     const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
@@ -170,9 +219,18 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            int tm, tn;
-            tile_coords(tile, tiles_m, tiles_n, tm, tn);
-            const int m0 = tm * 2 * BM + (int)rank * BM, n0 = tn * BN;
+            int tm, tn, m_base = 0, m_end = p.M;
+            float descale_t = descale;
+            if (GROUPED) {
+                const GroupTile gt = group_tile(g_tile_start, g_offs, p.n_groups, tiles_n, tile);
+                tm = gt.tm; tn = gt.tn;
+                m_base = gt.row0;
+                m_end = gt.row0 + gt.rows;         // rows past the group's end belong to the next group: not stored
+                descale_t = __ldg(p.sa_inv) * __ldg(p.sb_inv + gt.g);
+            } else {
+                tile_coords(tile, tiles_m, tiles_n, tm, tn);
+            }
+            const int m0 = m_base + tm * 2 * BM + (int)rank * BM, n0 = tn * BN;
             if (!mbar_wait_warp(tfull_bar(buf), acc_phase, ctx)) { ok = false; break; }
             tc_fence_after();
             const int row = m0 + quad * 32 + lane;
@@ -183,8 +241,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                 tmem_ld_32x32b_x32(taddr + (uint32_t)c, r);
                 tmem_ld_wait();
                 const int col = n0 + c;
-                if (row < p.M && col < p.N)
-                    gemm_store_chunk(r, descale, p.o, q_scale, p.N, row, col, min(32, p.N - col), amax2);
+                if (row < m_end && col < p.N)
+                    gemm_store_chunk(r, descale_t, p.o, q_scale, p.N, row, col, min(32, p.N - col), amax2);
             }
             tc_fence_before();
             __syncwarp();
@@ -223,7 +281,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     rc = b_mn ? make_tmap_2d_u8(&tb, b, (uint64_t)K, (uint64_t)N, (uint64_t)N, BK, BN / 2)
               : make_tmap_2d_u8(&tb, b, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
     if (rc != FP8_OK) return rc;
-    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
     static int max_clusters = -1;
     if (max_clusters < 0) {
         cudaLaunchConfig_t cfg = {};
@@ -236,7 +294,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, gemm_fp8_pair_kernel, &cfg) != cudaSuccess || n <= 0) {
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_fp8_pair_kernel<false>, &cfg) != cudaSuccess || n <= 0) {
             (void)cudaGetLastError();
             n = sm_count() / 2;
         }
@@ -250,7 +308,38 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     p.idesc = idesc;
     p.num_pairs = tiles < max_clusters ? tiles : max_clusters;
     p.status = status;
-    gemm_fp8_pair_kernel<<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
+    p.group_offsets = nullptr;
+    p.n_groups = 0;
+    gemm_fp8_pair_kernel<false><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+// Grouped form: Y[rows of group g] = sa_inv * sb_inv[g] * A[rows of group g] . B_g^T for every group, one launch.
+int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv,
+                             const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int K,
+                             uint32_t idesc, int *status, cudaStream_t st)
+{
+    using namespace g2;
+    CUtensorMap ta, tb;
+    int rc = make_tmap_2d_u8(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM, BK);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_2d_u8(&tb, b, (uint64_t)n_groups * N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
+    if (rc != FP8_OK) return rc;
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
+    // the host does not know the group sizes: at most ceil(M/256) + n_groups row tiles exist
+    const long tiles_bound = ((long)(M + 2 * BM - 1) / (2 * BM) + n_groups) * ((N + BN - 1) / BN);
+    const int pairs_max = sm_count() / 2;
+    Params p;
+    p.o = o; p.sa_inv = sa_inv; p.sb_inv = sb_inv;
+    p.M = M; p.N = N; p.K = K;
+    p.a_mn = 0; p.b_mn = 0;
+    p.idesc = idesc;
+    p.num_pairs = (int)(tiles_bound < pairs_max ? tiles_bound : pairs_max);
+    p.status = status;
+    p.group_offsets = group_offsets;
+    p.n_groups = n_groups;
+    gemm_fp8_pair_kernel<true><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }

@@ -233,6 +233,10 @@ gemm_fp8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
 int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, const GemmOut &o,
                      int M, int N, int K, int a_mn, int b_mn, uint32_t idesc, int *status, cudaStream_t st);
 
+int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv,
+                             const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int K,
+                             uint32_t idesc, int *status, cudaStream_t st);
+
 // FP8DPA_GEMM=1cta|2cta forces one kernel family (for A/B measurements); default: chosen per shape.
 static int gemm_family_override()
 {
@@ -423,4 +427,31 @@ extern "C" int fp8_linear_wgrad_rm(const uint8_t *dY8, const uint8_t *X8, const 
     const GemmOut o{dW, out_is_fp32, accumulate, nullptr, 0, nullptr};
     return gemm_fp8("fp8_linear_wgrad_rm", dY8, FP8_E5M2, X8, FP8_E4M3, sdY_inv, sX_inv, o, N, K, T,
                     static_cast<cudaStream_t>(stream), 1, 1);
+}
+
+// Grouped forward product for a mixture-of-experts FFN (Appendix D: 8 experts, 2 active): the token rows of X8 are
+// sorted by expert, expert g owns rows [group_offsets[g], group_offsets[g+1]) and the weight matrix W8[g] ([N,K]) with
+// its own scale.
+extern "C" int fp8_grouped_linear_fwd(const uint8_t *X8, const uint8_t *W8, const float *sX_inv, const float *sW_inv,
+                                      const int *group_offsets, int n_groups, void *Y, int out_is_fp32, int T, int N,
+                                      int K, void *stream)
+{
+    if (!group_offsets) {
+        set_error("fp8_grouped_linear_fwd: NULL group_offsets");
+        return FP8_ERR_NULL;
+    }
+    if (n_groups <= 0 || n_groups > 256) {
+        set_error("fp8_grouped_linear_fwd: n_groups %d must be in [1, 256]", n_groups);
+        return FP8_ERR_SHAPE;
+    }
+    int rc = validate_gemm("fp8_grouped_linear_fwd", X8, W8, sX_inv, sW_inv, Y, T, N, K);
+    if (rc != FP8_OK) return rc;
+    rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    int *status = device_status_ptr();
+    if (!status) return FP8_ERR_CUDA;
+    const GemmOut o{Y, out_is_fp32, 0, nullptr, 0, nullptr};
+    return launch_gemm_2cta_grouped(X8, W8, sX_inv, sW_inv, group_offsets, n_groups, o, T, N, K,
+                                    umma_idesc_f8(FP8_E4M3, FP8_E4M3, 256, 256), status,
+                                    static_cast<cudaStream_t>(stream));
 }

@@ -228,3 +228,52 @@ def test_gradients_with_operands_read_in_place(family, T, N, K, monkeypatch):
     fp8.fp8_linear_wgrad_rm(dy8, x8, sdy, sx, acc, accumulate=True)
     ref, mag = o.linear_wgrad(ody8, ox8, osdy, osx, prev=np.full((N, K), 0.5))
     check(acc, ref, mag + 0.5, TOL_FP32)
+
+
+@pytest.mark.parametrize("sizes,N,K", [([300, 0, 129, 512, 83], 528, 144), ([256, 256], 256, 256),
+                                        ([1000, 17, 2000, 1, 600, 0, 0, 350], 1024, 512), ([16], 16, 16)])
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_grouped_forward_matches_oracle_per_expert(sizes, N, K, out_dtype):
+    """Mixture-of-experts FFN product: token rows sorted by expert, one weight matrix and one weight scale per expert."""
+    E, T = len(sizes), sum(sizes)
+    Tpad = T + 37                                               # rows past the last group stay untouched
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    x = synth.normal_bf16((Tpad, K), 90 + E, 0, 1.0, synth.choose_columns(K, 2, 90, 1), 40.0)
+    x8, _, _, _, sx = gpu_quantize(x, o.E4M3, False)
+    ox8, _, _, osx = o.quantize(x, o.E4M3)
+    w8 = torch.empty((E, N, K), dtype=torch.uint8, device="cuda")
+    sw = torch.empty(E, dtype=torch.float32, device="cuda")
+    ow = []
+    for e in range(E):
+        w = synth.normal_bf16((N, K), 90 + E, 10 + e, synth.W_STD * (1 + e))      # a different range per expert
+        c, _, _, _, si = gpu_quantize(w, o.E4M3, False)
+        w8[e].copy_(c)
+        sw[e:e + 1].copy_(si)
+        ow.append(o.quantize(w, o.E4M3))
+    y = torch.full((Tpad, N), 7.0, dtype=out_dtype, device="cuda")
+    fp8.fp8_grouped_linear_fwd(x8, w8, sx, sw, torch.from_numpy(offs).cuda(), y)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    got = y.float().cpu().numpy().astype(np.float64)
+    tol = 2.0 ** -8 if out_dtype == torch.bfloat16 else TOL_FP32
+    for e in range(E):
+        r0, r1 = int(offs[e]), int(offs[e + 1])
+        if r1 == r0:
+            continue
+        ref, mag = o.linear_fwd(ox8[r0:r1], ow[e][0], osx, ow[e][3])
+        assert rel_err(got[r0:r1], ref, mag) <= tol, e
+    assert np.all(got[T:] == 7.0)
+
+
+def test_grouped_forward_argument_validation():
+    x8 = torch.zeros((32, 32), dtype=torch.uint8, device="cuda")
+    w8 = torch.zeros((2, 16, 32), dtype=torch.uint8, device="cuda")
+    s = scalar(1.0)
+    y = torch.empty((32, 16), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_grouped_linear_fwd(x8, w8, s, torch.ones(2, device="cuda"), None, y)
+    assert e.value.status == -1
+    big = torch.zeros((300, 16, 32), dtype=torch.uint8, device="cuda")
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_grouped_linear_fwd(x8, big, s, torch.ones(300, device="cuda"), torch.zeros(301, dtype=torch.int32, device="cuda"), y)
+    assert e.value.status == -3
