@@ -15,6 +15,7 @@
 #include <float.h>
 
 #include "common.cuh"
+#include "gemm_epilogue.cuh"
 
 namespace fp8dpa {
 namespace bw {
@@ -127,18 +128,6 @@ constexpr int TOTAL = BAR_OFFSET + (2 * STAGES + 4) * 8 + 16;
 constexpr int DYN_BYTES = TOTAL + 1024;
 constexpr int THREADS = 320;
 constexpr uint32_t TMEM_COLS = 256;
-
-// Tile order: bands of BAND tiles along the longer output dimension, the index along the shorter one advancing
-// slowest inside a band, so that the CTAs running at one time share a few operand panels that stay in L2.
-constexpr int BAND = 16;
-__device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
-{
-    const int per_band = BAND * n_short;
-    const int band = tile / per_band, within = tile - band * per_band;
-    const int len = min(BAND, n_long - band * BAND);
-    i_short = within / len;
-    i_long = band * BAND + (within - i_short * len);
-}
 
 struct Params {
     uint16_t *out;                 // [M,N] BF16

@@ -49,15 +49,6 @@ struct Params {
 };
 constexpr int MAX_GROUPS = 256;
 
-constexpr int BAND = 16;
-__device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
-{
-    const int per_band = BAND * n_short;
-    const int band = tile / per_band, within = tile - band * per_band;
-    const int len = min(BAND, n_long - band * BAND);
-    i_short = within / len;
-    i_long = band * BAND + (within - i_short * len);
-}
 __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int &tm, int &tn)
 {
     if (tiles_m >= tiles_n) band_coords(tile, tiles_m, tiles_n, tm, tn);

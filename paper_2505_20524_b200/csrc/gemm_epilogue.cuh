@@ -1,10 +1,24 @@
-// Epilogue of the FP8 GEMM kernels: 32 accumulator columns of one output row (binary32, straight from TMEM) ->
+// Pieces shared by the FP8 GEMM kernels: the tile order and the epilogue.
+// Epilogue: 32 accumulator columns of one output row (binary32, straight from TMEM) ->
 // descaled BF16 / FP32 values with 16-byte stores, or, for a producer under delayed scaling (Appendix E: the scale
 // comes from the amax history, so a single pass suffices), FP8 codes of the BF16-rounded result plus its amax.
 #pragma once
 #include "common.cuh"
 
 namespace fp8dpa {
+
+// Tile order shared by the GEMM kernels: bands of GEMM_BAND tiles along the longer output dimension; inside a band the
+// index along the shorter dimension advances slowest.  The CTAs that run at the same time then share one band of
+// one operand (a few MB) and a handful of panels of the other, and both stay in L2 however long the matrix is.
+constexpr int GEMM_BAND = 16;
+__device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
+{
+    const int per_band = GEMM_BAND * n_short;
+    const int band = tile / per_band, within = tile - band * per_band;
+    const int len = min(GEMM_BAND, n_long - band * GEMM_BAND);     // the last band may be short
+    i_short = within / len;
+    i_long = band * GEMM_BAND + (within - i_short * len);
+}
 
 struct GemmOut {
     void *out;                 // BF16 / FP32 / FP8 [M,N] row-major

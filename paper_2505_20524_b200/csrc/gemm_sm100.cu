@@ -49,18 +49,6 @@ struct GemmParams {
     int *status;
 };
 
-// Tile order: bands of G_BAND tiles along the longer output dimension; inside a band the index along the
-// shorter dimension advances slowest.  The CTAs that run at the same time then share one band of one operand
-// (a few MB) and a handful of panels of the other, and both stay in L2 however long the matrix is.
-constexpr int G_BAND = 16;
-__device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
-{
-    const int per_band = G_BAND * n_short;
-    const int band = tile / per_band, within = tile - band * per_band;
-    const int len = min(G_BAND, n_long - band * G_BAND);     // the last band may be short
-    i_short = within / len;
-    i_long = band * G_BAND + (within - i_short * len);
-}
 template <int TILE_M, int BN>
 __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int &tm, int &tn)
 {
