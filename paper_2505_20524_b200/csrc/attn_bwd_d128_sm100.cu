@@ -170,7 +170,9 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // KV head fastest: the CTAs that run at the same time then add their dQ tiles into different rows of a small,
     // L2-resident band of the accumulator instead of contending for the same rows
-    const int g = blockIdx.x, k_tile = blockIdx.y, b = blockIdx.z;
+    // ... and key tiles in ascending order over the whole grid (batch folded into x): with a causal mask the first key
+    // tiles see the most queries, so the longest CTAs of every batch start first
+    const int g = (int)(blockIdx.x % (unsigned)p.Hkv), b = (int)(blockIdx.x / (unsigned)p.Hkv), k_tile = blockIdx.y;
     const int G = p.Hq / p.Hkv;
     const int k0 = k_tile * KT;
     const int n_sub = p.Npad / QT;
@@ -521,7 +523,7 @@ int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8
     p.B = B; p.N = N; p.Npad = Npad; p.Hq = Hq; p.Hkv = Hkv;
     p.status = status;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_d128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::DYN_BYTES));
-    dim3 grid((unsigned)Hkv, (unsigned)((N + KT - 1) / KT), (unsigned)B);
+    dim3 grid((unsigned)(Hkv * B), (unsigned)((N + KT - 1) / KT), 1);
     attn_bwd_d128_kernel<<<grid, THREADS, Smem::DYN_BYTES, st>>>(tq, tk, tv, tdo, tdq, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     const size_t n4 = (size_t)B * N * Hq * D / 4;
