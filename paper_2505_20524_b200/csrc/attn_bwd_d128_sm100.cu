@@ -2,16 +2,18 @@
 //
 // One CTA per (128-key tile, KV head, batch) keeps K_j, V_j in shared memory and dK_j, dV_j in TMEM (256
 // columns).  It walks over 64-query sub-tiles t (and the query heads of the group).  With rows = keys:
-//   S^T  = K  Q_t^T   [128 x 64]     dP^T = V dO_t^T   [128 x 64]          (64 TMEM columns each)
-//   P~^T = 2^(c S^T - lse2_q),  P8^T = E4M3,  dS8^T = E5M2( P~^T o (a dP^T - db_q) )   (256 threads)
-//   dV  += P8^T dO_t      dK += dS8^T Q_t      dQ_t^T = K^T dS8^T  [128(d) x 64]  (64 TMEM columns)
-// The other 256 TMEM columns are four 64-column slots: S ping-pong (2), dP (1), dQ^T (1), so the scores of
-// sub-tile t+1 are in TMEM before the threads finish sub-tile t, and dP_{t+1}, dQ_t, dV_t, dK_t run on the
-// tensor pipe while the threads work on t+1.  dQ^T tiles leave through shared memory and one bulk
-// reduce-add (binary32 add in L2) per sub-tile into the FP32 accumulator.
+//   S^T  = K  Q_t^T   [128 x 64]     dP^T = V dO_t^T   [128 x 64]          (64 TMEM columns, one slot per group)
+//   P~^T = 2^(c S^T - lse2_q),  P8^T = E4M3,  dS8^T = E5M2( P~^T o (a dP^T - db_q) )
+//   dV  += P8^T dO_t      dK += dS8^T Q_t      dQ_t^T = K^T dS8^T  [128(d) x 64]  (64 TMEM columns, two slots)
+// Two element-wise warpgroups take the sub-tiles in turn (even t / odd t), one thread per key row and all 64
+// query columns, so the exponentials of one sub-tile overlap the dS arithmetic and the barrier round trips of
+// the other.  Each group owns one 64-column TMEM slot that holds S^T_t and then dP^T_t (issued as soon as the
+// group has S^T_t in registers), one P8/dS8 buffer in shared memory and one dQ^T slot.  dQ^T tiles leave through
+// two staging tiles in shared memory and one bulk reduce-add (binary32 add in L2) per sub-tile into the FP32
+// accumulator.
 //
-// Warps: 0 = TMA producer, 1 = MMA issuer, 2-9 = element-wise (two threads per key row, 32 query columns
-// each), 10-13 = dQ drain.  Every wait is bounded.
+// Warpgroups: 0 = control (warp 0 TMA producer, warp 1 MMA issuer), 1-2 = element-wise, 3 = dQ drain; registers
+// are moved from the control and drain groups to the element-wise groups (setmaxnreg).  Every wait is bounded.
 #include <cuda_fp16.h>
 #include <math.h>
 
@@ -24,9 +26,10 @@ namespace bwd128 {
 constexpr int D = 128;
 constexpr int KT = 128;            // keys per CTA
 constexpr int QT = 64;             // queries per sub-tile
-constexpr int STAGES = 6;          // (Q, dO, lse2, db) stages: a TMA load takes several sub-tile periods to land
-constexpr int THREADS = 14 * 32;
-constexpr int EW_WARPS = 8, DRAIN_WARPS = 4;
+constexpr int STAGES = 4;          // (Q, dO, lse2, db) stages: a TMA load takes several sub-tile periods to land
+constexpr int THREADS = 16 * 32;     // four warpgroups: control (TMA, MMA), two element-wise groups, dQ drain
+constexpr int DRAIN_WARPS = 4;
+constexpr int REGS_CTRL = 64, REGS_EW = 176, REGS_DRAIN = 88;   // per thread after setmaxnreg; sum <= 4 * 128
 constexpr int TMEM_COLS = 512;
 
 struct Smem {
@@ -42,18 +45,19 @@ struct Smem {
     static constexpr int PDS_BUF = 2 * PDS_TILE;                 // P8^T then dS8^T
     static constexpr int DQ_OFF = PDS_OFF + 2 * PDS_BUF;
     static constexpr int DQ_BYTES = QT * D * 4;                  // 32 KB: [64 q x 128 d] FP32
-    static constexpr int BAR_OFF = DQ_OFF + DQ_BYTES;
-    // kv_full, qdo_full[3], qdo_empty[3], s_full[2], dp_full, pds_full, pds_free[2], dq_full, dq_empty, all_done
-    static constexpr int N_BARS = 1 + 2 * STAGES + 2 + 1 + 1 + 2 + 1 + 1 + 1;
+    static constexpr int BAR_OFF = DQ_OFF + 2 * DQ_BYTES;          // two staging tiles
+    // kv_full, qdo_full[S], qdo_empty[S], then per group: s_full, dp_full, s_read, dp_read, pds_full, pds_free,
+    // dq_full, dq_empty; all_done
+    static constexpr int N_BARS = 1 + 2 * STAGES + 8 * 2 + 1;
     static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;
 };
 // TMEM columns
-constexpr uint32_t T_S0 = 0, T_S1 = 64, T_DP = 128, T_DQ = 192, T_DV = 256, T_DK = 384;
+constexpr uint32_t T_SD0 = 0, T_SD1 = 64, T_DQ0 = 128, T_DQ1 = 192, T_DV = 256, T_DK = 384;
 
 struct Params {
-    const float *lse2;     // [B,Hq,Npad]  LSE*log2(e) - log2(c_P); +inf in the padding
-    const float *db;       // [B,Hq,Npad]  D * ds_scale / c_P; 0 in the padding
+    const float *lse2;     // [B,Hq,Npad]  -(LSE*log2(e) - log2(c_P)); -inf in the padding
+    const float *db;       // [B,Hq,Npad]  -D * ds_scale / c_P; 0 in the padding
     uint16_t *dK, *dV;     // [B,N,Hkv,D] BF16
     const float *q_inv, *k_inv, *v_inv, *do_inv, *ds_scale;
     float *ds_amax;
@@ -70,7 +74,7 @@ __device__ __forceinline__ float e5m2_to_f32(uint32_t code)
 
 // ---------------------------------------------------------------- prep
 // Eight lanes per (b, i, h) with i < Npad (16-byte loads): D_i = do_inv * sum_d dec(dO8) * O, then
-// lse2 = LSE*log2e - log2(c_P), db = D * ds_scale / c_P; rows i >= N get (+inf, 0); the dQ accumulator row
+// lse2 = -(LSE*log2e - log2(c_P)), db = -D * ds_scale / c_P; rows i >= N get (-inf, 0); the dQ accumulator row
 // is zeroed.
 __global__ void __launch_bounds__(256) attn_bwd_d128_prep_kernel(const uint8_t *__restrict__ dO8, const uint16_t *__restrict__ O,
                                                    const float *__restrict__ LSE, const float *__restrict__ do_inv,
@@ -117,8 +121,8 @@ __global__ void __launch_bounds__(256) attn_bwd_d128_prep_kernel(const uint8_t *
             z[0] = zero; z[1] = zero; z[2] = zero; z[3] = zero;
         }
         if (j == 0) {
-            lse2[vi] = real ? __ldg(LSE + ((size_t)b * Hq + h) * N + i) * 1.4426950408889634f - log2_p_scale : INFINITY;
-            db[vi] = real ? acc * scale : 0.0f;
+            lse2[vi] = real ? log2_p_scale - __ldg(LSE + ((size_t)b * Hq + h) * N + i) * 1.4426950408889634f : -INFINITY;
+            db[vi] = real ? -acc * scale : 0.0f;
         }
     }
 }
@@ -145,6 +149,15 @@ __global__ void __launch_bounds__(256) attn_bwd_d128_finish_kernel(const float4 
     }
 }
 
+template <int N> __device__ __forceinline__ void reg_dec()
+{
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N> __device__ __forceinline__ void reg_inc()
+{
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 // ---------------------------------------------------------------- main
 __global__ void __launch_bounds__(THREADS, 1)
 attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -159,15 +172,22 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t kv_full = bar0;
     auto qdo_full = [&](int s) { return bar0 + 8u * (1 + s); };
     auto qdo_empty = [&](int s) { return bar0 + 8u * (1 + STAGES + s); };
-    auto s_full = [&](int s) { return bar0 + 8u * (1 + 2 * STAGES + s); };
-    const uint32_t dp_full = bar0 + 8u * (3 + 2 * STAGES);
-    const uint32_t pds_full = dp_full + 8u;
-    auto pds_free = [&](int s) { return dp_full + 16u + 8u * s; };
-    const uint32_t dq_full = dp_full + 32u, dq_empty = dp_full + 40u, all_done = dp_full + 48u;
+    const uint32_t bar1 = bar0 + 8u * (1 + 2 * STAGES);
+    // per element-wise group (= parity of the sub-tile index)
+    auto s_full = [&](int g) { return bar1 + 8u * g; };
+    auto dp_full = [&](int g) { return bar1 + 8u * (2 + g); };
+    auto s_read = [&](int g) { return bar1 + 8u * (4 + g); };
+    auto dp_read = [&](int g) { return bar1 + 8u * (6 + g); };
+    auto pds_full = [&](int g) { return bar1 + 8u * (8 + g); };
+    auto pds_free = [&](int g) { return bar1 + 8u * (10 + g); };
+    auto dq_full = [&](int g) { return bar1 + 8u * (12 + g); };
+    auto dq_empty = [&](int g) { return bar1 + 8u * (14 + g); };
+    const uint32_t all_done = bar1 + 8u * 16;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFF + L::N_BARS * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int wg = warp >> 2;
     // KV head fastest: the CTAs that run at the same time then add their dQ tiles into different rows of a small,
     // L2-resident band of the accumulator instead of contending for the same rows
     // ... and key tiles in ascending order over the whole grid (batch folded into x): with a causal mask the first key
@@ -188,14 +208,16 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             mbar_init(qdo_full(s), 1);
             mbar_init(qdo_empty(s), 1);
         }
-        mbar_init(s_full(0), 1);
-        mbar_init(s_full(1), 1);
-        mbar_init(dp_full, 1);
-        mbar_init(pds_full, EW_WARPS);
-        mbar_init(pds_free(0), 1);
-        mbar_init(pds_free(1), 1);
-        mbar_init(dq_full, 1);
-        mbar_init(dq_empty, DRAIN_WARPS);
+        for (int e = 0; e < 2; ++e) {
+            mbar_init(s_full(e), 1);
+            mbar_init(dp_full(e), 1);
+            mbar_init(s_read(e), 4);
+            mbar_init(dp_read(e), 4);
+            mbar_init(pds_full(e), 4);
+            mbar_init(pds_free(e), 1);
+            mbar_init(dq_full(e), 1);
+            mbar_init(dq_empty(e), DRAIN_WARPS);
+        }
         mbar_init(all_done, 1);
         *abort_flag = 0;
         mbar_init_fence();
@@ -215,188 +237,226 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const uint32_t tmem_base = *tmem_slot;
     const WaitCtx ctx{p.status, abort_flag};
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (elect_one()) {
-            mbar_expect_tx(kv_full, 2 * KT * D);
-            tma_load_3d(sbase + L::K_OFF, &tm_k, kv_full, g * D, k0, b);
-            tma_load_3d(sbase + L::V_OFF, &tm_v, kv_full, g * D, k0, b);
-            for (int t = 0; t < n_iter; ++t) {
-                const int st = t % STAGES;
-                const uint32_t ph = (uint32_t)(t / STAGES) & 1u;
-                const int h = head_of(t), q0 = q0_of(t);
-                if (!mbar_wait(qdo_empty(st), ph ^ 1u, ctx)) break;
-                const uint32_t sq = sbase + L::QDO_OFF + st * L::STAGE_BYTES, sdo = sq + L::Q_BYTES;
-                const uint32_t sl = sdo + L::Q_BYTES, sd = sl + 1024;
-                const size_t vi = ((size_t)b * p.Hq + h) * p.Npad + q0;
-                mbar_expect_tx(qdo_full(st), L::STAGE_TX);
-                tma_load_3d(sq, &tm_q, qdo_full(st), h * D, q0, b);
-                tma_load_3d(sdo, &tm_do, qdo_full(st), h * D, q0, b);
-                bulk_load_1d(sl, p.lse2 + vi, L::VEC_BYTES, qdo_full(st));
-                bulk_load_1d(sd, p.db + vi, L::VEC_BYTES, qdo_full(st));
+    if (wg == 0) {
+        reg_dec<REGS_CTRL>();
+        if (warp == 0) {
+            // -------------------------------------------------------- TMA producer
+            if (elect_one()) {
+                mbar_expect_tx(kv_full, 2 * KT * D);
+                tma_load_3d(sbase + L::K_OFF, &tm_k, kv_full, g * D, k0, b);
+                tma_load_3d(sbase + L::V_OFF, &tm_v, kv_full, g * D, k0, b);
+                for (int t = 0; t < n_iter; ++t) {
+                    const int st = t % STAGES;
+                    const uint32_t ph = (uint32_t)(t / STAGES) & 1u;
+                    const int h = head_of(t), q0 = q0_of(t);
+                    if (!mbar_wait(qdo_empty(st), ph ^ 1u, ctx)) break;
+                    const uint32_t sq = sbase + L::QDO_OFF + st * L::STAGE_BYTES, sdo = sq + L::Q_BYTES;
+                    const uint32_t sl = sdo + L::Q_BYTES, sd = sl + 1024;
+                    const size_t vi = ((size_t)b * p.Hq + h) * p.Npad + q0;
+                    mbar_expect_tx(qdo_full(st), L::STAGE_TX);
+                    tma_load_3d(sq, &tm_q, qdo_full(st), h * D, q0, b);
+                    tma_load_3d(sdo, &tm_do, qdo_full(st), h * D, q0, b);
+                    bulk_load_1d(sl, p.lse2 + vi, L::VEC_BYTES, qdo_full(st));
+                    bulk_load_1d(sd, p.db + vi, L::VEC_BYTES, qdo_full(st));
+                }
             }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (elect_one()) {
-            constexpr uint32_t E4 = 0, E5 = 1;
-            constexpr uint32_t id_s = umma_idesc_f8(E4, E4, 128, QT, 0, 0);      // K (K-major) x Q (K-major)
-            constexpr uint32_t id_dp = umma_idesc_f8(E4, E5, 128, QT, 0, 0);     // V x dO
-            constexpr uint32_t id_dv = umma_idesc_f8(E4, E5, 128, D, 0, 1);      // P8^T (K-major) x dO (MN)
-            constexpr uint32_t id_dk = umma_idesc_f8(E5, E4, 128, D, 0, 1);      // dS8^T (K-major) x Q (MN)
-            constexpr uint32_t id_dq = umma_idesc_f8(E4, E5, 128, QT, 1, 1);     // K^T (MN) x dS8^T (MN)
-            const uint64_t d_k = umma_desc(sbase + L::K_OFF, 128, 16);
-            const uint64_t d_v = umma_desc(sbase + L::V_OFF, 128, 16);
-            constexpr uint32_t ROWS32_128 = (32 * 128) >> 4;   // 32 rows of a 128-byte-row tile
-            constexpr uint32_t ROWS32_64 = (32 * 64) >> 4;     // 32 rows of a 64-byte-row tile
-            auto stage_q = [&](int t) { return sbase + L::QDO_OFF + (t % STAGES) * L::STAGE_BYTES; };
-            auto wait_stage = [&](int t) {
-                return mbar_wait(qdo_full(t % STAGES), (uint32_t)(t / STAGES) & 1u, ctx);
-            };
-            auto issue_s = [&](int t) {     // S^T_t = K Q_t^T into slot t & 1
-                const uint64_t d_q = umma_desc(stage_q(t), 128, 16);
-                const uint32_t dst = tmem_base + ((t & 1) ? T_S1 : T_S0);
+        } else if (warp == 1) {
+            // -------------------------------------------------------- MMA issuer
+            if (elect_one()) {
+                constexpr uint32_t E4 = 0, E5 = 1;
+                constexpr uint32_t id_s = umma_idesc_f8(E4, E4, 128, QT, 0, 0);      // K (K-major) x Q (K-major)
+                constexpr uint32_t id_dp = umma_idesc_f8(E4, E5, 128, QT, 0, 0);     // V x dO
+                constexpr uint32_t id_dv = umma_idesc_f8(E4, E5, 128, D, 0, 1);      // P8^T (K-major) x dO (MN)
+                constexpr uint32_t id_dk = umma_idesc_f8(E5, E4, 128, D, 0, 1);      // dS8^T (K-major) x Q (MN)
+                constexpr uint32_t id_dq = umma_idesc_f8(E4, E5, 128, QT, 1, 1);     // K^T (MN) x dS8^T (MN)
+                const uint64_t d_k = umma_desc(sbase + L::K_OFF, 128, 16);
+                const uint64_t d_v = umma_desc(sbase + L::V_OFF, 128, 16);
+                constexpr uint32_t ROWS32_128 = (32 * 128) >> 4;   // 32 rows of a 128-byte-row tile
+                constexpr uint32_t ROWS32_64 = (32 * 64) >> 4;     // 32 rows of a 64-byte-row tile
+                auto stage_q = [&](int t) { return sbase + L::QDO_OFF + (t % STAGES) * L::STAGE_BYTES; };
+                auto wait_stage = [&](int t) {
+                    return mbar_wait(qdo_full(t % STAGES), (uint32_t)(t / STAGES) & 1u, ctx);
+                };
+                auto issue_s = [&](int t) {     // S^T_t = K Q_t^T into the slot of group t & 1
+                    const uint64_t d_q = umma_desc(stage_q(t), 128, 16);
+                    const uint32_t dst = tmem_base + ((t & 1) ? T_SD1 : T_SD0);
 #pragma unroll
-                for (int k = 0; k < D / 32; ++k) umma_f8_ss(dst, d_k + 2u * k, d_q + 2u * k, id_s, k != 0);
-                umma_commit(s_full(t & 1));
-            };
-            auto issue_dp = [&](int t) {    // dP^T_t = V dO_t^T
-                const uint64_t d_do = umma_desc(stage_q(t) + L::Q_BYTES, 128, 16);
+                    for (int k = 0; k < D / 32; ++k) umma_f8_ss(dst, d_k + 2u * k, d_q + 2u * k, id_s, k != 0);
+                    umma_commit(s_full(t & 1));
+                };
+                auto issue_dp = [&](int t) {    // dP^T_t = V dO_t^T into the same slot, once S^T_t is in registers
+                    const uint64_t d_do = umma_desc(stage_q(t) + L::Q_BYTES, 128, 16);
+                    const uint32_t dst = tmem_base + ((t & 1) ? T_SD1 : T_SD0);
 #pragma unroll
-                for (int k = 0; k < D / 32; ++k) umma_f8_ss(tmem_base + T_DP, d_v + 2u * k, d_do + 2u * k, id_dp, k != 0);
-                umma_commit(dp_full);
-            };
-            bool ok = mbar_wait(kv_full, 0, ctx);
-            if (ok) ok = wait_stage(0);
-            if (ok) {
-                tc_fence_after();
-                issue_s(0);
-                issue_dp(0);
-            }
-            if (ok && n_iter > 1) {
-                ok = wait_stage(1);
+                    for (int k = 0; k < D / 32; ++k) umma_f8_ss(dst, d_v + 2u * k, d_do + 2u * k, id_dp, k != 0);
+                    umma_commit(dp_full(t & 1));
+                };
+                // dQ^T_t, dV, dK of sub-tile t, once P8^T_t and dS8^T_t are in shared memory
+                auto finish = [&](int t) {
+                    const int e = t & 1;
+                    const uint32_t u = (uint32_t)(t >> 1);
+                    if (!mbar_wait(pds_full(e), u & 1u, ctx)) return false;
+                    if (u > 0 && !mbar_wait(dq_empty(e), (u - 1) & 1u, ctx)) return false;
+                    tc_fence_after();
+                    const uint32_t sp = sbase + L::PDS_OFF + e * L::PDS_BUF, sds = sp + L::PDS_TILE;
+                    const uint64_t d_p = umma_desc(sp, 64, 16), d_ds = umma_desc(sds, 64, 16);
+                    const uint64_t d_q = umma_desc(stage_q(t), 128, 16), d_do = umma_desc(stage_q(t) + L::Q_BYTES, 128, 16);
+                    // dQ^T_t = K^T dS8^T_t: reduction over the 128 keys, 32 rows of either tile per step
+#pragma unroll
+                    for (int k = 0; k < KT / 32; ++k)
+                        umma_f8_ss(tmem_base + (e ? T_DQ1 : T_DQ0), d_k + ROWS32_128 * k, d_ds + ROWS32_64 * k, id_dq, k != 0);
+                    umma_commit(dq_full(e));
+                    // dV += P8^T dO_t, dK += dS8^T Q_t: reduction over the 64 queries, 32 per step
+#pragma unroll
+                    for (int k = 0; k < QT / 32; ++k)
+                        umma_f8_ss(tmem_base + T_DV, d_p + 2u * k, d_do + ROWS32_128 * k, id_dv, (t | k) != 0);
+#pragma unroll
+                    for (int k = 0; k < QT / 32; ++k)
+                        umma_f8_ss(tmem_base + T_DK, d_ds + 2u * k, d_q + ROWS32_128 * k, id_dk, (t | k) != 0);
+                    umma_commit(qdo_empty(t % STAGES));
+                    umma_commit(pds_free(e));
+                    return true;
+                };
+                bool ok = mbar_wait(kv_full, 0, ctx);
+                if (ok) ok = wait_stage(0);
                 if (ok) {
                     tc_fence_after();
-                    issue_s(1);
+                    issue_s(0);
                 }
-            }
-            for (int t = 0; t < n_iter && ok; ++t) {
-                const int pb = t & 1;
-                // P8^T_t and dS8^T_t are in shared memory; S_t and dP_t have been read
-                if (!mbar_wait(pds_full, (uint32_t)t & 1u, ctx)) { ok = false; break; }
-                tc_fence_after();
-                if (t + 1 < n_iter) issue_dp(t + 1);      // its stage was waited for when S_{t+1} was issued
-                const uint32_t sp = sbase + L::PDS_OFF + pb * L::PDS_BUF, sds = sp + L::PDS_TILE;
-                const uint64_t d_p = umma_desc(sp, 64, 16), d_ds = umma_desc(sds, 64, 16);
-                const uint64_t d_q = umma_desc(stage_q(t), 128, 16), d_do = umma_desc(stage_q(t) + L::Q_BYTES, 128, 16);
-                // dQ^T_t = K^T dS8^T_t: reduction over the 128 keys, 32 rows of either tile per step
-                if (t > 0 && !mbar_wait(dq_empty, (uint32_t)(t - 1) & 1u, ctx)) { ok = false; break; }
-                tc_fence_after();
-#pragma unroll
-                for (int k = 0; k < KT / 32; ++k)
-                    umma_f8_ss(tmem_base + T_DQ, d_k + ROWS32_128 * k, d_ds + ROWS32_64 * k, id_dq, k != 0);
-                umma_commit(dq_full);
-                if (t + 2 < n_iter) {
-                    if (!wait_stage(t + 2)) { ok = false; break; }
+                if (ok && n_iter > 1) {
+                    ok = wait_stage(1);
+                    if (ok) {
+                        tc_fence_after();
+                        issue_s(1);
+                    }
+                }
+                for (int t = 0; t < n_iter && ok; ++t) {
+                    if (t >= 1 && t + 1 < n_iter) {
+                        // the slot of sub-tile t+1 held dP_{t-1}: wait until the threads have read it
+                        if (!mbar_wait(dp_read((t + 1) & 1), (uint32_t)((t - 1) >> 1) & 1u, ctx)) { ok = false; break; }
+                        if (!wait_stage(t + 1)) { ok = false; break; }
+                        tc_fence_after();
+                        issue_s(t + 1);
+                    }
+                    if (!mbar_wait(s_read(t & 1), (uint32_t)(t >> 1) & 1u, ctx)) { ok = false; break; }
                     tc_fence_after();
-                    issue_s(t + 2);                        // slot t & 1: S_t has been read
+                    issue_dp(t);
+                    if (t >= 1 && !finish(t - 1)) { ok = false; break; }
                 }
-                // dV += P8^T dO_t, dK += dS8^T Q_t: reduction over the 64 queries, 32 per step
-#pragma unroll
-                for (int k = 0; k < QT / 32; ++k)
-                    umma_f8_ss(tmem_base + T_DV, d_p + 2u * k, d_do + ROWS32_128 * k, id_dv, (t | k) != 0);
-#pragma unroll
-                for (int k = 0; k < QT / 32; ++k)
-                    umma_f8_ss(tmem_base + T_DK, d_ds + 2u * k, d_q + ROWS32_128 * k, id_dk, (t | k) != 0);
-                umma_commit(qdo_empty(t % STAGES));
-                umma_commit(pds_free(pb));
+                if (ok) ok = finish(n_iter - 1);
+                if (ok) umma_commit(all_done);
             }
-            if (ok) umma_commit(all_done);
         }
-    } else if (warp < 2 + EW_WARPS) {
+    } else if (wg <= 2) {
+        reg_inc<REGS_EW>();
         // ------------------------------------------------------------ element-wise: P8^T, dS8^T
-        const int ew = warp - 2;
+        // Group e takes the sub-tiles t = e, e+2, ...; each thread one key row and all 64 query columns.  The two
+        // groups run half a period apart, so one group's exponentials overlap the other's dS arithmetic.
+        const int e = wg - 1;
         const int quad = warp & 3;                      // TMEM lanes 32*quad..: rows (keys) of this warp
-        const int half = ew >> 2;                       // query columns [32*half, 32*half + 32)
         const int r = quad * 32 + lane;                 // key row inside the tile
         const int key = k0 + r;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const uint32_t t_sd = tmem_base + (e ? T_SD1 : T_SD0) + lane_addr;
         const float c = p.softmax_scale * __ldg(p.q_inv) * __ldg(p.k_inv) * 1.4426950408889634f;
         const float dss = __ldg(p.ds_scale);
         const float a_dp = __ldg(p.do_inv) * __ldg(p.v_inv) * dss / p.p_scale;
         const uint64_t c2 = pack_f32x2(c, c), a2 = pack_f32x2(a_dp, a_dp);
         const int sw = (r >> 1) & 3;                    // 64-byte swizzle: 16-byte chunk index ^ ((row >> 1) & 3)
-        const int ch0 = half * 2;
+        uint8_t *prow = smem + L::PDS_OFF + e * L::PDS_BUF + r * 64;
+        uint8_t *dsrow = prow + L::PDS_TILE;
         float amax = 0.0f;
         bool ok = true;
-        for (int t = 0; t < n_iter; ++t) {
-            const int q0 = q0_of(t), st = t % STAGES, pb = t & 1;
-            const int qbase = q0 + half * 32;           // first query column of this thread
-            // valid iff key <= query (causal) and key < N; queries >= N carry lse2 = +inf
+        for (int t = e; t < n_iter; t += 2) {
+            const uint32_t u = (uint32_t)(t >> 1);
+            const int q0 = q0_of(t), st = t % STAGES;
+            // valid iff key <= query (causal) and key < N; queries >= N carry -lse2 = -inf
             const bool need_mask = (p.causal && q0 < k0 + KT - 1) || (k0 + KT > p.N);
-            const int first_ok = (key < p.N) ? (p.causal ? key - qbase : 0) : 64;   // columns >= first_ok are valid
-            const float *vec = reinterpret_cast<const float *>(smem + L::QDO_OFF + st * L::STAGE_BYTES + 2 * L::Q_BYTES);
-            const float *lse2 = vec + half * 32, *dbv = vec + 256 + half * 32;
+            const int first_ok = (key < p.N) ? (p.causal ? key - q0 : 0) : 64;   // columns >= first_ok are valid
+            const float *nlse2 = reinterpret_cast<const float *>(smem + L::QDO_OFF + st * L::STAGE_BYTES + 2 * L::Q_BYTES);
+            const float *ndb = nlse2 + 256;
             if (!mbar_wait_warp(qdo_full(st), (uint32_t)(t / STAGES) & 1u, ctx)) { ok = false; break; }
-            if (!mbar_wait_warp(s_full(pb), (uint32_t)(t >> 1) & 1u, ctx)) { ok = false; break; }
+            if (!mbar_wait_warp(s_full(e), u & 1u, ctx)) { ok = false; break; }
             tc_fence_after();
-            uint32_t sv[32];
-            tmem_ld_32x32b_x32(tmem_base + (pb ? T_S1 : T_S0) + lane_addr + (uint32_t)(half * 32), sv);
-            tmem_ld_wait();
-            float pe[32];
+            float pe[64];
+            {
+                uint32_t sa[32], sb[32];
+                tmem_ld_32x32b_x32(t_sd, sa);
+                tmem_ld_32x32b_x32(t_sd + 32u, sb);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(s_read(e));   // the slot may take dP^T_t
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-                const float2 l2 = *reinterpret_cast<const float2 *>(lse2 + i);
-                float x0, x1;
-                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), c2,
-                                       pack_f32x2(-l2.x, -l2.y)), x0, x1);
-                pe[i] = ex2_approx(x0);                 // c_P * P
-                pe[i + 1] = ex2_approx(x1);
+                for (int i = 0; i < 64; i += 2) {
+                    const float2 l2 = *reinterpret_cast<const float2 *>(nlse2 + i);     // -lse2 of two queries
+                    const uint32_t *sx = i < 32 ? sa + i : sb + (i - 32);
+                    float x0, x1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sx[0]), __uint_as_float(sx[1])), c2,
+                                           pack_f32x2(l2.x, l2.y)), x0, x1);
+                    pe[i] = ex2_approx(x0);             // c_P * P
+                    pe[i + 1] = ex2_approx(x1);
+                }
             }
             if (need_mask) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
+                for (int i = 0; i < 64; ++i)
                     if (i < first_ok) pe[i] = 0.0f;
             }
-            uint32_t w[8];
+            // the P8/dS8 buffer of this group was last read by the MMAs of sub-tile t-2
+            if (u > 0 && !mbar_wait_warp(pds_free(e), (u - 1) & 1u, ctx)) { ok = false; break; }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) w[i] = cvt_f32x4_to_fp8x4<0>(pe[4 * i], pe[4 * i + 1], pe[4 * i + 2], pe[4 * i + 3]);
-            // the P8/dS8 buffer pb was last read by the MMAs of sub-tile t-2
-            if (t >= 2 && !mbar_wait_warp(pds_free(pb), (uint32_t)((t >> 1) - 1) & 1u, ctx)) { ok = false; break; }
-            uint8_t *prow = smem + L::PDS_OFF + pb * L::PDS_BUF + r * 64;
-            uint8_t *dsrow = prow + L::PDS_TILE;
-            *reinterpret_cast<uint4 *>(prow + ((ch0 ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-            *reinterpret_cast<uint4 *>(prow + (((ch0 + 1) ^ sw) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-            if (!mbar_wait_warp(dp_full, (uint32_t)t & 1u, ctx)) { ok = false; break; }
-            tc_fence_after();
-            tmem_ld_32x32b_x32(tmem_base + T_DP + lane_addr + (uint32_t)(half * 32), sv);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-                const float2 d2 = *reinterpret_cast<const float2 *>(dbv + i);
-                float y0, y1;
-                unpack_f32x2(mul_f32x2(pack_f32x2(pe[i], pe[i + 1]),
-                                       fma_f32x2(pack_f32x2(__uint_as_float(sv[i]), __uint_as_float(sv[i + 1])), a2,
-                                                 pack_f32x2(-d2.x, -d2.y))), y0, y1);
-                pe[i] = y0;                              // ds_scale * dS
-                pe[i + 1] = y1;
-                amax = fmaxf(fmaxf(amax, fabsf(y0)), fabsf(y1));
+            for (int ch = 0; ch < 4; ++ch) {
+                uint4 w;
+                w.x = cvt_f32x4_to_fp8x4<0>(pe[16 * ch], pe[16 * ch + 1], pe[16 * ch + 2], pe[16 * ch + 3]);
+                w.y = cvt_f32x4_to_fp8x4<0>(pe[16 * ch + 4], pe[16 * ch + 5], pe[16 * ch + 6], pe[16 * ch + 7]);
+                w.z = cvt_f32x4_to_fp8x4<0>(pe[16 * ch + 8], pe[16 * ch + 9], pe[16 * ch + 10], pe[16 * ch + 11]);
+                w.w = cvt_f32x4_to_fp8x4<0>(pe[16 * ch + 12], pe[16 * ch + 13], pe[16 * ch + 14], pe[16 * ch + 15]);
+                *reinterpret_cast<uint4 *>(prow + ((ch ^ sw) << 4)) = w;
             }
+            if (!mbar_wait_warp(dp_full(e), u & 1u, ctx)) { ok = false; break; }
+            tc_fence_after();
 #pragma unroll
-            for (int i = 0; i < 8; ++i) w[i] = cvt_f32x4_to_fp8x4<1>(pe[4 * i], pe[4 * i + 1], pe[4 * i + 2], pe[4 * i + 3]);
-            *reinterpret_cast<uint4 *>(dsrow + ((ch0 ^ sw) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-            *reinterpret_cast<uint4 *>(dsrow + (((ch0 + 1) ^ sw) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-            tc_fence_before();
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t dv[32];
+                tmem_ld_32x32b_x32(t_sd + (uint32_t)(32 * hf), dv);
+                tmem_ld_wait();
+                if (hf == 1) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(dp_read(e));   // the slot may take S^T_{t+2}
+                }
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float2 d2 = *reinterpret_cast<const float2 *>(ndb + 32 * hf + i);   // -db of two queries
+                    float y0, y1;
+                    unpack_f32x2(mul_f32x2(pack_f32x2(pe[32 * hf + i], pe[32 * hf + i + 1]),
+                                           fma_f32x2(pack_f32x2(__uint_as_float(dv[i]), __uint_as_float(dv[i + 1])), a2,
+                                                     pack_f32x2(d2.x, d2.y))), y0, y1);
+                    pe[32 * hf + i] = y0;                // ds_scale * dS
+                    pe[32 * hf + i + 1] = y1;
+                    amax = fmaxf(amax, fmaxf(fabsf(y0), fabsf(y1)));
+                }
+#pragma unroll
+                for (int ch = 2 * hf; ch < 2 * hf + 2; ++ch) {
+                    uint4 w;
+                    w.x = cvt_f32x4_to_fp8x4<1>(pe[16 * ch], pe[16 * ch + 1], pe[16 * ch + 2], pe[16 * ch + 3]);
+                    w.y = cvt_f32x4_to_fp8x4<1>(pe[16 * ch + 4], pe[16 * ch + 5], pe[16 * ch + 6], pe[16 * ch + 7]);
+                    w.z = cvt_f32x4_to_fp8x4<1>(pe[16 * ch + 8], pe[16 * ch + 9], pe[16 * ch + 10], pe[16 * ch + 11]);
+                    w.w = cvt_f32x4_to_fp8x4<1>(pe[16 * ch + 12], pe[16 * ch + 13], pe[16 * ch + 14], pe[16 * ch + 15]);
+                    *reinterpret_cast<uint4 *>(dsrow + ((ch ^ sw) << 4)) = w;
+                }
+            }
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive(pds_full);
+            if (lane == 0) mbar_arrive(pds_full(e));
         }
-        // ---- epilogue: warps with half == 0 write dV, the others dK (TMEM lane = key)
+        // ---- epilogue: group 0 writes dV, group 1 dK (TMEM lane = key)
         if (ok && mbar_wait_warp(all_done, 0, ctx)) {
             tc_fence_after();
-            const float f = half == 0 ? __ldg(p.do_inv) / p.p_scale : p.softmax_scale * __ldg(p.q_inv) / dss;
-            uint16_t *dst = (half == 0 ? p.dV : p.dK) + (((size_t)b * p.N + key) * p.Hkv + g) * D;
-            const uint32_t tcol = half == 0 ? T_DV : T_DK;
+            const float f = e == 0 ? __ldg(p.do_inv) / p.p_scale : p.softmax_scale * __ldg(p.q_inv) / dss;
+            uint16_t *dst = (e == 0 ? p.dV : p.dK) + (((size_t)b * p.N + key) * p.Hkv + g) * D;
+            const uint32_t tcol = e == 0 ? T_DV : T_DK;
 #pragma unroll 1
             for (int cc = 0; cc < D; cc += 32) {
                 uint32_t v[32];
@@ -422,27 +482,29 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
         }
     } else {
+        reg_dec<REGS_DRAIN>();
         // ------------------------------------------------------------ dQ drain (4 warps)
         const int quad = warp & 3;                      // TMEM lane = d index
         const int dd = quad * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        float *dq_s = reinterpret_cast<float *>(smem + L::DQ_OFF);
-        const bool issuer = (warp == 2 + EW_WARPS) && lane == 0;
+        const bool issuer = (quad == 0) && lane == 0;
         for (int t = 0; t < n_iter; ++t) {
-            const int h = head_of(t), q0 = q0_of(t);
-            const bool got = mbar_wait_warp(dq_full, (uint32_t)t & 1u, ctx);
+            const int h = head_of(t), q0 = q0_of(t), e = t & 1;
+            float *dq_s = reinterpret_cast<float *>(smem + L::DQ_OFF + e * L::DQ_BYTES);
+            const bool got = mbar_wait_warp(dq_full(e), (uint32_t)(t >> 1) & 1u, ctx);
             uint32_t va[32], vb[32];
             if (got) {
                 tc_fence_after();
-                tmem_ld_32x32b_x32(tmem_base + T_DQ + lane_addr, va);
-                tmem_ld_32x32b_x32(tmem_base + T_DQ + lane_addr + 32u, vb);
+                const uint32_t src = tmem_base + (e ? T_DQ1 : T_DQ0) + lane_addr;
+                tmem_ld_32x32b_x32(src, va);
+                tmem_ld_32x32b_x32(src + 32u, vb);
                 tmem_ld_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(dq_empty);   // the dQ^T slot may be overwritten
+                if (lane == 0) mbar_arrive(dq_empty(e));   // the dQ^T slot may be overwritten
             }
-            // the previous bulk reduce must have finished reading the staging tile
-            if (issuer) bulk_wait_group_read0();
+            // the reduce issued two sub-tiles ago must have finished reading this staging tile
+            if (issuer) bulk_wait_group_read1();
             if (named_barrier_or(1, DRAIN_WARPS * 32, !got)) break;   // all four warps leave together
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
@@ -452,7 +514,7 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             fence_proxy_async_smem();
             named_barrier_sync(1, DRAIN_WARPS * 32);
             if (issuer) {
-                tma_reduce_add_3d(&tm_dq, sbase + L::DQ_OFF, h * D, q0, b);
+                tma_reduce_add_3d(&tm_dq, sbase + L::DQ_OFF + e * L::DQ_BYTES, h * D, q0, b);
                 bulk_commit_group();
             }
         }
