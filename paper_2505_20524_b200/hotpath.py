@@ -158,20 +158,23 @@ class BlockHotPath:
         return out
 
     # ------------------------------------------------------------------ host-to-host step
-    def step_host(self, h_in: dict, h_out: dict):
+    def step_host(self, h_in: dict, h_out: dict, wait: bool = True):
         """One step on pinned host buffers: inputs go up, every output comes back.
 
         Three streams: uploads, the kernels (the caller's current stream), downloads.  The copy engines run both
-        directions at once and under the kernels, so the step costs about max(upload, download) instead of their
-        sum.  h_in / h_out map the names of input_tensors() / output_tensors() to pinned host tensors.  On return
-        the current stream has waited for the last download.
+        directions at once and under the kernels, so a step costs about max(upload, download) instead of their
+        sum.  h_in / h_out map the names of input_tensors() / output_tensors() to pinned host tensors.  With
+        ``wait`` the current stream has waited for the last download on return.  Without it consecutive steps
+        overlap as well (the uploads of one step run while the previous step's outputs are still going down; a
+        group's kernels wait only for the previous download of their own outputs): call ``finish_host()`` before
+        reading the host buffers.
         """
         main = torch.cuda.current_stream(self.device)
         if not hasattr(self, "_up"):
             self._up, self._down = torch.cuda.Stream(self.device), torch.cuda.Stream(self.device)
+            self._downloaded = None
         up, down = self._up, self._down
         up.wait_stream(main)          # the previous step's kernels have read the device inputs
-        down.wait_stream(main)
         groups = []                   # (inputs, kernels, outputs) per independent piece of the step
         for lin in self.linears:
             ins = [("x_" + lin.name, lin.x.x), ("w_" + lin.name, lin.w.x), ("dy_" + lin.name, lin.dy.x)]
@@ -190,8 +193,11 @@ class BlockHotPath:
                 e = torch.cuda.Event()
                 e.record(up)
                 ready.append(e)
-        for (ins, run, outs), e in zip(groups, ready):
+        prev, downloaded = self._downloaded, []
+        for g, ((ins, run, outs), e) in enumerate(zip(groups, ready)):
             main.wait_event(e)
+            if prev is not None:
+                main.wait_event(prev[g])          # the previous step's copy of these outputs has left the device
             run()
             done = torch.cuda.Event()
             done.record(main)
@@ -199,7 +205,18 @@ class BlockHotPath:
                 down.wait_event(done)
                 for name, d in outs:
                     h_out[name].copy_(d, non_blocking=True)
-        main.wait_stream(down)
+                gone = torch.cuda.Event()
+                gone.record(down)
+            downloaded.append(gone)
+        self._downloaded = downloaded
+        if wait:
+            self.finish_host()
+
+    def finish_host(self):
+        """The current stream waits for every download issued by step_host()."""
+        if hasattr(self, "_down"):
+            torch.cuda.current_stream(self.device).wait_stream(self._down)
+            self._downloaded = None
 
     def _run_linear(self, lin):
         lin.x.quantize()

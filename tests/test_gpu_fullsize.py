@@ -175,6 +175,16 @@ def test_host_to_host_step_equals_device_step():
     for n, t in ref.items():
         a, b = hout[n], t.cpu()
         assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), n
+    # overlapped form: consecutive steps in flight, one wait at the end
+    for n in hout:
+        hout[n].zero_()
+    for _ in range(4):
+        hp.step_host(hin, hout, wait=False)
+    hp.finish_host()
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    for n, t in ref.items():
+        assert torch.equal(hout[n].view(torch.uint8), t.cpu().view(torch.uint8)), n
 
 
 def test_glue_and_producer_forms_at_c4_sizes():
