@@ -34,50 +34,86 @@ __device__ __forceinline__ float silu_mul(float g, float u)
     return g * r * u;
 }
 
-// 0.5 * erfc(y) for y >= 0 as 0.5 * t * exp(Q(t) - y^2), t = 1 / (1 + y/2): Q is a degree-9 least-squares fit of
-// log(erfcx(y) / t) on Chebyshev nodes of t in [0.2, 1] (y in [0, 8]); evaluated in binary32 the relative error
-// stays below 2e-6 up to y = 4 and 6e-6 up to y = 8, past which the result is below 1e-29.
-__device__ __forceinline__ float half_erfc_pos(float y)
+// The un-gated activations work on pairs of values with the packed binary32 instructions (one instruction, two
+// lanes): they are bound by instruction issue, not by memory, and the packed forms halve the count.
+__device__ __forceinline__ uint64_t splat2(float c) { return pack_f32x2(c, c); }
+__device__ __forceinline__ float rcp_approx(float x)
 {
-    float t;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.5f, y, 1.0f)));
-    float q = 1.227935892e-01f;
-    q = fmaf(q, t, -5.583772951e-01f);
-    q = fmaf(q, t, 8.634607687e-01f);
-    q = fmaf(q, t, -2.980391946e-01f);
-    q = fmaf(q, t, -4.172309384e-01f);
-    q = fmaf(q, t, 1.850209772e-01f);
-    q = fmaf(q, t, -2.980059381e-02f);
-    q = fmaf(q, t, 4.005914557e-01f);
-    q = fmaf(q, t, 9.969420963e-01f);
-    q = fmaf(q, t, -1.265360832e+00f);
-    return 0.5f * t * ex2_approx(1.4426950408889634f * fmaf(-y, y, q));
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
 }
 
-// activations: 0 = SiLU(gate) * up (two inputs), 1 = GeLU (exact form), 2 = xIELU with (a_p, a_n)
+// GeLU (exact form) of two values: x * Phi(x), Phi(x) = erfc(-x / sqrt 2) / 2.
+// With y = |x| / sqrt 2 and e = erfc(y) / 2 (taken from the tail side, so that the left tail keeps its relative
+// accuracy): x * Phi(x) = -|x| e for x < 0 and x - |x| e for x > 0, i.e. (x + |x|) / 2 - |x| e for both.
+// e = t * 2^(L Q(t) - 1 - L y^2), t = 1 / (1 + y/2), L = log2(e): Q is a degree-9 least-squares fit of
+// log(erfcx(y) / t) on Chebyshev nodes of t in [0.2, 1] (y in [0, 8]); evaluated in binary32 the relative error of
+// e stays below 2e-6 up to y = 4 and 6e-6 up to y = 8, past which e is below 1e-29.  The coefficients below are
+// those of L Q (the constant one with the -1 folded in).
+__device__ __forceinline__ uint64_t gelu2(float x0, float x1)
+{
+    constexpr float L = 1.4426950408889634f;
+    const uint64_t x = pack_f32x2(x0, x1);
+    const uint64_t nax = pack_f32x2(__uint_as_float(__float_as_uint(x0) | 0x80000000u),
+                                    __uint_as_float(__float_as_uint(x1) | 0x80000000u));     // -|x|
+    const uint64_t y = mul_f32x2(nax, splat2(-0.70710678118654752440f));
+    float d0, d1;
+    unpack_f32x2(fma_f32x2(y, splat2(0.5f), splat2(1.0f)), d0, d1);
+    const uint64_t t = pack_f32x2(rcp_approx(d0), rcp_approx(d1));
+    uint64_t q = splat2(1.227935892e-01f * L);
+    q = fma_f32x2(q, t, splat2(-5.583772951e-01f * L));
+    q = fma_f32x2(q, t, splat2(8.634607687e-01f * L));
+    q = fma_f32x2(q, t, splat2(-2.980391946e-01f * L));
+    q = fma_f32x2(q, t, splat2(-4.172309384e-01f * L));
+    q = fma_f32x2(q, t, splat2(1.850209772e-01f * L));
+    q = fma_f32x2(q, t, splat2(-2.980059381e-02f * L));
+    q = fma_f32x2(q, t, splat2(4.005914557e-01f * L));
+    q = fma_f32x2(q, t, splat2(9.969420963e-01f * L));
+    q = fma_f32x2(q, t, splat2(-1.265360832e+00f * L - 1.0f));
+    float z0, z1;
+    unpack_f32x2(fma_f32x2(mul_f32x2(y, y), splat2(-L), q), z0, z1);
+    const uint64_t e = mul_f32x2(t, pack_f32x2(ex2_approx(z0), ex2_approx(z1)));             // erfc(y) / 2
+    const uint64_t relu2x = fma_f32x2(nax, splat2(-1.0f), x);                                 // x + |x|, exact
+    return fma_f32x2(relu2x, splat2(0.5f), mul_f32x2(nax, e));
+}
+
+// xIELU of two values with (a_p, a_n): x > 0: a_p x^2 + x/2; x <= 0: a_n (e^x - 1 - x) + x/2, with e^x - 1 - x from
+// its series near 0 (|x| < 1/4, next term below 2e-9 of the first) and from the hardware exp2 elsewhere.
+__device__ __forceinline__ uint64_t xielu2(float x0, float x1, float a_p, float a_n)
+{
+    const uint64_t x = pack_f32x2(x0, x1);
+    const uint64_t hx = mul_f32x2(x, splat2(0.5f));
+    const uint64_t pos = fma_f32x2(mul_f32x2(x, splat2(a_p)), x, hx);
+    uint64_t ser = splat2(1.0f / 5040.0f);
+    ser = fma_f32x2(ser, x, splat2(1.0f / 720.0f));
+    ser = fma_f32x2(ser, x, splat2(1.0f / 120.0f));
+    ser = fma_f32x2(ser, x, splat2(1.0f / 24.0f));
+    ser = fma_f32x2(ser, x, splat2(1.0f / 6.0f));
+    ser = fma_f32x2(ser, x, splat2(0.5f));
+    ser = mul_f32x2(ser, mul_f32x2(x, x));
+    float a0, a1;
+    unpack_f32x2(mul_f32x2(x, splat2(1.4426950408889634f)), a0, a1);
+    const uint64_t big = add_f32x2(pack_f32x2(ex2_approx(a0), ex2_approx(a1)), fma_f32x2(x, splat2(-1.0f), splat2(-1.0f)));
+    float s0, s1, b0, b1, p0, p1, n0, n1;
+    unpack_f32x2(ser, s0, s1);
+    unpack_f32x2(big, b0, b1);
+    const uint64_t neg = fma_f32x2(splat2(a_n), pack_f32x2(x0 > -0.25f ? s0 : b0, x1 > -0.25f ? s1 : b1), hx);
+    unpack_f32x2(pos, p0, p1);
+    unpack_f32x2(neg, n0, n1);
+    return pack_f32x2(x0 > 0.0f ? p0 : n0, x1 > 0.0f ? p1 : n1);
+}
+
+// activations: 0 = SiLU(gate) * up (two inputs), 1 = GeLU (exact form), 2 = xIELU with (a_p, a_n);
+// two values in, one word of two BF16 values out
 constexpr int ACT_SWIGLU = 0;
 template <int ACT>
-__device__ __forceinline__ float act1(float x, float u, float a_p, float a_n)
+__device__ __forceinline__ uint32_t act2(float g0, float g1, float u0, float u1, float a_p, float a_n)
 {
-    if (ACT == ACT_SWIGLU) return silu_mul(x, u);
-    if (ACT == FP8_ACT_GELU) {
-        // x * Phi(x), Phi(x) = erfc(-x / sqrt 2) / 2; from the tail side, so that the left tail keeps its relative accuracy
-        const float e = half_erfc_pos(fabsf(x) * 0.70710678118654752440f);
-        return x * (x < 0.0f ? e : 1.0f - e);
-    }
-    // xIELU, x <= 0: a_n (e^x - 1 - x) + x / 2.  e^x - 1 - x from its series near 0 (|x| < 1/4, next term below 2e-9
-    // of the first), from the hardware exp2 elsewhere.
-    const float pos = fmaf(a_p * x, x, 0.5f * x);
-    float ser = 1.0f / 5040.0f;
-    ser = fmaf(ser, x, 1.0f / 720.0f);
-    ser = fmaf(ser, x, 1.0f / 120.0f);
-    ser = fmaf(ser, x, 1.0f / 24.0f);
-    ser = fmaf(ser, x, 1.0f / 6.0f);
-    ser = fmaf(ser, x, 0.5f);
-    ser = ser * x * x;
-    const float big = ex2_approx(1.4426950408889634f * x) - 1.0f - x;
-    const float neg = fmaf(a_n, x > -0.25f ? ser : big, 0.5f * x);
-    return x > 0.0f ? pos : neg;
+    if (ACT == ACT_SWIGLU) return pack_bf16x2(silu_mul(g0, u0), silu_mul(g1, u1));
+    float r0, r1;
+    unpack_f32x2(ACT == FP8_ACT_GELU ? gelu2(g0, g1) : xielu2(g0, g1, a_p, a_n), r0, r1);
+    return pack_bf16x2(r0, r1);
 }
 
 // 8 inputs (+ 8 up values for the gated form) -> 8 BF16 values of h (packed two per word)
@@ -88,8 +124,7 @@ __device__ __forceinline__ uint4 act8(const uint4 g, const uint4 u, float a_p, f
     uint32_t h[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
-        h[i] = pack_bf16x2(act1<ACT>(bf16_lo(gw[i]), bf16_lo(uw[i]), a_p, a_n),
-                           act1<ACT>(bf16_hi(gw[i]), bf16_hi(uw[i]), a_p, a_n));
+        h[i] = act2<ACT>(bf16_lo(gw[i]), bf16_hi(gw[i]), bf16_lo(uw[i]), bf16_hi(uw[i]), a_p, a_n);
     return make_uint4(h[0], h[1], h[2], h[3]);
 }
 
