@@ -26,7 +26,7 @@ namespace bwd128 {
 constexpr int D = 128;
 constexpr int KT = 128;            // keys per CTA
 constexpr int QT = 64;             // queries per sub-tile
-constexpr int STAGES = 4;          // (Q, dO, lse2, db) stages: a TMA load takes several sub-tile periods to land
+constexpr int STAGES = 5;          // (Q, dO, lse2, db) stages: a TMA load takes several sub-tile periods to land
 constexpr int THREADS = 16 * 32;     // four warpgroups: control (TMA, MMA), two element-wise groups, dQ drain
 constexpr int DRAIN_WARPS = 4;
 constexpr int REGS_CTRL = 64, REGS_EW = 176, REGS_DRAIN = 88;   // per thread after setmaxnreg; sum <= 4 * 128
