@@ -37,7 +37,8 @@ def run_fwd(qd, B, N, Hq, Hkv, d, causal, s):
 
 @pytest.mark.parametrize("name,B,N,causal", [("c1", 1, 256, True), ("c1", 2, 128, True), ("c1", 1, 400, True),
                                              ("c1", 1, 256, False), ("c1", 1, 16, True), ("c1", 1, 208, False),
-                                             ("c3", 1, 384, True), ("c4", 1, 272, True), ("c4", 1, 256, False)])
+                                             ("c3", 1, 384, True), ("c4", 1, 272, True), ("c4", 1, 256, False),
+                                             ("c3", 2, 144, True), ("c4", 2, 112, False)])
 def test_forward_matches_oracle(name, B, N, causal):
     cfg = synth.CONFIGS[name]
     Hq, Hkv, d = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
@@ -96,7 +97,11 @@ def run_bwd(qd, O_bits, lse32, B, N, Hq, Hkv, d, causal, s, ds_scale):
 
 @pytest.mark.parametrize("name,B,N,causal", [("c1", 1, 256, True), ("c1", 2, 128, True), ("c1", 1, 400, True),
                                              ("c1", 1, 256, False), ("c1", 1, 16, True),
-                                             ("c3", 1, 384, True), ("c4", 1, 272, True), ("c4", 1, 256, False)])
+                                             ("c3", 1, 384, True), ("c4", 1, 272, True), ("c4", 1, 256, False),
+                                             # d = 128 corner cases of the two-group kernel: a single sub-tile per CTA,
+                                             # an odd number of sub-tiles, a ragged tail, grouped heads on one tile
+                                             ("c3", 1, 64, True), ("c3", 2, 144, True), ("c3", 1, 192, False),
+                                             ("c4", 1, 64, True), ("c4", 2, 112, False)])
 def test_backward_matches_oracle(name, B, N, causal):
     cfg = synth.CONFIGS[name]
     Hq, Hkv, d = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
