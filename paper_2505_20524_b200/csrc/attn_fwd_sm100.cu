@@ -1,14 +1,17 @@
 // FP8 attention forward (Appendix B, Eq. (P) with QK^T and PV on FP8 tensor cores).
 //
 // One CTA per (128-query tile, query head, batch); two CTAs share an SM so that one CTA's softmax overlaps
-// the other's MMAs.  Per 128-key block j (ascending):
+// the other's MMAs.  Two warpgroups per CTA; registers move from the control group to the softmax group
+// (setmaxnreg 40 / 216, two CTAs fill the register file).  Per 128-key block j (ascending):
 //   warp 0  TMA: K_j and V_j tiles ([128 keys x d bytes], swizzled) into a 2-stage ring; Q once
-//   warp 1  MMA: S = Q K_j^T (d/32 MMAs, 128x128, accumulator in TMEM columns 0..127), then
-//                O += P8 V_j (4 MMAs, 128 x d, TMEM columns 128..128+d) with V read in place as an
-//                MN-major operand (no transposed copy of V)
-//   warps 2-5  softmax, one row per thread: running max m, l += sum P~, P~ = 2^(c*S - m) scaled by c_P and
-//              rounded to E4M3, written to shared memory in the K-major 128-byte-swizzled operand layout;
-//              O in TMEM is rescaled by 2^(m_old - m_new) when a row maximum grows
+//   warp 1  MMA: S = Q K_j^T (d/32 MMAs, 128x128, accumulator in TMEM columns 0..127), issued as soon as the
+//                softmax threads hold S_{j-1} in registers; then O += P8 V_j (4 MMAs, 128 x d, TMEM columns
+//                128..128+d) with V read in place as an MN-major operand (no transposed copy of V)
+//   warps 4-7  softmax, one row per thread: the whole score row (128 values) is read from TMEM once and the S
+//              columns released; running max m, l += sum P~, P~ = 2^(c*S - m) scaled by c_P and rounded to
+//              E4M3, all from registers; then (once the previous PV product is complete) O in TMEM is rescaled
+//              by 2^(m_old - m_new) when a row maximum grew, and P8 is written to shared memory in the K-major
+//              128-byte-swizzled operand layout
 // Final: O = v_inv * acc / (c_P * l) as BF16, LSE = ln2 * (m + log2 l).
 #include <math.h>
 
@@ -19,7 +22,8 @@ namespace fp8dpa {
 constexpr int A_BM = 128;          // query rows per CTA
 constexpr int A_BN = 128;          // keys per block
 constexpr int A_KV_STAGES = 2;
-constexpr int A_THREADS = 192;
+constexpr int A_THREADS = 256;      // warpgroup 0: TMA, MMA (+2 idle warps); warpgroup 1: softmax
+constexpr int A_REGS_CTRL = 40, A_REGS_SOFTMAX = 216;   // after setmaxnreg; 2 CTAs x 128 x (40 + 216) = the register file
 constexpr int A_TMEM_COLS = 256;   // S: [0,128)  O: [128, 128+d)
 
 template <int D>
@@ -32,8 +36,8 @@ struct AttnFwdSmem {
     static constexpr int KV_OFF = Q_OFF + Q_BYTES;
     static constexpr int P_OFF = KV_OFF + A_KV_STAGES * STAGE_BYTES;
     static constexpr int BAR_OFF = P_OFF + P_BYTES;
-    // q_full, kv_full[2], kv_empty[2], s_full, p_full, pv_done
-    static constexpr int N_BARS = 1 + 2 * A_KV_STAGES + 3;
+    // q_full, kv_full[2], kv_empty[2], s_full, p_full, pv_done, s_free
+    static constexpr int N_BARS = 1 + 2 * A_KV_STAGES + 4;
     static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;
 };
@@ -101,6 +105,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t s_full = bar0 + 8u * (1 + 2 * A_KV_STAGES);
     const uint32_t p_full = s_full + 8u;
     const uint32_t pv_done = s_full + 16u;
+    const uint32_t s_free = s_full + 24u;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFF + L::N_BARS * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
@@ -122,6 +127,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_init(s_full, 1);
         mbar_init(p_full, 4);     // one arrival per softmax warp
         mbar_init(pv_done, 1);
+        mbar_init(s_free, 4);     // the score row of every softmax warp is in registers
         *abort_flag = 0;
         mbar_init_fence();
         tma_prefetch_desc(&tm_q);
@@ -139,6 +145,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + 128u;
     const WaitCtx ctx{p.status, abort_flag};
 
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(A_REGS_CTRL));
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (elect_one()) {
@@ -177,11 +185,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (ok) ok = issue_s(0);
             for (int j = 0; j < n_kv && ok; ++j) {
                 const int st = j % A_KV_STAGES;
-                // P8_j is in shared memory, which also means S_j has been read: the S columns are free
+                // the threads hold S_j in registers: the S columns are free, so S_{j+1} runs under the softmax of block j
+                if (j + 1 < n_kv) {
+                    if (!mbar_wait(s_free, (uint32_t)j & 1u, ctx)) { ok = false; break; }
+                    tc_fence_after();
+                    if (!issue_s(j + 1)) { ok = false; break; }
+                }
+                // P8_j is in shared memory
                 if (!mbar_wait(p_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
                 tc_fence_after();
-                // next scores first, so that the softmax of block j+1 can start while P8_j V_j runs
-                if (j + 1 < n_kv && !issue_s(j + 1)) { ok = false; break; }
                 // O += P V: reduction over 128 keys in steps of 32; V advances 32 rows (32*D bytes) per step
                 const uint64_t dv = umma_desc(sbase + L::KV_OFF + st * L::STAGE_BYTES + L::KV_BYTES, D, 16);
 #pragma unroll
@@ -191,7 +203,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 umma_commit(pv_done);
             }
         }
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(A_REGS_SOFTMAX));
         // ------------------------------------------------------------ softmax / correction / epilogue
         const int quad = warp & 3;
         const int r = quad * 32 + lane;                  // row inside the tile = TMEM lane
@@ -208,31 +222,41 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const bool need_mask = (k0 + A_BN - 1 > q0 && p.causal) || (k0 + A_BN > p.N);
             if (!mbar_wait(s_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
             tc_fence_after();
-            // pass 1: row maximum (two chunk loads in flight per wait)
-            float mx = -INFINITY, mx1 = -INFINITY;
+            // the whole score row into registers, then the S columns are released
+            uint32_t sv[4][32];
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t va[32], vb[32];
-                tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(half * 64), va);
-                tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(half * 64 + 32), vb);
-                tmem_ld_wait();
+            for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(q * 32), sv[q]);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_free);
+            // four independent chains of 3-input maxima
+            float mq[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                mq[q] = -INFINITY;
                 if (need_mask) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        if (half * 64 + i <= limit) mx = fmaxf(mx, __uint_as_float(va[i]));
-                        if (half * 64 + 32 + i <= limit) mx1 = fmaxf(mx1, __uint_as_float(vb[i]));
-                    }
+                    for (int i = 0; i < 32; ++i)
+                        if (q * 32 + i <= limit) mq[q] = fmaxf(mq[q], __uint_as_float(sv[q][i]));
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        mx = fmax3(mx, __uint_as_float(va[i]), __uint_as_float(va[i + 1]));
-                        mx1 = fmax3(mx1, __uint_as_float(vb[i]), __uint_as_float(vb[i + 1]));
-                    }
+                    for (int i = 0; i < 32; i += 2)
+                        mq[q] = fmax3(mq[q], __uint_as_float(sv[q][i]), __uint_as_float(sv[q][i + 1]));
                 }
             }
-            mx = fmaxf(mx, mx1);
+            const float mx = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
             const float m_new = fmaxf(m, mx * c);
             const float alpha = ex2_approx(m - m_new);   // 0 on the first block (m = -inf)
+            // P~ * c_P = 2^(c*S - m_new + log2 c_P), row sum and E4M3 codes, all from registers: none of it needs the
+            // previous PV product, whose wait (and the rescale of O) therefore comes after it
+            const float neg_shift = p.log2_p_scale - m_new;
+            float lsum = 0.0f;
+            uint32_t w[4][8];
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                lsum += need_mask ? softmax_chunk<true>(sv[q], c, neg_shift, limit - q * 32, w[q])
+                                  : softmax_chunk<false>(sv[q], c, neg_shift, 0, w[q]);
             // the previous PV (issued after S_j) must be done before O is rescaled or the P tile overwritten
             if (j > 0) {
                 if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, ctx)) { ok = false; break; }
@@ -256,32 +280,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 tmem_st_wait();
             }
-            // pass 2: P~ * c_P = 2^(c*S - m_new + log2 c_P), row sum, E4M3 codes into the operand layout;
-            // the load of chunk q+1 is in flight while chunk q is processed
-            const float neg_shift = p.log2_p_scale - m_new;
-            float lsum = 0.0f;
-            {
-                uint32_t va[32], vb[32], w[8];
-                tmem_ld_32x32b_x32(tmem_s + lane_addr, va);
+            // two 16-byte chunks per 32 keys (keys cc..cc+15, cc+16..cc+31) at their swizzled positions
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int cc = q * 32;
-                    tmem_ld_wait();
-                    if (q < 3) {
-                        if (q & 1) tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(cc + 32), va);
-                        else tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(cc + 32), vb);
-                    }
-                    if (q & 1)
-                        lsum += need_mask ? softmax_chunk<true>(vb, c, neg_shift, limit - cc, w)
-                                          : softmax_chunk<false>(vb, c, neg_shift, 0, w);
-                    else
-                        lsum += need_mask ? softmax_chunk<true>(va, c, neg_shift, limit - cc, w)
-                                          : softmax_chunk<false>(va, c, neg_shift, 0, w);
-                    // two 16-byte chunks (keys cc..cc+15, cc+16..cc+31) at their swizzled positions
-                    const int ch = cc >> 4;
-                    *reinterpret_cast<uint4 *>(prow + (((ch) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-                    *reinterpret_cast<uint4 *>(prow + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-                }
+            for (int q = 0; q < 4; ++q) {
+                const int ch = q * 2;
+                *reinterpret_cast<uint4 *>(prow + (((ch) ^ (r & 7)) << 4)) = make_uint4(w[q][0], w[q][1], w[q][2], w[q][3]);
+                *reinterpret_cast<uint4 *>(prow + (((ch + 1) ^ (r & 7)) << 4)) = make_uint4(w[q][4], w[q][5], w[q][6], w[q][7]);
             }
             l = l * alpha + lsum;
             m = m_new;
