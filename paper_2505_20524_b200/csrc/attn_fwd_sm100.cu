@@ -12,7 +12,8 @@
 //              E4M3, all from registers; then (once the previous PV product is complete) O in TMEM is rescaled
 //              by 2^(m_old - m_new) when a row maximum grew, and P8 is written to shared memory in the K-major
 //              128-byte-swizzled operand layout
-// Final: O = v_inv * acc / (c_P * l) as BF16, LSE = ln2 * (m + log2 l).
+// Final: O = v_inv * acc / (c_P * l) as BF16, staged in the (by then free) K/V ring and written with one tiled
+// bulk store per 64 columns; LSE = ln2 * (m + log2 l).
 #include <math.h>
 
 #include "common.cuh"
@@ -92,7 +93,8 @@ __device__ __forceinline__ float softmax_chunk(const uint32_t (&v)[32], float c,
 template <int D>
 __global__ void __launch_bounds__(A_THREADS, 2)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                const __grid_constant__ CUtensorMap tm_v, const AttnFwdParams p)
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                const AttnFwdParams p)
 {
     using L = AttnFwdSmem<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -133,6 +135,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         tma_prefetch_desc(&tm_q);
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_o);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), A_TMEM_COLS);
@@ -294,10 +297,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(p_full);
         }
-        if (ok && mbar_wait(pv_done, (uint32_t)(n_kv - 1) & 1u, ctx)) {
+        // Epilogue: O = v_inv * acc / (c_P * l) as BF16 through shared memory (the K/V ring is free by now) and one
+        // tiled bulk store per 64 columns; rows past N are clipped by the tensor map.
+        const bool fin = ok && mbar_wait(pv_done, (uint32_t)(n_kv - 1) & 1u, ctx);
+        if (fin) {
             tc_fence_after();
             const float inv = __ldg(p.v_inv) / l;        // l already carries c_P
-            uint16_t *orow = p.O + (((size_t)b * p.N + row) * p.Hq + h) * D;
             uint8_t *o8row = p.O8 + (((size_t)b * p.N + row) * p.Hq + h) * D;
             const float o_scale = p.o_scale ? __ldg(p.o_scale) : 1.0f;
             uint32_t amax2 = 0;
@@ -306,27 +311,28 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 uint32_t v[32];
                 tmem_ld_32x32b_x32(tmem_o + lane_addr + (uint32_t)cc, v);
                 tmem_ld_wait();
-                if (row < p.N) {
+                // staging tile of 64 columns: [128 rows x 128 bytes], 128-byte swizzle
+                uint8_t *trow = smem + L::KV_OFF + (cc >> 6) * (A_BM * 128) + r * 128;
+                const int c0 = (cc & 63) >> 3;           // first 16-byte chunk of these 32 columns
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 o;
-                        o.x = pack_bf16x2(__uint_as_float(v[i]) * inv, __uint_as_float(v[i + 1]) * inv);
-                        o.y = pack_bf16x2(__uint_as_float(v[i + 2]) * inv, __uint_as_float(v[i + 3]) * inv);
-                        o.z = pack_bf16x2(__uint_as_float(v[i + 4]) * inv, __uint_as_float(v[i + 5]) * inv);
-                        o.w = pack_bf16x2(__uint_as_float(v[i + 6]) * inv, __uint_as_float(v[i + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + cc + i) = o;
-                        if (p.o_scale) {
-                            // the codes an unfused cast of the BF16 output would give
-                            amax2 = __vmaxu2(__vmaxu2(__vmaxu2(__vmaxu2(amax2, o.x & 0x7FFF7FFFu), o.y & 0x7FFF7FFFu),
-                                                      o.z & 0x7FFF7FFFu), o.w & 0x7FFF7FFFu);
-                            const uint32_t c0 = cvt_f32x4_to_fp8x4<0>(
-                                __fmul_rn(bf16_lo(o.x), o_scale), __fmul_rn(bf16_hi(o.x), o_scale),
-                                __fmul_rn(bf16_lo(o.y), o_scale), __fmul_rn(bf16_hi(o.y), o_scale));
-                            const uint32_t c1 = cvt_f32x4_to_fp8x4<0>(
-                                __fmul_rn(bf16_lo(o.z), o_scale), __fmul_rn(bf16_hi(o.z), o_scale),
-                                __fmul_rn(bf16_lo(o.w), o_scale), __fmul_rn(bf16_hi(o.w), o_scale));
-                            *reinterpret_cast<uint2 *>(o8row + cc + i) = make_uint2(c0, c1);
-                        }
+                for (int i = 0; i < 32; i += 8) {
+                    uint4 o;
+                    o.x = pack_bf16x2(__uint_as_float(v[i]) * inv, __uint_as_float(v[i + 1]) * inv);
+                    o.y = pack_bf16x2(__uint_as_float(v[i + 2]) * inv, __uint_as_float(v[i + 3]) * inv);
+                    o.z = pack_bf16x2(__uint_as_float(v[i + 4]) * inv, __uint_as_float(v[i + 5]) * inv);
+                    o.w = pack_bf16x2(__uint_as_float(v[i + 6]) * inv, __uint_as_float(v[i + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(trow + (((c0 + (i >> 3)) ^ (r & 7)) << 4)) = o;
+                    if (p.o_scale && row < p.N) {
+                        // the codes an unfused cast of the BF16 output would give
+                        amax2 = __vmaxu2(__vmaxu2(__vmaxu2(__vmaxu2(amax2, o.x & 0x7FFF7FFFu), o.y & 0x7FFF7FFFu),
+                                                  o.z & 0x7FFF7FFFu), o.w & 0x7FFF7FFFu);
+                        const uint32_t e0 = cvt_f32x4_to_fp8x4<0>(
+                            __fmul_rn(bf16_lo(o.x), o_scale), __fmul_rn(bf16_hi(o.x), o_scale),
+                            __fmul_rn(bf16_lo(o.y), o_scale), __fmul_rn(bf16_hi(o.y), o_scale));
+                        const uint32_t e1 = cvt_f32x4_to_fp8x4<0>(
+                            __fmul_rn(bf16_lo(o.z), o_scale), __fmul_rn(bf16_hi(o.z), o_scale),
+                            __fmul_rn(bf16_lo(o.w), o_scale), __fmul_rn(bf16_hi(o.w), o_scale));
+                        *reinterpret_cast<uint2 *>(o8row + cc + i) = make_uint2(e0, e1);
                     }
                 }
             }
@@ -337,6 +343,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             if (row < p.N)
                 p.LSE[((size_t)b * p.Hq + h) * p.N + row] = (m + log2f(l) - p.log2_p_scale) * 0.69314718055994531f;
+        }
+        fence_proxy_async_smem();
+        // all four softmax warps arrive, whatever happened to their waits; the store is issued only if every one finished
+        if (!named_barrier_or(1, 128, !fin) && warp == 4 && lane == 0) {
+#pragma unroll
+            for (int hf = 0; hf < D / 64; ++hf)
+                tma_store_3d(&tm_o, sbase + L::KV_OFF + hf * (A_BM * 128), (h * D + hf * 64) * 2, q0, b);
+            bulk_commit_group();
+            bulk_wait_group_read0();                     // shared memory is read before the CTA may exit
         }
     }
 
@@ -380,7 +395,7 @@ template <int D>
 static int launch_attn_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const AttnFwdParams &p,
                            cudaStream_t st)
 {
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     int rc = make_tmap_3d_u8(&tq, Q8, (uint64_t)p.Hq * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BM);
     if (rc != FP8_OK) return rc;
     rc = make_tmap_3d_u8(&tk, K8, (uint64_t)p.Hkv * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BN);
@@ -390,7 +405,10 @@ static int launch_attn_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *
     FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         AttnFwdSmem<D>::DYN_BYTES));
     dim3 grid((unsigned)((p.N + A_BM - 1) / A_BM), (unsigned)p.Hq, (unsigned)p.B);
-    attn_fwd_kernel<D><<<grid, A_THREADS, AttnFwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, p);
+    // the BF16 output as a byte tensor: 128-byte boxes (64 columns) of 128 rows
+    rc = make_tmap_3d_u8(&to, p.O, (uint64_t)p.Hq * D * 2, (uint64_t)p.N, (uint64_t)p.B, 128, A_BM);
+    if (rc != FP8_OK) return rc;
+    attn_fwd_kernel<D><<<grid, A_THREADS, AttnFwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, to, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }
