@@ -37,7 +37,7 @@ class AttnParams(C.Structure):
                 ("max_mode", C.c_int32), ("pad_", C.c_int32),
                 ("s", C.c_double), ("c_P", C.c_double),
                 ("q_inv", C.c_double), ("k_inv", C.c_double), ("v_inv", C.c_double), ("do_inv", C.c_double),
-                ("ds_scale", C.c_double), ("flip_eps", C.c_double)]
+                ("ds_scale", C.c_double), ("flip_eps", C.c_double), ("max_slack", C.c_double)]
 
 
 def _L():
@@ -300,12 +300,12 @@ def linear_fwd_blockwise(x8, w8, sx_inv, sw_inv, bk=128, bn=128, rows=None, cols
 
 # ---------------------------------------------------------------- attention
 def attn_params(B, N, Hq, Hkv, d, causal=True, quant=True, kv_block=0, max_mode=0, s=None, c_P=448.0,
-                q_inv=1.0, k_inv=1.0, v_inv=1.0, do_inv=1.0, ds_scale=1.0, flip_eps=0.0) -> AttnParams:
+                q_inv=1.0, k_inv=1.0, v_inv=1.0, do_inv=1.0, ds_scale=1.0, flip_eps=0.0, max_slack=0.0) -> AttnParams:
     return AttnParams(B=B, N=N, Hq=Hq, Hkv=Hkv, d=d, causal=int(causal), quant=int(quant),
                       kv_block=kv_block, max_mode=max_mode, pad_=0,
                       s=float(d ** -0.5 if s is None else s), c_P=float(c_P),
                       q_inv=float(q_inv), k_inv=float(k_inv), v_inv=float(v_inv), do_inv=float(do_inv),
-                      ds_scale=float(ds_scale), flip_eps=float(flip_eps))
+                      ds_scale=float(ds_scale), flip_eps=float(flip_eps), max_slack=float(max_slack))
 
 
 def _pairs(sel, nb, nh):

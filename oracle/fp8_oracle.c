@@ -404,6 +404,8 @@ typedef struct {
     double q_inv, k_inv, v_inv, do_inv;  /* descales of Q8, K8, V8, dO8 */
     double ds_scale;   /* backward: quantisation scale of dS */
     double flip_eps;   /* relative uncertainty of an FP32 evaluation (0 disables the slack outputs) */
+    double max_slack;  /* forward: tau >= 0 in powers of two; the reference maximum m moves only when a block maximum
+                        * exceeds it by more than 2^tau, i.e. by tau*ln2 in the exponent (0: whenever it grows) */
 } oracle_attn_params;
 
 typedef struct {
@@ -511,7 +513,7 @@ static void attention_fwd_core(const operand *Q, const operand *K, const operand
                     if (x[j - j0] > bm) bm = x[j - j0];
                 }
                 double cand = (p->max_mode == 1) ? ceil(bm * LOG2E) * LN2 : bm;
-                if (cand > m) {
+                if (cand > m + p->max_slack * LN2) {
                     double f = isinf(m) ? 0.0 : exp(m - cand);
                     l *= f;
                     for (int dd = 0; dd < d; ++dd) { acc[dd] *= f; am[dd] *= f; sl[dd] *= f; }

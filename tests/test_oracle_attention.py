@@ -117,6 +117,48 @@ def test_quantised_forward_matches_stepwise_definition():
             assert np.all((Pt.max(axis=1) > 0.5) & (Pt.max(axis=1) <= 1.0))
 
 
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("kv_block,tau", [(3, 1.0), (4, 3.0), (1, 2.5)])
+def test_reference_maximum_with_slack_leaves_unquantised_attention_unchanged(causal, kv_block, tau):
+    """O and LSE do not depend on the reference maximum: with quant off the slack mode is the textbook result."""
+    B, N, Hq, Hkv, d = 2, 13, 4, 2, 8
+    q, k, v = rand_codes((B, N, Hq, d), 31), rand_codes((B, N, Hkv, d), 32), rand_codes((B, N, Hkv, d), 33)
+    kw = dict(causal=causal, quant=False, kv_block=kv_block, s=0.3, q_inv=0.5, k_inv=2.0, v_inv=0.25)
+    O0, L0, _ = o.attention_fwd(q, k, v, o.attn_params(B, N, Hq, Hkv, d, **kw))
+    O1, L1, _ = o.attention_fwd(q, k, v, o.attn_params(B, N, Hq, Hkv, d, max_slack=tau, **kw))
+    assert np.allclose(O0, O1, rtol=1e-12, atol=1e-13)
+    assert np.allclose(L0, L1, rtol=1e-12)
+
+
+def test_quantised_forward_with_slack_matches_stepwise_definition():
+    """Slack tau: the reference maximum of a row moves only when a block maximum exceeds it by more than 2^tau, so
+    P~ reaches at most 2^tau and is quantised with c_P = 448 / 2^tau.  Reference maximum rebuilt here block by block."""
+    B, N, H, d, Bc, tau = 1, 12, 1, 8, 2, 2.0
+    cP = 448.0 / 2.0 ** tau
+    q, k, v = rand_codes((B, N, H, d), 42), rand_codes((B, N, H, d), 43), rand_codes((B, N, H, d), 44)
+    p = o.attn_params(B, N, H, H, d, quant=True, s=0.9, kv_block=Bc, c_P=cP, max_slack=tau)
+    O, LSE, _ = o.attention_fwd(q, k, v, p)
+    Q, K, V = dec(q)[0, :, 0], dec(k)[0, :, 0], dec(v)[0, :, 0]
+    x = np.where(np.tril(np.ones((N, N), dtype=bool)), 0.9 * Q @ K.T, -np.inf)
+    moved_late = 0
+    for i in range(N):
+        m, num, l = -np.inf, np.zeros(d), 0.0
+        for j0 in range(0, i + 1, Bc):
+            blk = x[i, j0:min(j0 + Bc, i + 1)]
+            if blk.max() > m + tau * np.log(2.0):
+                f = 0.0 if np.isinf(m) else np.exp(m - blk.max())
+                num, l, m = num * f, l * f, blk.max()
+                moved_late += j0 > 0
+            pt = np.exp(blk - m)
+            assert pt.max() <= 2.0 ** tau * (1 + 1e-12)
+            p8 = dec(o.encode_array(pt.astype(np.float32) * np.float32(cP), o.E4M3))
+            num = num + p8 @ V[j0:j0 + len(blk)]
+            l += pt.sum()
+        assert np.allclose(O[0, i], num / (cP * l), rtol=1e-12, atol=1e-14)
+        assert np.isclose(LSE[0, i], m + np.log(l), rtol=1e-13)
+    assert moved_late > 0                      # the case does exercise a later move of the reference
+
+
 def _fd_setup():
     rng = np.random.default_rng(21)
     B, N, Hq, Hkv, d = 1, 8, 2, 1, 4
