@@ -488,6 +488,9 @@ def run_report(args):
         fl = 2.0 * B * Hq * N * N * d
         shape = f"{cname} B{B} N{N} H{Hq}/{Hkv} d{d}"
         add("fp8_attention_fwd", shape, timed(lambda: fp8.fp8_attention_fwd(q8, k8, v8, s1, s1, s1, s, True, O, LSE, None)), flops=fl)
+        add("fp8_attention_fwd (reference maximum with slack 2^2, c_P = 112)", shape,
+            timed(lambda: fp8.fp8_attention_fwd(q8, k8, v8, s1, s1, s1, s, True, O, LSE, None, p_scale=112.0,
+                                                max_slack=2.0)), flops=fl)
         add("fp8_attention_bwd", shape,
             timed(lambda: fp8.fp8_attention_bwd(q8, k8, v8, do8, O, LSE, s1, s1, s1, s1, s, dss, True, dq, dk, dv, ws)),
             flops=2.5 * fl)

@@ -218,7 +218,8 @@ FP8_API int fp8_linear_fwd_blockwise(const uint8_t *X8, const uint8_t *W8, const
  *
  * Forward: scores and softmax in FP32; P~ = exp(x - running max) in (0,1] is re-quantised to E4M3 with
  * scale p_scale (448 = FP8Max / amax(P~)) before the PV product, keys taken in blocks of 128 in ascending
- * order; the row sum uses the un-quantised P~.  O is BF16, LSE[b,h,i] the FP32 log-sum-exp (natural log).
+ * order; the row sum uses the un-quantised P~.  With max_slack = tau > 0 the reference maximum of a row is the
+ * running maximum as of the last block that exceeded the previous reference by more than 2^tau (P~ in (0, 2^tau]).  O is BF16, LSE[b,h,i] the FP32 log-sum-exp (natural log).
  * Backward: recomputes P = exp(x - LSE); dV = P8^T dO, dP = dO V^T, dS = P o (dP - D) with
  * D = rowsum(dO o O), dS -> E5M2 with *ds_scale, dQ = s dS8 K, dK = s dS8^T Q; dK, dV summed over the
  * query heads of a group; *ds_amax (nullable) is overwritten with max|dS|. */
@@ -229,6 +230,10 @@ typedef struct {
     float p_scale;                      /* host value c_P; 448 */
     const float *ds_scale;              /* device scalar: quantisation scale of dS (backward only) */
     float *ds_amax;                     /* device scalar out, nullable (backward only) */
+    float max_slack;                    /* host value tau >= 0, in powers of two (forward only): a row keeps its reference
+                                         * maximum until a block maximum exceeds it by more than 2^tau, so that
+                                         * P~ <= 2^tau and O is rescaled rarely; pass p_scale = 448 / 2^tau (the scaling
+                                         * rule of Appendix E with margin m = tau).  0 = exact running maximum */
 } fp8_attn_scales;
 
 /* Scratch bytes the attention calls need (op: 0 = forward, 1 = backward). */

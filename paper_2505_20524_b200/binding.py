@@ -39,7 +39,7 @@ class Fp8Error(RuntimeError):
 class AttnScales(C.Structure):
     _fields_ = [("q_inv", C.c_void_p), ("k_inv", C.c_void_p), ("v_inv", C.c_void_p), ("do_inv", C.c_void_p),
                 ("softmax_scale", C.c_float), ("p_scale", C.c_float),
-                ("ds_scale", C.c_void_p), ("ds_amax", C.c_void_p)]
+                ("ds_scale", C.c_void_p), ("ds_amax", C.c_void_p), ("max_slack", C.c_float)]
 
 
 def load() -> C.CDLL:
@@ -249,16 +249,18 @@ def fp8_attention_workspace_bytes(op, B, N, Hq, Hkv, d) -> int:
     return int(load().fp8_attention_workspace_bytes(op, B, N, Hq, Hkv, d))
 
 
-def _scales(q_inv, k_inv, v_inv, do_inv, softmax_scale, p_scale, ds_scale, ds_amax):
+def _scales(q_inv, k_inv, v_inv, do_inv, softmax_scale, p_scale, ds_scale, ds_amax, max_slack=0.0):
     return AttnScales(_ptr(q_inv).value, _ptr(k_inv).value, _ptr(v_inv).value, _ptr(do_inv).value,
-                      float(softmax_scale), float(p_scale), _ptr(ds_scale).value, _ptr(ds_amax).value)
+                      float(softmax_scale), float(p_scale), _ptr(ds_scale).value, _ptr(ds_amax).value,
+                      float(max_slack))
 
 
 def fp8_attention_fwd(q8, k8, v8, q_inv, k_inv, v_inv, softmax_scale, causal, o, lse, ws, p_scale=448.0,
-                      stream=None):
+                      stream=None, max_slack=0.0):
+    """max_slack = tau > 0: a row keeps its reference maximum until exceeded by more than 2^tau; p_scale <= 448 / 2^tau."""
     B, N, Hq, d = q8.shape
     Hkv = k8.shape[2]
-    sc = _scales(q_inv, k_inv, v_inv, None, softmax_scale, p_scale, None, None)
+    sc = _scales(q_inv, k_inv, v_inv, None, softmax_scale, p_scale, None, None, max_slack)
     _check(load().fp8_attention_fwd(_ptr(q8), _ptr(k8), _ptr(v8), C.byref(sc), C.c_int(int(causal)), C.c_int(B),
                                     C.c_int(N), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), _ptr(o), _ptr(lse),
                                     _ptr(ws), C.c_size_t(0 if ws is None else ws.numel() * ws.element_size()),
@@ -266,11 +268,11 @@ def fp8_attention_fwd(q8, k8, v8, q_inv, k_inv, v_inv, softmax_scale, causal, o,
 
 
 def fp8_attention_fwd_q(q8, k8, v8, q_inv, k_inv, v_inv, softmax_scale, causal, o, lse, o_scale, o8, o_amax=None,
-                        p_scale=448.0, stream=None):
+                        p_scale=448.0, stream=None, max_slack=0.0):
     """Forward that also emits E4M3 codes of O under a caller (delayed) scale and amax(O)."""
     B, N, Hq, d = q8.shape
     Hkv = k8.shape[2]
-    sc = _scales(q_inv, k_inv, v_inv, None, softmax_scale, p_scale, None, None)
+    sc = _scales(q_inv, k_inv, v_inv, None, softmax_scale, p_scale, None, None, max_slack)
     _check(load().fp8_attention_fwd_q(_ptr(q8), _ptr(k8), _ptr(v8), C.byref(sc), C.c_int(int(causal)), C.c_int(B),
                                       C.c_int(N), C.c_int(Hq), C.c_int(Hkv), C.c_int(d), _ptr(o), _ptr(lse),
                                       _ptr(o_scale), _ptr(o8), _ptr(o_amax), _stream(stream)))

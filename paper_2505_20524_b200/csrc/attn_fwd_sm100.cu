@@ -49,6 +49,7 @@ struct AttnFwdParams {
     const float *q_inv, *k_inv, *v_inv;
     float softmax_scale;
     float log2_p_scale;
+    float max_slack;     // tau: the reference maximum of a row moves only when exceeded by more than 2^tau
     int causal;
     int B, N, Hq, Hkv;
     int *status;
@@ -249,8 +250,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
             }
             const float mx = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
-            const float m_new = fmaxf(m, mx * c);
-            const float alpha = ex2_approx(m - m_new);   // 0 on the first block (m = -inf)
+            // the reference maximum moves when the block maximum exceeds it by more than 2^tau (tau = 0: every time it
+            // grows); on the first block m = -inf, so it always moves and alpha = 0
+            const float m_blk = mx * c;
+            const float m_new = m_blk > m + p.max_slack ? m_blk : m;
+            const float alpha = ex2_approx(m - m_new);
             // P~ * c_P = 2^(c*S - m_new + log2 c_P), row sum and E4M3 codes, all from registers: none of it needs the
             // previous PV product, whose wait (and the rescale of O) therefore comes after it
             const float neg_shift = p.log2_p_scale - m_new;
@@ -431,6 +435,12 @@ static int attention_fwd_common(const char *who, const uint8_t *Q8, const uint8_
         set_error("%s: O must be 16-byte aligned", who);
         return FP8_ERR_ALIGN;
     }
+    // P~ reaches 2^max_slack: its scaled value must stay inside E4M3
+    if (!(sc->max_slack >= 0.0f) || !(sc->max_slack <= 8.0f) || sc->p_scale * exp2f(sc->max_slack) > 448.0f * 1.0001f) {
+        set_error("%s: max_slack must be in [0, 8] with p_scale * 2^max_slack <= 448 (p_scale %g, max_slack %g)", who,
+                  (double)sc->p_scale, (double)sc->max_slack);
+        return FP8_ERR_SHAPE;
+    }
     rc = check_arch();
     if (rc != FP8_OK) return rc;
     AttnFwdParams p;
@@ -439,6 +449,7 @@ static int attention_fwd_common(const char *who, const uint8_t *Q8, const uint8_
     p.q_inv = sc->q_inv; p.k_inv = sc->k_inv; p.v_inv = sc->v_inv;
     p.softmax_scale = sc->softmax_scale;
     p.log2_p_scale = log2f(sc->p_scale);
+    p.max_slack = sc->max_slack;
     p.causal = causal ? 1 : 0;
     p.B = B; p.N = N; p.Hq = Hq; p.Hkv = Hkv;
     p.status = device_status_ptr();

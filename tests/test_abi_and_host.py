@@ -36,7 +36,7 @@ def test_binding_mirrors_header_constants():
     for name, val in re.findall(r"(FP8_(?:OK|ERR_\w+))\s*=\s*(-?\d+)", text):
         assert binding.STATUS_NAMES[int(val)] == name
     assert "FP8_E4M3 = 0" in text and "FP8_E5M2 = 1" in text and binding.E4M3 == 0 and binding.E5M2 == 1
-    assert C.sizeof(binding.AttnScales) == 56          # 4 pointers, 2 floats, 2 pointers
+    assert C.sizeof(binding.AttnScales) == 64          # 4 pointers, 2 floats, 2 pointers, 1 float (+ padding)
     m = re.search(r"FP8_STATIC_SCRATCH_BYTES\s*\((\d+)u\s*<<\s*(\d+)\)", text)
     assert int(m.group(1)) << int(m.group(2)) == binding.STATIC_SCRATCH_BYTES
 

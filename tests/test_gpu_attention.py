@@ -24,12 +24,12 @@ def quantized_qkv(cfg, N, B, seed_shift=0):
     return out
 
 
-def run_fwd(qd, B, N, Hq, Hkv, d, causal, s):
+def run_fwd(qd, B, N, Hq, Hkv, d, causal, s, p_scale=448.0, max_slack=0.0):
     q8, k8, v8 = dev(qd["q"][0]), dev(qd["k"][0]), dev(qd["v"][0])
     O = torch.empty((B, N, Hq, d), dtype=torch.bfloat16, device="cuda")
     LSE = torch.empty((B, Hq, N), dtype=torch.float32, device="cuda")
     fp8.fp8_attention_fwd(q8, k8, v8, scalar(qd["q"][1]), scalar(qd["k"][1]), scalar(qd["v"][1]), s, causal,
-                          O, LSE, None)
+                          O, LSE, None, p_scale=p_scale, max_slack=max_slack)
     torch.cuda.synchronize()
     assert fp8.fp8_device_status() == 0
     return O, LSE
@@ -57,6 +57,44 @@ def test_forward_matches_oracle(name, B, N, causal):
     assert slack.sum() <= 1e-2 * mag.sum()    # tie decisions are the exception, not a blanket excuse
     glse = LSE.cpu().numpy().astype(np.float64).reshape(B * Hq, N)
     assert np.max(np.abs(glse - lse)) <= 1e-3 * max(1.0, np.abs(lse).max())
+
+
+@pytest.mark.parametrize("name,B,N,causal,tau", [("c1", 1, 400, True, 3.0), ("c3", 1, 384, True, 3.0),
+                                                 ("c4", 1, 272, True, 2.0), ("c4", 1, 256, False, 3.0)])
+def test_forward_with_reference_maximum_slack_matches_oracle(name, B, N, causal, tau):
+    """The reference maximum of a row moves only when exceeded by more than 2^tau; P~ is scaled by 448 / 2^tau."""
+    cfg = synth.CONFIGS[name]
+    Hq, Hkv, d = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    if name != "c1":
+        Hq, Hkv = Hq // 4, Hkv // 4
+        cfg = synth.BlockConfig(**{**cfg.__dict__, "n_q_heads": Hq, "n_kv_heads": Hkv})
+    qd = quantized_qkv(cfg, N, B)
+    s = d ** -0.5
+    c_P = 448.0 / 2.0 ** tau
+    O, LSE = run_fwd(qd, B, N, Hq, Hkv, d, causal, s, p_scale=c_P, max_slack=tau)
+    p = o.attn_params(B, N, Hq, Hkv, d, causal=causal, quant=True, kv_block=KV_BLOCK, max_mode=0, s=s, c_P=c_P,
+                      max_slack=tau, q_inv=qd["q"][1], k_inv=qd["k"][1], v_inv=qd["v"][1], flip_eps=FLIP_EPS)
+    ref, lse, mag, slack = o.attention_fwd(qd["q"][0], qd["k"][0], qd["v"][0], p, with_slack=True)
+    got = O.float().cpu().numpy().astype(np.float64).transpose(0, 2, 1, 3).reshape(B * Hq, N, d)
+    # a row whose block maximum sits within rounding of reference + 2^tau may move its reference on one side only:
+    # both results are valid there (O does not depend on the reference), they differ by quantisation noise of P8
+    err = np.maximum(np.abs(got - ref) - slack, 0.0) / np.maximum(mag, 1e-30)
+    assert np.quantile(err, 0.999) <= TOL_FWD, np.quantile(err, 0.999)
+    assert err.max() <= 4 * TOL_FWD, err.max()
+    glse = LSE.cpu().numpy().astype(np.float64).reshape(B * Hq, N)
+    assert np.max(np.abs(glse - lse)) <= 1e-3 * max(1.0, np.abs(lse).max())
+    # and against the exact-maximum result of the same kernel: the same attention up to P8 quantisation noise
+    O0, _ = run_fwd(qd, B, N, Hq, Hkv, d, causal, s)
+    g0 = O0.float().cpu().numpy().astype(np.float64).transpose(0, 2, 1, 3).reshape(B * Hq, N, d)
+    assert np.quantile(np.abs(got - g0) / np.maximum(mag, 1e-30), 0.999) <= 6e-2
+
+
+def test_reference_maximum_slack_validation():
+    cfg = synth.CONFIGS["c1"]
+    qd = quantized_qkv(cfg, 128, 1)
+    with pytest.raises(fp8.Fp8Error) as e:        # P~ would reach 8 * 448
+        run_fwd(qd, 1, 128, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, True, 0.125, p_scale=448.0, max_slack=3.0)
+    assert e.value.status == -3
 
 
 def test_softmax_scale_parameter():
