@@ -350,7 +350,7 @@ __global__ void __launch_bounds__(256) qk_norm_rope_kernel(const uint16_t *__res
             c[0] = c0.x; c[1] = c0.y; c[2] = c0.z; c[3] = c0.w; c[4] = c1.x; c[5] = c1.y; c[6] = c1.z; c[7] = c1.w;
             sn[0] = s0.x; sn[1] = s0.y; sn[2] = s0.z; sn[3] = s0.w; sn[4] = s1.x; sn[5] = s1.y; sn[6] = s1.z; sn[7] = s1.w;
         }
-#pragma unroll 2
+#pragma unroll 4
         for (int hh = 0; hh < QK_HC; ++hh) {
             const bool valid = item_valid && h0 + hh < H;
             const size_t v = tok * (size_t)H + (size_t)min(h0 + hh, H - 1);
@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(256) qk_norm_rope_kernel(const uint16_t *__res
                 for (int e = 0; e < 8; ++e) ss = fmaf(a[e], a[e], fmaf(b[e], b[e], ss));
 #pragma unroll
                 for (int off = LPV / 2; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
-                const float rinv = 1.0f / sqrtf(ss / (float)D + eps);
+                const float rinv = rsqrtf(fmaf(ss, 1.0f / (float)D, eps));
 #pragma unroll
                 for (int e = 0; e < 8; ++e) { a[e] *= rinv; b[e] *= rinv; }
             } else if (MODE == FP8_QK_TANH) {
