@@ -264,7 +264,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const float db = row_ok ? __ldg(p.Dsum + li) * b_d : 0.0f;
             const int limit = min(p.causal ? row : 0x7FFFFFFF, p.N - 1) - k0;   // last valid local key
             const bool need_mask = (p.causal && k0 + B_BN - 1 > q0) || (k0 + B_BN > p.N);
-            if (!mbar_wait(s_full, (uint32_t)t & 1u, ctx)) { ok = false; break; }
+            if (!mbar_wait_warp(s_full, (uint32_t)t & 1u, ctx)) { ok = false; break; }   // warp-uniform: .sync.aligned loads follow
             tc_fence_after();
 #pragma unroll 1
             for (int cc = 0; cc < B_BN; cc += 32) {
@@ -300,7 +300,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(pds_full);
             // drain the dQ tile of this pair into the FP32 accumulator
-            if (!mbar_wait(dq_full, (uint32_t)t & 1u, ctx)) { ok = false; break; }
+            if (!mbar_wait_warp(dq_full, (uint32_t)t & 1u, ctx)) { ok = false; break; }
             tc_fence_after();
             float *qacc = p.dQacc + (((size_t)b * p.N + (row_ok ? row : 0)) * p.Hq + h) * D;
 #pragma unroll 1

@@ -224,7 +224,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // keys beyond the row (causal, only the diagonal block) or beyond N get -inf
             const int limit = min(p.causal ? row : 0x7FFFFFFF, p.N - 1) - k0;   // last valid local column
             const bool need_mask = (k0 + A_BN - 1 > q0 && p.causal) || (k0 + A_BN > p.N);
-            if (!mbar_wait(s_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
+            // (warp-uniform waits: the warp-wide votes and barriers below name every lane)
+            if (!mbar_wait_warp(s_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
             tc_fence_after();
             // the whole score row into registers, then the S columns are released
             uint32_t sv[4][32];
@@ -266,7 +267,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                                   : softmax_chunk<false>(sv[q], c, neg_shift, 0, w[q]);
             // the previous PV (issued after S_j) must be done before O is rescaled or the P tile overwritten
             if (j > 0) {
-                if (!mbar_wait(pv_done, (uint32_t)(j - 1) & 1u, ctx)) { ok = false; break; }
+                if (!mbar_wait_warp(pv_done, (uint32_t)(j - 1) & 1u, ctx)) { ok = false; break; }
                 tc_fence_after();
             }
             if (j > 0 && __any_sync(0xffffffffu, m_new > m)) {
@@ -303,7 +304,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
         // Epilogue: O = v_inv * acc / (c_P * l) as BF16 through shared memory (the K/V ring is free by now) and one
         // tiled bulk store per 64 columns; rows past N are clipped by the tensor map.
-        const bool fin = ok && mbar_wait(pv_done, (uint32_t)(n_kv - 1) & 1u, ctx);
+        const bool fin = ok && mbar_wait_warp(pv_done, (uint32_t)(n_kv - 1) & 1u, ctx);
         if (fin) {
             tc_fence_after();
             const float inv = __ldg(p.v_inv) / l;        // l already carries c_P
