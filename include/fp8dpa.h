@@ -57,6 +57,12 @@ FP8_API const char *fp8_last_error(void);
  * or FP8_ERR_TIMEOUT) and clears it. */
 FP8_API int fp8_device_status(int *status_out, void *stream);
 
+/* Self-test of the bounded-wait path: one warp waits on a barrier that nothing ever completes, with a limit of
+ * `limit_cycles` SM clocks (0 < limit_cycles <= 2^31).  At the limit it gives up the way every kernel of the library
+ * does when a wait runs out: FP8_ERR_TIMEOUT goes into the device status word, *gave_up (device int) is set to 1 and
+ * the kernel returns; the context stays usable.  Enqueues on `stream` and returns FP8_OK. */
+FP8_API int fp8_selftest_wait_timeout(long long limit_cycles, int *gave_up, void *stream);
+
 /* ---- per-tensor scaling ---------------------------------------------------------------------------
  * Appendix C (definition above Theorem 1): s(x) = MaxFP8Value / absmax(x); Appendix E: rho(X) =
  * FP8MaxValue / (2^m max H) and FP8cast(rho(X) X).  MaxFP8Value is 448 (E4M3) / 57344 (E5M2). */

@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
-SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
+SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_qk_norm_rope", "fp8_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
@@ -82,6 +82,11 @@ def fp8_device_status(stream=None) -> int:
     out = C.c_int(0)
     _check(load().fp8_device_status(C.byref(out), _stream(stream)))
     return out.value
+
+
+def fp8_selftest_wait_timeout(limit_cycles, gave_up, stream=None):
+    """One warp waits on a barrier nothing completes and gives up after limit_cycles: status word = FP8_ERR_TIMEOUT."""
+    _check(load().fp8_selftest_wait_timeout(C.c_longlong(int(limit_cycles)), _ptr(gave_up), _stream(stream)))
 
 
 def fp8_amax(x, amax, stream=None):

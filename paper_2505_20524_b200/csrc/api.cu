@@ -165,6 +165,24 @@ int make_tmap_3d_f32(CUtensorMap *map, const void *base, uint64_t d0_cols, uint6
     return FP8_OK;
 }
 
+// One warp waits on a barrier that nothing ever completes, with a short limit: the path every kernel of the library
+// takes when a wait runs out (status word, shared abort flag, orderly return).
+__global__ void wait_timeout_selftest_kernel(int *status, long long limit, int *gave_up)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        abort_flag = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    const WaitCtx ctx{status, &abort_flag, limit};
+    const bool got = mbar_wait_warp(b, 0u, ctx);
+    if (threadIdx.x == 0) *gave_up = got ? 0 : 1;
+}
+
 }  // namespace fp8dpa
 
 extern "C" const char *fp8_last_error(void) { return fp8dpa::g_err; }
@@ -181,5 +199,24 @@ extern "C" int fp8_device_status(int *status_out, void *stream)
     FP8_CUDA_CHECK(cudaStreamSynchronize(s));
     FP8_CUDA_CHECK(cudaMemcpy(status_out, p, sizeof(int), cudaMemcpyDeviceToHost));
     FP8_CUDA_CHECK(cudaMemset(p, 0, sizeof(int)));
+    return FP8_OK;
+}
+
+extern "C" int fp8_selftest_wait_timeout(long long limit_cycles, int *gave_up, void *stream)
+{
+    if (!gave_up) {
+        fp8dpa::set_error("fp8_selftest_wait_timeout: gave_up is NULL");
+        return FP8_ERR_NULL;
+    }
+    if (limit_cycles <= 0 || limit_cycles > (1ll << 31)) {
+        fp8dpa::set_error("fp8_selftest_wait_timeout: limit_cycles must be in (0, 2^31], got %lld", limit_cycles);
+        return FP8_ERR_SHAPE;
+    }
+    int rc = fp8dpa::check_arch();
+    if (rc != FP8_OK) return rc;
+    int *status = fp8dpa::device_status_ptr();
+    if (!status) return FP8_ERR_CUDA;
+    fp8dpa::wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status, limit_cycles, gave_up);
+    FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }

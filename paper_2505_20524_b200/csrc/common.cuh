@@ -90,6 +90,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 struct WaitCtx {
     int *status;              // global status word
     volatile int *abort_flag; // shared, one per CTA
+    long long limit;          // SM clocks after which a wait gives up; 0 = the default
 };
 #ifndef FP8DPA_WAIT_LIMIT_CYCLES
 #define FP8DPA_WAIT_LIMIT_CYCLES 4000000000ll
@@ -102,7 +103,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0) {
             if (*ctx.abort_flag) return false;
-            if (clock64() - t0 > FP8DPA_WAIT_LIMIT_CYCLES) {
+            if (clock64() - t0 > (ctx.limit > 0 ? ctx.limit : FP8DPA_WAIT_LIMIT_CYCLES)) {
                 *ctx.abort_flag = 1;
                 atomicExch(ctx.status, (int)FP8_ERR_TIMEOUT);
                 return false;

@@ -146,3 +146,26 @@ def test_delayed_scaling_step_is_one_pass():
         fp8.fp8_scale_update(hist_d, head_d, a, o.E4M3, 0, s, si)
         head, es, _ = o.scale_update(hist, head, o.amax(x), o.E4M3)
         assert bits(s) == int(es.view(np.uint32))
+
+
+def test_bounded_wait_gives_up_and_reports():
+    """A wait that nothing completes runs out at its limit: FP8_ERR_TIMEOUT in the status word, the kernel returns,
+    and the context stays usable (the path every kernel of the library takes when a wait expires)."""
+    import time
+    assert fp8.fp8_device_status() == 0
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = time.time()
+    fp8.fp8_selftest_wait_timeout(1 << 22, flag)          # about 2 ms of SM clocks
+    torch.cuda.synchronize()
+    assert time.time() - t0 < 5.0
+    assert int(flag.item()) == 1
+    assert fp8.fp8_device_status() == -7                   # FP8_ERR_TIMEOUT, cleared by the read
+    assert fp8.fp8_device_status() == 0
+    x = torch.arange(-8, 8, dtype=torch.float32, device="cuda").to(torch.bfloat16)
+    a = torch.zeros(1, dtype=torch.float32, device="cuda")
+    fp8.fp8_amax(x, a)                                      # the next kernel runs as usual
+    torch.cuda.synchronize()
+    assert float(a.item()) == 8.0 and fp8.fp8_device_status() == 0
+    with pytest.raises(fp8.Fp8Error) as e:
+        fp8.fp8_selftest_wait_timeout(0, flag)
+    assert e.value.status == -3
