@@ -468,7 +468,11 @@ def run_report(args):
     s1, swg = f32(1e-2), torch.full((E,), 1e-2, device="cuda")
     add("fp8_grouped_linear_fwd (8 experts, uneven)", f"{Tr} rows x {Ng} x {Kg}",
         timed(lambda: fp8.fp8_grouped_linear_fwd(x8, w8, s1, swg, offs, yb)), flops=2.0 * Tr * Ng * Kg)
-    del x8, w8, yb
+    dy8 = codes(Tr, Ng)
+    dxb = torch.empty((Tr, Kg), dtype=torch.bfloat16, device="cuda")
+    add("fp8_grouped_linear_dgrad (8 experts, uneven, weights in place)", f"{Tr} rows x {Ng} x {Kg}",
+        timed(lambda: fp8.fp8_grouped_linear_dgrad(dy8, w8, s1, swg, offs, dxb)), flops=2.0 * Tr * Ng * Kg)
+    del x8, w8, yb, dy8, dxb
 
     # ---- attention of c3, c4, c5 (causal)
     for cname in ("c3", "c4", "c5"):

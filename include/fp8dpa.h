@@ -187,6 +187,12 @@ FP8_API int fp8_grouped_linear_fwd(const uint8_t *X8, const uint8_t *W8, const f
                            const int *group_offsets, int n_groups, void *Y, int out_is_fp32, int T, int N, int K,
                            void *stream);
 
+/* Its data gradient: dX[t, :] = sdY_inv * sW_inv[g(t)] * dY8[t, :] . W8[g(t)] with dY8 [T,N] in E5M2 (rows sorted by
+ * expert like X8) and the weights read in place ([N,K] per expert, no transposed copies).  N % 128 == 0. */
+FP8_API int fp8_grouped_linear_dgrad(const uint8_t *dY8, const uint8_t *W8, const float *sdY_inv, const float *sW_inv,
+                             const int *group_offsets, int n_groups, void *dX, int out_is_fp32, int T, int N, int K,
+                             void *stream);
+
 /* Producer forms for delayed scaling (Appendix E: rho comes from the amax history, so the producer of a tensor can
  * emit FP8 in its own epilogue, "a single pass on the data", Section 2).  Same products as fp8_linear_fwd /
  * fp8_linear_dgrad; the result is rounded to BF16 (the tensor an unfused chain would store), its amax is written to

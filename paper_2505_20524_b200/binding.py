@@ -21,7 +21,7 @@ _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_qk_norm_rope", "fp8_kurtosis",
-           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
+           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
 STATIC_SCRATCH_BYTES = 32 << 20
@@ -217,6 +217,15 @@ def fp8_grouped_linear_fwd(x8, w8, sx_inv, sw_inv, group_offsets, y, stream=None
     _check(load().fp8_grouped_linear_fwd(_ptr(x8), _ptr(w8), _ptr(sx_inv), _ptr(sw_inv), _ptr(group_offsets),
                                          C.c_int(E), _ptr(y), C.c_int(_is_fp32(y)), C.c_int(T), C.c_int(N), C.c_int(K),
                                          _stream(stream)))
+
+
+def fp8_grouped_linear_dgrad(dy8, w8, sdy_inv, sw_inv, group_offsets, dx, stream=None):
+    """Per-expert data gradient: dy8 [T, N] (E5M2) sorted by expert, w8 [E, N, K] read in place, dx [T, K]."""
+    T, N = dy8.shape
+    E, K = w8.shape[0], w8.shape[2]
+    _check(load().fp8_grouped_linear_dgrad(_ptr(dy8), _ptr(w8), _ptr(sdy_inv), _ptr(sw_inv), _ptr(group_offsets),
+                                           C.c_int(E), _ptr(dx), C.c_int(_is_fp32(dx)), C.c_int(T), C.c_int(N),
+                                           C.c_int(K), _stream(stream)))
 
 
 def fp8_quantize_blockwise(x, block_rows, fmt, out, scale_inv, stream=None):

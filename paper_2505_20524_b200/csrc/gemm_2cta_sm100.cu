@@ -144,12 +144,15 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             uint32_t phase = 0;
             bool ok = true;
             for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs) {
-                int tm, tn, m_base = 0, n_base = 0;
+                int tm, tn, m_base = 0, n_base = 0, kb_base_b = 0;
                 if (GROUPED) {
                     const GroupTile gt = group_tile(g_tile_start, g_offs, p.n_groups, tiles_n, tile);
                     tm = gt.tm; tn = gt.tn;
                     m_base = gt.row0;              // rows of A: the group's slice of the sorted token matrix
-                    n_base = gt.g * p.N;           // rows of B: the group's weight matrix
+                    // rows of B: the group's weight matrix -- its output rows (K-major B, forward) or its reduction
+                    // rows (MN-major B: the stored [reduction, output] matrix of the data gradient)
+                    if (p.b_mn) kb_base_b = gt.g * p.K;
+                    else n_base = gt.g * p.N;
                 } else {
                     tile_coords(tile, tiles_m, tiles_n, tm, tn);
                 }
@@ -162,7 +165,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                     // rows x 128 bytes of the output index (the matrix as it lies in memory, no transposed copy)
                     if (p.a_mn) tma_load_2d_pair(sa, &tmap_a, full_bar(stage), m0, kb * BK);
                     else tma_load_2d_pair(sa, &tmap_a, full_bar(stage), kb * BK, m0);
-                    if (p.b_mn) tma_load_2d_pair(sb, &tmap_b, full_bar(stage), n0, kb * BK);
+                    if (p.b_mn) tma_load_2d_pair(sb, &tmap_b, full_bar(stage), n0, kb_base_b + kb * BK);
                     else tma_load_2d_pair(sb, &tmap_b, full_bar(stage), kb * BK, n0);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -308,14 +311,17 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
 
 // Grouped form: Y[rows of group g] = sa_inv * sb_inv[g] * A[rows of group g] . B_g^T for every group, one launch.
 int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv,
-                             const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int K,
+                             const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int K, int b_mn,
                              uint32_t idesc, int *status, cudaStream_t st)
 {
     using namespace g2;
     CUtensorMap ta, tb;
     int rc = make_tmap_2d_u8(&ta, a, (uint64_t)M, (uint64_t)K, (uint64_t)K, BM, BK);
     if (rc != FP8_OK) return rc;
-    rc = make_tmap_2d_u8(&tb, b, (uint64_t)n_groups * N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
+    // K-major B: the groups' [N, K] matrices back to back; MN-major B: their [K, N] matrices back to back (K here is the
+    // reduction length of this product), 128 reduction rows x 128 bytes per box
+    rc = b_mn ? make_tmap_2d_u8(&tb, b, (uint64_t)n_groups * K, (uint64_t)N, (uint64_t)N, BK, BN / 2)
+              : make_tmap_2d_u8(&tb, b, (uint64_t)n_groups * N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
     if (rc != FP8_OK) return rc;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
     // the host does not know the group sizes: at most ceil(M/256) + n_groups row tiles exist
@@ -324,7 +330,7 @@ int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa
     Params p;
     p.o = o; p.sa_inv = sa_inv; p.sb_inv = sb_inv;
     p.M = M; p.N = N; p.K = K;
-    p.a_mn = 0; p.b_mn = 0;
+    p.a_mn = 0; p.b_mn = b_mn;
     p.idesc = idesc;
     p.num_pairs = (int)(tiles_bound < pairs_max ? tiles_bound : pairs_max);
     p.status = status;

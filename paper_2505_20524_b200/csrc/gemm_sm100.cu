@@ -222,7 +222,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
                      int M, int N, int K, int a_mn, int b_mn, uint32_t idesc, int *status, cudaStream_t st);
 
 int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv,
-                             const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int K,
+                             const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int K, int b_mn,
                              uint32_t idesc, int *status, cudaStream_t st);
 
 // FP8DPA_GEMM=1cta|2cta forces one kernel family (for A/B measurements); default: chosen per shape.
@@ -439,7 +439,37 @@ extern "C" int fp8_grouped_linear_fwd(const uint8_t *X8, const uint8_t *W8, cons
     int *status = device_status_ptr();
     if (!status) return FP8_ERR_CUDA;
     const GemmOut o{Y, out_is_fp32, 0, nullptr, 0, nullptr};
-    return launch_gemm_2cta_grouped(X8, W8, sX_inv, sW_inv, group_offsets, n_groups, o, T, N, K,
+    return launch_gemm_2cta_grouped(X8, W8, sX_inv, sW_inv, group_offsets, n_groups, o, T, N, K, 0,
                                     umma_idesc_f8(FP8_E4M3, FP8_E4M3, 256, 256), status,
+                                    static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int fp8_grouped_linear_dgrad(const uint8_t *dY8, const uint8_t *W8, const float *sdY_inv, const float *sW_inv,
+                                        const int *group_offsets, int n_groups, void *dX, int out_is_fp32, int T, int N,
+                                        int K, void *stream)
+{
+    if (!group_offsets) {
+        set_error("fp8_grouped_linear_dgrad: NULL group_offsets");
+        return FP8_ERR_NULL;
+    }
+    if (n_groups <= 0 || n_groups > 256) {
+        set_error("fp8_grouped_linear_dgrad: n_groups %d must be in [1, 256]", n_groups);
+        return FP8_ERR_SHAPE;
+    }
+    if (N % 128 != 0) {
+        // a reduction block of 128 rows must not reach into the next expert's weight matrix
+        set_error("fp8_grouped_linear_dgrad: N = %d must be a multiple of 128", N);
+        return FP8_ERR_SHAPE;
+    }
+    // dX[T,K] = dY8[T,N] . W8_g[N,K]: reduction length N, output width K
+    int rc = validate_gemm("fp8_grouped_linear_dgrad", dY8, W8, sdY_inv, sW_inv, dX, T, K, N);
+    if (rc != FP8_OK) return rc;
+    rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    int *status = device_status_ptr();
+    if (!status) return FP8_ERR_CUDA;
+    const GemmOut o{dX, out_is_fp32, 0, nullptr, 0, nullptr};
+    return launch_gemm_2cta_grouped(dY8, W8, sdY_inv, sW_inv, group_offsets, n_groups, o, T, K, N, 1,
+                                    umma_idesc_f8(FP8_E5M2, FP8_E4M3, 256, 256, 0, 1), status,
                                     static_cast<cudaStream_t>(stream));
 }

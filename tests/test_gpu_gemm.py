@@ -265,6 +265,45 @@ def test_grouped_forward_matches_oracle_per_expert(sizes, N, K, out_dtype):
     assert np.all(got[T:] == 7.0)
 
 
+@pytest.mark.parametrize("sizes,N,K", [([300, 0, 129, 512, 83], 512, 144), ([256, 256], 256, 256),
+                                        ([1000, 17, 2000, 1, 600, 0, 0, 350], 1024, 528), ([16], 128, 16)])
+@pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
+def test_grouped_data_gradient_matches_oracle_per_expert(sizes, N, K, out_dtype):
+    """dX of the mixture-of-experts product: gradient rows sorted by expert, every expert's [N, K] weights read in place."""
+    E, T = len(sizes), sum(sizes)
+    Tpad = T + 21
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    dy = synth.normal_bf16((Tpad, N), 70 + E, 0, synth.GRAD_STD)
+    dy8, _, _, _, sdy = gpu_quantize(dy, o.E5M2, False)
+    ody8, _, _, osdy = o.quantize(dy, o.E5M2)
+    w8 = torch.empty((E, N, K), dtype=torch.uint8, device="cuda")
+    sw = torch.empty(E, dtype=torch.float32, device="cuda")
+    ow = []
+    for e in range(E):
+        w = synth.normal_bf16((N, K), 70 + E, 10 + e, synth.W_STD * (1 + e))
+        c, _, _, _, si = gpu_quantize(w, o.E4M3, False)
+        w8[e].copy_(c)
+        sw[e:e + 1].copy_(si)
+        ow.append(o.quantize(w, o.E4M3))
+    dx = torch.full((Tpad, K), 7.0, dtype=out_dtype, device="cuda")
+    fp8.fp8_grouped_linear_dgrad(dy8, w8, sdy, sw, torch.from_numpy(offs).cuda(), dx)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    got = dx.float().cpu().numpy().astype(np.float64)
+    tol = 2.0 ** -8 if out_dtype == torch.bfloat16 else TOL_FP32
+    for e in range(E):
+        r0, r1 = int(offs[e]), int(offs[e + 1])
+        if r1 == r0:
+            continue
+        ref, mag = o.linear_dgrad(ody8[r0:r1], ow[e][0], osdy, ow[e][3])
+        assert rel_err(got[r0:r1], ref, mag) <= tol, e
+    assert np.all(got[T:] == 7.0)
+    with pytest.raises(fp8.Fp8Error) as err:                       # a reduction block must not span two experts
+        fp8.fp8_grouped_linear_dgrad(dy8[:, :N - 16].contiguous(), w8[:, :N - 16].contiguous(), sdy, sw,
+                                     torch.from_numpy(offs).cuda(), dx)
+    assert err.value.status == -3
+
+
 def test_grouped_forward_argument_validation():
     x8 = torch.zeros((32, 32), dtype=torch.uint8, device="cuda")
     w8 = torch.zeros((2, 16, 32), dtype=torch.uint8, device="cuda")
