@@ -43,7 +43,7 @@ def measured_peaks():
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
 
-    def __init__(self, index: int, period: float = 0.01):
+    def __init__(self, index: int, period: float = 0.005):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -70,6 +70,13 @@ class ClockSampler(threading.Thread):
             nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
             nv.nvmlClocksThrottleReasonHwPowerBrakeSlowdown: "hw_power_brake",
         }
+        # the benign ones too, so that a clock below the maximum never comes without its reason
+        for attr, name in (("nvmlClocksThrottleReasonGpuIdle", "gpu_idle"),
+                           ("nvmlClocksThrottleReasonApplicationsClocksSetting", "applications_clocks_setting"),
+                           ("nvmlClocksThrottleReasonSyncBoost", "sync_boost"),
+                           ("nvmlClocksThrottleReasonDisplayClockSetting", "display_clock_setting")):
+            if hasattr(nv, attr):
+                names[getattr(nv, attr)] = name
         while not self._halt.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
@@ -86,7 +93,7 @@ class ClockSampler(threading.Thread):
         self.join(timeout=2)
         s = sorted(self.samples)
         return {"sm_mhz": s[len(s) // 2] if s else None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(s)}
+                "samples": len(s), "sm_mhz_min": s[0] if s else None, "sm_mhz_max_seen": s[-1] if s else None}
 
 
 def physical_gpu_index(local_index: int) -> int:
