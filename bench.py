@@ -479,7 +479,11 @@ def run_report(args):
     dxb = torch.empty((Tr, Kg), dtype=torch.bfloat16, device="cuda")
     add("fp8_grouped_linear_dgrad (8 experts, uneven, weights in place)", f"{Tr} rows x {Ng} x {Kg}",
         timed(lambda: fp8.fp8_grouped_linear_dgrad(dy8, w8, s1, swg, offs, dxb)), flops=2.0 * Tr * Ng * Kg)
-    del x8, w8, yb, dy8, dxb
+    dwb = torch.empty((E, Ng, Kg), dtype=torch.bfloat16, device="cuda")
+    offs_host = [int(v) for v in offs.cpu().tolist()]
+    add("fp8_grouped_linear_wgrad (8 experts, uneven, one launch per expert)", f"{Tr} rows x {Ng} x {Kg}",
+        timed(lambda: fp8.fp8_grouped_linear_wgrad(dy8, x8, s1, s1, offs_host, dwb)), flops=2.0 * Tr * Ng * Kg)
+    del x8, w8, yb, dy8, dxb, dwb
 
     # ---- attention of c3, c4, c5 (causal)
     for cname in ("c3", "c4", "c5"):

@@ -193,6 +193,15 @@ FP8_API int fp8_grouped_linear_dgrad(const uint8_t *dY8, const uint8_t *W8, cons
                              const int *group_offsets, int n_groups, void *dX, int out_is_fp32, int T, int N, int K,
                              void *stream);
 
+/* Its weight gradients: dW[g] (+)= sdY_inv * sX_inv * dY8[rows of g]^T . X8[rows of g], dW [n_groups, N, K] (BF16 or
+ * FP32), both operands read in place.  One launch of the weight-gradient product per expert on its slice of rows;
+ * ragged and empty groups need no padding (an empty group gives zeros, or leaves dW[g] alone with `accumulate`).
+ * Unlike the two calls above the offsets are a HOST array (n_groups + 1 entries): the per-expert launches are set up
+ * on the host. */
+FP8_API int fp8_grouped_linear_wgrad(const uint8_t *dY8, const uint8_t *X8, const float *sdY_inv, const float *sX_inv,
+                             const int *group_offsets_host, int n_groups, void *dW, int out_is_fp32, int accumulate,
+                             int T, int N, int K, void *stream);
+
 /* Producer forms for delayed scaling (Appendix E: rho comes from the amax history, so the producer of a tensor can
  * emit FP8 in its own epilogue, "a single pass on the data", Section 2).  Same products as fp8_linear_fwd /
  * fp8_linear_dgrad; the result is rounded to BF16 (the tensor an unfused chain would store), its amax is written to

@@ -21,7 +21,7 @@ _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_qk_norm_rope", "fp8_kurtosis",
-           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
+           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
 STATIC_SCRATCH_BYTES = 32 << 20
@@ -225,6 +225,18 @@ def fp8_grouped_linear_dgrad(dy8, w8, sdy_inv, sw_inv, group_offsets, dx, stream
     E, K = w8.shape[0], w8.shape[2]
     _check(load().fp8_grouped_linear_dgrad(_ptr(dy8), _ptr(w8), _ptr(sdy_inv), _ptr(sw_inv), _ptr(group_offsets),
                                            C.c_int(E), _ptr(dx), C.c_int(_is_fp32(dx)), C.c_int(T), C.c_int(N),
+                                           C.c_int(K), _stream(stream)))
+
+
+def fp8_grouped_linear_wgrad(dy8, x8, sdy_inv, sx_inv, group_offsets_host, dw, accumulate=False, stream=None):
+    """Per-expert weight gradients: dy8 [T, N], x8 [T, K] sorted by expert, dw [E, N, K]; offsets are host integers."""
+    T, N = dy8.shape
+    K = x8.shape[1]
+    offs = [int(v) for v in group_offsets_host]
+    E = len(offs) - 1
+    arr = (C.c_int * len(offs))(*offs)
+    _check(load().fp8_grouped_linear_wgrad(_ptr(dy8), _ptr(x8), _ptr(sdy_inv), _ptr(sx_inv), arr, C.c_int(E), _ptr(dw),
+                                           C.c_int(_is_fp32(dw)), C.c_int(int(accumulate)), C.c_int(T), C.c_int(N),
                                            C.c_int(K), _stream(stream)))
 
 

@@ -233,13 +233,14 @@ static int gemm_family_override()
 }
 
 static int validate_gemm(const char *who, const void *a, const void *b, const float *sa, const float *sb, void *out,
-                         int M, int N, int K)
+                         int M, int N, int K, bool any_reduce = false)
 {
     if (!a || !b || !sa || !sb || !out) {
         set_error("%s: NULL pointer", who);
         return FP8_ERR_NULL;
     }
-    if (M <= 0 || N <= 0 || K <= 0 || (K % 16) || (N % 16)) {
+    // (with both operands read in place the reduction index counts rows, which the tensor maps zero-fill past the end)
+    if (M <= 0 || N <= 0 || K <= 0 || (!any_reduce && (K % 16)) || (N % 16)) {
         set_error("%s: unsupported shape (rows=%d cols=%d reduce=%d; cols and reduce must be positive multiples of 16)",
                   who, M, N, K);
         return FP8_ERR_SHAPE;
@@ -278,7 +279,7 @@ static int launch_gemm(const uint8_t *a, const uint8_t *b, const GemmParams &p, 
 int gemm_fp8(const char *who, const uint8_t *a, int fmt_a, const uint8_t *b, int fmt_b, const float *sa_inv,
              const float *sb_inv, const GemmOut &o, int M, int N, int K, cudaStream_t st, int a_mn = 0, int b_mn = 0)
 {
-    int rc = validate_gemm(who, a, b, sa_inv, sb_inv, o.out, M, N, K);
+    int rc = validate_gemm(who, a, b, sa_inv, sb_inv, o.out, M, N, K, a_mn && b_mn);
     if (rc != FP8_OK) return rc;
     if (o.q_scale && o.q_fmt != FP8_E4M3 && o.q_fmt != FP8_E5M2) {
         set_error("%s: output format %d is not FP8_E4M3 / FP8_E5M2", who, o.q_fmt);
@@ -472,4 +473,43 @@ extern "C" int fp8_grouped_linear_dgrad(const uint8_t *dY8, const uint8_t *W8, c
     return launch_gemm_2cta_grouped(dY8, W8, sdY_inv, sW_inv, group_offsets, n_groups, o, T, K, N, 1,
                                     umma_idesc_f8(FP8_E5M2, FP8_E4M3, 256, 256, 0, 1), status,
                                     static_cast<cudaStream_t>(stream));
+}
+
+// Weight gradients of the grouped product, dW[g] (+)= dY8[rows of g]^T . X8[rows of g]: one launch of the in-place
+// weight-gradient product per expert on that expert's slice of rows (the reduction runs over the slice; rows past its
+// end are zero-filled by the slice's tensor maps, so ragged groups need no padding).  The offsets are read on the host.
+extern "C" int fp8_grouped_linear_wgrad(const uint8_t *dY8, const uint8_t *X8, const float *sdY_inv, const float *sX_inv,
+                                        const int *group_offsets_host, int n_groups, void *dW, int out_is_fp32,
+                                        int accumulate, int T, int N, int K, void *stream)
+{
+    if (!group_offsets_host || !dY8 || !X8 || !dW) {
+        set_error("fp8_grouped_linear_wgrad: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if (n_groups <= 0 || n_groups > 256 || N <= 0 || K <= 0 || (N % 16) || (K % 16)) {
+        set_error("fp8_grouped_linear_wgrad: n_groups %d must be in [1, 256], N %d and K %d positive multiples of 16", n_groups,
+                  N, K);
+        return FP8_ERR_SHAPE;
+    }
+    for (int g = 0; g < n_groups; ++g) {
+        if (group_offsets_host[g] < 0 || group_offsets_host[g + 1] < group_offsets_host[g] || group_offsets_host[g + 1] > T) {
+            set_error("fp8_grouped_linear_wgrad: group_offsets must ascend from >= 0 to <= T (entry %d)", g);
+            return FP8_ERR_SHAPE;
+        }
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t elt = out_is_fp32 ? 4 : 2;
+    for (int g = 0; g < n_groups; ++g) {
+        const int r0 = group_offsets_host[g], rows = group_offsets_host[g + 1] - r0;
+        uint8_t *dw_g = static_cast<uint8_t *>(dW) + (size_t)g * N * K * elt;
+        if (rows == 0) {                      // an expert without tokens: a zero gradient
+            if (!accumulate) FP8_CUDA_CHECK(cudaMemsetAsync(dw_g, 0, (size_t)N * K * elt, st));
+            continue;
+        }
+        const GemmOut o{dw_g, out_is_fp32, accumulate, nullptr, 0, nullptr};
+        const int rc = gemm_fp8("fp8_grouped_linear_wgrad", dY8 + (size_t)r0 * N, FP8_E5M2, X8 + (size_t)r0 * K, FP8_E4M3,
+                                sdY_inv, sX_inv, o, N, K, rows, st, 1, 1);
+        if (rc != FP8_OK) return rc;
+    }
+    return FP8_OK;
 }

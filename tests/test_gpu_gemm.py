@@ -304,6 +304,39 @@ def test_grouped_data_gradient_matches_oracle_per_expert(sizes, N, K, out_dtype)
     assert err.value.status == -3
 
 
+@pytest.mark.parametrize("sizes,N,K", [([300, 0, 129, 512, 83], 528, 144), ([256, 256], 256, 256),
+                                        ([1000, 17, 2000, 1, 600, 0, 0, 350], 1024, 512), ([5], 16, 16)])
+def test_grouped_weight_gradient_matches_oracle_per_expert(sizes, N, K):
+    """dW of the mixture-of-experts product: per expert the reduction runs over its (ragged) slice of the sorted rows."""
+    E, T = len(sizes), sum(sizes)
+    Tpad = T + 9
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    dy = synth.normal_bf16((Tpad, N), 60 + E, 0, synth.GRAD_STD)
+    x = synth.normal_bf16((Tpad, K), 60 + E, 1, 1.0, synth.choose_columns(K, 2, 60, 1), 40.0)
+    dy8, _, _, _, sdy = gpu_quantize(dy, o.E5M2, False)
+    x8, _, _, _, sx = gpu_quantize(x, o.E4M3, False)
+    ody8, _, _, osdy = o.quantize(dy, o.E5M2)
+    ox8, _, _, osx = o.quantize(x, o.E4M3)
+    dw = torch.full((E, N, K), 7.0, dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_grouped_linear_wgrad(dy8, x8, sdy, sx, offs, dw)
+    acc = torch.full((E, N, K), 0.25, dtype=torch.float32, device="cuda")
+    fp8.fp8_grouped_linear_wgrad(dy8, x8, sdy, sx, offs, acc, accumulate=True)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    got, gacc = dw.float().cpu().numpy().astype(np.float64), acc.cpu().numpy().astype(np.float64)
+    for e in range(E):
+        r0, r1 = int(offs[e]), int(offs[e + 1])
+        if r1 == r0:
+            assert np.all(got[e] == 0.0) and np.all(gacc[e] == 0.25)      # no tokens: zero gradient / untouched
+            continue
+        ref, mag = o.linear_wgrad(ody8[r0:r1], ox8[r0:r1], osdy, osx)
+        assert rel_err(got[e], ref, mag) <= 2.0 ** -8, e
+        assert rel_err(gacc[e], ref + 0.25, mag + 0.25) <= TOL_FP32, e
+    with pytest.raises(fp8.Fp8Error) as err:
+        fp8.fp8_grouped_linear_wgrad(dy8, x8, sdy, sx, [0, T + 100], dw[:1])
+    assert err.value.status == -3
+
+
 def test_grouped_forward_argument_validation():
     x8 = torch.zeros((32, 32), dtype=torch.uint8, device="cuda")
     w8 = torch.zeros((2, 16, 32), dtype=torch.uint8, device="cuda")
