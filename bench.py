@@ -252,6 +252,27 @@ def run_ours(args, cfg):
     flops_step = hp.gemm_flops() + hp.attention_flops()
     value = job_tflops(world, flops_step, args.steps, ms_total)
 
+    graph_info = None
+    if args.graph:
+        # the same step submitted once per iteration: what is left of the step time when launch overhead is gone
+        g = hp.capture_graph()
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(args.steps):
+            g.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        barrier()
+        g_ms = max_over_ranks(g0.elapsed_time(g1), world, dev)
+        if fp8.fp8_device_status() != 0:
+            raise SystemExit("device status: a bounded wait expired inside a kernel (graph replay)")
+        graph_info = {"ms_per_step": g_ms / args.steps, "value": job_tflops(world, flops_step, args.steps, g_ms),
+                      "unit": UNIT}
+
     # ---- dominant kernel: the FP8 GEMM; duration from the events recorded around each launch
     gemm_ms = sum(a.elapsed_time(b) for evs in hp.gemm_events for a, b in evs)
     n_gemm = sum(len(evs) for evs in hp.gemm_events)
@@ -329,6 +350,8 @@ def run_ours(args, cfg):
                           "attention_tflop_per_step": hp.attention_flops() / 1e12,
                           "quantize_gb_per_step": hp.quantize_bytes() / 1e9},
         }
+        if graph_info is not None:
+            line["graph"] = graph_info
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -524,6 +547,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c4", choices=["c1", "c3", "c4", "c5"])
     ap.add_argument("--report", action="store_true", help="time every kernel of the library alone and print a table")
+    ap.add_argument("--graph", action="store_true",
+                    help="also time the step replayed from a CUDA graph (extra key \"graph\"; the contract keys stay eager)")
     args = ap.parse_args()
     if args.report:
         return run_report(args)

@@ -283,6 +283,21 @@ class BlockHotPath:
         fp8.fp8_scale(a["ds_amax"], fp8.E5M2, 0, a["ds_scale"], tmp_scale_inv)
         torch.cuda.synchronize(self.device)
 
+    def capture_graph(self):
+        """Captures one step (the same 48 launches) into a CUDA graph and returns it; ``graph.replay()`` then runs the
+        step with one submission.  The step makes no host synchronisation, so it is capturable as it is.  Worth it
+        where the step is launch-bound (small configurations); the large ones are bound by the kernels."""
+        side = torch.cuda.Stream(self.device)
+        side.wait_stream(torch.cuda.current_stream(self.device))
+        with torch.cuda.stream(side):
+            self.step()                       # every lazy initialisation happens outside the capture
+        torch.cuda.current_stream(self.device).wait_stream(side)
+        torch.cuda.synchronize(self.device)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.step()
+        return graph
+
     def step(self, time_gemms: bool = False):
         ev = []
 

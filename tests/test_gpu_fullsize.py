@@ -187,6 +187,27 @@ def test_host_to_host_step_equals_device_step():
         assert torch.equal(hout[n].view(torch.uint8), t.cpu().view(torch.uint8)), n
 
 
+def test_graph_replay_of_the_step_equals_the_step():
+    """The step makes no host synchronisation: captured into a CUDA graph and replayed it returns the same bits."""
+    cfg = synth.CONFIGS["c1"]
+    hp = BlockHotPath(cfg, "cuda")
+    hp.generate_host_inputs()
+    hp.allocate()
+    hp.calibrate_ds_scale()
+    hp.step()
+    torch.cuda.synchronize()
+    ref = {n: t.clone() for n, t in hp.output_tensors()}
+    g = hp.capture_graph()
+    for _, t in hp.output_tensors():
+        t.zero_()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    for n, t in hp.output_tensors():
+        assert torch.equal(t.view(torch.uint8), ref[n].view(torch.uint8)), n
+
+
 def test_glue_and_producer_forms_at_c4_sizes():
     """The (f)-row entry points at the 8B-class block's sizes, in the launch configurations bench.py --report times."""
     from gpu_util import dev, scalar
