@@ -107,6 +107,13 @@ def test_argument_validation_returns_errors_not_faults():
     with pytest.raises(fp8.Fp8Error) as e:
         fp8.fp8_cast(x.view(torch.int16).flatten()[1:].view(torch.bfloat16), scalar(1.0), 0, out)
     assert e.value.status == -2
+    # empty inputs are refused, not launched
+    empty = torch.empty(0, dtype=torch.bfloat16, device="cuda")
+    for call in (lambda: fp8.fp8_amax(empty, scalar(0.0)),
+                 lambda: fp8.fp8_cast(empty, scalar(1.0), 0, torch.empty(0, dtype=torch.uint8, device="cuda"))):
+        with pytest.raises(fp8.Fp8Error) as e:
+            call()
+        assert e.value.status in (-1, -3)       # an empty torch tensor has a null data pointer
     assert fp8.fp8_device_status() == 0
 
 
