@@ -80,9 +80,12 @@ class BlockHotPath:
     KERNELS_PER_ATTN_BWD = 3    # prep, main, finish
 
     def __init__(self, cfg: synth.BlockConfig, device="cuda", with_linears=None, with_attention=True,
-                 seq=None, batch=None, transposed_copies=False):
+                 seq=None, batch=None, transposed_copies=False, attn_max_slack=0.0):
         # transposed_copies: also write [cols, rows] FP8 copies in the cast and run dgrad / wgrad on them (the
         # form a K-major-only tensor core needs); off by default, tcgen05 reads the operands in place
+        # attn_max_slack: tau of the attention forward's reference maximum (0 = exact running maximum); P~ is then
+        # scaled by 448 / 2^tau
+        self.attn_max_slack = float(attn_max_slack)
         self.cfg = cfg
         self.device = torch.device(device)
         self.transposed_copies = transposed_copies
@@ -235,7 +238,8 @@ class BlockHotPath:
         for n in ("q", "k", "v", "do"):
             a[n].quantize()
         fp8.fp8_attention_fwd(a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv, a["v"].scale_inv,
-                              a["softmax_scale"], True, a["o"], a["lse"], None)
+                              a["softmax_scale"], True, a["o"], a["lse"], None,
+                              p_scale=448.0 / 2.0 ** self.attn_max_slack, max_slack=self.attn_max_slack)
         fp8.fp8_attention_bwd(a["q"].q, a["k"].q, a["v"].q, a["do"].q, a["o"], a["lse"], a["q"].scale_inv,
                               a["k"].scale_inv, a["v"].scale_inv, a["do"].scale_inv, a["softmax_scale"],
                               a["ds_scale"], True, a["dq"], a["dk"], a["dv"], a["ws"], ds_amax=a["ds_amax"])
@@ -327,7 +331,8 @@ class BlockHotPath:
             for n in ("q", "k", "v", "do"):
                 a[n].quantize()
             fp8.fp8_attention_fwd(a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv, a["v"].scale_inv,
-                                  a["softmax_scale"], True, a["o"], a["lse"], None)
+                                  a["softmax_scale"], True, a["o"], a["lse"], None,
+                                  p_scale=448.0 / 2.0 ** self.attn_max_slack, max_slack=self.attn_max_slack)
             fp8.fp8_attention_bwd(a["q"].q, a["k"].q, a["v"].q, a["do"].q, a["o"], a["lse"], a["q"].scale_inv,
                                   a["k"].scale_inv, a["v"].scale_inv, a["do"].scale_inv, a["softmax_scale"],
                                   a["ds_scale"], True, a["dq"], a["dk"], a["dv"], a["ws"], ds_amax=a["ds_amax"])
