@@ -464,6 +464,12 @@ def run_report(args):
             yb, dxb, dwb = (torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in ((Tt, N), (Tt, K), (N, K)))
             fl = 2.0 * Tt * N * K
             add("fp8_linear_fwd", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_fwd(x8, w8, s1, s2, yb)), flops=fl)
+            try:        # context only: the library's FP8 product on the same operands (a cuBLASLt call through torch)
+                xf, wf = x8.view(torch.float8_e4m3fn), w8.view(torch.float8_e4m3fn)
+                add("library FP8 GEMM, torch._scaled_mm (context)", f"{cname} {layer} {Tt}x{N}x{K}",
+                    timed(lambda: torch._scaled_mm(xf, wf.t(), scale_a=s1, scale_b=s2, out_dtype=torch.bfloat16)), flops=fl)
+            except Exception:
+                pass
             add("fp8_linear_dgrad", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_dgrad(dy8, w8t, s1, s2, dxb)), flops=fl)
             add("fp8_linear_wgrad", f"{cname} {layer} {Tt}x{N}x{K}", timed(lambda: fp8.fp8_linear_wgrad(dy8t, x8t, s1, s2, dwb)), flops=fl)
             add("fp8_linear_dgrad_rm (W8 read in place)", f"{cname} {layer} {Tt}x{N}x{K}",
