@@ -150,64 +150,64 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const WaitCtx ctx{p.status, abort_flag};
 
     if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(A_REGS_CTRL));
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (elect_one()) {
-            mbar_expect_tx(q_full, L::Q_BYTES);
-            tma_load_3d(sbase + L::Q_OFF, &tm_q, q_full, h * D, q0, b);
-            for (int j = 0; j < n_kv; ++j) {
-                const int st = j % A_KV_STAGES;
-                const uint32_t ph = (uint32_t)(j / A_KV_STAGES) & 1u;
-                if (!mbar_wait(kv_empty(st), ph ^ 1u, ctx)) break;
-                const uint32_t sk = sbase + L::KV_OFF + st * L::STAGE_BYTES, sv = sk + L::KV_BYTES;
-                mbar_expect_tx(kv_full(st), L::STAGE_BYTES);
-                tma_load_3d(sk, &tm_k, kv_full(st), g * D, j * A_BN, b);
-                tma_load_3d(sv, &tm_v, kv_full(st), g * D, j * A_BN, b);
-            }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (elect_one()) {
-            constexpr uint32_t idesc_s = umma_idesc_f8(0, 0, A_BM, A_BN, 0, 0);
-            constexpr uint32_t idesc_o = umma_idesc_f8(0, 0, A_BM, D, 0, 1);      // V is MN-major
-            const uint64_t dq = umma_desc(sbase + L::Q_OFF, D, 16);
-            const uint64_t dp = umma_desc(sbase + L::P_OFF, 128, 16);
-            bool ok = mbar_wait(q_full, 0, ctx);
-            // S = Q K_j^T: reduction over d in steps of 32 bytes inside the swizzle span
-            auto issue_s = [&](int j) -> bool {
-                const int st = j % A_KV_STAGES;
-                const uint32_t ph = (uint32_t)(j / A_KV_STAGES) & 1u;
-                if (!mbar_wait(kv_full(st), ph, ctx)) return false;
-                tc_fence_after();
-                const uint64_t dk = umma_desc(sbase + L::KV_OFF + st * L::STAGE_BYTES, D, 16);
-#pragma unroll
-                for (int k = 0; k < D / 32; ++k) umma_f8_ss(tmem_s, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
-                umma_commit(s_full);
-                return true;
-            };
-            if (ok) ok = issue_s(0);
-            for (int j = 0; j < n_kv && ok; ++j) {
-                const int st = j % A_KV_STAGES;
-                // the threads hold S_j in registers: the S columns are free, so S_{j+1} runs under the softmax of block j
-                if (j + 1 < n_kv) {
-                    if (!mbar_wait(s_free, (uint32_t)j & 1u, ctx)) { ok = false; break; }
-                    tc_fence_after();
-                    if (!issue_s(j + 1)) { ok = false; break; }
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(A_REGS_CTRL));
+        if (warp == 0) {
+            // ------------------------------------------------------------ TMA producer
+            if (elect_one()) {
+                mbar_expect_tx(q_full, L::Q_BYTES);
+                tma_load_3d(sbase + L::Q_OFF, &tm_q, q_full, h * D, q0, b);
+                for (int j = 0; j < n_kv; ++j) {
+                    const int st = j % A_KV_STAGES;
+                    const uint32_t ph = (uint32_t)(j / A_KV_STAGES) & 1u;
+                    if (!mbar_wait(kv_empty(st), ph ^ 1u, ctx)) break;
+                    const uint32_t sk = sbase + L::KV_OFF + st * L::STAGE_BYTES, sv = sk + L::KV_BYTES;
+                    mbar_expect_tx(kv_full(st), L::STAGE_BYTES);
+                    tma_load_3d(sk, &tm_k, kv_full(st), g * D, j * A_BN, b);
+                    tma_load_3d(sv, &tm_v, kv_full(st), g * D, j * A_BN, b);
                 }
-                // P8_j is in shared memory
-                if (!mbar_wait(p_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
-                tc_fence_after();
-                // O += P V: reduction over 128 keys in steps of 32; V advances 32 rows (32*D bytes) per step
-                const uint64_t dv = umma_desc(sbase + L::KV_OFF + st * L::STAGE_BYTES + L::KV_BYTES, D, 16);
+            }
+        } else if (warp == 1) {
+            // ------------------------------------------------------------ MMA issuer
+            if (elect_one()) {
+                constexpr uint32_t idesc_s = umma_idesc_f8(0, 0, A_BM, A_BN, 0, 0);
+                constexpr uint32_t idesc_o = umma_idesc_f8(0, 0, A_BM, D, 0, 1);      // V is MN-major
+                const uint64_t dq = umma_desc(sbase + L::Q_OFF, D, 16);
+                const uint64_t dp = umma_desc(sbase + L::P_OFF, 128, 16);
+                bool ok = mbar_wait(q_full, 0, ctx);
+                // S = Q K_j^T: reduction over d in steps of 32 bytes inside the swizzle span
+                auto issue_s = [&](int j) -> bool {
+                    const int st = j % A_KV_STAGES;
+                    const uint32_t ph = (uint32_t)(j / A_KV_STAGES) & 1u;
+                    if (!mbar_wait(kv_full(st), ph, ctx)) return false;
+                    tc_fence_after();
+                    const uint64_t dk = umma_desc(sbase + L::KV_OFF + st * L::STAGE_BYTES, D, 16);
 #pragma unroll
-                for (int k = 0; k < A_BN / 32; ++k)
-                    umma_f8_ss(tmem_o, dp + 2u * k, dv + (uint32_t)((32 * D) >> 4) * k, idesc_o, (j | k) != 0);
-                umma_commit(kv_empty(st));
-                umma_commit(pv_done);
+                    for (int k = 0; k < D / 32; ++k) umma_f8_ss(tmem_s, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
+                    umma_commit(s_full);
+                    return true;
+                };
+                if (ok) ok = issue_s(0);
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    const int st = j % A_KV_STAGES;
+                    // the threads hold S_j in registers: the S columns are free, so S_{j+1} runs under the softmax of block j
+                    if (j + 1 < n_kv) {
+                        if (!mbar_wait(s_free, (uint32_t)j & 1u, ctx)) { ok = false; break; }
+                        tc_fence_after();
+                        if (!issue_s(j + 1)) { ok = false; break; }
+                    }
+                    // P8_j is in shared memory
+                    if (!mbar_wait(p_full, (uint32_t)j & 1u, ctx)) { ok = false; break; }
+                    tc_fence_after();
+                    // O += P V: reduction over 128 keys in steps of 32; V advances 32 rows (32*D bytes) per step
+                    const uint64_t dv = umma_desc(sbase + L::KV_OFF + st * L::STAGE_BYTES + L::KV_BYTES, D, 16);
+#pragma unroll
+                    for (int k = 0; k < A_BN / 32; ++k)
+                        umma_f8_ss(tmem_o, dp + 2u * k, dv + (uint32_t)((32 * D) >> 4) * k, idesc_o, (j | k) != 0);
+                    umma_commit(kv_empty(st));
+                    umma_commit(pv_done);
+                }
             }
         }
-    }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(A_REGS_SOFTMAX));
         // ------------------------------------------------------------ softmax / correction / epilogue
