@@ -338,7 +338,8 @@ def attention_bwd(q, k, v, do, O, LSE, p: AttnParams, kv_heads=None, q_rows=None
     """Gradients for the (batch, kv head) pairs given, over query rows x key rows.
 
     O: [B,N,Hq,d] float64 (the values handed to the backward, e.g. BF16-rounded), LSE: [B,Hq,N] float64.
-    Returns dict with dQ[pair,G,nq,d], dK/dV[pair,nk,d], mag_* (error-metric denominators), slack_* (how far
+    Returns dict with dQ[pair,G,nq,d], dK/dV[pair,nk,d], mag_* (error-metric denominators; for code operands also
+    mag8_dQ / mag8_dK, the sums over the quantised |dS8|), slack_* (how far
     each output may move through FP32-vs-double tie decisions of the two encodes; zero unless p.flip_eps > 0)
     and amax_dS."""
     dt = np.float64 if real else np.uint8
@@ -358,12 +359,27 @@ def attention_bwd(q, k, v, do, O, LSE, p: AttnParams, kv_heads=None, q_rows=None
         out["mag_" + key] = np.empty_like(out[key])
         out["slack_" + key] = np.zeros_like(out[key])
     am = C.c_double()
-    f = _L().oracle_attention_bwd_real if real else _L().oracle_attention_bwd
+    args = [_p(q), _p(k), _p(v), _p(do), _p(O), _p(LSE), C.byref(p), _p(bg), C.c_int(n),
+            C.c_int(q0), C.c_int(q1), C.c_int(k0), C.c_int(k1),
+            _p(out["dQ"]), _p(out["dK"]), _p(out["dV"]),
+            _p(out["mag_dQ"]), _p(out["mag_dK"]), _p(out["mag_dV"]), C.byref(am),
+            _p(out["slack_dQ"]), _p(out["slack_dK"]), _p(out["slack_dV"])]
+    if real:
+        f = _L().oracle_attention_bwd_real
+    else:
+        # also the denominators built from the quantised dS8 (sum of |dS8|/ds_scale |K| resp. |Q|)
+        out["mag8_dQ"] = np.empty_like(out["dQ"])
+        out["mag8_dK"] = np.empty_like(out["dK"])
+        args += [_p(out["mag8_dQ"]), _p(out["mag8_dK"])]
+        f = _L().oracle_attention_bwd_mag8
     f.restype = None
-    f(_p(q), _p(k), _p(v), _p(do), _p(O), _p(LSE), C.byref(p), _p(bg), C.c_int(n),
-      C.c_int(q0), C.c_int(q1), C.c_int(k0), C.c_int(k1),
-      _p(out["dQ"]), _p(out["dK"]), _p(out["dV"]),
-      _p(out["mag_dQ"]), _p(out["mag_dK"]), _p(out["mag_dV"]), C.byref(am),
-      _p(out["slack_dQ"]), _p(out["slack_dK"]), _p(out["slack_dV"]))
+    f(*args)
     out["amax_dS"] = am.value
     return out
+
+
+def flip_step(y: float, band: float, fmt: int) -> float:
+    """Distance between the two candidate FP8 values when y lies within `band` of a rounding midpoint, else 0."""
+    f = _L().oracle_flip_step
+    f.restype = C.c_double
+    return float(f(C.c_double(y), C.c_double(band), C.c_int(fmt)))

@@ -15,10 +15,11 @@
  * Where the paper is silent (rounding mode, saturation, where FP8 enters inside attention, the backward
  * pass) the reading taken is written at the function.
  *
- * Parity status: codec, amax, scale, cast, GEMM, attention forward and the un-quantised attention
- * backward are pinned by tests (tables, worked values, brute force, closed forms, finite differences).
+ * Parity status: codec, amax, scale, cast, GEMM, attention forward and backward (un-quantised: finite
+ * differences; quantised: rebuilt step by step in numpy with two query heads per key/value head and a
+ * saturating dS scale) and the tie-band rule (hand-worked values) are pinned by tests.
  * The *placement* of the two FP8 encodes inside the attention backward is our reading of "FP8 in forward
- * and backward"; no published value exists for it: "parity unpinned" for that placement only.
+ * and backward"; the paper prints no value for it, so that placement stays a reading; its arithmetic is pinned.
  */
 #include <float.h>
 #include <math.h>
@@ -592,7 +593,8 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
                                const int32_t *bg, int nbg, int q0, int q1, int k0, int k1,
                                double *dQ, double *dK, double *dV,
                                double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS,
-                               double *slack_dQ, double *slack_dK, double *slack_dV)
+                               double *slack_dQ, double *slack_dK, double *slack_dV,
+                               double *mag8_dQ, double *mag8_dK)
 {
     const int d = p->d, G = p->Hq / p->Hkv, nq = q1 - q0, nk = k1 - k0;
     const double cP = p->quant ? p->c_P : 1.0;
@@ -626,7 +628,13 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
             double *out = dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d;
             double *mout = mag_dQ ? mag_dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d : NULL;
             double *sout = want_slack ? slack_dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d : NULL;
-            for (int dd = 0; dd < d; ++dd) { out[dd] = 0.0; if (mout) mout[dd] = 0.0; if (sout) sout[dd] = 0.0; }
+            double *m8out = mag8_dQ ? mag8_dQ + (((int64_t)pi * G + hg) * nq + (i - q0)) * d : NULL;
+            for (int dd = 0; dd < d; ++dd) {
+                out[dd] = 0.0;
+                if (mout) mout[dd] = 0.0;
+                if (sout) sout[dd] = 0.0;
+                if (m8out) m8out[dd] = 0.0;
+            }
             for (int j = k0; j < k1; ++j) {
                 if (p->causal && j > i) break;
                 double P = exp(score(p, Q, K, b, h, g, i, j) - lse);
@@ -657,6 +665,7 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
                     out[dd] += p->s * p->k_inv * u * kv;
                     if (mout) mout[dd] += p->s * p->k_inv * m_ds * fabs(kv);
                     if (sout) sout[dd] += p->s * p->k_inv * step * fabs(kv);
+                    if (m8out) m8out[dd] += p->s * p->k_inv * fabs(u) * fabs(kv);
                 }
             }
         }
@@ -672,8 +681,10 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
             double *mV = mag_dV ? mag_dV + ((int64_t)pi * nk + (j - k0)) * d : NULL;
             double *sK = want_slack ? slack_dK + ((int64_t)pi * nk + (j - k0)) * d : NULL;
             double *sV = want_slack ? slack_dV + ((int64_t)pi * nk + (j - k0)) * d : NULL;
+            double *m8K = mag8_dK ? mag8_dK + ((int64_t)pi * nk + (j - k0)) * d : NULL;
             for (int dd = 0; dd < d; ++dd) {
                 oK[dd] = 0.0; oV[dd] = 0.0;
+                if (m8K) m8K[dd] = 0.0;
                 if (mK) mK[dd] = 0.0;
                 if (mV) mV[dd] = 0.0;
                 if (sK) { sK[dd] = 0.0; sV[dd] = 0.0; }
@@ -715,6 +726,7 @@ static void attention_bwd_core(const operand *Q, const operand *K, const operand
                         oK[dd] += p->s * p->q_inv * u * qv;
                         if (mV) mV[dd] += p->do_inv * w * fabs(dov);
                         if (mK) mK[dd] += p->s * p->q_inv * m_ds * fabs(qv);
+                        if (m8K) m8K[dd] += p->s * p->q_inv * fabs(u) * fabs(qv);
                         if (sK) {
                             sK[dd] += p->s * p->q_inv * stepS * fabs(qv);
                             sV[dd] += p->do_inv * stepP * fabs(dov);
@@ -741,7 +753,7 @@ void oracle_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V
     operand_init(&V, V8, NULL, ORACLE_E4M3);
     operand_init(&dO, dO8, NULL, ORACLE_E5M2);
     attention_bwd_core(&Q, &K, &V, &dO, O, LSE, p, bg, nbg, q0, q1, k0, k1,
-                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS, slack_dQ, slack_dK, slack_dV);
+                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS, slack_dQ, slack_dK, slack_dV, NULL, NULL);
 }
 
 void oracle_attention_bwd_real(const double *Qd, const double *Kd, const double *Vd, const double *dOd,
@@ -757,8 +769,31 @@ void oracle_attention_bwd_real(const double *Qd, const double *Kd, const double 
     operand_init(&V, NULL, Vd, ORACLE_E4M3);
     operand_init(&dO, NULL, dOd, ORACLE_E5M2);
     attention_bwd_core(&Q, &K, &V, &dO, O, LSE, p, bg, nbg, q0, q1, k0, k1,
-                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS, slack_dQ, slack_dK, slack_dV);
+                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS, slack_dQ, slack_dK, slack_dV, NULL, NULL);
 }
+
+/* oracle_attention_bwd plus two more error-metric denominators: the sums of |dS8|/ds_scale * |K| (for dQ) and
+ * |dS8|/ds_scale * |Q| (for dK), i.e. the magnitude of the product as the FP8 GEMM sees it, after dP - D has
+ * cancelled.  Smaller than mag_dQ / mag_dK wherever the softmax row is nearly one-hot. */
+void oracle_attention_bwd_mag8(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const uint8_t *dO8,
+                               const double *O, const double *LSE, const oracle_attn_params *p,
+                               const int32_t *bg, int nbg, int q0, int q1, int k0, int k1,
+                               double *dQ, double *dK, double *dV,
+                               double *mag_dQ, double *mag_dK, double *mag_dV, double *amax_dS,
+                               double *slack_dQ, double *slack_dK, double *slack_dV,
+                               double *mag8_dQ, double *mag8_dK)
+{
+    operand Q, K, V, dO;
+    operand_init(&Q, Q8, NULL, ORACLE_E4M3);
+    operand_init(&K, K8, NULL, ORACLE_E4M3);
+    operand_init(&V, V8, NULL, ORACLE_E4M3);
+    operand_init(&dO, dO8, NULL, ORACLE_E5M2);
+    attention_bwd_core(&Q, &K, &V, &dO, O, LSE, p, bg, nbg, q0, q1, k0, k1,
+                       dQ, dK, dV, mag_dQ, mag_dK, mag_dV, amax_dS, slack_dQ, slack_dK, slack_dV, mag8_dQ, mag8_dK);
+}
+
+/* The tie-band rule on its own, so that tests can pin it on hand-worked values. */
+double oracle_flip_step(double y, double band, int fmt) { return flip_step(y, band, fmt); }
 
 int oracle_num_threads(void)
 {

@@ -283,3 +283,158 @@ def test_tie_slack_outputs():
     p = o.attn_params(B, N, H, H, d, quant=True, flip_eps=1e-6)
     _, _, _, slack = o.attention_fwd(np.zeros_like(q), k, v, p, with_slack=True)
     assert slack.sum() == 0.0
+
+
+def _stepwise_quantised_backward(q, k, v, do, O, LSE, s, q_inv, k_inv, v_inv, do_inv, ds_scale, causal, cP=448.0):
+    """The quantised backward rebuilt in numpy, one (batch, head) at a time, in the order of the definition:
+    P = exp(x - LSE); P8 = E4M3(fl32(P) fl32(c_P)); dV += P8^T dO / c_P; dP = dO V^T; D = rowsum(dO * O);
+    dS = P (dP - D); dS8 = E5M2(fl32(dS) fl32(ds_scale)); dQ = s dS8 K / ds_scale; dK += s dS8^T Q / ds_scale."""
+    B, N, Hq, d = q.shape
+    Hkv = k.shape[2]
+    G = Hq // Hkv
+    Qc, Kc, Vc, dOc = dec(q), dec(k), dec(v), dec(do, o.E5M2)
+    dQ = np.zeros((B, Hq, N, d))
+    dK = np.zeros((B, Hkv, N, d))
+    dV = np.zeros((B, Hkv, N, d))
+    m8Q = np.zeros_like(dQ)
+    m8K = np.zeros_like(dK)
+    amax, nsat = 0.0, 0
+    mask = np.tril(np.ones((N, N), dtype=bool)) if causal else np.ones((N, N), dtype=bool)
+    for b in range(B):
+        for h in range(Hq):
+            g = h // G
+            x = s * q_inv * k_inv * (Qc[b, :, h] @ Kc[b, :, g].T)
+            P = np.where(mask, np.exp(x - LSE[b, h][:, None]), 0.0)
+            P8 = dec(o.encode_array(P.astype(np.float32) * np.float32(cP), o.E4M3))
+            dOr = do_inv * dOc[b, :, h]
+            D = (dOr * O[b, :, h]).sum(axis=1)
+            dV[b, g] += P8.T @ dOr / cP
+            dP = do_inv * v_inv * (dOc[b, :, h] @ Vc[b, :, g].T)
+            dS = np.where(mask, P * (dP - D[:, None]), 0.0)
+            amax = max(amax, np.abs(dS).max())
+            prod = dS.astype(np.float32) * np.float32(ds_scale)
+            nsat += int((np.abs(prod) > 57344.0).sum())
+            dS8 = dec(o.encode_array(prod, o.E5M2), o.E5M2) / ds_scale
+            dQ[b, h] = s * k_inv * (dS8 @ Kc[b, :, g])
+            dK[b, g] += s * q_inv * (dS8.T @ Qc[b, :, h])
+            m8Q[b, h] = s * k_inv * (np.abs(dS8) @ np.abs(Kc[b, :, g]))
+            m8K[b, g] += s * q_inv * (np.abs(dS8).T @ np.abs(Qc[b, :, h]))
+    return dQ, dK, dV, m8Q, m8K, amax, nsat
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("ds_scale,expect_saturation", [(2048.0, False), (3.0e7, True)])
+def test_quantised_backward_matches_stepwise_definition(causal, ds_scale, expect_saturation):
+    """quant=on differs from the textbook gradient only by the two encodes, placed where a product's operand is
+    formed: P8 feeds dV, dS8 feeds dQ and dK.  Two query heads per key/value head, so the group sum is covered;
+    the large ds_scale pushes dS * ds_scale past 57344, where the cast saturates."""
+    B, N, Hq, Hkv, d = 2, 10, 4, 2, 8
+    q, k, v = rand_codes((B, N, Hq, d), 70), rand_codes((B, N, Hkv, d), 71), rand_codes((B, N, Hkv, d), 72)
+    do = rand_codes((B, N, Hq, d), 73, 0x10, 0x30)           # read as E5M2 codes
+    kw = dict(s=0.35, q_inv=0.5, k_inv=1.5, v_inv=0.25, do_inv=0.125)
+    p = o.attn_params(B, N, Hq, Hkv, d, causal=causal, quant=True, ds_scale=ds_scale, **kw)
+    # O and LSE are inputs of the backward: LSE is the log-sum-exp of the scores, O any tensor (here the textbook one)
+    Qr, Kr, Vr = dec(q) * 0.5, dec(k) * 1.5, dec(v) * 0.25
+    O = np.empty((B, N, Hq, d))
+    LSE = np.empty((B, Hq, N))
+    for b in range(B):
+        for h in range(Hq):
+            g = h // (Hq // Hkv)
+            P, O[b, :, h] = softmax_reference(Qr[b, :, h], Kr[b, :, g], Vr[b, :, g], 0.35, causal)
+            x = 0.35 * Qr[b, :, h] @ Kr[b, :, g].T
+            if causal:
+                x = np.where(np.tril(np.ones_like(x, dtype=bool)), x, -np.inf)
+            LSE[b, h] = np.log(np.exp(x).sum(axis=1))
+    g_ = o.attention_bwd(q, k, v, do, O, LSE, p)
+    dQ, dK, dV, m8Q, m8K, amax, nsat = _stepwise_quantised_backward(q, k, v, do, O, LSE, ds_scale=ds_scale,
+                                                                    causal=causal, **kw)
+    assert (nsat > 0) == expect_saturation
+    G = Hq // Hkv
+    got_dQ = g_["dQ"].reshape(B, Hkv, G, N, d).reshape(B, Hq, N, d)
+    assert np.allclose(got_dQ, dQ, rtol=1e-11, atol=1e-300)
+    assert np.allclose(g_["dK"].reshape(B, Hkv, N, d), dK, rtol=1e-11, atol=1e-300)
+    assert np.allclose(g_["dV"].reshape(B, Hkv, N, d), dV, rtol=1e-11, atol=1e-300)
+    assert np.isclose(g_["amax_dS"], amax, rtol=1e-12)
+    assert np.allclose(g_["mag8_dQ"].reshape(B, Hq, N, d), m8Q, rtol=1e-11)
+    assert np.allclose(g_["mag8_dK"].reshape(B, Hkv, N, d), m8K, rtol=1e-11)
+    assert np.all(np.abs(dK).max(axis=(0, 2, 3)) > 0) and np.abs(dQ).max() > 0
+    if expect_saturation:
+        # a saturated dS8 is +-57344 / ds_scale: the result differs from the un-saturated product
+        unsat = o.attention_bwd(q, k, v, do, O, LSE, o.attn_params(B, N, Hq, Hkv, d, causal=causal, quant=False, **kw))
+        assert not np.allclose(unsat["dQ"], g_["dQ"], rtol=0.2)
+
+
+def test_quantised_backward_pin_catches_plausible_mistakes():
+    """The step-wise rebuild separates the variants a mistaken oracle could implement: dS quantised in E4M3,
+    P8 (not P) inside dS, a missing 1/ds_scale — each moves the result by far more than the pin's tolerance."""
+    B, N, H, d = 1, 10, 1, 8
+    q, k, v = rand_codes((B, N, H, d), 80), rand_codes((B, N, H, d), 81), rand_codes((B, N, H, d), 82)
+    do = rand_codes((B, N, H, d), 83, 0x10, 0x30)
+    p = o.attn_params(B, N, H, H, d, quant=True, s=0.4, ds_scale=512.0)
+    O, LSE, _ = o.attention_fwd(q, k, v, p)
+    g_ = o.attention_bwd(q, k, v, do, O.reshape(B, N, H, d), LSE.reshape(B, H, N), p)
+    Qc, Kc, Vc, dOc = dec(q)[0, :, 0], dec(k)[0, :, 0], dec(v)[0, :, 0], dec(do, o.E5M2)[0, :, 0]
+    mask = np.tril(np.ones((N, N), dtype=bool))
+    P = np.where(mask, np.exp(0.4 * Qc @ Kc.T - LSE[0][:, None]), 0.0)
+    P8 = dec(o.encode_array(P.astype(np.float32) * np.float32(448.0), o.E4M3)) / 448.0
+    D = (dOc * O[0]).sum(axis=1)
+    dP = dOc @ Vc.T
+    right = P * (dP - D[:, None])
+    variants = {
+        "e4m3": dec(o.encode_array((right * 512.0).astype(np.float32), o.E4M3)) / 512.0,
+        "p8_in_dS": dec(o.encode_array((P8 * (dP - D[:, None]) * 512.0).astype(np.float32), o.E5M2), o.E5M2) / 512.0,
+        "no_descale": dec(o.encode_array((right * 512.0).astype(np.float32), o.E5M2), o.E5M2),
+    }
+    good = dec(o.encode_array((right * 512.0).astype(np.float32), o.E5M2), o.E5M2) / 512.0
+    assert np.allclose(g_["dQ"][0, 0], 0.4 * good @ Kc, rtol=1e-11, atol=1e-300)
+    for name, ds8 in variants.items():
+        assert not np.allclose(g_["dQ"][0, 0], 0.4 * ds8 @ Kc, rtol=1e-6, atol=1e-300), name
+
+
+def test_flip_step_hand_worked_values():
+    """The tie band: a value within `band` of the midpoint between two neighbouring codes may go to either, and
+    the function returns the gap between them; anywhere else it returns 0."""
+    f = o.flip_step
+    E4, E5 = o.E4M3, o.E5M2
+    # E4M3 around 1: codes 0x38 = 1, 0x39 = 1.125, midpoint 1.0625, gap 0.125
+    assert f(1.0625, 1e-9, E4) == 0.125
+    assert f(-1.0625, 1e-9, E4) == 0.125                      # sign-symmetric
+    assert f(1.0625 + 0.004, 0.005, E4) == 0.125              # inside the band, above the midpoint (code 0x39)
+    assert f(1.0625 - 0.004, 0.005, E4) == 0.125              # inside the band, below it (code 0x38)
+    assert f(1.0625 + 0.006, 0.005, E4) == 0.0                # just outside
+    assert f(1.0625 - 0.006, 0.005, E4) == 0.0
+    assert f(1.0, 0.01, E4) == 0.0                            # on a code, far from both midpoints
+    assert f(1.0625, 0.0, E4) == 0.0                          # band 0 switches the rule off
+    # binade boundary: 1.875 | 2.0 | 2.25 — the gap differs on the two sides of 2
+    assert f(1.9375, 1e-9, E4) == 0.125
+    assert f(2.125, 1e-9, E4) == 0.25
+    # top of the range: 416 | 448, nothing above 448 (the cast saturates, so no flip there)
+    assert f(432.0, 1e-6, E4) == 32.0
+    assert f(448.0, 1.0, E4) == 0.0
+    assert f(449.0, 2.0, E4) == 0.0
+    assert f(1e4, 1.0, E4) == 0.0
+    assert f(450.0, 20.0, E4) == 32.0                         # saturated, but the band reaches down to 432
+    assert f(464.0, 20.0, E4) == 0.0                          # 32 above the midpoint: out of a band of 20
+    # subnormal range of E4M3: grid of 2^-9 up to 2^-6
+    u = 2.0 ** -9
+    assert f(0.5 * u, 1e-12, E4) == u                         # between 0 and the smallest subnormal
+    assert f(1.5 * u, 1e-12, E4) == u
+    assert f(7.5 * u, 1e-12, E4) == u                         # last subnormal | first normal
+    assert f(8.5 * u, 1e-12, E4) == u                         # first normal binade has the same spacing
+    assert f(16.5 * u, 1e-12, E4) == 0.0                      # 2^-5 binade: spacing 2u, 16.5u is not a midpoint
+    assert f(17.0 * u, 1e-12, E4) == 2 * u
+    assert f(0.0, 1e-12, E4) == 0.0
+    # E5M2: 1 | 1.25 (gap 0.25), top 49152 | 57344 (gap 8192), subnormal grid 2^-16
+    assert f(1.125, 1e-9, E5) == 0.25
+    assert f(1.125 + 0.02, 0.01, E5) == 0.0
+    assert f(53248.0, 1e-3, E5) == 8192.0
+    assert f(57344.0, 100.0, E5) == 0.0
+    assert f(1.5 * 2.0 ** -16, 1e-15, E5) == 2.0 ** -16
+    # consistency with the encoder on every pair of neighbouring finite codes
+    for fmt, top in ((E4, 0x7E), (E5, 0x7B)):
+        t = o.decode_table(fmt)
+        for c in range(top):
+            mid, gap = 0.5 * (t[c] + t[c + 1]), t[c + 1] - t[c]
+            assert f(mid, gap * 1e-6, fmt) == gap
+            assert f(mid + 0.26 * gap, 0.25 * gap, fmt) == 0.0
+            assert f(mid - 0.26 * gap, 0.25 * gap, fmt) == 0.0
