@@ -64,3 +64,40 @@ BWD_FLOOR = 1e-6
 # relative uncertainty of the kernel's FP32 evaluation of a length-128 dot product and an exp2:
 # measured tcgen05 accumulation error is 2^-22 of the magnitude sum at K = 128; 8x margin
 FLIP_EPS = 2.0 ** -19
+
+
+def quantile_err(got, ref, mag, slack=None, q=0.999, floor_frac=0.0):
+    """(q-quantile, maximum) of (|got - ref| - slack)+ / mag over all elements."""
+    den = np.maximum(mag, max(1e-30, floor_frac * float(np.mean(mag))))
+    diff = np.abs(got - ref)
+    if slack is not None:
+        diff = np.maximum(diff - slack, 0.0)
+    e = (diff / den).ravel()
+    return float(np.quantile(e, q)), float(e.max())
+
+
+def norm_ratios(got, ref):
+    """(Frobenius, max-norm) ratios ||got - ref|| / ||ref||."""
+    d = got - ref
+    return (float(np.linalg.norm(d.ravel()) / max(np.linalg.norm(ref.ravel()), 1e-300)),
+            float(np.abs(d).max() / max(np.abs(ref).max(), 1e-300)))
+
+
+def report(case: str, **metrics):
+    """Print one line of parity figures (pytest -s shows it) and, when FP8DPA_PARITY_REPORT names a file, append
+    it there as JSON so that the figures quoted in the design notes can be regenerated."""
+    import json
+    import os
+    line = json.dumps({"case": case, **{k: (float("%.4g" % v) if isinstance(v, float) else v)
+                                        for k, v in metrics.items()}})
+    print("parity:", line)
+    path = os.environ.get("FP8DPA_PARITY_REPORT")
+    if path:
+        with open(path, "a") as f:
+            f.write(line + "\n")
+
+
+# Frobenius-norm gates (||gpu - oracle||_F / ||oracle||_F).  O and the gradients are BF16 (2^-9 relative per element)
+# and inherit the re-quantisation ties of P8 / dS8 on a small share of the terms.
+FRO_FWD = 5e-3
+FRO_BWD = 5e-3

@@ -12,12 +12,13 @@ import oracle as o
 import paper_2505_20524_b200 as fp8
 from paper_2505_20524_b200 import synth
 from paper_2505_20524_b200.hotpath import BlockHotPath
-from gpu_util import dev, host, scalar, rel_err, BWD_FLOOR, FLIP_EPS
+from gpu_util import (dev, host, scalar, rel_err, quantile_err, norm_ratios, report, BWD_FLOOR, FLIP_EPS, FRO_FWD,
+                      FRO_BWD)
 
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("log2n,fmts", [(27, (o.E4M3, o.E5M2)), (29, (o.E4M3,))])
+@pytest.mark.parametrize("log2n,fmts", [(27, (o.E4M3, o.E5M2)), (29, (o.E4M3, o.E5M2))])
 def test_quantize_sweep_sizes_bit_exact(log2n, fmts):
     n = 1 << log2n
     x = synth.flat_tensor(n)
@@ -112,6 +113,9 @@ def _attention_case(name, kv_heads, head_rows):
         for n_, (b, hh) in enumerate(heads):
             e = rel_err(gO[b, rng[0]:rng[1], hh], O_[n_], mag_[n_], slack_[n_])
             assert e <= 2e-2, ("O", rng, b, hh, e)
+            fro = norm_ratios(gO[b, rng[0]:rng[1], hh], O_[n_])[0]
+            assert fro <= FRO_FWD, ("O", rng, b, hh, fro)
+            report("fwd %s full size rows %d:%d b%d h%d" % (name, rng[0], rng[1], b, hh), max_rel=e, fro=fro)
             assert np.max(np.abs(gL[b, hh, rng[0]:rng[1]] - lse_[n_])) <= 1e-3 * max(1.0, np.abs(lse_[n_]).max())
 
     # backward again on the oracle's O / LSE for the sampled (head, row) ranges, so both sides see equal inputs
@@ -136,13 +140,31 @@ def _attention_case(name, kv_heads, head_rows):
     gv = a["dv"].float().cpu().numpy().astype(np.float64)
     for n_, (b, g) in enumerate(kv_heads):
         for j in range(G):
-            e = rel_err(gq[b, lo[0]:lo[1], g * G + j], first["dQ"][n_, j], first["mag_dQ"][n_, j],
-                        first["slack_dQ"][n_, j], BWD_FLOOR)
+            got = gq[b, lo[0]:lo[1], g * G + j]
+            e = rel_err(got, first["dQ"][n_, j], first["mag_dQ"][n_, j], first["slack_dQ"][n_, j], BWD_FLOOR)
             assert e <= 3e-2, ("dQ", b, g, j, e)
+            q999, mx = quantile_err(got, first["dQ"][n_, j], first["mag8_dQ"][n_, j], first["slack_dQ"][n_, j],
+                                    0.999, BWD_FLOOR)
+            fro = norm_ratios(got, first["dQ"][n_, j])[0]
+            assert fro <= FRO_BWD and mx <= 3e-2, ("dQ", b, g, j, fro, mx)
+            report("bwd %s full size dQ b%d h%d" % (name, b, g * G + j), max_rel=e, mag8_q999=q999, mag8_max=mx,
+                   fro=fro)
         for nm, got in (("dK", gk), ("dV", gv)):
-            e = rel_err(got[b, hi[0]:hi[1], g], last[nm][n_], last["mag_" + nm][n_], last["slack_" + nm][n_],
-                        BWD_FLOOR)
+            gt = got[b, hi[0]:hi[1], g]
+            e = rel_err(gt, last[nm][n_], last["mag_" + nm][n_], last["slack_" + nm][n_], BWD_FLOOR)
             assert e <= 3e-2, (nm, b, g, e)
+            fro = norm_ratios(gt, last[nm][n_])[0]
+            assert fro <= FRO_BWD, (nm, b, g, fro)
+            m = dict(max_rel=e, fro=fro)
+            if nm == "dK":
+                q999, mx = quantile_err(gt, last[nm][n_], last["mag8_dK"][n_], last["slack_dK"][n_], 0.999, BWD_FLOOR)
+                assert mx <= 3e-2, (nm, b, g, mx)
+                m.update(mag8_q999=q999, mag8_max=mx)
+            report("bwd %s full size %s b%d g%d" % (name, nm, b, g), **m)
+
+
+def test_attention_1p5b_block_sampled():
+    _attention_case("c3", kv_heads=[(0, 0), (3, 15)], head_rows=256)
 
 
 def test_attention_8b_block_sampled():
