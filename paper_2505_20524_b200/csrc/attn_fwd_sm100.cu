@@ -15,6 +15,10 @@
 // Final: O = v_inv * acc / (c_P * l) as BF16, staged in the (by then free) K/V ring and written with one tiled
 // bulk store per 64 columns; LSE = ln2 * (m + log2 l).
 #include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -373,6 +377,452 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------------
+// d = 128: one CTA per SM on 256 query rows, taken as two 128-row tiles with a softmax warpgroup each.
+//
+//   warps 0-3   softmax of tile 0, warps 4-7 softmax of tile 1 (one row per thread): score row from TMEM into
+//               registers, block maximum, new reference maximum m, factor 2^(m_old - m) published to the correction
+//               warps, P~ = 2^(c S - m) (row sum from the un-rounded values), E4M3 codes of c_P P~ stored back to TMEM
+//               over the first 32 of the tile's 128 score columns.  Only a tile's last key block can need a mask
+//               (the causal diagonal, the end of the sequence); it runs through a separate instance of the block code
+//   warps 8-11  correction: multiply a tile's O accumulator in TMEM by the published factor when a row maximum
+//               grew (off the softmax threads' chain, under their exponentials); at the end normalise O by l,
+//               write BF16 (and the optional E4M3 copy) through shared memory with tiled bulk stores.  The two tiles
+//               are served in the order their events arrive
+//   warp 12     TMA: Q tiles once, K_j and V_j through two rings
+//   warps 13,14 MMA issuers of tile 0 and tile 1: S_i = Q_i K_j^T (operands in shared memory), O_i += P8_i V_j with
+//               P8 read from TMEM as the A operand and V in place as an MN-major B operand.  Per tile the order is
+//               PV_i(j), QK_i(j+1): the tensor pipe runs one thread's products in issue order, so S_i(j+1) overwrites
+//               the columns of P8_i(j) only after PV_i(j) has read them.  One issuer per tile, so that neither tile
+//               waits for the other's turn
+// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 columns each.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int P_THREADS = 512;
+constexpr int P_STAGES = 4;
+constexpr int P_REGS_SOFTMAX = 184, P_REGS_CORR = 80, P_REGS_CTRL = 64;   // 2*128*184 + 128*80 + 128*64 = 65536
+constexpr int P_TMEM_COLS = 512;
+
+struct AttnFwdPairSmem {
+    static constexpr int D = 128;
+    static constexpr int TILE_BYTES = 128 * D;                 // one Q, K or V tile
+    static constexpr int Q_OFF = 0;                            // two Q tiles
+    static constexpr int K_OFF = Q_OFF + 2 * TILE_BYTES;
+    static constexpr int V_OFF = K_OFF + P_STAGES * TILE_BYTES;
+    // output staging of tile i ([128 x 128] BF16 = two 64-column halves): its Q tile (idle by then) and OST_i
+    static constexpr int OST_OFF = V_OFF + P_STAGES * TILE_BYTES;
+    static constexpr int ALPHA_OFF = OST_OFF + 2 * TILE_BYTES; // float[2][128]: rescale factor of the current block
+    static constexpr int L_OFF = ALPHA_OFF + 2 * 128 * 4;      // float[2][128]: final row sums
+    static constexpr int BAR_OFF = L_OFF + 2 * 128 * 4;
+    // q_full[2], k_full[S], k_empty[S], v_full[S], v_empty[S], s_full[2], pv_go[2], o_final[2], alpha_ready[2][4],
+    // l_ready[2][4]
+    static constexpr int N_BARS = 2 + 4 * P_STAGES + 6 + 16;
+    static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
+    static constexpr int DYN_BYTES = TOTAL + 1024;
+};
+
+
+// D[tmem] (+)= A[tmem] * B[smem]: A = 128 rows (lanes) x 32 FP8 values in 8 consecutive 32-bit columns.
+__device__ __forceinline__ void umma_f8_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Event loop of a role that serves both tiles: gives up like the bounded waits do.
+struct IdleGuard {
+    long long t0;
+    uint32_t n;
+    __device__ __forceinline__ void reset() { n = 0; }
+    __device__ __forceinline__ bool expired(const WaitCtx &ctx)
+    {
+        if (n == 0) t0 = clock64();
+        if ((++n & 63u) != 0) return false;
+        if (*ctx.abort_flag) return true;
+        if (clock64() - t0 > (ctx.limit > 0 ? ctx.limit : FP8DPA_WAIT_LIMIT_CYCLES)) {
+            *ctx.abort_flag = 1;
+            atomicExch(ctx.status, (int)FP8_ERR_TIMEOUT);
+            return true;
+        }
+        return false;
+    }
+};
+
+__global__ void __launch_bounds__(P_THREADS, 1)
+attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                     const AttnFwdParams p)
+{
+    using L = AttnFwdPairSmem;
+    constexpr int D = 128;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::BAR_OFF;
+    auto q_full = [&](int i) { return bar0 + 8u * i; };
+    auto k_full = [&](int s) { return bar0 + 8u * (2 + s); };
+    auto k_empty = [&](int s) { return bar0 + 8u * (2 + P_STAGES + s); };
+    auto v_full = [&](int s) { return bar0 + 8u * (2 + 2 * P_STAGES + s); };
+    auto v_empty = [&](int s) { return bar0 + 8u * (2 + 3 * P_STAGES + s); };
+    constexpr int B1 = 2 + 4 * P_STAGES;
+    auto s_full = [&](int i) { return bar0 + 8u * (B1 + i); };
+    auto pv_go = [&](int i) { return bar0 + 8u * (B1 + 2 + i); };
+    auto o_final = [&](int i) { return bar0 + 8u * (B1 + 4 + i); };
+    auto alpha_ready = [&](int i, int q) { return bar0 + 8u * (B1 + 6 + i * 4 + q); };
+    auto l_ready = [&](int i, int q) { return bar0 + 8u * (B1 + 14 + i * 4 + q); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFF + L::N_BARS * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    float *alpha_s = reinterpret_cast<float *>(smem + L::ALPHA_OFF);
+    float *l_s = reinterpret_cast<float *>(smem + L::L_OFF);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // heavy (late) query tiles first: with a causal mask a later tile attends to more key blocks
+    const int q_tile = (int)gridDim.x - 1 - (int)blockIdx.x;
+    const int h = blockIdx.y, b = blockIdx.z;
+    const int g = h / (p.Hq / p.Hkv);
+    const int q0 = q_tile * 256;
+    const int n_kv_all = (p.N + A_BN - 1) / A_BN;
+    // key blocks of the two tiles (tile 1 may lie wholly past N)
+    const int n0 = p.causal ? min(n_kv_all, 2 * q_tile + 1) : n_kv_all;
+    const int n1 = (q0 + 128 < p.N) ? (p.causal ? min(n_kv_all, 2 * q_tile + 2) : n_kv_all) : 0;
+    const int nmax = max(n0, n1);
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(q_full(i), 1);
+            mbar_init(s_full(i), 1);
+            mbar_init(pv_go(i), 8);        // four softmax warps (P8 stored) + four correction warps (O rescaled)
+            mbar_init(o_final(i), 1);
+            for (int q = 0; q < 4; ++q) {
+                mbar_init(alpha_ready(i, q), 1);
+                mbar_init(l_ready(i, q), 1);
+            }
+        }
+        for (int s = 0; s < P_STAGES; ++s) {
+            mbar_init(k_full(s), 1);
+            mbar_init(k_empty(s), n1 > 0 ? 2 : 1);     // one release per active tile
+            mbar_init(v_full(s), 1);
+            mbar_init(v_empty(s), n1 > 0 ? 2 : 1);
+        }
+        *abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_o);
+    }
+    if (warp == 13) {
+        tmem_alloc(smem_u32(tmem_slot), P_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const WaitCtx ctx{p.status, abort_flag};
+
+    if (warp >= 12) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(P_REGS_CTRL));
+        if (warp == 12) {
+            // ------------------------------------------------------------ TMA producer
+            if (elect_one()) {
+                mbar_expect_tx(q_full(0), L::TILE_BYTES);
+                tma_load_3d(sbase + L::Q_OFF, &tm_q, q_full(0), h * D, q0, b);
+                if (n1 > 0) {
+                    mbar_expect_tx(q_full(1), L::TILE_BYTES);
+                    tma_load_3d(sbase + L::Q_OFF + L::TILE_BYTES, &tm_q, q_full(1), h * D, q0 + 128, b);
+                }
+                for (int j = 0; j < nmax; ++j) {
+                    const int st = j % P_STAGES;
+                    const uint32_t ph = (uint32_t)(j / P_STAGES) & 1u;
+                    if (!mbar_wait_relaxed(k_empty(st), ph ^ 1u, ctx)) break;
+                    mbar_expect_tx(k_full(st), L::TILE_BYTES);
+                    tma_load_3d(sbase + L::K_OFF + st * L::TILE_BYTES, &tm_k, k_full(st), g * D, j * A_BN, b);
+                    if (!mbar_wait_relaxed(v_empty(st), ph ^ 1u, ctx)) break;
+                    mbar_expect_tx(v_full(st), L::TILE_BYTES);
+                    tma_load_3d(sbase + L::V_OFF + st * L::TILE_BYTES, &tm_v, v_full(st), g * D, j * A_BN, b);
+                }
+            }
+        } else if (warp == 13 || warp == 14) {
+            // ------------------------------------------------------------ MMA issuer of tile i
+            const int i = warp - 13;
+            const int n_kv = i ? n1 : n0;
+            if (n_kv > 0 && elect_one()) {
+                constexpr uint32_t idesc_s = umma_idesc_f8(0, 0, 128, A_BN, 0, 0);
+                constexpr uint32_t idesc_o = umma_idesc_f8(0, 0, 128, D, 0, 1);       // V is MN-major
+                const uint64_t dq = umma_desc(sbase + L::Q_OFF + i * L::TILE_BYTES, D, 16);
+                const uint32_t ts = tmem_base + (uint32_t)(i * 128), to = tmem_base + 256u + (uint32_t)(i * 128);
+                auto issue_qk = [&](int j) {
+                    const uint64_t dk = umma_desc(sbase + L::K_OFF + (j % P_STAGES) * L::TILE_BYTES, D, 16);
+#pragma unroll
+                    for (int k = 0; k < D / 32; ++k) umma_f8_ss(ts, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
+                    umma_commit(s_full(i));
+                    umma_commit(k_empty(j % P_STAGES));
+                };
+                bool ok = mbar_wait(q_full(i), 0, ctx) && mbar_wait(k_full(0), 0, ctx);
+                if (ok) {
+                    tc_fence_after();
+                    issue_qk(0);
+                }
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    const int st = j % P_STAGES;
+                    // V_j and K_{j+1} land long before P8_i(j): take those waits off the chain
+                    if (!mbar_wait(v_full(st), (uint32_t)(j / P_STAGES) & 1u, ctx)) { ok = false; break; }
+                    if (j + 1 < n_kv &&
+                        !mbar_wait(k_full((j + 1) % P_STAGES), (uint32_t)((j + 1) / P_STAGES) & 1u, ctx)) {
+                        ok = false;
+                        break;
+                    }
+                    // P8_i(j) is in TMEM and O_i carries the new reference maximum
+                    if (!mbar_wait(pv_go(i), (uint32_t)j & 1u, ctx)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t dv = umma_desc(sbase + L::V_OFF + st * L::TILE_BYTES, D, 16);
+#pragma unroll
+                    for (int k = 0; k < A_BN / 32; ++k)
+                        umma_f8_ts(to, ts + 8u * k, dv + (uint32_t)((32 * D) >> 4) * k, idesc_o, (j | k) != 0);
+                    if (j == n_kv - 1) {
+                        umma_commit(o_final(i));
+                    } else {
+                        issue_qk(j + 1);
+                    }
+                    umma_commit(v_empty(st));
+                }
+                // key blocks only the other tile uses: hand this tile's share of their stages back once they have
+                // landed (an earlier arrival would count for the stage's previous use)
+                for (int j = n_kv; j < nmax && ok; ++j) {
+                    const int st = j % P_STAGES;
+                    const uint32_t ph = (uint32_t)(j / P_STAGES) & 1u;
+                    if (!mbar_wait_relaxed(k_full(st), ph, ctx) || !mbar_wait_relaxed(v_full(st), ph, ctx)) break;
+                    mbar_arrive(k_empty(st));
+                    mbar_arrive(v_empty(st));
+                }
+            }
+        }
+    } else if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(P_REGS_SOFTMAX));
+        // ------------------------------------------------------------ softmax of tile i
+        const int i = warp >> 2, quad = warp & 3;
+        const int r = quad * 32 + lane;
+        const int qs = q0 + i * 128;                       // first row of the tile
+        const int row = qs + r;
+        const int n_kv = i ? n1 : n0;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const uint32_t tmem_s = tmem_base + (uint32_t)(i * 128);
+        const float c = p.softmax_scale * __ldg(p.q_inv) * __ldg(p.k_inv) * 1.4426950408889634f;
+        float m = -INFINITY, l = 0.0f;
+        // one key block; MASK: columns past `limit` (the causal diagonal, the end of the sequence) count as -inf
+        auto block = [&](auto masked, const int j) -> bool {
+            constexpr bool MASK = decltype(masked)::value;
+            const int limit = min(p.causal ? row : 0x7FFFFFFF, p.N - 1) - j * A_BN;   // last valid local column
+            if (!mbar_wait_warp(s_full(i), (uint32_t)j & 1u, ctx)) return false;
+            tc_fence_after();
+            uint32_t sv[4][32];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(tmem_s + lane_addr + (uint32_t)(q * 32), sv[q]);
+            tmem_ld_wait();
+            float mq[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                mq[q] = -INFINITY;
+                if (MASK) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (q * 32 + e <= limit) mq[q] = fmaxf(mq[q], __uint_as_float(sv[q][e]));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2)
+                        mq[q] = fmax3(mq[q], __uint_as_float(sv[q][e]), __uint_as_float(sv[q][e + 1]));
+                }
+            }
+            const float mx = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3]));
+            const float m_blk = mx * c;
+            const bool grew = m_blk > m + p.max_slack;
+            const float m_new = grew ? m_blk : m;
+            const float alpha = grew ? ex2_approx(m - m_new) : 1.0f;      // first block: m = -inf, alpha = 0
+            // the correction warps rescale O_i while this thread evaluates its exponentials
+            alpha_s[i * 128 + r] = alpha;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(alpha_ready(i, quad));
+            const float neg_shift = p.log2_p_scale - m_new;
+            float lsum = 0.0f;
+            uint32_t w[32];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t wq[8];
+                lsum += softmax_chunk<MASK>(sv[q], c, neg_shift, limit - q * 32, wq);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) w[q * 8 + e] = wq[e];
+            }
+            // P8 over the first 32 score columns (this thread's own row, already in registers)
+            tmem_st_32x32b_x32(tmem_s + lane_addr, w);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pv_go(i));
+            l = l * alpha + lsum;
+            m = m_new;
+            return true;
+        };
+        bool ok = true;
+        // Causal: tile 0 has one key block fewer than tile 1.  It starts when tile 1 has stored its first P8, so that
+        // the two tiles' exponential phases start out apart on the exponential unit instead of coinciding.
+        if (i == 0 && n1 > n0) ok = mbar_wait_warp(pv_go(1), 0, ctx);
+        if (n_kv > 0) {
+            const int k_last = (n_kv - 1) * A_BN;
+            const bool last_masked = (k_last + A_BN - 1 > qs && p.causal) || (k_last + A_BN > p.N);
+            const int n_plain = last_masked ? n_kv - 1 : n_kv;
+            for (int j = 0; j < n_plain && ok; ++j) ok = block(std::false_type{}, j);
+            if (ok && last_masked) ok = block(std::true_type{}, n_kv - 1);
+        }
+        if (ok && n_kv > 0) {
+            l_s[i * 128 + r] = l;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(l_ready(i, quad));
+            if (row < p.N)
+                p.LSE[((size_t)b * p.Hq + h) * p.N + row] = (m + log2f(l) - p.log2_p_scale) * 0.69314718055994531f;
+        }
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(P_REGS_CORR));
+        // ------------------------------------------------------------ correction and epilogue
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const int nt[2] = {n0, n1};
+        // jc[i]: next event of tile i: block jc[i] to correct; == nt[i]: the epilogue; > nt[i]: done
+        int jc[2] = {0, n1 > 0 ? 0 : 1};
+        bool ok = true, stored = false;
+        IdleGuard idle;
+        idle.reset();
+        // lane 0 looks at the barrier, the warp follows it (the TMEM instructions below need the whole warp)
+        auto ready = [&](uint32_t bar, uint32_t parity) -> bool {
+            int v = 0;
+            if (lane == 0) v = mbar_test_wait(bar, parity) ? 1 : 0;
+            return __shfl_sync(0xffffffffu, v, 0) != 0;
+        };
+        while (ok && (jc[0] <= n0 || jc[1] <= n1)) {
+            bool progressed = false;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int j = jc[i];
+                if (j < nt[i]) {
+                    if (!ready(alpha_ready(i, quad), (uint32_t)j & 1u)) continue;
+                    __syncwarp();
+                    if (j > 0) {
+                        const float a = alpha_s[i * 128 + r];
+                        if (__any_sync(0xffffffffu, a != 1.0f)) {
+                            // S_i(j) complete implies PV_i(j-1) complete: O_i is at rest
+                            tc_fence_after();
+                            const uint32_t to = tmem_base + 256u + (uint32_t)(i * 128) + lane_addr;
+                            const uint64_t a2 = pack_f32x2(a, a);
+#pragma unroll 1
+                            for (int cc = 0; cc < D; cc += 32) {
+                                uint32_t v[32];
+                                tmem_ld_32x32b_x32(to + (uint32_t)cc, v);
+                                tmem_ld_wait();
+#pragma unroll
+                                for (int e = 0; e < 32; e += 2) {
+                                    float x, y;
+                                    unpack_f32x2(mul_f32x2(pack_f32x2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), a2), x, y);
+                                    v[e] = __float_as_uint(x);
+                                    v[e + 1] = __float_as_uint(y);
+                                }
+                                tmem_st_32x32b_x32(to + (uint32_t)cc, v);
+                            }
+                            tmem_st_wait();
+                            tc_fence_before();
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(pv_go(i));
+                    jc[i] = j + 1;
+                    progressed = true;
+                } else if (j == nt[i]) {
+                    // the tile has passed its last key block: normalise and store it once its last PV is complete
+                    if (!ready(l_ready(i, quad), 0) || !ready(o_final(i), 0)) continue;
+                    __syncwarp();
+                    tc_fence_after();
+                    const int row = q0 + i * 128 + r;
+                    const float inv = __ldg(p.v_inv) / l_s[i * 128 + r];     // l already carries c_P
+                    uint8_t *o8row = p.O8 + (((size_t)b * p.N + row) * p.Hq + h) * D;
+                    const float o_scale = p.o_scale ? __ldg(p.o_scale) : 1.0f;
+                    const uint32_t to = tmem_base + 256u + (uint32_t)(i * 128) + lane_addr;
+                    uint32_t amax2 = 0;
+#pragma unroll 1
+                    for (int cc = 0; cc < D; cc += 32) {
+                        uint32_t v[32];
+                        tmem_ld_32x32b_x32(to + (uint32_t)cc, v);
+                        tmem_ld_wait();
+                        // staging tile of 64 columns: [128 rows x 128 bytes], 128-byte swizzle; columns 0-63 over the
+                        // tile's Q buffer, columns 64-127 in OST_i
+                        uint8_t *trow = smem + (cc < 64 ? L::Q_OFF : L::OST_OFF) + i * L::TILE_BYTES + r * 128;
+                        const int c0 = (cc & 63) >> 3;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            uint4 o;
+                            o.x = pack_bf16x2(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv);
+                            o.y = pack_bf16x2(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
+                            o.z = pack_bf16x2(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
+                            o.w = pack_bf16x2(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(trow + (((c0 + (e >> 3)) ^ (r & 7)) << 4)) = o;
+                            if (p.o_scale && row < p.N) {
+                                amax2 = __vmaxu2(__vmaxu2(__vmaxu2(__vmaxu2(amax2, o.x & 0x7FFF7FFFu), o.y & 0x7FFF7FFFu),
+                                                          o.z & 0x7FFF7FFFu), o.w & 0x7FFF7FFFu);
+                                const uint32_t e0 = cvt_f32x4_to_fp8x4<0>(
+                                    __fmul_rn(bf16_lo(o.x), o_scale), __fmul_rn(bf16_hi(o.x), o_scale),
+                                    __fmul_rn(bf16_lo(o.y), o_scale), __fmul_rn(bf16_hi(o.y), o_scale));
+                                const uint32_t e1 = cvt_f32x4_to_fp8x4<0>(
+                                    __fmul_rn(bf16_lo(o.z), o_scale), __fmul_rn(bf16_hi(o.z), o_scale),
+                                    __fmul_rn(bf16_lo(o.w), o_scale), __fmul_rn(bf16_hi(o.w), o_scale));
+                                *reinterpret_cast<uint2 *>(o8row + cc + e) = make_uint2(e0, e1);
+                            }
+                        }
+                    }
+                    if (p.o_scale && p.o_amax_bits) {
+                        uint32_t mm = row < p.N ? max(amax2 & 0xFFFFu, amax2 >> 16) : 0u;
+                        mm = __reduce_max_sync(0xffffffffu, mm);
+                        if (lane == 0 && mm != 0u) atomicMax(p.o_amax_bits, mm << 16);
+                    }
+                    // every warp stores its own 32 rows (the output map's box is 32 rows x 64 columns)
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_3d(&tm_o, sbase + L::Q_OFF + i * L::TILE_BYTES + quad * 4096, (h * D) * 2,
+                                     q0 + i * 128 + quad * 32, b);
+                        tma_store_3d(&tm_o, sbase + L::OST_OFF + i * L::TILE_BYTES + quad * 4096, (h * D + 64) * 2,
+                                     q0 + i * 128 + quad * 32, b);
+                        bulk_commit_group();
+                        stored = true;
+                    }
+                    jc[i] = j + 1;
+                    progressed = true;
+                }
+            }
+            if (progressed) idle.reset();
+            else {
+                if (__shfl_sync(0xffffffffu, (int)(lane == 0 && idle.expired(ctx)), 0)) ok = false;
+            }
+        }
+        if (stored) bulk_wait_group_read0();               // shared memory is read before the CTA may exit
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+        __syncthreads();
+    }
+    if (warp == 13) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, P_TMEM_COLS);
+    }
+}
+
 int validate_attn(const char *who, const void *q, const void *k, const void *v, const fp8_attn_scales *sc, int B, int N,
                   int Hq, int Hkv, int d)
 {
@@ -418,6 +868,39 @@ static int launch_attn_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *
     return FP8_OK;
 }
 
+
+static int launch_attn_fwd_pair(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const AttnFwdParams &p,
+                                cudaStream_t st)
+{
+    constexpr int D = 128;
+    CUtensorMap tq, tk, tv, to;
+    int rc = make_tmap_3d_u8(&tq, Q8, (uint64_t)p.Hq * D, (uint64_t)p.N, (uint64_t)p.B, D, 128);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tk, K8, (uint64_t)p.Hkv * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BN);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tv, V8, (uint64_t)p.Hkv * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BN);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&to, p.O, (uint64_t)p.Hq * D * 2, (uint64_t)p.N, (uint64_t)p.B, 128, 32);
+    if (rc != FP8_OK) return rc;
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        AttnFwdPairSmem::DYN_BYTES));
+    dim3 grid((unsigned)((p.N + 255) / 256), (unsigned)p.Hq, (unsigned)p.B);
+    attn_fwd_pair_kernel<<<grid, P_THREADS, AttnFwdPairSmem::DYN_BYTES, st>>>(tq, tk, tv, to, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+// FP8DPA_ATTN_FWD=single forces the one-tile-per-CTA kernel at d = 128 (for A/B measurements)
+static bool attn_fwd_use_pair()
+{
+    static int v = -1;
+    if (v < 0) {
+        const char *e = getenv("FP8DPA_ATTN_FWD");
+        v = (e && strcmp(e, "single") == 0) ? 0 : 1;
+    }
+    return v != 0;
+}
+
 }  // namespace fp8dpa
 
 using namespace fp8dpa;
@@ -460,7 +943,8 @@ static int attention_fwd_common(const char *who, const uint8_t *Q8, const uint8_
     p.o_amax_bits = reinterpret_cast<unsigned int *>(o_amax);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (o_scale && o_amax) FP8_CUDA_CHECK(cudaMemsetAsync(o_amax, 0, sizeof(float), st));
-    return d == 128 ? launch_attn_fwd<128>(Q8, K8, V8, p, st) : launch_attn_fwd<64>(Q8, K8, V8, p, st);
+    if (d == 128) return attn_fwd_use_pair() ? launch_attn_fwd_pair(Q8, K8, V8, p, st) : launch_attn_fwd<128>(Q8, K8, V8, p, st);
+    return launch_attn_fwd<64>(Q8, K8, V8, p, st);
 }
 
 extern "C" int fp8_attention_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const fp8_attn_scales *sc,

@@ -84,6 +84,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// non-blocking look at a barrier phase (for roles that serve several event sources in arrival order)
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
 // Bounded wait.  Gives up after ~2 s (or as soon as another role of the CTA has given up), records
 // FP8_ERR_TIMEOUT in the device status word and returns false; the caller then leaves its loop and
 // falls through to the common teardown.
@@ -110,6 +122,31 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
             }
         }
     }
+}
+
+// The same wait for roles that are not on the critical path of their CTA (producers waiting for a free stage, helpers
+// waiting for work): between polls the thread sleeps, so that it does not take issue slots from the warps that
+// share its scheduler.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, const WaitCtx &ctx, unsigned ns = 64)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        __nanosleep(ns);
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0) {
+            if (*ctx.abort_flag) return false;
+            if (clock64() - t0 > (ctx.limit > 0 ? ctx.limit : FP8DPA_WAIT_LIMIT_CYCLES)) {
+                *ctx.abort_flag = 1;
+                atomicExch(ctx.status, (int)FP8_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait_relaxed_warp(uint32_t bar, uint32_t parity, const WaitCtx &ctx, unsigned ns = 64)
+{
+    return __all_sync(0xffffffffu, mbar_wait_relaxed(bar, parity, ctx, ns) ? 1 : 0) != 0;
 }
 
 // Warp-uniform form for warps whose 32 lanes wait together and then run .sync.aligned instructions:
