@@ -98,14 +98,18 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     if (GROUPED) {
         // every CTA builds the same tile table from the device-side offsets
         if (threadIdx.x == 0) {
-            int acc = 0;
+            // The offsets come from the router on the device and the host never sees them: force them into
+            // 0 <= offs[0] <= offs[1] <= ... <= M, so that an array that breaks the contract gives wrong (clipped)
+            // groups, never a store past the end of the output.
+            int acc = 0, prev = min(max(__ldg(p.group_offsets), 0), p.M);
             for (int g = 0; g < p.n_groups; ++g) {
-                const int o0 = __ldg(p.group_offsets + g), o1 = __ldg(p.group_offsets + g + 1);
-                g_offs[g] = o0;
+                const int o1 = min(max(__ldg(p.group_offsets + g + 1), prev), p.M);
+                g_offs[g] = prev;
                 g_tile_start[g] = acc;
-                acc += ((max(o1 - o0, 0) + 2 * BM - 1) / (2 * BM)) * tiles_n;
+                acc += ((o1 - prev + 2 * BM - 1) / (2 * BM)) * tiles_n;
+                prev = o1;
             }
-            g_offs[p.n_groups] = __ldg(p.group_offsets + p.n_groups);
+            g_offs[p.n_groups] = prev;
             g_tile_start[p.n_groups] = acc;
         }
         __syncthreads();

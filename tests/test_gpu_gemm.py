@@ -265,6 +265,25 @@ def test_grouped_forward_matches_oracle_per_expert(sizes, N, K, out_dtype):
     assert np.all(got[T:] == 7.0)
 
 
+def test_grouped_forward_with_offsets_that_break_the_contract_stays_inside_the_output():
+    """The group offsets live on the device, so the host cannot validate them.  An array that is not ascending or
+    runs past T must not make the kernel store outside the [T, N] output: the kernel clips every offset into
+    [previous offset, T]."""
+    T, N, K, E = 1024, 256, 128, 4
+    guard = 64
+    x8 = torch.randint(0x20, 0x48, (T + guard, K), dtype=torch.uint8, device="cuda")
+    w8 = torch.randint(0x20, 0x48, (E, N, K), dtype=torch.uint8, device="cuda")
+    sx, sw = scalar(2.0 ** -4), torch.full((E,), 2.0 ** -5, device="cuda")
+    for bad in ([0, 300, 200, 900, 5000], [-7, 100, 100, 2000, 1500], [0, 1 << 30, 3, 4, 5]):
+        y = torch.full((T + guard, N), 7.0, dtype=torch.bfloat16, device="cuda")
+        offs = torch.tensor(bad, dtype=torch.int32, device="cuda")
+        fp8.fp8_grouped_linear_fwd(x8[:T], w8, sx, sw, offs, y[:T])
+        torch.cuda.synchronize()
+        assert fp8.fp8_device_status() == 0
+        assert torch.all(y[T:] == 7.0)
+        assert torch.isfinite(y.float()).all()
+
+
 @pytest.mark.parametrize("sizes,N,K", [([300, 0, 129, 512, 83], 512, 144), ([256, 256], 256, 256),
                                         ([1000, 17, 2000, 1, 600, 0, 0, 350], 1024, 528), ([16], 128, 16)])
 @pytest.mark.parametrize("out_dtype", [torch.bfloat16, torch.float32])
