@@ -183,6 +183,113 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------------------- other workloads
+def quantize_sweep(peaks):
+    """Workload c2: amax / cast / quantize on flat BF16 tensors of 2^20 .. 2^29 elements, N(0,1) with 1e-4 of the
+    entries set to +-200.  `cold`: the calls walk a pool of tensors larger than twice the L2, so nothing is resident
+    from the previous call; `warm`: the same tensor again and again (flagged: at the small sizes this is an L2 figure)."""
+    import torch
+    import paper_2505_20524_b200 as fp8
+    out = []
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(2)
+    f32 = lambda v=0.0: torch.full((1,), float(v), dtype=torch.float32, device="cuda")
+    for log2n in (20, 24, 27, 29):
+        n = 1 << log2n
+        nbuf = max(1, min(160, -(-(300 << 20) // (2 * n))))
+        xs = []
+        for _ in range(nbuf):
+            x = torch.randn(n, device="cuda", generator=gen)
+            hit = torch.rand(n, device="cuda", generator=gen) < 1e-4
+            x = torch.where(hit, torch.where(x > 0, 200.0, -200.0), x).to(torch.bfloat16)
+            xs.append(x)
+            del hit
+        q = torch.empty(n, dtype=torch.uint8, device="cuda")
+        a, sc, si = f32(), f32(2.24), f32(1.0)
+        ops = (("amax", 2, lambda x: fp8.fp8_amax(x, a)),
+               ("cast_e4m3", 3, lambda x: fp8.fp8_cast(x, sc, fp8.E4M3, q)),
+               ("cast_e5m2", 3, lambda x: fp8.fp8_cast(x, sc, fp8.E5M2, q)),
+               ("quantize_e4m3", 5, lambda x: fp8.fp8_quantize(x, fp8.E4M3, q, None, a, sc, si)))
+        row = {"elements": n, "pool_tensors": nbuf}
+        for name, bpe, fn in ops:
+            for mode in ("cold", "warm"):
+                reps = max(8, nbuf) if mode == "cold" else 20
+                for i in range(3):
+                    fn(xs[i % nbuf])
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                e0.record()
+                for i in range(reps):
+                    fn(xs[i % nbuf] if mode == "cold" else xs[0])
+                e1.record()
+                torch.cuda.synchronize()
+                gbs = bpe * n * reps / (e0.elapsed_time(e1) / 1e3) / 1e9
+                row[f"{name}_{mode}_gbs"] = round(gbs, 1)
+        row["quantize_cold_frac_of_measured_hbm"] = round(row["quantize_e4m3_cold_gbs"] / peaks["hbm"], 3)
+        out.append(row)
+        del xs, q
+        torch.cuda.empty_cache()
+    return {"workload": "c2: flat BF16 tensors, N(0,1) with 1e-4 of the entries +-200 (drawn on the device, seed 2)",
+            "bytes_per_element": {"amax": 2, "cast": 3, "quantize": 5}, "hbm_gbs_measured": peaks["hbm"],
+            "note": "warm = same tensor repeated (L2-resident below 2^26 elements); cold = pool of tensors > 2 x L2",
+            "sizes": out}
+
+
+def long_context_attention(peaks, steps=5):
+    """Workload c5: causal FP8 attention forward + backward at B = 1, N = 16384, 32 heads x 128; Q/K/V N(0,1) with 1% of
+    the (head, dim) columns x 40, dO N(0, 1e-3); drawn on the device (seed 5) and quantised by fp8_quantize."""
+    import torch
+    import paper_2505_20524_b200 as fp8
+    B, N, H, d = 1, 16384, 32, 128
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    f32 = lambda v=0.0: torch.full((1,), float(v), dtype=torch.float32, device="cuda")
+    t = {}
+    for name, std, fmt in (("q", 1.0, fp8.E4M3), ("k", 1.0, fp8.E4M3), ("v", 1.0, fp8.E4M3), ("do", 1e-3, fp8.E5M2)):
+        x = torch.randn((B, N, H, d), device="cuda", generator=gen) * std
+        if name != "do":
+            cols = torch.randperm(H * d, device="cuda", generator=gen)[:41]
+            x.view(B, N, H * d)[:, :, cols] *= 40.0
+        x = x.to(torch.bfloat16)
+        q8 = torch.empty((B, N, H, d), dtype=torch.uint8, device="cuda")
+        a, sc, si = f32(), f32(), f32()
+        fp8.fp8_quantize(x, fmt, q8, None, a, sc, si)
+        t[name] = (q8, si)
+        del x
+    O = torch.empty((B, N, H, d), dtype=torch.bfloat16, device="cuda")
+    LSE = torch.empty((B, H, N), dtype=torch.float32, device="cuda")
+    dq, dk, dv = torch.empty_like(O), torch.empty_like(O), torch.empty_like(O)
+    ws = torch.empty(fp8.fp8_attention_workspace_bytes(1, B, N, H, H, d), dtype=torch.uint8, device="cuda")
+    s, dss, amax = d ** -0.5, f32(1.0), f32()
+    fwd = lambda: fp8.fp8_attention_fwd(t["q"][0], t["k"][0], t["v"][0], t["q"][1], t["k"][1], t["v"][1], s, True, O,
+                                        LSE, None)
+    bwd = lambda: fp8.fp8_attention_bwd(t["q"][0], t["k"][0], t["v"][0], t["do"][0], O, LSE, t["q"][1], t["k"][1],
+                                        t["v"][1], t["do"][1], s, dss, True, dq, dk, dv, ws, ds_amax=amax)
+    fwd()
+    bwd()                                        # calibration of the dS scale, delayed-scaling style
+    fp8.fp8_scale(amax, fp8.E5M2, 0, dss, f32())
+    res = {}
+    for name, fn in (("fwd", fwd), ("bwd", bwd)):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        res[name] = e0.elapsed_time(e1) / steps
+    fl = 2.0 * B * H * N * N * d
+    tot = 3.5 * fl / (res["fwd"] + res["bwd"]) / 1e9
+    return {"workload": "c5: B 1, N 16384, 32 heads x 128, causal; synthetic, drawn on the device (seed 5)",
+            "fwd_ms": res["fwd"], "bwd_ms": res["bwd"], "fwd_tflops": fl / res["fwd"] / 1e9,
+            "bwd_tflops": 2.5 * fl / res["bwd"] / 1e9, "fwd_bwd_tflops": tot,
+            "fwd_bwd_frac_of_nominal_4500": tot / FP8_NOMINAL_TFLOPS,
+            "fwd_bwd_frac_of_2x_burst": tot / (2.0 * peaks["bf16_burst"]), "steps": steps,
+            "l2": "operands (4 x 67 MB) and outputs exceed the L2 together; no flush", "device_status": fp8.fp8_device_status()}
+
+
 # ---------------------------------------------------------------------------------------------- our arm
 def max_over_ranks(ms_local: float, world: int, device=None) -> float:
     """Device time of the slowest rank (every rank gets the same number)."""
@@ -278,18 +385,49 @@ def run_ours(args, cfg):
     n_gemm = sum(len(evs) for evs in hp.gemm_events)
     gemm_tflops = hp.gemm_flops() * args.steps / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else None
     peaks = measured_peaks()
-    fp8_peak = 2.0 * peaks["bf16_sustained"]          # FP8 = 2x the BF16 rate; kernel timed inside a long step
+    # Which measured peak the in-step rate is compared with.  FP8 is nominally 2x the BF16 rate, so the denominators
+    # are 2 x the measured BF16 GEMM figures.  The sustained figure was taken over seconds at a power-capped clock;
+    # a timed region shorter than a second that ran at (nearly) the maximum SM clock is a burst, and is compared
+    # with the burst figure.  All three fractions are carried; `frac` is the one the rule picks.
+    region_s = ms_total / 1e3
+    clk_ok = bool(clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and
+                  clocks["sm_mhz"] >= 0.97 * clocks["sm_max_mhz"])
+    use_burst = region_s < 1.0 or clk_ok
+    fp8_peak = 2.0 * (peaks["bf16_burst"] if use_burst else peaks["bf16_sustained"])
     roofline = None
     if gemm_tflops is not None:
+        traffic = GEMM_DRAM_CAPTURE.get(cfg.name)
         roofline = {
             "bound": "tensor", "kernel": "gemm_fp8_pair_kernel", "achieved": gemm_tflops, "peak": fp8_peak,
             "unit": "TFLOP/s", "frac": gemm_tflops / fp8_peak,
-            "traffic": GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name),
-            "peak_source": f"2 x bf16_tflops_sustained ({peaks['source']})",
+            "traffic": traffic["bytes_per_launch"] if traffic else None,
+            "traffic_source": traffic["source"] if traffic else None,
+            "peak_source": (f"2 x bf16_tflops{'' if use_burst else '_sustained'} ({peaks['source']}); rule: burst figure "
+                            f"when the timed region is < 1 s or the sampled SM clock stays within 3% of its maximum "
+                            f"(region {region_s:.2f} s, median clock {clocks.get('sm_mhz')} MHz), else sustained"),
             "launches": n_gemm, "avg_launch_ms": gemm_ms / max(n_gemm, 1),
             "flops_per_launch": hp.gemm_flops() / 12.0,
+            "frac_vs_2x_burst": gemm_tflops / (2.0 * peaks["bf16_burst"]),
+            "frac_vs_2x_sustained": gemm_tflops / (2.0 * peaks["bf16_sustained"]),
             "frac_of_nominal_4500": gemm_tflops / FP8_NOMINAL_TFLOPS,
         }
+
+    # ---- the other parts of the step, from their own events: attention forward / backward and the quantize groups
+    attention, quantize = None, None
+    if hp.attn_events and hp.attn_events[0]:
+        f_ms = sum(evs[0][0].elapsed_time(evs[0][1]) for evs in hp.attn_events) / args.steps
+        b_ms = sum(evs[1][0].elapsed_time(evs[1][1]) for evs in hp.attn_events) / args.steps
+        fwd_fl = hp.attention_flops() / 3.5
+        attention = {"fwd_ms": f_ms, "bwd_ms": b_ms, "fwd_tflops": fwd_fl / f_ms / 1e9, "bwd_tflops": 2.5 * fwd_fl / b_ms / 1e9,
+                     "fwd_frac_of_nominal_4500": fwd_fl / f_ms / 1e9 / FP8_NOMINAL_TFLOPS,
+                     "bwd_frac_of_nominal_4500": 2.5 * fwd_fl / b_ms / 1e9 / FP8_NOMINAL_TFLOPS,
+                     "fwd_bwd_tflops": 3.5 * fwd_fl / (f_ms + b_ms) / 1e9,
+                     "fwd_bwd_frac_of_2x_burst": 3.5 * fwd_fl / (f_ms + b_ms) / 1e9 / (2.0 * peaks["bf16_burst"])}
+    if hp.quant_events and hp.quant_events[0]:
+        q_ms = sum(a.elapsed_time(b) for evs in hp.quant_events for a, b in evs) / args.steps
+        gbs = hp.quantize_bytes() / q_ms / 1e6
+        quantize = {"ms_per_step": q_ms, "gb_per_step": hp.quantize_bytes() / 1e9, "gbs": gbs,
+                    "frac_of_measured_hbm": gbs / peaks["hbm"], "hbm_gbs": peaks["hbm"], "peak_source": peaks["source"]}
 
     # ---- end to end: pinned host inputs -> device, step, every output -> pinned host
     ins, outs = hp.input_tensors(), hp.output_tensors()
@@ -327,6 +465,16 @@ def run_ours(args, cfg):
         cpu_baseline = {"value": f / s / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"{reps} x ({desc})", "seconds": s}
 
+    acct = {"launches": hp.launches_per_step() * args.steps, "gemm_tflop": hp.gemm_flops() / 1e12,
+            "attn_tflop": hp.attention_flops() / 1e12, "quant_gb": hp.quantize_bytes() / 1e9}
+    c2, c5 = None, None
+    if rank == 0 and world == 1 and not args.no_extra and cfg.name == "c4":
+        del hp, h_in, h_out, hin, hout
+        torch.cuda.empty_cache()
+        c2 = quantize_sweep(peaks)
+        c5 = long_context_attention(peaks)
+        hp = None
+
     if rank == 0:
         c = cfg
         line = {
@@ -342,13 +490,17 @@ def run_ours(args, cfg):
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
-            "gpu_launches": hp.launches_per_step() * args.steps,
+            "gpu_launches": acct["launches"],
             "roofline": roofline,
             "cpu_baseline": cpu_baseline,
+            "attention": attention,
+            "quantize": quantize,
+            "c2_quantize_sweep": c2,
+            "c5_long_context_attention": c5,
             "breakdown": {"gemm_ms_per_step": gemm_ms / args.steps, "gemm_tflops": gemm_tflops,
-                          "gemm_tflop_per_step": hp.gemm_flops() / 1e12,
-                          "attention_tflop_per_step": hp.attention_flops() / 1e12,
-                          "quantize_gb_per_step": hp.quantize_bytes() / 1e9},
+                          "gemm_tflop_per_step": acct["gemm_tflop"],
+                          "attention_tflop_per_step": acct["attn_tflop"],
+                          "quantize_gb_per_step": acct["quant_gb"]},
         }
         if graph_info is not None:
             line["graph"] = graph_info
@@ -357,9 +509,11 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) per GEMM launch, averaged over the 12 launches of one step, from the single-pass ncu
-# capture summarised in profiles/gemm_fp8_pair_kernel.md (null for workloads without a capture).
-GEMM_DRAM_BYTES_PER_LAUNCH = {"c4": 416.15e6}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per GEMM launch, averaged over the 12 launches of one step:
+# from one single-pass ncu capture of this benchmark (`--metrics dram__bytes_read.sum,dram__bytes_write.sum,
+# gpu__time_duration.sum --clock-control none -k regex:gemm_fp8`), taken on the commit named in `source`.  None for
+# workloads without a capture: a figure from another build says nothing about this one.
+GEMM_DRAM_CAPTURE = {}
 
 
 # ---------------------------------------------------------------------------------------------- per-kernel report
@@ -410,6 +564,14 @@ def run_report(args):
     def codes(*shape):
         return torch.randint(0x20, 0x48, shape, dtype=torch.uint8, device="cuda")
 
+    def cast_codes(shape, std, fmt):
+        """FP8 codes of a normal tensor under just-in-time scaling: the bit activity of real operands (uniformly drawn
+        codes run several per cent faster on a power-capped board)."""
+        x = (std * torch.randn(shape, device="cuda")).to(torch.bfloat16)
+        q = torch.empty(shape, dtype=torch.uint8, device="cuda")
+        fp8.fp8_quantize(x, fmt, q, None, f32(), f32(), f32())
+        return q
+
     # ---- quantize family (HBM): the flat sweep of workload c2 and the block tensors of c4
     for n in (1 << 24, 1 << 27, 1 << 29):
         x = bf16(n)
@@ -458,8 +620,8 @@ def run_report(args):
     for cname in ("c3", "c4"):
         cfg = synth.CONFIGS[cname]
         for layer, (Tt, N, K) in cfg.linear_shapes().items():
-            x8, w8, dy8 = codes(Tt, K), codes(N, K), codes(Tt, N)
-            x8t, w8t, dy8t = codes(K, Tt), codes(K, N), codes(N, Tt)
+            x8, w8, dy8 = cast_codes((Tt, K), 1.0, fp8.E4M3), cast_codes((N, K), 0.02, fp8.E4M3), cast_codes((Tt, N), 1e-3, fp8.E5M2)
+            x8t, w8t, dy8t = x8.t().contiguous(), w8.t().contiguous(), dy8.t().contiguous()
             s1, s2 = f32(1e-2), f32(1e-2)
             yb, dxb, dwb = (torch.empty(sh, dtype=torch.bfloat16, device="cuda") for sh in ((Tt, N), (Tt, K), (N, K)))
             fl = 2.0 * Tt * N * K
@@ -556,6 +718,8 @@ def main():
     ap.add_argument("--attn-slack", type=float, default=0.0,
                     help="tau of the attention forward's reference maximum (default 0 = exact running maximum; the "
                          "contract line is quoted with 0)")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the two extra workloads of the default line (c2 quantize sweep, c5 attention)")
     ap.add_argument("--graph", action="store_true",
                     help="also time the step replayed from a CUDA graph (extra key \"graph\"; the contract keys stay eager)")
     args = ap.parse_args()

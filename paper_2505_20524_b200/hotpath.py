@@ -97,6 +97,8 @@ class BlockHotPath:
         self.attn = None
         self.host_inputs: dict[str, np.ndarray] = {}
         self.gemm_events = []
+        self.quant_events = []
+        self.attn_events = []
 
     # ------------------------------------------------------------------ inputs
     def generate_host_inputs(self):
@@ -303,22 +305,26 @@ class BlockHotPath:
         return graph
 
     def step(self, time_gemms: bool = False):
-        ev = []
+        """One pass of the hot path.  With ``time_gemms`` every GEMM launch, every quantize group and the two attention
+        calls are bracketed by CUDA events on the launching stream (appended to gemm_events / quant_events /
+        attn_events, one list per step)."""
+        ev, qev, aev = [], [], []
 
-        def gemm(fn, *args, **kw):
+        def timed(dst, fn, *args, **kw):
             if time_gemms:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
                 fn(*args, **kw)
                 e1.record()
-                ev.append((e0, e1))
+                dst.append((e0, e1))
             else:
                 fn(*args, **kw)
 
+        def gemm(fn, *args, **kw):
+            timed(ev, fn, *args, **kw)
+
         for lin in self.linears:
-            lin.x.quantize()
-            lin.w.quantize()
-            lin.dy.quantize()
+            timed(qev, lambda: (lin.x.quantize(), lin.w.quantize(), lin.dy.quantize()))
             gemm(fp8.fp8_linear_fwd, lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
             if self.transposed_copies:
                 gemm(fp8.fp8_linear_dgrad, lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
@@ -328,13 +334,14 @@ class BlockHotPath:
                 gemm(fp8.fp8_linear_wgrad_rm, lin.dy.q, lin.x.q, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
         if self.attn is not None:
             a = self.attn
-            for n in ("q", "k", "v", "do"):
-                a[n].quantize()
-            fp8.fp8_attention_fwd(a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv, a["v"].scale_inv,
-                                  a["softmax_scale"], True, a["o"], a["lse"], None,
-                                  p_scale=448.0 / 2.0 ** self.attn_max_slack, max_slack=self.attn_max_slack)
-            fp8.fp8_attention_bwd(a["q"].q, a["k"].q, a["v"].q, a["do"].q, a["o"], a["lse"], a["q"].scale_inv,
-                                  a["k"].scale_inv, a["v"].scale_inv, a["do"].scale_inv, a["softmax_scale"],
-                                  a["ds_scale"], True, a["dq"], a["dk"], a["dv"], a["ws"], ds_amax=a["ds_amax"])
+            timed(qev, lambda: [a[n].quantize() for n in ("q", "k", "v", "do")])
+            timed(aev, fp8.fp8_attention_fwd, a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv,
+                  a["v"].scale_inv, a["softmax_scale"], True, a["o"], a["lse"], None,
+                  p_scale=448.0 / 2.0 ** self.attn_max_slack, max_slack=self.attn_max_slack)
+            timed(aev, fp8.fp8_attention_bwd, a["q"].q, a["k"].q, a["v"].q, a["do"].q, a["o"], a["lse"],
+                  a["q"].scale_inv, a["k"].scale_inv, a["v"].scale_inv, a["do"].scale_inv, a["softmax_scale"],
+                  a["ds_scale"], True, a["dq"], a["dk"], a["dv"], a["ws"], ds_amax=a["ds_amax"])
         if time_gemms:
             self.gemm_events.append(ev)
+            self.quant_events.append(qev)
+            self.attn_events.append(aev)
