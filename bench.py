@@ -605,6 +605,10 @@ def run_report(args):
             nbytes=2 * T * F)
         add(f"fp8_act_cast {name} (cast + transposed copy)", f"{T}x{F}",
             timed(lambda: fp8.fp8_act_cast(xa, act, par, sc, 0, h8, h8t, None)), nbytes=4 * T * F)
+    for act, name in ((fp8.ACT_GELU, "gelu"), (fp8.ACT_XIELU, "xielu")):
+        # delayed scaling: codes and amax in one pass over the input (2 B read + 1 B written per element)
+        add(f"fp8_act_cast {name} (single pass: cast + amax under a delayed scale)", f"{T}x{F}",
+            timed(lambda: fp8.fp8_act_cast(xa, act, par, sc, 0, h8, None, a)), nbytes=3 * T * F)
     add("fp8_kurtosis", f"{T}x{2 * F}", timed(lambda: fp8.fp8_kurtosis(x, a)), nbytes=2 * T * 2 * F)
     del x, q, qt, h8, h8t, xa
     r, y, g = bf16(2 * T, H), bf16(2 * T, H, std=0.02), torch.ones(H, device="cuda")
@@ -612,13 +616,21 @@ def run_report(args):
     for mode, name in ((fp8.NORM_RMS, "rmsnorm"), (fp8.NORM_LAYERSCALE, "layerscale")):
         add(f"fp8_postnorm_residual {name}", f"{2 * T}x{H}", timed(lambda: fp8.fp8_postnorm_residual(r, y, g, mode, 1e-5, o_, a)),
             nbytes=6 * 2 * T * H)
+    o8 = torch.empty((2 * T, H), dtype=torch.uint8, device="cuda")
+    add("fp8_postnorm_residual_q rmsnorm (BF16 + FP8 codes + amax, delayed scale)", f"{2 * T}x{H}",
+        timed(lambda: fp8.fp8_postnorm_residual_q(r, y, g, fp8.NORM_RMS, 1e-5, sc, 0, o_, o8, a)), nbytes=7 * 2 * T * H)
+    del o8
     qk = bf16(2 * T, c4.n_q_heads, c4.head_dim)
     qo = torch.empty_like(qk)
     cos, sin = torch.rand((c4.seq, c4.head_dim // 2), device="cuda"), torch.rand((c4.seq, c4.head_dim // 2), device="cuda")
     for mode, name in ((fp8.QK_RMS, "rms"), (fp8.QK_TANH, "tanh"), (fp8.QK_NONE, "none")):
         add(f"fp8_qk_norm_rope {name} + rotary", f"{2 * T}x{c4.n_q_heads}x{c4.head_dim}",
             timed(lambda: fp8.fp8_qk_norm_rope(qk, mode, 0.5, 1e-6, cos, sin, c4.seq, qo, a)), nbytes=4 * qk.numel())
-    del r, y, o_, qk, qo
+    q8_ = torch.empty(qk.shape, dtype=torch.uint8, device="cuda")
+    add("fp8_qk_norm_rope_q rms + rotary (FP8 codes only + amax, delayed scale)", f"{2 * T}x{c4.n_q_heads}x{c4.head_dim}",
+        timed(lambda: fp8.fp8_qk_norm_rope_q(qk, fp8.QK_RMS, 0.5, 1e-6, cos, sin, c4.seq, sc, 0, None, q8_, a)),
+        nbytes=3 * qk.numel())
+    del r, y, o_, qk, qo, q8_
 
     # ---- GEMMs of c3 and c4: forward / dgrad / wgrad, the producer form and the blockwise recipe
     for cname in ("c3", "c4"):

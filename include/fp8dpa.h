@@ -129,6 +129,17 @@ enum { FP8_NORM_RMS = 0, FP8_NORM_LAYERSCALE = 1 };
 FP8_API int fp8_postnorm_residual(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D,
                           int mode, float eps, void *out_bf16, float *amax_out, void *stream);
 
+/* Producer form under delayed scaling (Appendix E: rho from the amax history; Section 3 / Appendix B: without a
+ * pre-normalisation the post-norm output IS the operand of the next FP8 GEMM): the same result, and in the same
+ * pass its FP8 codes out8[T,D] = FP8cast(*scale * out) of the BF16-rounded values (bit-identical to fp8_cast of
+ * out_bf16) and *amax_out = amax(out) for fp8_scale_update.  x_scale multiplies the residual input x before the
+ * sum: 1 inside the network; sigma_0^-1 for the first block, whose input is scaled by the inverse of the
+ * initialisation standard deviation (Section 3; Appendix B, architecture table, column "input scaling").
+ * out_bf16 is required (it is the residual stream), out8 and scale are required, amax_out may be NULL. */
+FP8_API int fp8_postnorm_residual_q(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D,
+                            int mode, float eps, float x_scale, const float *scale, int fmt, void *out_bf16,
+                            uint8_t *out8, float *amax_out, void *stream);
+
 /* QK entropy regulariser and rotary embedding of per-head query / key vectors (Section 3; Appendix B:
  * attnhead = selfattn(N_QK(X W_Q), N_QK(X W_K), X W_V) with rotary position embeddings), fused with the amax that
  * the FP8 cast of Q / K needs.  x, out: [T,H,d] BF16 (out may alias x), d in {64, 128}.
@@ -141,6 +152,14 @@ enum { FP8_QK_RMS = 0, FP8_QK_TANH = 1, FP8_QK_NONE = 2 };
 FP8_API int fp8_qk_norm_rope(const void *x_bf16, size_t T, size_t H, size_t d, int mode, float alpha, float eps,
                      const float *cos_table, const float *sin_table, size_t seq_len, void *out_bf16,
                      float *amax_out, void *stream);
+
+/* Producer form under delayed scaling (Appendix E): the regularised, rotated vectors are the Q / K operands of the
+ * FP8 attention (Appendix E, table "Comparison between FP8 methods": QK^T runs in FP8), so the same pass also
+ * writes their FP8 codes out8[T,H,d] = FP8cast(*scale * out) of the BF16-rounded values (bit-identical to fp8_cast
+ * of out_bf16) and *amax_out = amax(out).  out_bf16 may be NULL when only the codes are wanted. */
+FP8_API int fp8_qk_norm_rope_q(const void *x_bf16, size_t T, size_t H, size_t d, int mode, float alpha, float eps,
+                       const float *cos_table, const float *sin_table, size_t seq_len, const float *scale, int fmt,
+                       void *out_bf16, uint8_t *out8, float *amax_out, void *stream);
 
 /* Kurtosis monitor (Section 4): *out = mean over rows of mu[x^4] / mu[x^2]^2 of a [rows, cols] BF16 tensor
  * (un-centred; rows are token vectors).  *out is overwritten.  cols % 8 == 0. */

@@ -162,15 +162,16 @@ NORM_RMS, NORM_LAYERSCALE = 0, 1
 QK_RMS, QK_TANH, QK_NONE = 0, 1, 2
 
 
-def postnorm_residual(x_bf16, y_bf16, gamma, mode: int = NORM_RMS, eps: float = 0.0) -> np.ndarray:
-    """x + gamma * y / rms(y) (mode 0) or x + gamma * y (mode 1), rounded to BF16 (Section 3, Appendix B)."""
+def postnorm_residual(x_bf16, y_bf16, gamma, mode: int = NORM_RMS, eps: float = 0.0, x_scale: float = 1.0) -> np.ndarray:
+    """x_scale * x + gamma * y / rms(y) (mode 0) or x_scale * x + gamma * y (mode 1), rounded to BF16 (Section 3,
+    Appendix B); x_scale = sigma_0^-1 on the first block's input, 1 elsewhere."""
     x, y = _c(x_bf16, np.uint16), _c(y_bf16, np.uint16)
     g = _c(gamma, np.float32)
     T, D = x.shape
     out = np.empty_like(x)
-    f = _L().oracle_postnorm_residual_bf16
+    f = _L().oracle_postnorm_residual_scaled_bf16
     f.restype = None
-    f(_p(x), _p(y), _p(g), C.c_size_t(T), C.c_size_t(D), C.c_int(mode), C.c_double(eps), _p(out))
+    f(_p(x), _p(y), _p(g), C.c_size_t(T), C.c_size_t(D), C.c_int(mode), C.c_double(eps), C.c_double(x_scale), _p(out))
     return out
 
 

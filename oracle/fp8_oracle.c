@@ -255,8 +255,11 @@ void oracle_activation_bf16(const uint16_t *x, size_t n, int act, double alpha_p
  *   mode 1  LayerScale  out = x + gamma (.) y
  * x (residual stream), y (branch output): [T,D] BF16; gamma: D binary32; out rounded to BF16.
  * ---------------------------------------------------------------------------------------------- */
-void oracle_postnorm_residual_bf16(const uint16_t *x, const uint16_t *y, const float *gamma, size_t T, size_t D,
-                                   int mode, double eps, uint16_t *out)
+/* x_scale multiplies the residual input: 1 inside the network, sigma_0^-1 on the first block's input (Section 3: the
+ * input of the first block is scaled by the inverse of the initialisation standard deviation; Appendix B,
+ * architecture table, column "input scaling"). */
+void oracle_postnorm_residual_scaled_bf16(const uint16_t *x, const uint16_t *y, const float *gamma, size_t T, size_t D,
+                                          int mode, double eps, double x_scale, uint16_t *out)
 {
 #pragma omp parallel for schedule(static)
     for (long t = 0; t < (long)T; ++t) {
@@ -267,11 +270,17 @@ void oracle_postnorm_residual_bf16(const uint16_t *x, const uint16_t *y, const f
         }
         double rinv = mode == 0 ? 1.0 / sqrt(ss / (double)D + eps) : 1.0;
         for (size_t d = 0; d < D; ++d) {
-            double r = (double)bf16_bits_to_float(x[(size_t)t * D + d]) +
+            double r = x_scale * (double)bf16_bits_to_float(x[(size_t)t * D + d]) +
                        (double)gamma[d] * (double)bf16_bits_to_float(y[(size_t)t * D + d]) * rinv;
             out[(size_t)t * D + d] = f32_to_bf16_rne((float)r);
         }
     }
+}
+
+void oracle_postnorm_residual_bf16(const uint16_t *x, const uint16_t *y, const float *gamma, size_t T, size_t D,
+                                   int mode, double eps, uint16_t *out)
+{
+    oracle_postnorm_residual_scaled_bf16(x, y, gamma, T, D, mode, eps, 1.0, out);
 }
 
 /* ------------------------------------------------------------------------------------------------

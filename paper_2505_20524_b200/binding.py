@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
-           "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_qk_norm_rope", "fp8_kurtosis",
+           "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
@@ -132,6 +132,26 @@ def fp8_postnorm_residual(x, y, gamma, mode, eps, out, amax_out=None, stream=Non
     T, D = x.shape
     _check(load().fp8_postnorm_residual(_ptr(x), _ptr(y), _ptr(gamma), C.c_size_t(T), C.c_size_t(D), C.c_int(mode),
                                         C.c_float(eps), _ptr(out), _ptr(amax_out), _stream(stream)))
+
+
+def fp8_postnorm_residual_q(x, y, gamma, mode, eps, scale, fmt, out, out8, amax_out=None, x_scale=1.0, stream=None):
+    """fp8_postnorm_residual that also writes the FP8 codes of its (BF16-rounded) result under the delayed `scale`;
+    x_scale multiplies the residual input (sigma_0^-1 for the first block's input, else 1)."""
+    T, D = x.shape
+    _check(load().fp8_postnorm_residual_q(_ptr(x), _ptr(y), _ptr(gamma), C.c_size_t(T), C.c_size_t(D), C.c_int(mode),
+                                          C.c_float(eps), C.c_float(x_scale), _ptr(scale), C.c_int(fmt), _ptr(out),
+                                          _ptr(out8), _ptr(amax_out), _stream(stream)))
+
+
+def fp8_qk_norm_rope_q(x, mode, alpha, eps, cos_table, sin_table, seq_len, scale, fmt, out, out8, amax_out=None,
+                       stream=None):
+    """fp8_qk_norm_rope that also writes the FP8 codes of its (BF16-rounded) result under the delayed `scale`
+    (out may be None when only the codes are wanted)."""
+    T, H, d = x.shape
+    _check(load().fp8_qk_norm_rope_q(_ptr(x), C.c_size_t(T), C.c_size_t(H), C.c_size_t(d), C.c_int(mode),
+                                     C.c_float(alpha), C.c_float(eps), _ptr(cos_table), _ptr(sin_table),
+                                     C.c_size_t(seq_len), _ptr(scale), C.c_int(fmt), _ptr(out), _ptr(out8),
+                                     _ptr(amax_out), _stream(stream)))
 
 
 def fp8_qk_norm_rope(x, mode, alpha, eps, cos_table, sin_table, seq_len, out, amax_out=None, stream=None):

@@ -250,14 +250,30 @@ __global__ void __launch_bounds__(256) kurtosis_kernel(const uint16_t *__restric
 // Post-norm + residual, one CTA per token row.  The row of y stays in registers between the sum of squares and the
 // update: KG 16-byte groups per thread at 256 threads (KG = 1, 2, 4, 8 for up to 2048 ... 16384 columns, chosen at
 // launch so that short rows do not pay for the registers of long ones).
+
+// Eight BF16 values (four packed words) -> eight FP8 codes under `scale`: the codes fp8_cast gives for the same
+// values (binary32 product, one rounding to FP8).  fmt: 0 = E4M3, 1 = E5M2.
+__device__ __forceinline__ uint2 bf16x8_to_fp8x8(const uint32_t (&w)[4], float scale, int fmt)
+{
+    const float v0 = __fmul_rn(bf16_lo(w[0]), scale), v1 = __fmul_rn(bf16_hi(w[0]), scale);
+    const float v2 = __fmul_rn(bf16_lo(w[1]), scale), v3 = __fmul_rn(bf16_hi(w[1]), scale);
+    const float v4 = __fmul_rn(bf16_lo(w[2]), scale), v5 = __fmul_rn(bf16_hi(w[2]), scale);
+    const float v6 = __fmul_rn(bf16_lo(w[3]), scale), v7 = __fmul_rn(bf16_hi(w[3]), scale);
+    if (fmt == 0) return make_uint2(cvt_f32x4_to_fp8x4<0>(v0, v1, v2, v3), cvt_f32x4_to_fp8x4<0>(v4, v5, v6, v7));
+    return make_uint2(cvt_f32x4_to_fp8x4<1>(v0, v1, v2, v3), cvt_f32x4_to_fp8x4<1>(v4, v5, v6, v7));
+}
+
 template <int MODE, int KG>
 __global__ void __launch_bounds__(256) postnorm_residual_kernel(const uint16_t *__restrict__ x,
                                                                 const uint16_t *__restrict__ y,
                                                                 const float *__restrict__ gamma, int D, float eps,
                                                                 uint16_t *__restrict__ out,
-                                                                unsigned int *__restrict__ amax_bits)
+                                                                unsigned int *__restrict__ amax_bits, float x_scale,
+                                                                const float *__restrict__ q_scale,
+                                                                uint8_t *__restrict__ out8, int fmt)
 {
     __shared__ float red[8];
+    const float qs = out8 ? __ldg(q_scale) : 1.0f;
     const size_t base = (size_t)blockIdx.x * D;
     const uint4 *py = reinterpret_cast<const uint4 *>(y + base);
     const uint4 *px = reinterpret_cast<const uint4 *>(x + base);
@@ -303,12 +319,13 @@ __global__ void __launch_bounds__(256) postnorm_residual_kernel(const uint16_t *
             uint32_t o[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const float lo = fmaf(g[2 * q] * rinv, bf16_lo(yw[q]), bf16_lo(xw[q]));
-                const float hi = fmaf(g[2 * q + 1] * rinv, bf16_hi(yw[q]), bf16_hi(xw[q]));
+                const float lo = fmaf(g[2 * q] * rinv, bf16_lo(yw[q]), x_scale * bf16_lo(xw[q]));
+                const float hi = fmaf(g[2 * q + 1] * rinv, bf16_hi(yw[q]), x_scale * bf16_hi(xw[q]));
                 o[q] = pack_bf16x2(lo, hi);
                 m = absmax2e(m, o[q]);
             }
             po[i] = make_uint4(o[0], o[1], o[2], o[3]);
+            if (out8) *reinterpret_cast<uint2 *>(out8 + base + (size_t)i * 8) = bf16x8_to_fp8x8(o, qs, fmt);
         }
     }
     if (amax_bits) block_max_bf16_to(m, amax_bits);
@@ -325,9 +342,12 @@ __global__ void __launch_bounds__(256) qk_norm_rope_kernel(const uint16_t *__res
                                                            float alpha, float eps, const float *__restrict__ cos_t,
                                                            const float *__restrict__ sin_t, int seq_len,
                                                            uint16_t *__restrict__ out,
-                                                           unsigned int *__restrict__ amax_bits)
+                                                           unsigned int *__restrict__ amax_bits,
+                                                           const float *__restrict__ q_scale,
+                                                           uint8_t *__restrict__ out8, int fmt)
 {
     constexpr int LPV = D / 16;             // lanes per vector: 8 (d = 128) or 4 (d = 64)
+    const float qs = out8 ? __ldg(q_scale) : 1.0f;
     constexpr int GPB = 256 / LPV;          // lane groups per CTA
     const int j = threadIdx.x % LPV;
     const int chunks = (H + QK_HC - 1) / QK_HC;
@@ -392,10 +412,15 @@ __global__ void __launch_bounds__(256) qk_norm_rope_kernel(const uint16_t *__res
                 ob[q] = pack_bf16x2(b[2 * q], b[2 * q + 1]);
                 if (valid) m = absmax2e(absmax2e(m, oa[q]), ob[q]);
             }
-            if (valid) {
+            if (valid && out) {
                 uint16_t *po = out + v * D + j * 8;
                 *reinterpret_cast<uint4 *>(po) = make_uint4(oa[0], oa[1], oa[2], oa[3]);
                 *reinterpret_cast<uint4 *>(po + D / 2) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+            }
+            if (valid && out8) {
+                uint8_t *p8 = out8 + v * D + j * 8;
+                *reinterpret_cast<uint2 *>(p8) = bf16x8_to_fp8x8(oa, qs, fmt);
+                *reinterpret_cast<uint2 *>(p8 + D / 2) = bf16x8_to_fp8x8(ob, qs, fmt);
             }
         }
     }
@@ -489,12 +514,21 @@ extern "C" int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float 
     return FP8_OK;
 }
 
-extern "C" int fp8_postnorm_residual(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D,
-                                     int mode, float eps, void *out_bf16, float *amax_out, void *stream)
+static int postnorm_common(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D, int mode,
+                           float eps, float x_scale, const float *q_scale, int fmt, void *out_bf16, uint8_t *out8,
+                           float *amax_out, void *stream)
 {
-    if (!x_bf16 || !y_bf16 || !gamma || !out_bf16) {
+    if (!x_bf16 || !y_bf16 || !gamma || !out_bf16 || (out8 && !q_scale)) {
         set_error("fp8_postnorm_residual: NULL pointer");
         return FP8_ERR_NULL;
+    }
+    if (out8 && fmt != FP8_E4M3 && fmt != FP8_E5M2) {
+        set_error("fp8_postnorm_residual_q: fmt %d is not FP8_E4M3 / FP8_E5M2", fmt);
+        return FP8_ERR_ENUM;
+    }
+    if (!aligned16(out8) || !(x_scale == x_scale)) {
+        set_error("fp8_postnorm_residual_q: out8 must be 16-byte aligned and x_scale a number");
+        return FP8_ERR_ALIGN;
     }
     if (mode != FP8_NORM_RMS && mode != FP8_NORM_LAYERSCALE) {
         set_error("fp8_postnorm_residual: mode %d is not FP8_NORM_RMS / FP8_NORM_LAYERSCALE", mode);
@@ -516,7 +550,7 @@ extern "C" int fp8_postnorm_residual(const void *x_bf16, const void *y_bf16, con
     uint16_t *o = static_cast<uint16_t *>(out_bf16);
     unsigned int *ab = reinterpret_cast<unsigned int *>(amax_out);
 #define FP8DPA_LAUNCH_PN(MM, KG) \
-    postnorm_residual_kernel<MM, KG><<<(unsigned)T, 256, 0, st>>>(x, y, gamma, (int)D, eps, o, ab)
+    postnorm_residual_kernel<MM, KG><<<(unsigned)T, 256, 0, st>>>(x, y, gamma, (int)D, eps, o, ab, x_scale, q_scale, out8, fmt)
 #define FP8DPA_LAUNCH_PN_KG(MM) \
     do { \
         if (D <= 2048) FP8DPA_LAUNCH_PN(MM, 1); \
@@ -532,13 +566,38 @@ extern "C" int fp8_postnorm_residual(const void *x_bf16, const void *y_bf16, con
     return FP8_OK;
 }
 
-extern "C" int fp8_qk_norm_rope(const void *x_bf16, size_t T, size_t H, size_t d, int mode, float alpha, float eps,
-                                const float *cos_table, const float *sin_table, size_t seq_len, void *out_bf16,
-                                float *amax_out, void *stream)
+extern "C" int fp8_postnorm_residual(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D,
+                                     int mode, float eps, void *out_bf16, float *amax_out, void *stream)
 {
-    if (!x_bf16 || !out_bf16 || ((cos_table == nullptr) != (sin_table == nullptr))) {
-        set_error("fp8_qk_norm_rope: NULL pointer (cos and sin tables come together)");
+    return postnorm_common(x_bf16, y_bf16, gamma, T, D, mode, eps, 1.0f, nullptr, 0, out_bf16, nullptr, amax_out, stream);
+}
+
+extern "C" int fp8_postnorm_residual_q(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D,
+                                       int mode, float eps, float x_scale, const float *scale, int fmt, void *out_bf16,
+                                       uint8_t *out8, float *amax_out, void *stream)
+{
+    if (!out8 || !scale) {
+        set_error("fp8_postnorm_residual_q: NULL scale / out8");
         return FP8_ERR_NULL;
+    }
+    return postnorm_common(x_bf16, y_bf16, gamma, T, D, mode, eps, x_scale, scale, fmt, out_bf16, out8, amax_out, stream);
+}
+
+static int qk_common(const void *x_bf16, size_t T, size_t H, size_t d, int mode, float alpha, float eps,
+                     const float *cos_table, const float *sin_table, size_t seq_len, const float *q_scale, int fmt,
+                     void *out_bf16, uint8_t *out8, float *amax_out, void *stream)
+{
+    if (!x_bf16 || (!out_bf16 && !out8) || ((cos_table == nullptr) != (sin_table == nullptr)) || (out8 && !q_scale)) {
+        set_error("fp8_qk_norm_rope: NULL pointer (cos and sin tables come together; FP8 output needs its scale)");
+        return FP8_ERR_NULL;
+    }
+    if (out8 && fmt != FP8_E4M3 && fmt != FP8_E5M2) {
+        set_error("fp8_qk_norm_rope_q: fmt %d is not FP8_E4M3 / FP8_E5M2", fmt);
+        return FP8_ERR_ENUM;
+    }
+    if (!aligned16(out8)) {
+        set_error("fp8_qk_norm_rope_q: out8 must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
     }
     if (mode < FP8_QK_RMS || mode > FP8_QK_NONE) {
         set_error("fp8_qk_norm_rope: mode %d is not FP8_QK_RMS / FP8_QK_TANH / FP8_QK_NONE", mode);
@@ -567,7 +626,7 @@ extern "C" int fp8_qk_norm_rope(const void *x_bf16, size_t T, size_t H, size_t d
     unsigned int *ab = reinterpret_cast<unsigned int *>(amax_out);
 #define FP8DPA_LAUNCH_QK(DD, MM) \
     qk_norm_rope_kernel<DD, MM><<<(unsigned)blocks, 256, 0, st>>>(x, T, (int)H, alpha, eps, cos_table, sin_table, \
-                                                                 (int)(seq_len ? seq_len : 1), o, ab)
+                                                                 (int)(seq_len ? seq_len : 1), o, ab, q_scale, out8, fmt)
     if (d == 128) {
         if (mode == FP8_QK_RMS) FP8DPA_LAUNCH_QK(128, FP8_QK_RMS);
         else if (mode == FP8_QK_TANH) FP8DPA_LAUNCH_QK(128, FP8_QK_TANH);
@@ -580,4 +639,28 @@ extern "C" int fp8_qk_norm_rope(const void *x_bf16, size_t T, size_t H, size_t d
 #undef FP8DPA_LAUNCH_QK
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
+}
+
+extern "C" int fp8_qk_norm_rope(const void *x_bf16, size_t T, size_t H, size_t d, int mode, float alpha, float eps,
+                                const float *cos_table, const float *sin_table, size_t seq_len, void *out_bf16,
+                                float *amax_out, void *stream)
+{
+    if (!out_bf16) {
+        set_error("fp8_qk_norm_rope: NULL output");
+        return FP8_ERR_NULL;
+    }
+    return qk_common(x_bf16, T, H, d, mode, alpha, eps, cos_table, sin_table, seq_len, nullptr, 0, out_bf16, nullptr,
+                     amax_out, stream);
+}
+
+extern "C" int fp8_qk_norm_rope_q(const void *x_bf16, size_t T, size_t H, size_t d, int mode, float alpha, float eps,
+                                  const float *cos_table, const float *sin_table, size_t seq_len, const float *scale,
+                                  int fmt, void *out_bf16, uint8_t *out8, float *amax_out, void *stream)
+{
+    if (!out8 || !scale) {
+        set_error("fp8_qk_norm_rope_q: NULL scale / out8");
+        return FP8_ERR_NULL;
+    }
+    return qk_common(x_bf16, T, H, d, mode, alpha, eps, cos_table, sin_table, seq_len, scale, fmt, out_bf16, out8,
+                     amax_out, stream);
 }

@@ -161,6 +161,62 @@ def test_qk_norm_rope_matches_oracle(mode, rope, T, H, d, N):
     assert float(a.item()) == float(o.amax(got))
 
 
+@pytest.mark.parametrize("mode,fmt,x_scale", [(o.NORM_RMS, o.E4M3, 1.0), (o.NORM_LAYERSCALE, o.E4M3, 1.0),
+                                               (o.NORM_RMS, o.E5M2, 1.0), (o.NORM_RMS, o.E4M3, 50.0)])
+@pytest.mark.parametrize("T,D", [(64, 2048), (100, 4096), (7, 264)])
+def test_postnorm_residual_producer_form_equals_unfused_chain(mode, fmt, x_scale, T, D):
+    """Delayed scaling: the same pass writes the FP8 codes of its result; they are the codes fp8_cast gives for the
+    BF16 output, the amax is that of the BF16 output, and the BF16 output matches the oracle (with the input factor)."""
+    c = synth.choose_columns(D, max(1, D // 200), 4, 1)
+    xb = synth.normal_bf16((T, D), 11, 1, 1.0 / x_scale, c, 20.0)
+    yb = synth.normal_bf16((T, D), 11, 2, 0.02, c, 20.0)
+    gamma = (np.full(D, 1.0 / np.sqrt(32.0)) * (1.0 + 0.01 * np.arange(D) / D)).astype(np.float32)
+    gd = torch.from_numpy(gamma).cuda()
+    exp = o.postnorm_residual(xb, yb, gamma, mode, 1e-5, x_scale)
+    sc = scalar(3.7)                                           # a "history" scale, not the tensor's own
+    out = torch.empty((T, D), dtype=torch.int16, device="cuda")
+    out8 = torch.full((T, D), 0x55, dtype=torch.uint8, device="cuda")
+    a = scalar(-1.0)
+    fp8.fp8_postnorm_residual_q(dev(xb), dev(yb), gd, mode, 1e-5, sc, fmt, out, out8, a, x_scale=x_scale)
+    torch.cuda.synchronize()
+    got = host(out).view(np.uint16)
+    bf16_close(got, exp)
+    assert float(a.item()) == float(o.amax(got))
+    assert np.array_equal(host(out8), o.cast(got, np.float32(3.7), fmt))      # the oracle's cast of the same BF16 values
+    if D % 16 == 0:                                                               # (fp8_cast wants whole 16-byte rows)
+        ref8 = torch.empty_like(out8)
+        fp8.fp8_cast(out.view(torch.bfloat16), sc, fmt, ref8)                    # and the library's own unfused chain
+        assert torch.equal(out8, ref8)
+    if x_scale == 1.0:
+        plain = torch.empty_like(out)
+        fp8.fp8_postnorm_residual(dev(xb), dev(yb), gd, mode, 1e-5, plain, None)
+        assert torch.equal(plain, out)
+
+
+@pytest.mark.parametrize("mode,fmt", [(o.QK_RMS, o.E4M3), (o.QK_TANH, o.E4M3), (o.QK_NONE, o.E5M2)])
+@pytest.mark.parametrize("T,H,d,N", [(256, 8, 128, 64), (96, 4, 64, 32), (33, 3, 128, 11)])
+def test_qk_norm_rope_producer_form_equals_unfused_chain(mode, fmt, T, H, d, N):
+    xb = synth.normal_bf16((T, H * d), 13, 3, 1.5).reshape(T, H, d)
+    inv = 10000.0 ** (-np.arange(d // 2) * 2.0 / d)
+    ang = np.arange(N)[:, None] * inv[None]
+    cos, sin = torch.from_numpy(np.cos(ang).astype(np.float32)).cuda(), torch.from_numpy(np.sin(ang).astype(np.float32)).cuda()
+    plain = torch.empty((T, H, d), dtype=torch.int16, device="cuda")
+    a0 = scalar(-1.0)
+    fp8.fp8_qk_norm_rope(dev(xb), mode, 0.5, 1e-6, cos, sin, N, plain, a0)
+    sc = scalar(100.0)
+    out = torch.empty_like(plain)
+    out8 = torch.full((T, H, d), 0x55, dtype=torch.uint8, device="cuda")
+    a = scalar(-1.0)
+    fp8.fp8_qk_norm_rope_q(dev(xb), mode, 0.5, 1e-6, cos, sin, N, sc, fmt, out, out8, a)
+    torch.cuda.synchronize()
+    assert torch.equal(out, plain) and float(a.item()) == float(a0.item())
+    assert np.array_equal(host(out8), o.cast(host(out).view(np.uint16), np.float32(100.0), fmt))
+    # codes only
+    only8 = torch.full((T, H, d), 0x55, dtype=torch.uint8, device="cuda")
+    fp8.fp8_qk_norm_rope_q(dev(xb), mode, 0.5, 1e-6, cos, sin, N, sc, fmt, None, only8, None)
+    assert torch.equal(only8, out8)
+
+
 def test_glue_argument_validation():
     x = dev(synth.normal_bf16((8, 64), 0, 0, 1.0))
     g = torch.ones(64, device="cuda")

@@ -113,6 +113,26 @@ def test_postnorm_residual_closed_forms():
     assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-30)
 
 
+def test_postnorm_residual_input_scaling():
+    """x_scale multiplies the residual input only (the first block's input is scaled by sigma_0^-1, Section 3)."""
+    D = 64
+    g = np.full(D, 0.5, dtype=np.float32)
+    xx, yy = synth.normal_bf16((8, D), 3, 6, 1.0), synth.normal_bf16((8, D), 3, 7, 1.0)
+    # factor 1 is the plain form
+    assert np.array_equal(o.postnorm_residual(xx, yy, g, o.NORM_RMS, 1e-5, 1.0), o.postnorm_residual(xx, yy, g, o.NORM_RMS, 1e-5))
+    # zero branch output: out = BF16(u x); a power of two is exact
+    zero = bf16(np.zeros((8, D)))
+    out = synth.bf16_to_f32(o.postnorm_residual(xx, zero, g, o.NORM_LAYERSCALE, 0.0, 4.0))
+    assert np.array_equal(out, 4.0 * synth.bf16_to_f32(xx))
+    out = synth.bf16_to_f32(o.postnorm_residual(xx, zero, g, o.NORM_LAYERSCALE, 0.0, 1.0 / 0.02))
+    assert np.array_equal(out, synth.bf16_to_f32(bf16(synth.bf16_to_f32(xx).astype(np.float64) * 50.0)))
+    # the factor does not touch the branch: u x + gamma y / rms(y) against numpy
+    xf, yf = synth.bf16_to_f32(xx).astype(np.float64), synth.bf16_to_f32(yy).astype(np.float64)
+    ref = 50.0 * xf + 0.5 * yf / np.sqrt((yf ** 2).mean(axis=1, keepdims=True))
+    got = synth.bf16_to_f32(o.postnorm_residual(xx, yy, g, o.NORM_RMS, 0.0, 50.0))
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-30)
+
+
 def test_qk_norm_rope_closed_forms():
     T, H, d, N = 6, 2, 64, 3
     q = synth.normal_bf16((T, H * d), 5, 6, 2.0).reshape(T, H, d)
