@@ -610,6 +610,9 @@ def run_report(args):
         add(f"fp8_act_cast {name} (single pass: cast + amax under a delayed scale)", f"{T}x{F}",
             timed(lambda: fp8.fp8_act_cast(xa, act, par, sc, 0, h8, None, a)), nbytes=3 * T * F)
     add("fp8_kurtosis", f"{T}x{2 * F}", timed(lambda: fp8.fp8_kurtosis(x, a)), nbytes=2 * T * 2 * F)
+    kk = f32()
+    add("fp8_amax_kurtosis (amax + kurtosis, one pass)", f"{T}x{2 * F}", timed(lambda: fp8.fp8_amax_kurtosis(x, a, kk)),
+        nbytes=2 * T * 2 * F)
     del x, q, qt, h8, h8t, xa
     r, y, g = bf16(2 * T, H), bf16(2 * T, H, std=0.02), torch.ones(H, device="cuda")
     o_ = torch.empty_like(r)

@@ -165,6 +165,12 @@ FP8_API int fp8_qk_norm_rope_q(const void *x_bf16, size_t T, size_t H, size_t d,
  * (un-centred; rows are token vectors).  *out is overwritten.  cols % 8 == 0. */
 FP8_API int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *out, void *stream);
 
+/* The monitor folded into the amax pass of a just-in-time quantisation (Section 4 tracks the kurtosis of tensors
+ * that are quantised anyway: FFN-2 input, QKV output, block output; Appendix C: s(x) = MaxFP8Value / absmax(x)):
+ * one read of x gives *amax = max |x| (as fp8_amax, bit-exact) and *kurtosis (as fp8_kurtosis).  Both device
+ * scalars are overwritten.  cols % 8 == 0. */
+FP8_API int fp8_amax_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *amax, float *kurtosis, void *stream);
+
 /* ---- linear layers --------------------------------------------------------------------------------
  * Appendix E: GEMM(X,Y) = 1/(rho_X rho_Y) * FP8GEMM(FP8cast(rho_X X), FP8cast(rho_Y Y)), BF16 result;
  * Table "Comparison between FP8 methods": Linear_W(X) = XW for the FFN, QKV and output projections.

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
-           "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis",
+           "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis", "fp8_amax_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
@@ -179,6 +179,13 @@ def fp8_swiglu_cast(gate_up, scale, fmt, out, out_t=None, amax_out=None, stream=
 def fp8_kurtosis(x, out, stream=None):
     rows, cols = _rows_cols(x)
     _check(load().fp8_kurtosis(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), _ptr(out), _stream(stream)))
+
+
+def fp8_amax_kurtosis(x, amax, kurtosis, stream=None):
+    """amax and the kurtosis monitor of a [rows, cols] BF16 tensor from one read of it."""
+    rows, cols = _rows_cols(x)
+    _check(load().fp8_amax_kurtosis(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), _ptr(amax), _ptr(kurtosis),
+                                    _stream(stream)))
 
 
 def _is_fp32(t):

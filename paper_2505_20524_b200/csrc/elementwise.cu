@@ -210,15 +210,18 @@ __global__ void __launch_bounds__(256) act_cast_kernel(const uint16_t *__restric
 }
 
 // One CTA per row: sums of x^2 and x^4, then kurt = mean(x^4) / mean(x^2)^2 added (scaled by 1/rows) to *out.
+// With amax_bits the same pass also takes the tensor's amax (the pass a just-in-time quantisation makes anyway).
 __global__ void __launch_bounds__(256) kurtosis_kernel(const uint16_t *__restrict__ x, int cols, float inv_rows,
-                                                       float *__restrict__ out)
+                                                       float *__restrict__ out, unsigned int *__restrict__ amax_bits)
 {
     __shared__ float red2[8], red4[8];
     const uint4 *row = reinterpret_cast<const uint4 *>(x + (size_t)blockIdx.x * cols);
     float s2 = 0.0f, s4 = 0.0f;
+    uint32_t m = 0;
     for (int i = threadIdx.x; i < cols / 8; i += blockDim.x) {
         const uint4 v = __ldg(row + i);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        m = absmax2e(absmax2e(absmax2e(absmax2e(m, v.x), v.y), v.z), v.w);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const float a = bf16_lo(w[k]), b = bf16_hi(w[k]);
@@ -245,6 +248,7 @@ __global__ void __launch_bounds__(256) kurtosis_kernel(const uint16_t *__restric
             atomicAdd(out, m4 / (m2 * m2) * inv_rows);
         }
     }
+    if (amax_bits) block_max_bf16_to(m, amax_bits);
 }
 
 // Post-norm + residual, one CTA per token row.  The row of y stays in registers between the sum of squares and the
@@ -490,7 +494,7 @@ extern "C" int fp8_act_cast(const void *x_bf16, size_t T, size_t F, int act, con
     return act_cast("fp8_act_cast", x_bf16, T, F, act, act_params, scale, fmt, out, out_t, amax_out, stream);
 }
 
-extern "C" int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *out, void *stream)
+static int kurtosis_common(const void *x_bf16, size_t rows, size_t cols, float *out, float *amax_out, void *stream)
 {
     if (!x_bf16 || !out) {
         set_error("fp8_kurtosis: NULL pointer");
@@ -508,10 +512,25 @@ extern "C" int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float 
     if (rc != FP8_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     FP8_CUDA_CHECK(cudaMemsetAsync(out, 0, sizeof(float), st));
+    if (amax_out) FP8_CUDA_CHECK(cudaMemsetAsync(amax_out, 0, sizeof(float), st));
     kurtosis_kernel<<<(unsigned)rows, 256, 0, st>>>(static_cast<const uint16_t *>(x_bf16), (int)cols,
-                                                   1.0f / (float)rows, out);
+                                                   1.0f / (float)rows, out, reinterpret_cast<unsigned int *>(amax_out));
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
+}
+
+extern "C" int fp8_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *out, void *stream)
+{
+    return kurtosis_common(x_bf16, rows, cols, out, nullptr, stream);
+}
+
+extern "C" int fp8_amax_kurtosis(const void *x_bf16, size_t rows, size_t cols, float *amax, float *kurtosis, void *stream)
+{
+    if (!amax) {
+        set_error("fp8_amax_kurtosis: NULL amax");
+        return FP8_ERR_NULL;
+    }
+    return kurtosis_common(x_bf16, rows, cols, kurtosis, amax, stream);
 }
 
 static int postnorm_common(const void *x_bf16, const void *y_bf16, const float *gamma, size_t T, size_t D, int mode,

@@ -30,6 +30,21 @@ def neighbours(code, ref, fmt):
     return np.abs(rank[code] - rank[ref]) <= 2            # +0 and -0 sit next to each other in the ordering
 
 
+def test_amax_and_kurtosis_from_one_pass():
+    """The monitor folded into the amax pass: amax bit-exact as fp8_amax, kurtosis as fp8_kurtosis."""
+    for rows, cols in ((64, 4096), (1000, 264), (8192, 2048)):
+        c = synth.choose_columns(cols, max(1, cols // 100), 6, 1)
+        xb = synth.normal_bf16((rows, cols), 14, 1, 1.0, c, 30.0)
+        a, k, k0 = scalar(-1.0), scalar(-1.0), scalar(-1.0)
+        fp8.fp8_amax_kurtosis(dev(xb), a, k)
+        fp8.fp8_kurtosis(dev(xb), k0)
+        torch.cuda.synchronize()
+        assert float(a.item()) == float(o.amax(xb))
+        ref = o.kurtosis(xb)
+        assert abs(float(k.item()) - ref) <= 2e-5 * ref
+        assert abs(float(k.item()) - float(k0.item())) <= 1e-5 * ref
+
+
 @pytest.mark.parametrize("fmt", [o.E4M3, o.E5M2])
 @pytest.mark.parametrize("T,F", [(256, 1024), (144, 272), (1024, 5632)])
 def test_swiglu_cast_matches_oracle(fmt, T, F):
