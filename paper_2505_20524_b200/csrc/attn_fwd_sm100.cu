@@ -63,9 +63,40 @@ struct AttnFwdParams {
     unsigned int *o_amax_bits;   // nullable
 };
 
+// 2^t for two values at once on the FMA pipe instead of the exponential unit: t = n + f with n the nearest integer
+// (adding 1.5 * 2^23 leaves n in the low mantissa bits) and |f| <= 1/2, 2^f from a degree-5 polynomial (interpolated at
+// Chebyshev nodes; relative error 2.9e-7 = 2^-21.7 in binary32 Horner form, the accuracy class of ex2.approx), the
+// exponent n added to the result's bit pattern.  t is clamped at -126 so that the result stays a normal number
+// (anything below 2^-10 rounds to the zero code of P8 anyway and adds nothing visible to the row sum).
+__device__ __forceinline__ void exp2_poly_x2(uint64_t t2, float &ea, float &eb)
+{
+    float ta, tb;
+    unpack_f32x2(t2, ta, tb);
+    ta = fmaxf(ta, -126.0f);
+    tb = fmaxf(tb, -126.0f);
+    const uint64_t tc = pack_f32x2(ta, tb);
+    const uint64_t magic = pack_f32x2(12582912.0f, 12582912.0f), nmagic = pack_f32x2(-12582912.0f, -12582912.0f);
+    const uint64_t r2 = add_f32x2(tc, magic);
+    const uint64_t n2 = add_f32x2(r2, nmagic);
+    const uint64_t f2 = fma_f32x2(n2, pack_f32x2(-1.0f, -1.0f), tc);
+    uint64_t p2 = pack_f32x2(0.0013390866806730628f, 0.0013390866806730628f);
+    p2 = fma_f32x2(p2, f2, pack_f32x2(0.009666373953223228f, 0.009666373953223228f));
+    p2 = fma_f32x2(p2, f2, pack_f32x2(0.055503569543361664f, 0.055503569543361664f));
+    p2 = fma_f32x2(p2, f2, pack_f32x2(0.2402234822511673f, 0.2402234822511673f));
+    p2 = fma_f32x2(p2, f2, pack_f32x2(0.6931471824645996f, 0.6931471824645996f));
+    p2 = fma_f32x2(p2, f2, pack_f32x2(1.0f, 1.0f));
+    float pa, pb, ra, rb;
+    unpack_f32x2(p2, pa, pb);
+    unpack_f32x2(r2, ra, rb);
+    ea = __uint_as_float(__float_as_uint(pa) + (__float_as_uint(ra) << 23));
+    eb = __uint_as_float(__float_as_uint(pb) + (__float_as_uint(rb) << 23));
+}
+
 // One 32-column chunk of a score row -> 32 values of c_P * P~ = 2^(c*S - shift), their sum, and 32 E4M3 codes.
 // MASK: columns beyond `limit` (relative to the chunk start) contribute exactly 0.
-template <bool MASK>
+// POLY: one pair of columns in every POLY pairs takes its exponentials on the FMA pipe (0: none); the exponential unit
+// does 16 per clock and SM against 32 scores per clock from the FP8 tensor pipe, so it is the scarcer of the two.
+template <bool MASK, int POLY = 0>
 __device__ __forceinline__ float softmax_chunk(const uint32_t (&v)[32], float c, float neg_shift, int limit,
                                                uint32_t (&w)[8])
 {
@@ -73,10 +104,15 @@ __device__ __forceinline__ float softmax_chunk(const uint32_t (&v)[32], float c,
     float e[32];
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
-        float a, b;
-        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, s2), a, b);
-        e[i] = ex2_approx(a);
-        e[i + 1] = ex2_approx(b);
+        const uint64_t t2 = fma_f32x2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), c2, s2);
+        if (POLY > 0 && !MASK && ((i / 2) % POLY) == POLY - 1) {
+            exp2_poly_x2(t2, e[i], e[i + 1]);
+        } else {
+            float a, b;
+            unpack_f32x2(t2, a, b);
+            e[i] = ex2_approx(a);
+            e[i + 1] = ex2_approx(b);
+        }
         if (MASK) {
             if (i > limit) e[i] = 0.0f;
             if (i + 1 > limit) e[i + 1] = 0.0f;
@@ -402,6 +438,14 @@ constexpr int P_THREADS = 512;
 constexpr int P_STAGES = 4;
 constexpr int P_REGS_SOFTMAX = 184, P_REGS_CORR = 80, P_REGS_CTRL = 64;   // 2*128*184 + 128*80 + 128*64 = 65536
 constexpr int P_TMEM_COLS = 512;
+// Share of the exponentials evaluated on the FMA pipe: one pair of score columns in FP8DPA_FWD_POLY (0 = none, the
+// default).  Measured at N = 16384: 0 -> 1.70 ms, 8 -> 1.72, 4 -> 2.02, 2 -> 1.98: the softmax warps are bound by
+// instruction issue and dependent-issue latency, not by the exponential unit, so the extra instructions cost more than the
+// unit's relief returns.
+#ifndef FP8DPA_FWD_POLY
+#define FP8DPA_FWD_POLY 0
+#endif
+constexpr int P_POLY = FP8DPA_FWD_POLY;
 
 struct AttnFwdPairSmem {
     static constexpr int D = 128;
@@ -654,7 +698,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 uint32_t wq[8];
-                lsum += softmax_chunk<MASK>(sv[q], c, neg_shift, limit - q * 32, wq);
+                lsum += softmax_chunk<MASK, P_POLY>(sv[q], c, neg_shift, limit - q * 32, wq);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) w[q * 8 + e] = wq[e];
             }
