@@ -665,10 +665,21 @@ def run_report(args):
                 sw = torch.full(((N + 127) // 128, K // 128), 1e-2, device="cuda")
                 add("fp8_linear_fwd_blockwise", f"{cname} {layer} {Tt}x{N}x{K}",
                     timed(lambda: fp8.fp8_linear_fwd_blockwise(x8, w8, sx, sw, yb)), flops=fl)
+                if N % 128 == 0:
+                    sdy = torch.full((N // 128, Tt), 1e-2, device="cuda")
+                    add("fp8_linear_dgrad_blockwise (W8 and its block scales read in place)", f"{cname} {layer} {Tt}x{N}x{K}",
+                        timed(lambda: fp8.fp8_linear_dgrad_blockwise(dy8, w8, sdy, sw, dxb)), flops=fl)
+                    del sdy
+                sdt = torch.full(((Tt + 127) // 128, N), 1e-2, device="cuda")
+                sxt = torch.full(((Tt + 127) // 128, K), 1e-2, device="cuda")
+                add("fp8_linear_wgrad_blockwise (128x1 blocks, operands read in place)", f"{cname} {layer} {Tt}x{N}x{K}",
+                    timed(lambda: fp8.fp8_linear_wgrad_blockwise(dy8, x8, sdt, sxt, dwb)), flops=fl)
                 xb = bf16(Tt, K)
                 add("fp8_quantize_blockwise 1x128", f"{Tt}x{K}", timed(lambda: fp8.fp8_quantize_blockwise(xb, 1, 0, x8, sx)),
                     nbytes=3 * Tt * K)
-                del xb, y8, sx, sw
+                add("fp8_quantize_blockwise 128x1", f"{Tt}x{K}",
+                    timed(lambda: fp8.fp8_quantize_blockwise(xb, fp8.FP8_BLOCK_128x1, 0, x8, sxt)), nbytes=3 * Tt * K)
+                del xb, y8, sx, sw, sdt, sxt
             del x8, w8, dy8, x8t, w8t, dy8t, yb, dxb, dwb
 
     # ---- grouped (mixture-of-experts) forward product: 8 experts, 2 active, c3-sized FFN

@@ -250,12 +250,26 @@ FP8_API int fp8_linear_dgrad_q(const uint8_t *dY8, const uint8_t *W8t, const flo
  * fp8_quantize_blockwise: x [rows, cols] BF16 -> out [rows, cols] codes, one pass.  block_rows = 1: 1 x 128 blocks,
  * scale_inv laid out K-block-major, [cols/128][rows] (the order the product reads it in).  block_rows = 128:
  * 128 x 128 blocks, scale_inv [ceil(rows/128)][cols/128].  cols % 128 == 0.  Inputs are finite.
+ * block_rows = FP8_BLOCK_128x1: blocks of 128 consecutive rows of one column (what the weight-gradient product needs,
+ * whose reduction runs over the token rows), scale_inv [ceil(rows/128)][cols].
  * fp8_linear_fwd_blockwise: Y[t,n] = sum_kb sx_inv[kb][t] * sw_inv[n/128][kb] * sum_{k in kb} X8[t,k] W8[n,k], BF16
- * result; X8 [T,K], W8 [N,K] in E4M3; K % 128 == 0, N % 16 == 0. */
+ * result; X8 [T,K], W8 [N,K] in E4M3; K % 128 == 0, N % 16 == 0.
+ * fp8_linear_dgrad_blockwise: dX[t,k] = sum_nb sdy_inv[nb][t] * sw_inv[nb][k/128] * sum_{n in nb} dY8[t,n] W8[n,k];
+ * dY8 [T,N] E5M2 quantised in 1 x 128 blocks (scales [N/128][T]), W8 [N,K] and its 128 x 128 scales exactly as the
+ * forward uses them (read in place, no transposed copy); N % 128 == 0, K % 128 == 0.
+ * fp8_linear_wgrad_blockwise: dW[n,k] = sum_tb sdy_inv_t[tb][n] * sx_inv_t[tb][k] * sum_{t in tb} dY8[t,n] X8[t,k];
+ * dY8 [T,N] E5M2 and X8 [T,K] E4M3 both quantised in 128 x 1 blocks (FP8_BLOCK_128x1), read in place; BF16 result
+ * [N,K]; N % 16 == 0, K % 16 == 0, T arbitrary (the last block of tokens may be short).
+ * (Appendix E, throughput table: the recipe's cost is measured over a whole training step, forward and backward.) */
+#define FP8_BLOCK_128x1 (-128)
 FP8_API int fp8_quantize_blockwise(const void *x_bf16, size_t rows, size_t cols, int block_rows, int fmt,
                            uint8_t *out, float *scale_inv, void *stream);
 FP8_API int fp8_linear_fwd_blockwise(const uint8_t *X8, const uint8_t *W8, const float *sx_inv, const float *sw_inv,
                              void *Y_bf16, int T, int N, int K, void *stream);
+FP8_API int fp8_linear_dgrad_blockwise(const uint8_t *dY8, const uint8_t *W8, const float *sdy_inv, const float *sw_inv,
+                               void *dX_bf16, int T, int N, int K, void *stream);
+FP8_API int fp8_linear_wgrad_blockwise(const uint8_t *dY8, const uint8_t *X8, const float *sdy_inv_t,
+                               const float *sx_inv_t, void *dW_bf16, int T, int N, int K, void *stream);
 
 /* ---- attention ------------------------------------------------------------------------------------
  * Appendix B, Eq. (P): P = Softmax(s Q K^T + M), output P V, grouped-query heads; Appendix E table: both

@@ -299,6 +299,43 @@ def linear_fwd_blockwise(x8, w8, sx_inv, sw_inv, bk=128, bn=128, rows=None, cols
     return ref, mag
 
 
+def linear_dgrad_blockwise(dy8, w8, sdy_inv, sw_inv, bn=128, bk=128, rows=None, cols=None):
+    """dX with one descale per (row, N-block) of dY and per (bn x bk) block of W; returns (ref, mag) on rows x cols."""
+    dy8, w8 = _c(dy8, np.uint8), _c(w8, np.uint8)
+    T, N = dy8.shape
+    K = w8.shape[1]
+    sdy, sw = _c(sdy_inv, np.float32), _c(sw_inv, np.float32)
+    assert sdy.shape == (T, (N + bn - 1) // bn) and sw.shape == ((N + bn - 1) // bn, (K + bk - 1) // bk)
+    r = np.arange(T, dtype=np.int64) if rows is None else _c(rows, np.int64)
+    c = np.arange(K, dtype=np.int64) if cols is None else _c(cols, np.int64)
+    ref = np.empty((r.size, c.size), dtype=np.float64)
+    mag = np.empty_like(ref)
+    f = _L().oracle_linear_dgrad_blockwise
+    f.restype = None
+    f(_p(dy8), _p(w8), _p(sdy), _p(sw), C.c_int64(T), C.c_int64(N), C.c_int64(K), C.c_int64(bn), C.c_int64(bk),
+      _p(r), C.c_int64(r.size), _p(c), C.c_int64(c.size), _p(ref), _p(mag))
+    return ref, mag
+
+
+def linear_wgrad_blockwise(dy8, x8, sdy_inv_t, sx_inv_t, bt=128, rows=None, cols=None):
+    """dW with one descale per (token block, channel) of dY and of X; returns (ref, mag) on rows x cols of [N, K]."""
+    dy8, x8 = _c(dy8, np.uint8), _c(x8, np.uint8)
+    T, N = dy8.shape
+    K = x8.shape[1]
+    sdy, sx = _c(sdy_inv_t, np.float32), _c(sx_inv_t, np.float32)
+    ntb = (T + bt - 1) // bt
+    assert sdy.shape == (ntb, N) and sx.shape == (ntb, K)
+    r = np.arange(N, dtype=np.int64) if rows is None else _c(rows, np.int64)
+    c = np.arange(K, dtype=np.int64) if cols is None else _c(cols, np.int64)
+    ref = np.empty((r.size, c.size), dtype=np.float64)
+    mag = np.empty_like(ref)
+    f = _L().oracle_linear_wgrad_blockwise
+    f.restype = None
+    f(_p(dy8), _p(x8), _p(sdy), _p(sx), C.c_int64(T), C.c_int64(N), C.c_int64(K), C.c_int64(bt),
+      _p(r), C.c_int64(r.size), _p(c), C.c_int64(c.size), _p(ref), _p(mag))
+    return ref, mag
+
+
 # ---------------------------------------------------------------- attention
 def attn_params(B, N, Hq, Hkv, d, causal=True, quant=True, kv_block=0, max_mode=0, s=None, c_P=448.0,
                 q_inv=1.0, k_inv=1.0, v_inv=1.0, do_inv=1.0, ds_scale=1.0, flip_eps=0.0, max_slack=0.0) -> AttnParams:

@@ -880,3 +880,73 @@ void oracle_linear_fwd_blockwise(const uint8_t *X8, const uint8_t *W8, const flo
             mag[i * ncols + j] = am;
         }
 }
+
+/* Data gradient of the same recipe (Appendix E measures the recipe over whole training steps, forward and backward):
+ * dX[t,k] = sum over N-blocks nb of sdy_inv[t,nb] * sw_inv[nb, k/bk] * sum_{n in nb} dec(dY8[t,n]) dec(W8[n,k]).
+ * dY8: [T,N] E5M2 codes quantised in 1 x bn blocks, sdy_inv [T, N/bn]; W8: [N,K] E4M3 in bn x bk blocks, sw_inv
+ * [N/bn, K/bk] (the forward's own weight blocks, now cut along the reduction index). */
+void oracle_linear_dgrad_blockwise(const uint8_t *dY8, const uint8_t *W8, const float *sdy_inv, const float *sw_inv,
+                                   int64_t T, int64_t N, int64_t K, int64_t bn, int64_t bk,
+                                   const int64_t *rows, int64_t nrows, const int64_t *cols, int64_t ncols,
+                                   double *ref, double *mag)
+{
+    double t5[256], t4[256];
+    oracle_fp8_decode_table(ORACLE_E5M2, t5);
+    oracle_fp8_decode_table(ORACLE_E4M3, t4);
+    int64_t nnb = (N + bn - 1) / bn, nkb = (K + bk - 1) / bk;
+    (void)T;
+#pragma omp parallel for schedule(static)
+    for (long i = 0; i < (long)nrows; ++i)
+        for (int64_t j = 0; j < ncols; ++j) {
+            int64_t t = rows[i], k = cols[j];
+            double acc = 0.0, am = 0.0;
+            for (int64_t nb = 0; nb < nnb; ++nb) {
+                double part = 0.0, pm = 0.0;
+                int64_t n1 = (nb + 1) * bn < N ? (nb + 1) * bn : N;
+                for (int64_t n = nb * bn; n < n1; ++n) {
+                    double a = t5[dY8[t * N + n]], b = t4[W8[n * K + k]];
+                    part += a * b;
+                    pm += fabs(a * b);
+                }
+                double sc = (double)sdy_inv[t * nnb + nb] * (double)sw_inv[nb * nkb + k / bk];
+                acc += sc * part;
+                am += sc * pm;
+            }
+            ref[i * ncols + j] = acc;
+            mag[i * ncols + j] = am;
+        }
+}
+
+/* Weight gradient: the reduction runs over tokens, so both operands are quantised in bt x 1 blocks (bt consecutive
+ * tokens of one channel): dW[n,k] = sum over token blocks tb of sdy_inv_t[tb,n] * sx_inv_t[tb,k] *
+ * sum_{t in tb} dec(dY8[t,n]) dec(X8[t,k]).  sdy_inv_t: [ceil(T/bt), N]; sx_inv_t: [ceil(T/bt), K]. */
+void oracle_linear_wgrad_blockwise(const uint8_t *dY8, const uint8_t *X8, const float *sdy_inv_t, const float *sx_inv_t,
+                                   int64_t T, int64_t N, int64_t K, int64_t bt,
+                                   const int64_t *rows, int64_t nrows, const int64_t *cols, int64_t ncols,
+                                   double *ref, double *mag)
+{
+    double t5[256], t4[256];
+    oracle_fp8_decode_table(ORACLE_E5M2, t5);
+    oracle_fp8_decode_table(ORACLE_E4M3, t4);
+    int64_t ntb = (T + bt - 1) / bt;
+#pragma omp parallel for schedule(static)
+    for (long i = 0; i < (long)nrows; ++i)
+        for (int64_t j = 0; j < ncols; ++j) {
+            int64_t n = rows[i], k = cols[j];
+            double acc = 0.0, am = 0.0;
+            for (int64_t tb = 0; tb < ntb; ++tb) {
+                double part = 0.0, pm = 0.0;
+                int64_t t1 = (tb + 1) * bt < T ? (tb + 1) * bt : T;
+                for (int64_t t = tb * bt; t < t1; ++t) {
+                    double a = t5[dY8[t * N + n]], b = t4[X8[t * K + k]];
+                    part += a * b;
+                    pm += fabs(a * b);
+                }
+                double sc = (double)sdy_inv_t[tb * N + n] * (double)sx_inv_t[tb * K + k];
+                acc += sc * part;
+                am += sc * pm;
+            }
+            ref[i * ncols + j] = acc;
+            mag[i * ncols + j] = am;
+        }
+}

@@ -14,6 +14,7 @@ import torch
 
 E4M3 = 0
 E5M2 = 1
+FP8_BLOCK_128x1 = -128        # block_rows value of fp8_quantize_blockwise: 128 consecutive rows of one column
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
@@ -21,7 +22,7 @@ _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis", "fp8_amax_kurtosis",
-           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_attention_workspace_bytes",
+           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_linear_dgrad_blockwise", "fp8_linear_wgrad_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
 
 STATIC_SCRATCH_BYTES = 32 << 20
@@ -268,7 +269,8 @@ def fp8_grouped_linear_wgrad(dy8, x8, sdy_inv, sx_inv, group_offsets_host, dw, a
 
 
 def fp8_quantize_blockwise(x, block_rows, fmt, out, scale_inv, stream=None):
-    """Block-by-block quantisation: 1 x 128 (scale_inv [cols/128, rows]) or 128 x 128 (scale_inv [rows/128, cols/128])."""
+    """Block-by-block quantisation: 1 x 128 (scale_inv [cols/128, rows]), 128 x 128 (scale_inv [rows/128, cols/128])
+    or, with block_rows = FP8_BLOCK_128x1, 128 x 1 (scale_inv [ceil(rows/128), cols])."""
     rows, cols = x.shape
     _check(load().fp8_quantize_blockwise(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), C.c_int(block_rows), C.c_int(fmt),
                                          _ptr(out), _ptr(scale_inv), _stream(stream)))
@@ -279,6 +281,22 @@ def fp8_linear_fwd_blockwise(x8, w8, sx_inv, sw_inv, y, stream=None):
     N = w8.shape[0]
     _check(load().fp8_linear_fwd_blockwise(_ptr(x8), _ptr(w8), _ptr(sx_inv), _ptr(sw_inv), _ptr(y), C.c_int(T),
                                            C.c_int(N), C.c_int(K), _stream(stream)))
+
+
+def fp8_linear_dgrad_blockwise(dy8, w8, sdy_inv, sw_inv, dx, stream=None):
+    """dX = dY W under the blockwise recipe: dy8 [T,N] in 1 x 128 blocks, w8 [N,K] in the forward's 128 x 128 blocks."""
+    T, N = dy8.shape
+    K = w8.shape[1]
+    _check(load().fp8_linear_dgrad_blockwise(_ptr(dy8), _ptr(w8), _ptr(sdy_inv), _ptr(sw_inv), _ptr(dx), C.c_int(T),
+                                             C.c_int(N), C.c_int(K), _stream(stream)))
+
+
+def fp8_linear_wgrad_blockwise(dy8, x8, sdy_inv_t, sx_inv_t, dw, stream=None):
+    """dW = dY^T X under the blockwise recipe: both operands in 128 x 1 blocks along the token axis."""
+    T, N = dy8.shape
+    K = x8.shape[1]
+    _check(load().fp8_linear_wgrad_blockwise(_ptr(dy8), _ptr(x8), _ptr(sdy_inv_t), _ptr(sx_inv_t), _ptr(dw), C.c_int(T),
+                                             C.c_int(N), C.c_int(K), _stream(stream)))
 
 
 def fp8_linear_dgrad(dy8, w8t, sdy_inv, sw_inv, dx, ws=None, stream=None):

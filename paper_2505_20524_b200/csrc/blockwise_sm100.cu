@@ -118,6 +118,62 @@ __global__ void __launch_bounds__(256) quantize_128x128_kernel(const uint16_t *_
     }
 }
 
+// 128 x 1 blocks (128 consecutive rows of one column; the layout the weight-gradient product needs, whose reduction
+// runs over the rows): one CTA per 128 x 128 tile as above, column maxima combined through shared memory.
+// scale_inv: [ceil(R/128)][C].
+template <int FMT>
+__global__ void __launch_bounds__(256) quantize_128x1_kernel(const uint16_t *__restrict__ x, int R, int C,
+                                                             uint8_t *__restrict__ out, float *__restrict__ scale_inv)
+{
+    __shared__ uint4 col_max[16][16];                 // [row group][column group]: packed maxima of 8 columns
+    const int r0 = blockIdx.y * 128, c0 = blockIdx.x * 128;
+    const int rg = threadIdx.x >> 4, cg = threadIdx.x & 15;
+    uint4 v[8];
+    uint4 m = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int r = r0 + k * 16 + rg, c = c0 + cg * 8;
+        v[k] = make_uint4(0, 0, 0, 0);
+        if (r < R) v[k] = __ldg(reinterpret_cast<const uint4 *>(x + (size_t)r * C + c));
+        m.x = __vmaxu2(m.x, v[k].x & 0x7FFF7FFFu);
+        m.y = __vmaxu2(m.y, v[k].y & 0x7FFF7FFFu);
+        m.z = __vmaxu2(m.z, v[k].z & 0x7FFF7FFFu);
+        m.w = __vmaxu2(m.w, v[k].w & 0x7FFF7FFFu);
+    }
+    col_max[rg][cg] = m;
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < 16; ++g) {
+        const uint4 o = col_max[g][cg];
+        m.x = __vmaxu2(m.x, o.x); m.y = __vmaxu2(m.y, o.y); m.z = __vmaxu2(m.z, o.z); m.w = __vmaxu2(m.w, o.w);
+    }
+    const uint32_t mw[4] = {m.x, m.y, m.z, m.w};
+    float sc[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        sc[2 * i] = block_scale_from_amax(__uint_as_float((mw[i] & 0xFFFFu) << 16), FMT == 0 ? 448.0f : 57344.0f);
+        sc[2 * i + 1] = block_scale_from_amax(__uint_as_float(mw[i] & 0xFFFF0000u), FMT == 0 ? 448.0f : 57344.0f);
+    }
+    if (rg == 0) {
+        float *dst = scale_inv + (size_t)blockIdx.y * C + c0 + cg * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) dst[i] = __fdiv_rn(1.0f, sc[i]);
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int r = r0 + k * 16 + rg, c = c0 + cg * 8;
+        if (r < R) {
+            const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+            uint16_t h[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                h[i] = cvt_f32x2_to_fp8x2<FMT>(__fmul_rn(bf16_lo(w[i]), sc[2 * i]), __fmul_rn(bf16_hi(w[i]), sc[2 * i + 1]));
+            *reinterpret_cast<uint2 *>(out + (size_t)r * C + c) =
+                make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ GEMM
 constexpr int BM = 128, BN = 128, BK = 128;
 constexpr int STAGES = 6;
@@ -129,14 +185,21 @@ constexpr int DYN_BYTES = TOTAL + 1024;
 constexpr int THREADS = 320;
 constexpr uint32_t TMEM_COLS = 256;
 
+// MODE_FWD    Y[t,n]  = sum_kb sx[kb][t] sw[n/128][kb] sum_{k in kb} X8[t,k] W8[n,k]      A, B reduction-contiguous
+// MODE_DGRAD  dX[t,k] = sum_nb sdy[nb][t] sw[nb][k/128] sum_{n in nb} dY8[t,n] W8[n,k]    B = W8 read in place (MN-major)
+// MODE_WGRAD  dW[n,k] = sum_tb sdy[tb][n] sx[tb][k] sum_{t in tb} dY8[t,n] X8[t,k]        A and B read in place (MN-major),
+//             one descale per output row and one per output column for every block of 128 tokens
+enum { MODE_FWD = 0, MODE_DGRAD = 1, MODE_WGRAD = 2 };
 struct Params {
     uint16_t *out;                 // [M,N] BF16
-    const float *sx_inv;           // [K/128][M]
-    const float *sw_inv;           // [ceil(N/128)][K/128]
-    int M, N, K;
+    const float *sx_inv;           // row descales, [reduction blocks][M]
+    const float *sw_inv;           // fwd: [ceil(N/128)][K/128]; dgrad: [K/128][ceil(N/128)] (the same array, read across);
+                                   // wgrad: column descales [reduction blocks][N]
+    int M, N, K;                   // output rows, output columns, reduction length
     int *status;
 };
 
+template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                       const Params p)
@@ -156,7 +219,7 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
     const int num_tiles = tiles_m * tiles_n;
-    const int k_blocks = p.K / BK;
+    const int k_blocks = (p.K + BK - 1) / BK;      // (the weight-gradient reduction over tokens may end ragged: zero-filled)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -198,15 +261,20 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctx)) { ok = false; break; }
                     const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
                     mbar_expect_tx(full_bar(stage), STAGE_BYTES);
-                    tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BK, tm * BM);
-                    tma_load_2d(sb, &tmap_b, full_bar(stage), kb * BK, tn * BN);
+                    // an operand read in place has the reduction index as its row index
+                    if (MODE == MODE_WGRAD) tma_load_2d(sa, &tmap_a, full_bar(stage), tm * BM, kb * BK);
+                    else tma_load_2d(sa, &tmap_a, full_bar(stage), kb * BK, tm * BM);
+                    if (MODE == MODE_FWD) tma_load_2d(sb, &tmap_b, full_bar(stage), kb * BK, tn * BN);
+                    else tma_load_2d(sb, &tmap_b, full_bar(stage), tn * BN, kb * BK);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         if (elect_one()) {
-            constexpr uint32_t idesc = umma_idesc_f8(0, 0, BM, BN);
+            constexpr int A_MN = MODE == MODE_WGRAD, B_MN = MODE != MODE_FWD;
+            constexpr uint32_t idesc = umma_idesc_f8(MODE == MODE_FWD ? 0 : 1, 0, BM, BN, A_MN, B_MN);   // gradients: E5M2
+            constexpr uint32_t STEP_K = 2u, STEP_MN = (32u * 128u) >> 4;      // descriptor advance per 32 reduction steps
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -218,10 +286,12 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     if (!mbar_wait(full_bar(stage), phase, ctx)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
-                    const uint64_t da = umma_desc_k_sw128(sa), db = umma_desc_k_sw128(sb);
+                    const uint64_t da = A_MN ? umma_desc(sa, 128, 16) : umma_desc_k_sw128(sa);
+                    const uint64_t db = B_MN ? umma_desc(sb, 128, 16) : umma_desc_k_sw128(sb);
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)
-                        umma_f8_ss(tmem_base + (uint32_t)(buf * BN), da + 2u * k, db + 2u * k, idesc, k != 0 ? 1u : 0u);
+                        umma_f8_ss(tmem_base + (uint32_t)(buf * BN), da + (A_MN ? STEP_MN : STEP_K) * k,
+                                   db + (B_MN ? STEP_MN : STEP_K) * k, idesc, k != 0 ? 1u : 0u);
                     umma_commit(empty_bar(stage));
                     umma_commit(pfull_bar(buf));
                     if (++stage == S) { stage = 0; phase ^= 1u; }
@@ -241,7 +311,13 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             const int row = tm * BM + quad * 32 + lane;
             const int n0 = tn * BN + half * HC;
             const float *sx = p.sx_inv + (row < p.M ? row : 0);
-            const float *sw = p.sw_inv + (size_t)tn * k_blocks;
+            const int tiles_n_all = (p.N + BN - 1) / BN;
+            // weight-block descale of (this output tile, reduction block kb): consecutive along kb in the forward,
+            // one row of the [K/128][N/128] array apart in the data gradient
+            const float *sw = MODE == MODE_DGRAD ? p.sw_inv + tn : p.sw_inv + (size_t)tn * k_blocks;
+            const size_t sw_step = MODE == MODE_DGRAD ? (size_t)tiles_n_all : 1;
+            // weight gradient: column descales of this thread's 64 output columns, [reduction blocks][N]
+            const float *scol = p.sw_inv + (n0 < p.N ? n0 : 0);
             float acc[HC];
 #pragma unroll
             for (int c = 0; c < HC; ++c) acc[c] = 0.0f;
@@ -252,7 +328,7 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 #pragma unroll
             for (int i = 0; i < PF; ++i) {
                 sxq[i] = i < k_blocks ? __ldg(sx + (size_t)i * p.M) : 0.0f;
-                swq[i] = i < k_blocks ? __ldg(sw + i) : 0.0f;
+                swq[i] = (MODE != MODE_WGRAD && i < k_blocks) ? __ldg(sw + (size_t)i * sw_step) : 1.0f;
             }
             for (int kb = 0; kb < k_blocks; ++kb, ++n) {
                 const int buf = (int)(n & 1u);
@@ -260,7 +336,7 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 #pragma unroll
                 for (int i = 0; i + 1 < PF; ++i) { sxq[i] = sxq[i + 1]; swq[i] = swq[i + 1]; }
                 sxq[PF - 1] = kb + PF < k_blocks ? __ldg(sx + (size_t)(kb + PF) * p.M) : 0.0f;
-                swq[PF - 1] = kb + PF < k_blocks ? __ldg(sw + kb + PF) : 0.0f;
+                swq[PF - 1] = (MODE != MODE_WGRAD && kb + PF < k_blocks) ? __ldg(sw + (size_t)(kb + PF) * sw_step) : 1.0f;
                 if (!mbar_wait_warp(pfull_bar(buf), (n >> 1) & 1u, ctx)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + lane_addr + (uint32_t)(buf * BN);
@@ -268,14 +344,39 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 tmem_ld_32x32b_x32(taddr, r0);
                 tmem_ld_wait();
                 tmem_ld_32x32b_x32(taddr + 32u, r1);           // in flight during the first 32 FMAs
+                if (MODE == MODE_WGRAD) {
+                    // every column has its own descale for this block of tokens (the same 64 values for all lanes)
+                    const float4 *pc = reinterpret_cast<const float4 *>(scol + (size_t)kb * p.N);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) acc[i] = fmaf(__uint_as_float(r0[i]), sc, acc[i]);
+                    for (int i = 0; i < 32; i += 4) {
+                        const float4 c4 = (n0 + i < p.N) ? __ldg(pc + (i >> 2)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        acc[i] = fmaf(__uint_as_float(r0[i]) * c4.x, sc, acc[i]);
+                        acc[i + 1] = fmaf(__uint_as_float(r0[i + 1]) * c4.y, sc, acc[i + 1]);
+                        acc[i + 2] = fmaf(__uint_as_float(r0[i + 2]) * c4.z, sc, acc[i + 2]);
+                        acc[i + 3] = fmaf(__uint_as_float(r0[i + 3]) * c4.w, sc, acc[i + 3]);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[i] = fmaf(__uint_as_float(r0[i]), sc, acc[i]);
+                }
                 tmem_ld_wait();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pempty_bar(buf));   // the partial is in registers: the buffer is free
+                if (MODE == MODE_WGRAD) {
+                    const float4 *pc = reinterpret_cast<const float4 *>(scol + (size_t)kb * p.N + 32);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) acc[32 + i] = fmaf(__uint_as_float(r1[i]), sc, acc[32 + i]);
+                    for (int i = 0; i < 32; i += 4) {
+                        const float4 c4 = (n0 + 32 + i < p.N) ? __ldg(pc + (i >> 2)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        acc[32 + i] = fmaf(__uint_as_float(r1[i]) * c4.x, sc, acc[32 + i]);
+                        acc[33 + i] = fmaf(__uint_as_float(r1[i + 1]) * c4.y, sc, acc[33 + i]);
+                        acc[34 + i] = fmaf(__uint_as_float(r1[i + 2]) * c4.z, sc, acc[34 + i]);
+                        acc[35 + i] = fmaf(__uint_as_float(r1[i + 3]) * c4.w, sc, acc[35 + i]);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[32 + i] = fmaf(__uint_as_float(r1[i]), sc, acc[32 + i]);
+                }
             }
             if (ok && row < p.M) {
                 uint16_t *dst = p.out + (size_t)row * p.N + n0;
@@ -315,8 +416,9 @@ extern "C" int fp8_quantize_blockwise(const void *x_bf16, size_t rows, size_t co
         set_error("fp8_quantize_blockwise: NULL pointer");
         return FP8_ERR_NULL;
     }
-    if ((fmt != FP8_E4M3 && fmt != FP8_E5M2) || (block_rows != 1 && block_rows != 128)) {
-        set_error("fp8_quantize_blockwise: fmt %d / block_rows %d not supported (E4M3 or E5M2; 1 or 128)", fmt, block_rows);
+    if ((fmt != FP8_E4M3 && fmt != FP8_E5M2) || (block_rows != 1 && block_rows != 128 && block_rows != FP8_BLOCK_128x1)) {
+        set_error("fp8_quantize_blockwise: fmt %d / block_rows %d not supported (E4M3 or E5M2; 1, 128 or FP8_BLOCK_128x1)", fmt,
+                  block_rows);
         return FP8_ERR_ENUM;
     }
     if (rows == 0 || cols == 0 || (cols % 128) || rows > 0x7FFFFFFFull || cols > 0x7FFFFFFFull) {
@@ -338,6 +440,10 @@ extern "C" int fp8_quantize_blockwise(const void *x_bf16, size_t rows, size_t co
         if (blocks > cap) blocks = cap;
         if (fmt == FP8_E4M3) bw::quantize_1x128_kernel<0><<<(unsigned)blocks, 256, 0, st>>>(x, rows, (int)cols, out, scale_inv);
         else bw::quantize_1x128_kernel<1><<<(unsigned)blocks, 256, 0, st>>>(x, rows, (int)cols, out, scale_inv);
+    } else if (block_rows == FP8_BLOCK_128x1) {
+        dim3 grid((unsigned)(cols / 128), (unsigned)((rows + 127) / 128));
+        if (fmt == FP8_E4M3) bw::quantize_128x1_kernel<0><<<grid, 256, 0, st>>>(x, (int)rows, (int)cols, out, scale_inv);
+        else bw::quantize_128x1_kernel<1><<<grid, 256, 0, st>>>(x, (int)rows, (int)cols, out, scale_inv);
     } else {
         dim3 grid((unsigned)(cols / 128), (unsigned)((rows + 127) / 128));
         if (fmt == FP8_E4M3) bw::quantize_128x128_kernel<0><<<grid, 256, 0, st>>>(x, (int)rows, (int)cols, out, scale_inv);
@@ -347,39 +453,80 @@ extern "C" int fp8_quantize_blockwise(const void *x_bf16, size_t rows, size_t co
     return FP8_OK;
 }
 
-extern "C" int fp8_linear_fwd_blockwise(const uint8_t *X8, const uint8_t *W8, const float *sx_inv, const float *sw_inv,
-                                        void *Y_bf16, int T, int N, int K, void *stream)
+static int launch_blockwise(const char *who, int mode, const uint8_t *A8, const uint8_t *B8, const float *sa_inv,
+                            const float *sb_inv, void *out_bf16, int M, int N, int Kred, uint64_t a_rows, uint64_t a_cols,
+                            uint64_t b_rows, uint64_t b_cols, void *stream)
 {
-    if (!X8 || !W8 || !sx_inv || !sw_inv || !Y_bf16) {
-        set_error("fp8_linear_fwd_blockwise: NULL pointer");
+    if (!A8 || !B8 || !sa_inv || !sb_inv || !out_bf16) {
+        set_error("%s: NULL pointer", who);
         return FP8_ERR_NULL;
     }
-    if (T <= 0 || N <= 0 || K <= 0 || (K % 128) || (N % 16)) {
-        set_error("fp8_linear_fwd_blockwise: unsupported shape T=%d N=%d K=%d (K %% 128 == 0, N %% 16 == 0)", T, N, K);
-        return FP8_ERR_SHAPE;
-    }
-    if (!aligned16(X8) || !aligned16(W8) || !aligned16(Y_bf16)) {
-        set_error("fp8_linear_fwd_blockwise: tensor pointers must be 16-byte aligned");
+    if (!aligned16(A8) || !aligned16(B8) || !aligned16(out_bf16) || !aligned16(sb_inv)) {
+        set_error("%s: tensor pointers must be 16-byte aligned", who);
         return FP8_ERR_ALIGN;
     }
     int rc = check_arch();
     if (rc != FP8_OK) return rc;
     CUtensorMap ta, tb;
-    rc = make_tmap_2d_u8(&ta, X8, (uint64_t)T, (uint64_t)K, (uint64_t)K, bw::BM, bw::BK);
+    // every operand tile is 128 rows of 128 bytes, whichever index its rows count
+    rc = make_tmap_2d_u8(&ta, A8, a_rows, a_cols, a_cols, 128, 128);
     if (rc != FP8_OK) return rc;
-    rc = make_tmap_2d_u8(&tb, W8, (uint64_t)N, (uint64_t)K, (uint64_t)K, bw::BN, bw::BK);
+    rc = make_tmap_2d_u8(&tb, B8, b_rows, b_cols, b_cols, 128, 128);
     if (rc != FP8_OK) return rc;
-    FP8_CUDA_CHECK(cudaFuncSetAttribute(bw::gemm_blockwise_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        bw::DYN_BYTES));
     bw::Params p;
-    p.out = static_cast<uint16_t *>(Y_bf16);
-    p.sx_inv = sx_inv; p.sw_inv = sw_inv;
-    p.M = T; p.N = N; p.K = K;
+    p.out = static_cast<uint16_t *>(out_bf16);
+    p.sx_inv = sa_inv; p.sw_inv = sb_inv;
+    p.M = M; p.N = N; p.K = Kred;
     p.status = device_status_ptr();
     if (!p.status) return FP8_ERR_CUDA;
-    const int tiles = ((T + bw::BM - 1) / bw::BM) * ((N + bw::BN - 1) / bw::BN);
+    const int tiles = ((M + bw::BM - 1) / bw::BM) * ((N + bw::BN - 1) / bw::BN);
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    bw::gemm_blockwise_kernel<<<grid, bw::THREADS, bw::DYN_BYTES, static_cast<cudaStream_t>(stream)>>>(ta, tb, p);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+#define FP8DPA_LAUNCH_BW(MODE) \
+    do { \
+        FP8_CUDA_CHECK(cudaFuncSetAttribute(bw::gemm_blockwise_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                            bw::DYN_BYTES)); \
+        bw::gemm_blockwise_kernel<MODE><<<grid, bw::THREADS, bw::DYN_BYTES, st>>>(ta, tb, p); \
+    } while (0)
+    if (mode == bw::MODE_FWD) FP8DPA_LAUNCH_BW(bw::MODE_FWD);
+    else if (mode == bw::MODE_DGRAD) FP8DPA_LAUNCH_BW(bw::MODE_DGRAD);
+    else FP8DPA_LAUNCH_BW(bw::MODE_WGRAD);
+#undef FP8DPA_LAUNCH_BW
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
+}
+
+extern "C" int fp8_linear_fwd_blockwise(const uint8_t *X8, const uint8_t *W8, const float *sx_inv, const float *sw_inv,
+                                        void *Y_bf16, int T, int N, int K, void *stream)
+{
+    if (T <= 0 || N <= 0 || K <= 0 || (K % 128) || (N % 16)) {
+        set_error("fp8_linear_fwd_blockwise: unsupported shape T=%d N=%d K=%d (K %% 128 == 0, N %% 16 == 0)", T, N, K);
+        return FP8_ERR_SHAPE;
+    }
+    return launch_blockwise("fp8_linear_fwd_blockwise", bw::MODE_FWD, X8, W8, sx_inv, sw_inv, Y_bf16, T, N, K,
+                            (uint64_t)T, (uint64_t)K, (uint64_t)N, (uint64_t)K, stream);
+}
+
+extern "C" int fp8_linear_dgrad_blockwise(const uint8_t *dY8, const uint8_t *W8, const float *sdy_inv,
+                                          const float *sw_inv, void *dX_bf16, int T, int N, int K, void *stream)
+{
+    if (T <= 0 || N <= 0 || K <= 0 || (N % 128) || (K % 128)) {
+        set_error("fp8_linear_dgrad_blockwise: unsupported shape T=%d N=%d K=%d (N %% 128 == 0, K %% 128 == 0)", T, N, K);
+        return FP8_ERR_SHAPE;
+    }
+    // output [T, K], reduction over N: A = dY8 [T, N] as stored, B = W8 [N, K] read in place
+    return launch_blockwise("fp8_linear_dgrad_blockwise", bw::MODE_DGRAD, dY8, W8, sdy_inv, sw_inv, dX_bf16, T, K, N,
+                            (uint64_t)T, (uint64_t)N, (uint64_t)N, (uint64_t)K, stream);
+}
+
+extern "C" int fp8_linear_wgrad_blockwise(const uint8_t *dY8, const uint8_t *X8, const float *sdy_inv_t,
+                                          const float *sx_inv_t, void *dW_bf16, int T, int N, int K, void *stream)
+{
+    if (T <= 0 || N <= 0 || K <= 0 || (N % 16) || (K % 16)) {
+        set_error("fp8_linear_wgrad_blockwise: unsupported shape T=%d N=%d K=%d (N %% 16 == 0, K %% 16 == 0)", T, N, K);
+        return FP8_ERR_SHAPE;
+    }
+    // output [N, K], reduction over T: A = dY8 [T, N] and B = X8 [T, K], both read in place
+    return launch_blockwise("fp8_linear_wgrad_blockwise", bw::MODE_WGRAD, dY8, X8, sdy_inv_t, sx_inv_t, dW_bf16, N, K, T,
+                            (uint64_t)T, (uint64_t)N, (uint64_t)T, (uint64_t)K, stream);
 }

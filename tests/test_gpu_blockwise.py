@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 def gpu_quantize_blockwise(xb, block_rows, fmt):
     R, C = xb.shape
     out = torch.empty((R, C), dtype=torch.uint8, device="cuda")
-    shape = (C // 128, R) if block_rows == 1 else ((R + 127) // 128, C // 128)
+    shape = {1: (C // 128, R), 128: ((R + 127) // 128, C // 128), fp8.FP8_BLOCK_128x1: ((R + 127) // 128, C)}[block_rows]
     si = torch.full(shape, -1.0, dtype=torch.float32, device="cuda")
     fp8.fp8_quantize_blockwise(dev(xb), block_rows, fmt, out, si)
     return out, si
@@ -36,6 +36,49 @@ def test_block_quantisers_bit_exact(fmt, R, C):
     codes, osi = o.quantize_blockwise(xb, 128, 128, fmt)
     assert np.array_equal(host(out), codes)
     assert np.array_equal(host(si).view(np.uint32), osi.view(np.uint32))
+    # 128 x 1
+    out, si = gpu_quantize_blockwise(xb, fp8.FP8_BLOCK_128x1, fmt)
+    codes, osi = o.quantize_blockwise(xb, 128, 1, fmt)
+    assert np.array_equal(host(out), codes)
+    assert np.array_equal(host(si).view(np.uint32), osi.view(np.uint32))
+
+
+@pytest.mark.parametrize("T,N,K", [(256, 256, 256), (400, 384, 640), (1000, 512, 2048), (16, 128, 128), (130, 1024, 256)])
+def test_blockwise_dgrad_matches_oracle(T, N, K):
+    seed = T + 5 * N + K
+    dy = synth.normal_bf16((T, N), seed, 0, 1e-3, synth.choose_columns(N, 2, seed, 2), 30.0)
+    w = synth.normal_bf16((N, K), seed, 1, synth.W_STD)
+    dy8, sdy = gpu_quantize_blockwise(dy, 1, o.E5M2)
+    w8, sw = gpu_quantize_blockwise(w, 128, o.E4M3)
+    dx = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_linear_dgrad_blockwise(dy8, w8, sdy, sw, dx)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    ody8, osdy = o.quantize_blockwise(dy, 1, 128, o.E5M2)
+    ow8, osw = o.quantize_blockwise(w, 128, 128, o.E4M3)
+    assert np.array_equal(host(dy8), ody8) and np.array_equal(host(w8), ow8)
+    ref, mag = o.linear_dgrad_blockwise(ody8, ow8, osdy, osw)
+    err = rel_err(dx.float().cpu().numpy().astype(np.float64), ref, mag)
+    assert err <= 2.0 ** -8, err
+
+
+@pytest.mark.parametrize("T,N,K", [(256, 256, 256), (400, 384, 640), (1000, 512, 2048), (77, 128, 128), (2048, 1024, 256)])
+def test_blockwise_wgrad_matches_oracle(T, N, K):
+    seed = T + 7 * N + K
+    dy = synth.normal_bf16((T, N), seed, 0, 1e-3, synth.choose_columns(N, 2, seed, 2), 30.0)
+    x = synth.normal_bf16((T, K), seed, 1, 1.0, synth.choose_columns(K, 3, seed, 1), 50.0)
+    dy8, sdy = gpu_quantize_blockwise(dy, fp8.FP8_BLOCK_128x1, o.E5M2)
+    x8, sx = gpu_quantize_blockwise(x, fp8.FP8_BLOCK_128x1, o.E4M3)
+    dw = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_linear_wgrad_blockwise(dy8, x8, sdy, sx, dw)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    ody8, osdy = o.quantize_blockwise(dy, 128, 1, o.E5M2)
+    ox8, osx = o.quantize_blockwise(x, 128, 1, o.E4M3)
+    assert np.array_equal(host(dy8), ody8) and np.array_equal(host(x8), ox8)
+    ref, mag = o.linear_wgrad_blockwise(ody8, ox8, osdy, osx)
+    err = rel_err(dw.float().cpu().numpy().astype(np.float64), ref, mag)
+    assert err <= 2.0 ** -8, err
 
 
 @pytest.mark.parametrize("T,N,K", [(256, 256, 256), (400, 272, 384), (128, 1040, 1024), (1000, 512, 2048), (16, 16, 128)])

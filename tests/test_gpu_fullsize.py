@@ -302,6 +302,34 @@ def test_glue_and_producer_forms_at_c4_sizes():
     ref, mag = o.linear_fwd_blockwise(ox8, ow8, osx, osw)
     got = y.float().cpu().numpy().astype(np.float64)[rows]
     assert rel_err(got, ref, mag) <= 2.0 ** -8
+    # its data gradient on sampled token rows, and its weight gradient on sampled entries
+    dyq = synth.normal_bf16((Tt, N), 4, 82, 1e-3, synth.choose_columns(N, 8, 4, 82), 20.0)
+    dy8 = torch.empty((Tt, N), dtype=torch.uint8, device="cuda")
+    sdy = torch.empty((N // 128, Tt), device="cuda")
+    fp8.fp8_quantize_blockwise(dev(dyq), 1, o.E5M2, dy8, sdy)
+    dx = torch.empty((Tt, K), dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_linear_dgrad_blockwise(dy8, w8, sdy, sw, dx)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    ody8, osdy = o.quantize_blockwise(np.ascontiguousarray(dyq[rows]), 1, 128, o.E5M2)
+    assert np.array_equal(host(dy8)[rows], ody8)
+    ref, mag = o.linear_dgrad_blockwise(ody8, ow8, osdy, osw)
+    assert rel_err(dx.float().cpu().numpy().astype(np.float64)[rows], ref, mag) <= 2.0 ** -8
+    del dx, y
+    nb = (Tt + 127) // 128
+    sdt, sxt = torch.empty((nb, N), device="cuda"), torch.empty((nb, K), device="cuda")
+    fp8.fp8_quantize_blockwise(dev(dyq), fp8.FP8_BLOCK_128x1, o.E5M2, dy8, sdt)
+    fp8.fp8_quantize_blockwise(dev(xq), fp8.FP8_BLOCK_128x1, o.E4M3, x8, sxt)
+    dw = torch.empty((N, K), dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_linear_wgrad_blockwise(dy8, x8, sdt, sxt, dw)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    ns, ks = _sample(N, 12, 7), _sample(K, 12, 8)
+    ody8, osdt = o.quantize_blockwise(np.ascontiguousarray(dyq[:, ns]), 128, 1, o.E5M2)
+    ox8, osxt = o.quantize_blockwise(np.ascontiguousarray(xq[:, ks]), 128, 1, o.E4M3)
+    assert np.array_equal(host(dy8)[:, ns], ody8) and np.array_equal(host(x8)[:, ks], ox8)
+    ref, mag = o.linear_wgrad_blockwise(ody8, ox8, osdt, osxt)
+    assert rel_err(dw.float().cpu().numpy().astype(np.float64)[np.ix_(ns, ks)], ref, mag) <= 2.0 ** -8
 
 
 def test_bench_line_carries_the_contract_keys():

@@ -87,3 +87,68 @@ def test_blockwise_pipeline_is_exact_on_powers_of_two():
     xd = tab[x8] * np.repeat(sx.astype(np.float64), 128, axis=1)
     wd = tab[w8] * np.repeat(np.repeat(sw.astype(np.float64), 128, axis=0), 128, axis=1)
     assert np.allclose(ref, xd @ wd.T, rtol=1e-6)
+
+
+def test_column_block_quantiser_is_the_row_block_one_transposed():
+    # 128 x 1 blocks of x are the 1 x 128 blocks of x^T: same codes, same descales, transposed
+    x = synth.normal_bf16((300, 40), 61, 0, 3.0)
+    codes, si = o.quantize_blockwise(x, 128, 1, o.E5M2)
+    codes_t, si_t = o.quantize_blockwise(np.ascontiguousarray(x.T), 1, 128, o.E5M2)
+    assert si.shape == (3, 40)
+    assert np.array_equal(codes, codes_t.T) and np.array_equal(si.view(np.uint32), si_t.T.view(np.uint32))
+
+
+def test_blockwise_gradients_reduce_to_plain_matrix_products():
+    T, N, K = 200, 256, 384                      # T ragged against the 128-token blocks of the weight gradient
+    tab4, tab5 = o.decode_table(o.E4M3), o.decode_table(o.E5M2)
+    dy8 = o.quantize(synth.normal_bf16((T, N), 35, 1, 1.0), o.E5M2)[0]
+    w8 = o.quantize(synth.normal_bf16((N, K), 35, 2, 0.02), o.E4M3)[0]
+    x8 = o.quantize(synth.normal_bf16((T, K), 35, 3, 1.0), o.E4M3)[0]
+    g, w, x = tab5[dy8], tab4[w8], tab4[x8]
+    # constant scales: the plain products times the two factors
+    ref, mag = o.linear_dgrad_blockwise(dy8, w8, np.full((T, 2), 0.25, np.float32), np.full((2, 3), 0.5, np.float32))
+    assert np.allclose(ref, 0.125 * (g @ w), rtol=1e-12, atol=1e-300)
+    assert np.allclose(mag, 0.125 * (np.abs(g) @ np.abs(w)), rtol=1e-12)
+    ntb = 2
+    ref, mag = o.linear_wgrad_blockwise(dy8, x8, np.full((ntb, N), 0.25, np.float32), np.full((ntb, K), 2.0, np.float32))
+    assert np.allclose(ref, 0.5 * (g.T @ x), rtol=1e-12, atol=1e-300)
+    assert np.allclose(mag, 0.5 * (np.abs(g).T @ np.abs(x)), rtol=1e-12)
+    # distinct scales per block: every factor lands on its own block and nowhere else
+    rng = np.random.default_rng(9)
+    sdy = rng.uniform(0.5, 2.0, size=(T, 2)).astype(np.float32)
+    sw = rng.uniform(0.5, 2.0, size=(2, 3)).astype(np.float32)
+    gd = g * np.repeat(sdy.astype(np.float64), 128, axis=1)
+    wd = w * np.repeat(np.repeat(sw.astype(np.float64), 128, axis=0), 128, axis=1)
+    ref, mag = o.linear_dgrad_blockwise(dy8, w8, sdy, sw)
+    assert np.max(np.abs(ref - gd @ wd) / mag) < 1e-13          # sums that cancel: measure against the magnitude
+    assert np.max(np.abs(ref - (g * np.repeat(sdy[:, ::-1].astype(np.float64), 128, axis=1)) @ wd) / mag) > 1e-2
+    sdt = rng.uniform(0.5, 2.0, size=(ntb, N)).astype(np.float32)
+    sxt = rng.uniform(0.5, 2.0, size=(ntb, K)).astype(np.float32)
+    gd = g * np.repeat(sdt.astype(np.float64), 128, axis=0)[:T]
+    xd = x * np.repeat(sxt.astype(np.float64), 128, axis=0)[:T]
+    ref, mag = o.linear_wgrad_blockwise(dy8, x8, sdt, sxt)
+    assert np.max(np.abs(ref - gd.T @ xd) / mag) < 1e-13
+    assert np.max(np.abs(ref - (g * np.repeat(sdt[::-1].astype(np.float64), 128, axis=0)[:T]).T @ xd) / mag) > 1e-2
+    # sampled rows and columns pick the same entries
+    rows, cols = np.array([3, 255]), np.array([0, 129, 383])
+    sub, _ = o.linear_wgrad_blockwise(dy8, x8, sdt, sxt, rows=rows, cols=cols)
+    assert np.array_equal(sub, ref[np.ix_(rows, cols)])
+
+
+def test_blockwise_gradient_pipeline_recovers_the_unquantised_products():
+    # quantise -> product -> descale reproduces the BF16 operands' product to the formats' precision
+    T, N, K = 256, 128, 256
+    dy = synth.normal_bf16((T, N), 36, 1, 1e-3)
+    w = synth.normal_bf16((N, K), 36, 2, 0.02)
+    x = synth.normal_bf16((T, K), 36, 3, 1.0)
+    f = lambda a: (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    dy8, sdy = o.quantize_blockwise(dy, 1, 128, o.E5M2)
+    w8, sw = o.quantize_blockwise(w, 128, 128, o.E4M3)
+    ref, mag = o.linear_dgrad_blockwise(dy8, w8, sdy, sw)
+    exact = f(dy) @ f(w)
+    assert np.max(np.abs(ref - exact) / mag) < 0.07          # E5M2 half-ulp 2^-3 and E4M3 2^-4, averaged over a sum
+    dy8t, sdt = o.quantize_blockwise(dy, 128, 1, o.E5M2)
+    x8t, sxt = o.quantize_blockwise(x, 128, 1, o.E4M3)
+    ref, mag = o.linear_wgrad_blockwise(dy8t, x8t, sdt, sxt)
+    exact = f(dy).T @ f(x)
+    assert np.max(np.abs(ref - exact) / mag) < 0.07
