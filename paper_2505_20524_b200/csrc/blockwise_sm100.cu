@@ -13,6 +13,8 @@
 //             each); acc[64] (registers) += partial[c] * sx_inv[kb,row] * sw_inv[tile,kb], the TMEM load of the next
 //             32 columns in flight during the FMAs; after the last K-block the row is written as BF16
 #include <float.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "gemm_epilogue.cuh"
@@ -318,9 +320,11 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             const size_t sw_step = MODE == MODE_DGRAD ? (size_t)tiles_n_all : 1;
             // weight gradient: column descales of this thread's 64 output columns, [reduction blocks][N]
             const float *scol = p.sw_inv + (n0 < p.N ? n0 : 0);
-            float acc[HC];
+            // accumulators as packed pairs: the promotion is one fma.rn.f32x2 per two outputs and K-block (per lane an
+            // ordinary FP32 FMA, so the result is the scalar one bit for bit), which halves its issue slots
+            uint64_t acc2[HC / 2];
 #pragma unroll
-            for (int c = 0; c < HC; ++c) acc[c] = 0.0f;
+            for (int c = 0; c < HC / 2; ++c) acc2[c] = 0ull;
             // the two descale factors of a K-block are fetched PF K-blocks ahead: a global load per K-block on the
             // critical path would cost more than the K-block's MMAs
             constexpr int PF = 4;
@@ -333,6 +337,7 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             for (int kb = 0; kb < k_blocks; ++kb, ++n) {
                 const int buf = (int)(n & 1u);
                 const float sc = sxq[0] * swq[0];
+                const uint64_t sc2 = pack_f32x2(sc, sc);
 #pragma unroll
                 for (int i = 0; i + 1 < PF; ++i) { sxq[i] = sxq[i + 1]; swq[i] = swq[i + 1]; }
                 sxq[PF - 1] = kb + PF < k_blocks ? __ldg(sx + (size_t)(kb + PF) * p.M) : 0.0f;
@@ -350,14 +355,12 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 #pragma unroll
                     for (int i = 0; i < 32; i += 4) {
                         const float4 c4 = (n0 + i < p.N) ? __ldg(pc + (i >> 2)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        acc[i] = fmaf(__uint_as_float(r0[i]) * c4.x, sc, acc[i]);
-                        acc[i + 1] = fmaf(__uint_as_float(r0[i + 1]) * c4.y, sc, acc[i + 1]);
-                        acc[i + 2] = fmaf(__uint_as_float(r0[i + 2]) * c4.z, sc, acc[i + 2]);
-                        acc[i + 3] = fmaf(__uint_as_float(r0[i + 3]) * c4.w, sc, acc[i + 3]);
+                        acc2[i >> 1] = fma_f32x2(mul_f32x2(pack_u32x2(r0[i], r0[i + 1]), pack_f32x2(c4.x, c4.y)), sc2, acc2[i >> 1]);
+                        acc2[(i >> 1) + 1] = fma_f32x2(mul_f32x2(pack_u32x2(r0[i + 2], r0[i + 3]), pack_f32x2(c4.z, c4.w)), sc2, acc2[(i >> 1) + 1]);
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) acc[i] = fmaf(__uint_as_float(r0[i]), sc, acc[i]);
+                    for (int i = 0; i < 32; i += 2) acc2[i >> 1] = fma_f32x2(pack_u32x2(r0[i], r0[i + 1]), sc2, acc2[i >> 1]);
                 }
                 tmem_ld_wait();
                 tc_fence_before();
@@ -368,17 +371,18 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 #pragma unroll
                     for (int i = 0; i < 32; i += 4) {
                         const float4 c4 = (n0 + 32 + i < p.N) ? __ldg(pc + (i >> 2)) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        acc[32 + i] = fmaf(__uint_as_float(r1[i]) * c4.x, sc, acc[32 + i]);
-                        acc[33 + i] = fmaf(__uint_as_float(r1[i + 1]) * c4.y, sc, acc[33 + i]);
-                        acc[34 + i] = fmaf(__uint_as_float(r1[i + 2]) * c4.z, sc, acc[34 + i]);
-                        acc[35 + i] = fmaf(__uint_as_float(r1[i + 3]) * c4.w, sc, acc[35 + i]);
+                        acc2[16 + (i >> 1)] = fma_f32x2(mul_f32x2(pack_u32x2(r1[i], r1[i + 1]), pack_f32x2(c4.x, c4.y)), sc2, acc2[16 + (i >> 1)]);
+                        acc2[17 + (i >> 1)] = fma_f32x2(mul_f32x2(pack_u32x2(r1[i + 2], r1[i + 3]), pack_f32x2(c4.z, c4.w)), sc2, acc2[17 + (i >> 1)]);
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) acc[32 + i] = fmaf(__uint_as_float(r1[i]), sc, acc[32 + i]);
+                    for (int i = 0; i < 32; i += 2) acc2[16 + (i >> 1)] = fma_f32x2(pack_u32x2(r1[i], r1[i + 1]), sc2, acc2[16 + (i >> 1)]);
                 }
             }
             if (ok && row < p.M) {
+                float acc[HC];
+#pragma unroll
+                for (int c = 0; c < HC / 2; ++c) unpack_f32x2(acc2[c], acc[2 * c], acc[2 * c + 1]);
                 uint16_t *dst = p.out + (size_t)row * p.N + n0;
 #pragma unroll
                 for (int c = 0; c < HC; c += 8) {
@@ -405,6 +409,10 @@ gemm_blockwise_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 }
 
 }  // namespace bw
+
+// the CTA-pair form of the same products (blockwise_2cta_sm100.cu)
+int launch_blockwise_pair(int mode, const CUtensorMap &ta, const CUtensorMap &tb, const float *sa_inv, const float *sb_inv,
+                          uint16_t *out, int M, int N, int Kred, int *status, cudaStream_t st);
 }  // namespace fp8dpa
 
 using namespace fp8dpa;
@@ -479,9 +487,17 @@ static int launch_blockwise(const char *who, int mode, const uint8_t *A8, const 
     p.M = M; p.N = N; p.K = Kred;
     p.status = device_status_ptr();
     if (!p.status) return FP8_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // 256 x 256 tiles on CTA pairs wherever the output has more than one 128 x 128 tile in both directions; the
+    // single-CTA kernel for narrow outputs (FP8DPA_BLOCKWISE=1cta forces it, for comparison)
+    static const bool force_1cta = [] {
+        const char *e = getenv("FP8DPA_BLOCKWISE");
+        return e && !strcmp(e, "1cta");
+    }();
+    if (!force_1cta && M > bw::BM && N > bw::BN)
+        return launch_blockwise_pair(mode, ta, tb, sa_inv, sb_inv, p.out, M, N, Kred, p.status, st);
     const int tiles = ((M + bw::BM - 1) / bw::BM) * ((N + bw::BN - 1) / bw::BN);
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
 #define FP8DPA_LAUNCH_BW(MODE) \
     do { \
         FP8_CUDA_CHECK(cudaFuncSetAttribute(bw::gemm_blockwise_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
