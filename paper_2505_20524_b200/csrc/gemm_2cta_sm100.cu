@@ -14,6 +14,9 @@
 //   tfull[b]  multicast commit after the last MMA of a tile (lands in both CTAs)
 //   tempty[b] used in the even CTA only: 8 arrivals (4 epilogue warps of each CTA; the odd CTA arrives remotely)
 // Every wait is bounded; a cluster barrier before exit keeps either CTA alive while its peer can still reach it.
+#include <stdlib.h>
+#include <string.h>
+
 #include "common.cuh"
 #include "gemm_epilogue.cuh"
 
@@ -46,13 +49,18 @@ struct Params {
     // descale sb_inv[g]; the offsets live on the device (they come out of the router)
     const int *group_offsets;
     int n_groups;
+    // Tile order of the plain form: bands of band_w tiles along the rows (band_on_m) or the columns of the output; inside
+    // a band the other index advances slowest.  The operand of the banded dimension is then shared by consecutive
+    // waves; where its band is sized to stay in L2 its loads carry evict_last and the other operand's evict_first
+    // (hint_a / hint_b: 0 none, 1 evict_last, 2 evict_first).
+    int band_w, band_on_m, hint_a, hint_b;
 };
 constexpr int MAX_GROUPS = 256;
 
-__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int &tm, int &tn)
+__device__ __forceinline__ void tile_coords(const Params &p, int tile, int tiles_m, int tiles_n, int &tm, int &tn)
 {
-    if (tiles_m >= tiles_n) band_coords(tile, tiles_m, tiles_n, tm, tn);
-    else band_coords(tile, tiles_n, tiles_m, tn, tm);
+    if (p.band_on_m) band_coords_w(tile, tiles_m, tiles_n, p.band_w, tm, tn);
+    else band_coords_w(tile, tiles_n, tiles_m, p.band_w, tn, tm);
 }
 
 // Tile -> (group, row offset of the group, rows of the group, tile coordinates inside the group) for the grouped form:
@@ -147,6 +155,8 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            const uint64_t pol_last = l2_policy_evict_last(), pol_first = l2_policy_evict_first();
+            const uint64_t pol_a = p.hint_a == 1 ? pol_last : pol_first, pol_b = p.hint_b == 1 ? pol_last : pol_first;
             for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs) {
                 int tm, tn, m_base = 0, n_base = 0, kb_base_b = 0;
                 if (GROUPED) {
@@ -158,7 +168,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                     if (p.b_mn) kb_base_b = gt.g * p.K;
                     else n_base = gt.g * p.N;
                 } else {
-                    tile_coords(tile, tiles_m, tiles_n, tm, tn);
+                    tile_coords(p, tile, tiles_m, tiles_n, tm, tn);
                 }
                 const int m0 = m_base + tm * 2 * BM + (int)rank * BM, n0 = n_base + tn * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < k_blocks; ++kb) {
@@ -167,10 +177,12 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                     if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
                     // K-major tile: 128 rows of the output index x 128 reduction bytes; MN-major tile: 128 reduction
                     // rows x 128 bytes of the output index (the matrix as it lies in memory, no transposed copy)
-                    if (p.a_mn) tma_load_2d_pair(sa, &tmap_a, full_bar(stage), m0, kb * BK);
-                    else tma_load_2d_pair(sa, &tmap_a, full_bar(stage), kb * BK, m0);
-                    if (p.b_mn) tma_load_2d_pair(sb, &tmap_b, full_bar(stage), n0, kb_base_b + kb * BK);
-                    else tma_load_2d_pair(sb, &tmap_b, full_bar(stage), kb * BK, n0);
+                    const int a0 = p.a_mn ? m0 : kb * BK, a1 = p.a_mn ? kb * BK : m0;
+                    const int b0 = p.b_mn ? n0 : kb * BK, b1 = p.b_mn ? kb_base_b + kb * BK : n0;
+                    if (!GROUPED && p.hint_a) tma_load_2d_pair_hint(sa, &tmap_a, full_bar(stage), a0, a1, pol_a);
+                    else tma_load_2d_pair(sa, &tmap_a, full_bar(stage), a0, a1);
+                    if (!GROUPED && p.hint_b) tma_load_2d_pair_hint(sb, &tmap_b, full_bar(stage), b0, b1, pol_b);
+                    else tma_load_2d_pair(sb, &tmap_b, full_bar(stage), b0, b1);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -226,7 +238,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                 m_end = gt.row0 + gt.rows;         // rows past the group's end belong to the next group: not stored
                 descale_t = __ldg(p.sa_inv) * __ldg(p.sb_inv + gt.g);
             } else {
-                tile_coords(tile, tiles_m, tiles_n, tm, tn);
+                tile_coords(p, tile, tiles_m, tiles_n, tm, tn);
             }
             const int m0 = m_base + tm * 2 * BM + (int)rank * BM, n0 = tn * BN;
             if (!mbar_wait_warp(tfull_bar(buf), acc_phase, ctx)) { ok = false; break; }
@@ -265,6 +277,53 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
 }
 
 }  // namespace g2
+
+// Tile order and L2 priority of one product.  Every wave of 74 tiles streams its row panels and column panels
+// (256 x K bytes each) once, in step along the reduction, so tiles of a wave share panels through L2 whatever their
+// size; what matters is what the NEXT wave still finds.  One output dimension is cut into bands of w tiles, the other
+// index advances slowest inside a band: consecutive waves then reuse the band's w panels and stream the others.
+// w = as many panels as fit RESIDENT_BYTES (measured: the band survives a wave's streaming up to about 36 MB, well
+// under the 126 MB of L2), but never under 8, since a wave of 8 x 9.25 tiles touches the fewest panels when nothing
+// survives.  DRAM reads of the operands are then P * (n1 + ceil(n1 / w) * n2) for n1 banded tiles, n2 streamed ones
+// and panel size P; the cheaper choice of the banded dimension wins.  The band's loads carry an evict_last policy
+// (worth 0-10 % of the reads); evict_first on the streamed operand was measured and doubles the reads (tiles of a
+// wave drift apart by more than such a line lives).  Measured on the 8B-class shapes (DRAM read MB, old order ->
+// this one): 8192x28672x4096 350 -> 183, 8192x4096x28672 1217 -> 968, 28672x4096x8192 640 -> 328,
+// 8192x4096x14336 583 -> 406, 4096x14336x8192 303 -> 172; durations equal within 2 % (the products are bound by the
+// tensor pipe and board power, not by DRAM).  Small products (operands under FITS_BYTES) keep bands of 16 along the
+// longer dimension.  FP8DPA_GEMM_ORDER=legacy keeps that form everywhere (for comparison; read per call).
+static void choose_tile_order(g2::Params &p)
+{
+    using namespace g2;
+    const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
+    p.band_on_m = tiles_m >= tiles_n;
+    p.band_w = GEMM_BAND;
+    p.hint_a = p.hint_b = 0;
+    const char *eo = getenv("FP8DPA_GEMM_ORDER");        // read per call: one process can compare the two orders
+    const bool legacy = eo && !strcmp(eo, "legacy");
+    const char *er = getenv("FP8DPA_GEMM_RESIDENT_MB");
+    const double FITS_BYTES = 48e6, RESIDENT_BYTES = er ? atof(er) * 1e6 : 36e6;
+    const double panel = 256.0 * p.K;
+    if (legacy || ((double)p.M + p.N) * p.K <= FITS_BYTES) return;
+    // at least 8 tiles wide: a wave of 74 tiles is then no longer than 8 x 9.25, the shape with the fewest panels
+    const int wmax = (int)(RESIDENT_BYTES / panel) < 8 ? 8 : (int)(RESIDENT_BYTES / panel);
+    double best = 0.0;
+    for (int on_m = 0; on_m < 2; ++on_m) {
+        const int n1 = on_m ? tiles_m : tiles_n, n2 = on_m ? tiles_n : tiles_m;
+        const int w = wmax < n1 ? wmax : n1;
+        const double reads = panel * (n1 + (double)((n1 + w - 1) / w) * n2);
+        if (best == 0.0 || reads < best) {
+            best = reads;
+            p.band_on_m = on_m;
+            p.band_w = w;
+        }
+    }
+    const char *eh = getenv("FP8DPA_GEMM_HINTS");        // experiments: 0 none, 1 evict_last only, 2 both
+    const int hint_mode = eh ? atoi(eh) : 1;
+    const int resident = hint_mode >= 1 ? 1 : 0, streamed = hint_mode >= 2 ? 2 : 0;
+    p.hint_a = p.band_on_m ? resident : streamed;
+    p.hint_b = p.band_on_m ? streamed : resident;
+}
 
 // Returns FP8_OK after launching, or a negative status.  `max_pairs` = 0 lets the runtime size the grid.
 int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv, const GemmOut &o,
@@ -308,6 +367,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     p.status = status;
     p.group_offsets = nullptr;
     p.n_groups = 0;
+    choose_tile_order(p);
     gemm_fp8_pair_kernel<false><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
@@ -340,6 +400,7 @@ int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa
     p.status = status;
     p.group_offsets = group_offsets;
     p.n_groups = n_groups;
+    p.band_w = GEMM_BAND; p.band_on_m = 1; p.hint_a = p.hint_b = 0;      // (the grouped form has its own tile table)
     gemm_fp8_pair_kernel<true><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;

@@ -11,13 +11,17 @@ namespace fp8dpa {
 // index along the shorter dimension advances slowest.  The CTAs that run at the same time then share one band of
 // one operand (a few MB) and a handful of panels of the other, and both stay in L2 however long the matrix is.
 constexpr int GEMM_BAND = 16;
+__device__ __forceinline__ void band_coords_w(int tile, int n_long, int n_short, int band_w, int &i_long, int &i_short)
+{
+    const int per_band = band_w * n_short;
+    const int band = tile / per_band, within = tile - band * per_band;
+    const int len = min(band_w, n_long - band * band_w);     // the last band may be short
+    i_short = within / len;
+    i_long = band * band_w + (within - i_short * len);
+}
 __device__ __forceinline__ void band_coords(int tile, int n_long, int n_short, int &i_long, int &i_short)
 {
-    const int per_band = GEMM_BAND * n_short;
-    const int band = tile / per_band, within = tile - band * per_band;
-    const int len = min(GEMM_BAND, n_long - band * GEMM_BAND);     // the last band may be short
-    i_short = within / len;
-    i_long = band * GEMM_BAND + (within - i_short * len);
+    band_coords_w(tile, n_long, n_short, GEMM_BAND, i_long, i_short);
 }
 
 struct GemmOut {
