@@ -38,6 +38,10 @@ class QTensor:
     amax: torch.Tensor = None
     scale: torch.Tensor = None
     scale_inv: torch.Tensor = None
+    history: torch.Tensor = None       # delayed scaling: the last HISTORY_LEN abs-max values and the ring position
+    head: torch.Tensor = None
+
+    HISTORY_LEN = 1024                 # the length the paper trains with (Appendix E)
 
     def __post_init__(self):
         dev = self.x.device
@@ -49,6 +53,23 @@ class QTensor:
 
     def quantize(self):
         fp8.fp8_quantize(self.x, self.fmt, self.q, self.qt, self.amax, self.scale, self.scale_inv)
+
+    def quantize_delayed(self):
+        """Delayed scaling (Appendix E): one pass casts under the scale of the history and records this step's
+        abs-max; the history and the scale for the next step are updated afterwards.  The first call seeds the
+        history with a just-in-time pass."""
+        if self.history is None:
+            dev = self.x.device
+            self.history = torch.zeros(self.HISTORY_LEN, dtype=torch.float32, device=dev)
+            self.head = torch.zeros(1, dtype=torch.int32, device=dev)
+            self._next = (_f32(dev), _f32(dev))
+            fp8.fp8_amax(self.x, self.amax)
+            fp8.fp8_scale_update(self.history, self.head, self.amax, self.fmt, 0, *self._next)
+        # the scale computed after the previous step becomes this step's; this step's products read scale_inv, so the
+        # update for the next step is written to the other pair of scalars
+        (self.scale, self.scale_inv), self._next = self._next, (self.scale, self.scale_inv)
+        fp8.fp8_cast(self.x, self.scale, self.fmt, self.q, self.qt, self.amax)
+        fp8.fp8_scale_update(self.history, self.head, self.amax, self.fmt, 0, *self._next)
 
     @property
     def nbytes_in(self):
@@ -80,11 +101,15 @@ class BlockHotPath:
     KERNELS_PER_ATTN_BWD = 3    # prep, main, finish
 
     def __init__(self, cfg: synth.BlockConfig, device="cuda", with_linears=None, with_attention=True,
-                 seq=None, batch=None, transposed_copies=False, attn_max_slack=0.0):
+                 seq=None, batch=None, transposed_copies=False, attn_max_slack=0.0, scaling="jit"):
         # transposed_copies: also write [cols, rows] FP8 copies in the cast and run dgrad / wgrad on them (the
         # form a K-major-only tensor core needs); off by default, tcgen05 reads the operands in place
         # attn_max_slack: tau of the attention forward's reference maximum (0 = exact running maximum); P~ is then
         # scaled by 448 / 2^tau
+        # scaling: "jit" = amax pass, scale, cast pass per tensor and step (fp8_quantize); "delayed" = one cast pass under
+        # the scale of the abs-max history, which the pass itself feeds (Appendix E; the recipe the paper trains with)
+        assert scaling in ("jit", "delayed")
+        self.scaling = scaling
         self.attn_max_slack = float(attn_max_slack)
         self.cfg = cfg
         self.device = torch.device(device)
@@ -261,20 +286,22 @@ class BlockHotPath:
     def quantize_bytes(self):
         """Algorithmic HBM bytes of the JIT quantize calls: 2 (amax read) + 2 (cast read) + 1 per FP8 copy."""
         b = 0
+        rd = 4 if self.scaling == "jit" else 2          # BF16 read twice (amax pass, cast pass) or once
         for lin in self.linears:
             for t in (lin.x, lin.w, lin.dy):
-                b += t.x.numel() * (4 + 1 + (1 if t.transpose else 0))
+                b += t.x.numel() * (rd + 1 + (1 if t.transpose else 0))
         if self.attn is not None:
             for n in ("q", "k", "v", "do"):
-                b += self.attn[n].x.numel() * 5
+                b += self.attn[n].x.numel() * (rd + 1)
         return b
 
     def launches_per_step(self):
         n = 0
+        kq = self.KERNELS_PER_QUANTIZE         # delayed scaling: cast (+amax) and the history update, also two
         for _ in self.linears:
-            n += 3 * self.KERNELS_PER_QUANTIZE + 3
+            n += 3 * kq + 3
         if self.attn is not None:
-            n += 4 * self.KERNELS_PER_QUANTIZE + 1 + self.KERNELS_PER_ATTN_BWD
+            n += 4 * kq + 1 + self.KERNELS_PER_ATTN_BWD
         return n
 
     # ------------------------------------------------------------------ the step
@@ -323,8 +350,10 @@ class BlockHotPath:
         def gemm(fn, *args, **kw):
             timed(ev, fn, *args, **kw)
 
+        quant = QTensor.quantize if self.scaling == "jit" else QTensor.quantize_delayed
+
         for lin in self.linears:
-            timed(qev, lambda: (lin.x.quantize(), lin.w.quantize(), lin.dy.quantize()))
+            timed(qev, lambda: [quant(t) for t in (lin.x, lin.w, lin.dy)])
             gemm(fp8.fp8_linear_fwd, lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
             if self.transposed_copies:
                 gemm(fp8.fp8_linear_dgrad, lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
@@ -334,7 +363,7 @@ class BlockHotPath:
                 gemm(fp8.fp8_linear_wgrad_rm, lin.dy.q, lin.x.q, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
         if self.attn is not None:
             a = self.attn
-            timed(qev, lambda: [a[n].quantize() for n in ("q", "k", "v", "do")])
+            timed(qev, lambda: [quant(a[n]) for n in ("q", "k", "v", "do")])
             timed(aev, fp8.fp8_attention_fwd, a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv,
                   a["v"].scale_inv, a["softmax_scale"], True, a["o"], a["lse"], None,
                   p_scale=448.0 / 2.0 ** self.attn_max_slack, max_slack=self.attn_max_slack)

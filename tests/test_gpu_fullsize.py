@@ -209,6 +209,44 @@ def test_host_to_host_step_equals_device_step():
         assert torch.equal(hout[n].view(torch.uint8), t.cpu().view(torch.uint8)), n
 
 
+def test_delayed_scaling_step_equals_the_just_in_time_step_on_repeated_inputs():
+    """With the same inputs every step, the abs-max history holds one value: the delayed-scaling step (one cast pass per
+    tensor under the history's scale, Appendix E) must return the bits of the just-in-time step; and when an input grows,
+    the step that sees it still casts (saturating) under the old scale and the next one under the new."""
+    cfg = synth.CONFIGS["c1"]
+    jit = BlockHotPath(cfg, "cuda")
+    h = jit.generate_host_inputs()
+    jit.allocate()
+    jit.calibrate_ds_scale()
+    jit.step()
+    torch.cuda.synchronize()
+    ref = {n: t.clone() for n, t in jit.output_tensors()}
+    dl = BlockHotPath(cfg, "cuda", scaling="delayed")
+    dl.allocate(h)
+    dl.attn["ds_scale"].copy_(jit.attn["ds_scale"])
+    for _ in range(3):
+        dl.step()
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    for n, t in dl.output_tensors():
+        assert torch.equal(t.view(torch.uint8), ref[n].view(torch.uint8)), n
+    assert dl.quantize_bytes() * 5 == jit.quantize_bytes() * 3            # 3 instead of 5 bytes per element
+    # an input doubles: this step's codes are those of the old scale, the next step's those of the new one
+    x = dl.linears[0].x
+    old_scale = float(x.scale.item())
+    x.x.copy_((x.x.float() * 2).to(torch.bfloat16))
+    dl.step()
+    torch.cuda.synchronize()
+    assert float(x.scale.item()) == old_scale
+    want = torch.empty_like(x.q)
+    fp8.fp8_cast(x.x, x.scale, x.fmt, want)
+    assert torch.equal(x.q, want)
+    dl.step()
+    torch.cuda.synchronize()
+    assert float(x.scale.item()) == old_scale / 2
+    assert fp8.fp8_device_status() == 0
+
+
 def test_graph_replay_of_the_step_equals_the_step():
     """The step makes no host synchronisation: captured into a CUDA graph and replayed it returns the same bits."""
     cfg = synth.CONFIGS["c1"]
