@@ -4,13 +4,15 @@
 // columns).  It walks over 64-query sub-tiles t (and the query heads of the group).  With rows = keys:
 //   S^T  = K  Q_t^T   [128 x 64]     dP^T = V dO_t^T   [128 x 64]          (64 TMEM columns, one slot per group)
 //   P~^T = 2^(c S^T - lse2_q),  P8^T = E4M3,  dS8^T = E5M2( P~^T o (a dP^T - db_q) )
-//   dV  += P8^T dO_t      dK += dS8^T Q_t      dQ_t^T = K^T dS8^T  [128(d) x 64]  (64 TMEM columns, two slots)
+//   dV  += P8^T dO_t      dK += dS8^T Q_t      dQ_t^T = K^T dS8^T  [128(d) x 64]  (64 TMEM columns, one slot)
 // Two element-wise warpgroups take the sub-tiles in turn (even t / odd t), one thread per key row and all 64
 // query columns, so the exponentials of one sub-tile overlap the dS arithmetic and the barrier round trips of
 // the other.  Each group owns one 64-column TMEM slot that holds S^T_t and then dP^T_t (issued as soon as the
-// group has S^T_t in registers), one P8/dS8 buffer in shared memory and one dQ^T slot.  dQ^T tiles leave through
-// two staging tiles in shared memory and one bulk reduce-add (binary32 add in L2) per sub-tile into the FP32
-// accumulator.
+// group has S^T_t in registers), 2 x 16 TMEM columns for P8^T_t and dS8^T_t (rows = keys is exactly the layout of
+// a left operand in TMEM: dV += P8^T dO and dK += dS8^T Q read them from there, four codes per column) and one
+// dS8^T tile in shared memory (the right operand of dQ^T = K^T dS8^T).  dQ^T tiles have one TMEM slot and leave
+// through two staging tiles in shared memory and one bulk reduce-add (binary32 add in L2) per sub-tile into the
+// FP32 accumulator.
 //
 // Warpgroups: 0 = control (warp 0 TMA producer, warp 1 MMA issuer), 1-2 = element-wise, 3 = dQ drain; registers
 // are moved from the control and drain groups to the element-wise groups (setmaxnreg).  Every wait is bounded.
@@ -42,18 +44,20 @@ struct Smem {
     static constexpr int STAGE_TX = 2 * Q_BYTES + 2 * VEC_BYTES;
     static constexpr int PDS_OFF = QDO_OFF + STAGES * STAGE_BYTES;
     static constexpr int PDS_TILE = KT * QT;                     // 8 KB: [128 key rows x 64 B]
-    static constexpr int PDS_BUF = 2 * PDS_TILE;                 // P8^T then dS8^T
+    static constexpr int PDS_BUF = PDS_TILE;                     // dS8^T (P8^T lives in TMEM only)
     static constexpr int DQ_OFF = PDS_OFF + 2 * PDS_BUF;
     static constexpr int DQ_BYTES = QT * D * 4;                  // 32 KB: [64 q x 128 d] FP32
     static constexpr int BAR_OFF = DQ_OFF + 2 * DQ_BYTES;          // two staging tiles
     // kv_full, qdo_full[S], qdo_empty[S], then per group: s_full, dp_full, s_read, dp_read, pds_full, pds_free,
-    // dq_full, dq_empty; all_done
+    // dq_full, dq_empty (of the two, index 0 serves the one dQ^T slot); all_done
     static constexpr int N_BARS = 1 + 2 * STAGES + 8 * 2 + 1;
     static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;
 };
 // TMEM columns
-constexpr uint32_t T_SD0 = 0, T_SD1 = 64, T_DQ0 = 128, T_DQ1 = 192, T_DV = 256, T_DK = 384;
+// S^T/dP^T slot per group, one dQ^T slot, per group 16 columns of P8^T and 16 of dS8^T (A operands of the dV and dK
+// products: lane = key, four codes per column), dV, dK
+constexpr uint32_t T_SD0 = 0, T_SD1 = 64, T_DQ = 128, T_P0 = 192, T_DS0 = 208, T_P1 = 224, T_DS1 = 240, T_DV = 256, T_DK = 384;
 
 struct Params {
     const float *lse2;     // [B,Hq,Npad]  -(LSE*log2(e) - log2(c_P)); -inf in the padding
@@ -147,6 +151,18 @@ __global__ void __launch_bounds__(256) attn_bwd_d128_finish_kernel(const float4 
         const float4 v = acc[i];
         dQ[i] = make_uint2(pack_bf16x2(v.x * f, v.y * f), pack_bf16x2(v.z * f, v.w * f));
     }
+}
+
+// D[tmem] (+)= A[tmem] * B[smem]: A = 128 rows (lanes) x 32 FP8 values in 8 consecutive 32-bit columns.
+__device__ __forceinline__ void umma_f8_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                           uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 
 template <int N> __device__ __forceinline__ void reg_dec()
@@ -296,23 +312,25 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const int e = t & 1;
                     const uint32_t u = (uint32_t)(t >> 1);
                     if (!mbar_wait(pds_full(e), u & 1u, ctx)) return false;
-                    if (u > 0 && !mbar_wait(dq_empty(e), (u - 1) & 1u, ctx)) return false;
+                    // one dQ^T slot: the drain must have taken sub-tile t-1 out of it
+                    if (t > 0 && !mbar_wait(dq_empty(0), (uint32_t)(t - 1) & 1u, ctx)) return false;
                     tc_fence_after();
-                    const uint32_t sp = sbase + L::PDS_OFF + e * L::PDS_BUF, sds = sp + L::PDS_TILE;
-                    const uint64_t d_p = umma_desc(sp, 64, 16), d_ds = umma_desc(sds, 64, 16);
+                    const uint32_t sds = sbase + L::PDS_OFF + e * L::PDS_BUF;
+                    const uint64_t d_ds = umma_desc(sds, 64, 16);
                     const uint64_t d_q = umma_desc(stage_q(t), 128, 16), d_do = umma_desc(stage_q(t) + L::Q_BYTES, 128, 16);
                     // dQ^T_t = K^T dS8^T_t: reduction over the 128 keys, 32 rows of either tile per step
 #pragma unroll
                     for (int k = 0; k < KT / 32; ++k)
-                        umma_f8_ss(tmem_base + (e ? T_DQ1 : T_DQ0), d_k + ROWS32_128 * k, d_ds + ROWS32_64 * k, id_dq, k != 0);
-                    umma_commit(dq_full(e));
-                    // dV += P8^T dO_t, dK += dS8^T Q_t: reduction over the 64 queries, 32 per step
+                        umma_f8_ss(tmem_base + T_DQ, d_k + ROWS32_128 * k, d_ds + ROWS32_64 * k, id_dq, k != 0);
+                    umma_commit(dq_full(0));
+                    // dV += P8^T dO_t, dK += dS8^T Q_t: reduction over the 64 queries, 32 per step; the left operands
+                    // come straight from TMEM (rows = keys is the layout the element-wise threads produce)
 #pragma unroll
                     for (int k = 0; k < QT / 32; ++k)
-                        umma_f8_ss(tmem_base + T_DV, d_p + 2u * k, d_do + ROWS32_128 * k, id_dv, (t | k) != 0);
+                        umma_f8_ts(tmem_base + T_DV, tmem_base + (e ? T_P1 : T_P0) + 8u * k, d_do + ROWS32_128 * k, id_dv, (t | k) != 0);
 #pragma unroll
                     for (int k = 0; k < QT / 32; ++k)
-                        umma_f8_ss(tmem_base + T_DK, d_ds + 2u * k, d_q + ROWS32_128 * k, id_dk, (t | k) != 0);
+                        umma_f8_ts(tmem_base + T_DK, tmem_base + (e ? T_DS1 : T_DS0) + 8u * k, d_q + ROWS32_128 * k, id_dk, (t | k) != 0);
                     umma_commit(qdo_empty(t % STAGES));
                     umma_commit(pds_free(e));
                     return true;
@@ -363,8 +381,7 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const float a_dp = __ldg(p.do_inv) * __ldg(p.v_inv) * dss / p.p_scale;
         const uint64_t c2 = pack_f32x2(c, c), a2 = pack_f32x2(a_dp, a_dp);
         const int sw = (r >> 1) & 3;                    // 64-byte swizzle: 16-byte chunk index ^ ((row >> 1) & 3)
-        uint8_t *prow = smem + L::PDS_OFF + e * L::PDS_BUF + r * 64;
-        uint8_t *dsrow = prow + L::PDS_TILE;
+        uint8_t *dsrow = smem + L::PDS_OFF + e * L::PDS_BUF + r * 64;
         float amax = 0.0f;
         bool ok = true;
         for (int t = e; t < n_iter; t += 2) {
@@ -405,17 +422,16 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
             // the P8/dS8 buffer of this group was last read by the MMAs of sub-tile t-2
             if (u > 0 && !mbar_wait_warp(pds_free(e), (u - 1) & 1u, ctx)) { ok = false; break; }
+            {
+                uint32_t wp[16];                         // P8^T row of this key: 64 codes, four per word
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                uint4 w;
-                w.x = cvt_f32x4_to_fp8x4<0>(pe[16 * ch], pe[16 * ch + 1], pe[16 * ch + 2], pe[16 * ch + 3]);
-                w.y = cvt_f32x4_to_fp8x4<0>(pe[16 * ch + 4], pe[16 * ch + 5], pe[16 * ch + 6], pe[16 * ch + 7]);
-                w.z = cvt_f32x4_to_fp8x4<0>(pe[16 * ch + 8], pe[16 * ch + 9], pe[16 * ch + 10], pe[16 * ch + 11]);
-                w.w = cvt_f32x4_to_fp8x4<0>(pe[16 * ch + 12], pe[16 * ch + 13], pe[16 * ch + 14], pe[16 * ch + 15]);
-                *reinterpret_cast<uint4 *>(prow + ((ch ^ sw) << 4)) = w;
+                for (int q = 0; q < 16; ++q)
+                    wp[q] = cvt_f32x4_to_fp8x4<0>(pe[4 * q], pe[4 * q + 1], pe[4 * q + 2], pe[4 * q + 3]);
+                tmem_st_32x32b_x16(tmem_base + (e ? T_P1 : T_P0) + lane_addr, wp);
             }
             if (!mbar_wait_warp(dp_full(e), u & 1u, ctx)) { ok = false; break; }
             tc_fence_after();
+            uint32_t wds[16];
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 uint32_t dv[32];
@@ -444,9 +460,13 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     w.y = cvt_f32x4_to_fp8x4<1>(pe[16 * ch + 4], pe[16 * ch + 5], pe[16 * ch + 6], pe[16 * ch + 7]);
                     w.z = cvt_f32x4_to_fp8x4<1>(pe[16 * ch + 8], pe[16 * ch + 9], pe[16 * ch + 10], pe[16 * ch + 11]);
                     w.w = cvt_f32x4_to_fp8x4<1>(pe[16 * ch + 12], pe[16 * ch + 13], pe[16 * ch + 14], pe[16 * ch + 15]);
-                    *reinterpret_cast<uint4 *>(dsrow + ((ch ^ sw) << 4)) = w;
+                    *reinterpret_cast<uint4 *>(dsrow + ((ch ^ sw) << 4)) = w;       // right operand of dQ^T
+                    wds[4 * ch] = w.x; wds[4 * ch + 1] = w.y; wds[4 * ch + 2] = w.z; wds[4 * ch + 3] = w.w;
                 }
             }
+            tmem_st_32x32b_x16(tmem_base + (e ? T_DS1 : T_DS0) + lane_addr, wds);      // left operand of dK
+            tmem_st_wait();
+            tc_fence_before();
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(pds_full(e));
@@ -491,17 +511,17 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         for (int t = 0; t < n_iter; ++t) {
             const int h = head_of(t), q0 = q0_of(t), e = t & 1;
             float *dq_s = reinterpret_cast<float *>(smem + L::DQ_OFF + e * L::DQ_BYTES);
-            const bool got = mbar_wait_warp(dq_full(e), (uint32_t)(t >> 1) & 1u, ctx);
+            const bool got = mbar_wait_warp(dq_full(0), (uint32_t)t & 1u, ctx);
             uint32_t va[32], vb[32];
             if (got) {
                 tc_fence_after();
-                const uint32_t src = tmem_base + (e ? T_DQ1 : T_DQ0) + lane_addr;
+                const uint32_t src = tmem_base + T_DQ + lane_addr;
                 tmem_ld_32x32b_x32(src, va);
                 tmem_ld_32x32b_x32(src + 32u, vb);
                 tmem_ld_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(dq_empty(e));   // the dQ^T slot may be overwritten
+                if (lane == 0) mbar_arrive(dq_empty(0));   // the dQ^T slot may be overwritten
             }
             // the reduce issued two sub-tiles ago must have finished reading this staging tile
             if (issuer) bulk_wait_group_read1();
