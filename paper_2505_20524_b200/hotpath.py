@@ -331,6 +331,50 @@ class BlockHotPath:
             self.step()
         return graph
 
+    def step_overlapped(self):
+        """The launches of step() on two streams: every quantize call goes to a side stream, the products and the
+        attention stay on the current one and wait (events) only for the operands they read.  The quantize passes are
+        HBM-bound and their CTAs fit beside the persistent GEMM CTAs of an SM, so they run in the shadow of the
+        products of the groups before them; only the first group's quantize is exposed.  Same kernels, same bits."""
+        main = torch.cuda.current_stream(self.device)
+        if getattr(self, "_qstream", None) is None:
+            self._qstream = torch.cuda.Stream(self.device)
+        side = self._qstream
+        side.wait_stream(main)              # the previous step's products have read the FP8 buffers about to be rewritten
+        quant = QTensor.quantize if self.scaling == "jit" else QTensor.quantize_delayed
+        ready = []
+        with torch.cuda.stream(side):
+            for lin in self.linears:
+                for t in (lin.x, lin.w, lin.dy):
+                    quant(t)
+                ev = torch.cuda.Event()
+                ev.record(side)
+                ready.append(ev)
+            if self.attn is not None:
+                for n in ("q", "k", "v", "do"):
+                    quant(self.attn[n])
+                ev = torch.cuda.Event()
+                ev.record(side)
+                ready.append(ev)
+        for lin, ev in zip(self.linears, ready):
+            main.wait_event(ev)
+            fp8.fp8_linear_fwd(lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
+            if self.transposed_copies:
+                fp8.fp8_linear_dgrad(lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+                fp8.fp8_linear_wgrad(lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+            else:
+                fp8.fp8_linear_dgrad_rm(lin.dy.q, lin.w.q, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+                fp8.fp8_linear_wgrad_rm(lin.dy.q, lin.x.q, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+        if self.attn is not None:
+            a = self.attn
+            main.wait_event(ready[-1])
+            fp8.fp8_attention_fwd(a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv, a["v"].scale_inv,
+                                  a["softmax_scale"], True, a["o"], a["lse"], None,
+                                  p_scale=448.0 / 2.0 ** self.attn_max_slack, max_slack=self.attn_max_slack)
+            fp8.fp8_attention_bwd(a["q"].q, a["k"].q, a["v"].q, a["do"].q, a["o"], a["lse"], a["q"].scale_inv,
+                                  a["k"].scale_inv, a["v"].scale_inv, a["do"].scale_inv, a["softmax_scale"],
+                                  a["ds_scale"], True, a["dq"], a["dk"], a["dv"], a["ws"], ds_amax=a["ds_amax"])
+
     def step(self, time_gemms: bool = False):
         """One pass of the hot path.  With ``time_gemms`` every GEMM launch, every quantize group and the two attention
         calls are bracketed by CUDA events on the launching stream (appended to gemm_events / quant_events /

@@ -247,6 +247,35 @@ def test_delayed_scaling_step_equals_the_just_in_time_step_on_repeated_inputs():
     assert fp8.fp8_device_status() == 0
 
 
+def test_overlapped_step_equals_the_step():
+    """Quantize calls on a side stream, products on the current one, ordered by events: the bits of step()."""
+    for name in ("c1", "c3"):
+        cfg = synth.CONFIGS[name]
+        hp = BlockHotPath(cfg, "cuda")
+        hp.generate_host_inputs()
+        hp.allocate()
+        hp.calibrate_ds_scale()
+        hp.step()
+        torch.cuda.synchronize()
+        ref = {n: t.clone() for n, t in hp.output_tensors()}
+        for _, t in hp.output_tensors():
+            t.zero_()
+        for _ in range(3):
+            hp.step_overlapped()
+        torch.cuda.synchronize()
+        assert fp8.fp8_device_status() == 0
+        for n, t in hp.output_tensors():
+            if n == "dq" and cfg.head_dim == 128:
+                # dQ is summed over key tiles by FP32 adds in L2 whose order follows the CTA schedule: equal up to that
+                # rounding from run to run, whichever streams the step uses
+                a, b = t.float(), ref[n].float()
+                assert float((a - b).abs().max()) <= 2.0 ** -7 * float(b.abs().max()), (name, n)
+            else:
+                assert torch.equal(t.view(torch.uint8), ref[n].view(torch.uint8)), (name, n)
+        del hp, ref
+        torch.cuda.empty_cache()
+
+
 def test_graph_replay_of_the_step_equals_the_step():
     """The step makes no host synchronisation: captured into a CUDA graph and replayed it returns the same bits."""
     cfg = synth.CONFIGS["c1"]
