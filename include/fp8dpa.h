@@ -326,7 +326,8 @@ FP8_API int fp8_attention_bwd(const uint8_t *Q8, const uint8_t *K8, const uint8_
  * holds that array until the process exits.  The call allocates nothing (no cudaMalloc / cudaFree, no
  * allocating library routine).
  *
- * Limit: fp8_attention_workspace_bytes(1, B, N, Hq, Hkv, d), about B*N*Hq*(d+1)*4 bytes, must not exceed
+ * Limit: fp8_attention_workspace_bytes(1, B, N, Hq, Hkv, d), about B*N*Hq*(d+1)*4 bytes for d = 64 and
+ * B*N*Hq*(d+8)*4 for d = 128, must not exceed
  * FP8_STATIC_SCRATCH_BYTES; larger problems return FP8_ERR_WORKSPACE and launch nothing.
  * The first call on each device looks up the array's device address (with that device current); make that
  * first call before any stream capture begins.

@@ -165,6 +165,27 @@ int make_tmap_3d_f32(CUtensorMap *map, const void *base, uint64_t d0_cols, uint6
     return FP8_OK;
 }
 
+// Rank-2 map over a [rows, 16] BF16 array (32-byte rows) with the 32-byte swizzle: the right operand of a K = 16
+// tcgen05.mma.kind::f16 step, one row per output column.
+int make_tmap_2d_bf16x16(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows)
+{
+    int rc = load_encoder();
+    if (rc != FP8_OK) return rc;
+    cuuint64_t dims[2] = {16, rows};
+    cuuint64_t strides[1] = {32};
+    cuuint32_t box[2] = {16, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled (rank 2, bf16 x 16) failed (CUresult %d) rows=%llu box=%u", (int)r,
+                  (unsigned long long)rows, box_rows);
+        return FP8_ERR_CUDA;
+    }
+    return FP8_OK;
+}
+
 // One warp waits on a barrier that nothing ever completes, with a short limit: the path every kernel of the library
 // takes when a wait runs out (status word, shared abort flag, orderly return).
 __global__ void wait_timeout_selftest_kernel(int *status, long long limit, int *gave_up)

@@ -5,6 +5,12 @@
 //   S^T  = K  Q_t^T   [128 x 64]     dP^T = V dO_t^T   [128 x 64]          (64 TMEM columns, one slot per group)
 //   P~^T = 2^(c S^T - lse2_q),  P8^T = E4M3,  dS8^T = E5M2( P~^T o (a dP^T - db_q) )
 //   dV  += P8^T dO_t      dK += dS8^T Q_t      dQ_t^T = K^T dS8^T  [128(d) x 64]  (64 TMEM columns, one slot)
+// The per-query terms lse2_q and db_q never reach the element-wise threads as data: the prep kernel writes them,
+// divided by c resp. a and split into three BF16 terms, as one row of 16 BF16 per query, and the tensor core adds them
+// to the accumulators with one K = 16 BF16 product each (a tile of ones x that row), so that S^T and dP^T arrive as
+// S^T - lse2_q / c and dP^T - db_q / a and one multiplication is left.  A shared-memory load in front of every pair
+// of columns was what bounded these threads: while the tensor core streams operands out of shared memory, a
+// dependent ld.shared takes several times its idle latency (measured: the exponential phase 1375 -> 650 clk).
 // Two element-wise warpgroups take the sub-tiles in turn (even t / odd t), one thread per key row and all 64
 // query columns, so the exponentials of one sub-tile overlap the dS arithmetic and the barrier round trips of
 // the other.  Each group owns one 64-column TMEM slot that holds S^T_t and then dP^T_t (issued as soon as the
@@ -16,6 +22,7 @@
 //
 // Warpgroups: 0 = control (warp 0 TMA producer, warp 1 MMA issuer), 1-2 = element-wise, 3 = dQ drain; registers
 // are moved from the control and drain groups to the element-wise groups (setmaxnreg).  Every wait is bounded.
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <math.h>
 
@@ -39,13 +46,17 @@ struct Smem {
     static constexpr int V_OFF = K_OFF + KT * D;
     static constexpr int QDO_OFF = V_OFF + KT * D;
     static constexpr int Q_BYTES = QT * D;                       // 8 KB
-    static constexpr int VEC_BYTES = QT * 4;                     // 256 B
-    static constexpr int STAGE_BYTES = 2 * Q_BYTES + 2 * 1024;   // Q, dO, lse2 (padded to 1 KB), db (1 KB)
-    static constexpr int STAGE_TX = 2 * Q_BYTES + 2 * VEC_BYTES;
+    static constexpr int VEC_BYTES = QT * 32;                    // 2 KB: per query 16 BF16 (shift of S^T, shift of dP^T)
+    static constexpr int STAGE_BYTES = 2 * Q_BYTES + VEC_BYTES;  // Q, dO, the per-query shifts
+    static constexpr int STAGE_TX = STAGE_BYTES;
     static constexpr int PDS_OFF = QDO_OFF + STAGES * STAGE_BYTES;
     static constexpr int PDS_TILE = KT * QT;                     // 8 KB: [128 key rows x 64 B]
     static constexpr int PDS_BUF = PDS_TILE;                     // dS8^T (P8^T lives in TMEM only)
-    static constexpr int DQ_OFF = PDS_OFF + 2 * PDS_BUF;
+    // left operands of the two rank-one products that add the per-query shifts: [128 keys x 16 BF16], ones in the
+    // columns of the shift they pick (32-byte swizzle)
+    static constexpr int ONES_OFF = PDS_OFF + 2 * PDS_BUF;
+    static constexpr int ONES_BYTES = KT * 32;                   // 4 KB each
+    static constexpr int DQ_OFF = ONES_OFF + 2 * ONES_BYTES;
     static constexpr int DQ_BYTES = QT * D * 4;                  // 32 KB: [64 q x 128 d] FP32
     static constexpr int BAR_OFF = DQ_OFF + 2 * DQ_BYTES;          // two staging tiles
     // kv_full, qdo_full[S], qdo_empty[S], then per group: s_full, dp_full, s_read, dp_read, pds_full, pds_free,
@@ -60,8 +71,6 @@ struct Smem {
 constexpr uint32_t T_SD0 = 0, T_SD1 = 64, T_DQ = 128, T_P0 = 192, T_DS0 = 208, T_P1 = 224, T_DS1 = 240, T_DV = 256, T_DK = 384;
 
 struct Params {
-    const float *lse2;     // [B,Hq,Npad]  -(LSE*log2(e) - log2(c_P)); -inf in the padding
-    const float *db;       // [B,Hq,Npad]  -D * ds_scale / c_P; 0 in the padding
     uint16_t *dK, *dV;     // [B,N,Hkv,D] BF16
     const float *q_inv, *k_inv, *v_inv, *do_inv, *ds_scale;
     float *ds_amax;
@@ -77,19 +86,38 @@ __device__ __forceinline__ float e5m2_to_f32(uint32_t code)
 }
 
 // ---------------------------------------------------------------- prep
-// Eight lanes per (b, i, h) with i < Npad (16-byte loads): D_i = do_inv * sum_d dec(dO8) * O, then
-// lse2 = -(LSE*log2e - log2(c_P)), db = -D * ds_scale / c_P; rows i >= N get (-inf, 0); the dQ accumulator row
-// is zeroed.
+// Eight lanes per (b, i, h) with i < Npad (16-byte loads): D_i = do_inv * sum_d dec(dO8) * O, then the two per-query
+// shifts of the main kernel, each already divided by the factor its accumulator is multiplied with afterwards:
+//   L_i  = (log2(c_P) - LSE_i * log2(e)) / c      so that c * (S^T + L)  = c S^T - lse2        (exponent of c_P * P)
+//   Db_i = (-D_i * ds_scale / c_P) / a            so that a * (dP^T + Db) = a dP^T - db        (factor of dS)
+// Both go out as three BF16 terms (hi + mid + lo = the binary32 value exactly) in a row of 16 BF16: L in columns 0-2,
+// Db in columns 8-10, zeros elsewhere.  The main kernel adds them to its accumulators with one K = 16 BF16 product each
+// (ones x row), so its element-wise threads never load a per-query value.  Rows i >= N get L = -2^100 (P = 0) and
+// Db = 0; the dQ accumulator row is zeroed.
+__device__ __forceinline__ uint32_t bf16_rn_bits(float x) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+__device__ __forceinline__ void split3_bf16(float x, uint32_t &hi, uint32_t &mid, uint32_t &lo)
+{
+    hi = bf16_rn_bits(x);
+    const float r1 = x - __uint_as_float(hi << 16);
+    mid = bf16_rn_bits(r1);
+    const float r2 = r1 - __uint_as_float(mid << 16);
+    lo = bf16_rn_bits(r2);
+}
 __global__ void __launch_bounds__(256) attn_bwd_d128_prep_kernel(const uint8_t *__restrict__ dO8, const uint16_t *__restrict__ O,
-                                                   const float *__restrict__ LSE, const float *__restrict__ do_inv,
-                                                   const float *__restrict__ ds_scale, float p_scale,
-                                                   float log2_p_scale, float *__restrict__ lse2,
-                                                   float *__restrict__ db, float *__restrict__ dQacc, int B, int N,
+                                                   const float *__restrict__ LSE, const float *__restrict__ q_inv,
+                                                   const float *__restrict__ k_inv, const float *__restrict__ v_inv,
+                                                   const float *__restrict__ do_inv,
+                                                   const float *__restrict__ ds_scale, float softmax_scale, float p_scale,
+                                                   float log2_p_scale, uint4 *__restrict__ vec,
+                                                   float *__restrict__ dQacc, int B, int N,
                                                    int Npad, int Hq)
 {
     const long n_rows = (long)B * Npad * Hq;
     const int j = threadIdx.x & 7;
     const float scale = __ldg(do_inv) * __ldg(ds_scale) / p_scale;
+    // the same expressions as in the main kernel
+    const float c = softmax_scale * __ldg(q_inv) * __ldg(k_inv) * 1.4426950408889634f;
+    const float a_dp = __ldg(do_inv) * __ldg(v_inv) * __ldg(ds_scale) / p_scale;
     // the trip count is uniform over the CTA: the shuffles below name every lane
     for (long base = (long)blockIdx.x * 32; base < n_rows; base += (long)gridDim.x * 32) {
         const long w_raw = base + (threadIdx.x >> 3);            // (b*Npad + i)*Hq + h
@@ -103,10 +131,10 @@ __global__ void __launch_bounds__(256) attn_bwd_d128_prep_kernel(const uint8_t *
         const size_t row = ((size_t)b * N + (real ? i : 0)) * Hq + h;
         float acc = 0.0f;
         if (real) {
-            const uint4 c = __ldg(reinterpret_cast<const uint4 *>(dO8 + row * D + j * 16));
+            const uint4 cw4 = __ldg(reinterpret_cast<const uint4 *>(dO8 + row * D + j * 16));
             const uint4 o0 = __ldg(reinterpret_cast<const uint4 *>(O + row * D + j * 16));
             const uint4 o1 = __ldg(reinterpret_cast<const uint4 *>(O + row * D + j * 16 + 8));
-            const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
+            const uint32_t cw[4] = {cw4.x, cw4.y, cw4.z, cw4.w};
             const uint32_t ow[8] = {o0.x, o0.y, o0.z, o0.w, o1.x, o1.y, o1.z, o1.w};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -125,8 +153,16 @@ __global__ void __launch_bounds__(256) attn_bwd_d128_prep_kernel(const uint8_t *
             z[0] = zero; z[1] = zero; z[2] = zero; z[3] = zero;
         }
         if (j == 0) {
-            lse2[vi] = real ? log2_p_scale - __ldg(LSE + ((size_t)b * Hq + h) * N + i) * 1.4426950408889634f : -INFINITY;
-            db[vi] = real ? -acc * scale : 0.0f;
+            uint32_t l0 = 0xF180u, l1 = 0, l2 = 0, d0 = 0, d1 = 0, d2 = 0;          // 0xF180 = -2^100 in BF16
+            if (real) {
+                const float nl = log2_p_scale - __ldg(LSE + ((size_t)b * Hq + h) * N + i) * 1.4426950408889634f;
+                const float L = fminf(fmaxf(__fdiv_rn(nl, c), -1e30f), 1e30f);
+                const float Db = fminf(fmaxf(__fdiv_rn(-acc * scale, a_dp), -1e30f), 1e30f);
+                split3_bf16(L, l0, l1, l2);
+                split3_bf16(Db, d0, d1, d2);
+            }
+            vec[2 * vi] = make_uint4(l0 | (l1 << 16), l2, 0u, 0u);
+            vec[2 * vi + 1] = make_uint4(d0 | (d1 << 16), d2, 0u, 0u);
         }
     }
 }
@@ -178,7 +214,7 @@ template <int N> __device__ __forceinline__ void reg_inc()
 __global__ void __launch_bounds__(THREADS, 1)
 attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
             const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-            const __grid_constant__ CUtensorMap tm_dq, const Params p)
+            const __grid_constant__ CUtensorMap tm_dq, const __grid_constant__ CUtensorMap tm_vec, const Params p)
 {
     using L = Smem;
     extern __shared__ uint8_t smem_raw[];
@@ -242,7 +278,19 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         tma_prefetch_desc(&tm_v);
         tma_prefetch_desc(&tm_do);
         tma_prefetch_desc(&tm_dq);
+        tma_prefetch_desc(&tm_vec);
     }
+    // the two ones-tiles: row r holds BF16 ones in columns 0-3 (picks L) resp. 8-11 (picks Db), zeros elsewhere; under
+    // the 32-byte swizzle the 16-byte half c of row r lies at half c ^ ((r >> 2) & 1)
+    if (threadIdx.x < 2 * KT) {
+        const int which = threadIdx.x / KT, r = threadIdx.x % KT;
+        uint4 *rowp = reinterpret_cast<uint4 *>(smem + L::ONES_OFF + which * L::ONES_BYTES + r * 32);
+        const uint4 ones = make_uint4(0x3F803F80u, 0x3F803F80u, 0u, 0u), zero = make_uint4(0u, 0u, 0u, 0u);
+        const int flip = (r >> 2) & 1;
+        rowp[which ^ flip] = ones;
+        rowp[(which ^ 1) ^ flip] = zero;
+    }
+    fence_proxy_async_smem();
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
@@ -267,13 +315,12 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const int h = head_of(t), q0 = q0_of(t);
                     if (!mbar_wait(qdo_empty(st), ph ^ 1u, ctx)) break;
                     const uint32_t sq = sbase + L::QDO_OFF + st * L::STAGE_BYTES, sdo = sq + L::Q_BYTES;
-                    const uint32_t sl = sdo + L::Q_BYTES, sd = sl + 1024;
-                    const size_t vi = ((size_t)b * p.Hq + h) * p.Npad + q0;
+                    const uint32_t sl = sdo + L::Q_BYTES;
+                    const int vrow = (b * p.Hq + h) * p.Npad + q0;
                     mbar_expect_tx(qdo_full(st), L::STAGE_TX);
                     tma_load_3d(sq, &tm_q, qdo_full(st), h * D, q0, b);
                     tma_load_3d(sdo, &tm_do, qdo_full(st), h * D, q0, b);
-                    bulk_load_1d(sl, p.lse2 + vi, L::VEC_BYTES, qdo_full(st));
-                    bulk_load_1d(sd, p.db + vi, L::VEC_BYTES, qdo_full(st));
+                    tma_load_2d(sl, &tm_vec, qdo_full(st), 0, vrow);
                 }
             }
         } else if (warp == 1) {
@@ -285,6 +332,9 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 constexpr uint32_t id_dv = umma_idesc_f8(E4, E5, 128, D, 0, 1);      // P8^T (K-major) x dO (MN)
                 constexpr uint32_t id_dk = umma_idesc_f8(E5, E4, 128, D, 0, 1);      // dS8^T (K-major) x Q (MN)
                 constexpr uint32_t id_dq = umma_idesc_f8(E4, E5, 128, QT, 1, 1);     // K^T (MN) x dS8^T (MN)
+                constexpr uint32_t id_vec = umma_idesc_f8(1, 1, 128, QT, 0, 0);      // kind::f16: BF16 ones x BF16 shifts
+                const uint64_t d_ones_l = umma_desc_k_sw32(sbase + L::ONES_OFF);
+                const uint64_t d_ones_d = umma_desc_k_sw32(sbase + L::ONES_OFF + L::ONES_BYTES);
                 const uint64_t d_k = umma_desc(sbase + L::K_OFF, 128, 16);
                 const uint64_t d_v = umma_desc(sbase + L::V_OFF, 128, 16);
                 constexpr uint32_t ROWS32_128 = (32 * 128) >> 4;   // 32 rows of a 128-byte-row tile
@@ -298,6 +348,8 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const uint32_t dst = tmem_base + ((t & 1) ? T_SD1 : T_SD0);
 #pragma unroll
                     for (int k = 0; k < D / 32; ++k) umma_f8_ss(dst, d_k + 2u * k, d_q + 2u * k, id_s, k != 0);
+                    // + 1 x L_q: the accumulator leaves as S^T - lse2 / c
+                    umma_bf16_ss(dst, d_ones_l, umma_desc_k_sw32(stage_q(t) + 2 * L::Q_BYTES), id_vec, 1u);
                     umma_commit(s_full(t & 1));
                 };
                 auto issue_dp = [&](int t) {    // dP^T_t = V dO_t^T into the same slot, once S^T_t is in registers
@@ -305,6 +357,8 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const uint32_t dst = tmem_base + ((t & 1) ? T_SD1 : T_SD0);
 #pragma unroll
                     for (int k = 0; k < D / 32; ++k) umma_f8_ss(dst, d_v + 2u * k, d_do + 2u * k, id_dp, k != 0);
+                    // + 1 x Db_q: the accumulator leaves as dP^T - db / a
+                    umma_bf16_ss(dst, d_ones_d, umma_desc_k_sw32(stage_q(t) + 2 * L::Q_BYTES), id_vec, 1u);
                     umma_commit(dp_full(t & 1));
                 };
                 // dQ^T_t, dV, dK of sub-tile t, once P8^T_t and dS8^T_t are in shared memory
@@ -386,13 +440,10 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         bool ok = true;
         for (int t = e; t < n_iter; t += 2) {
             const uint32_t u = (uint32_t)(t >> 1);
-            const int q0 = q0_of(t), st = t % STAGES;
+            const int q0 = q0_of(t);
             // valid iff key <= query (causal) and key < N; queries >= N carry -lse2 = -inf
             const bool need_mask = (p.causal && q0 < k0 + KT - 1) || (k0 + KT > p.N);
             const int first_ok = (key < p.N) ? (p.causal ? key - q0 : 0) : 64;   // columns >= first_ok are valid
-            const float *nlse2 = reinterpret_cast<const float *>(smem + L::QDO_OFF + st * L::STAGE_BYTES + 2 * L::Q_BYTES);
-            const float *ndb = nlse2 + 256;
-            if (!mbar_wait_warp(qdo_full(st), (uint32_t)(t / STAGES) & 1u, ctx)) { ok = false; break; }
             if (!mbar_wait_warp(s_full(e), u & 1u, ctx)) { ok = false; break; }
             tc_fence_after();
             float pe[64];
@@ -406,11 +457,10 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (lane == 0) mbar_arrive(s_read(e));   // the slot may take dP^T_t
 #pragma unroll
                 for (int i = 0; i < 64; i += 2) {
-                    const float2 l2 = *reinterpret_cast<const float2 *>(nlse2 + i);     // -lse2 of two queries
+                    // the accumulator already carries the per-query shift (rank-one product): one multiply is left
                     const uint32_t *sx = i < 32 ? sa + i : sb + (i - 32);
                     float x0, x1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sx[0]), __uint_as_float(sx[1])), c2,
-                                           pack_f32x2(l2.x, l2.y)), x0, x1);
+                    unpack_f32x2(mul_f32x2(pack_u32x2(sx[0], sx[1]), c2), x0, x1);
                     pe[i] = ex2_approx(x0);             // c_P * P
                     pe[i + 1] = ex2_approx(x1);
                 }
@@ -444,11 +494,9 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 }
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const float2 d2 = *reinterpret_cast<const float2 *>(ndb + 32 * hf + i);   // -db of two queries
                     float y0, y1;
                     unpack_f32x2(mul_f32x2(pack_f32x2(pe[32 * hf + i], pe[32 * hf + i + 1]),
-                                           fma_f32x2(pack_f32x2(__uint_as_float(dv[i]), __uint_as_float(dv[i + 1])), a2,
-                                                     pack_f32x2(d2.x, d2.y))), y0, y1);
+                                           mul_f32x2(pack_u32x2(dv[i], dv[i + 1]), a2)), y0, y1);
                     pe[32 * hf + i] = y0;                // ds_scale * dS
                     pe[32 * hf + i + 1] = y1;
                     amax = fmaxf(amax, fmaxf(fabsf(y0), fabsf(y1)));
@@ -558,9 +606,10 @@ attn_bwd_d128_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
 size_t attn_bwd_d128_ws_bytes(int B, int N, int Hq)
 {
+    // per (batch, head, padded query) one row of 16 BF16 (the two shifts), then the FP32 dQ accumulator
     const size_t Npad = ((size_t)N + bwd128::QT - 1) / bwd128::QT * bwd128::QT;
-    const size_t vec = (((size_t)B * Hq * Npad * sizeof(float)) + 255) & ~(size_t)255;
-    return 2 * vec + (size_t)B * N * Hq * bwd128::D * sizeof(float);
+    const size_t vec = (((size_t)B * Hq * Npad * 32) + 255) & ~(size_t)255;
+    return vec + (size_t)B * N * Hq * bwd128::D * sizeof(float);
 }
 
 int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const uint8_t *dO8,
@@ -570,11 +619,10 @@ int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8
 {
     using namespace bwd128;
     const int Npad = (N + QT - 1) / QT * QT;
-    const size_t vec = (((size_t)B * Hq * Npad * sizeof(float)) + 255) & ~(size_t)255;
-    float *lse2 = static_cast<float *>(ws);
-    float *db = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + vec);
-    float *dQacc = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + 2 * vec);
-    CUtensorMap tq, tk, tv, tdo, tdq;
+    const size_t vec = (((size_t)B * Hq * Npad * 32) + 255) & ~(size_t)255;
+    uint4 *shifts = static_cast<uint4 *>(ws);
+    float *dQacc = reinterpret_cast<float *>(static_cast<uint8_t *>(ws) + vec);
+    CUtensorMap tq, tk, tv, tdo, tdq, tvec;
     int rc = make_tmap_3d_u8(&tq, Q8, (uint64_t)Hq * D, (uint64_t)N, (uint64_t)B, D, QT);
     if (rc != FP8_OK) return rc;
     rc = make_tmap_3d_u8(&tk, K8, (uint64_t)Hkv * D, (uint64_t)N, (uint64_t)B, D, KT);
@@ -585,16 +633,18 @@ int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8
     if (rc != FP8_OK) return rc;
     rc = make_tmap_3d_f32(&tdq, dQacc, (uint64_t)Hq * D, (uint64_t)N, (uint64_t)B, D, QT);
     if (rc != FP8_OK) return rc;
+    rc = make_tmap_2d_bf16x16(&tvec, shifts, (uint64_t)B * Hq * Npad, QT);
+    if (rc != FP8_OK) return rc;
     if (sc->ds_amax) FP8_CUDA_CHECK(cudaMemsetAsync(sc->ds_amax, 0, sizeof(float), st));
     const float log2_p = log2f(sc->p_scale);
     const long prep_rows = (long)B * Npad * Hq;
     long prep_blocks = (prep_rows + 31) / 32;                   // 32 rows per CTA and sweep
     if (prep_blocks > (long)sm_count() * 16) prep_blocks = (long)sm_count() * 16;
-    attn_bwd_d128_prep_kernel<<<(unsigned)prep_blocks, 256, 0, st>>>(dO8, O, LSE, sc->do_inv, sc->ds_scale, sc->p_scale, log2_p,
-                                                            lse2, db, dQacc, B, N, Npad, Hq);
+    attn_bwd_d128_prep_kernel<<<(unsigned)prep_blocks, 256, 0, st>>>(dO8, O, LSE, sc->q_inv, sc->k_inv, sc->v_inv, sc->do_inv,
+                                                            sc->ds_scale, sc->softmax_scale, sc->p_scale, log2_p, shifts,
+                                                            dQacc, B, N, Npad, Hq);
     FP8_CUDA_CHECK(cudaGetLastError());
     Params p;
-    p.lse2 = lse2; p.db = db;
     p.dK = dK; p.dV = dV;
     p.q_inv = sc->q_inv; p.k_inv = sc->k_inv; p.v_inv = sc->v_inv; p.do_inv = sc->do_inv;
     p.ds_scale = sc->ds_scale;
@@ -606,7 +656,7 @@ int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8
     p.status = status;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_d128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::DYN_BYTES));
     dim3 grid((unsigned)(Hkv * B), (unsigned)((N + KT - 1) / KT), 1);
-    attn_bwd_d128_kernel<<<grid, THREADS, Smem::DYN_BYTES, st>>>(tq, tk, tv, tdo, tdq, p);
+    attn_bwd_d128_kernel<<<grid, THREADS, Smem::DYN_BYTES, st>>>(tq, tk, tv, tdo, tdq, tvec, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     const size_t n4 = (size_t)B * N * Hq * D / 4;
     size_t blocks = (n4 + 255) / 256;

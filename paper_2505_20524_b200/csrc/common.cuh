@@ -22,6 +22,7 @@ int make_tmap_2d_u8(CUtensorMap *map, const void *base, uint64_t rows, uint64_t 
 
 int make_tmap_3d_u8(CUtensorMap *map, const void *base, uint64_t d0_cols, uint64_t d1_rows, uint64_t d2_batch,
                     uint32_t box_cols, uint32_t box_rows);
+int make_tmap_2d_bf16x16(CUtensorMap *map, const void *base, uint64_t rows, uint32_t box_rows);
 
 int make_tmap_3d_f32(CUtensorMap *map, const void *base, uint64_t d0_cols, uint64_t d1_rows, uint64_t d2_batch,
                      uint32_t box_cols, uint32_t box_rows);
@@ -276,6 +277,29 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, int swizzle_bytes,
     d |= (uint64_t)1 << 46;
     d |= (uint64_t)(swizzle_bytes == 128 ? 2 : 4) << 61;   // SWIZZLE_128B = 2, SWIZZLE_64B = 4
     return d;
+}
+// K-major operand whose rows are 32 bytes (16 BF16 of the reduction index), 32-byte swizzle: 8 rows per 256-byte atom.
+__device__ __forceinline__ uint64_t umma_desc_k_sw32(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(256 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)6 << 61;                       // SWIZZLE_32B
+    return d;
+}
+// D[tmem] (+)= A[smem] * B[smem] with BF16 operands (K = 16 per instruction), FP32 accumulate; the instruction descriptor
+// has the layout of umma_idesc_f8 with format 1 = BF16 in both operand fields.
+__device__ __forceinline__ void umma_bf16_ss(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 // Instruction descriptor of tcgen05.mma.kind::f8f6f4 with FP32 accumulate.  fmt: 0 = E4M3, 1 = E5M2;
 // *_mn = 1 when that operand is MN-major (output index contiguous) instead of K-major.

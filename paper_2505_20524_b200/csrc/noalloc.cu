@@ -53,7 +53,7 @@ extern "C" int fp8_attention_bwd_static(const uint8_t *Q8, const uint8_t *K8, co
     }
     if (need > (size_t)FP8_STATIC_SCRATCH_BYTES) {
         set_error("fp8_attention_bwd_static: this problem needs %zu bytes of scratch but the built-in array holds %zu "
-                  "(B*N*Hq*(d+1)*4 must not exceed it); use fp8_attention_bwd with a caller workspace",
+                  "(about B*N*Hq*(d+8)*4 must not exceed it); use fp8_attention_bwd with a caller workspace",
                   need, (size_t)FP8_STATIC_SCRATCH_BYTES);
         return FP8_ERR_WORKSPACE;
     }
