@@ -331,7 +331,7 @@ class BlockHotPath:
             self.step()
         return graph
 
-    def step_overlapped(self):
+    def step_overlapped(self, time_gemms: bool = False):
         """The launches of step() on two streams: every quantize call goes to a side stream, the products and the
         attention stay on the current one and wait (events) only for the operands they read.  The quantize passes are
         HBM-bound and their CTAs fit beside the persistent GEMM CTAs of an SM, so they run in the shadow of the
@@ -356,15 +356,29 @@ class BlockHotPath:
                 ev = torch.cuda.Event()
                 ev.record(side)
                 ready.append(ev)
+        gev = []
+
+        def gemm(fn, *args):
+            if time_gemms:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                fn(*args)
+                e1.record()
+                gev.append((e0, e1))
+            else:
+                fn(*args)
+
         for lin, ev in zip(self.linears, ready):
             main.wait_event(ev)
-            fp8.fp8_linear_fwd(lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
+            gemm(fp8.fp8_linear_fwd, lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
             if self.transposed_copies:
-                fp8.fp8_linear_dgrad(lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
-                fp8.fp8_linear_wgrad(lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+                gemm(fp8.fp8_linear_dgrad, lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+                gemm(fp8.fp8_linear_wgrad, lin.dy.qt, lin.x.qt, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
             else:
-                fp8.fp8_linear_dgrad_rm(lin.dy.q, lin.w.q, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
-                fp8.fp8_linear_wgrad_rm(lin.dy.q, lin.x.q, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+                gemm(fp8.fp8_linear_dgrad_rm, lin.dy.q, lin.w.q, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
+                gemm(fp8.fp8_linear_wgrad_rm, lin.dy.q, lin.x.q, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
+        if time_gemms:
+            self.gemm_events.append(gev)
         if self.attn is not None:
             a = self.attn
             main.wait_event(ready[-1])
