@@ -341,6 +341,42 @@ FP8_API int fp8_attention_bwd_static(const uint8_t *Q8, const uint8_t *K8, const
                              int causal, int B, int N, int Hq, int Hkv, int d,
                              void *dQ_bf16, void *dK_bf16, void *dV_bf16, void *stream);
 
+/* ---- host-buffer forms ------------------------------------------------------------------------------
+ * (No counterpart in the paper: packaging of the calls above for a caller whose tensors live in HOST memory.)
+ *
+ * fp8_linear_step_host: one linear layer's training step (Appendix E, throughput table) from BF16 HOST tensors
+ * X[T,K], W[N,K], dY[T,N] to BF16 HOST tensors Y[T,N], dX[T,K], dW[N,K]: upload, fp8_quantize of X and W
+ * (E4M3) and dY (E5M2) with just-in-time scales, fp8_linear_fwd, fp8_linear_dgrad_rm, fp8_linear_wgrad_rm,
+ * download.  T, N, K multiples of 16.
+ * fp8_attention_step_host: one attention's training step (Appendix B, Eq. (P)) from BF16 HOST tensors
+ * Q, dO [B,N,Hq,d] and K, V [B,N,Hkv,d] to HOST O, dQ [B,N,Hq,d] (BF16), LSE [B,Hq,N] (FP32) and
+ * dK, dV [B,N,Hkv,d] (BF16): upload, fp8_quantize of Q, K, V (E4M3) and dO (E5M2), fp8_attention_fwd with
+ * p_scale = 448 and max_slack = 0, fp8_attention_bwd with the given ds_scale (a host value), download.
+ * Results are bit-identical to the same chain of device-pointer calls.
+ *
+ * Pointers: every h* argument is HOST memory, owned by the caller; pinned (page-locked) memory is needed
+ * for the copies to overlap anything, pageable memory is correct but serialises.  `ws` is DEVICE memory,
+ * 256-byte aligned, of at least fp8_*_step_host_workspace_bytes(...) bytes (0 = unsupported shape); it
+ * holds the uploaded tensors, their FP8 copies, the results and the scratch, and its contents are
+ * unspecified afterwards.
+ * Ordering: the calls enqueue on three streams owned by the library (uploads, kernels, downloads; one
+ * set per device) and return without waiting, so that with two or more workspaces in rotation the
+ * copies of one call run under the kernels of another.  A workspace may be reused at once: the library
+ * orders the new call after the previous call on the same `ws` address.  Inputs must stay unchanged and
+ * outputs are undefined until fp8_host_sync() has returned FP8_OK; it waits for every host-buffer call made
+ * so far on the current device.  The calls are serialised by an internal lock and may come from any
+ * host thread.  Errors: FP8_ERR_NULL, FP8_ERR_SHAPE, FP8_ERR_WORKSPACE before anything is enqueued; an
+ * error of an inner call is returned as is, with the work enqueued before it left to finish. */
+FP8_API size_t fp8_linear_step_host_workspace_bytes(int T, int N, int K);
+FP8_API int fp8_linear_step_host(const void *hX_bf16, const void *hW_bf16, const void *hdY_bf16, int T, int N, int K,
+                         void *hY_bf16, void *hdX_bf16, void *hdW_bf16, void *ws, size_t ws_bytes);
+FP8_API size_t fp8_attention_step_host_workspace_bytes(int B, int N, int Hq, int Hkv, int d);
+FP8_API int fp8_attention_step_host(const void *hQ_bf16, const void *hK_bf16, const void *hV_bf16, const void *hdO_bf16,
+                            int B, int N, int Hq, int Hkv, int d, float softmax_scale, float ds_scale, int causal,
+                            void *hO_bf16, float *hLSE, void *hdQ_bf16, void *hdK_bf16, void *hdV_bf16,
+                            void *ws, size_t ws_bytes);
+FP8_API int fp8_host_sync(void);
+
 #ifdef __cplusplus
 }
 #endif

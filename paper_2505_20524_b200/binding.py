@@ -23,7 +23,9 @@ _lib = None
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis", "fp8_amax_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_linear_dgrad_blockwise", "fp8_linear_wgrad_blockwise", "fp8_attention_workspace_bytes",
-           "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static"]
+           "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static",
+           "fp8_linear_step_host_workspace_bytes", "fp8_linear_step_host", "fp8_attention_step_host_workspace_bytes",
+           "fp8_attention_step_host", "fp8_host_sync"]
 
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -54,6 +56,11 @@ def load() -> C.CDLL:
         if hasattr(lib, "fp8_attention_workspace_bytes"):
             lib.fp8_attention_workspace_bytes.restype = C.c_size_t
             lib.fp8_attention_workspace_bytes.argtypes = [C.c_int] * 6
+        if hasattr(lib, "fp8_linear_step_host_workspace_bytes"):
+            lib.fp8_linear_step_host_workspace_bytes.restype = C.c_size_t
+            lib.fp8_linear_step_host_workspace_bytes.argtypes = [C.c_int] * 3
+            lib.fp8_attention_step_host_workspace_bytes.restype = C.c_size_t
+            lib.fp8_attention_step_host_workspace_bytes.argtypes = [C.c_int] * 5
         _lib = lib
     return _lib
 
@@ -371,3 +378,40 @@ def fp8_attention_bwd_static(q8, k8, v8, do8, o, lse, q_inv, k_inv, v_inv, do_in
     _check(load().fp8_attention_bwd_static(_ptr(q8), _ptr(k8), _ptr(v8), _ptr(do8), _ptr(o), _ptr(lse),
                                            C.byref(sc), C.c_int(int(causal)), C.c_int(B), C.c_int(N), C.c_int(Hq),
                                            C.c_int(Hkv), C.c_int(d), _ptr(dq), _ptr(dk), _ptr(dv), _stream(stream)))
+
+
+def _hptr(t):
+    assert not t.is_cuda and t.is_contiguous(), "expects contiguous HOST tensors"
+    return C.c_void_p(t.data_ptr())
+
+
+def fp8_linear_step_host_workspace_bytes(T, N, K) -> int:
+    return int(load().fp8_linear_step_host_workspace_bytes(T, N, K))
+
+
+def fp8_linear_step_host(hx, hw, hdy, hy, hdx, hdw, ws):
+    """hx [T,K], hw [N,K], hdy [T,N] and the outputs hy, hdx, hdw: BF16 HOST tensors (pinned for overlap); ws: a uint8
+    CUDA tensor of fp8_linear_step_host_workspace_bytes(T, N, K).  Returns once enqueued: see fp8_host_sync."""
+    (T, K), N = hx.shape, hw.shape[0]
+    _check(load().fp8_linear_step_host(_hptr(hx), _hptr(hw), _hptr(hdy), C.c_int(T), C.c_int(N), C.c_int(K), _hptr(hy),
+                                       _hptr(hdx), _hptr(hdw), _ptr(ws), C.c_size_t(ws.numel())))
+
+
+def fp8_attention_step_host_workspace_bytes(B, N, Hq, Hkv, d) -> int:
+    return int(load().fp8_attention_step_host_workspace_bytes(B, N, Hq, Hkv, d))
+
+
+def fp8_attention_step_host(hq, hk, hv, hdo, softmax_scale, ds_scale, causal, ho, hlse, hdq, hdk, hdv, ws):
+    """hq, hdo, ho, hdq [B,N,Hq,d] and hk, hv, hdk, hdv [B,N,Hkv,d]: BF16 HOST tensors; hlse [B,Hq,N] FP32 HOST;
+    softmax_scale and ds_scale host floats; ws: a uint8 CUDA tensor of fp8_attention_step_host_workspace_bytes(...)."""
+    B, N, Hq, d = hq.shape
+    Hkv = hk.shape[2]
+    _check(load().fp8_attention_step_host(_hptr(hq), _hptr(hk), _hptr(hv), _hptr(hdo), C.c_int(B), C.c_int(N), C.c_int(Hq),
+                                          C.c_int(Hkv), C.c_int(d), C.c_float(softmax_scale), C.c_float(ds_scale),
+                                          C.c_int(int(causal)), _hptr(ho), _hptr(hlse), _hptr(hdq), _hptr(hdk), _hptr(hdv),
+                                          _ptr(ws), C.c_size_t(ws.numel())))
+
+
+def fp8_host_sync():
+    """Waits for every host-buffer call made so far on the current device."""
+    _check(load().fp8_host_sync())

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(CSRC, "libfp8dpa.so")
-SOURCES = ["api.cu", "quantize.cu", "elementwise.cu", "gemm_sm100.cu", "gemm_2cta_sm100.cu", "blockwise_sm100.cu", "blockwise_2cta_sm100.cu", "attn_fwd_sm100.cu", "attn_bwd_sm100.cu", "attn_bwd_d128_sm100.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "quantize.cu", "elementwise.cu", "gemm_sm100.cu", "gemm_2cta_sm100.cu", "blockwise_sm100.cu", "blockwise_2cta_sm100.cu", "attn_fwd_sm100.cu", "attn_bwd_sm100.cu", "attn_bwd_d128_sm100.cu", "noalloc.cu", "hoststep.cu"]
 
 
 def sources():

@@ -248,6 +248,31 @@ class BlockHotPath:
             torch.cuda.current_stream(self.device).wait_stream(self._down)
             self._downloaded = None
 
+    def step_host_abi(self, h_in: dict, h_out: dict):
+        """The same step through the host-buffer entry points of the C ABI: one fp8_linear_step_host per projection
+        and one fp8_attention_step_host, each on a device workspace of its own, so that the library overlaps the
+        copies of one group with the kernels of another.  Returns once enqueued; ``fp8.fp8_host_sync()`` before
+        reading h_out.  dS is quantised with the scale this object holds at the first call (a host value)."""
+        if not hasattr(self, "_host_ws"):
+            ws = {}
+            for lin in self.linears:
+                ws[lin.name] = torch.empty(fp8.fp8_linear_step_host_workspace_bytes(lin.T, lin.N, lin.K),
+                                           dtype=torch.uint8, device=self.device)
+            if self.attn is not None:
+                c = self.cfg
+                ws["attn"] = torch.empty(fp8.fp8_attention_step_host_workspace_bytes(
+                    self.B, self.N, c.n_q_heads, c.n_kv_heads, c.head_dim), dtype=torch.uint8, device=self.device)
+                self._host_ds_scale = float(self.attn["ds_scale"].item())
+            self._host_ws = ws
+        for lin in self.linears:
+            n = lin.name
+            fp8.fp8_linear_step_host(h_in["x_" + n], h_in["w_" + n], h_in["dy_" + n], h_out["y_" + n], h_out["dx_" + n],
+                                     h_out["dw_" + n], self._host_ws[n])
+        if self.attn is not None:
+            fp8.fp8_attention_step_host(h_in["q"], h_in["k"], h_in["v"], h_in["do"], self.attn["softmax_scale"],
+                                        self._host_ds_scale, True, h_out["o"], h_out["lse"], h_out["dq"], h_out["dk"],
+                                        h_out["dv"], self._host_ws["attn"])
+
     def _run_linear(self, lin):
         lin.x.quantize()
         lin.w.quantize()

@@ -209,6 +209,34 @@ def test_host_to_host_step_equals_device_step():
         assert torch.equal(hout[n].view(torch.uint8), t.cpu().view(torch.uint8)), n
 
 
+@pytest.mark.parametrize("name", ["c1", "c4"])
+def test_host_buffer_entry_points_equal_device_step(name):
+    """The step through fp8_linear_step_host / fp8_attention_step_host (the form bench.py times end to end), three
+    steps in flight on the same workspaces, returns the bits of step(); dQ at head_dim 128 within its summation-order
+    noise."""
+    cfg = synth.CONFIGS[name]
+    hp = BlockHotPath(cfg, "cuda")
+    h = hp.generate_host_inputs()
+    hp.allocate()
+    hp.calibrate_ds_scale()
+    hp.step()
+    torch.cuda.synchronize()
+    ref = {n: t.cpu() for n, t in hp.output_tensors()}
+    hin = {n: torch.from_numpy(h[n].view("int16")).view(torch.bfloat16).reshape(t.shape).pin_memory()
+           for n, t in hp.input_tensors()}
+    hout = {n: torch.zeros(t.shape, dtype=t.dtype).pin_memory() for n, t in hp.output_tensors()}
+    for _ in range(3):
+        hp.step_host_abi(hin, hout)
+    fp8.fp8_host_sync()
+    assert fp8.fp8_device_status() == 0
+    for n, t in ref.items():
+        if n == "dq" and cfg.head_dim == 128:
+            a, b = hout[n].float(), t.float()
+            assert (a - b).abs().max() <= 2.0 ** -7 * b.abs().max()
+        else:
+            assert torch.equal(hout[n].view(torch.uint8), t.view(torch.uint8)), n
+
+
 def test_delayed_scaling_step_equals_the_just_in_time_step_on_repeated_inputs():
     """With the same inputs every step, the abs-max history holds one value: the delayed-scaling step (one cast pass per
     tensor under the history's scale, Appendix E) must return the bits of the just-in-time step; and when an input grows,
