@@ -867,6 +867,493 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Forward for d = 128, persistent form: one CTA per SM walks a list of (128-query tile, head, batch) items, and the key
+// blocks of all its items form one stream G = 0, 1, 2, ...  Two softmax warpgroups take the blocks of the stream in
+// turn (warpgroup G & 1), one row per thread, so that the exponentials of block G + 1 run while block G is still being
+// finished: with FP8 operands a 128 x 128 tile costs 512 clocks of MMAs against 1024 clocks of the exponential unit, so the
+// softmax chain of a single tile, not the tensor pipe, sets the pace, and two blocks of the same tile in flight hide
+// each other's latencies.  The scores are three blocks ahead: S(G), S(G+1), S(G+2) live in three TMEM buffers, so a
+// warpgroup never waits for the tensor pipe in steady state, also across the boundary between two items.
+//   warps 0-3 / 4-7  softmax warpgroups 0 / 1.  Block G of an item: score row TMEM -> registers, block maximum; the
+//               block maximum of G-1 that the other warpgroup published (shared memory, slot (G-1) & 3, fetched under the
+//               score loads) and this warpgroup's own m(G-2) give m(G-1); publishes its block maximum and the factor
+//               2^(m(G-1) - m(G)) for the accumulator, evaluates the exponentials, stores P8(G) over the first 32 columns
+//               of S(G).  Each warpgroup keeps the row sum of its own blocks with its own reference maximum; the
+//               epilogue merges the two
+//   warps 8-11  correction: rescales O when the running maximum grew (after PV(G-1) has completed), lets PV(G) go;
+//               per item normalises O, merges the row sums, writes O (BF16, tiled bulk stores) and LSE
+//   warp 12     TMA producer: Q (two buffers), K and V (4 stages each)
+//   warp 13     MMA issuer: QK(G+3) right after PV(G) (same TMEM buffer: the tensor pipe runs one thread's products in
+//               issue order, so S(G+3) overwrites P8(G) only after PV(G) has read it)
+// TMEM (512 columns): S buffers 0..2 | O.
+// setmaxnreg only moves registers inside the CTA's own allocation at launch (an increase beyond what the other warpgroups
+// release waits for ever), so the three register counts below must add up to it; the launcher checks the allocation.
+// Every ring (score buffers mod 3, maximum / factor / go / done slots mod 4) is indexed by G, and a slot's next use
+// depends, through PV(G) -> QK(G+3) -> S(G+3), on its previous use having been consumed, so no barrier can complete
+// twice before a waiter has seen it once.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int X_THREADS = 512;
+constexpr int X_KS = 4, X_VS = 4;
+constexpr int X_REGS_LAUNCH = 128;
+static_assert(2 * 128 * P_REGS_SOFTMAX + 128 * P_REGS_CORR + 128 * P_REGS_CTRL <= X_THREADS * X_REGS_LAUNCH, "register budget");
+
+struct AttnFwdStreamSmem {
+    static constexpr int D = 128;
+    static constexpr int TILE_BYTES = 128 * D;
+    static constexpr int Q_OFF = 0;                              // two Q tiles
+    static constexpr int K_OFF = Q_OFF + 2 * TILE_BYTES;
+    static constexpr int V_OFF = K_OFF + X_KS * TILE_BYTES;
+    static constexpr int OST_OFF = V_OFF + X_VS * TILE_BYTES;    // output staging: [128 x 128] BF16 as two 64-column halves
+    static constexpr int ALPHA_OFF = OST_OFF + 2 * TILE_BYTES;   // float[4][128]
+    static constexpr int M_OFF = ALPHA_OFF + 4 * 128 * 4;        // float[4][128]: block maxima (scaled scores), slot G & 3
+    static constexpr int L_OFF = M_OFF + 4 * 128 * 4;            // float[2][128]: row sums of the two warpgroups
+    static constexpr int ML_OFF = L_OFF + 2 * 128 * 4;           // float[2][128]: their reference maxima
+    static constexpr int BAR_OFF = ML_OFF + 2 * 128 * 4;
+    // q_full[2] q_empty[2] k_full[KS] k_empty[KS] v_full[VS] v_empty[VS] s_full[3] pv_go[4] pv_done[4] am_ready[4][4]
+    // l_ready[2][4] epi_done
+    static constexpr int N_BARS = 4 + 2 * X_KS + 2 * X_VS + 3 + 4 + 4 + 16 + 8 + 1;
+    static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
+    static constexpr int DYN_BYTES = TOTAL + 1024;
+};
+
+// The items of one CTA: item k = round * gridDim.x + (CTA index, reversed in odd rounds), heaviest query tiles first.
+struct FwdItems {
+    int round;
+    int q_tile, h, b, n_kv;      // current item
+    __device__ __forceinline__ void init() { round = -1; }
+    __device__ __forceinline__ bool next(const AttnFwdParams &p)
+    {
+        const int n_qt = (p.N + 127) / 128, per_level = p.Hq * p.B;
+        const int n_items = n_qt * per_level;
+        for (;;) {
+            ++round;
+            const long long base = (long long)round * (long long)gridDim.x;
+            if (base >= n_items) return false;
+            const int k = (int)base + ((round & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x);
+            if (k >= n_items) continue;
+            const int level = k / per_level, hb = k - level * per_level;
+            q_tile = n_qt - 1 - level;
+            b = hb / p.Hq;
+            h = hb - b * p.Hq;
+            n_kv = p.causal ? min(n_qt, q_tile + 1) : n_qt;
+            return true;
+        }
+    }
+};
+
+__global__ void __launch_bounds__(X_THREADS, 1)
+attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                       const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                       const AttnFwdParams p)
+{
+    using L = AttnFwdStreamSmem;
+    constexpr int D = 128;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar0 = sbase + L::BAR_OFF;
+    auto q_full = [&](int i) { return bar0 + 8u * i; };
+    auto q_empty = [&](int i) { return bar0 + 8u * (2 + i); };
+    auto k_full = [&](int s) { return bar0 + 8u * (4 + s); };
+    auto k_empty = [&](int s) { return bar0 + 8u * (4 + X_KS + s); };
+    auto v_full = [&](int s) { return bar0 + 8u * (4 + 2 * X_KS + s); };
+    auto v_empty = [&](int s) { return bar0 + 8u * (4 + 2 * X_KS + X_VS + s); };
+    constexpr int B1 = 4 + 2 * X_KS + 2 * X_VS;
+    auto s_full = [&](int s) { return bar0 + 8u * (B1 + s); };
+    auto pv_go = [&](int s) { return bar0 + 8u * (B1 + 3 + s); };
+    auto pv_done = [&](int s) { return bar0 + 8u * (B1 + 7 + s); };
+    auto am_ready = [&](int s, int q) { return bar0 + 8u * (B1 + 11 + s * 4 + q); };
+    auto l_ready = [&](int w, int q) { return bar0 + 8u * (B1 + 27 + w * 4 + q); };
+    const uint32_t epi_done = bar0 + 8u * (B1 + 35);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFF + L::N_BARS * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    float *alpha_s = reinterpret_cast<float *>(smem + L::ALPHA_OFF);
+    float *m_s = reinterpret_cast<float *>(smem + L::M_OFF);
+    float *l_s = reinterpret_cast<float *>(smem + L::L_OFF);
+    float *ml_s = reinterpret_cast<float *>(smem + L::ML_OFF);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(q_full(i), 1);
+            mbar_init(q_empty(i), 1);
+        }
+        for (int s = 0; s < X_KS; ++s) {
+            mbar_init(k_full(s), 1);
+            mbar_init(k_empty(s), 1);
+        }
+        for (int s = 0; s < X_VS; ++s) {
+            mbar_init(v_full(s), 1);
+            mbar_init(v_empty(s), 1);
+        }
+        for (int s = 0; s < 3; ++s) mbar_init(s_full(s), 1);
+        for (int s = 0; s < 4; ++s) {
+            mbar_init(pv_go(s), 8);          // four softmax warps (P8 stored) + four correction warps (O rescaled)
+            mbar_init(pv_done(s), 1);
+            for (int q = 0; q < 4; ++q) mbar_init(am_ready(s, q), 1);
+        }
+        for (int w = 0; w < 2; ++w)
+            for (int q = 0; q < 4; ++q) mbar_init(l_ready(w, q), 1);
+        mbar_init(epi_done, 4);
+        *abort_flag = 0;
+        mbar_init_fence();
+        tma_prefetch_desc(&tm_q);
+        tma_prefetch_desc(&tm_k);
+        tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_o);
+    }
+    if (warp == 13) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_o = tmem_base + 384u;
+    const WaitCtx ctx{p.status, abort_flag};
+    FwdItems it;
+    it.init();
+
+    if (warp >= 12) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(P_REGS_CTRL));
+        if (warp == 12) {
+            // ------------------------------------------------------------ TMA producer
+            if (elect_one()) {
+                uint32_t gk = 0, gv = 0, n_it = 0;
+                bool ok = true;
+                // Q of item t + 1 is requested early in item t (two buffers), so that the first scores of the next item
+                // can be issued before the current item has finished
+                FwdItems nx = it;
+                bool have_next = nx.next(p);
+                auto load_q = [&](const FwdItems &x, uint32_t idx) -> bool {
+                    const int qb = (int)(idx & 1u);
+                    if (!mbar_wait_relaxed(q_empty(qb), ((idx >> 1) & 1u) ^ 1u, ctx)) return false;
+                    mbar_expect_tx(q_full(qb), L::TILE_BYTES);
+                    tma_load_3d(sbase + L::Q_OFF + qb * L::TILE_BYTES, &tm_q, q_full(qb), x.h * D, x.q_tile * 128, x.b);
+                    return true;
+                };
+                if (have_next) ok = load_q(nx, 0);
+                while (ok && it.next(p)) {
+                    have_next = nx.next(p);
+                    const int g = it.h / (p.Hq / p.Hkv);
+                    auto load_k = [&](int j) -> bool {
+                        const uint32_t st = gk % X_KS, ph = (gk / X_KS) & 1u;
+                        if (!mbar_wait_relaxed(k_empty(st), ph ^ 1u, ctx)) return false;
+                        mbar_expect_tx(k_full(st), L::TILE_BYTES);
+                        tma_load_3d(sbase + L::K_OFF + st * L::TILE_BYTES, &tm_k, k_full(st), g * D, j * A_BN, it.b);
+                        ++gk;
+                        return true;
+                    };
+                    auto load_v = [&](int j) -> bool {
+                        const uint32_t st = gv % X_VS, ph = (gv / X_VS) & 1u;
+                        if (!mbar_wait_relaxed(v_empty(st), ph ^ 1u, ctx)) return false;
+                        mbar_expect_tx(v_full(st), L::TILE_BYTES);
+                        tma_load_3d(sbase + L::V_OFF + st * L::TILE_BYTES, &tm_v, v_full(st), g * D, j * A_BN, it.b);
+                        ++gv;
+                        return true;
+                    };
+                    // K runs two blocks ahead of V: the scores are issued three blocks ahead of the PV products
+                    for (int j = 0; j < min(2, it.n_kv) && ok; ++j) ok = load_k(j);
+                    for (int j = 0; j < it.n_kv && ok; ++j) {
+                        ok = load_v(j);
+                        if (ok && j + 2 < it.n_kv) ok = load_k(j + 2);
+                        if (ok && j == 0 && have_next) ok = load_q(nx, n_it + 1u);
+                    }
+                    ++n_it;
+                }
+            }
+        } else if (warp == 13) {
+            // ------------------------------------------------------------ MMA issuer
+            if (elect_one()) {
+                constexpr uint32_t idesc_s = umma_idesc_f8(0, 0, 128, A_BN, 0, 0);
+                constexpr uint32_t idesc_o = umma_idesc_f8(0, 0, 128, D, 0, 1);       // V is MN-major
+                // two cursors over the same item list: the next QK to issue and the next PV
+                FwdItems qi = it;
+                uint32_t gq = 0, gkq = 0;      // stream index and K count of the next QK
+                int jq = 0;                    // its block within item qi
+                uint32_t nq_it = 0;            // items begun by the QK cursor
+                bool q_valid = qi.next(p), ok = true;
+                auto issue_next_qk = [&]() -> bool {
+                    const int qb = (int)(nq_it & 1u);
+                    if (jq == 0 && !mbar_wait(q_full(qb), (nq_it >> 1) & 1u, ctx)) return false;
+                    const uint32_t st = gkq % X_KS;
+                    if (!mbar_wait(k_full(st), (gkq / X_KS) & 1u, ctx)) return false;
+                    tc_fence_after();
+                    const uint64_t dq = umma_desc(sbase + L::Q_OFF + qb * L::TILE_BYTES, D, 16);
+                    const uint64_t dk = umma_desc(sbase + L::K_OFF + st * L::TILE_BYTES, D, 16);
+                    const uint32_t ts = tmem_base + (gq % 3u) * 128u;
+#pragma unroll
+                    for (int k = 0; k < D / 32; ++k) umma_f8_ss(ts, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
+                    umma_commit(s_full((int)(gq % 3u)));
+                    umma_commit(k_empty((int)st));
+                    ++gq;
+                    ++gkq;
+                    if (++jq == qi.n_kv) {
+                        umma_commit(q_empty(qb));          // the item's last QK has read Q
+                        jq = 0;
+                        ++nq_it;
+                        q_valid = qi.next(p);
+                    }
+                    return true;
+                };
+                for (int i = 0; i < 3 && ok && q_valid; ++i) ok = issue_next_qk();
+                uint32_t gp = 0, gvp = 0, np_it = 0;
+                while (ok && it.next(p)) {
+                    for (int j = 0; j < it.n_kv && ok; ++j, ++gp, ++gvp) {
+                        const uint32_t st = gvp % X_VS;
+                        if (!mbar_wait(v_full(st), (gvp / X_VS) & 1u, ctx)) { ok = false; break; }
+                        // the epilogue of the previous item has read O
+                        if (j == 0 && np_it > 0 && !mbar_wait(epi_done, (np_it - 1u) & 1u, ctx)) { ok = false; break; }
+                        if (!mbar_wait(pv_go((int)(gp & 3u)), (gp >> 2) & 1u, ctx)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t dv = umma_desc(sbase + L::V_OFF + st * L::TILE_BYTES, D, 16);
+                        const uint32_t ts = tmem_base + (gp % 3u) * 128u;
+#pragma unroll
+                        for (int k = 0; k < A_BN / 32; ++k)
+                            umma_f8_ts(tmem_o, ts + 8u * k, dv + (uint32_t)((32 * D) >> 4) * k, idesc_o, (j | k) != 0);
+                        umma_commit(pv_done((int)(gp & 3u)));
+                        umma_commit(v_empty((int)st));
+                        if (q_valid) ok = issue_next_qk();
+                    }
+                    ++np_it;
+                }
+            }
+        }
+    }
+    else if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(P_REGS_SOFTMAX));
+        // ------------------------------------------------------------ softmax warpgroup w: blocks G with (G & 1) == w
+        const int w = warp >> 2, quad = warp & 3;
+        const int r = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const float c = p.softmax_scale * __ldg(p.q_inv) * __ldg(p.k_inv) * 1.4426950408889634f;
+        uint32_t gbase = 0, n_it = 0;
+        bool ok = true;
+        while (ok && it.next(p)) {
+            const int qs = it.q_tile * 128;
+            const int row = qs + r;
+            const int n_kv = it.n_kv;
+            float m_own = -INFINITY, l = 0.0f;     // reference maximum and row sum of this warpgroup's blocks
+            // one key block; MASK: columns past `limit` (the causal diagonal, the end of the sequence) count as -inf
+            auto block = [&](auto masked, const int j) -> bool {
+                constexpr bool MASK = decltype(masked)::value;
+                const uint32_t G = gbase + (uint32_t)j;
+                const int limit = min(p.causal ? row : 0x7FFFFFFF, p.N - 1) - j * A_BN;   // last valid local column
+                const uint32_t sb = G % 3u;
+                if (!mbar_wait_warp(s_full((int)sb), (G / 3u) & 1u, ctx)) return false;
+                tc_fence_after();
+                const uint32_t tmem_s = tmem_base + sb * 128u + lane_addr;
+                uint32_t sv[4][32];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x32(tmem_s + (uint32_t)(q * 32), sv[q]);
+                // under the loads: the running maximum up to the previous block of this item, from this warpgroup's own
+                // m(G-2) and the block maximum the other warpgroup published for G-1
+                float m_prev = m_own;
+                if (j > 0) {
+                    const uint32_t Gp = G - 1u;
+                    if (!mbar_wait_warp(am_ready((int)(Gp & 3u), quad), (Gp >> 2) & 1u, ctx)) return false;
+                    const float mb = m_s[(Gp & 3u) * 128u + r];
+                    m_prev = (mb > m_own + p.max_slack) ? mb : m_own;
+                }
+                tmem_ld_wait();
+                float mq[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    mq[q] = -INFINITY;
+                    if (MASK) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (q * 32 + e <= limit) mq[q] = fmaxf(mq[q], __uint_as_float(sv[q][e]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2)
+                            mq[q] = fmax3(mq[q], __uint_as_float(sv[q][e]), __uint_as_float(sv[q][e + 1]));
+                    }
+                }
+                const float m_blk = fmaxf(fmaxf(mq[0], mq[1]), fmaxf(mq[2], mq[3])) * c;
+                const bool grew = m_blk > m_prev + p.max_slack;
+                const float m_new = grew ? m_blk : m_prev;
+                // for the other warpgroup (this block's maximum) and the correction warps (the factor for the accumulator)
+                alpha_s[(G & 3u) * 128u + r] = grew ? ex2_approx(m_prev - m_new) : 1.0f;      // first block: 0
+                m_s[(G & 3u) * 128u + r] = m_blk;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(am_ready((int)(G & 3u), quad));
+                const float neg_shift = p.log2_p_scale - m_new;
+                float lsum = 0.0f;
+                uint32_t pw[32];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t wq[8];
+                    lsum += softmax_chunk<MASK, P_POLY>(sv[q], c, neg_shift, limit - q * 32, wq);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) pw[q * 8 + e] = wq[e];
+                }
+                // P8 over the first 32 score columns of this buffer (this thread's own row, already in registers)
+                tmem_st_32x32b_x32(tmem_s, pw);
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pv_go((int)(G & 3u)));
+                l = l * ((m_own == m_new) ? 1.0f : ex2_approx(m_own - m_new)) + lsum;
+                m_own = m_new;
+                return true;
+            };
+            const int k_last = (n_kv - 1) * A_BN;
+            const bool last_masked = (k_last + A_BN - 1 > qs && p.causal) || (k_last + A_BN > p.N);
+            for (int j = (int)((gbase ^ (uint32_t)w) & 1u); j < n_kv && ok; j += 2) {
+                if (j == n_kv - 1 && last_masked) ok = block(std::true_type{}, j);
+                else ok = block(std::false_type{}, j);
+            }
+            if (!ok) break;
+            // the epilogue of the previous item has read the row sums
+            if (n_it > 0 && !mbar_wait_warp(epi_done, (n_it - 1u) & 1u, ctx)) break;
+            l_s[w * 128 + r] = l;
+            ml_s[w * 128 + r] = m_own;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(l_ready(w, quad));
+            gbase += (uint32_t)n_kv;
+            ++n_it;
+        }
+    } else if (warp < 12) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(P_REGS_CORR));
+        // ------------------------------------------------------------ correction and epilogue
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        const uint32_t to = tmem_o + lane_addr;
+        uint32_t gbase = 0, n_it = 0;
+        bool ok = true, stored = false;
+        while (ok && it.next(p)) {
+            const int n_kv = it.n_kv;
+            for (int j = 0; j < n_kv && ok; ++j) {
+                const uint32_t G = gbase + (uint32_t)j;
+                if (!mbar_wait_warp(am_ready((int)(G & 3u), quad), (G >> 2) & 1u, ctx)) { ok = false; break; }
+                if (j > 0) {
+                    const float a = alpha_s[(G & 3u) * 128u + r];
+                    if (__any_sync(0xffffffffu, a != 1.0f)) {
+                        // O is at rest once PV(G-1) has completed
+                        const uint32_t Gp = G - 1u;
+                        if (!mbar_wait_warp(pv_done((int)(Gp & 3u)), (Gp >> 2) & 1u, ctx)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t a2 = pack_f32x2(a, a);
+#pragma unroll 1
+                        for (int cc = 0; cc < D; cc += 32) {
+                            uint32_t v[32];
+                            tmem_ld_32x32b_x32(to + (uint32_t)cc, v);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int e = 0; e < 32; e += 2) {
+                                float x, y;
+                                unpack_f32x2(mul_f32x2(pack_f32x2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), a2), x, y);
+                                v[e] = __float_as_uint(x);
+                                v[e + 1] = __float_as_uint(y);
+                            }
+                            tmem_st_32x32b_x32(to + (uint32_t)cc, v);
+                        }
+                        tmem_st_wait();
+                        tc_fence_before();
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pv_go((int)(G & 3u)));
+            }
+            if (!ok) break;
+            // ---- epilogue of the item: merge the two row sums, normalise, store
+            const uint32_t Gl = gbase + (uint32_t)n_kv - 1u;
+            if (!mbar_wait_warp(l_ready(0, quad), n_it & 1u, ctx) || !mbar_wait_warp(l_ready(1, quad), n_it & 1u, ctx) ||
+                !mbar_wait_warp(pv_done((int)(Gl & 3u)), (Gl >> 2) & 1u, ctx)) {
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            const int row = it.q_tile * 128 + r;
+            const float m0 = ml_s[r], m1 = ml_s[128 + r];
+            const float mf = fmaxf(m0, m1);
+            const float lt = l_s[r] * (m0 == mf ? 1.0f : ex2_approx(m0 - mf)) +
+                             l_s[128 + r] * (m1 == mf ? 1.0f : ex2_approx(m1 - mf));
+            const float inv = __ldg(p.v_inv) / lt;                 // lt already carries c_P
+            if (row < p.N)
+                p.LSE[((size_t)it.b * p.Hq + it.h) * p.N + row] = (mf + log2f(lt) - p.log2_p_scale) * 0.69314718055994531f;
+            uint8_t *o8row = p.O8 + (((size_t)it.b * p.N + row) * p.Hq + it.h) * D;
+            const float o_scale = p.o_scale ? __ldg(p.o_scale) : 1.0f;
+            // the previous item's stores have read this warp's rows of the staging tile
+            if (stored) {
+                if (lane == 0) bulk_wait_group_read0();
+                __syncwarp();
+            }
+            uint32_t amax2 = 0;
+#pragma unroll 1
+            for (int cc = 0; cc < D; cc += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32b_x32(to + (uint32_t)cc, v);
+                tmem_ld_wait();
+                if (cc == D - 32) {
+                    // O and the row sums have been read: the next item may overwrite them
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(epi_done);
+                }
+                // staging tile of 64 columns: [128 rows x 128 bytes], 128-byte swizzle
+                uint8_t *trow = smem + L::OST_OFF + (cc < 64 ? 0 : L::TILE_BYTES) + r * 128;
+                const int c0 = (cc & 63) >> 3;
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    uint4 o;
+                    o.x = pack_bf16x2(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv);
+                    o.y = pack_bf16x2(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
+                    o.z = pack_bf16x2(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
+                    o.w = pack_bf16x2(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(trow + (((c0 + (e >> 3)) ^ (r & 7)) << 4)) = o;
+                    if (p.o_scale && row < p.N) {
+                        amax2 = __vmaxu2(__vmaxu2(__vmaxu2(__vmaxu2(amax2, o.x & 0x7FFF7FFFu), o.y & 0x7FFF7FFFu),
+                                                  o.z & 0x7FFF7FFFu), o.w & 0x7FFF7FFFu);
+                        const uint32_t e0 = cvt_f32x4_to_fp8x4<0>(
+                            __fmul_rn(bf16_lo(o.x), o_scale), __fmul_rn(bf16_hi(o.x), o_scale),
+                            __fmul_rn(bf16_lo(o.y), o_scale), __fmul_rn(bf16_hi(o.y), o_scale));
+                        const uint32_t e1 = cvt_f32x4_to_fp8x4<0>(
+                            __fmul_rn(bf16_lo(o.z), o_scale), __fmul_rn(bf16_hi(o.z), o_scale),
+                            __fmul_rn(bf16_lo(o.w), o_scale), __fmul_rn(bf16_hi(o.w), o_scale));
+                        *reinterpret_cast<uint2 *>(o8row + cc + e) = make_uint2(e0, e1);
+                    }
+                }
+            }
+            if (p.o_scale && p.o_amax_bits) {
+                uint32_t mm = row < p.N ? max(amax2 & 0xFFFFu, amax2 >> 16) : 0u;
+                mm = __reduce_max_sync(0xffffffffu, mm);
+                if (lane == 0 && mm != 0u) atomicMax(p.o_amax_bits, mm << 16);
+            }
+            // every warp stores its own 32 rows (the output map's box is 32 rows x 64 columns)
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_3d(&tm_o, sbase + L::OST_OFF + quad * 4096, (it.h * D) * 2, it.q_tile * 128 + quad * 32, it.b);
+                tma_store_3d(&tm_o, sbase + L::OST_OFF + L::TILE_BYTES + quad * 4096, (it.h * D + 64) * 2,
+                             it.q_tile * 128 + quad * 32, it.b);
+                bulk_commit_group();
+            }
+            stored = true;
+            gbase += (uint32_t)n_kv;
+            ++n_it;
+        }
+        if (stored && lane == 0) bulk_wait_group_read0();               // shared memory is read before the CTA may exit
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(20000);
+        __syncthreads();
+    }
+    if (warp == 13) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
 int validate_attn(const char *who, const void *q, const void *k, const void *v, const fp8_attn_scales *sc, int B, int N,
                   int Hq, int Hkv, int d)
 {
@@ -934,15 +1421,44 @@ static int launch_attn_fwd_pair(const uint8_t *Q8, const uint8_t *K8, const uint
     return FP8_OK;
 }
 
-// FP8DPA_ATTN_FWD=single forces the one-tile-per-CTA kernel at d = 128 (for A/B measurements)
-static bool attn_fwd_use_pair()
+static int launch_attn_fwd_stream(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const AttnFwdParams &p,
+                                  cudaStream_t st)
 {
-    static int v = -1;
-    if (v < 0) {
-        const char *e = getenv("FP8DPA_ATTN_FWD");
-        v = (e && strcmp(e, "single") == 0) ? 0 : 1;
+    constexpr int D = 128;
+    CUtensorMap tq, tk, tv, to;
+    int rc = make_tmap_3d_u8(&tq, Q8, (uint64_t)p.Hq * D, (uint64_t)p.N, (uint64_t)p.B, D, 128);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tk, K8, (uint64_t)p.Hkv * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BN);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&tv, V8, (uint64_t)p.Hkv * D, (uint64_t)p.N, (uint64_t)p.B, D, A_BN);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_3d_u8(&to, p.O, (uint64_t)p.Hq * D * 2, (uint64_t)p.N, (uint64_t)p.B, 128, 32);
+    if (rc != FP8_OK) return rc;
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        AttnFwdStreamSmem::DYN_BYTES));
+    // the kernel's register hand-over between its warpgroups is balanced for this allocation at launch
+    cudaFuncAttributes fa;
+    FP8_CUDA_CHECK(cudaFuncGetAttributes(&fa, attn_fwd_stream_kernel));
+    if (fa.numRegs != X_REGS_LAUNCH) {
+        set_error("attn_fwd_stream_kernel: built with %d registers per thread, expected %d", fa.numRegs, X_REGS_LAUNCH);
+        return FP8_ERR_CUDA;
     }
-    return v != 0;
+    const long long n_items = (long long)((p.N + 127) / 128) * p.Hq * p.B;
+    const int sms = sm_count();
+    if (sms <= 0) return FP8_ERR_CUDA;
+    dim3 grid((unsigned)(n_items < sms ? n_items : sms));
+    attn_fwd_stream_kernel<<<grid, X_THREADS, AttnFwdStreamSmem::DYN_BYTES, st>>>(tq, tk, tv, to, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+// The d = 128 kernel: the persistent one ("stream": two softmax warpgroups on alternating key blocks) unless
+// FP8DPA_ATTN_FWD names another for A/B measurements: "single" = one 128-row tile per CTA, two CTAs per SM; "pair" = two
+// tiles per CTA
+static int attn_fwd_choice()
+{
+    const char *e = getenv("FP8DPA_ATTN_FWD");      // read per call: tests switch it
+    return (e && strcmp(e, "single") == 0) ? 0 : (e && strcmp(e, "pair") == 0) ? 1 : 2;
 }
 
 }  // namespace fp8dpa
@@ -987,7 +1503,11 @@ static int attention_fwd_common(const char *who, const uint8_t *Q8, const uint8_
     p.o_amax_bits = reinterpret_cast<unsigned int *>(o_amax);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (o_scale && o_amax) FP8_CUDA_CHECK(cudaMemsetAsync(o_amax, 0, sizeof(float), st));
-    if (d == 128) return attn_fwd_use_pair() ? launch_attn_fwd_pair(Q8, K8, V8, p, st) : launch_attn_fwd<128>(Q8, K8, V8, p, st);
+    if (d == 128) {
+        const int ch = attn_fwd_choice();
+        return ch == 2 ? launch_attn_fwd_stream(Q8, K8, V8, p, st)
+                       : ch == 1 ? launch_attn_fwd_pair(Q8, K8, V8, p, st) : launch_attn_fwd<128>(Q8, K8, V8, p, st);
+    }
     return launch_attn_fwd<64>(Q8, K8, V8, p, st);
 }
 

@@ -73,6 +73,30 @@ def test_forward_matches_oracle(name, B, N, causal):
            oracle_whole_row_vs_blocked_fro=norm_ratios(ref0, ref)[0])
 
 
+@pytest.mark.parametrize("family", ["single", "pair", "stream"])
+@pytest.mark.parametrize("name,B,N,causal", [("c3", 1, 656, True), ("c4", 2, 400, True), ("c4", 1, 272, False),
+                                             ("c3", 3, 128, True)])
+def test_forward_kernel_families_at_head_dim_128(family, name, B, N, causal, monkeypatch):
+    """FP8DPA_ATTN_FWD picks the d = 128 kernel: one tile per CTA, two tiles per CTA, or the persistent kernel whose CTAs
+    walk several (tile, head, batch) items with two softmax warpgroups on alternating key blocks (the default).  All
+    three must agree with the oracle; the shapes give CTAs of the persistent kernel items of different lengths, odd and
+    even block counts (the warpgroups swap roles from item to item), a ragged last tile and grouped heads."""
+    monkeypatch.setenv("FP8DPA_ATTN_FWD", family)
+    cfg = synth.CONFIGS[name]
+    Hq, Hkv, d = cfg.n_q_heads // 4, cfg.n_kv_heads // 4, cfg.head_dim
+    cfg = synth.BlockConfig(**{**cfg.__dict__, "n_q_heads": Hq, "n_kv_heads": Hkv})
+    qd = quantized_qkv(cfg, N, B)
+    s = d ** -0.5
+    O, LSE = run_fwd(qd, B, N, Hq, Hkv, d, causal, s)
+    p = o.attn_params(B, N, Hq, Hkv, d, causal=causal, quant=True, kv_block=KV_BLOCK, max_mode=0, s=s,
+                      q_inv=qd["q"][1], k_inv=qd["k"][1], v_inv=qd["v"][1], flip_eps=FLIP_EPS)
+    ref, lse, mag, slack = o.attention_fwd(qd["q"][0], qd["k"][0], qd["v"][0], p, with_slack=True)
+    got = O.float().cpu().numpy().astype(np.float64).transpose(0, 2, 1, 3).reshape(B * Hq, N, d)
+    assert rel_err(got, ref, mag, slack) <= TOL_FWD
+    glse = LSE.cpu().numpy().astype(np.float64).reshape(B * Hq, N)
+    assert np.max(np.abs(glse - lse)) <= 1e-3 * max(1.0, np.abs(lse).max())
+
+
 @pytest.mark.parametrize("name,B,N,causal,tau", [("c1", 1, 400, True, 3.0), ("c3", 1, 384, True, 3.0),
                                                  ("c4", 1, 272, True, 2.0), ("c4", 1, 256, False, 3.0)])
 def test_forward_with_reference_maximum_slack_matches_oracle(name, B, N, causal, tau):
