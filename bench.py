@@ -778,7 +778,10 @@ def run_report(args):
     offs_host = [int(v) for v in offs.cpu().tolist()]
     add("fp8_grouped_linear_wgrad (8 experts, uneven, one launch per expert)", f"{Tr} rows x {Ng} x {Kg}",
         timed(lambda: fp8.fp8_grouped_linear_wgrad(dy8, x8, s1, s1, offs_host, dwb)), flops=2.0 * Tr * Ng * Kg)
-    del x8, w8, yb, dy8, dxb, dwb
+    wsg = torch.empty(fp8.fp8_grouped_linear_wgrad_workspace_bytes(E, Ng), dtype=torch.uint8, device="cuda")
+    add("fp8_grouped_linear_wgrad_dev (8 experts, uneven, one launch, device offsets)", f"{Tr} rows x {Ng} x {Kg}",
+        timed(lambda: fp8.fp8_grouped_linear_wgrad_dev(dy8, x8, s1, s1, offs, dwb, wsg)), flops=2.0 * Tr * Ng * Kg)
+    del x8, w8, yb, dy8, dxb, dwb, wsg
 
     # ---- attention of c3, c4, c5 (causal)
     for cname in ("c3", "c4", "c5"):

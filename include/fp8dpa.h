@@ -227,6 +227,18 @@ FP8_API int fp8_grouped_linear_wgrad(const uint8_t *dY8, const uint8_t *X8, cons
                              const int *group_offsets_host, int n_groups, void *dW, int out_is_fp32, int accumulate,
                              int T, int N, int K, void *stream);
 
+/* The same weight gradients in one launch with the offsets on the DEVICE (group_offsets as in fp8_grouped_linear_fwd:
+ * n_groups + 1 ascending int32 entries, clamped to [0, T] by the kernel), so that the router's output never has to reach
+ * the host.  ws: device scratch of fp8_grouped_linear_wgrad_workspace_bytes(n_groups, N) = n_groups * 128 * N bytes,
+ * 16-byte aligned, overwritten (it receives a zero-padded copy of the last, possibly ragged block of 128 rows of dY8 of
+ * every expert; all other blocks are read in place).  Same arithmetic, outputs, `accumulate` and empty-group behaviour as
+ * fp8_grouped_linear_wgrad (an empty group gives zeros, or leaves dW[g] unchanged in value with `accumulate`).
+ * Errors: FP8_ERR_NULL, FP8_ERR_SHAPE, FP8_ERR_ALIGN, FP8_ERR_WORKSPACE before anything is launched. */
+FP8_API size_t fp8_grouped_linear_wgrad_workspace_bytes(int n_groups, int N);
+FP8_API int fp8_grouped_linear_wgrad_dev(const uint8_t *dY8, const uint8_t *X8, const float *sdY_inv, const float *sX_inv,
+                                 const int *group_offsets, int n_groups, void *dW, int out_is_fp32, int accumulate,
+                                 int T, int N, int K, void *ws, size_t ws_bytes, void *stream);
+
 /* Producer forms for delayed scaling (Appendix E: rho comes from the amax history, so the producer of a tensor can
  * emit FP8 in its own epilogue, "a single pass on the data", Section 2).  Same products as fp8_linear_fwd /
  * fp8_linear_dgrad; the result is rounded to BF16 (the tensor an unfused chain would store), its amax is written to

@@ -9,7 +9,7 @@ from . import binding  # noqa: F401
 from .binding import (ACT_GELU, ACT_XIELU, E4M3, E5M2, FP8_BLOCK_128x1, NORM_LAYERSCALE, NORM_RMS, QK_NONE, QK_RMS, QK_TANH,  # noqa: F401
                       Fp8Error, fp8_act_cast, fp8_amax, fp8_attention_bwd, fp8_attention_bwd_static,
                       fp8_attention_fwd, fp8_attention_fwd_q, fp8_attention_workspace_bytes, fp8_cast,
-                      fp8_device_status, fp8_grouped_linear_dgrad, fp8_grouped_linear_fwd, fp8_grouped_linear_wgrad, fp8_kurtosis, fp8_amax_kurtosis, fp8_last_error, fp8_linear_dgrad,
+                      fp8_device_status, fp8_grouped_linear_dgrad, fp8_grouped_linear_fwd, fp8_grouped_linear_wgrad, fp8_grouped_linear_wgrad_dev, fp8_grouped_linear_wgrad_workspace_bytes, fp8_kurtosis, fp8_amax_kurtosis, fp8_last_error, fp8_linear_dgrad,
                       fp8_linear_dgrad_q, fp8_linear_dgrad_rm, fp8_linear_fwd, fp8_linear_fwd_blockwise,
                       fp8_linear_dgrad_blockwise, fp8_linear_wgrad_blockwise,
                       fp8_linear_fwd_q, fp8_linear_wgrad, fp8_linear_wgrad_rm, fp8_postnorm_residual, fp8_postnorm_residual_q,

@@ -22,7 +22,7 @@ _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
            "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis", "fp8_amax_kurtosis",
-           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_linear_dgrad_blockwise", "fp8_linear_wgrad_blockwise", "fp8_attention_workspace_bytes",
+           "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_grouped_linear_wgrad_workspace_bytes", "fp8_grouped_linear_wgrad_dev", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_linear_dgrad_blockwise", "fp8_linear_wgrad_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static",
            "fp8_linear_step_host_workspace_bytes", "fp8_linear_step_host", "fp8_attention_step_host_workspace_bytes",
            "fp8_attention_step_host", "fp8_host_sync"]
@@ -56,6 +56,9 @@ def load() -> C.CDLL:
         if hasattr(lib, "fp8_attention_workspace_bytes"):
             lib.fp8_attention_workspace_bytes.restype = C.c_size_t
             lib.fp8_attention_workspace_bytes.argtypes = [C.c_int] * 6
+        if hasattr(lib, "fp8_grouped_linear_wgrad_workspace_bytes"):
+            lib.fp8_grouped_linear_wgrad_workspace_bytes.restype = C.c_size_t
+            lib.fp8_grouped_linear_wgrad_workspace_bytes.argtypes = [C.c_int] * 2
         if hasattr(lib, "fp8_linear_step_host_workspace_bytes"):
             lib.fp8_linear_step_host_workspace_bytes.restype = C.c_size_t
             lib.fp8_linear_step_host_workspace_bytes.argtypes = [C.c_int] * 3
@@ -273,6 +276,22 @@ def fp8_grouped_linear_wgrad(dy8, x8, sdy_inv, sx_inv, group_offsets_host, dw, a
     _check(load().fp8_grouped_linear_wgrad(_ptr(dy8), _ptr(x8), _ptr(sdy_inv), _ptr(sx_inv), arr, C.c_int(E), _ptr(dw),
                                            C.c_int(_is_fp32(dw)), C.c_int(int(accumulate)), C.c_int(T), C.c_int(N),
                                            C.c_int(K), _stream(stream)))
+
+
+def fp8_grouped_linear_wgrad_workspace_bytes(n_groups, N) -> int:
+    return int(load().fp8_grouped_linear_wgrad_workspace_bytes(n_groups, N))
+
+
+def fp8_grouped_linear_wgrad_dev(dy8, x8, sdy_inv, sx_inv, group_offsets, dw, ws, accumulate=False, stream=None):
+    """The same weight gradients in one launch; group_offsets is an int32 CUDA tensor (E + 1 entries), ws a uint8 CUDA tensor
+    of fp8_grouped_linear_wgrad_workspace_bytes(E, N)."""
+    T, N = dy8.shape
+    K = x8.shape[1]
+    E = group_offsets.numel() - 1
+    _check(load().fp8_grouped_linear_wgrad_dev(_ptr(dy8), _ptr(x8), _ptr(sdy_inv), _ptr(sx_inv), _ptr(group_offsets),
+                                               C.c_int(E), _ptr(dw), C.c_int(_is_fp32(dw)), C.c_int(int(accumulate)),
+                                               C.c_int(T), C.c_int(N), C.c_int(K), _ptr(ws), C.c_size_t(ws.numel()),
+                                               _stream(stream)))
 
 
 def fp8_quantize_blockwise(x, block_rows, fmt, out, scale_inv, stream=None):

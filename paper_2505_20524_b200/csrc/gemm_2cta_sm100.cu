@@ -80,12 +80,21 @@ __device__ __forceinline__ GroupTile group_tile(const int *tile_start, const int
     return t;
 }
 
-template <bool GROUPED>
+// MODE 0: one product.  MODE 1: grouped along the rows (forward / data gradient of the mixture-of-experts FFN).
+// MODE 2: grouped along the reduction (its weight gradients): group g reduces over the rows [offs[g], offs[g+1]) of both
+// operands (read in place, MN-major) into its own [M, N] output.  Every block of 128 reduction rows but a group's last comes
+// from the operands themselves; the last one, which may be ragged, takes its A tile from a zero-padded copy of those rows
+// (tmap_a_tail: [n_groups * 128, M], written by grouped_tail_kernel), so whatever rows of the next group the B tile
+// carries meet zeros.  A group without rows reduces over one all-zero block.
+template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
-gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const Params p)
+gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                     const __grid_constant__ CUtensorMap tmap_a_tail, const Params p)
 {
+    constexpr bool GROUPED = MODE == 1;
+    constexpr bool GRED = MODE == 2;
     __shared__ int g_tile_start[GROUPED ? MAX_GROUPS + 1 : 1];
-    __shared__ int g_offs[GROUPED ? MAX_GROUPS + 1 : 1];
+    __shared__ int g_offs[MODE != 0 ? MAX_GROUPS + 1 : 1];
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
@@ -103,6 +112,19 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
     const int tiles_m = (p.M + 2 * BM - 1) / (2 * BM), tiles_n = (p.N + BN - 1) / BN;
     int num_tiles = tiles_m * tiles_n;
     const int k_blocks = (p.K + BK - 1) / BK;
+    if (GRED) {
+        // the same clamping of the device-side offsets as below; the tiles do not depend on them
+        if (threadIdx.x == 0) {
+            int prev = min(max(__ldg(p.group_offsets), 0), p.K);
+            for (int g = 0; g < p.n_groups; ++g) {
+                g_offs[g] = prev;
+                prev = min(max(__ldg(p.group_offsets + g + 1), prev), p.K);
+            }
+            g_offs[p.n_groups] = prev;
+        }
+        __syncthreads();
+        num_tiles *= p.n_groups;
+    }
     if (GROUPED) {
         // every CTA builds the same tile table from the device-side offsets
         if (threadIdx.x == 0) {
@@ -158,8 +180,15 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
             const uint64_t pol_last = l2_policy_evict_last(), pol_first = l2_policy_evict_first();
             const uint64_t pol_a = p.hint_a == 1 ? pol_last : pol_first, pol_b = p.hint_b == 1 ? pol_last : pol_first;
             for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs) {
-                int tm, tn, m_base = 0, n_base = 0, kb_base_b = 0;
-                if (GROUPED) {
+                int tm, tn, m_base = 0, n_base = 0, kb_base_b = 0, kbs = k_blocks, red0 = 0, g_red = 0;
+                if (GRED) {
+                    const int per = tiles_m * tiles_n, local = tile % per;
+                    g_red = tile / per;
+                    tn = local / tiles_m;
+                    tm = local - tn * tiles_m;
+                    red0 = g_offs[g_red];
+                    kbs = max(1, (g_offs[g_red + 1] - red0 + BK - 1) / BK);
+                } else if (GROUPED) {
                     const GroupTile gt = group_tile(g_tile_start, g_offs, p.n_groups, tiles_n, tile);
                     tm = gt.tm; tn = gt.tn;
                     m_base = gt.row0;              // rows of A: the group's slice of the sorted token matrix
@@ -171,10 +200,18 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                     tile_coords(p, tile, tiles_m, tiles_n, tm, tn);
                 }
                 const int m0 = m_base + tm * 2 * BM + (int)rank * BM, n0 = n_base + tn * BN + (int)rank * (BN / 2);
-                for (int kb = 0; kb < k_blocks; ++kb) {
+                for (int kb = 0; kb < kbs; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, ctx)) { ok = false; break; }
                     const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
                     if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+                    if (GRED) {
+                        // both operands MN-major: [reduction rows, output index]
+                        if (kb == kbs - 1) tma_load_2d_pair(sa, &tmap_a_tail, full_bar(stage), m0, g_red * BK);
+                        else tma_load_2d_pair(sa, &tmap_a, full_bar(stage), m0, red0 + kb * BK);
+                        tma_load_2d_pair(sb, &tmap_b, full_bar(stage), n0, red0 + kb * BK);
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     // K-major tile: 128 rows of the output index x 128 reduction bytes; MN-major tile: 128 reduction
                     // rows x 128 bytes of the output index (the matrix as it lies in memory, no transposed copy)
                     const int a0 = p.a_mn ? m0 : kb * BK, a1 = p.a_mn ? kb * BK : m0;
@@ -200,7 +237,12 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                 if (!mbar_wait(tempty_bar(buf), acc_phase ^ 1u, ctx)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < k_blocks; ++kb) {
+                int kbs = k_blocks;
+                if (GRED) {
+                    const int g = tile / (tiles_m * tiles_n);
+                    kbs = max(1, (g_offs[g + 1] - g_offs[g] + BK - 1) / BK);
+                }
+                for (int kb = 0; kb < kbs; ++kb) {
                     if (!mbar_wait(full_bar(stage), phase, ctx)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = sbase + stage * STAGE_BYTES, sb = sa + A_BYTES;
@@ -229,9 +271,14 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
         for (int tile = pair; tile < num_tiles && ok; tile += p.num_pairs, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            int tm, tn, m_base = 0, m_end = p.M;
+            int tm, tn, m_base = 0, m_end = p.M, row_shift = 0;
             float descale_t = descale;
-            if (GROUPED) {
+            if (GRED) {
+                const int per = tiles_m * tiles_n, local = tile % per;
+                tn = local / tiles_m;
+                tm = local - tn * tiles_m;
+                row_shift = (tile / per) * p.M;            // the group's [M, N] output follows the previous group's
+            } else if (GROUPED) {
                 const GroupTile gt = group_tile(g_tile_start, g_offs, p.n_groups, tiles_n, tile);
                 tm = gt.tm; tn = gt.tn;
                 m_base = gt.row0;
@@ -252,7 +299,7 @@ gemm_fp8_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_co
                 tmem_ld_wait();
                 const int col = n0 + c;
                 if (row < m_end && col < p.N)
-                    gemm_store_chunk(r, descale_t, p.o, q_scale, p.N, row, col, min(32, p.N - col), amax2);
+                    gemm_store_chunk(r, descale_t, p.o, q_scale, p.N, row_shift + row, col, min(32, p.N - col), amax2);
             }
             tc_fence_before();
             __syncwarp();
@@ -338,7 +385,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     rc = b_mn ? make_tmap_2d_u8(&tb, b, (uint64_t)K, (uint64_t)N, (uint64_t)N, BK, BN / 2)
               : make_tmap_2d_u8(&tb, b, (uint64_t)N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
     if (rc != FP8_OK) return rc;
-    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
     static int max_clusters = -1;
     if (max_clusters < 0) {
         cudaLaunchConfig_t cfg = {};
@@ -351,7 +398,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, gemm_fp8_pair_kernel<false>, &cfg) != cudaSuccess || n <= 0) {
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_fp8_pair_kernel<0>, &cfg) != cudaSuccess || n <= 0) {
             (void)cudaGetLastError();
             n = sm_count() / 2;
         }
@@ -368,7 +415,7 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
     p.group_offsets = nullptr;
     p.n_groups = 0;
     choose_tile_order(p);
-    gemm_fp8_pair_kernel<false><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
+    gemm_fp8_pair_kernel<0><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, ta, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }
@@ -387,7 +434,7 @@ int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa
     rc = b_mn ? make_tmap_2d_u8(&tb, b, (uint64_t)n_groups * K, (uint64_t)N, (uint64_t)N, BK, BN / 2)
               : make_tmap_2d_u8(&tb, b, (uint64_t)n_groups * N, (uint64_t)K, (uint64_t)K, BN / 2, BK);
     if (rc != FP8_OK) return rc;
-    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
     // the host does not know the group sizes: at most ceil(M/256) + n_groups row tiles exist
     const long tiles_bound = ((long)(M + 2 * BM - 1) / (2 * BM) + n_groups) * ((N + BN - 1) / BN);
     const int pairs_max = sm_count() / 2;
@@ -401,7 +448,64 @@ int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa
     p.group_offsets = group_offsets;
     p.n_groups = n_groups;
     p.band_w = GEMM_BAND; p.band_on_m = 1; p.hint_a = p.hint_b = 0;      // (the grouped form has its own tile table)
-    gemm_fp8_pair_kernel<true><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, p);
+    gemm_fp8_pair_kernel<1><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, ta, p);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+// Zero-padded copies of the last (possibly ragged) block of 128 reduction rows of every group: tail[g * 128 + i, :] =
+// a[offs[g] + 128 * (blocks_g - 1) + i, :] for the rows of group g, zero beyond them (blocks_g = max(1, ceil(rows_g / 128))).
+// The offsets are clamped like in the product kernel.  cols % 16 == 0.
+__global__ void __launch_bounds__(256) grouped_tail_kernel(const uint8_t *__restrict__ a, const int *__restrict__ offs,
+                                                           int n_rows, int cols, uint8_t *__restrict__ tail)
+{
+    const int g = blockIdx.x;
+    int prev = min(max(__ldg(offs), 0), n_rows);
+    for (int i = 0; i < g; ++i) prev = min(max(__ldg(offs + i + 1), prev), n_rows);
+    const int r0 = prev, r1 = min(max(__ldg(offs + g + 1), prev), n_rows);
+    const int rows = r1 - r0, blocks = max(1, (rows + 127) / 128);
+    const int t0 = r0 + (blocks - 1) * 128, valid = rows - (blocks - 1) * 128;       // 0 .. 128 rows to copy
+    const int vec = cols / 16;
+    const long n = 128l * vec;
+    for (long i = (long)blockIdx.y * blockDim.x + threadIdx.x; i < n; i += (long)gridDim.y * blockDim.x) {
+        const int row = (int)(i / vec), cv = (int)(i - (long)row * vec);
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (row < valid) v = __ldg(reinterpret_cast<const uint4 *>(a + (size_t)(t0 + row) * cols) + cv);
+        reinterpret_cast<uint4 *>(tail + ((size_t)g * 128 + row) * cols)[cv] = v;
+    }
+}
+
+// Weight gradients of the grouped product in one launch: C[g] (+)= sa_inv * sb_inv * A[rows of g]^T . B[rows of g] for every
+// group, A [T, M] and B [T, N] read in place, C [n_groups, M, N]; `tail` holds n_groups * 128 * M bytes of scratch.
+int launch_gemm_2cta_grouped_red(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv,
+                                 const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int T,
+                                 uint32_t idesc, uint8_t *tail, int *status, cudaStream_t st)
+{
+    using namespace g2;
+    CUtensorMap ta, tb, tt;
+    int rc = make_tmap_2d_u8(&ta, a, (uint64_t)T, (uint64_t)M, (uint64_t)M, BK, BM);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_2d_u8(&tb, b, (uint64_t)T, (uint64_t)N, (uint64_t)N, BK, BN / 2);
+    if (rc != FP8_OK) return rc;
+    rc = make_tmap_2d_u8(&tt, tail, (uint64_t)n_groups * BK, (uint64_t)M, (uint64_t)M, BK, BM);
+    if (rc != FP8_OK) return rc;
+    dim3 tgrid((unsigned)n_groups, (unsigned)((128l * (M / 16) + 255) / 256 < 64 ? (128l * (M / 16) + 255) / 256 : 64));
+    grouped_tail_kernel<<<tgrid, 256, 0, st>>>(a, group_offsets, T, M, tail);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(gemm_fp8_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN_BYTES));
+    const long tiles = (long)n_groups * ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
+    const int pairs_max = sm_count() / 2;
+    Params p;
+    p.o = o; p.sa_inv = sa_inv; p.sb_inv = sb_inv;
+    p.M = M; p.N = N; p.K = T;
+    p.a_mn = 1; p.b_mn = 1;
+    p.idesc = idesc;
+    p.num_pairs = (int)(tiles < pairs_max ? tiles : pairs_max);
+    p.status = status;
+    p.group_offsets = group_offsets;
+    p.n_groups = n_groups;
+    p.band_w = GEMM_BAND; p.band_on_m = 1; p.hint_a = p.hint_b = 0;
+    gemm_fp8_pair_kernel<2><<<2 * p.num_pairs, THREADS, DYN_BYTES, st>>>(ta, tb, tt, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }

@@ -224,6 +224,9 @@ int launch_gemm_2cta(const uint8_t *a, const uint8_t *b, const float *sa_inv, co
 int launch_gemm_2cta_grouped(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv,
                              const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int K, int b_mn,
                              uint32_t idesc, int *status, cudaStream_t st);
+int launch_gemm_2cta_grouped_red(const uint8_t *a, const uint8_t *b, const float *sa_inv, const float *sb_inv,
+                                 const int *group_offsets, int n_groups, const GemmOut &o, int M, int N, int T,
+                                 uint32_t idesc, uint8_t *tail, int *status, cudaStream_t st);
 
 // FP8DPA_GEMM=1cta|2cta forces one kernel family (for A/B measurements); default: chosen per shape.
 static int gemm_family_override()
@@ -512,4 +515,48 @@ extern "C" int fp8_grouped_linear_wgrad(const uint8_t *dY8, const uint8_t *X8, c
         if (rc != FP8_OK) return rc;
     }
     return FP8_OK;
+}
+
+// The same weight gradients in ONE launch with the offsets on the device (the router's output, as in the forward and the
+// data gradient): the CTA-pair kernel walks (expert, output tile) and reduces over that expert's rows; the last, possibly
+// ragged block of 128 rows of every expert is read from a zero-padded copy in `ws` (made by a small kernel first), so the
+// rows of the next expert that share the block contribute nothing.
+extern "C" size_t fp8_grouped_linear_wgrad_workspace_bytes(int n_groups, int N)
+{
+    if (n_groups <= 0 || N <= 0) return 0;
+    return (size_t)n_groups * 128 * (size_t)N;
+}
+
+extern "C" int fp8_grouped_linear_wgrad_dev(const uint8_t *dY8, const uint8_t *X8, const float *sdY_inv,
+                                            const float *sX_inv, const int *group_offsets, int n_groups, void *dW,
+                                            int out_is_fp32, int accumulate, int T, int N, int K, void *ws, size_t ws_bytes,
+                                            void *stream)
+{
+    if (!group_offsets || !dY8 || !X8 || !dW || !sdY_inv || !sX_inv) {
+        set_error("fp8_grouped_linear_wgrad_dev: NULL pointer");
+        return FP8_ERR_NULL;
+    }
+    if (n_groups <= 0 || n_groups > 256 || T <= 0 || N <= 0 || K <= 0 || (N % 16) || (K % 16)) {
+        set_error("fp8_grouped_linear_wgrad_dev: n_groups %d must be in [1, 256], T %d positive, N %d and K %d positive "
+                  "multiples of 16", n_groups, T, N, K);
+        return FP8_ERR_SHAPE;
+    }
+    if (!aligned16(dY8) || !aligned16(X8) || !aligned16(dW)) {
+        set_error("fp8_grouped_linear_wgrad_dev: tensor pointers must be 16-byte aligned");
+        return FP8_ERR_ALIGN;
+    }
+    const size_t need = fp8_grouped_linear_wgrad_workspace_bytes(n_groups, N);
+    if (!ws || ws_bytes < need || !aligned16(ws)) {
+        set_error("fp8_grouped_linear_wgrad_dev: workspace must be 16-byte aligned and hold %zu bytes (got %zu)", need,
+                  ws_bytes);
+        return FP8_ERR_WORKSPACE;
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    int *status = device_status_ptr();
+    if (!status) return FP8_ERR_CUDA;
+    const GemmOut o{dW, out_is_fp32, accumulate, nullptr, 0, nullptr};
+    return launch_gemm_2cta_grouped_red(dY8, X8, sdY_inv, sX_inv, group_offsets, n_groups, o, N, K, T,
+                                        umma_idesc_f8(FP8_E5M2, FP8_E4M3, 256, 256, 1, 1), static_cast<uint8_t *>(ws), status,
+                                        static_cast<cudaStream_t>(stream));
 }

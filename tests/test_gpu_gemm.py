@@ -356,6 +356,58 @@ def test_grouped_weight_gradient_matches_oracle_per_expert(sizes, N, K):
     assert err.value.status == -3
 
 
+@pytest.mark.parametrize("sizes,N,K", [([300, 0, 129, 512, 83], 528, 144), ([256, 256], 256, 256),
+                                        ([1000, 17, 2000, 1, 600, 0, 0, 350], 1024, 512), ([5], 16, 16),
+                                        ([0, 0, 384], 272, 1040), ([127, 1, 128, 129], 256, 512)])
+def test_grouped_weight_gradient_in_one_launch_with_device_offsets(sizes, N, K):
+    """The same gradients from fp8_grouped_linear_wgrad_dev: one launch over (expert, output tile), the offsets read on
+    the device, the ragged last block of every expert taken from a zero-padded copy.  Rows past the last offset and the
+    rows of the neighbouring experts that share a block of 128 must not leak into a gradient; out-of-range offsets are
+    clamped, not followed."""
+    E, T = len(sizes), sum(sizes)
+    Tpad = T + 9
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    dy = synth.normal_bf16((Tpad, N), 80 + E, 0, synth.GRAD_STD)
+    x = synth.normal_bf16((Tpad, K), 80 + E, 1, 1.0, synth.choose_columns(K, 2, 80, 1), 40.0)
+    dy8, _, _, _, sdy = gpu_quantize(dy, o.E5M2, False)
+    x8, _, _, _, sx = gpu_quantize(x, o.E4M3, False)
+    ody8, _, _, osdy = o.quantize(dy, o.E5M2)
+    ox8, _, _, osx = o.quantize(x, o.E4M3)
+    doffs = torch.from_numpy(offs).cuda()
+    ws = torch.full((fp8.fp8_grouped_linear_wgrad_workspace_bytes(E, N),), 0x7B, dtype=torch.uint8, device="cuda")
+    dw = torch.full((E, N, K), 7.0, dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_grouped_linear_wgrad_dev(dy8, x8, sdy, sx, doffs, dw, ws)
+    acc = torch.full((E, N, K), 0.25, dtype=torch.float32, device="cuda")
+    fp8.fp8_grouped_linear_wgrad_dev(dy8, x8, sdy, sx, doffs, acc, ws, accumulate=True)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    got, gacc = dw.float().cpu().numpy().astype(np.float64), acc.cpu().numpy().astype(np.float64)
+    for e in range(E):
+        r0, r1 = int(offs[e]), int(offs[e + 1])
+        if r1 == r0:
+            assert np.all(got[e] == 0.0) and np.all(gacc[e] == 0.25)      # no tokens: zero gradient / unchanged
+            continue
+        ref, mag = o.linear_wgrad(ody8[r0:r1], ox8[r0:r1], osdy, osx)
+        assert rel_err(got[e], ref, mag) <= 2.0 ** -8, e
+        assert rel_err(gacc[e], ref + 0.25, mag + 0.25) <= TOL_FP32, e
+    # bit-equal to the per-expert launches (same kernel arithmetic, same order of the reduction blocks)
+    dw2 = torch.full((E, N, K), 7.0, dtype=torch.bfloat16, device="cuda")
+    fp8.fp8_grouped_linear_wgrad(dy8, x8, sdy, sx, offs, dw2)
+    if N >= 256 and K >= 256:
+        assert torch.equal(dw.view(torch.int16), dw2.view(torch.int16))
+    # offsets that break the contract are clamped to [0, T] and made ascending: no access past the tensors
+    bad = torch.tensor([0, Tpad + 500] + [Tpad + 900] * (E - 1), dtype=torch.int32, device="cuda")
+    fp8.fp8_grouped_linear_wgrad_dev(dy8, x8, sdy, sx, bad, dw, ws)
+    torch.cuda.synchronize()
+    assert fp8.fp8_device_status() == 0
+    ref, mag = o.linear_wgrad(ody8, ox8, osdy, osx)
+    assert rel_err(dw[0].float().cpu().numpy().astype(np.float64), ref, mag) <= 2.0 ** -8
+    assert all(bool((dw[e] == 0).all()) for e in range(1, E))
+    with pytest.raises(fp8.Fp8Error) as err:
+        fp8.fp8_grouped_linear_wgrad_dev(dy8, x8, sdy, sx, doffs, dw, ws[:16])
+    assert err.value.status == -5
+
+
 def test_grouped_forward_argument_validation():
     x8 = torch.zeros((32, 32), dtype=torch.uint8, device="cuda")
     w8 = torch.zeros((2, 16, 32), dtype=torch.uint8, device="cuda")
