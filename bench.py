@@ -584,9 +584,9 @@ def run_ours(args, cfg):
 # gpu__time_duration.sum --clock-control none -k regex:gemm_fp8`), taken on the commit named in `source`.  None for
 # workloads without a capture: a figure from another build says nothing about this one.
 GEMM_DRAM_CAPTURE = {
-    "c4": {"bytes_per_launch": 314.13e6,
-           "source": "ncu, 12 launches of one c4 step, commit 2c45df1 (GEMM kernels unchanged since): read 213.3 MB + "
-                     "write 100.9 MB per launch on average, against 263 MB of operands and outputs"},
+    "c4": {"bytes_per_launch": 316.73e6,
+           "source": "ncu, 12 launches of one c4 step, commit 2df078f: read 215.6 MB + write 101.1 MB per launch on "
+                     "average, against 263 MB of operands and outputs"},
 }
 
 
