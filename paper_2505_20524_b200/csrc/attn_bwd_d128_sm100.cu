@@ -656,6 +656,10 @@ int launch_attn_bwd_d128(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8
     p.status = status;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_bwd_d128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::DYN_BYTES));
     dim3 grid((unsigned)(Hkv * B), (unsigned)((N + KT - 1) / KT), 1);
+    {
+        const int rc_regs = check_launch_registers(attn_bwd_d128_kernel, 128, "attn_bwd_d128_kernel");
+        if (rc_regs != FP8_OK) return rc_regs;
+    }
     attn_bwd_d128_kernel<<<grid, THREADS, Smem::DYN_BYTES, st>>>(tq, tk, tv, tdo, tdq, tvec, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     const size_t n4 = (size_t)B * N * Hq * D / 4;

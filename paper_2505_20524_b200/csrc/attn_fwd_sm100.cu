@@ -1394,6 +1394,8 @@ static int launch_attn_fwd(const uint8_t *Q8, const uint8_t *K8, const uint8_t *
     // the BF16 output as a byte tensor: 128-byte boxes (64 columns) of 128 rows
     rc = make_tmap_3d_u8(&to, p.O, (uint64_t)p.Hq * D * 2, (uint64_t)p.N, (uint64_t)p.B, 128, A_BM);
     if (rc != FP8_OK) return rc;
+    rc = check_launch_registers(attn_fwd_kernel<D>, 128, "attn_fwd_kernel");
+    if (rc != FP8_OK) return rc;
     attn_fwd_kernel<D><<<grid, A_THREADS, AttnFwdSmem<D>::DYN_BYTES, st>>>(tq, tk, tv, to, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
@@ -1415,6 +1417,8 @@ static int launch_attn_fwd_pair(const uint8_t *Q8, const uint8_t *K8, const uint
     if (rc != FP8_OK) return rc;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         AttnFwdPairSmem::DYN_BYTES));
+    rc = check_launch_registers(attn_fwd_pair_kernel, 128, "attn_fwd_pair_kernel");
+    if (rc != FP8_OK) return rc;
     dim3 grid((unsigned)((p.N + 255) / 256), (unsigned)p.Hq, (unsigned)p.B);
     attn_fwd_pair_kernel<<<grid, P_THREADS, AttnFwdPairSmem::DYN_BYTES, st>>>(tq, tk, tv, to, p);
     FP8_CUDA_CHECK(cudaGetLastError());
@@ -1436,13 +1440,8 @@ static int launch_attn_fwd_stream(const uint8_t *Q8, const uint8_t *K8, const ui
     if (rc != FP8_OK) return rc;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         AttnFwdStreamSmem::DYN_BYTES));
-    // the kernel's register hand-over between its warpgroups is balanced for this allocation at launch
-    cudaFuncAttributes fa;
-    FP8_CUDA_CHECK(cudaFuncGetAttributes(&fa, attn_fwd_stream_kernel));
-    if (fa.numRegs != X_REGS_LAUNCH) {
-        set_error("attn_fwd_stream_kernel: built with %d registers per thread, expected %d", fa.numRegs, X_REGS_LAUNCH);
-        return FP8_ERR_CUDA;
-    }
+    rc = check_launch_registers(attn_fwd_stream_kernel, X_REGS_LAUNCH, "attn_fwd_stream_kernel");
+    if (rc != FP8_OK) return rc;
     const long long n_items = (long long)((p.N + 127) / 128) * p.Hq * p.B;
     const int sms = sm_count();
     if (sms <= 0) return FP8_ERR_CUDA;

@@ -36,6 +36,21 @@ int make_tmap_3d_f32(CUtensorMap *map, const void *base, uint64_t d0_cols, uint6
         }                                                                                           \
     } while (0)
 
+// Kernels that move registers between their warpgroups (setmaxnreg) are balanced for one allocation at launch: an increase
+// beyond what the CTA's other warpgroups release would wait for ever, and no bounded wait covers that instruction.  Their
+// launchers call this first.
+template <typename F>
+inline int check_launch_registers(F *kernel, int expected, const char *name)
+{
+    cudaFuncAttributes fa;
+    FP8_CUDA_CHECK(cudaFuncGetAttributes(&fa, kernel));
+    if (fa.numRegs != expected) {
+        set_error("%s: built with %d registers per thread, its register hand-over expects %d", name, fa.numRegs, expected);
+        return FP8_ERR_CUDA;
+    }
+    return FP8_OK;
+}
+
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---------------------------------------------------------------- device side
