@@ -869,22 +869,26 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 
 // ---------------------------------------------------------------------------------------------------------------
 // Forward for d = 128, persistent form: one CTA per SM walks a list of (128-query tile, head, batch) items, and the key
-// blocks of all its items form one stream G = 0, 1, 2, ...  Two softmax warpgroups take the blocks of the stream in
-// turn (warpgroup G & 1), one row per thread, so that the exponentials of block G + 1 run while block G is still being
-// finished: with FP8 operands a 128 x 128 tile costs 512 clocks of MMAs against 1024 clocks of the exponential unit, so the
-// softmax chain of a single tile, not the tensor pipe, sets the pace, and two blocks of the same tile in flight hide
-// each other's latencies.  The scores are three blocks ahead: S(G), S(G+1), S(G+2) live in three TMEM buffers, so a
-// warpgroup never waits for the tensor pipe in steady state, also across the boundary between two items.
-//   warps 0-3 / 4-7  softmax warpgroups 0 / 1.  Block G of an item: score row TMEM -> registers, block maximum; the
-//               block maximum of G-1 that the other warpgroup published (shared memory, slot (G-1) & 3, fetched under the
-//               score loads) and this warpgroup's own m(G-2) give m(G-1); publishes its block maximum and the factor
-//               2^(m(G-1) - m(G)) for the accumulator, evaluates the exponentials, stores P8(G) over the first 32 columns
-//               of S(G).  Each warpgroup keeps the row sum of its own blocks with its own reference maximum; the
-//               epilogue merges the two
-//   warps 8-11  correction: rescales O when the running maximum grew (after PV(G-1) has completed), lets PV(G) go;
+// blocks of all its items form one stream G = 0, 1, 2, ...  NWG softmax warpgroups take the blocks of the stream in turn
+// (warpgroup G % NWG), one row per thread, so that the exponentials of one block run while its neighbours are being
+// started and finished: with FP8 operands a 128 x 128 tile costs 512 clocks of MMAs against 1024 clocks of the exponential
+// unit, so the softmax chain of a single tile, not the tensor pipe, sets the pace, and several blocks of the same tile in
+// flight hide each other's latencies.  The scores are three blocks ahead: S(G), S(G+1), S(G+2) live in three TMEM buffers.
+// With two warpgroups a warpgroup never waits for the tensor pipe in steady state, also across the boundary between two
+// items; with three (the default) every warpgroup has one buffer of its own and the other two cover the round trip of its
+// next scores through the tensor pipe.
+//   warps 0 .. 4 NWG - 1  softmax warpgroups.  Block G of an item: block maximum; the running maximum m(G-1) from what
+//               the neighbouring warpgroup published (shared memory, slot (G-1) & 3, fetched under the score loads);
+//               publishes its own and the factor 2^(m(G-1) - m(G)) for the accumulator, evaluates the exponentials, stores
+//               P8(G) over the first 32 columns of S(G).  NWG = 2: the score row sits in registers (184 per thread), the
+//               published value is the block maximum and m(G-1) follows from it and the warpgroup's own m(G-2).  NWG = 3:
+//               the row stays in TMEM and is read twice in chunks of 32 columns (112 registers per thread), the
+//               published value is the running maximum.  Each warpgroup keeps the row sum of its own blocks with its own
+//               reference maximum; the epilogue merges them
+//   next 4 warps  correction: rescales O when the running maximum grew (after PV(G-1) has completed), lets PV(G) go;
 //               per item normalises O, merges the row sums, writes O (BF16, tiled bulk stores) and LSE
-//   warp 12     TMA producer: Q (two buffers), K and V (4 stages each)
-//   warp 13     MMA issuer: QK(G+3) right after PV(G) (same TMEM buffer: the tensor pipe runs one thread's products in
+//   next warp   TMA producer: Q (two buffers), K and V (4 stages each)
+//   next warp   MMA issuer: QK(G+3) right after PV(G) (same TMEM buffer: the tensor pipe runs one thread's products in
 //               issue order, so S(G+3) overwrites P8(G) only after PV(G) has read it)
 // TMEM (512 columns): S buffers 0..2 | O.
 // setmaxnreg only moves registers inside the CTA's own allocation at launch (an increase beyond what the other warpgroups
@@ -893,10 +897,16 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 // depends, through PV(G) -> QK(G+3) -> S(G+3), on its previous use having been consumed, so no barrier can complete
 // twice before a waiter has seen it once.
 // ---------------------------------------------------------------------------------------------------------------
-constexpr int X_THREADS = 512;
+// NWG softmax warpgroups.  2: one row of 128 scores per thread held in registers (184 registers).  3: blocks G % 3, every
+// warpgroup with a score buffer of its own; the row stays in TMEM and is read twice in chunks of 32 columns (maximum, then
+// exponentials), which fits 112 registers; a warpgroup's next scores are issued when its P8 has been consumed, and the
+// other two warpgroups cover that round trip.
+template <int NWG> struct XCfg;
+template <> struct XCfg<2> { static constexpr int THREADS = 512, LAUNCH = 128, SOFTMAX = 184, CORR = 80, CTRL = 64; };
+template <> struct XCfg<3> { static constexpr int THREADS = 640, LAUNCH = 96, SOFTMAX = 112, CORR = 80, CTRL = 64; };
+static_assert(2 * 128 * XCfg<2>::SOFTMAX + 128 * XCfg<2>::CORR + 128 * XCfg<2>::CTRL <= XCfg<2>::THREADS * XCfg<2>::LAUNCH, "register budget");
+static_assert(3 * 128 * XCfg<3>::SOFTMAX + 128 * XCfg<3>::CORR + 128 * XCfg<3>::CTRL <= XCfg<3>::THREADS * XCfg<3>::LAUNCH, "register budget");
 constexpr int X_KS = 4, X_VS = 4;
-constexpr int X_REGS_LAUNCH = 128;
-static_assert(2 * 128 * P_REGS_SOFTMAX + 128 * P_REGS_CORR + 128 * P_REGS_CTRL <= X_THREADS * X_REGS_LAUNCH, "register budget");
 
 struct AttnFwdStreamSmem {
     static constexpr int D = 128;
@@ -907,12 +917,12 @@ struct AttnFwdStreamSmem {
     static constexpr int OST_OFF = V_OFF + X_VS * TILE_BYTES;    // output staging: [128 x 128] BF16 as two 64-column halves
     static constexpr int ALPHA_OFF = OST_OFF + 2 * TILE_BYTES;   // float[4][128]
     static constexpr int M_OFF = ALPHA_OFF + 4 * 128 * 4;        // float[4][128]: block maxima (scaled scores), slot G & 3
-    static constexpr int L_OFF = M_OFF + 4 * 128 * 4;            // float[2][128]: row sums of the two warpgroups
-    static constexpr int ML_OFF = L_OFF + 2 * 128 * 4;           // float[2][128]: their reference maxima
-    static constexpr int BAR_OFF = ML_OFF + 2 * 128 * 4;
+    static constexpr int L_OFF = M_OFF + 4 * 128 * 4;            // float[3][128]: row sums of the softmax warpgroups
+    static constexpr int ML_OFF = L_OFF + 3 * 128 * 4;           // float[3][128]: their reference maxima
+    static constexpr int BAR_OFF = ML_OFF + 3 * 128 * 4;
     // q_full[2] q_empty[2] k_full[KS] k_empty[KS] v_full[VS] v_empty[VS] s_full[3] pv_go[4] pv_done[4] am_ready[4][4]
-    // l_ready[2][4] epi_done
-    static constexpr int N_BARS = 4 + 2 * X_KS + 2 * X_VS + 3 + 4 + 4 + 16 + 8 + 1;
+    // l_ready[3][4] epi_done
+    static constexpr int N_BARS = 4 + 2 * X_KS + 2 * X_VS + 3 + 4 + 4 + 16 + 12 + 1;
     static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;
 };
@@ -942,7 +952,8 @@ struct FwdItems {
     }
 };
 
-__global__ void __launch_bounds__(X_THREADS, 1)
+template <int NWG>
+__global__ void __launch_bounds__(XCfg<NWG>::THREADS, 1)
 attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
                        const AttnFwdParams p)
@@ -965,7 +976,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     auto pv_done = [&](int s) { return bar0 + 8u * (B1 + 7 + s); };
     auto am_ready = [&](int s, int q) { return bar0 + 8u * (B1 + 11 + s * 4 + q); };
     auto l_ready = [&](int w, int q) { return bar0 + 8u * (B1 + 27 + w * 4 + q); };
-    const uint32_t epi_done = bar0 + 8u * (B1 + 35);
+    const uint32_t epi_done = bar0 + 8u * (B1 + 39);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFF + L::N_BARS * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     float *alpha_s = reinterpret_cast<float *>(smem + L::ALPHA_OFF);
@@ -974,6 +985,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     float *ml_s = reinterpret_cast<float *>(smem + L::ML_OFF);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int W_CORR = 4 * NWG, W_TMA = 4 * NWG + 4, W_MMA = 4 * NWG + 5;      // first correction warp, producer, issuer
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < 2; ++i) {
@@ -994,7 +1006,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             mbar_init(pv_done(s), 1);
             for (int q = 0; q < 4; ++q) mbar_init(am_ready(s, q), 1);
         }
-        for (int w = 0; w < 2; ++w)
+        for (int w = 0; w < 3; ++w)
             for (int q = 0; q < 4; ++q) mbar_init(l_ready(w, q), 1);
         mbar_init(epi_done, 4);
         *abort_flag = 0;
@@ -1004,7 +1016,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         tma_prefetch_desc(&tm_v);
         tma_prefetch_desc(&tm_o);
     }
-    if (warp == 13) {
+    if (warp == W_MMA) {
         tmem_alloc(smem_u32(tmem_slot), 512);
         tmem_relinquish();
     }
@@ -1017,9 +1029,9 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     FwdItems it;
     it.init();
 
-    if (warp >= 12) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(P_REGS_CTRL));
-        if (warp == 12) {
+    if (warp >= W_TMA) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(XCfg<NWG>::CTRL));
+        if (warp == W_TMA) {
             // ------------------------------------------------------------ TMA producer
             if (elect_one()) {
                 uint32_t gk = 0, gv = 0, n_it = 0;
@@ -1065,7 +1077,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     ++n_it;
                 }
             }
-        } else if (warp == 13) {
+        } else if (warp == W_MMA) {
             // ------------------------------------------------------------ MMA issuer
             if (elect_one()) {
                 constexpr uint32_t idesc_s = umma_idesc_f8(0, 0, 128, A_BN, 0, 0);
@@ -1123,8 +1135,8 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
         }
     }
-    else if (warp < 8) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(P_REGS_SOFTMAX));
+    else if (warp < W_CORR) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(XCfg<NWG>::SOFTMAX));
         // ------------------------------------------------------------ softmax warpgroup w: blocks G with (G & 1) == w
         const int w = warp >> 2, quad = warp & 3;
         const int r = quad * 32 + lane;
@@ -1201,11 +1213,91 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 m_own = m_new;
                 return true;
             };
+            // The same block for three warpgroups: the row stays in TMEM (buffer w) and is read twice in chunks of 32.
+            auto block3 = [&](auto masked, const int j) -> bool {
+                constexpr bool MASK = decltype(masked)::value;
+                const uint32_t G = gbase + (uint32_t)j;
+                const int limit = min(p.causal ? row : 0x7FFFFFFF, p.N - 1) - j * A_BN;   // last valid local column
+                const uint32_t sb = G % 3u;
+                if (!mbar_wait_warp(s_full((int)sb), (G / 3u) & 1u, ctx)) return false;
+                tc_fence_after();
+                const uint32_t tmem_s = tmem_base + sb * 128u + lane_addr;
+                uint32_t va[32], vb[32];
+                float mq[2] = {-INFINITY, -INFINITY};
+                auto chunk_max = [&](const uint32_t (&v)[32], int q, float &acc) {
+                    if (MASK) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (q * 32 + e <= limit) acc = fmaxf(acc, __uint_as_float(v[e]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) acc = fmax3(acc, __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+                    }
+                };
+                // first pass: the block maximum, two chunks in flight; the last load is chunk 0 again, for the second pass
+                tmem_ld_32x32b_x32(tmem_s + 64u, va);
+                tmem_ld_32x32b_x32(tmem_s + 96u, vb);
+                float m_prev = -INFINITY;
+                tmem_ld_wait();
+                chunk_max(va, 2, mq[0]);
+                chunk_max(vb, 3, mq[1]);
+                tmem_ld_32x32b_x32(tmem_s + 32u, vb);
+                tmem_ld_32x32b_x32(tmem_s, va);
+                // under the loads: the running maximum up to the previous block of this item
+                if (j > 0) {
+                    const uint32_t Gp = G - 1u;
+                    if (!mbar_wait_warp(am_ready((int)(Gp & 3u), quad), (Gp >> 2) & 1u, ctx)) return false;
+                    m_prev = m_s[(Gp & 3u) * 128u + r];
+                }
+                tmem_ld_wait();
+                chunk_max(vb, 1, mq[1]);
+                chunk_max(va, 0, mq[0]);
+                const float m_blk = fmaxf(mq[0], mq[1]) * c;
+                const bool grew = m_blk > m_prev + p.max_slack;
+                const float m_new = grew ? m_blk : m_prev;
+                // for the next warpgroup (the running maximum) and the correction warps (the factor for the accumulator)
+                alpha_s[(G & 3u) * 128u + r] = grew ? ex2_approx(m_prev - m_new) : 1.0f;      // first block: 0
+                m_s[(G & 3u) * 128u + r] = m_new;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(am_ready((int)(G & 3u), quad));
+                const float neg_shift = p.log2_p_scale - m_new;
+                float lsum = 0.0f;
+                // second pass: chunk q from registers while chunk q + 1 is on its way; P8 of chunk q goes over score columns
+                // 8q .. 8q+7, all inside chunk 0, which is in registers by now
+                {
+                    uint32_t wq[8];
+                    lsum += softmax_chunk<MASK, P_POLY>(va, c, neg_shift, limit, wq);             // chunk 0 (vb holds chunk 1)
+                    tmem_ld_32x32b_x32(tmem_s + 64u, va);
+                    tmem_st_32x32b_x8(tmem_s, wq);
+                    lsum += softmax_chunk<MASK, P_POLY>(vb, c, neg_shift, limit - 32, wq);        // chunk 1
+                    tmem_ld_wait();
+                    tmem_ld_32x32b_x32(tmem_s + 96u, vb);
+                    tmem_st_32x32b_x8(tmem_s + 8u, wq);
+                    lsum += softmax_chunk<MASK, P_POLY>(va, c, neg_shift, limit - 64, wq);        // chunk 2
+                    tmem_ld_wait();
+                    tmem_st_32x32b_x8(tmem_s + 16u, wq);
+                    lsum += softmax_chunk<MASK, P_POLY>(vb, c, neg_shift, limit - 96, wq);        // chunk 3
+                    tmem_st_32x32b_x8(tmem_s + 24u, wq);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pv_go((int)(G & 3u)));
+                l = l * ((m_own == m_new) ? 1.0f : ex2_approx(m_own - m_new)) + lsum;
+                m_own = m_new;
+                return true;
+            };
             const int k_last = (n_kv - 1) * A_BN;
             const bool last_masked = (k_last + A_BN - 1 > qs && p.causal) || (k_last + A_BN > p.N);
-            for (int j = (int)((gbase ^ (uint32_t)w) & 1u); j < n_kv && ok; j += 2) {
-                if (j == n_kv - 1 && last_masked) ok = block(std::true_type{}, j);
-                else ok = block(std::false_type{}, j);
+            // this warpgroup's blocks of the item: G = gbase + j with G % NWG == w
+            for (int j = (int)(((uint32_t)w + (uint32_t)NWG - gbase % (uint32_t)NWG) % (uint32_t)NWG); j < n_kv && ok; j += NWG) {
+                if (NWG == 2) {
+                    if (j == n_kv - 1 && last_masked) ok = block(std::true_type{}, j);
+                    else ok = block(std::false_type{}, j);
+                } else {
+                    if (j == n_kv - 1 && last_masked) ok = block3(std::true_type{}, j);
+                    else ok = block3(std::false_type{}, j);
+                }
             }
             if (!ok) break;
             // the epilogue of the previous item has read the row sums
@@ -1217,8 +1309,8 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             gbase += (uint32_t)n_kv;
             ++n_it;
         }
-    } else if (warp < 12) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(P_REGS_CORR));
+    } else if (warp < W_TMA) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(XCfg<NWG>::CORR));
         // ------------------------------------------------------------ correction and epilogue
         const int quad = warp & 3;
         const int r = quad * 32 + lane;
@@ -1263,17 +1355,22 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             if (!ok) break;
             // ---- epilogue of the item: merge the two row sums, normalise, store
             const uint32_t Gl = gbase + (uint32_t)n_kv - 1u;
-            if (!mbar_wait_warp(l_ready(0, quad), n_it & 1u, ctx) || !mbar_wait_warp(l_ready(1, quad), n_it & 1u, ctx) ||
-                !mbar_wait_warp(pv_done((int)(Gl & 3u)), (Gl >> 2) & 1u, ctx)) {
+            bool lr = true;
+            for (int w = 0; w < NWG && lr; ++w) lr = mbar_wait_warp(l_ready(w, quad), n_it & 1u, ctx);
+            if (!lr || !mbar_wait_warp(pv_done((int)(Gl & 3u)), (Gl >> 2) & 1u, ctx)) {
                 ok = false;
                 break;
             }
             tc_fence_after();
             const int row = it.q_tile * 128 + r;
-            const float m0 = ml_s[r], m1 = ml_s[128 + r];
-            const float mf = fmaxf(m0, m1);
-            const float lt = l_s[r] * (m0 == mf ? 1.0f : ex2_approx(m0 - mf)) +
-                             l_s[128 + r] * (m1 == mf ? 1.0f : ex2_approx(m1 - mf));
+            float mf = -INFINITY, lt = 0.0f;
+#pragma unroll
+            for (int w = 0; w < NWG; ++w) mf = fmaxf(mf, ml_s[w * 128 + r]);
+#pragma unroll
+            for (int w = 0; w < NWG; ++w) {
+                const float mw = ml_s[w * 128 + r];
+                lt += l_s[w * 128 + r] * (mw == mf ? 1.0f : ex2_approx(mw - mf));
+            }
             const float inv = __ldg(p.v_inv) / lt;                 // lt already carries c_P
             if (row < p.N)
                 p.LSE[((size_t)it.b * p.Hq + it.h) * p.N + row] = (mf + log2f(lt) - p.log2_p_scale) * 0.69314718055994531f;
@@ -1348,7 +1445,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int i = 0; i < 64; ++i) __nanosleep(20000);
         __syncthreads();
     }
-    if (warp == 13) {
+    if (warp == W_MMA) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);
     }
@@ -1425,6 +1522,7 @@ static int launch_attn_fwd_pair(const uint8_t *Q8, const uint8_t *K8, const uint
     return FP8_OK;
 }
 
+template <int NWG>
 static int launch_attn_fwd_stream(const uint8_t *Q8, const uint8_t *K8, const uint8_t *V8, const AttnFwdParams &p,
                                   cudaStream_t st)
 {
@@ -1438,26 +1536,26 @@ static int launch_attn_fwd_stream(const uint8_t *Q8, const uint8_t *K8, const ui
     if (rc != FP8_OK) return rc;
     rc = make_tmap_3d_u8(&to, p.O, (uint64_t)p.Hq * D * 2, (uint64_t)p.N, (uint64_t)p.B, 128, 32);
     if (rc != FP8_OK) return rc;
-    FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_stream_kernel<NWG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         AttnFwdStreamSmem::DYN_BYTES));
-    rc = check_launch_registers(attn_fwd_stream_kernel, X_REGS_LAUNCH, "attn_fwd_stream_kernel");
+    rc = check_launch_registers(attn_fwd_stream_kernel<NWG>, XCfg<NWG>::LAUNCH, "attn_fwd_stream_kernel");
     if (rc != FP8_OK) return rc;
     const long long n_items = (long long)((p.N + 127) / 128) * p.Hq * p.B;
     const int sms = sm_count();
     if (sms <= 0) return FP8_ERR_CUDA;
     dim3 grid((unsigned)(n_items < sms ? n_items : sms));
-    attn_fwd_stream_kernel<<<grid, X_THREADS, AttnFwdStreamSmem::DYN_BYTES, st>>>(tq, tk, tv, to, p);
+    attn_fwd_stream_kernel<NWG><<<grid, XCfg<NWG>::THREADS, AttnFwdStreamSmem::DYN_BYTES, st>>>(tq, tk, tv, to, p);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }
 
-// The d = 128 kernel: the persistent one ("stream": two softmax warpgroups on alternating key blocks) unless
-// FP8DPA_ATTN_FWD names another for A/B measurements: "single" = one 128-row tile per CTA, two CTAs per SM; "pair" = two
-// tiles per CTA
+// The d = 128 kernel: the persistent one with three softmax warpgroups unless FP8DPA_ATTN_FWD names another for A/B
+// measurements: "stream2" = the persistent kernel with two warpgroups (score rows in registers); "pair" = two tiles per CTA;
+// "single" = one 128-row tile per CTA, two CTAs per SM
 static int attn_fwd_choice()
 {
     const char *e = getenv("FP8DPA_ATTN_FWD");      // read per call: tests switch it
-    return (e && strcmp(e, "single") == 0) ? 0 : (e && strcmp(e, "pair") == 0) ? 1 : 2;
+    return (e && strcmp(e, "single") == 0) ? 0 : (e && strcmp(e, "pair") == 0) ? 1 : (e && strcmp(e, "stream2") == 0) ? 2 : 3;
 }
 
 }  // namespace fp8dpa
@@ -1504,7 +1602,8 @@ static int attention_fwd_common(const char *who, const uint8_t *Q8, const uint8_
     if (o_scale && o_amax) FP8_CUDA_CHECK(cudaMemsetAsync(o_amax, 0, sizeof(float), st));
     if (d == 128) {
         const int ch = attn_fwd_choice();
-        return ch == 2 ? launch_attn_fwd_stream(Q8, K8, V8, p, st)
+        return ch == 3 ? launch_attn_fwd_stream<3>(Q8, K8, V8, p, st)
+               : ch == 2 ? launch_attn_fwd_stream<2>(Q8, K8, V8, p, st)
                        : ch == 1 ? launch_attn_fwd_pair(Q8, K8, V8, p, st) : launch_attn_fwd<128>(Q8, K8, V8, p, st);
     }
     return launch_attn_fwd<64>(Q8, K8, V8, p, st);

@@ -73,14 +73,14 @@ def test_forward_matches_oracle(name, B, N, causal):
            oracle_whole_row_vs_blocked_fro=norm_ratios(ref0, ref)[0])
 
 
-@pytest.mark.parametrize("family", ["single", "pair", "stream"])
+@pytest.mark.parametrize("family", ["single", "pair", "stream2", "stream"])
 @pytest.mark.parametrize("name,B,N,causal", [("c3", 1, 656, True), ("c4", 2, 400, True), ("c4", 1, 272, False),
                                              ("c3", 3, 128, True)])
 def test_forward_kernel_families_at_head_dim_128(family, name, B, N, causal, monkeypatch):
     """FP8DPA_ATTN_FWD picks the d = 128 kernel: one tile per CTA, two tiles per CTA, or the persistent kernel whose CTAs
-    walk several (tile, head, batch) items with two softmax warpgroups on alternating key blocks (the default).  All
-    three must agree with the oracle; the shapes give CTAs of the persistent kernel items of different lengths, odd and
-    even block counts (the warpgroups swap roles from item to item), a ragged last tile and grouped heads."""
+    walk several (tile, head, batch) items with two or three (the default) softmax warpgroups taking the key blocks in turn.
+    All four must agree with the oracle; the shapes give CTAs of the persistent kernel items of different lengths, block
+    counts of every residue (the warpgroups change roles from item to item), a ragged last tile and grouped heads."""
     monkeypatch.setenv("FP8DPA_ATTN_FWD", family)
     cfg = synth.CONFIGS[name]
     Hq, Hkv, d = cfg.n_q_heads // 4, cfg.n_kv_heads // 4, cfg.head_dim
