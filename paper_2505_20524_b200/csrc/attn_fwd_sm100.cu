@@ -921,8 +921,8 @@ struct AttnFwdStreamSmem {
     static constexpr int ML_OFF = L_OFF + 3 * 128 * 4;           // float[3][128]: their reference maxima
     static constexpr int BAR_OFF = ML_OFF + 3 * 128 * 4;
     // q_full[2] q_empty[2] k_full[KS] k_empty[KS] v_full[VS] v_empty[VS] s_full[3] pv_go[4] pv_done[4] am_ready[4][4]
-    // l_ready[3][4] epi_done
-    static constexpr int N_BARS = 4 + 2 * X_KS + 2 * X_VS + 3 + 4 + 4 + 16 + 12 + 1;
+    // l_ready[3][4] epi_done m_ready[4][4]
+    static constexpr int N_BARS = 4 + 2 * X_KS + 2 * X_VS + 3 + 4 + 4 + 16 + 12 + 1 + 16;
     static constexpr int TOTAL = BAR_OFF + N_BARS * 8 + 16;
     static constexpr int DYN_BYTES = TOTAL + 1024;
 };
@@ -952,6 +952,14 @@ struct FwdItems {
     }
 };
 
+// ex2.approx that the compiler keeps where it is written (its result is wanted long before its use)
+__device__ __forceinline__ float ex2_approx_pinned(float x)
+{
+    float y;
+    asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <int NWG>
 __global__ void __launch_bounds__(XCfg<NWG>::THREADS, 1)
 attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -977,6 +985,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     auto am_ready = [&](int s, int q) { return bar0 + 8u * (B1 + 11 + s * 4 + q); };
     auto l_ready = [&](int w, int q) { return bar0 + 8u * (B1 + 27 + w * 4 + q); };
     const uint32_t epi_done = bar0 + 8u * (B1 + 39);
+    auto m_ready = [&](int s, int q) { return bar0 + 8u * (B1 + 40 + s * 4 + q); };      // three warpgroups only
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + L::BAR_OFF + L::N_BARS * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
     float *alpha_s = reinterpret_cast<float *>(smem + L::ALPHA_OFF);
@@ -1004,7 +1013,10 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int s = 0; s < 4; ++s) {
             mbar_init(pv_go(s), 8);          // four softmax warps (P8 stored) + four correction warps (O rescaled)
             mbar_init(pv_done(s), 1);
-            for (int q = 0; q < 4; ++q) mbar_init(am_ready(s, q), 1);
+            for (int q = 0; q < 4; ++q) {
+                mbar_init(am_ready(s, q), 1);
+                mbar_init(m_ready(s, q), 1);
+            }
         }
         for (int w = 0; w < 3; ++w)
             for (int q = 0; q < 4; ++q) mbar_init(l_ready(w, q), 1);
@@ -1088,30 +1100,40 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 int jq = 0;                    // its block within item qi
                 uint32_t nq_it = 0;            // items begun by the QK cursor
                 bool q_valid = qi.next(p), ok = true;
-                auto issue_next_qk = [&]() -> bool {
-                    const int qb = (int)(nq_it & 1u);
-                    if (jq == 0 && !mbar_wait(q_full(qb), (nq_it >> 1) & 1u, ctx)) return false;
-                    const uint32_t st = gkq % X_KS;
-                    if (!mbar_wait(k_full(st), (gkq / X_KS) & 1u, ctx)) return false;
+                // the next QK in two steps, so that its waits (loads that landed long ago, but every look at a barrier
+                // costs a round trip) are taken before the wait for P8 and not between PV(G) and QK(G+3)
+                uint64_t nq_dq = 0, nq_dk = 0;
+                uint32_t nq_st = 0;
+                int nq_qb = 0;
+                auto prepare_next_qk = [&]() -> bool {
+                    nq_qb = (int)(nq_it & 1u);
+                    if (jq == 0 && !mbar_wait(q_full(nq_qb), (nq_it >> 1) & 1u, ctx)) return false;
+                    nq_st = gkq % X_KS;
+                    if (!mbar_wait(k_full((int)nq_st), (gkq / X_KS) & 1u, ctx)) return false;
+                    nq_dq = umma_desc(sbase + L::Q_OFF + nq_qb * L::TILE_BYTES, D, 16);
+                    nq_dk = umma_desc(sbase + L::K_OFF + nq_st * L::TILE_BYTES, D, 16);
+                    return true;
+                };
+                auto fire_next_qk = [&]() {
                     tc_fence_after();
-                    const uint64_t dq = umma_desc(sbase + L::Q_OFF + qb * L::TILE_BYTES, D, 16);
-                    const uint64_t dk = umma_desc(sbase + L::K_OFF + st * L::TILE_BYTES, D, 16);
                     const uint32_t ts = tmem_base + (gq % 3u) * 128u;
 #pragma unroll
-                    for (int k = 0; k < D / 32; ++k) umma_f8_ss(ts, dq + 2u * k, dk + 2u * k, idesc_s, k != 0);
+                    for (int k = 0; k < D / 32; ++k) umma_f8_ss(ts, nq_dq + 2u * k, nq_dk + 2u * k, idesc_s, k != 0);
                     umma_commit(s_full((int)(gq % 3u)));
-                    umma_commit(k_empty((int)st));
+                    umma_commit(k_empty((int)nq_st));
                     ++gq;
                     ++gkq;
                     if (++jq == qi.n_kv) {
-                        umma_commit(q_empty(qb));          // the item's last QK has read Q
+                        umma_commit(q_empty(nq_qb));       // the item's last QK has read Q
                         jq = 0;
                         ++nq_it;
                         q_valid = qi.next(p);
                     }
-                    return true;
                 };
-                for (int i = 0; i < 3 && ok && q_valid; ++i) ok = issue_next_qk();
+                for (int i = 0; i < 3 && ok && q_valid; ++i) {
+                    ok = prepare_next_qk();
+                    if (ok) fire_next_qk();
+                }
                 uint32_t gp = 0, gvp = 0, np_it = 0;
                 while (ok && it.next(p)) {
                     for (int j = 0; j < it.n_kv && ok; ++j, ++gp, ++gvp) {
@@ -1119,6 +1141,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         if (!mbar_wait(v_full(st), (gvp / X_VS) & 1u, ctx)) { ok = false; break; }
                         // the epilogue of the previous item has read O
                         if (j == 0 && np_it > 0 && !mbar_wait(epi_done, (np_it - 1u) & 1u, ctx)) { ok = false; break; }
+                        if (q_valid && !prepare_next_qk()) { ok = false; break; }
                         if (!mbar_wait(pv_go((int)(gp & 3u)), (gp >> 2) & 1u, ctx)) { ok = false; break; }
                         tc_fence_after();
                         const uint64_t dv = umma_desc(sbase + L::V_OFF + st * L::TILE_BYTES, D, 16);
@@ -1128,7 +1151,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                             umma_f8_ts(tmem_o, ts + 8u * k, dv + (uint32_t)((32 * D) >> 4) * k, idesc_o, (j | k) != 0);
                         umma_commit(pv_done((int)(gp & 3u)));
                         umma_commit(v_empty((int)st));
-                        if (q_valid) ok = issue_next_qk();
+                        if (q_valid) fire_next_qk();
                     }
                     ++np_it;
                 }
@@ -1246,7 +1269,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 // under the loads: the running maximum up to the previous block of this item
                 if (j > 0) {
                     const uint32_t Gp = G - 1u;
-                    if (!mbar_wait_warp(am_ready((int)(Gp & 3u), quad), (Gp >> 2) & 1u, ctx)) return false;
+                    if (!mbar_wait_warp(m_ready((int)(Gp & 3u), quad), (Gp >> 2) & 1u, ctx)) return false;
                     m_prev = m_s[(Gp & 3u) * 128u + r];
                 }
                 tmem_ld_wait();
@@ -1255,11 +1278,14 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 const float m_blk = fmaxf(mq[0], mq[1]) * c;
                 const bool grew = m_blk > m_prev + p.max_slack;
                 const float m_new = grew ? m_blk : m_prev;
-                // for the next warpgroup (the running maximum) and the correction warps (the factor for the accumulator)
-                alpha_s[(G & 3u) * 128u + r] = grew ? ex2_approx(m_prev - m_new) : 1.0f;      // first block: 0
+                // the next warpgroup needs the running maximum first
                 m_s[(G & 3u) * 128u + r] = m_new;
                 __syncwarp();
-                if (lane == 0) mbar_arrive(am_ready((int)(G & 3u), quad));
+                if (lane == 0) mbar_arrive(m_ready((int)(G & 3u), quad));
+                // The two factors 2^(..) are started here and used further down: a result of the exponential unit arrives only
+                // after it has queued behind the other warpgroups' exponentials, and a warp issues in order.
+                const float a_raw = ex2_approx_pinned(m_prev - m_new);      // first block: 2^-inf = 0
+                const float f_raw = ex2_approx_pinned(m_own - m_new);
                 const float neg_shift = p.log2_p_scale - m_new;
                 float lsum = 0.0f;
                 // second pass: chunk q from registers while chunk q + 1 is on its way; P8 of chunk q goes over score columns
@@ -1269,6 +1295,10 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     lsum += softmax_chunk<MASK, P_POLY>(va, c, neg_shift, limit, wq);             // chunk 0 (vb holds chunk 1)
                     tmem_ld_32x32b_x32(tmem_s + 64u, va);
                     tmem_st_32x32b_x8(tmem_s, wq);
+                    // the factor for the accumulator, for the correction warps
+                    alpha_s[(G & 3u) * 128u + r] = grew ? a_raw : 1.0f;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(am_ready((int)(G & 3u), quad));
                     lsum += softmax_chunk<MASK, P_POLY>(vb, c, neg_shift, limit - 32, wq);        // chunk 1
                     tmem_ld_wait();
                     tmem_ld_32x32b_x32(tmem_s + 96u, vb);
@@ -1283,7 +1313,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pv_go((int)(G & 3u)));
-                l = l * ((m_own == m_new) ? 1.0f : ex2_approx(m_own - m_new)) + lsum;
+                l = l * ((m_own == m_new) ? 1.0f : f_raw) + lsum;
                 m_own = m_new;
                 return true;
             };
