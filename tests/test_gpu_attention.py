@@ -97,6 +97,40 @@ def test_forward_kernel_families_at_head_dim_128(family, name, B, N, causal, mon
     assert np.max(np.abs(glse - lse)) <= 1e-3 * max(1.0, np.abs(lse).max())
 
 
+@pytest.mark.parametrize("N,B,Hq,Hkv", [(16, 1, 1, 1), (112, 2, 4, 2), (128, 1, 8, 1), (144, 3, 2, 2), (272, 1, 40, 8),
+                                        (400, 2, 4, 2), (784, 1, 8, 1), (1296, 1, 4, 2), (3088, 1, 8, 1)])
+def test_forward_kernel_families_agree_over_many_item_layouts(N, B, Hq, Hkv, monkeypatch):
+    """The persistent kernels give every CTA a different list of items (1 to 25 key blocks each, more or fewer items than
+    CTAs, warpgroups changing roles at every item boundary).  Random codes, all four d = 128 kernels, causal and not, exact
+    and slack reference maximum: the same codes must come out up to the BF16 rounding of O (the kernels differ only in the
+    order of the row sum) and no bounded wait may expire."""
+    d = 128
+    g = torch.Generator(device="cuda").manual_seed(N * 131 + B * 17 + Hq)
+    def codes(*shape):
+        c = torch.randint(0x20, 0x50, shape, dtype=torch.uint8, device="cuda", generator=g)
+        return c | (torch.randint(0, 2, shape, dtype=torch.uint8, device="cuda", generator=g) << 7)
+    q8, k8, v8 = codes(B, N, Hq, d), codes(B, N, Hkv, d), codes(B, N, Hkv, d)
+    s1 = scalar(0.04)
+    def run(kind, causal, tau):
+        monkeypatch.setenv("FP8DPA_ATTN_FWD", kind)
+        O = torch.zeros((B, N, Hq, d), dtype=torch.bfloat16, device="cuda")
+        LSE = torch.zeros((B, Hq, N), dtype=torch.float32, device="cuda")
+        fp8.fp8_attention_fwd(q8, k8, v8, s1, s1, s1, d ** -0.5, causal, O, LSE, None, p_scale=448.0 / 2 ** tau, max_slack=tau)
+        torch.cuda.synchronize()
+        assert fp8.fp8_device_status() == 0, kind
+        return O.float(), LSE
+    for causal in (True, False):
+        if not causal and N > 1300:
+            continue
+        for tau in (0.0, 2.0):
+            ref = run("single", causal, tau)
+            for kind in ("pair", "stream2", "stream"):
+                O, LSE = run(kind, causal, tau)
+                assert torch.isfinite(O).all()
+                assert (O - ref[0]).abs().max() <= 2.0 ** -7 * ref[0].abs().max(), (kind, causal, tau)
+                assert (LSE - ref[1]).abs().max() <= 1e-4, (kind, causal, tau)
+
+
 @pytest.mark.parametrize("name,B,N,causal,tau", [("c1", 1, 400, True, 3.0), ("c3", 1, 384, True, 3.0),
                                                  ("c4", 1, 272, True, 2.0), ("c4", 1, 256, False, 3.0)])
 def test_forward_with_reference_maximum_slack_matches_oracle(name, B, N, causal, tau):
