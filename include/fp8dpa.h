@@ -87,6 +87,19 @@ FP8_API int fp8_cast(const void *x_bf16, size_t rows, size_t cols, const float *
 FP8_API int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fmt, uint8_t *out, uint8_t *out_t,
                  float *amax, float *scale, float *scale_inv, void *stream);
 
+/* fp8_quantize of up to 8 flat tensors (the operands of one layer) in two launches instead of two per tensor: one
+ * reduction over all of them, one cast of all of them (the just-in-time recipe of Section 2, unchanged arithmetic: every
+ * tensor has its own amax, scale and codes, bit-identical to fp8_quantize).  `items` is a HOST array; item i casts the
+ * n BF16 values at x_bf16 to out (no transposed copy).  scalars: device array of 3 * n_items floats, overwritten with
+ * (amax, scale, 1 / scale) of item i at scalars[3 i .. 3 i + 2]. */
+typedef struct {
+    const void *x_bf16;   /* device, 16-byte aligned */
+    size_t n;             /* number of BF16 values, > 0 */
+    int fmt;              /* FP8_E4M3 / FP8_E5M2 */
+    uint8_t *out;         /* device, 16-byte aligned, n bytes */
+} fp8_quant_item;
+FP8_API int fp8_quantize_multi(const fp8_quant_item *items, int n_items, float *scalars, void *stream);
+
 /* Delayed scaling (Appendix E): H holds the last `len` abs-max values of one tensor (the paper trains with
  * len = 1024, margin 0); rho = FP8Max / (2^margin * max H); after a step, H <- {amax} u H minus its oldest
  * entry, "to use in the next iteration".  This call does that update on the device: history[*head] = *amax_new,

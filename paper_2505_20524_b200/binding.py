@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
-           "fp8_quantize", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis", "fp8_amax_kurtosis",
+           "fp8_quantize", "fp8_quantize_multi", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis", "fp8_amax_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_grouped_linear_wgrad_workspace_bytes", "fp8_grouped_linear_wgrad_dev", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_linear_dgrad_blockwise", "fp8_linear_wgrad_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static",
            "fp8_linear_step_host_workspace_bytes", "fp8_linear_step_host", "fp8_attention_step_host_workspace_bytes",
@@ -131,6 +131,21 @@ def fp8_quantize(x, fmt, out, out_t, amax, scale, scale_inv, stream=None):
     rows, cols = _rows_cols(x)
     _check(load().fp8_quantize(_ptr(x), C.c_size_t(rows), C.c_size_t(cols), C.c_int(fmt), _ptr(out), _ptr(out_t),
                                _ptr(amax), _ptr(scale), _ptr(scale_inv), _stream(stream)))
+
+
+class QuantItem(C.Structure):
+    _fields_ = [("x_bf16", C.c_void_p), ("n", C.c_size_t), ("fmt", C.c_int), ("out", C.c_void_p)]
+
+
+def fp8_quantize_multi(xs, fmts, outs, scalars, stream=None):
+    """Just-in-time quantize of up to 8 tensors in two launches: xs BF16 CUDA tensors, outs uint8 CUDA tensors of the same
+    sizes, scalars a float32 CUDA tensor of 3 * len(xs) entries receiving (amax, scale, 1 / scale) per tensor."""
+    n = len(xs)
+    assert len(fmts) == n and len(outs) == n and scalars.numel() >= 3 * n
+    items = (QuantItem * n)()
+    for i, (x, f, o) in enumerate(zip(xs, fmts, outs)):
+        items[i] = QuantItem(_ptr(x).value, x.numel(), int(f), _ptr(o).value)
+    _check(load().fp8_quantize_multi(items, C.c_int(n), _ptr(scalars), _stream(stream)))
 
 
 ACT_GELU, ACT_XIELU = 1, 2

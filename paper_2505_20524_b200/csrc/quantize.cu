@@ -29,13 +29,13 @@ __device__ __forceinline__ void block_atomic_max_bf16(uint32_t m2, unsigned int 
     }
 }
 
-__global__ void __launch_bounds__(512) amax_kernel(const uint4 *__restrict__ x, size_t n_vec,
-                                                   const uint16_t *__restrict__ tail, int n_tail,
-                                                   unsigned int *__restrict__ amax_bits)
+// The reduction over one tensor as seen by block `rank` of the `nblk` blocks that share it.
+__device__ __forceinline__ void amax_body(const uint4 *__restrict__ x, size_t n_vec, const uint16_t *__restrict__ tail,
+                                          int n_tail, unsigned int *__restrict__ amax_bits, unsigned rank, unsigned nblk)
 {
     uint32_t m = 0;
-    const size_t stride = (size_t)gridDim.x * blockDim.x;
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t stride = (size_t)nblk * blockDim.x;
+    size_t i = (size_t)rank * blockDim.x + threadIdx.x;
     // four independent 16-byte loads in flight per thread
     for (; i + 3 * stride < n_vec; i += 4 * stride) {
         const uint4 a = __ldg(x + i), b = __ldg(x + i + stride), c = __ldg(x + i + 2 * stride),
@@ -49,8 +49,42 @@ __global__ void __launch_bounds__(512) amax_kernel(const uint4 *__restrict__ x, 
         const uint4 a = __ldg(x + i);
         m = absmax2(absmax2(absmax2(absmax2(m, a.x), a.y), a.z), a.w);
     }
-    if (blockIdx.x == 0 && (int)threadIdx.x < n_tail) m = absmax2(m, (uint32_t)tail[threadIdx.x]);
+    if (rank == 0 && (int)threadIdx.x < n_tail) m = absmax2(m, (uint32_t)tail[threadIdx.x]);
     block_atomic_max_bf16(m, amax_bits);
+}
+
+__global__ void __launch_bounds__(512) amax_kernel(const uint4 *__restrict__ x, size_t n_vec,
+                                                   const uint16_t *__restrict__ tail, int n_tail,
+                                                   unsigned int *__restrict__ amax_bits)
+{
+    amax_body(x, n_vec, tail, n_tail, amax_bits, blockIdx.x, gridDim.x);
+}
+
+// Several tensors in one launch (the operands of one layer): block b works on the tensor whose block range holds b.
+constexpr int MULTI_MAX = 8;
+struct MultiItem {
+    const uint16_t *x;
+    uint8_t *out;
+    size_t n;
+    int fmt;
+    unsigned blk0;       // first block of this tensor
+};
+struct MultiArgs {
+    MultiItem it[MULTI_MAX];
+    int n_items;
+    unsigned n_blocks;
+    float *scalars;      // per tensor: amax, scale, 1 / scale
+};
+
+__global__ void __launch_bounds__(512) amax_multi_kernel(const MultiArgs a)
+{
+    int t = 0;
+    while (t + 1 < a.n_items && blockIdx.x >= a.it[t + 1].blk0) ++t;
+    const MultiItem &m = a.it[t];
+    const unsigned nblk = (t + 1 < a.n_items ? a.it[t + 1].blk0 : a.n_blocks) - m.blk0;
+    const size_t n_vec = m.n / 8;
+    amax_body(reinterpret_cast<const uint4 *>(m.x), n_vec, m.x + n_vec * 8, (int)(m.n - n_vec * 8),
+              reinterpret_cast<unsigned int *>(a.scalars + 3 * t), blockIdx.x - m.blk0, nblk);
 }
 
 // ---------------------------------------------------------------- scale
@@ -142,17 +176,17 @@ __device__ __forceinline__ uint2 cast8(const uint4 v, const float s)
     return make_uint2((uint32_t)h[0] | ((uint32_t)h[1] << 16), (uint32_t)h[2] | ((uint32_t)h[3] << 16));
 }
 
+// The cast of one tensor as seen by block `rank` of the `nblk` blocks that share it.
 template <int FMT, bool AMAX>
-__global__ void __launch_bounds__(256) cast_flat_kernel(const uint4 *__restrict__ x, size_t n16,
-                                                        const uint16_t *__restrict__ tail_in,
-                                                        uint8_t *__restrict__ tail_out, int n_tail,
-                                                        const ScaleSrc scale_src,
-                                                        uint4 *__restrict__ out, unsigned int *__restrict__ amax_bits)
+__device__ __forceinline__ void cast_flat_body(const uint4 *__restrict__ x, size_t n16, const uint16_t *__restrict__ tail_in,
+                                               uint8_t *__restrict__ tail_out, int n_tail, const ScaleSrc &scale_src,
+                                               uint4 *__restrict__ out, unsigned int *__restrict__ amax_bits, unsigned rank,
+                                               unsigned nblk)
 {
-    const float s = resolve_scale(scale_src, blockIdx.x == 0 && threadIdx.x == 0);
+    const float s = resolve_scale(scale_src, rank == 0 && threadIdx.x == 0);
     uint32_t m = 0;
-    const size_t stride = (size_t)gridDim.x * blockDim.x;
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t stride = (size_t)nblk * blockDim.x;
+    size_t i = (size_t)rank * blockDim.x + threadIdx.x;
     // Back to front: the amax pass that precedes a just-in-time cast walked the tensor front to back, so its
     // tail is what the L2 still holds.
     if (n16 > 0) {
@@ -182,13 +216,43 @@ __global__ void __launch_bounds__(256) cast_flat_kernel(const uint4 *__restrict_
         const uint2 p0 = cast8<FMT>(a0, s), p1 = cast8<FMT>(a1, s);
         *(out - i) = make_uint4(p0.x, p0.y, p1.x, p1.y);
     }
-    if (blockIdx.x == 0 && (int)threadIdx.x < n_tail) {
+    if (rank == 0 && (int)threadIdx.x < n_tail) {
         const uint32_t w = tail_in[threadIdx.x];
         if (AMAX) m = absmax2(m, w);
         const float p = __fmul_rn(bf16_lo(w), s);
         tail_out[threadIdx.x] = (uint8_t)(cvt_f32x2_to_fp8x2<FMT>(p, 0.0f) & 0xFF);
     }
     if (AMAX) block_atomic_max_bf16(m, amax_bits);
+}
+
+template <int FMT, bool AMAX>
+__global__ void __launch_bounds__(256) cast_flat_kernel(const uint4 *__restrict__ x, size_t n16,
+                                                        const uint16_t *__restrict__ tail_in,
+                                                        uint8_t *__restrict__ tail_out, int n_tail,
+                                                        const ScaleSrc scale_src,
+                                                        uint4 *__restrict__ out, unsigned int *__restrict__ amax_bits)
+{
+    cast_flat_body<FMT, AMAX>(x, n16, tail_in, tail_out, n_tail, scale_src, out, amax_bits, blockIdx.x, gridDim.x);
+}
+
+// Just-in-time casts of several tensors in one launch: each takes its scale from the amax the reduction left in scalars.
+__global__ void __launch_bounds__(256) cast_multi_kernel(const MultiArgs a)
+{
+    int t = 0;
+    while (t + 1 < a.n_items && blockIdx.x >= a.it[t + 1].blk0) ++t;
+    const MultiItem &m = a.it[t];
+    const unsigned nblk = (t + 1 < a.n_items ? a.it[t + 1].blk0 : a.n_blocks) - m.blk0, rank = blockIdx.x - m.blk0;
+    const size_t n16 = m.n / 16;
+    const int n_tail = (int)(m.n - n16 * 16);
+    float *sc = a.scalars + 3 * t;
+    const ScaleSrc src{nullptr, sc, m.fmt == FP8_E4M3 ? 448.0f : 57344.0f, sc + 1, sc + 2};
+    const uint4 *x = reinterpret_cast<const uint4 *>(m.x);
+    if (m.fmt == FP8_E4M3)
+        cast_flat_body<0, false>(x, n16, m.x + n16 * 16, m.out + n16 * 16, n_tail, src, reinterpret_cast<uint4 *>(m.out),
+                                 nullptr, rank, nblk);
+    else
+        cast_flat_body<1, false>(x, n16, m.x + n16 * 16, m.out + n16 * 16, n_tail, src, reinterpret_cast<uint4 *>(m.out),
+                                 nullptr, rank, nblk);
 }
 
 // Cast + transposed copy: one CTA per 128 x 128 tile.  Codes go straight to `out` (16-byte stores) and
@@ -411,6 +475,75 @@ extern "C" int fp8_quantize(const void *x_bf16, size_t rows, size_t cols, int fm
     if (rc != FP8_OK) return rc;
     const ScaleSrc src{nullptr, amax, fmt == FP8_E4M3 ? 448.0f : 57344.0f, scale, scale_inv};
     return do_cast(x_bf16, rows, cols, src, fmt, out, out_t, nullptr, st);
+}
+
+extern "C" int fp8_quantize_multi(const fp8_quant_item *items, int n_items, float *scalars, void *stream)
+{
+    if (!items || !scalars) {
+        set_error("fp8_quantize_multi: NULL items / scalars");
+        return FP8_ERR_NULL;
+    }
+    if (n_items < 1 || n_items > MULTI_MAX) {
+        set_error("fp8_quantize_multi: n_items %d must be in [1, %d]", n_items, MULTI_MAX);
+        return FP8_ERR_SHAPE;
+    }
+    MultiArgs am, ac;
+    am.n_items = ac.n_items = n_items;
+    am.scalars = ac.scalars = scalars;
+    // the grids of the two passes: every tensor gets the blocks it would get alone, scaled down together at the cap
+    size_t want_a[MULTI_MAX], want_c[MULTI_MAX], tot_a = 0, tot_c = 0;
+    for (int t = 0; t < n_items; ++t) {
+        const fp8_quant_item &q = items[t];
+        if (!q.x_bf16 || !q.out) {
+            set_error("fp8_quantize_multi: NULL pointer in item %d", t);
+            return FP8_ERR_NULL;
+        }
+        if (q.fmt != FP8_E4M3 && q.fmt != FP8_E5M2) {
+            set_error("fp8_quantize_multi: item %d: fmt %d is not FP8_E4M3 / FP8_E5M2", t, q.fmt);
+            return FP8_ERR_ENUM;
+        }
+        if (q.n == 0) {
+            set_error("fp8_quantize_multi: item %d is empty", t);
+            return FP8_ERR_SHAPE;
+        }
+        if (!aligned16(q.x_bf16) || !aligned16(q.out)) {
+            set_error("fp8_quantize_multi: tensor pointers must be 16-byte aligned (item %d)", t);
+            return FP8_ERR_ALIGN;
+        }
+        am.it[t].x = ac.it[t].x = static_cast<const uint16_t *>(q.x_bf16);
+        am.it[t].out = ac.it[t].out = q.out;
+        am.it[t].n = ac.it[t].n = q.n;
+        am.it[t].fmt = ac.it[t].fmt = q.fmt;
+        want_a[t] = (q.n / 8 + 4 * 512 - 1) / (4 * 512);
+        want_c[t] = (q.n / 16 + 2 * 256 - 1) / (2 * 256);
+        if (want_a[t] == 0) want_a[t] = 1;
+        if (want_c[t] == 0) want_c[t] = 1;
+        tot_a += want_a[t];
+        tot_c += want_c[t];
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    const size_t cap_a = (size_t)sm_count() * 4, cap_c = (size_t)sm_count() * 8;
+    unsigned ba = 0, bc = 0;
+    for (int t = 0; t < n_items; ++t) {
+        size_t na = tot_a > cap_a ? want_a[t] * cap_a / tot_a : want_a[t];
+        size_t nc = tot_c > cap_c ? want_c[t] * cap_c / tot_c : want_c[t];
+        if (na == 0) na = 1;
+        if (nc == 0) nc = 1;
+        am.it[t].blk0 = ba;
+        ac.it[t].blk0 = bc;
+        ba += (unsigned)na;
+        bc += (unsigned)nc;
+    }
+    am.n_blocks = ba;
+    ac.n_blocks = bc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    FP8_CUDA_CHECK(cudaMemsetAsync(scalars, 0, 3 * sizeof(float) * (size_t)n_items, st));
+    amax_multi_kernel<<<ba, 512, 0, st>>>(am);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    cast_multi_kernel<<<bc, 256, 0, st>>>(ac);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
 }
 
 extern "C" int fp8_scale_update(float *history, int len, int *head, const float *amax_new, int fmt, int margin,

@@ -76,6 +76,15 @@ class QTensor:
         return self.x.numel() * 2
 
 
+def _share_scalars(*tensors):
+    """Puts the (amax, scale, 1 / scale) scalars of several QTensors side by side in one buffer, the layout
+    fp8_quantize_multi fills; every QTensor keeps its own one-element views."""
+    buf = torch.zeros(3 * len(tensors), dtype=torch.float32, device=tensors[0].x.device)
+    for i, t in enumerate(tensors):
+        t.amax, t.scale, t.scale_inv = buf[3 * i:3 * i + 1], buf[3 * i + 1:3 * i + 2], buf[3 * i + 2:3 * i + 3]
+    return buf
+
+
 @dataclass
 class Linear:
     name: str
@@ -88,6 +97,7 @@ class Linear:
     y: torch.Tensor = None
     dx: torch.Tensor = None
     dw: torch.Tensor = None
+    scalars: torch.Tensor = None       # the nine scaling scalars of x, w, dy side by side
 
     @property
     def flops(self):            # forward + dgrad + wgrad
@@ -101,15 +111,19 @@ class BlockHotPath:
     KERNELS_PER_ATTN_BWD = 3    # prep, main, finish
 
     def __init__(self, cfg: synth.BlockConfig, device="cuda", with_linears=None, with_attention=True,
-                 seq=None, batch=None, transposed_copies=False, attn_max_slack=0.0, scaling="jit"):
+                 seq=None, batch=None, transposed_copies=False, attn_max_slack=0.0, scaling="jit", multi_quantize=True):
         # transposed_copies: also write [cols, rows] FP8 copies in the cast and run dgrad / wgrad on them (the
         # form a K-major-only tensor core needs); off by default, tcgen05 reads the operands in place
         # attn_max_slack: tau of the attention forward's reference maximum (0 = exact running maximum); P~ is then
         # scaled by 448 / 2^tau
         # scaling: "jit" = amax pass, scale, cast pass per tensor and step (fp8_quantize); "delayed" = one cast pass under
         # the scale of the abs-max history, which the pass itself feeds (Appendix E; the recipe the paper trains with)
+        # multi_quantize: the just-in-time quantize of a group's tensors (x, w, dy of a projection; q, k, v, do) as one
+        # reduction launch and one cast launch for the group (fp8_quantize_multi) instead of two launches per tensor:
+        # the same codes and scales, fewer kernel boundaries
         assert scaling in ("jit", "delayed")
         self.scaling = scaling
+        self.multi_quantize = bool(multi_quantize)
         self.attn_max_slack = float(attn_max_slack)
         self.cfg = cfg
         self.device = torch.device(device)
@@ -151,6 +165,7 @@ class BlockHotPath:
                 lin.y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
                 lin.dx = torch.empty((T, K), dtype=torch.bfloat16, device=dev)
                 lin.dw = torch.empty((N, K), dtype=torch.bfloat16, device=dev)
+                lin.scalars = _share_scalars(lin.x, lin.w, lin.dy)
                 self.linears.append(lin)
         if self.with_attention:
             c = self.cfg
@@ -167,6 +182,7 @@ class BlockHotPath:
             a["ds_scale"] = _f32(dev, 1.0)
             a["ds_amax"] = _f32(dev)
             a["softmax_scale"] = float(d) ** -0.5
+            a["scalars"] = _share_scalars(a["q"], a["k"], a["v"], a["do"])
             self.attn = a
         return self
 
@@ -273,10 +289,19 @@ class BlockHotPath:
                                         self._host_ds_scale, True, h_out["o"], h_out["lse"], h_out["dq"], h_out["dk"],
                                         h_out["dv"], self._host_ws["attn"])
 
+    def _quantize_group(self, tensors, scalars):
+        """Quantize of the tensors of one group under the configured recipe."""
+        if self.scaling == "delayed":
+            for t in tensors:
+                t.quantize_delayed()
+        elif self.multi_quantize and not self.transposed_copies:
+            fp8.fp8_quantize_multi([t.x for t in tensors], [t.fmt for t in tensors], [t.q for t in tensors], scalars)
+        else:
+            for t in tensors:
+                t.quantize()
+
     def _run_linear(self, lin):
-        lin.x.quantize()
-        lin.w.quantize()
-        lin.dy.quantize()
+        self._quantize_group((lin.x, lin.w, lin.dy), lin.scalars)
         fp8.fp8_linear_fwd(lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
         if self.transposed_copies:
             fp8.fp8_linear_dgrad(lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
@@ -287,8 +312,7 @@ class BlockHotPath:
 
     def _run_attention(self):
         a = self.attn
-        for n in ("q", "k", "v", "do"):
-            a[n].quantize()
+        self._quantize_group([a[n] for n in ("q", "k", "v", "do")], a["scalars"])
         fp8.fp8_attention_fwd(a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv, a["v"].scale_inv,
                               a["softmax_scale"], True, a["o"], a["lse"], None,
                               p_scale=448.0 / 2.0 ** self.attn_max_slack, max_slack=self.attn_max_slack)
@@ -323,10 +347,11 @@ class BlockHotPath:
     def launches_per_step(self):
         n = 0
         kq = self.KERNELS_PER_QUANTIZE         # delayed scaling: cast (+amax) and the history update, also two
+        grouped = self.scaling == "jit" and self.multi_quantize and not self.transposed_copies
         for _ in self.linears:
-            n += 3 * kq + 3
+            n += (kq if grouped else 3 * kq) + 3       # one reduction + one cast for the group, or two per tensor
         if self.attn is not None:
-            n += 4 * kq + 1 + self.KERNELS_PER_ATTN_BWD
+            n += (kq if grouped else 4 * kq) + 1 + self.KERNELS_PER_ATTN_BWD
         return n
 
     # ------------------------------------------------------------------ the step
@@ -342,7 +367,7 @@ class BlockHotPath:
         torch.cuda.synchronize(self.device)
 
     def capture_graph(self):
-        """Captures one step (the same 48 launches) into a CUDA graph and returns it; ``graph.replay()`` then runs the
+        """Captures one step (the same launches) into a CUDA graph and returns it; ``graph.replay()`` then runs the
         step with one submission.  The step makes no host synchronisation, so it is capturable as it is.  Worth it
         where the step is launch-bound (small configurations); the large ones are bound by the kernels."""
         side = torch.cuda.Stream(self.device)
@@ -366,18 +391,15 @@ class BlockHotPath:
             self._qstream = torch.cuda.Stream(self.device)
         side = self._qstream
         side.wait_stream(main)              # the previous step's products have read the FP8 buffers about to be rewritten
-        quant = QTensor.quantize if self.scaling == "jit" else QTensor.quantize_delayed
         ready = []
         with torch.cuda.stream(side):
             for lin in self.linears:
-                for t in (lin.x, lin.w, lin.dy):
-                    quant(t)
+                self._quantize_group((lin.x, lin.w, lin.dy), lin.scalars)
                 ev = torch.cuda.Event()
                 ev.record(side)
                 ready.append(ev)
             if self.attn is not None:
-                for n in ("q", "k", "v", "do"):
-                    quant(self.attn[n])
+                self._quantize_group([self.attn[n] for n in ("q", "k", "v", "do")], self.attn["scalars"])
                 ev = torch.cuda.Event()
                 ev.record(side)
                 ready.append(ev)
@@ -433,10 +455,8 @@ class BlockHotPath:
         def gemm(fn, *args, **kw):
             timed(ev, fn, *args, **kw)
 
-        quant = QTensor.quantize if self.scaling == "jit" else QTensor.quantize_delayed
-
         for lin in self.linears:
-            timed(qev, lambda: [quant(t) for t in (lin.x, lin.w, lin.dy)])
+            timed(qev, self._quantize_group, (lin.x, lin.w, lin.dy), lin.scalars)
             gemm(fp8.fp8_linear_fwd, lin.x.q, lin.w.q, lin.x.scale_inv, lin.w.scale_inv, lin.y)
             if self.transposed_copies:
                 gemm(fp8.fp8_linear_dgrad, lin.dy.q, lin.w.qt, lin.dy.scale_inv, lin.w.scale_inv, lin.dx)
@@ -446,7 +466,7 @@ class BlockHotPath:
                 gemm(fp8.fp8_linear_wgrad_rm, lin.dy.q, lin.x.q, lin.dy.scale_inv, lin.x.scale_inv, lin.dw)
         if self.attn is not None:
             a = self.attn
-            timed(qev, lambda: [quant(a[n]) for n in ("q", "k", "v", "do")])
+            timed(qev, self._quantize_group, [a[n] for n in ("q", "k", "v", "do")], a["scalars"])
             timed(aev, fp8.fp8_attention_fwd, a["q"].q, a["k"].q, a["v"].q, a["q"].scale_inv, a["k"].scale_inv,
                   a["v"].scale_inv, a["softmax_scale"], True, a["o"], a["lse"], None,
                   p_scale=448.0 / 2.0 ** self.attn_max_slack, max_slack=self.attn_max_slack)

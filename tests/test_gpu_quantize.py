@@ -176,3 +176,34 @@ def test_bounded_wait_gives_up_and_reports():
     with pytest.raises(fp8.Fp8Error) as e:
         fp8.fp8_selftest_wait_timeout(0, flag)
     assert e.value.status == -3
+
+
+def test_quantize_multi_equals_per_tensor_quantize_and_oracle():
+    """fp8_quantize_multi (one reduction launch and one cast launch for a group of tensors) gives every tensor the codes
+    and the three scalars of its own fp8_quantize: sizes from 1 element to several blocks, ragged tails, both formats,
+    an all-zero tensor (scale 1), eight tensors (the maximum) and a single one."""
+    sizes = [1, 15, 16, 4096 + 7, 300_000, 1 << 20, (1 << 20) + 24, 2_500_000]
+    fmts = [fp8.E4M3, fp8.E5M2, fp8.E4M3, fp8.E5M2, fp8.E4M3, fp8.E4M3, fp8.E5M2, fp8.E4M3]
+    xs_host = [synth.flat_tensor(n, seed=40 + i) if n >= 16 else synth.normal_bf16((1, n), 40 + i, 0, 3.0).reshape(-1)
+               for i, n in enumerate(sizes)]
+    xs_host[4] = np.zeros(sizes[4], dtype=np.uint16)            # amax 0: scale 1
+    for take in (slice(0, 8), slice(3, 4), slice(4, 7)):
+        xs = [dev(x) for x in xs_host[take]]
+        f = fmts[take]
+        outs = [torch.full((x.numel(),), 0xAA, dtype=torch.uint8, device="cuda") for x in xs]
+        scal = torch.full((3 * len(xs),), -1.0, dtype=torch.float32, device="cuda")
+        fp8.fp8_quantize_multi(xs, f, outs, scal)
+        torch.cuda.synchronize()
+        sc = scal.cpu().numpy()
+        for i, (x, xh, fmt, out) in enumerate(zip(xs, xs_host[take], f, outs)):
+            q = torch.empty(x.numel(), dtype=torch.uint8, device="cuda")
+            a, s_, si = scalar(), scalar(), scalar()
+            fp8.fp8_quantize(x.reshape(1, -1), fmt, q, None, a, s_, si)
+            assert torch.equal(out, q), i
+            assert sc[3 * i] == a.item() and sc[3 * i + 1] == s_.item() and sc[3 * i + 2] == si.item(), i
+            oc, oa, osc, osi = o.quantize(xh.reshape(1, -1), fmt)
+            assert np.array_equal(out.cpu().numpy(), oc.reshape(-1)), i
+            assert np.float32(sc[3 * i]) == np.float32(oa) and np.float32(sc[3 * i + 1]) == np.float32(osc), i
+    with pytest.raises(fp8.Fp8Error):
+        fp8.fp8_quantize_multi([dev(xs_host[2])] * 9, [fp8.E4M3] * 9, [torch.empty(16, dtype=torch.uint8, device="cuda")] * 9,
+                               torch.empty(27, device="cuda"))
