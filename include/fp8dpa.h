@@ -370,12 +370,12 @@ FP8_API int fp8_attention_bwd_static(const uint8_t *Q8, const uint8_t *K8, const
  * (No counterpart in the paper: packaging of the calls above for a caller whose tensors live in HOST memory.)
  *
  * fp8_linear_step_host: one linear layer's training step (Appendix E, throughput table) from BF16 HOST tensors
- * X[T,K], W[N,K], dY[T,N] to BF16 HOST tensors Y[T,N], dX[T,K], dW[N,K]: upload, fp8_quantize of X and W
+ * X[T,K], W[N,K], dY[T,N] to BF16 HOST tensors Y[T,N], dX[T,K], dW[N,K]: upload, fp8_quantize_multi of X and W
  * (E4M3) and dY (E5M2) with just-in-time scales, fp8_linear_fwd, fp8_linear_dgrad_rm, fp8_linear_wgrad_rm,
  * download.  T, N, K multiples of 16.
  * fp8_attention_step_host: one attention's training step (Appendix B, Eq. (P)) from BF16 HOST tensors
  * Q, dO [B,N,Hq,d] and K, V [B,N,Hkv,d] to HOST O, dQ [B,N,Hq,d] (BF16), LSE [B,Hq,N] (FP32) and
- * dK, dV [B,N,Hkv,d] (BF16): upload, fp8_quantize of Q, K, V (E4M3) and dO (E5M2), fp8_attention_fwd with
+ * dK, dV [B,N,Hkv,d] (BF16): upload, fp8_quantize_multi of Q, K, V (E4M3) and dO (E5M2), fp8_attention_fwd with
  * p_scale = 448 and max_slack = 0, fp8_attention_bwd with the given ds_scale (a host value), download.
  * Results are bit-identical to the same chain of device-pointer calls.
  *

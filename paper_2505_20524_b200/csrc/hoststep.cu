@@ -137,9 +137,10 @@ extern "C" int fp8_linear_step_host(const void *hX, const void *hW, const void *
     FP8_CUDA_CHECK(cudaStreamWaitEvent(c->main, up_done, 0));
     FP8_CUDA_CHECK(cudaEventDestroy(up_done));                  // released once the wait has consumed it
     // amax, scale, scale_inv of x, w, dy
-    rc = fp8_quantize(x, (size_t)T, (size_t)K, FP8_E4M3, x8, nullptr, sc + 0, sc + 1, sc + 2, c->main);
-    if (rc == FP8_OK) rc = fp8_quantize(w, (size_t)N, (size_t)K, FP8_E4M3, w8, nullptr, sc + 3, sc + 4, sc + 5, c->main);
-    if (rc == FP8_OK) rc = fp8_quantize(dy, (size_t)T, (size_t)N, FP8_E5M2, dy8, nullptr, sc + 6, sc + 7, sc + 8, c->main);
+    {
+        const fp8_quant_item items[3] = {{x, tk, FP8_E4M3, x8}, {w, nk, FP8_E4M3, w8}, {dy, tn, FP8_E5M2, dy8}};
+        rc = fp8_quantize_multi(items, 3, sc, c->main);
+    }
     if (rc == FP8_OK) rc = fp8_linear_fwd(x8, w8, sc + 2, sc + 5, y, 0, T, N, K, nullptr, 0, c->main);
     if (rc == FP8_OK) rc = fp8_linear_dgrad_rm(dy8, w8, sc + 8, sc + 5, dx, 0, T, N, K, c->main);
     if (rc == FP8_OK) rc = fp8_linear_wgrad_rm(dy8, x8, sc + 8, sc + 2, dw, 0, 0, T, N, K, c->main);
@@ -211,11 +212,10 @@ extern "C" int fp8_attention_step_host(const void *hQ, const void *hK, const voi
     FP8_CUDA_CHECK(cudaStreamWaitEvent(c->main, up_done, 0));
     FP8_CUDA_CHECK(cudaEventDestroy(up_done));
     // scalars: (amax, scale, scale_inv) of q, k, v, do; then ds_scale and ds_amax
-    const size_t rows = (size_t)B * N;
-    rc = fp8_quantize(q, rows, (size_t)Hq * d, FP8_E4M3, q8, nullptr, sc + 0, sc + 1, sc + 2, c->main);
-    if (rc == FP8_OK) rc = fp8_quantize(k, rows, (size_t)Hkv * d, FP8_E4M3, k8, nullptr, sc + 3, sc + 4, sc + 5, c->main);
-    if (rc == FP8_OK) rc = fp8_quantize(v, rows, (size_t)Hkv * d, FP8_E4M3, v8, nullptr, sc + 6, sc + 7, sc + 8, c->main);
-    if (rc == FP8_OK) rc = fp8_quantize(dO, rows, (size_t)Hq * d, FP8_E5M2, do8, nullptr, sc + 9, sc + 10, sc + 11, c->main);
+    {
+        const fp8_quant_item items[4] = {{q, nq, FP8_E4M3, q8}, {k, nkv, FP8_E4M3, k8}, {v, nkv, FP8_E4M3, v8}, {dO, nq, FP8_E5M2, do8}};
+        rc = fp8_quantize_multi(items, 4, sc, c->main);
+    }
     if (rc != FP8_OK) return rc;
     set_scalar_kernel<<<1, 1, 0, c->main>>>(sc + 12, ds_scale);
     FP8_CUDA_CHECK(cudaGetLastError());
