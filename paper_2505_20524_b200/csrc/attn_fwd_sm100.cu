@@ -1319,15 +1319,16 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             };
             const int k_last = (n_kv - 1) * A_BN;
             const bool last_masked = (k_last + A_BN - 1 > qs && p.causal) || (k_last + A_BN > p.N);
-            // this warpgroup's blocks of the item: G = gbase + j with G % NWG == w
-            for (int j = (int)(((uint32_t)w + (uint32_t)NWG - gbase % (uint32_t)NWG) % (uint32_t)NWG); j < n_kv && ok; j += NWG) {
-                if (NWG == 2) {
-                    if (j == n_kv - 1 && last_masked) ok = block(std::true_type{}, j);
-                    else ok = block(std::false_type{}, j);
-                } else {
-                    if (j == n_kv - 1 && last_masked) ok = block3(std::true_type{}, j);
-                    else ok = block3(std::false_type{}, j);
-                }
+            // this warpgroup's blocks of the item: G = gbase + j with G % NWG == w.  Only the item's last block can need the
+            // mask; it runs after the loop, so that the loop holds one instance of the block code
+            const int n_plain = last_masked ? n_kv - 1 : n_kv;
+            int j = (int)(((uint32_t)w + (uint32_t)NWG - gbase % (uint32_t)NWG) % (uint32_t)NWG);
+            if (NWG == 2) {
+                for (; j < n_plain && ok; j += NWG) ok = block(std::false_type{}, j);
+                if (ok && j == n_kv - 1 && last_masked) ok = block(std::true_type{}, j);
+            } else {
+                for (; j < n_plain && ok; j += NWG) ok = block3(std::false_type{}, j);
+                if (ok && j == n_kv - 1 && last_masked) ok = block3(std::true_type{}, j);
             }
             if (!ok) break;
             // the epilogue of the previous item has read the row sums
