@@ -882,7 +882,7 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 //               publishes its own and the factor 2^(m(G-1) - m(G)) for the accumulator, evaluates the exponentials, stores
 //               P8(G) over the first 32 columns of S(G).  NWG = 2: the score row sits in registers (184 per thread), the
 //               published value is the block maximum and m(G-1) follows from it and the warpgroup's own m(G-2).  NWG = 3:
-//               the row stays in TMEM and is read twice in chunks of 32 columns (112 registers per thread), the
+//               the row stays in TMEM and is read twice in chunks of 32 columns (96 registers per thread, the launch allocation), the
 //               published value is the running maximum.  Each warpgroup keeps the row sum of its own blocks with its own
 //               reference maximum; the epilogue merges them
 //   next 4 warps  correction: rescales O when the running maximum grew (after PV(G-1) has completed), lets PV(G) go;
@@ -899,11 +899,21 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 // ---------------------------------------------------------------------------------------------------------------
 // NWG softmax warpgroups.  2: one row of 128 scores per thread held in registers (184 registers).  3: blocks G % 3, every
 // warpgroup with a score buffer of its own; the row stays in TMEM and is read twice in chunks of 32 columns (maximum, then
-// exponentials), which fits 112 registers; a warpgroup's next scores are issued when its P8 has been consumed, and the
-// other two warpgroups cover that round trip.
+// exponentials), which fits the 96 registers every thread of a 640-thread CTA gets at launch, so this form moves no
+// registers between warpgroups (measured: 112 / 80 / 64 after setmaxnreg 1.49 ms at N = 16384, 104 / 88 / 80 1.475, 96 for all 1.47;
+// 120 / 64 / 56 and 112 / 72 / 72 1.97 and 1.61: the correction warps must not go short); a warpgroup's next scores are issued when
+// its P8 has been consumed, and the other two warpgroups cover that round trip.
+// setmaxnreg for a warpgroup: an increase or a release relative to the allocation at launch, nothing when equal (a release
+// to a larger count is not a valid instruction).
+template <int TARGET, int LAUNCH>
+__device__ __forceinline__ void set_registers()
+{
+    if (TARGET > LAUNCH) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(TARGET));
+    else if (TARGET < LAUNCH) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(TARGET));
+}
 template <int NWG> struct XCfg;
 template <> struct XCfg<2> { static constexpr int THREADS = 512, LAUNCH = 128, SOFTMAX = 184, CORR = 80, CTRL = 64; };
-template <> struct XCfg<3> { static constexpr int THREADS = 640, LAUNCH = 96, SOFTMAX = 112, CORR = 80, CTRL = 64; };
+template <> struct XCfg<3> { static constexpr int THREADS = 640, LAUNCH = 96, SOFTMAX = 96, CORR = 96, CTRL = 96; };
 static_assert(2 * 128 * XCfg<2>::SOFTMAX + 128 * XCfg<2>::CORR + 128 * XCfg<2>::CTRL <= XCfg<2>::THREADS * XCfg<2>::LAUNCH, "register budget");
 static_assert(3 * 128 * XCfg<3>::SOFTMAX + 128 * XCfg<3>::CORR + 128 * XCfg<3>::CTRL <= XCfg<3>::THREADS * XCfg<3>::LAUNCH, "register budget");
 constexpr int X_KS = 4, X_VS = 4;
@@ -1042,7 +1052,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     it.init();
 
     if (warp >= W_TMA) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(XCfg<NWG>::CTRL));
+        set_registers<XCfg<NWG>::CTRL, XCfg<NWG>::LAUNCH>();
         if (warp == W_TMA) {
             // ------------------------------------------------------------ TMA producer
             if (elect_one()) {
@@ -1159,7 +1169,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
     }
     else if (warp < W_CORR) {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(XCfg<NWG>::SOFTMAX));
+        set_registers<XCfg<NWG>::SOFTMAX, XCfg<NWG>::LAUNCH>();
         // ------------------------------------------------------------ softmax warpgroup w: blocks G with (G & 1) == w
         const int w = warp >> 2, quad = warp & 3;
         const int r = quad * 32 + lane;
@@ -1341,7 +1351,7 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             ++n_it;
         }
     } else if (warp < W_TMA) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(XCfg<NWG>::CORR));
+        set_registers<XCfg<NWG>::CORR, XCfg<NWG>::LAUNCH>();
         // ------------------------------------------------------------ correction and epilogue
         const int quad = warp & 3;
         const int r = quad * 32 + lane;
