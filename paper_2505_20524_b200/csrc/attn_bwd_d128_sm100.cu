@@ -38,7 +38,10 @@ constexpr int QT = 64;             // queries per sub-tile
 constexpr int STAGES = 5;          // (Q, dO, lse2, db) stages: a TMA load takes several sub-tile periods to land
 constexpr int THREADS = 16 * 32;     // four warpgroups: control (TMA, MMA), two element-wise groups, dQ drain
 constexpr int DRAIN_WARPS = 4;
-constexpr int REGS_CTRL = 64, REGS_EW = 176, REGS_DRAIN = 88;   // per thread after setmaxnreg; sum <= 4 * 128
+// per thread after setmaxnreg (splits of 56/176/104, 80/168/96, 96/160/96 measured the same within 0.5%; those that spill lose 2-4%)
+constexpr int REGS_CTRL = 64, REGS_EW = 176, REGS_DRAIN = 88;
+static_assert(REGS_CTRL + 2 * REGS_EW + REGS_DRAIN <= 4 * 128 && REGS_CTRL <= 128 && REGS_DRAIN <= 128 && REGS_EW >= 128,
+              "register hand-over: releases must cover the increases inside the 512 x 128 of the launch");
 constexpr int TMEM_COLS = 512;
 
 struct Smem {
