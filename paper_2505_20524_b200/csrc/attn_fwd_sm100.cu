@@ -1415,26 +1415,14 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const float inv = __ldg(p.v_inv) / lt;                 // lt already carries c_P
             if (row < p.N)
                 p.LSE[((size_t)it.b * p.Hq + it.h) * p.N + row] = (mf + log2f(lt) - p.log2_p_scale) * 0.69314718055994531f;
-            uint8_t *o8row = p.O8 + (((size_t)it.b * p.N + row) * p.Hq + it.h) * D;
-            const float o_scale = p.o_scale ? __ldg(p.o_scale) : 1.0f;
             // the previous item's stores have read this warp's rows of the staging tile
             if (stored) {
                 if (lane == 0) bulk_wait_group_read0();
                 __syncwarp();
             }
-            uint32_t amax2 = 0;
-#pragma unroll 1
-            for (int cc = 0; cc < D; cc += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32b_x32(to + (uint32_t)cc, v);
-                tmem_ld_wait();
-                if (cc == D - 32) {
-                    // O and the row sums have been read: the next item may overwrite them
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(epi_done);
-                }
-                // staging tile of 64 columns: [128 rows x 128 bytes], 128-byte swizzle
+            // 32 accumulator columns of this thread's row -> BF16 into the staging tile (64 columns per tile: [128 rows x 128
+            // bytes], 128-byte swizzle)
+            auto emit32 = [&](const uint32_t (&v)[32], const int cc) {
                 uint8_t *trow = smem + L::OST_OFF + (cc < 64 ? 0 : L::TILE_BYTES) + r * 128;
                 const int c0 = (cc & 63) >> 3;
 #pragma unroll
@@ -1445,17 +1433,58 @@ attn_fwd_stream_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     o.z = pack_bf16x2(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
                     o.w = pack_bf16x2(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
                     *reinterpret_cast<uint4 *>(trow + (((c0 + (e >> 3)) ^ (r & 7)) << 4)) = o;
-                    if (p.o_scale && row < p.N) {
-                        amax2 = __vmaxu2(__vmaxu2(__vmaxu2(__vmaxu2(amax2, o.x & 0x7FFF7FFFu), o.y & 0x7FFF7FFFu),
-                                                  o.z & 0x7FFF7FFFu), o.w & 0x7FFF7FFFu);
-                        const uint32_t e0 = cvt_f32x4_to_fp8x4<0>(
-                            __fmul_rn(bf16_lo(o.x), o_scale), __fmul_rn(bf16_hi(o.x), o_scale),
-                            __fmul_rn(bf16_lo(o.y), o_scale), __fmul_rn(bf16_hi(o.y), o_scale));
-                        const uint32_t e1 = cvt_f32x4_to_fp8x4<0>(
-                            __fmul_rn(bf16_lo(o.z), o_scale), __fmul_rn(bf16_hi(o.z), o_scale),
-                            __fmul_rn(bf16_lo(o.w), o_scale), __fmul_rn(bf16_hi(o.w), o_scale));
-                        *reinterpret_cast<uint2 *>(o8row + cc + e) = make_uint2(e0, e1);
+                }
+            };
+            if (XCfg<NWG>::CORR >= 96) {
+                // the next item's first PV waits for these reads: two loads in flight, the last pair requested early
+                uint32_t va[32], vb[32];
+                tmem_ld_32x32b_x32(to, va);
+                tmem_ld_32x32b_x32(to + 32u, vb);
+                tmem_ld_wait();
+                emit32(va, 0);
+                tmem_ld_32x32b_x32(to + 64u, va);
+                emit32(vb, 32);
+                tmem_ld_32x32b_x32(to + 96u, vb);
+                tmem_ld_wait();
+                // O and the row sums have been read: the next item may overwrite them
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(epi_done);
+                emit32(va, 64);
+                emit32(vb, 96);
+            } else {
+                // (80 registers: one buffer; two would spill and cost more than the overlap returns)
+#pragma unroll 1
+                for (int cc = 0; cc < D; cc += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32x32b_x32(to + (uint32_t)cc, v);
+                    tmem_ld_wait();
+                    if (cc == D - 32) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(epi_done);
                     }
+                    emit32(v, cc);
+                }
+            }
+            // the FP8 copy of the producer form and its amax, from this thread's own row of the staging tile
+            uint32_t amax2 = 0;
+            if (p.o_scale && row < p.N) {
+                uint8_t *o8row = p.O8 + (((size_t)it.b * p.N + row) * p.Hq + it.h) * D;
+                const float o_scale = __ldg(p.o_scale);
+#pragma unroll 4
+                for (int ch = 0; ch < 16; ++ch) {
+                    const uint8_t *trow = smem + L::OST_OFF + (ch < 8 ? 0 : L::TILE_BYTES) + r * 128;
+                    const uint4 o = *reinterpret_cast<const uint4 *>(trow + (((ch & 7) ^ (r & 7)) << 4));
+                    amax2 = __vmaxu2(__vmaxu2(__vmaxu2(__vmaxu2(amax2, o.x & 0x7FFF7FFFu), o.y & 0x7FFF7FFFu),
+                                              o.z & 0x7FFF7FFFu), o.w & 0x7FFF7FFFu);
+                    const uint32_t e0 = cvt_f32x4_to_fp8x4<0>(
+                        __fmul_rn(bf16_lo(o.x), o_scale), __fmul_rn(bf16_hi(o.x), o_scale),
+                        __fmul_rn(bf16_lo(o.y), o_scale), __fmul_rn(bf16_hi(o.y), o_scale));
+                    const uint32_t e1 = cvt_f32x4_to_fp8x4<0>(
+                        __fmul_rn(bf16_lo(o.z), o_scale), __fmul_rn(bf16_hi(o.z), o_scale),
+                        __fmul_rn(bf16_lo(o.w), o_scale), __fmul_rn(bf16_hi(o.w), o_scale));
+                    *reinterpret_cast<uint2 *>(o8row + ch * 8) = make_uint2(e0, e1);
                 }
             }
             if (p.o_scale && p.o_amax_bits) {
