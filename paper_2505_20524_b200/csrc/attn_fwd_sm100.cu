@@ -899,8 +899,8 @@ attn_fwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 // ---------------------------------------------------------------------------------------------------------------
 // NWG softmax warpgroups.  2: one row of 128 scores per thread held in registers (184 registers).  3: blocks G % 3, every
 // warpgroup with a score buffer of its own; the row stays in TMEM and is read twice in chunks of 32 columns (maximum, then
-// exponentials), which fits the 96 registers every thread of a 640-thread CTA gets at launch, so this form moves no
-// registers between warpgroups (measured: 112 / 80 / 64 after setmaxnreg 1.49 ms at N = 16384, 104 / 88 / 80 1.475, 96 for all 1.47;
+// exponentials), which fits the 96 registers a thread gets when a scheduler holds five warps (18 warps: 12 softmax, 4
+// correction, producer, issuer), so this form moves no registers between warpgroups (measured: 112 / 80 / 64 after setmaxnreg 1.49 ms at N = 16384, 104 / 88 / 80 1.475, 96 for all 1.47;
 // 120 / 64 / 56 and 112 / 72 / 72 1.97 and 1.61: the correction warps must not go short); a warpgroup's next scores are issued when
 // its P8 has been consumed, and the other two warpgroups cover that round trip.
 // setmaxnreg for a warpgroup: an increase or a release relative to the allocation at launch, nothing when equal (a release
@@ -913,9 +913,10 @@ __device__ __forceinline__ void set_registers()
 }
 template <int NWG> struct XCfg;
 template <> struct XCfg<2> { static constexpr int THREADS = 512, LAUNCH = 128, SOFTMAX = 184, CORR = 80, CTRL = 64; };
-template <> struct XCfg<3> { static constexpr int THREADS = 640, LAUNCH = 96, SOFTMAX = 96, CORR = 96, CTRL = 96; };
+template <> struct XCfg<3> { static constexpr int THREADS = 576, LAUNCH = 112, SOFTMAX = 112, CORR = 112, CTRL = 112; };
 static_assert(2 * 128 * XCfg<2>::SOFTMAX + 128 * XCfg<2>::CORR + 128 * XCfg<2>::CTRL <= XCfg<2>::THREADS * XCfg<2>::LAUNCH, "register budget");
-static_assert(3 * 128 * XCfg<3>::SOFTMAX + 128 * XCfg<3>::CORR + 128 * XCfg<3>::CTRL <= XCfg<3>::THREADS * XCfg<3>::LAUNCH, "register budget");
+static_assert(XCfg<3>::SOFTMAX == XCfg<3>::LAUNCH && XCfg<3>::CORR == XCfg<3>::LAUNCH && XCfg<3>::CTRL == XCfg<3>::LAUNCH,
+              "no register hand-over in the three-warpgroup form (its 18 warps are not a whole number of warpgroups)");
 constexpr int X_KS = 4, X_VS = 4;
 
 struct AttnFwdStreamSmem {
@@ -1608,8 +1609,10 @@ static int launch_attn_fwd_stream(const uint8_t *Q8, const uint8_t *K8, const ui
     if (rc != FP8_OK) return rc;
     FP8_CUDA_CHECK(cudaFuncSetAttribute(attn_fwd_stream_kernel<NWG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         AttnFwdStreamSmem::DYN_BYTES));
-    rc = check_launch_registers(attn_fwd_stream_kernel<NWG>, XCfg<NWG>::LAUNCH, "attn_fwd_stream_kernel");
-    if (rc != FP8_OK) return rc;
+    if (XCfg<NWG>::SOFTMAX != XCfg<NWG>::LAUNCH) {          // only the form that hands registers over depends on the allocation
+        rc = check_launch_registers(attn_fwd_stream_kernel<NWG>, XCfg<NWG>::LAUNCH, "attn_fwd_stream_kernel");
+        if (rc != FP8_OK) return rc;
+    }
     const long long n_items = (long long)((p.N + 127) / 128) * p.Hq * p.B;
     const int sms = sm_count();
     if (sms <= 0) return FP8_ERR_CUDA;
