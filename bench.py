@@ -237,9 +237,10 @@ def quantize_sweep(peaks):
 
 def delayed_scaling_step(cfg, host, args, flops_step):
     """The same step under delayed scaling (Appendix E, the recipe the paper trains with): every tensor is cast in one
-    pass under the scale of its abs-max history (length 1024), the pass records the new abs-max and a small kernel
-    updates history and scale for the next step.  Same inputs, same products and attention; the headline `value`
-    stays the just-in-time form."""
+    pass under the scale of its abs-max history (length 1024), the pass records the new abs-max and the last block to
+    finish a tensor updates history and scale for the next step (one launch per group of operands:
+    fp8_quantize_delayed_multi).  Same inputs, same products and attention; the headline `value` stays the
+    just-in-time form."""
     import torch
     from paper_2505_20524_b200.hotpath import BlockHotPath
     hp = BlockHotPath(cfg, attn_max_slack=args.attn_slack, scaling="delayed")
@@ -667,6 +668,21 @@ def run_report(args):
     a, sc, si = f32(), f32(1.0), f32(1.0)
     add("fp8_quantize e5m2 + transposed copy", f"{T}x{2 * F}",
         timed(lambda: fp8.fp8_quantize(x, fp8.E5M2, q, qt, a, sc, si)), nbytes=6 * T * 2 * F)
+    # the operands of the c4 QKV projection as one group: X [T,H], W [3H/2,H], dY [T,3H/2]
+    gx = [bf16(T, H), bf16(3 * H // 2, H), bf16(T, 3 * H // 2)]
+    gf = [fp8.E4M3, fp8.E4M3, fp8.E5M2]
+    gq = [torch.empty(t.shape, dtype=torch.uint8, device="cuda") for t in gx]
+    gn = sum(t.numel() for t in gx)
+    gsc = torch.zeros(9, dtype=torch.float32, device="cuda")
+    add("fp8_quantize_multi (X, W, dY of the QKV projection; two launches)", f"{gn}",
+        timed(lambda: fp8.fp8_quantize_multi(gx, gf, gq, gsc)), nbytes=5 * gn)
+    gh = [torch.zeros(1024, dtype=torch.float32, device="cuda") for _ in gx]
+    ghd = [torch.zeros(1, dtype=torch.int32, device="cuda") for _ in gx]
+    gs, ga, gs1, gsi1 = [f32(1.0) for _ in gx], [f32() for _ in gx], [f32() for _ in gx], [f32() for _ in gx]
+    gsync = torch.zeros(6, dtype=torch.int32, device="cuda")
+    add("fp8_quantize_delayed_multi (same group: codes, amax, history update, next scale; one launch)", f"{gn}",
+        timed(lambda: fp8.fp8_quantize_delayed_multi(gx, gf, gq, gh, ghd, gs, ga, gs1, gsi1, 0, gsync)), nbytes=3 * gn)
+    del gx, gq
     h8, h8t = torch.empty((T, F), dtype=torch.uint8, device="cuda"), torch.empty((F, T), dtype=torch.uint8, device="cuda")
     add("fp8_swiglu_cast (amax pass)", f"{T}x{F}", timed(lambda: fp8.fp8_swiglu_cast(x, None, 0, None, None, a)),
         nbytes=4 * T * F)

@@ -13,6 +13,6 @@ from .binding import (ACT_GELU, ACT_XIELU, E4M3, E5M2, FP8_BLOCK_128x1, NORM_LAY
                       fp8_linear_dgrad_q, fp8_linear_dgrad_rm, fp8_linear_fwd, fp8_linear_fwd_blockwise,
                       fp8_linear_dgrad_blockwise, fp8_linear_wgrad_blockwise,
                       fp8_linear_fwd_q, fp8_linear_wgrad, fp8_linear_wgrad_rm, fp8_postnorm_residual, fp8_postnorm_residual_q,
-                      fp8_qk_norm_rope, fp8_qk_norm_rope_q, fp8_quantize, fp8_quantize_multi, fp8_quantize_blockwise, fp8_scale, fp8_scale_update,
+                      fp8_qk_norm_rope, fp8_qk_norm_rope_q, fp8_quantize, fp8_quantize_multi, fp8_quantize_delayed_multi, fp8_quantize_blockwise, fp8_scale, fp8_scale_update,
                       fp8_selftest_wait_timeout, fp8_swiglu_cast, fp8_linear_step_host, fp8_linear_step_host_workspace_bytes,
                       fp8_attention_step_host, fp8_attention_step_host_workspace_bytes, fp8_host_sync)

@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "csrc", "libfp8dpa.so")
 _lib = None
 
 SYMBOLS = ["fp8_last_error", "fp8_device_status", "fp8_selftest_wait_timeout", "fp8_amax", "fp8_scale", "fp8_scale_update", "fp8_cast",
-           "fp8_quantize", "fp8_quantize_multi", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis", "fp8_amax_kurtosis",
+           "fp8_quantize", "fp8_quantize_multi", "fp8_quantize_delayed_multi", "fp8_swiglu_cast", "fp8_act_cast", "fp8_postnorm_residual", "fp8_postnorm_residual_q", "fp8_qk_norm_rope", "fp8_qk_norm_rope_q", "fp8_kurtosis", "fp8_amax_kurtosis",
            "fp8_linear_fwd", "fp8_linear_dgrad", "fp8_linear_wgrad", "fp8_linear_fwd_q", "fp8_linear_dgrad_q", "fp8_linear_dgrad_rm", "fp8_linear_wgrad_rm", "fp8_grouped_linear_fwd", "fp8_grouped_linear_dgrad", "fp8_grouped_linear_wgrad", "fp8_grouped_linear_wgrad_workspace_bytes", "fp8_grouped_linear_wgrad_dev", "fp8_quantize_blockwise", "fp8_linear_fwd_blockwise", "fp8_linear_dgrad_blockwise", "fp8_linear_wgrad_blockwise", "fp8_attention_workspace_bytes",
            "fp8_attention_fwd", "fp8_attention_fwd_q", "fp8_attention_bwd", "fp8_attention_bwd_static",
            "fp8_linear_step_host_workspace_bytes", "fp8_linear_step_host", "fp8_attention_step_host_workspace_bytes",
@@ -146,6 +146,30 @@ def fp8_quantize_multi(xs, fmts, outs, scalars, stream=None):
     for i, (x, f, o) in enumerate(zip(xs, fmts, outs)):
         items[i] = QuantItem(_ptr(x).value, x.numel(), int(f), _ptr(o).value)
     _check(load().fp8_quantize_multi(items, C.c_int(n), _ptr(scalars), _stream(stream)))
+
+
+class DelayedItem(C.Structure):
+    _fields_ = [("x_bf16", C.c_void_p), ("n", C.c_size_t), ("fmt", C.c_int), ("out", C.c_void_p),
+                ("history", C.c_void_p), ("head", C.c_void_p), ("scale", C.c_void_p), ("amax", C.c_void_p),
+                ("scale_next", C.c_void_p), ("scale_inv_next", C.c_void_p)]
+
+
+def fp8_quantize_delayed_multi(xs, fmts, outs, histories, heads, scales, amaxes, scales_next, scales_inv_next, margin,
+                               sync, stream=None):
+    """Delayed-scaling quantize of up to 8 tensors in one launch (cast under `scales`, amax, history update and the next
+    step's scale): lists of CUDA tensors, one entry per tensor; all histories have the same length; sync an int32 /
+    uint32 CUDA tensor of 2 * len(xs) words that is zero before the first call."""
+    n = len(xs)
+    assert all(len(v) == n for v in (fmts, outs, histories, heads, scales, amaxes, scales_next, scales_inv_next))
+    assert sync.numel() >= 2 * n and sync.element_size() == 4
+    assert all(h.numel() == histories[0].numel() for h in histories)
+    items = (DelayedItem * n)()
+    for i in range(n):
+        items[i] = DelayedItem(_ptr(xs[i]).value, xs[i].numel(), int(fmts[i]), _ptr(outs[i]).value,
+                               _ptr(histories[i]).value, _ptr(heads[i]).value, _ptr(scales[i]).value,
+                               _ptr(amaxes[i]).value, _ptr(scales_next[i]).value, _ptr(scales_inv_next[i]).value)
+    _check(load().fp8_quantize_delayed_multi(items, C.c_int(n), C.c_int(histories[0].numel()), C.c_int(margin),
+                                             _ptr(sync), _stream(stream)))
 
 
 ACT_GELU, ACT_XIELU = 1, 2

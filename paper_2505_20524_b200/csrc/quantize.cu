@@ -124,17 +124,16 @@ __device__ __forceinline__ float resolve_scale(const ScaleSrc &src, bool first_t
 }
 
 // ---------------------------------------------------------------- delayed scaling: history ring update
-// One CTA: insert the new amax at the position of the oldest entry, then scale = FP8Max / (2^m max H).
-__global__ void __launch_bounds__(256) scale_update_kernel(float *__restrict__ history, int len, int *__restrict__ head,
-                                                           const float *__restrict__ amax_new, float fp8_max,
-                                                           int margin, float *__restrict__ scale,
-                                                           float *__restrict__ scale_inv)
+// One CTA (256 threads): insert the new amax at the position of the oldest entry, then scale = FP8Max / (2^m max H).
+__device__ __forceinline__ void ring_update_body(float *__restrict__ history, int len, int *__restrict__ head,
+                                                 float amax_new, float fp8_max, int margin, float *__restrict__ scale,
+                                                 float *__restrict__ scale_inv)
 {
     __shared__ float warp_max[8];
     __shared__ int s_nan;
     if (threadIdx.x == 0) {
         const int h = *head;
-        history[h] = *amax_new;
+        history[h] = amax_new;
         *head = (h + 1) % len;
         s_nan = 0;
     }
@@ -161,6 +160,14 @@ __global__ void __launch_bounds__(256) scale_update_kernel(float *__restrict__ h
         *scale = s;
         *scale_inv = __fdiv_rn(1.0f, s);
     }
+}
+
+__global__ void __launch_bounds__(256) scale_update_kernel(float *__restrict__ history, int len, int *__restrict__ head,
+                                                           const float *__restrict__ amax_new, float fp8_max,
+                                                           int margin, float *__restrict__ scale,
+                                                           float *__restrict__ scale_inv)
+{
+    ring_update_body(history, len, head, *amax_new, fp8_max, margin, scale, scale_inv);
 }
 
 // ---------------------------------------------------------------- cast
@@ -253,6 +260,66 @@ __global__ void __launch_bounds__(256) cast_multi_kernel(const MultiArgs a)
     else
         cast_flat_body<1, false>(x, n16, m.x + n16 * 16, m.out + n16 * 16, n_tail, src, reinterpret_cast<uint4 *>(m.out),
                                  nullptr, rank, nblk);
+}
+
+// Delayed scaling of several tensors in ONE launch: every tensor is cast under the scale its history gave after the
+// previous step while the same pass takes its amax; the last block of a tensor to finish (a counter per tensor) then
+// does that tensor's ring update and writes the scale of the next step.  sync[2 t] collects the amax bits, sync[2 t + 1]
+// counts finished blocks; the last block leaves both at zero for the next call.
+struct DelayedItem {
+    const uint16_t *x;
+    uint8_t *out;
+    size_t n;
+    int fmt;
+    unsigned blk0;
+    float *history;
+    int *head;
+    const float *scale;
+    float *amax, *scale_next, *scale_inv_next;
+};
+struct DelayedArgs {
+    DelayedItem it[MULTI_MAX];
+    int n_items;
+    unsigned n_blocks;
+    int len, margin;
+    unsigned int *sync;
+};
+
+__global__ void __launch_bounds__(256) cast_delayed_multi_kernel(const DelayedArgs a)
+{
+    __shared__ int s_last;
+    int t = 0;
+    while (t + 1 < a.n_items && blockIdx.x >= a.it[t + 1].blk0) ++t;
+    const DelayedItem &m = a.it[t];
+    const unsigned nblk = (t + 1 < a.n_items ? a.it[t + 1].blk0 : a.n_blocks) - m.blk0, rank = blockIdx.x - m.blk0;
+    const size_t n16 = m.n / 16;
+    const int n_tail = (int)(m.n - n16 * 16);
+    const ScaleSrc src{m.scale, nullptr, 0.0f, nullptr, nullptr};
+    const uint4 *x = reinterpret_cast<const uint4 *>(m.x);
+    unsigned int *acc = a.sync + 2 * t;
+    if (m.fmt == FP8_E4M3)
+        cast_flat_body<0, true>(x, n16, m.x + n16 * 16, m.out + n16 * 16, n_tail, src, reinterpret_cast<uint4 *>(m.out),
+                                acc, rank, nblk);
+    else
+        cast_flat_body<1, true>(x, n16, m.x + n16 * 16, m.out + n16 * 16, n_tail, src, reinterpret_cast<uint4 *>(m.out),
+                                acc, rank, nblk);
+    // the block's atomic max was issued by thread 0 (if it had anything to add): make it visible, then count
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(acc + 1, 1u) == nblk - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __shared__ float s_amax;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_amax = __uint_as_float(atomicExch(acc, 0u));
+        acc[1] = 0u;
+        *m.amax = s_amax;
+    }
+    __syncthreads();
+    ring_update_body(m.history, a.len, m.head, s_amax, m.fmt == FP8_E4M3 ? 448.0f : 57344.0f, a.margin, m.scale_next,
+                     m.scale_inv_next);
 }
 
 // Cast + transposed copy: one CTA per 128 x 128 tile.  Codes go straight to `out` (16-byte stores) and
@@ -542,6 +609,81 @@ extern "C" int fp8_quantize_multi(const fp8_quant_item *items, int n_items, floa
     amax_multi_kernel<<<ba, 512, 0, st>>>(am);
     FP8_CUDA_CHECK(cudaGetLastError());
     cast_multi_kernel<<<bc, 256, 0, st>>>(ac);
+    FP8_CUDA_CHECK(cudaGetLastError());
+    return FP8_OK;
+}
+
+extern "C" int fp8_quantize_delayed_multi(const fp8_delayed_item *items, int n_items, int history_len, int margin,
+                                          uint32_t *sync, void *stream)
+{
+    if (!items || !sync) {
+        set_error("fp8_quantize_delayed_multi: NULL items / sync");
+        return FP8_ERR_NULL;
+    }
+    if (n_items < 1 || n_items > MULTI_MAX) {
+        set_error("fp8_quantize_delayed_multi: n_items %d must be in [1, %d]", n_items, MULTI_MAX);
+        return FP8_ERR_SHAPE;
+    }
+    if (history_len <= 0 || history_len > (1 << 20) || margin < -64 || margin > 64) {
+        set_error("fp8_quantize_delayed_multi: history_len %d must be in [1, 2^20] and margin %d in [-64, 64]",
+                  history_len, margin);
+        return FP8_ERR_SHAPE;
+    }
+    DelayedArgs a;
+    a.n_items = n_items;
+    a.len = history_len;
+    a.margin = margin;
+    a.sync = sync;
+    size_t want[MULTI_MAX], tot = 0;
+    for (int t = 0; t < n_items; ++t) {
+        const fp8_delayed_item &q = items[t];
+        if (!q.x_bf16 || !q.out || !q.history || !q.head || !q.scale || !q.amax || !q.scale_next || !q.scale_inv_next) {
+            set_error("fp8_quantize_delayed_multi: NULL pointer in item %d", t);
+            return FP8_ERR_NULL;
+        }
+        if (q.fmt != FP8_E4M3 && q.fmt != FP8_E5M2) {
+            set_error("fp8_quantize_delayed_multi: item %d: fmt %d is not FP8_E4M3 / FP8_E5M2", t, q.fmt);
+            return FP8_ERR_ENUM;
+        }
+        if (q.n == 0) {
+            set_error("fp8_quantize_delayed_multi: item %d is empty", t);
+            return FP8_ERR_SHAPE;
+        }
+        if (!aligned16(q.x_bf16) || !aligned16(q.out)) {
+            set_error("fp8_quantize_delayed_multi: tensor pointers must be 16-byte aligned (item %d)", t);
+            return FP8_ERR_ALIGN;
+        }
+        if (q.scale == q.scale_next || q.scale == q.scale_inv_next) {
+            set_error("fp8_quantize_delayed_multi: item %d: scale_next / scale_inv_next must not alias scale", t);
+            return FP8_ERR_SHAPE;
+        }
+        DelayedItem &d = a.it[t];
+        d.x = static_cast<const uint16_t *>(q.x_bf16);
+        d.out = q.out;
+        d.n = q.n;
+        d.fmt = q.fmt;
+        d.history = q.history;
+        d.head = q.head;
+        d.scale = q.scale;
+        d.amax = q.amax;
+        d.scale_next = q.scale_next;
+        d.scale_inv_next = q.scale_inv_next;
+        want[t] = (q.n / 16 + 2 * 256 - 1) / (2 * 256);
+        if (want[t] == 0) want[t] = 1;
+        tot += want[t];
+    }
+    int rc = check_arch();
+    if (rc != FP8_OK) return rc;
+    const size_t cap = (size_t)sm_count() * 8;
+    unsigned nb = 0;
+    for (int t = 0; t < n_items; ++t) {
+        size_t n = tot > cap ? want[t] * cap / tot : want[t];
+        if (n == 0) n = 1;
+        a.it[t].blk0 = nb;
+        nb += (unsigned)n;
+    }
+    a.n_blocks = nb;
+    cast_delayed_multi_kernel<<<nb, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
     FP8_CUDA_CHECK(cudaGetLastError());
     return FP8_OK;
 }

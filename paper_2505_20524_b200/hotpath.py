@@ -58,6 +58,12 @@ class QTensor:
         """Delayed scaling (Appendix E): one pass casts under the scale of the history and records this step's
         abs-max; the history and the scale for the next step are updated afterwards.  The first call seeds the
         history with a just-in-time pass."""
+        self.begin_delayed_step()
+        fp8.fp8_cast(self.x, self.scale, self.fmt, self.q, self.qt, self.amax)
+        fp8.fp8_scale_update(self.history, self.head, self.amax, self.fmt, 0, *self._next)
+
+    def begin_delayed_step(self):
+        """Seeds the history on the first call; then makes the scale computed after the previous step this step's."""
         if self.history is None:
             dev = self.x.device
             self.history = torch.zeros(self.HISTORY_LEN, dtype=torch.float32, device=dev)
@@ -65,11 +71,8 @@ class QTensor:
             self._next = (_f32(dev), _f32(dev))
             fp8.fp8_amax(self.x, self.amax)
             fp8.fp8_scale_update(self.history, self.head, self.amax, self.fmt, 0, *self._next)
-        # the scale computed after the previous step becomes this step's; this step's products read scale_inv, so the
-        # update for the next step is written to the other pair of scalars
+        # this step's products read scale_inv, so the update for the next step is written to the other pair of scalars
         (self.scale, self.scale_inv), self._next = self._next, (self.scale, self.scale_inv)
-        fp8.fp8_cast(self.x, self.scale, self.fmt, self.q, self.qt, self.amax)
-        fp8.fp8_scale_update(self.history, self.head, self.amax, self.fmt, 0, *self._next)
 
     @property
     def nbytes_in(self):
@@ -120,7 +123,8 @@ class BlockHotPath:
         # the scale of the abs-max history, which the pass itself feeds (Appendix E; the recipe the paper trains with)
         # multi_quantize: the just-in-time quantize of a group's tensors (x, w, dy of a projection; q, k, v, do) as one
         # reduction launch and one cast launch for the group (fp8_quantize_multi) instead of two launches per tensor:
-        # the same codes and scales, fewer kernel boundaries
+        # the same codes and scales, fewer kernel boundaries; under delayed scaling the whole quantize of a group (casts,
+        # amaxes, history updates, next scales) is one launch (fp8_quantize_delayed_multi)
         assert scaling in ("jit", "delayed")
         self.scaling = scaling
         self.multi_quantize = bool(multi_quantize)
@@ -135,6 +139,7 @@ class BlockHotPath:
         self.linears: list[Linear] = []
         self.attn = None
         self.host_inputs: dict[str, np.ndarray] = {}
+        self._delayed_sync = {}       # per group: the counter words of the one-launch delayed-scaling quantize
         self.gemm_events = []
         self.quant_events = []
         self.attn_events = []
@@ -291,7 +296,19 @@ class BlockHotPath:
 
     def _quantize_group(self, tensors, scalars):
         """Quantize of the tensors of one group under the configured recipe."""
-        if self.scaling == "delayed":
+        if self.scaling == "delayed" and self.multi_quantize and not self.transposed_copies:
+            # one launch for the group: casts under last step's scales, amaxes, history updates, next scales
+            for t in tensors:
+                t.begin_delayed_step()
+            key = id(tensors[0])
+            if key not in self._delayed_sync:
+                self._delayed_sync[key] = torch.zeros(2 * len(tensors), dtype=torch.int32, device=self.device)
+            fp8.fp8_quantize_delayed_multi([t.x for t in tensors], [t.fmt for t in tensors], [t.q for t in tensors],
+                                           [t.history for t in tensors], [t.head for t in tensors],
+                                           [t.scale for t in tensors], [t.amax for t in tensors],
+                                           [t._next[0] for t in tensors], [t._next[1] for t in tensors], 0,
+                                           self._delayed_sync[key])
+        elif self.scaling == "delayed":
             for t in tensors:
                 t.quantize_delayed()
         elif self.multi_quantize and not self.transposed_copies:
@@ -347,11 +364,13 @@ class BlockHotPath:
     def launches_per_step(self):
         n = 0
         kq = self.KERNELS_PER_QUANTIZE         # delayed scaling: cast (+amax) and the history update, also two
-        grouped = self.scaling == "jit" and self.multi_quantize and not self.transposed_copies
+        grouped = self.multi_quantize and not self.transposed_copies
+        # per group: one reduction + one cast (just-in-time) or one launch (delayed); else two launches per tensor
+        kg = 1 if self.scaling == "delayed" else kq
         for _ in self.linears:
-            n += (kq if grouped else 3 * kq) + 3       # one reduction + one cast for the group, or two per tensor
+            n += (kg if grouped else 3 * kq) + 3
         if self.attn is not None:
-            n += (kq if grouped else 4 * kq) + 1 + self.KERNELS_PER_ATTN_BWD
+            n += (kg if grouped else 4 * kq) + 1 + self.KERNELS_PER_ATTN_BWD
         return n
 
     # ------------------------------------------------------------------ the step

@@ -237,7 +237,8 @@ def test_host_buffer_entry_points_equal_device_step(name):
             assert torch.equal(hout[n].view(torch.uint8), t.view(torch.uint8)), n
 
 
-def test_delayed_scaling_step_equals_the_just_in_time_step_on_repeated_inputs():
+@pytest.mark.parametrize("multi", [True, False], ids=["one_launch_per_group", "two_launches_per_tensor"])
+def test_delayed_scaling_step_equals_the_just_in_time_step_on_repeated_inputs(multi):
     """With the same inputs every step, the abs-max history holds one value: the delayed-scaling step (one cast pass per
     tensor under the history's scale, Appendix E) must return the bits of the just-in-time step; and when an input grows,
     the step that sees it still casts (saturating) under the old scale and the next one under the new."""
@@ -249,7 +250,7 @@ def test_delayed_scaling_step_equals_the_just_in_time_step_on_repeated_inputs():
     jit.step()
     torch.cuda.synchronize()
     ref = {n: t.clone() for n, t in jit.output_tensors()}
-    dl = BlockHotPath(cfg, "cuda", scaling="delayed")
+    dl = BlockHotPath(cfg, "cuda", scaling="delayed", multi_quantize=multi)
     dl.allocate(h)
     dl.attn["ds_scale"].copy_(jit.attn["ds_scale"])
     for _ in range(3):
