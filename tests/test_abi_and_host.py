@@ -41,6 +41,35 @@ def test_binding_mirrors_header_constants():
     assert int(m.group(1)) << int(m.group(2)) == binding.STATIC_SCRATCH_BYTES
 
 
+def test_binding_structures_have_the_header_layout(tmp_path):
+    """The ctypes structures that cross the boundary by pointer match the C compiler's layout of the header's structs:
+    size and the offset of every field, from a program compiled against include/fp8dpa.h."""
+    from paper_2505_20524_b200 import binding
+    pairs = {"fp8_quant_item": binding.QuantItem, "fp8_delayed_item": binding.DelayedItem,
+             "fp8_attn_scales": binding.AttnScales}
+    text = open(os.path.join(ROOT, "include", "fp8dpa.h")).read()
+    lines = ["#include <stdio.h>", "#include <stddef.h>", '#include "fp8dpa.h"', "int main(void) {"]
+    for cname, st in pairs.items():
+        body = re.search(r"typedef struct \{([^{}]*)\}\s*" + cname + r"\s*;", text, re.S).group(1)
+        body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+        fields = [re.findall(r"\w+", part)[-1] for d in body.split(";") if d.strip() for part in d.split(",")]
+        assert fields == [f[0] for f in st._fields_], (cname, fields)         # same names in the same order
+        lines.append(f'printf("{cname} %zu", sizeof({cname}));')
+        lines += [f'printf(" %zu", offsetof({cname}, {f}));' for f in fields]
+        lines.append('printf("\\n");')
+    lines.append("return 0; }")
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
+    for line in filter(None, out):
+        name, size, *offs = line.split()
+        st = pairs[name]
+        assert C.sizeof(st) == int(size), name
+        assert [getattr(st, f[0]).offset for f in st._fields_] == [int(v) for v in offs], name
+
+
 def test_workspace_size_is_host_only_arithmetic():
     from paper_2505_20524_b200 import binding
     n = binding.fp8_attention_workspace_bytes(1, 2, 4096, 32, 8, 128)
