@@ -285,7 +285,7 @@ struct DelayedArgs {
     unsigned int *sync;
 };
 
-__global__ void __launch_bounds__(256) cast_delayed_multi_kernel(const DelayedArgs a)
+__global__ void __launch_bounds__(256, 8) cast_delayed_multi_kernel(const DelayedArgs a)
 {
     __shared__ int s_last;
     int t = 0;
