@@ -388,7 +388,12 @@ class BlockHotPath:
     def capture_graph(self):
         """Captures one step (the same launches) into a CUDA graph and returns it; ``graph.replay()`` then runs the
         step with one submission.  The step makes no host synchronisation, so it is capturable as it is.  Worth it
-        where the step is launch-bound (small configurations); the large ones are bound by the kernels."""
+        where the step is launch-bound (small configurations); the large ones are bound by the kernels.  Just-in-time
+        scaling only: under delayed scaling consecutive steps alternate between two pairs of scale scalars on the host,
+        which one captured step cannot express."""
+        if self.scaling != "jit":
+            raise ValueError("capture_graph: a delayed-scaling step alternates its scale buffers between steps; "
+                             "capture is supported for scaling='jit'")
         side = torch.cuda.Stream(self.device)
         side.wait_stream(torch.cuda.current_stream(self.device))
         with torch.cuda.stream(side):
