@@ -110,13 +110,15 @@ FP8_API int fp8_quantize_multi(const fp8_quant_item *items, int n_items, float *
 FP8_API int fp8_scale_update(float *history, int len, int *head, const float *amax_new, int fmt, int margin,
                      float *scale, float *scale_inv, void *stream);
 
-/* The whole delayed-scaling quantize (Appendix E) of up to 8 flat tensors in ONE launch: item i casts its n BF16
- * values to out under *scale (the scale its history gave after the previous step), the same pass takes amax(x), and
- * the last block to finish a tensor does that tensor's fp8_scale_update: history[*head] = amax, *head advances,
- * *scale_next / *scale_inv_next = the scale of the next step from the maximum of the updated history; *amax is
- * overwritten with amax(x).  Codes, amax, history, head and scales are bit-identical to fp8_cast(..., amax_out)
- * followed by fp8_scale_update.  `items` is a HOST array; every pointer inside it is a device pointer.  scale_next and
- * scale_inv_next must not alias scale (the caller swaps the two pairs between steps).  sync: device array of
+/* The whole delayed-scaling quantize (Appendix E) of up to 8 flat tensors in ONE launch.  Item i: *scale_next, as the
+ * call finds it, is this step's scale (what the previous call left there from the history; before the first call the
+ * caller sets it, e.g. to 1 or from fp8_amax + fp8_scale_update).  The n BF16 values are cast to out under it, the same
+ * pass takes amax(x), *scale and *scale_inv receive this step's scale and its reciprocal (what the products of this
+ * step read), and the last block to finish the tensor does its fp8_scale_update: history[*head] = amax, *head advances,
+ * *scale_next = the scale of the next step from the maximum of the updated history; *amax = amax(x).  No pointer
+ * changes between steps, so a step built on this call can be captured in a CUDA graph.  Codes, amax, history, head
+ * and scales are bit-identical to fp8_cast(..., amax_out) followed by fp8_scale_update.  `items` is a HOST array;
+ * every pointer inside it is a device pointer; scale and scale_inv must not alias scale_next.  sync: device array of
  * 2 * n_items 32-bit words, zero before the first call and left zero by every call (amax bits and a block counter
  * per tensor); calls that share `sync` must be ordered on one stream. */
 typedef struct {
@@ -126,10 +128,10 @@ typedef struct {
     uint8_t *out;            /* device, 16-byte aligned, n bytes */
     float *history;          /* device ring of history_len floats (zero-initialised by the caller) */
     int *head;               /* device int, initially 0 */
-    const float *scale;      /* device: the scale of this step */
+    float *scale_next;       /* device, read then overwritten: this step's scale in, the next step's out */
     float *amax;             /* device, overwritten */
-    float *scale_next;       /* device, overwritten */
-    float *scale_inv_next;   /* device, overwritten */
+    float *scale;            /* device, overwritten: this step's scale */
+    float *scale_inv;        /* device, overwritten: its reciprocal */
 } fp8_delayed_item;
 FP8_API int fp8_quantize_delayed_multi(const fp8_delayed_item *items, int n_items, int history_len, int margin,
                                uint32_t *sync, void *stream);

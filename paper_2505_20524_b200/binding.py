@@ -150,24 +150,25 @@ def fp8_quantize_multi(xs, fmts, outs, scalars, stream=None):
 
 class DelayedItem(C.Structure):
     _fields_ = [("x_bf16", C.c_void_p), ("n", C.c_size_t), ("fmt", C.c_int), ("out", C.c_void_p),
-                ("history", C.c_void_p), ("head", C.c_void_p), ("scale", C.c_void_p), ("amax", C.c_void_p),
-                ("scale_next", C.c_void_p), ("scale_inv_next", C.c_void_p)]
+                ("history", C.c_void_p), ("head", C.c_void_p), ("scale_next", C.c_void_p), ("amax", C.c_void_p),
+                ("scale", C.c_void_p), ("scale_inv", C.c_void_p)]
 
 
-def fp8_quantize_delayed_multi(xs, fmts, outs, histories, heads, scales, amaxes, scales_next, scales_inv_next, margin,
+def fp8_quantize_delayed_multi(xs, fmts, outs, histories, heads, scales_next, amaxes, scales, scales_inv, margin,
                                sync, stream=None):
-    """Delayed-scaling quantize of up to 8 tensors in one launch (cast under `scales`, amax, history update and the next
-    step's scale): lists of CUDA tensors, one entry per tensor; all histories have the same length; sync an int32 /
+    """Delayed-scaling quantize of up to 8 tensors in one launch: cast under scales_next[i] as the call finds it (also
+    written to scales[i] with its reciprocal in scales_inv[i]), amax, history update, and the next step's scale left in
+    scales_next[i].  Lists of CUDA tensors, one entry per tensor; all histories have the same length; sync an int32 /
     uint32 CUDA tensor of 2 * len(xs) words that is zero before the first call."""
     n = len(xs)
-    assert all(len(v) == n for v in (fmts, outs, histories, heads, scales, amaxes, scales_next, scales_inv_next))
+    assert all(len(v) == n for v in (fmts, outs, histories, heads, scales_next, amaxes, scales, scales_inv))
     assert sync.numel() >= 2 * n and sync.element_size() == 4
     assert all(h.numel() == histories[0].numel() for h in histories)
     items = (DelayedItem * n)()
     for i in range(n):
         items[i] = DelayedItem(_ptr(xs[i]).value, xs[i].numel(), int(fmts[i]), _ptr(outs[i]).value,
-                               _ptr(histories[i]).value, _ptr(heads[i]).value, _ptr(scales[i]).value,
-                               _ptr(amaxes[i]).value, _ptr(scales_next[i]).value, _ptr(scales_inv_next[i]).value)
+                               _ptr(histories[i]).value, _ptr(heads[i]).value, _ptr(scales_next[i]).value,
+                               _ptr(amaxes[i]).value, _ptr(scales[i]).value, _ptr(scales_inv[i]).value)
     _check(load().fp8_quantize_delayed_multi(items, C.c_int(n), C.c_int(histories[0].numel()), C.c_int(margin),
                                              _ptr(sync), _stream(stream)))
 

@@ -188,9 +188,10 @@ template <int FMT, bool AMAX>
 __device__ __forceinline__ void cast_flat_body(const uint4 *__restrict__ x, size_t n16, const uint16_t *__restrict__ tail_in,
                                                uint8_t *__restrict__ tail_out, int n_tail, const ScaleSrc &scale_src,
                                                uint4 *__restrict__ out, unsigned int *__restrict__ amax_bits, unsigned rank,
-                                               unsigned nblk)
+                                               unsigned nblk, float scale_value = -1.0f)
 {
-    const float s = resolve_scale(scale_src, rank == 0 && threadIdx.x == 0);
+    // scale_value >= 0: the caller has the scale already (the delayed-scaling launch); scales are never negative
+    const float s = scale_value >= 0.0f ? scale_value : resolve_scale(scale_src, rank == 0 && threadIdx.x == 0);
     uint32_t m = 0;
     const size_t stride = (size_t)nblk * blockDim.x;
     size_t i = (size_t)rank * blockDim.x + threadIdx.x;
@@ -263,8 +264,9 @@ __global__ void __launch_bounds__(256) cast_multi_kernel(const MultiArgs a)
 }
 
 // Delayed scaling of several tensors in ONE launch: every tensor is cast under the scale its history gave after the
-// previous step while the same pass takes its amax; the last block of a tensor to finish (a counter per tensor) then
-// does that tensor's ring update and writes the scale of the next step.  sync[2 t] collects the amax bits, sync[2 t + 1]
+// previous step (*scale_next as the launch finds it; the first block also publishes it and its reciprocal for the
+// products) while the same pass takes its amax; the last block of a tensor to finish (a counter per tensor) then does
+// that tensor's ring update and leaves the scale of the next step in *scale_next.  sync[2 t] collects the amax bits, sync[2 t + 1]
 // counts finished blocks; the last block leaves both at zero for the next call.
 struct DelayedItem {
     const uint16_t *x;
@@ -274,8 +276,8 @@ struct DelayedItem {
     unsigned blk0;
     float *history;
     int *head;
-    const float *scale;
-    float *amax, *scale_next, *scale_inv_next;
+    float *scale_next;                  // in: this step's scale; out (last block): the next step's
+    float *amax, *scale, *scale_inv;    // out: amax(x); this step's scale and its reciprocal, for the products
 };
 struct DelayedArgs {
     DelayedItem it[MULTI_MAX];
@@ -294,15 +296,22 @@ __global__ void __launch_bounds__(256, 8) cast_delayed_multi_kernel(const Delaye
     const unsigned nblk = (t + 1 < a.n_items ? a.it[t + 1].blk0 : a.n_blocks) - m.blk0, rank = blockIdx.x - m.blk0;
     const size_t n16 = m.n / 16;
     const int n_tail = (int)(m.n - n16 * 16);
-    const ScaleSrc src{m.scale, nullptr, 0.0f, nullptr, nullptr};
+    // A plain load, not the read-only path: the last block overwrites *scale_next at the end of this launch.  It does so
+    // only after every block has counted in, and a block counts in after it has read the scale here.
+    const float s = *reinterpret_cast<const volatile float *>(m.scale_next);
+    if (rank == 0 && threadIdx.x == 0) {
+        *m.scale = s;
+        *m.scale_inv = __fdiv_rn(1.0f, s);
+    }
+    const ScaleSrc src{nullptr, nullptr, 0.0f, nullptr, nullptr};
     const uint4 *x = reinterpret_cast<const uint4 *>(m.x);
     unsigned int *acc = a.sync + 2 * t;
     if (m.fmt == FP8_E4M3)
         cast_flat_body<0, true>(x, n16, m.x + n16 * 16, m.out + n16 * 16, n_tail, src, reinterpret_cast<uint4 *>(m.out),
-                                acc, rank, nblk);
+                                acc, rank, nblk, s);
     else
         cast_flat_body<1, true>(x, n16, m.x + n16 * 16, m.out + n16 * 16, n_tail, src, reinterpret_cast<uint4 *>(m.out),
-                                acc, rank, nblk);
+                                acc, rank, nblk, s);
     // the block's atomic max was issued by thread 0 (if it had anything to add): make it visible, then count
     if (threadIdx.x == 0) {
         __threadfence();
@@ -318,8 +327,9 @@ __global__ void __launch_bounds__(256, 8) cast_delayed_multi_kernel(const Delaye
         *m.amax = s_amax;
     }
     __syncthreads();
+    __shared__ float s_unused_inv;
     ring_update_body(m.history, a.len, m.head, s_amax, m.fmt == FP8_E4M3 ? 448.0f : 57344.0f, a.margin, m.scale_next,
-                     m.scale_inv_next);
+                     &s_unused_inv);
 }
 
 // Cast + transposed copy: one CTA per 128 x 128 tile.  Codes go straight to `out` (16-byte stores) and
@@ -637,7 +647,7 @@ extern "C" int fp8_quantize_delayed_multi(const fp8_delayed_item *items, int n_i
     size_t want[MULTI_MAX], tot = 0;
     for (int t = 0; t < n_items; ++t) {
         const fp8_delayed_item &q = items[t];
-        if (!q.x_bf16 || !q.out || !q.history || !q.head || !q.scale || !q.amax || !q.scale_next || !q.scale_inv_next) {
+        if (!q.x_bf16 || !q.out || !q.history || !q.head || !q.scale_next || !q.amax || !q.scale || !q.scale_inv) {
             set_error("fp8_quantize_delayed_multi: NULL pointer in item %d", t);
             return FP8_ERR_NULL;
         }
@@ -653,8 +663,8 @@ extern "C" int fp8_quantize_delayed_multi(const fp8_delayed_item *items, int n_i
             set_error("fp8_quantize_delayed_multi: tensor pointers must be 16-byte aligned (item %d)", t);
             return FP8_ERR_ALIGN;
         }
-        if (q.scale == q.scale_next || q.scale == q.scale_inv_next) {
-            set_error("fp8_quantize_delayed_multi: item %d: scale_next / scale_inv_next must not alias scale", t);
+        if (q.scale == q.scale_next || q.scale_inv == q.scale_next) {
+            set_error("fp8_quantize_delayed_multi: item %d: scale / scale_inv must not alias scale_next", t);
             return FP8_ERR_SHAPE;
         }
         DelayedItem &d = a.it[t];
@@ -664,10 +674,10 @@ extern "C" int fp8_quantize_delayed_multi(const fp8_delayed_item *items, int n_i
         d.fmt = q.fmt;
         d.history = q.history;
         d.head = q.head;
-        d.scale = q.scale;
-        d.amax = q.amax;
         d.scale_next = q.scale_next;
-        d.scale_inv_next = q.scale_inv_next;
+        d.amax = q.amax;
+        d.scale = q.scale;
+        d.scale_inv = q.scale_inv;
         want[t] = (q.n / 16 + 2 * 256 - 1) / (2 * 256);
         if (want[t] == 0) want[t] = 1;
         tot += want[t];

@@ -58,12 +58,15 @@ class QTensor:
         """Delayed scaling (Appendix E): one pass casts under the scale of the history and records this step's
         abs-max; the history and the scale for the next step are updated afterwards.  The first call seeds the
         history with a just-in-time pass."""
-        self.begin_delayed_step()
+        self.seed_history()
+        # the scale computed after the previous step becomes this step's; this step's products read scale_inv, so the
+        # update for the next step is written to the other pair of scalars
+        (self.scale, self.scale_inv), self._next = self._next, (self.scale, self.scale_inv)
         fp8.fp8_cast(self.x, self.scale, self.fmt, self.q, self.qt, self.amax)
         fp8.fp8_scale_update(self.history, self.head, self.amax, self.fmt, 0, *self._next)
 
-    def begin_delayed_step(self):
-        """Seeds the history on the first call; then makes the scale computed after the previous step this step's."""
+    def seed_history(self):
+        """First call only: the history ring, and the first step's scale from a just-in-time amax pass."""
         if self.history is None:
             dev = self.x.device
             self.history = torch.zeros(self.HISTORY_LEN, dtype=torch.float32, device=dev)
@@ -71,8 +74,6 @@ class QTensor:
             self._next = (_f32(dev), _f32(dev))
             fp8.fp8_amax(self.x, self.amax)
             fp8.fp8_scale_update(self.history, self.head, self.amax, self.fmt, 0, *self._next)
-        # this step's products read scale_inv, so the update for the next step is written to the other pair of scalars
-        (self.scale, self.scale_inv), self._next = self._next, (self.scale, self.scale_inv)
 
     @property
     def nbytes_in(self):
@@ -297,16 +298,18 @@ class BlockHotPath:
     def _quantize_group(self, tensors, scalars):
         """Quantize of the tensors of one group under the configured recipe."""
         if self.scaling == "delayed" and self.multi_quantize and not self.transposed_copies:
-            # one launch for the group: casts under last step's scales, amaxes, history updates, next scales
+            # one launch for the group: casts under the scales the previous step left in _next[0] (published to scale /
+            # scale_inv for the products), amaxes, history updates, and the next step's scales back into _next[0]; the same
+            # pointers every step
             for t in tensors:
-                t.begin_delayed_step()
+                t.seed_history()
             key = id(tensors[0])
             if key not in self._delayed_sync:
                 self._delayed_sync[key] = torch.zeros(2 * len(tensors), dtype=torch.int32, device=self.device)
             fp8.fp8_quantize_delayed_multi([t.x for t in tensors], [t.fmt for t in tensors], [t.q for t in tensors],
                                            [t.history for t in tensors], [t.head for t in tensors],
-                                           [t.scale for t in tensors], [t.amax for t in tensors],
-                                           [t._next[0] for t in tensors], [t._next[1] for t in tensors], 0,
+                                           [t._next[0] for t in tensors], [t.amax for t in tensors],
+                                           [t.scale for t in tensors], [t.scale_inv for t in tensors], 0,
                                            self._delayed_sync[key])
         elif self.scaling == "delayed":
             for t in tensors:
@@ -388,12 +391,12 @@ class BlockHotPath:
     def capture_graph(self):
         """Captures one step (the same launches) into a CUDA graph and returns it; ``graph.replay()`` then runs the
         step with one submission.  The step makes no host synchronisation, so it is capturable as it is.  Worth it
-        where the step is launch-bound (small configurations); the large ones are bound by the kernels.  Just-in-time
-        scaling only: under delayed scaling consecutive steps alternate between two pairs of scale scalars on the host,
-        which one captured step cannot express."""
-        if self.scaling != "jit":
-            raise ValueError("capture_graph: a delayed-scaling step alternates its scale buffers between steps; "
-                             "capture is supported for scaling='jit'")
+        where the step is launch-bound (small configurations); the large ones are bound by the kernels.  Delayed
+        scaling is capturable in its one-launch form (the same pointers every step); the per-tensor form alternates
+        between two pairs of scale scalars on the host, which one captured step cannot express."""
+        if self.scaling != "jit" and not (self.multi_quantize and not self.transposed_copies):
+            raise ValueError("capture_graph: the per-tensor delayed-scaling step alternates its scale buffers between "
+                             "steps on the host; capture needs scaling='jit' or the one-launch group quantize")
         side = torch.cuda.Stream(self.device)
         side.wait_stream(torch.cuda.current_stream(self.device))
         with torch.cuda.stream(side):

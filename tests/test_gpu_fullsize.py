@@ -324,9 +324,29 @@ def test_graph_replay_of_the_step_equals_the_step():
     assert fp8.fp8_device_status() == 0
     for n, t in hp.output_tensors():
         assert torch.equal(t.view(torch.uint8), ref[n].view(torch.uint8)), n
-    # a delayed-scaling step swaps its scale buffers on the host between steps: one captured step cannot do that
+    # delayed scaling: the one-launch group quantize keeps its pointers from step to step, so three replays of one
+    # captured step equal three eager steps (the history advances on the device); the per-tensor form swaps its scale
+    # buffers on the host between steps and refuses capture
+    eager = BlockHotPath(cfg, "cuda", scaling="delayed")
+    eager.allocate(hp.host_inputs)
+    eager.attn["ds_scale"].copy_(hp.attn["ds_scale"])
+    for _ in range(4):
+        eager.step()
+    torch.cuda.synchronize()
+    want = {n: t.clone() for n, t in eager.output_tensors()}
+    dl = BlockHotPath(cfg, "cuda", scaling="delayed")
+    dl.allocate(hp.host_inputs)
+    dl.attn["ds_scale"].copy_(hp.attn["ds_scale"])
+    g = dl.capture_graph()                       # runs one eager step itself
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    for n, t in dl.output_tensors():
+        assert torch.equal(t.view(torch.uint8), want[n].view(torch.uint8)), n
+    assert torch.equal(dl.linears[0].x.history, eager.linears[0].x.history)
+    assert int(dl.linears[0].x.head.item()) == int(eager.linears[0].x.head.item())
     with pytest.raises(ValueError):
-        BlockHotPath(cfg, "cuda", scaling="delayed").capture_graph()
+        BlockHotPath(cfg, "cuda", scaling="delayed", multi_quantize=False).capture_graph()
 
 
 def test_glue_and_producer_forms_at_c4_sizes():

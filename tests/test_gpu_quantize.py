@@ -210,18 +210,19 @@ def test_quantize_multi_equals_per_tensor_quantize_and_oracle():
 
 
 def test_delayed_multi_is_the_oracle_chain_in_one_launch():
-    """fp8_quantize_delayed_multi over more steps than the history holds: per tensor and step the codes equal the
-    oracle's cast under the scale of the history so far, and amax, history, position and next scale equal the oracle's
-    scale_update; sizes from 1 element to several blocks per tensor, both formats, an all-zero tensor, a ring of
-    length 3 (wraps twice) with margin 1; the counter words are zero after every call."""
+    """fp8_quantize_delayed_multi over more steps than the history holds, with the same pointers every step: per tensor
+    and step the codes equal the oracle's cast under the scale of the history so far, the published scale and reciprocal
+    are that scale's, and amax, history, position and next scale equal the oracle's scale_update; sizes from 1 element
+    to several blocks per tensor, both formats, an all-zero tensor, a ring of length 3 (wraps twice) with margin 1; the
+    counter words are zero after every call."""
     l, margin, steps = 3, 1, 8
     sizes = [1, 15, 4096 + 7, 300_000, (1 << 20) + 24, 2_500_000]
     fmts = [fp8.E4M3, fp8.E5M2, fp8.E4M3, fp8.E5M2, fp8.E5M2, fp8.E4M3]
     n = len(sizes)
     hist_d = [torch.zeros(l, dtype=torch.float32, device="cuda") for _ in range(n)]
     head_d = [torch.zeros(1, dtype=torch.int32, device="cuda") for _ in range(n)]
-    cur = [(scalar(1.0), scalar(1.0)) for _ in range(n)]
-    nxt = [(scalar(-1.0), scalar(-1.0)) for _ in range(n)]
+    nxt = [scalar(1.0) for _ in range(n)]                     # the first step casts under scale 1
+    cur, cur_inv = [scalar(-1.0) for _ in range(n)], [scalar(-1.0) for _ in range(n)]
     amax_d = [scalar(-1.0) for _ in range(n)]
     sync = torch.zeros(2 * n, dtype=torch.int32, device="cuda")
     hist = [np.zeros(l, dtype=np.float32) for _ in range(n)]
@@ -238,29 +239,29 @@ def test_delayed_multi_is_the_oracle_chain_in_one_launch():
                 xs_host.append(synth.normal_bf16((1, sz), 100 + 10 * step + i, 0, 1.0 + step).reshape(-1))
         xs = [dev(x) for x in xs_host]
         outs = [torch.full((sz,), 0xAA, dtype=torch.uint8, device="cuda") for sz in sizes]
-        fp8.fp8_quantize_delayed_multi(xs, fmts, outs, hist_d, head_d, [c[0] for c in cur], amax_d,
-                                       [c[0] for c in nxt], [c[1] for c in nxt], margin, sync)
+        fp8.fp8_quantize_delayed_multi(xs, fmts, outs, hist_d, head_d, nxt, amax_d, cur, cur_inv, margin, sync)
         torch.cuda.synchronize()
         assert int(sync.abs().sum().item()) == 0
         for i in range(n):
             assert np.array_equal(outs[i].cpu().numpy(), o.cast(xs_host[i].reshape(1, -1), es[i], fmts[i]).reshape(-1)), (step, i)
+            assert np.float32(cur[i].item()) == es[i], (step, i)
+            assert np.float32(cur_inv[i].item()) == np.float32(1.0) / es[i], (step, i)
             a = o.amax(xs_host[i])
             assert np.float32(amax_d[i].item()) == np.float32(a), (step, i)
-            head[i], s_new, si_new = o.scale_update(hist[i], head[i], a, fmts[i], margin)
-            assert bits(nxt[i][0]) == int(s_new.view(np.uint32)) and bits(nxt[i][1]) == int(si_new.view(np.uint32)), (step, i)
+            head[i], s_new, _ = o.scale_update(hist[i], head[i], a, fmts[i], margin)
+            assert bits(nxt[i]) == int(s_new.view(np.uint32)), (step, i)
             assert int(head_d[i].item()) == head[i] and np.array_equal(hist_d[i].cpu().numpy(), hist[i]), (step, i)
             es[i] = s_new
-        cur, nxt = nxt, cur
     # a single tensor, and the argument checks
     one = dev(synth.flat_tensor(70_000, seed=7))
     out = torch.empty(70_000, dtype=torch.uint8, device="cuda")
-    fp8.fp8_quantize_delayed_multi([one], [fp8.E4M3], [out], hist_d[:1], head_d[:1], [cur[0][0]], amax_d[:1],
-                                   [nxt[0][0]], [nxt[0][1]], 0, sync)
+    fp8.fp8_quantize_delayed_multi([one], [fp8.E4M3], [out], hist_d[:1], head_d[:1], nxt[:1], amax_d[:1], cur[:1],
+                                   cur_inv[:1], 0, sync)
     assert np.array_equal(out.cpu().numpy(), o.cast(host(one).reshape(1, -1), es[0], fp8.E4M3).reshape(-1))
-    with pytest.raises(fp8.Fp8Error):      # the next scale may not overwrite the scale being read
-        fp8.fp8_quantize_delayed_multi([one], [fp8.E4M3], [out], hist_d[:1], head_d[:1], [cur[0][0]], amax_d[:1],
-                                       [cur[0][0]], [nxt[0][1]], 0, sync)
+    with pytest.raises(fp8.Fp8Error):      # this step's scale may not be published over the state it is read from
+        fp8.fp8_quantize_delayed_multi([one], [fp8.E4M3], [out], hist_d[:1], head_d[:1], nxt[:1], amax_d[:1], nxt[:1],
+                                       cur_inv[:1], 0, sync)
     with pytest.raises(fp8.Fp8Error):
         fp8.fp8_quantize_delayed_multi([one] * 9, [fp8.E4M3] * 9, [out] * 9, hist_d[:1] * 9, head_d[:1] * 9,
-                                       [cur[0][0]] * 9, amax_d[:1] * 9, [nxt[0][0]] * 9, [nxt[0][1]] * 9, 0,
+                                       nxt[:1] * 9, amax_d[:1] * 9, cur[:1] * 9, cur_inv[:1] * 9, 0,
                                        torch.zeros(18, dtype=torch.int32, device="cuda"))
