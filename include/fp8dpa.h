@@ -102,7 +102,7 @@ FP8_API int fp8_quantize_multi(const fp8_quant_item *items, int n_items, float *
 
 /* Delayed scaling (Appendix E): H holds the last `len` abs-max values of one tensor (the paper trains with
  * len = 1024, margin 0); rho = FP8Max / (2^margin * max H); after a step, H <- {amax} u H minus its oldest
- * entry, "to use in the next iteration".  This call does that update on the device: history[*head] = *amax_new,
+ * entry, and the updated history serves the following step.  This call does that update on the device: history[*head] = *amax_new,
  * *head = (*head + 1) % len, then *scale / *scale_inv from the maximum of the updated history (guards as in
  * fp8_scale; an all-zero history gives 1).  history: `len` floats, zero-initialised by the caller; head: device
  * int, initially 0, the position of the oldest entry.  A training step then needs a single pass per tensor:

@@ -144,8 +144,8 @@ void oracle_scale(float amax, int fmt, int margin, float *scale, float *scale_in
 
 /* ------------------------------------------------------------------------------------------------
  * Delayed scaling (Appendix E): H = {h_1..h_l} holds the last l abs-max values of a tensor,
- * rho = FP8Max / (2^m max H), and after a step H <- {amax(X)} u {h_t}_{t=2..l}, "to use in the next
- * iteration".  Reading of the set notation: a FIFO, the dropped h_1 is the oldest entry; the new scale is
+ * rho = FP8Max / (2^m max H), and after a step H <- {amax(X)} u {h_t}_{t=2..l}; the updated history
+ * serves the following step.  Reading of the set notation: a FIFO, the dropped h_1 is the oldest entry; the new scale is
  * computed from the history *after* the insertion and is the one the next step casts with.  `head` is
  * the position of the oldest entry.  Entries that were never written are 0 and an all-zero history
  * gives scale 1 (same guard as oracle_scale).
@@ -185,8 +185,8 @@ void oracle_cast_bf16(const uint16_t *x, size_t rows, size_t cols, float scale, 
  * Kurtosis monitor (Section 4, "Long-term outlier dynamics"): kurt(x) = mu[x^4] / sigma^2[x]^2 for one token
  * vector x, without centring, averaged over the tokens of the tensor.  Reading of the printed formula
  * (its denominator is typeset as the variance of x^2): the un-centred second moment of x, squared, i.e.
- * mu[x^4] / mu[x^2]^2 - the only reading under which "maximised when few elements are extremely large"
- * holds (a one-hot vector of length D gives D, a constant vector 1, a Gaussian about 3).
+ * mu[x^4] / mu[x^2]^2 - the only reading under which the quantity peaks for a vector dominated by a handful of
+ * outliers, as the section says it does (a one-hot vector of length D gives D, a constant vector 1, a Gaussian about 3).
  * A row of zeros contributes 0.
  * ---------------------------------------------------------------------------------------------- */
 double oracle_kurtosis_bf16(const uint16_t *x, size_t rows, size_t cols)
